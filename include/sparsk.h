@@ -1,0 +1,181 @@
+/*
+ * sparsk.h -- C ABI of the B200 (sm_100a) SPAR-K decode library.
+ *
+ * SPAR-K (scheduled periodic alternating early exit) decodes an interleaved
+ * text/speech token stream with a stack of L transformer layers.  Text steps run
+ * all L layers.  A speech step whose index c inside its chunk satisfies
+ * c mod K == r runs all L layers too ("refresh"); every other speech step leaves
+ * at layer e = l_EE and reads its token from that layer's own head (Sec. IV-B.1,
+ * Eq. 2).  An early-exit step caches K/V of layers 1..e only, keeps h^(e) and
+ * marks its position pending; the next full-depth step pushes the pending
+ * positions together with its own through layers e+1..L as one causal block,
+ * which fills their K/V, and clears the pending set; tokens already emitted are
+ * never revised (Sec. IV-B.3, Algorithm 1).
+ *
+ * Every step of that path runs in hand-written CUDA kernels inside this library.
+ * There is no CPU fallback.  The library never calls cudaMalloc on the step path:
+ * all device memory is a caller-supplied workspace.
+ *
+ * Conventions
+ *   - "device" / "host" in a comment says where the pointer must live.
+ *   - All weights are bfloat16, row-major [out_features, in_features], BORROWED:
+ *     the caller keeps them alive until sparsk_destroy.
+ *   - Token ids [0, vocab_text) are text, [vocab_text, vocab_text+vocab_speech)
+ *     are speech.
+ *   - Calls enqueue work on the stream given at create and return without
+ *     synchronising unless stated.  Outputs are valid once the stream has been
+ *     synchronised.
+ *   - Return value 0 is success, negative values are the SPARSK_E* codes.  Every
+ *     error that can be found from host-side arguments is found before anything
+ *     is launched, and leaves all state unchanged.  Nothing aborts or traps.
+ */
+#ifndef SPARSK_H
+#define SPARSK_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SPARSK_OK 0
+#define SPARSK_EINVAL (-1)    /* bad dims, NULL pointer, value out of range, duplicate slot   */
+#define SPARSK_ECAPACITY (-2) /* a sequence would exceed max_seq_len or max_pending           */
+#define SPARSK_ENOHEAD (-3)   /* the step needs an exit head whose pointers are NULL          */
+#define SPARSK_ECUDA (-4)     /* a CUDA call failed; text in sparsk_last_error                */
+#define SPARSK_ESTATE (-5)    /* slot never prefilled / context destroyed                     */
+#define SPARSK_ETIMEOUT (-6)  /* a bounded in-kernel wait ran out (reported by the next call) */
+
+typedef struct sparsk_ctx sparsk_ctx; /* opaque */
+
+/* Model and schedule description (Sec. III for L and d; Sec. IV-B.1 for e, K, r). */
+typedef struct {
+    int32_t n_layers;       /* L */
+    int32_t d_model;        /* d, multiple of 8 */
+    int32_t n_q_heads;      /* H_q, multiple of n_kv_heads */
+    int32_t n_kv_heads;     /* H_kv */
+    int32_t head_dim;       /* 64 or 128 */
+    int32_t d_ffn;          /* F, multiple of 8 */
+    int32_t vocab_text;     /* V_t */
+    int32_t vocab_speech;   /* V_s */
+    float rms_eps;
+    float rope_base;
+    int32_t exit_layer;     /* e in 1..L; e == L disables early exit */
+    int32_t refresh_period; /* K >= 1; K == 1 makes every step full depth */
+    int32_t refresh_phase;  /* r in [0, K): in-chunk index c is full depth iff c % K == r */
+    int32_t text_exit;      /* 0: text steps always run L layers (the paper's main rows);
+                               1: text steps follow the same (K, r, e) rule (Sec. V-E) */
+    int32_t max_seqs;       /* number of sequence slots */
+    int32_t max_seq_len;    /* positions per slot */
+    int32_t max_pending;    /* pending positions per slot; >= K-1 for the periodic schedule */
+    int32_t prefill_rows;   /* rows per prefill pass (0 = default) */
+} sparsk_dims;
+
+/* All pointers are DEVICE pointers to bfloat16 data; the arrays of pointers themselves
+ * are HOST arrays of length n_layers.  head_norm[l-1] / head_proj[l-1] are the head g_l of
+ * layer l (Eq. 2; g_L is the ordinary LM head of Eq. 1) and may be NULL for layers that are
+ * never used as an exit. */
+typedef struct {
+    const void *embed;             /* [V_t+V_s, d] */
+    const void *const *attn_norm;  /* [d]          */
+    const void *const *wq;         /* [H_q*hd, d]  */
+    const void *const *wk;         /* [H_kv*hd, d] */
+    const void *const *wv;         /* [H_kv*hd, d] */
+    const void *const *wo;         /* [d, H_q*hd]  */
+    const void *const *mlp_norm;   /* [d]          */
+    const void *const *w_gate;     /* [F, d]       */
+    const void *const *w_up;       /* [F, d]       */
+    const void *const *w_down;     /* [d, F]       */
+    const void *const *head_norm;  /* [d] or NULL  */
+    const void *const *head_proj;  /* [V_t+V_s, d] or NULL */
+} sparsk_weights;
+
+/* Bytes of device workspace sparsk_create needs for these dims; 0 if the dims are invalid.
+ * The workspace holds the KV cache ([L][slot][H_kv][max_seq_len][hd] bf16, keys and values),
+ * the pending store ([slot][max_pending][d] fp32), per-slot lengths, the step descriptor,
+ * activation buffers, split-KV scratch and the rotary table. */
+size_t sparsk_workspace_bytes(const sparsk_dims *dims /*host*/);
+
+/* Build a context.  `workspace` (device, 256-byte aligned, >= sparsk_workspace_bytes) and the
+ * weights stay owned by the caller.  `cuda_stream` is a cudaStream_t (NULL = default stream).
+ * Synchronises the stream once (table upload).  Sec. III / IV-B define what is being set up. */
+int sparsk_create(const sparsk_dims *dims /*host*/, const sparsk_weights *weights /*host*/,
+                  void *workspace /*device*/, size_t workspace_bytes, void *cuda_stream,
+                  sparsk_ctx **out /*host*/);
+
+/* Ingest prompt tokens at full depth: K/V of every layer is written for every token, nothing
+ * is emitted, pending sets stay empty (the standard-decoding state of Sec. III).  `slots`
+ * [n_seqs] host, distinct; `tokens` device int32, the prompts concatenated; `offsets`
+ * [n_seqs+1] host.  Appends to whatever the slot already holds. */
+int sparsk_prefill(sparsk_ctx *ctx, int32_t n_seqs, const int32_t *slots /*host*/,
+                   const int32_t *tokens /*device*/, const int32_t *offsets /*host*/);
+
+/* One decoding step for n_seqs sequences (one iteration of Algorithm 1's loop, for text and
+ * speech alike).  token_ids[i]: input token of sequence i (the token emitted by its previous
+ * step, or the last prompt token).  modality[i]: 0 text / 1 speech, the modality of the token
+ * this step EMITS; the argmax is restricted to that id range (lowest id on ties).
+ * speech_counters[i]: index c of that token inside its chunk.  Outputs: next_tokens[i] and
+ * exit_depths[i] (e or L).  Host arrays are read before the call returns. */
+int sparsk_decode_step(sparsk_ctx *ctx, int32_t n_seqs, const int32_t *slots /*host*/,
+                       const int32_t *token_ids /*device [n]*/, const uint8_t *modality /*host [n]*/,
+                       const int32_t *speech_counters /*host [n]*/,
+                       int32_t *next_tokens /*device [n]*/, int32_t *exit_depths /*device [n]*/);
+
+/* Same step with HOST token and result buffers: copies token_ids to the device, runs the step,
+ * copies both results back and synchronises the stream.  This is the call a host-side
+ * generation loop makes when it consumes every token as it is produced. */
+int sparsk_decode_step_host(sparsk_ctx *ctx, int32_t n_seqs, const int32_t *slots /*host*/,
+                            const int32_t *token_ids /*host [n]*/, const uint8_t *modality /*host*/,
+                            const int32_t *speech_counters /*host*/,
+                            int32_t *next_tokens /*host [n]*/, int32_t *exit_depths /*host [n]*/);
+
+/* Forget a slot: length 0, pending set empty. */
+int sparsk_reset_slot(sparsk_ctx *ctx, int32_t slot);
+
+/* Load / read cache contents of one layer (1-based) of a slot: n positions starting at
+ * first_pos, keys already rotated, layout [n][H_kv*hd] bf16, device pointers.  set_len declares
+ * that positions [0, len) are complete at every layer (pending set empty).  These let a caller
+ * restore a saved prefix, and let tests inspect the KV invariant of Sec. IV-B.3. */
+int sparsk_import_kv(sparsk_ctx *ctx, int32_t slot, int32_t layer, int32_t first_pos, int32_t n,
+                     const void *k /*device*/, const void *v /*device*/);
+int sparsk_export_kv(sparsk_ctx *ctx, int32_t slot, int32_t layer, int32_t first_pos, int32_t n,
+                     void *k /*device*/, void *v /*device*/);
+int sparsk_set_len(sparsk_ctx *ctx, int32_t slot, int32_t len);
+/* Host view of a slot: positions held and pending count (no device access). */
+int sparsk_slot_state(const sparsk_ctx *ctx, int32_t slot, int32_t *len /*host*/,
+                      int32_t *pending /*host*/);
+
+/* Parity hooks.  While non-NULL, every decode step also writes, for sequence i of the step,
+ * the hidden state its head read (exit_hidden [n, d] fp32) and its logits (exit_logits
+ * [n, V_t+V_s] fp32, -inf outside the modality's id range).  Device pointers, caller-owned. */
+int sparsk_set_debug(sparsk_ctx *ctx, float *exit_hidden /*device or NULL*/,
+                     float *exit_logits /*device or NULL*/);
+
+/* Tuning knobs, by name: "gemm_min_rows" (row count from which the tcgen05 path is used; a
+ * large value keeps everything on the GEMV path), "use_graph" (0/1), "attn_split" (positions
+ * per KV split), "pdl" (0/1, programmatic dependent launch between the kernels of a step),
+ * "gemv_ks" / "gemv_r" (override the GEMV team width / rows per group; 0 = automatic),
+ * "time_kernel" (see sparsk_kernel_time).  Returns SPARSK_EINVAL for an unknown name or value. */
+int sparsk_set_option(sparsk_ctx *ctx, const char *name /*host*/, int64_t value);
+
+/* Per-kernel timing for roofline reports.  sparsk_set_option(ctx, "time_kernel", c) with c =
+ * 1 QKV, 2 attention, 3 O-projection, 4 gate/up, 5 down-projection, 6 exit head brackets every
+ * later launch of that class with CUDA events on the context's stream (up to 8192 launches; 0
+ * stops).  sparsk_kernel_time synchronises the stream and returns the summed device time of the
+ * bracketed launches and their number.  No counterpart in the paper: measurement only. */
+int sparsk_kernel_time(sparsk_ctx *ctx, double *total_ms /*host*/, int64_t *n_launches /*host*/);
+
+/* Number of kernels this library has launched on behalf of the context so far. */
+int64_t sparsk_launch_count(const sparsk_ctx *ctx);
+
+/* Text of the last error of this context (host string, valid until the next call). */
+const char *sparsk_last_error(const sparsk_ctx *ctx);
+
+/* Release host-side state.  The workspace and weights are the caller's to free. */
+int sparsk_destroy(sparsk_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPARSK_H */

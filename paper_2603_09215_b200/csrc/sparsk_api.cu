@@ -1,0 +1,787 @@
+// Host side of the SPAR-K decode library: argument checks, the host mirror of the exit
+// schedule (which only sizes launches; the device kernels are authoritative), workspace
+// carving and the launch sequence of a step.  C ABI declared in include/sparsk.h.
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <vector>
+
+#include "../../include/sparsk.h"
+#include "sparsk_attn.cuh"
+#include "sparsk_common.cuh"
+#include "sparsk_gemv.cuh"
+#include "sparsk_step.cuh"
+
+using namespace sparsk;
+
+namespace {
+
+constexpr int MAX_SPLITS = 32;
+constexpr int MIN_SPLIT_LEN = 64;
+constexpr int STAGE_RING = 16;
+constexpr uint32_t CTX_MAGIC = 0x5350524bu;  // "SPRK"
+constexpr size_t TIME_POOL = 8192;           // event pairs available to the kernel timer
+enum { KC_MISC = 0, KC_QKV = 1, KC_ATTN = 2, KC_OPROJ = 3, KC_GATEUP = 4, KC_DOWN = 5, KC_HEAD = 6 };
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Carve {
+    char *base;
+    size_t off;
+    template <class T>
+    T *take(size_t n)
+    {
+        off = align_up(off, 256);
+        T *p = base ? reinterpret_cast<T *>(base + off) : nullptr;
+        off += n * sizeof(T);
+        return p;
+    }
+};
+
+}  // namespace
+
+struct sparsk_ctx {
+    uint32_t magic;
+    sparsk_dims dm;
+    std::vector<const bf16 *> attn_norm, wq, wk, wv, wo, mlp_norm, w_gate, w_up, w_down, head_norm, head_proj;
+    const bf16 *embed;
+    cudaStream_t stream;
+    int n_sm;
+    int cap_rows;  // rows any pass may have
+    // workspace
+    bf16 *kcache, *vcache;
+    float *pend_h;
+    int *kv_len, *pend_cnt;
+    float2 *rope;
+    StepDesc sd;
+    int *staged, *tok_dev, *out_tok_dev, *out_depth_dev;
+    int *pf_slot, *pf_pos, *pf_grp_row0, *pf_grp_nrows, *pf_ngrp, *pf_nrows;
+    float *h_lo, *h_up;
+    bf16 *qbuf, *attn_o, *act;
+    float *part_o;
+    float2 *part_ml;
+    // pinned staging ring for the per-step host arrays
+    int *stage_host[STAGE_RING];
+    cudaEvent_t stage_ev[STAGE_RING];
+    int stage_next;
+    // host mirror of per-slot state
+    std::vector<int> h_len, h_pend;
+    // options
+    int pdl, attn_split, gemm_min_rows, use_graph, gv_ks, gv_r, gv_grid_mult;
+    float *dbg_hidden, *dbg_logits;
+    int64_t launches;
+    // optional per-kernel-class timing (events around every launch of one class)
+    int cur_class, time_class;
+    std::vector<cudaEvent_t> tev;
+    size_t tev_used;
+    char err[512];
+};
+
+namespace {
+
+int fail(sparsk_ctx *c, int code, const char *fmt, ...)
+{
+    if (c) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(c->err, sizeof c->err, fmt, ap);
+        va_end(ap);
+    }
+    return code;
+}
+
+#define CU(call)                                                                                   \
+    do {                                                                                           \
+        cudaError_t e_ = (call);                                                                   \
+        if (e_ != cudaSuccess)                                                                     \
+            return fail(ctx, SPARSK_ECUDA, "%s failed: %s (%s:%d)", #call, cudaGetErrorString(e_), \
+                        __FILE__, __LINE__);                                                       \
+    } while (0)
+
+bool dims_ok(const sparsk_dims *d)
+{
+    if (!d) return false;
+    if (d->n_layers < 1 || d->d_model < 8 || d->d_model % 8) return false;
+    if (d->n_q_heads < 1 || d->n_kv_heads < 1 || d->n_q_heads % d->n_kv_heads) return false;
+    if (d->head_dim != 64 && d->head_dim != 128) return false;
+    if (d->d_ffn < 8 || d->d_ffn % 8) return false;
+    if (d->vocab_text < 1 || d->vocab_speech < 0) return false;
+    if (!(d->rms_eps >= 0.f) || !(d->rope_base > 0.f)) return false;
+    if (d->exit_layer < 1 || d->exit_layer > d->n_layers) return false;
+    if (d->refresh_period < 1 || d->refresh_phase < 0 || d->refresh_phase >= d->refresh_period) return false;
+    if (d->text_exit != 0 && d->text_exit != 1) return false;
+    if (d->max_seqs < 1 || d->max_seqs > 1024 || d->max_seq_len < 1) return false;
+    if (d->max_pending < 0 || d->prefill_rows < 0) return false;
+    return true;
+}
+
+int cap_rows_of(const sparsk_dims *d)
+{
+    const int pf = d->prefill_rows > 0 ? d->prefill_rows : 64;
+    const long dec = (long)d->max_seqs * (d->max_pending + 1);
+    return (int)std::max<long>(dec, pf);
+}
+
+// Lays the workspace out; with base == NULL only measures it.
+size_t carve(sparsk_ctx *c, const sparsk_dims *d, char *base)
+{
+    Carve w{base, 0};
+    const size_t B = d->max_seqs, S = d->max_seq_len, L = d->n_layers;
+    const size_t kvrow = (size_t)d->n_kv_heads * d->head_dim, qrow = (size_t)d->n_q_heads * d->head_dim;
+    const size_t R = cap_rows_of(d);
+    bf16 *kc = w.take<bf16>(L * B * S * kvrow);
+    bf16 *vc = w.take<bf16>(L * B * S * kvrow);
+    float *ph = w.take<float>(B * (size_t)std::max(1, d->max_pending) * d->d_model);
+    int *kl = w.take<int>(B), *pc = w.take<int>(B);
+    float2 *rope = w.take<float2>(S * (d->head_dim / 2));
+    StepDesc sd;
+    sd.slot = w.take<int>(B); sd.modality = w.take<int>(B); sd.counter = w.take<int>(B);
+    sd.token = w.take<int>(B); sd.depth = w.take<int>(B); sd.lo_pos = w.take<int>(B);
+    sd.lo_grp_row0 = w.take<int>(B); sd.lo_grp_nrows = w.take<int>(B);
+    sd.up_slot = w.take<int>(R); sd.up_pos = w.take<int>(R); sd.up_src = w.take<int>(R);
+    sd.up_grp_row0 = w.take<int>(B); sd.up_grp_nrows = w.take<int>(B); sd.cur_row = w.take<int>(B);
+    sd.list_seq = w.take<int>(4 * B); sd.list_row = w.take<int>(4 * B);
+    sd.counts = w.take<int>(8);
+    sd.argmax = w.take<unsigned long long>(B);
+    int *staged = w.take<int>(3 * B), *tok = w.take<int>(B), *ot = w.take<int>(B), *od = w.take<int>(B);
+    int *pfs = w.take<int>(R), *pfp = w.take<int>(R), *pfg0 = w.take<int>(1), *pfgn = w.take<int>(1);
+    int *pfng = w.take<int>(1), *pfnr = w.take<int>(1);
+    float *hlo = w.take<float>(B * d->d_model), *hup = w.take<float>(R * d->d_model);
+    bf16 *q = w.take<bf16>(R * qrow), *ao = w.take<bf16>(R * qrow), *act = w.take<bf16>(R * d->d_ffn);
+    float *po = w.take<float>(R * d->n_q_heads * MAX_SPLITS * d->head_dim);
+    float2 *pml = w.take<float2>(R * d->n_q_heads * MAX_SPLITS);
+    if (c) {
+        c->kcache = kc; c->vcache = vc; c->pend_h = ph; c->kv_len = kl; c->pend_cnt = pc; c->rope = rope;
+        c->sd = sd; c->staged = staged; c->tok_dev = tok; c->out_tok_dev = ot; c->out_depth_dev = od;
+        c->pf_slot = pfs; c->pf_pos = pfp; c->pf_grp_row0 = pfg0; c->pf_grp_nrows = pfgn;
+        c->pf_ngrp = pfng; c->pf_nrows = pfnr;
+        c->h_lo = hlo; c->h_up = hup; c->qbuf = q; c->attn_o = ao; c->act = act;
+        c->part_o = po; c->part_ml = pml;
+    }
+    return align_up(w.off, 256);
+}
+
+template <class... KArgs, class... Args>
+cudaError_t launch(sparsk_ctx *c, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, Args... args)
+{
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = c->stream;
+    cudaLaunchAttribute attr[1];
+    if (c->pdl) {
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+    c->launches++;
+    const bool timed = c->time_class == c->cur_class && c->time_class != KC_MISC && c->tev_used + 2 <= c->tev.size();
+    if (timed) cudaEventRecord(c->tev[c->tev_used++], c->stream);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+    if (timed) cudaEventRecord(c->tev[c->tev_used++], c->stream);
+    return e;
+}
+
+// ---------------------------------------------------------------- GEMV dispatch
+struct GvPlan {
+    int ks, grid_x;
+};
+
+GvPlan plan_gemv(const sparsk_ctx *c, int n_groups, int K)
+{
+    const int chunks = (K + 255) / 256;
+    int best_ks = 1;
+    double best = 1e30;
+    for (int ks = 1; ks <= GV_WARPS; ks *= 2) {
+        if (ks > 1 && ks > chunks) break;
+        const long T = (long)c->n_sm * (GV_WARPS / ks);
+        const long iters = (n_groups + T - 1) / T;
+        const double cost = (double)iters * ((chunks + ks - 1) / ks + 3.0);
+        if (cost < best - 1e-9) {
+            best = cost;
+            best_ks = ks;
+        }
+    }
+    if (c->gv_ks > 0) best_ks = c->gv_ks;
+    GvPlan p;
+    p.ks = best_ks;
+    p.grid_x = std::min(c->n_sm, n_groups);
+    if (p.grid_x < 1) p.grid_x = 1;
+    return p;
+}
+
+template <class Op, int R, int M, bool NORM>
+cudaError_t launch_gemv_inst(sparsk_ctx *c, const Op &op, GvIn in, int n_groups)
+{
+    static bool attr_set = false;
+    auto kern = gemv_kernel<Op, R, M, NORM>;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    const GvPlan p = plan_gemv(c, n_groups, in.K);
+    in.ks = p.ks;
+    const size_t smem = align_up((size_t)M * in.K * 2, 16) + (size_t)2 * GV_WARPS * R * M * sizeof(float);
+    if (smem > 200 * 1024) return cudaErrorInvalidValue;
+    const int passes = (M == GV_MC) ? (in.n_rows + GV_MC - 1) / GV_MC : 1;
+    return launch(c, kern, dim3(p.grid_x, passes), dim3(GV_THREADS), smem, op, in);
+}
+
+// M template: 1, 2 or 4 (three rows run as four with one masked).
+#define GV_DISPATCH_M(OPT, RR, NORM, op, in, ng)                                    \
+    ((in).n_rows == 1   ? launch_gemv_inst<OPT<RR>, RR, 1, NORM>(c, op, in, ng)     \
+     : (in).n_rows == 2 ? launch_gemv_inst<OPT<RR>, RR, 2, NORM>(c, op, in, ng)     \
+                        : launch_gemv_inst<OPT<RR>, RR, 4, NORM>(c, op, in, ng))
+
+int pick_r(const sparsk_ctx *c, int n_rows, bool paired)
+{
+    if (c->gv_r > 0) return (paired && c->gv_r < 2) ? 2 : c->gv_r;
+    if (n_rows >= 3) return 4;
+    return 2;
+}
+
+struct RowSet {
+    const int *slot, *pos, *grp_row0, *grp_nrows, *n_groups, *n_rows_dev;
+    int n_rows;     // host count (sizes the launches)
+    int n_groups_h; // host count
+    int max_grp_rows;
+    int max_len;    // longest prefix any row attends to (host)
+};
+
+cudaError_t run_qkv(sparsk_ctx *c, int layer, const float *h, const RowSet &rs)
+{
+    const sparsk_dims &d = c->dm;
+    const int li = layer - 1;
+    GvIn in{};
+    in.h = h; in.gain = c->attn_norm[li]; in.eps = d.rms_eps; in.K = d.d_model; in.n_rows = rs.n_rows;
+    const size_t lstride = (size_t)d.max_seqs * d.n_kv_heads * d.max_seq_len * d.head_dim;
+    const int R = pick_r(c, rs.n_rows, true);
+#define QKV_CASE(RR)                                                                                   \
+    {                                                                                                  \
+        QkvOp<RR> op;                                                                                  \
+        op.wq = c->wq[li]; op.wk = c->wk[li]; op.wv = c->wv[li]; op.q_out = c->qbuf;                   \
+        op.kc = c->kcache + li * lstride; op.vc = c->vcache + li * lstride; op.rope = c->rope;         \
+        op.row_slot = rs.slot; op.row_pos = rs.pos; op.d = d.d_model; op.Hq = d.n_q_heads;             \
+        op.Hkv = d.n_kv_heads; op.hd = d.head_dim; op.S = d.max_seq_len;                               \
+        const int P = RR / 2;                                                                          \
+        const int ng = (d.n_q_heads + d.n_kv_heads) * (d.head_dim / 2) / P + d.n_kv_heads * d.head_dim / RR; \
+        return GV_DISPATCH_M(QkvOp, RR, true, op, in, ng);                                             \
+    }
+    if (R == 4) QKV_CASE(4) else QKV_CASE(2)
+#undef QKV_CASE
+}
+
+cudaError_t run_resid(sparsk_ctx *c, const bf16 *w, const bf16 *x, float *h, int K, int n_out, int n_rows)
+{
+    GvIn in{};
+    in.x = x; in.K = K; in.n_rows = n_rows;
+    int R = c->gv_r > 0 ? c->gv_r : (n_rows >= 3 ? 4 : 2);
+#define RES_CASE(RR)                                            \
+    {                                                           \
+        ResidOp<RR> op;                                         \
+        op.w = w; op.h = h; op.K = K; op.n_out = n_out;         \
+        const int ng = (n_out + RR - 1) / RR;                   \
+        return GV_DISPATCH_M(ResidOp, RR, false, op, in, ng);   \
+    }
+    if (R == 4) RES_CASE(4) else if (R == 2) RES_CASE(2) else RES_CASE(1)
+#undef RES_CASE
+}
+
+cudaError_t run_gateup(sparsk_ctx *c, int layer, const float *h, int n_rows)
+{
+    const sparsk_dims &d = c->dm;
+    const int li = layer - 1;
+    GvIn in{};
+    in.h = h; in.gain = c->mlp_norm[li]; in.eps = d.rms_eps; in.K = d.d_model; in.n_rows = n_rows;
+    const int R = pick_r(c, n_rows, true);
+#define GU_CASE(RR)                                                              \
+    {                                                                            \
+        GateUpOp<RR> op;                                                         \
+        op.wg = c->w_gate[li]; op.wu = c->w_up[li]; op.u = c->act;               \
+        op.d = d.d_model; op.F = d.d_ffn;                                        \
+        const int P = RR / 2;                                                    \
+        const int ng = (d.d_ffn + P - 1) / P;                                    \
+        return GV_DISPATCH_M(GateUpOp, RR, true, op, in, ng);                    \
+    }
+    if (R == 4) GU_CASE(4) else GU_CASE(2)
+#undef GU_CASE
+}
+
+// Head of `layer` over list `l` (0 early/text, 1 early/speech, 2 full/text, 3 full/speech).
+cudaError_t run_head(sparsk_ctx *c, int layer, const float *h, int list, int n_rows)
+{
+    const sparsk_dims &d = c->dm;
+    const int li = layer - 1, B = d.max_seqs;
+    GvIn in{};
+    in.h = h; in.gain = c->head_norm[li]; in.eps = d.rms_eps; in.K = d.d_model; in.n_rows = n_rows;
+    in.row_idx = c->sd.list_row + (size_t)list * B;
+    const int speech = list & 1;
+    const int R = c->gv_r > 0 ? c->gv_r : 4;
+    struct ClassScope {
+        sparsk_ctx *c;
+        ~ClassScope() { c->cur_class = KC_MISC; }
+    } scope{c};
+    c->cur_class = KC_HEAD;
+#define HD_CASE(RR)                                                                              \
+    {                                                                                            \
+        HeadOp<RR> op;                                                                           \
+        op.w = c->head_proj[li]; op.seq_of_row = c->sd.list_seq + (size_t)list * B;              \
+        op.argmax = c->sd.argmax; op.logits = c->dbg_logits; op.d = d.d_model;                   \
+        op.lo = speech ? d.vocab_text : 0; op.hi = speech ? d.vocab_text + d.vocab_speech : d.vocab_text; \
+        op.V = d.vocab_text + d.vocab_speech;                                                    \
+        const int ng = (op.hi - op.lo + RR - 1) / RR;                                            \
+        return GV_DISPATCH_M(HeadOp, RR, true, op, in, ng);                                      \
+    }
+    if (R == 4) HD_CASE(4) else if (R == 2) HD_CASE(2) else HD_CASE(1)
+#undef HD_CASE
+}
+
+cudaError_t run_attn(sparsk_ctx *c, int layer, const RowSet &rs)
+{
+    const sparsk_dims &d = c->dm;
+    const int G = d.n_q_heads / d.n_kv_heads;
+    const size_t lstride = (size_t)d.max_seqs * d.n_kv_heads * d.max_seq_len * d.head_dim;
+    AttnArgs a{};
+    a.q = c->qbuf;
+    a.kc = c->kcache + (layer - 1) * lstride;
+    a.vc = c->vcache + (layer - 1) * lstride;
+    a.grp_row0 = rs.grp_row0; a.grp_nrows = rs.grp_nrows; a.row_slot = rs.slot; a.row_pos = rs.pos;
+    a.n_groups = rs.n_groups;
+    a.part_o = c->part_o; a.part_ml = c->part_ml; a.out = c->attn_o;
+    a.Hq = d.n_q_heads; a.Hkv = d.n_kv_heads; a.S = d.max_seq_len;
+    a.n_qblk = (rs.max_grp_rows * G + AT_QB - 1) / AT_QB;
+    // enough splits to fill the machine, none shorter than MIN_SPLIT_LEN
+    int split = c->attn_split;
+    if (split <= 0) {
+        const long base = (long)rs.n_groups_h * a.n_qblk * d.n_kv_heads;
+        long want = std::max<long>(1, (2L * c->n_sm + base - 1) / base);
+        want = std::min<long>(want, MAX_SPLITS);
+        split = (int)((rs.max_len + want - 1) / want);
+        split = std::max(split, MIN_SPLIT_LEN);
+    }
+    split = (split + AT_TILE - 1) / AT_TILE * AT_TILE;
+    int n_splits = (rs.max_len + split - 1) / split;
+    if (n_splits > MAX_SPLITS) {
+        n_splits = MAX_SPLITS;
+        split = ((rs.max_len + n_splits - 1) / n_splits + AT_TILE - 1) / AT_TILE * AT_TILE;
+        n_splits = (rs.max_len + split - 1) / split;
+    }
+    a.split_len = split;
+    a.n_splits = n_splits;
+    dim3 grid(rs.n_groups_h * a.n_qblk, d.n_kv_heads, n_splits);
+    cudaError_t e;
+    if (d.head_dim == 128) {
+        e = launch(c, attn_partial_kernel<128>, grid, dim3(AT_THREADS), 0, a);
+        if (e != cudaSuccess) return e;
+        return launch(c, attn_merge_kernel<128>, dim3(rs.n_rows, d.n_q_heads), dim3(128), 0, a, rs.n_rows_dev);
+    }
+    e = launch(c, attn_partial_kernel<64>, grid, dim3(AT_THREADS), 0, a);
+    if (e != cudaSuccess) return e;
+    return launch(c, attn_merge_kernel<64>, dim3(rs.n_rows, d.n_q_heads), dim3(64), 0, a, rs.n_rows_dev);
+}
+
+// One transformer layer over a row set: h <- h^(layer).
+cudaError_t run_layer(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
+{
+    const sparsk_dims &d = c->dm;
+    const int li = layer - 1;
+    cudaError_t e;
+    c->cur_class = KC_QKV;
+    if ((e = run_qkv(c, layer, h, rs)) != cudaSuccess) return e;
+    c->cur_class = KC_ATTN;
+    if ((e = run_attn(c, layer, rs)) != cudaSuccess) return e;
+    c->cur_class = KC_OPROJ;
+    if ((e = run_resid(c, c->wo[li], c->attn_o, h, d.n_q_heads * d.head_dim, d.d_model, rs.n_rows)) != cudaSuccess) return e;
+    c->cur_class = KC_GATEUP;
+    if ((e = run_gateup(c, layer, h, rs.n_rows)) != cudaSuccess) return e;
+    c->cur_class = KC_DOWN;
+    e = run_resid(c, c->w_down[li], c->act, h, d.d_ffn, d.d_model, rs.n_rows);
+    c->cur_class = KC_MISC;
+    return e;
+}
+
+bool good(const sparsk_ctx *c) { return c && c->magic == CTX_MAGIC; }
+
+}  // namespace
+
+// =============================================================================== C ABI
+
+extern "C" size_t sparsk_workspace_bytes(const sparsk_dims *dims)
+{
+    if (!dims_ok(dims)) return 0;
+    return carve(nullptr, dims, nullptr);
+}
+
+extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, void *workspace,
+                             size_t workspace_bytes, void *cuda_stream, sparsk_ctx **out)
+{
+    if (!out) return SPARSK_EINVAL;
+    *out = nullptr;
+    if (!dims_ok(dims) || !w || !workspace) return SPARSK_EINVAL;
+    if ((uintptr_t)workspace % 256) return SPARSK_EINVAL;
+    if (workspace_bytes < sparsk_workspace_bytes(dims)) return SPARSK_EINVAL;
+    const int L = dims->n_layers, e = dims->exit_layer;
+    const void *const *arrs[] = {w->attn_norm, w->wq, w->wk, w->wv, w->wo, w->mlp_norm, w->w_gate, w->w_up, w->w_down};
+    if (!w->embed || ((uintptr_t)w->embed % 16) || !w->head_norm || !w->head_proj) return SPARSK_EINVAL;
+    for (auto a : arrs) {
+        if (!a) return SPARSK_EINVAL;
+        for (int l = 0; l < L; l++)
+            if (!a[l] || ((uintptr_t)a[l] % 16)) return SPARSK_EINVAL;
+    }
+    for (int l = 0; l < L; l++)
+        if (((uintptr_t)w->head_norm[l] % 16) || ((uintptr_t)w->head_proj[l] % 16)) return SPARSK_EINVAL;
+    if (((size_t)dims->vocab_text * dims->d_model * 2) % 16) return SPARSK_EINVAL;
+    // the heads of layers e and L are what the periodic schedule reads
+    if (!w->head_norm[L - 1] || !w->head_proj[L - 1]) return SPARSK_ENOHEAD;
+    if (dims->refresh_period > 1 && e < L && (!w->head_norm[e - 1] || !w->head_proj[e - 1])) return SPARSK_ENOHEAD;
+
+    sparsk_ctx *ctx = new (std::nothrow) sparsk_ctx();
+    if (!ctx) return SPARSK_EINVAL;
+    ctx->magic = CTX_MAGIC;
+    ctx->dm = *dims;
+    if (ctx->dm.prefill_rows <= 0) ctx->dm.prefill_rows = 64;
+    ctx->stream = (cudaStream_t)cuda_stream;
+    ctx->err[0] = 0;
+    auto cp = [&](std::vector<const bf16 *> &dst, const void *const *src) {
+        dst.resize(L);
+        for (int l = 0; l < L; l++) dst[l] = (const bf16 *)src[l];
+    };
+    cp(ctx->attn_norm, w->attn_norm); cp(ctx->wq, w->wq); cp(ctx->wk, w->wk); cp(ctx->wv, w->wv);
+    cp(ctx->wo, w->wo); cp(ctx->mlp_norm, w->mlp_norm); cp(ctx->w_gate, w->w_gate); cp(ctx->w_up, w->w_up);
+    cp(ctx->w_down, w->w_down); cp(ctx->head_norm, w->head_norm); cp(ctx->head_proj, w->head_proj);
+    ctx->embed = (const bf16 *)w->embed;
+    ctx->cap_rows = cap_rows_of(&ctx->dm);
+    carve(ctx, &ctx->dm, (char *)workspace);
+    ctx->h_len.assign(dims->max_seqs, 0);
+    ctx->h_pend.assign(dims->max_seqs, 0);
+    ctx->pdl = 0; ctx->attn_split = 0; ctx->gemm_min_rows = 1 << 30; ctx->use_graph = 0;
+    ctx->gv_ks = 0; ctx->gv_r = 0; ctx->gv_grid_mult = 1;
+    ctx->dbg_hidden = nullptr; ctx->dbg_logits = nullptr;
+    ctx->launches = 0;
+    ctx->cur_class = KC_MISC; ctx->time_class = KC_MISC; ctx->tev_used = 0;
+    ctx->stage_next = 0;
+    for (int i = 0; i < STAGE_RING; i++) { ctx->stage_host[i] = nullptr; ctx->stage_ev[i] = nullptr; }
+
+    int rc = SPARSK_OK;
+    do {
+        int dev = 0;
+        cudaError_t ce;
+        if ((ce = cudaGetDevice(&dev)) != cudaSuccess ||
+            (ce = cudaDeviceGetAttribute(&ctx->n_sm, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) {
+            rc = fail(ctx, SPARSK_ECUDA, "device query failed: %s", cudaGetErrorString(ce));
+            break;
+        }
+        for (int i = 0; i < STAGE_RING && rc == SPARSK_OK; i++) {
+            if ((ce = cudaHostAlloc((void **)&ctx->stage_host[i], 3 * sizeof(int) * dims->max_seqs, cudaHostAllocDefault)) != cudaSuccess ||
+                (ce = cudaEventCreateWithFlags(&ctx->stage_ev[i], cudaEventDisableTiming)) != cudaSuccess)
+                rc = fail(ctx, SPARSK_ECUDA, "staging setup failed: %s", cudaGetErrorString(ce));
+        }
+        if (rc) break;
+        // rotary table in double, stored as float (cos, sin)
+        const int half = dims->head_dim / 2;
+        std::vector<float2> tab((size_t)dims->max_seq_len * half);
+        for (int i = 0; i < half; i++) {
+            const double inv = std::pow((double)dims->rope_base, -2.0 * i / dims->head_dim);
+            for (int p = 0; p < dims->max_seq_len; p++) {
+                const double th = (double)p * inv;
+                tab[(size_t)p * half + i] = make_float2((float)std::cos(th), (float)std::sin(th));
+            }
+        }
+        if ((ce = cudaMemcpyAsync(ctx->rope, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess ||
+            (ce = cudaMemsetAsync(ctx->kv_len, 0, sizeof(int) * dims->max_seqs, ctx->stream)) != cudaSuccess ||
+            (ce = cudaMemsetAsync(ctx->pend_cnt, 0, sizeof(int) * dims->max_seqs, ctx->stream)) != cudaSuccess ||
+            (ce = cudaMemsetAsync(ctx->sd.counts, 0, sizeof(int) * 8, ctx->stream)) != cudaSuccess ||
+            (ce = cudaStreamSynchronize(ctx->stream)) != cudaSuccess) {
+            rc = fail(ctx, SPARSK_ECUDA, "table upload failed: %s", cudaGetErrorString(ce));
+            break;
+        }
+    } while (0);
+    if (rc != SPARSK_OK) {
+        sparsk_destroy(ctx);
+        return rc;
+    }
+    *out = ctx;
+    return SPARSK_OK;
+}
+
+extern "C" int sparsk_destroy(sparsk_ctx *ctx)
+{
+    if (!good(ctx)) return SPARSK_ESTATE;
+    cudaStreamSynchronize(ctx->stream);
+    for (int i = 0; i < STAGE_RING; i++) {
+        if (ctx->stage_host[i]) cudaFreeHost(ctx->stage_host[i]);
+        if (ctx->stage_ev[i]) cudaEventDestroy(ctx->stage_ev[i]);
+    }
+    for (cudaEvent_t ev : ctx->tev) cudaEventDestroy(ev);
+    ctx->magic = 0;
+    delete ctx;
+    return SPARSK_OK;
+}
+
+extern "C" const char *sparsk_last_error(const sparsk_ctx *ctx) { return good(ctx) ? ctx->err : "invalid context"; }
+extern "C" int64_t sparsk_launch_count(const sparsk_ctx *ctx) { return good(ctx) ? ctx->launches : -1; }
+
+extern "C" int sparsk_set_debug(sparsk_ctx *ctx, float *exit_hidden, float *exit_logits)
+{
+    if (!good(ctx)) return SPARSK_ESTATE;
+    ctx->dbg_hidden = exit_hidden;
+    ctx->dbg_logits = exit_logits;
+    return SPARSK_OK;
+}
+
+extern "C" int sparsk_set_option(sparsk_ctx *ctx, const char *name, int64_t value)
+{
+    if (!good(ctx)) return SPARSK_ESTATE;
+    if (!name) return fail(ctx, SPARSK_EINVAL, "option name is NULL");
+    if (!strcmp(name, "gemm_min_rows") && value >= 1) ctx->gemm_min_rows = (int)std::min<int64_t>(value, 1 << 30);
+    else if (!strcmp(name, "use_graph") && (value == 0 || value == 1)) ctx->use_graph = (int)value;
+    else if (!strcmp(name, "pdl") && (value == 0 || value == 1)) ctx->pdl = (int)value;
+    else if (!strcmp(name, "attn_split") && value >= 0 && value <= (1 << 24)) ctx->attn_split = (int)value;
+    else if (!strcmp(name, "gemv_ks") && (value == 0 || value == 1 || value == 2 || value == 4 || value == 8 || value == 16)) ctx->gv_ks = (int)value;
+    else if (!strcmp(name, "gemv_r") && (value == 0 || value == 1 || value == 2 || value == 4)) ctx->gv_r = (int)value;
+    else if (!strcmp(name, "time_kernel") && value >= 0 && value <= KC_HEAD) {
+        // start (or stop, with 0) timing every launch of one kernel class; resets the totals
+        if (value && ctx->tev.empty()) {
+            ctx->tev.resize(2 * TIME_POOL);
+            for (auto &ev : ctx->tev) CU(cudaEventCreate(&ev));
+        }
+        ctx->time_class = (int)value;
+        ctx->tev_used = 0;
+    } else return fail(ctx, SPARSK_EINVAL, "unknown option or bad value: %s=%lld", name, (long long)value);
+    return SPARSK_OK;
+}
+
+extern "C" int sparsk_kernel_time(sparsk_ctx *ctx, double *total_ms, int64_t *n_launches)
+{
+    if (!good(ctx)) return SPARSK_ESTATE;
+    if (!total_ms || !n_launches) return fail(ctx, SPARSK_EINVAL, "kernel_time: NULL output");
+    CU(cudaStreamSynchronize(ctx->stream));
+    double tot = 0.0;
+    for (size_t i = 0; i + 1 < ctx->tev_used; i += 2) {
+        float ms = 0.f;
+        CU(cudaEventElapsedTime(&ms, ctx->tev[i], ctx->tev[i + 1]));
+        tot += ms;
+    }
+    *total_ms = tot;
+    *n_launches = (int64_t)(ctx->tev_used / 2);
+    return SPARSK_OK;
+}
+
+extern "C" int sparsk_reset_slot(sparsk_ctx *ctx, int32_t slot) { return sparsk_set_len(ctx, slot, 0); }
+
+extern "C" int sparsk_set_len(sparsk_ctx *ctx, int32_t slot, int32_t len)
+{
+    if (!good(ctx)) return SPARSK_ESTATE;
+    if (slot < 0 || slot >= ctx->dm.max_seqs || len < 0 || len > ctx->dm.max_seq_len)
+        return fail(ctx, SPARSK_EINVAL, "set_len: slot %d / len %d out of range", slot, len);
+    CU(launch(ctx, set_int_kernel, dim3(1), dim3(1), 0, ctx->kv_len + slot, (int)len));
+    CU(launch(ctx, set_int_kernel, dim3(1), dim3(1), 0, ctx->pend_cnt + slot, 0));
+    ctx->h_len[slot] = len;
+    ctx->h_pend[slot] = 0;
+    return SPARSK_OK;
+}
+
+extern "C" int sparsk_slot_state(const sparsk_ctx *ctx, int32_t slot, int32_t *len, int32_t *pending)
+{
+    if (!good(ctx)) return SPARSK_ESTATE;
+    if (slot < 0 || slot >= ctx->dm.max_seqs) return SPARSK_EINVAL;
+    if (len) *len = ctx->h_len[slot];
+    if (pending) *pending = ctx->h_pend[slot];
+    return SPARSK_OK;
+}
+
+static int kv_io(sparsk_ctx *ctx, int32_t slot, int32_t layer, int32_t first_pos, int32_t n, void *k, void *v, int to_cache)
+{
+    if (!good(ctx)) return SPARSK_ESTATE;
+    const sparsk_dims &d = ctx->dm;
+    if (slot < 0 || slot >= d.max_seqs || layer < 1 || layer > d.n_layers || first_pos < 0 || n < 0 ||
+        (long)first_pos + n > d.max_seq_len || !k || !v)
+        return fail(ctx, SPARSK_EINVAL, "kv import/export: argument out of range");
+    if (n == 0) return SPARSK_OK;
+    const size_t per_slot = (size_t)d.n_kv_heads * d.max_seq_len * d.head_dim;
+    const size_t off = ((size_t)(layer - 1) * d.max_seqs + slot) * per_slot;
+    const size_t total = (size_t)n * d.n_kv_heads * d.head_dim;
+    const int blocks = (int)std::min<size_t>((total + 255) / 256, 4096);
+    CU(launch(ctx, kv_copy_kernel, dim3(blocks), dim3(256), 0, ctx->kcache + off, ctx->vcache + off, (bf16 *)k,
+              (bf16 *)v, (int)first_pos, (int)n, d.n_kv_heads, d.head_dim, d.max_seq_len, to_cache));
+    return SPARSK_OK;
+}
+extern "C" int sparsk_import_kv(sparsk_ctx *ctx, int32_t slot, int32_t layer, int32_t first_pos, int32_t n,
+                                const void *k, const void *v)
+{
+    return kv_io(ctx, slot, layer, first_pos, n, const_cast<void *>(k), const_cast<void *>(v), 1);
+}
+extern "C" int sparsk_export_kv(sparsk_ctx *ctx, int32_t slot, int32_t layer, int32_t first_pos, int32_t n,
+                                void *k, void *v)
+{
+    return kv_io(ctx, slot, layer, first_pos, n, k, v, 0);
+}
+
+// --------------------------------------------------------------------------- prefill
+extern "C" int sparsk_prefill(sparsk_ctx *ctx, int32_t n_seqs, const int32_t *slots, const int32_t *tokens,
+                              const int32_t *offsets)
+{
+    if (!good(ctx)) return SPARSK_ESTATE;
+    const sparsk_dims &d = ctx->dm;
+    if (n_seqs < 0 || n_seqs > d.max_seqs || (n_seqs && (!slots || !tokens || !offsets)))
+        return fail(ctx, SPARSK_EINVAL, "prefill: bad arguments");
+    std::vector<char> seen(d.max_seqs, 0);
+    for (int i = 0; i < n_seqs; i++) {
+        const int s = slots[i];
+        if (s < 0 || s >= d.max_seqs || seen[s]) return fail(ctx, SPARSK_EINVAL, "prefill: slot %d invalid or repeated", s);
+        seen[s] = 1;
+        const long n = (long)offsets[i + 1] - offsets[i];
+        if (n < 0 || offsets[i] < 0) return fail(ctx, SPARSK_EINVAL, "prefill: offsets must not decrease");
+        if (ctx->h_pend[s]) return fail(ctx, SPARSK_ESTATE, "prefill: slot %d has pending positions", s);
+        if (ctx->h_len[s] + n > d.max_seq_len) return fail(ctx, SPARSK_ECAPACITY, "prefill: slot %d would hold %ld > %d positions", s, ctx->h_len[s] + n, d.max_seq_len);
+    }
+    const int chunk = std::min(d.prefill_rows, ctx->cap_rows);
+    for (int i = 0; i < n_seqs; i++) {
+        const int s = slots[i];
+        const int total = offsets[i + 1] - offsets[i];
+        for (int done = 0; done < total; done += chunk) {
+            const int n = std::min(chunk, total - done);
+            const int pos0 = ctx->h_len[s];
+            CU(launch(ctx, prefill_rows_kernel, dim3((n + 255) / 256), dim3(256), 0, ctx->pf_slot, ctx->pf_pos,
+                      ctx->pf_grp_row0, ctx->pf_grp_nrows, s, pos0, n));
+            CU(launch(ctx, set_int_kernel, dim3(1), dim3(1), 0, ctx->pf_ngrp, 1));
+            CU(launch(ctx, set_int_kernel, dim3(1), dim3(1), 0, ctx->pf_nrows, n));
+            CU(launch(ctx, embed_kernel, dim3(n), dim3(128), 0, tokens + offsets[i] + done, ctx->embed, ctx->h_up, n, d.d_model,
+                      d.vocab_text + d.vocab_speech, ctx->sd.counts + CNT_STATUS));
+            RowSet rs{ctx->pf_slot, ctx->pf_pos, ctx->pf_grp_row0, ctx->pf_grp_nrows, ctx->pf_ngrp, ctx->pf_nrows,
+                      n, 1, n, pos0 + n};
+            for (int l = 1; l <= d.n_layers; l++) CU(run_layer(ctx, l, ctx->h_up, rs));
+            CU(launch(ctx, set_int_kernel, dim3(1), dim3(1), 0, ctx->kv_len + s, pos0 + n));
+            ctx->h_len[s] = pos0 + n;
+        }
+    }
+    return SPARSK_OK;
+}
+
+// --------------------------------------------------------------------------- decode step
+extern "C" int sparsk_decode_step(sparsk_ctx *ctx, int32_t n, const int32_t *slots, const int32_t *token_ids,
+                                  const uint8_t *modality, const int32_t *counters, int32_t *next_tokens,
+                                  int32_t *exit_depths)
+{
+    if (!good(ctx)) return SPARSK_ESTATE;
+    const sparsk_dims &d = ctx->dm;
+    const int L = d.n_layers, e = d.exit_layer, K = d.refresh_period, r = d.refresh_phase, B = d.max_seqs;
+    if (n < 1 || n > B || !slots || !token_ids || !modality || !counters || !next_tokens || !exit_depths)
+        return fail(ctx, SPARSK_EINVAL, "decode_step: bad arguments (n=%d)", n);
+    // ---- host mirror of the schedule: validates, and sizes the launches
+    std::vector<char> seen(B, 0);
+    int n_list[4] = {0, 0, 0, 0};
+    int m_up = 0, n_grp = 0, max_grp = 1, max_len_lo = 0, max_len_up = 0;
+    for (int i = 0; i < n; i++) {
+        const int s = slots[i];
+        if (s < 0 || s >= B || seen[s]) return fail(ctx, SPARSK_EINVAL, "decode_step: slot %d invalid or repeated", s);
+        seen[s] = 1;
+        if (modality[i] > 1) return fail(ctx, SPARSK_EINVAL, "decode_step: modality[%d]=%d", i, modality[i]);
+        if (counters[i] < 0) return fail(ctx, SPARSK_EINVAL, "decode_step: counter[%d]=%d", i, counters[i]);
+        if (ctx->h_len[s] + 1 > d.max_seq_len) return fail(ctx, SPARSK_ECAPACITY, "decode_step: slot %d is full (%d positions)", s, ctx->h_len[s]);
+        const int depth = (modality[i] == 0 && !d.text_exit) ? L : ((counters[i] % K == r) ? L : e);
+        const bool full = depth == L;
+        if (!full && ctx->h_pend[s] + 1 > d.max_pending)
+            return fail(ctx, SPARSK_ECAPACITY, "decode_step: slot %d would hold %d pending positions (max_pending %d)", s, ctx->h_pend[s] + 1, d.max_pending);
+        n_list[(full ? 2 : 0) + (modality[i] ? 1 : 0)]++;
+        max_len_lo = std::max(max_len_lo, ctx->h_len[s] + 1);
+        if (full && e < L) {
+            m_up += ctx->h_pend[s] + 1;
+            n_grp++;
+            max_grp = std::max(max_grp, ctx->h_pend[s] + 1);
+            max_len_up = std::max(max_len_up, ctx->h_len[s] + 1);
+        }
+    }
+    if ((n_list[0] + n_list[1]) && (!ctx->head_norm[e - 1] || !ctx->head_proj[e - 1]))
+        return fail(ctx, SPARSK_ENOHEAD, "decode_step: layer %d has no exit head", e);
+    if (m_up > ctx->cap_rows) return fail(ctx, SPARSK_ECAPACITY, "decode_step: %d upper rows exceed capacity %d", m_up, ctx->cap_rows);
+
+    // ---- stage the host arrays
+    const int ring = ctx->stage_next;
+    ctx->stage_next = (ring + 1) % STAGE_RING;
+    CU(cudaEventSynchronize(ctx->stage_ev[ring]));
+    int *st = ctx->stage_host[ring];
+    for (int i = 0; i < n; i++) {
+        st[i] = slots[i];
+        st[n + i] = modality[i];
+        st[2 * n + i] = counters[i];
+    }
+    CU(cudaMemcpyAsync(ctx->staged, st, sizeof(int) * 3 * n, cudaMemcpyHostToDevice, ctx->stream));
+    CU(cudaEventRecord(ctx->stage_ev[ring], ctx->stream));
+
+    // ---- schedule, compaction, embedding
+    const int V = d.vocab_text + d.vocab_speech;
+    CU(launch(ctx, schedule_kernel, dim3((n + 127) / 128), dim3(128), 0, ctx->sd, (int)n, (const int *)ctx->staged,
+              (const int *)token_ids, V, L, e, K, r, d.text_exit));
+    CU(launch(ctx, compact_kernel, dim3(1), dim3(1024), 0, ctx->sd, (int)n, (const int *)ctx->kv_len,
+              (const int *)ctx->pend_cnt, L, e, B));
+    CU(launch(ctx, embed_kernel, dim3(n), dim3(128), 0, (const int *)ctx->sd.token, ctx->embed, ctx->h_lo, (int)n, d.d_model,
+              V, ctx->sd.counts + CNT_STATUS));
+    if (ctx->dbg_logits) {
+        const size_t cnt = (size_t)n * V;
+        CU(launch(ctx, fill_kernel, dim3((unsigned)std::min<size_t>((cnt + 255) / 256, 2048)), dim3(256), 0, ctx->dbg_logits, cnt, -INFINITY));
+    }
+    // ---- lower pass: layers 1..e over all sequences
+    RowSet lo{ctx->sd.slot, ctx->sd.lo_pos, ctx->sd.lo_grp_row0, ctx->sd.lo_grp_nrows, ctx->sd.counts + CNT_NSEQ,
+              ctx->sd.counts + CNT_NSEQ, n, n, 1, max_len_lo};
+    for (int l = 1; l <= e; l++) CU(run_layer(ctx, l, ctx->h_lo, lo));
+    // ---- early exits: keep h^(e), read the token from g_e
+    if (n_list[0] + n_list[1]) {
+        CU(launch(ctx, stash_kernel, dim3(n), dim3(128), 0, ctx->sd, (const float *)ctx->h_lo, ctx->pend_h,
+                  (const int *)ctx->pend_cnt, (int)n, d.d_model, L, d.max_pending));
+        for (int l = 0; l < 2; l++)
+            if (n_list[l]) CU(run_head(ctx, e, ctx->h_lo, l, n_list[l]));
+    }
+    // ---- upper pass: pending and current positions of full-depth sequences through e+1..L
+    const float *h_full = ctx->h_lo;
+    if (m_up) {
+        CU(launch(ctx, gather_upper_kernel, dim3(m_up), dim3(128), 0, ctx->sd, (const float *)ctx->h_lo,
+                  (const float *)ctx->pend_h, ctx->h_up, d.d_model, d.max_pending));
+        RowSet up{ctx->sd.up_slot, ctx->sd.up_pos, ctx->sd.up_grp_row0, ctx->sd.up_grp_nrows, ctx->sd.counts + CNT_NGRP,
+                  ctx->sd.counts + CNT_MUP, m_up, n_grp, max_grp, max_len_up};
+        for (int l = e + 1; l <= L; l++) CU(run_layer(ctx, l, ctx->h_up, up));
+        h_full = ctx->h_up;
+    }
+    for (int l = 2; l < 4; l++)
+        if (n_list[l]) CU(run_head(ctx, L, h_full, l, n_list[l]));
+    if (ctx->dbg_hidden)
+        CU(launch(ctx, debug_hidden_kernel, dim3(n), dim3(128), 0, ctx->sd, (const float *)ctx->h_lo,
+                  (const float *)ctx->h_up, ctx->dbg_hidden, (int)n, d.d_model));
+    CU(launch(ctx, finish_kernel, dim3((n + 127) / 128), dim3(128), 0, ctx->sd, (int)n, ctx->kv_len, ctx->pend_cnt,
+              next_tokens, exit_depths, L));
+    // ---- host mirror follows
+    for (int i = 0; i < n; i++) {
+        const int s = slots[i];
+        const int depth = (modality[i] == 0 && !d.text_exit) ? L : ((counters[i] % K == r) ? L : e);
+        ctx->h_len[s] += 1;
+        ctx->h_pend[s] = (depth == L) ? 0 : ctx->h_pend[s] + 1;
+    }
+    return SPARSK_OK;
+}
+
+extern "C" int sparsk_decode_step_host(sparsk_ctx *ctx, int32_t n, const int32_t *slots, const int32_t *token_ids,
+                                       const uint8_t *modality, const int32_t *counters, int32_t *next_tokens,
+                                       int32_t *exit_depths)
+{
+    if (!good(ctx)) return SPARSK_ESTATE;
+    if (n < 1 || n > ctx->dm.max_seqs || !token_ids || !next_tokens || !exit_depths)
+        return fail(ctx, SPARSK_EINVAL, "decode_step_host: bad arguments (n=%d)", n);
+    CU(cudaMemcpyAsync(ctx->tok_dev, token_ids, sizeof(int) * n, cudaMemcpyHostToDevice, ctx->stream));
+    const int rc = sparsk_decode_step(ctx, n, slots, ctx->tok_dev, modality, counters, ctx->out_tok_dev, ctx->out_depth_dev);
+    if (rc != SPARSK_OK) return rc;
+    CU(cudaMemcpyAsync(next_tokens, ctx->out_tok_dev, sizeof(int) * n, cudaMemcpyDeviceToHost, ctx->stream));
+    CU(cudaMemcpyAsync(exit_depths, ctx->out_depth_dev, sizeof(int) * n, cudaMemcpyDeviceToHost, ctx->stream));
+    int status = 0;
+    CU(cudaMemcpyAsync(&status, ctx->sd.counts + CNT_STATUS, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+    CU(cudaStreamSynchronize(ctx->stream));
+    if (status) CU(cudaMemsetAsync(ctx->sd.counts + CNT_STATUS, 0, sizeof(int), ctx->stream));
+    if (status & ST_TIMEOUT) return fail(ctx, SPARSK_ETIMEOUT, "a bounded in-kernel wait ran out");
+    if (status & ST_BAD_TOKEN) return fail(ctx, SPARSK_EINVAL, "a token id was outside the vocabulary (clamped)");
+    return SPARSK_OK;
+}

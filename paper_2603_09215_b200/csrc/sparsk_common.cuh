@@ -1,0 +1,86 @@
+// Shared device helpers of the SPAR-K decode kernels (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace sparsk {
+
+typedef __nv_bfloat16 bf16;
+
+// Row bookkeeping of one decode step, all device arrays inside the workspace.
+// "Lower" rows are the step's sequences themselves (one row each, layers 1..e);
+// "upper" rows are, for every sequence that runs full depth, its pending positions
+// followed by its current position (layers e+1..L; Algorithm 1, full-depth branch).
+struct StepDesc {
+    int *slot, *modality, *counter, *token, *depth;  // [B]
+    int *lo_pos;                                     // [B] position of the row = slot length
+    int *lo_grp_row0, *lo_grp_nrows;                 // [B] identity groups (1 row each)
+    int *up_slot, *up_pos, *up_src;                  // [R] src >= 0: pending index; < 0: lower row -1-src
+    int *up_grp_row0, *up_grp_nrows;                 // [B] one group per full-depth sequence
+    int *cur_row;                                    // [B] upper row of the current position, or -1
+    int *list_seq, *list_row;                        // [4][B]: ee/text, ee/speech, full/text, full/speech
+    int *counts;                                     // [8]: see CNT_* below
+    unsigned long long *argmax;                      // [B] packed (logit, ~id)
+};
+enum { CNT_NSEQ = 0, CNT_MUP = 1, CNT_NGRP = 2, CNT_LIST0 = 3 /* ..6 */, CNT_STATUS = 7 };
+enum { ST_BAD_TOKEN = 1, ST_TIMEOUT = 2 };
+
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;"); }
+
+// 16-byte streaming load that does not allocate in L1 (weights and cache lines are read once).
+__device__ __forceinline__ uint4 ld_stream16(const void *p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void prefetch_l2(const void *p)
+{
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+}
+
+// bf16 pair packed in 32 bits -> two floats (element at the lower address first).
+__device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+__device__ __forceinline__ void unpack8(const uint4 &v, float (&f)[8])
+{
+    f[0] = bf_lo(v.x); f[1] = bf_hi(v.x); f[2] = bf_lo(v.y); f[3] = bf_hi(v.y);
+    f[4] = bf_lo(v.z); f[5] = bf_hi(v.z); f[6] = bf_lo(v.w); f[7] = bf_hi(v.w);
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float a, float b)
+{
+    __nv_bfloat162 t = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t *>(&t);
+}
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// Order-preserving map float -> uint32, and the 64-bit key whose maximum is the largest logit
+// with the lowest id among equals.
+__device__ __forceinline__ uint32_t float_key(float f)
+{
+    uint32_t u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ unsigned long long argmax_key(float logit, int id)
+{
+    return ((unsigned long long)float_key(logit) << 32) | (unsigned long long)(0xffffffffu - (uint32_t)id);
+}
+
+}  // namespace sparsk
