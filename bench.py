@@ -1,0 +1,431 @@
+#!/usr/bin/env python
+"""Benchmark of the SPAR-K decode hot path on B200.
+
+A "step" is one interleave cycle (N_text + N_speech decode steps) of the workload for all of its
+sequences: it contains text steps, early-exit speech steps and full-depth refresh steps that
+flush pending positions, i.e. every stage of the path.  `value` is decode tokens per second with
+tokens resident on the device; `e2e` is the same loop through sparsk_decode_step_host with host
+token buffers and a device->host read of every result.  Prints ONE JSON line on rank 0.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2_step_b1]
+  python bench.py --impl reference ...     # times the CPU oracle on a bounded sample
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2603_09215_b200 import synth  # noqa: E402
+
+KC = {"qkv": 1, "attn": 2, "oproj": 3, "gateup": 4, "down": 5, "head": 6}
+
+
+# --------------------------------------------------------------------------- byte model
+def layer_weight_bytes(d):
+    qd, kd = d["n_q_heads"] * d["head_dim"], d["n_kv_heads"] * d["head_dim"]
+    return 2 * (qd * d["d_model"] + 2 * kd * d["d_model"] + d["d_model"] * qd + 3 * d["d_ffn"] * d["d_model"]
+                + 2 * d["d_model"])
+
+
+def step_bytes(d, depths, mods, lens, pend):
+    """Algorithmic HBM bytes of one decode step: each active layer's weights once, each active
+    (sequence, layer) pair's KV prefix once plus the rows it appends, each (head, modality)
+    slice used once, the embedding rows."""
+    L, e = d["n_layers"], d["exit_layer"]
+    kvb = 2 * d["n_kv_heads"] * d["head_dim"] * 2
+    wl = layer_weight_bytes(d)
+    any_full = any(x == L for x in depths) and e < L
+    total = wl * e + (wl * (L - e) if any_full else 0)
+    for dep, ln, pn in zip(depths, lens, pend):
+        total += e * ((ln + 1) * kvb + kvb)
+        if dep == L and e < L:
+            total += (L - e) * ((ln + 1) * kvb + (pn + 1) * kvb)
+    for head, mod in {(dep, m) for dep, m in zip(depths, mods)}:
+        rows = d["vocab_speech"] if mod else d["vocab_text"]
+        total += rows * d["d_model"] * 2 + d["d_model"] * 2
+    total += len(depths) * d["d_model"] * 2
+    return total
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid):
+        self.uuid, self.lines, self.proc = uuid, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", self.uuid, f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for ln in self.proc.stdout:
+            self.lines.append(ln.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); pw.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------- workload
+def workload_setup(name, rank):
+    wl = dict(synth.WORKLOADS[name])
+    dims = synth.model_dims(wl["shape"], wl["exit_layer"], wl["refresh_period"], wl["refresh_phase"])
+    B = wl["batch"]
+    prompts = synth.make_prompts(dims, B, wl["prompt"][0], wl["prompt"][1], seed=1 + 1000 * rank,
+                                 len_seed=2 + 1000 * rank)
+    phi, off = synth.make_phases(B, wl["n_text"], wl["n_speech"], wl["refresh_period"], wl["random_phase"],
+                                 seed=3 + 1000 * rank)
+    return wl, dims, prompts, phi, off
+
+
+def cycle_schedule(wl, phi, off, g0, n):
+    out = []
+    for g in range(g0, g0 + n):
+        mc = [synth.interleave(g, wl["n_text"], wl["n_speech"], int(p), int(o)) for p, o in zip(phi, off)]
+        out.append((np.array([m for m, _ in mc], np.uint8), np.array([c for _, c in mc], np.int32)))
+    return out
+
+
+class Runner:
+    """Drives one library context through decode steps with tokens kept on the device."""
+
+    def __init__(self, dims, gw, wl, prompts, phi, off, total_steps, options=None, synthetic_kv=False):
+        import torch
+        from paper_2603_09215_b200 import binding
+        self.torch = torch
+        self.wl, self.dims, self.phi, self.off = wl, dims, phi, off
+        B = wl["batch"]
+        self.B = B
+        K = dims["refresh_period"]
+        max_len = max(len(p) for p in prompts) + total_steps + 8
+        self.ctx = binding.Sparsk(dims, gw, B, max_len, max(K - 1, 1) if dims["exit_layer"] < dims["n_layers"] else 1,
+                                  prefill_rows=64)
+        for k, v in (options or {}).items():
+            self.ctx.set_option(k, v)
+        self.slots = list(range(B))
+        if synthetic_kv:
+            self._fill_synthetic(prompts)
+        else:
+            self.ctx.prefill(self.slots, [p[:-1] for p in prompts])
+        self.tok = [torch.tensor([int(p[-1]) for p in prompts], dtype=torch.int32, device="cuda"),
+                    torch.zeros(B, dtype=torch.int32, device="cuda")]
+        self.dep = torch.zeros(B, dtype=torch.int32, device="cuda")
+        self.host_tok = np.array([int(p[-1]) for p in prompts], np.int32)
+        self.g = 0
+        self.lens = [len(p) - 1 for p in prompts]
+        self.pend = [0] * B
+        self.depth_log = []     # (modality, depth) per emitted token
+        self.bytes = 0
+
+    def _fill_synthetic(self, prompts):
+        torch = self.torch
+        for s, p in enumerate(prompts):
+            n = len(p) - 1
+            k, v = synth.synth_kv(self.dims, n, seed=100 + s)
+            for layer in range(1, self.dims["n_layers"] + 1):
+                kt = torch.from_numpy(k[layer - 1].view(np.int16)).cuda().view(torch.bfloat16)
+                vt = torch.from_numpy(v[layer - 1].view(np.int16)).cuda().view(torch.bfloat16)
+                self.ctx.import_kv(s, layer, 0, kt, vt)
+            self.ctx.set_len(s, n)
+        torch.cuda.synchronize()
+
+    def _account(self, mods, ctrs):
+        d = self.dims
+        L, e, K, r = d["n_layers"], d["exit_layer"], d["refresh_period"], d["refresh_phase"]
+        depths = [L if m == 0 else (L if c % K == r else e) for m, c in zip(mods, ctrs)]
+        self.bytes += step_bytes(d, depths, mods, self.lens, self.pend)
+        for i, dep in enumerate(depths):
+            self.lens[i] += 1
+            self.pend[i] = 0 if dep == L else self.pend[i] + 1
+            self.depth_log.append((int(mods[i]), dep))
+
+    def run_cycles(self, n_cycles, host=False):
+        cyc = self.wl["n_text"] + self.wl["n_speech"]
+        sched = cycle_schedule(self.wl, self.phi, self.off, self.g, n_cycles * cyc)
+        if host:
+            nt, dp = np.zeros(self.B, np.int32), np.zeros(self.B, np.int32)
+            for mods, ctrs in sched:
+                self.ctx.decode_step_host(self.slots, self.host_tok, mods, ctrs, nt, dp)
+                self.host_tok[:] = nt
+                self._account(mods, ctrs)
+        else:
+            for mods, ctrs in sched:
+                self.ctx.decode_step(self.slots, self.tok[0], mods, ctrs, self.tok[1], self.dep)
+                self.tok.reverse()
+                self._account(mods, ctrs)
+        self.g += n_cycles * cyc
+        return n_cycles * cyc * self.B
+
+    def sync_host_tokens(self):
+        self.host_tok[:] = self.tok[0].cpu().numpy()
+
+    def push_host_tokens(self):
+        self.tok[0].copy_(self.torch.from_numpy(self.host_tok))
+
+
+def layer_saving(log, L):
+    sp = [dep for m, dep in log if m == 1]
+    al = [dep for _, dep in log]
+    f = lambda xs: (1 - (sum(xs) / len(xs)) / L) * 100 if xs else 0.0
+    return {"speech_mean_depth": sum(sp) / max(1, len(sp)), "speech_saving_pct": f(sp), "all_saving_pct": f(al)}
+
+
+# --------------------------------------------------------------------------- CPU oracle timing
+def oracle_sample(wl, dims, w, prompts, phi, off, n_steps, start_g=0, seqs=1):
+    """Times the C oracle, as it stands, for `n_steps` consecutive decode steps of the first
+    `seqs` sequences, starting from a cache of the workload's prompt length filled with stand-in
+    values (the oracle's cost does not depend on the cache contents)."""
+    from oracle import oracle as ora
+    from oracle.bruteforce import bf16_to_f64
+    n = max(len(p) for p in prompts[:seqs]) - 1
+    om = ora.OracleModel(dims, w, max_len=n + n_steps + 2)
+    seq = []
+    for s in range(seqs):
+        sq = om.new_seq(max(1, dims["refresh_period"]))
+        k, v = synth.synth_kv(dims, len(prompts[s]) - 1, seed=100 + s)
+        for layer in range(1, dims["n_layers"] + 1):
+            kf, vf = bf16_to_f64(k[layer - 1]), bf16_to_f64(v[layer - 1])
+            for p in range(kf.shape[0]):
+                sq.set_kv(layer, p, kf[p], vf[p])
+        sq.set_len(len(prompts[s]) - 1)
+        seq.append(sq)
+    toks = [int(prompts[s][-1]) for s in range(seqs)]
+    t0 = time.perf_counter()
+    for g in range(start_g, start_g + n_steps):
+        for s in range(seqs):
+            m, c = synth.interleave(g, wl["n_text"], wl["n_speech"], int(phi[s]), int(off[s]))
+            r = seq[s].decode_step(toks[s], m, c, want_logits=False)
+            toks[s] = r["token"]
+    dt = time.perf_counter() - t0
+    return dt, n_steps * seqs
+
+
+def omp_threads():
+    return int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
+
+
+# --------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=4)
+    ap.add_argument("--impl", default="sparsk", choices=["sparsk", "reference"])
+    ap.add_argument("--workload", default="cfg2_step_b1", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-full-depth", action="store_true")
+    ap.add_argument("--option", action="append", default=[], help="library option name=value")
+    ap.add_argument("--time-kernel", default="gateup", choices=sorted(KC))
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    W = max(args.warmup, 3)
+    wl, dims, prompts, phi, off = workload_setup(args.workload, rank)
+    cyc = wl["n_text"] + wl["n_speech"]
+    L = dims["n_layers"]
+    cfg = {"workload": args.workload, "shape": wl["shape"], "batch_per_gpu": wl["batch"],
+           "prompt_len": list(wl["prompt"]), "interleave": f'{wl["n_text"]}:{wl["n_speech"]}',
+           "exit_layer": wl["exit_layer"], "refresh_period": wl["refresh_period"],
+           "refresh_phase": wl["refresh_phase"], "decode_steps_per_step": cyc,
+           "l2": "inputs larger than L2 (all active layers' weights are streamed every decode step)",
+           "parallelism": f"replicas x{world}" if world > 1 else "single GPU"}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        w = synth.make_weights(dims, seed=0, head_layers=[wl["exit_layer"], L])
+        seqs = min(wl["batch"], 1)
+        times, toks = [], 0
+        for i in range(W + args.steps):
+            dt, n = oracle_sample(wl, dims, w, prompts, phi, off, 1, start_g=i, seqs=seqs)
+            if i >= W:
+                times.append(dt)
+                toks += n
+        tot = sum(times)
+        val = toks / tot
+        base = {"value": val, "unit": "tokens/s", "cores": omp_threads(), "kind": "oracle",
+                "sample": f"each step = 1 decode step of 1 sequence at cache length {len(prompts[0]) - 1} "
+                          f"(stand-in cache values), walking the interleave cycle"}
+        print(json.dumps({"impl": "reference", "metric": "decode_tokens_per_s", "value": val, "unit": "tokens/s",
+                          "n_gpus": args.gpus, "steps": args.steps, "warmup": W,
+                          "ms_per_step": 1e3 * tot / args.steps, "higher_is_better": True, "scaling": "weak",
+                          "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": cfg,
+                          "cpu_baseline": base,
+                          "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0,
+                                  "d2h_bytes_per_step": 0}}))
+        return
+
+    import torch
+    from paper_2603_09215_b200 import binding
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    t_setup = time.time()
+    w = synth.make_weights(dims, seed=0, head_layers=[wl["exit_layer"], L])
+    gw = binding.upload_weights(w)
+    opts = {}
+    for o in args.option:
+        k, v = o.split("=")
+        opts[k] = int(v)
+    synthetic_kv = max(wl["prompt"]) > 4096      # long prompts: cache contents are stand-ins
+    extra = (W + args.steps) * 2 + 8
+    total_steps = extra * cyc
+    run = Runner(dims, gw, wl, prompts, phi, off, total_steps, opts, synthetic_kv)
+    cfg["cache_fill"] = "stand-in values (imported)" if synthetic_kv else "real prefill of random prompts"
+    setup_s = time.time() - t_setup
+
+    def timed(runner, cycles, host=False):
+        barrier()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0 = runner.ctx.launch_count()
+        ev0.record()
+        n = runner.run_cycles(cycles, host=host)
+        ev1.record()
+        barrier()
+        ms = ev0.elapsed_time(ev1)
+        if world > 1:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, n, runner.ctx.launch_count() - l0
+
+    # ---- SPAR-K schedule, tokens on the device
+    run.run_cycles(W)
+    torch.cuda.synchronize()
+    uuid = str(torch.cuda.get_device_properties(local).uuid)
+    uuid = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+    sampler = ClockSampler(uuid)
+    sampler.start()
+    b0 = run.bytes
+    ms, ntok, launches = timed(run, args.steps)
+    clocks = sampler.stop()
+    step_b = (run.bytes - b0)
+    value = world * ntok / (ms / 1e3)
+    peaks = {}
+    pk_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(pk_path):
+        peaks = json.load(open(pk_path))
+    hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
+    peak_kind = "measured" if "hbm_gbs" in peaks else "fallback"
+
+    # ---- the same loop through the host-buffer entry point
+    run.sync_host_tokens()
+    run.run_cycles(1, host=True)
+    ms_e2e, ntok_e2e, _ = timed(run, args.steps, host=True)
+    run.push_host_tokens()
+    B = wl["batch"]
+    e2e = {"value": world * ntok_e2e / (ms_e2e / 1e3), "unit": "tokens/s",
+           "h2d_bytes_per_step": cyc * (4 * B + 12 * B), "d2h_bytes_per_step": cyc * (8 * B + 4)}
+
+    # ---- dominant kernel, timed live with events around each of its launches
+    kname = args.time_kernel
+    run.ctx.set_option("time_kernel", KC[kname])
+    run.run_cycles(min(args.steps, 8))
+    kms, kn = run.ctx.kernel_time()
+    run.ctx.set_option("time_kernel", 0)
+    d = dims
+    kbytes = {"gateup": 2 * d["d_ffn"] * d["d_model"] * 2, "down": d["d_ffn"] * d["d_model"] * 2,
+              "qkv": (d["n_q_heads"] + 2 * d["n_kv_heads"]) * d["head_dim"] * d["d_model"] * 2,
+              "oproj": d["n_q_heads"] * d["head_dim"] * d["d_model"] * 2}.get(kname)
+    roof = {"bound": "hbm", "kernel": kname, "unit": "GB/s", "peak": hbm_peak, "peak_kind": peak_kind,
+            "traffic": None}
+    if kbytes and kn:
+        ach = kbytes / (kms / kn * 1e-3) / 1e9
+        roof.update(achieved=ach, frac=ach / hbm_peak, launches_timed=kn, avg_launch_us=1e3 * kms / kn,
+                    bytes_per_launch=kbytes)
+    else:
+        roof.update(achieved=None, frac=None)
+
+    # ---- full depth (K = 1) on the same weights
+    full = None
+    if not args.no_full_depth:
+        wl_f = dict(wl, refresh_period=1, refresh_phase=0)
+        dims_f = synth.model_dims(wl["shape"], wl["exit_layer"], 1, 0)
+        rf = Runner(dims_f, gw, wl_f, prompts, phi, off, total_steps, opts, synthetic_kv)
+        rf.run_cycles(W)
+        fb0 = rf.bytes
+        ms_f, ntok_f, _ = timed(rf, args.steps)
+        full = {"value": world * ntok_f / (ms_f / 1e3), "unit": "tokens/s", "ms_per_step": ms_f / args.steps,
+                "bytes_per_step": (rf.bytes - fb0) / args.steps,
+                "hbm_frac": ((rf.bytes - fb0) / (ms_f * 1e-3) / 1e9) / hbm_peak}
+        rf.ctx.close()
+
+    sav = layer_saving(run.depth_log, L)
+    n_text = sum(1 for m, _ in run.depth_log[-ntok:] if m == 0)
+    out = {"metric": "decode_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world,
+           "steps": args.steps, "warmup": W, "ms_per_step": ms / args.steps, "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": cfg,
+           "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roof,
+           "step_hbm": {"bytes_per_step": step_b / args.steps, "achieved_gbs": step_b / (ms * 1e-3) / 1e9,
+                        "frac_of_measured_copy": step_b / (ms * 1e-3) / 1e9 / hbm_peak,
+                        "frac_of_nominal_8tbs": step_b / (ms * 1e-3) / 1e9 / 8000.0},
+           "layer_saving": sav, "setup_s": setup_s}
+    if full:
+        out["full_depth"] = full
+        out["reduction"] = {"wall_time_pct": (1 - (ms / args.steps) / full["ms_per_step"]) * 100,
+                            "byte_model_pct": (1 - (step_b / args.steps) / full["bytes_per_step"]) * 100,
+                            "layer_saving_all_tokens_pct": sav["all_saving_pct"]}
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        seqs = 1
+        dt, n = oracle_sample(wl, dims, w, prompts, phi, off, cyc, start_g=0, seqs=seqs)
+        out["cpu_baseline"] = {"value": n / dt, "unit": "tokens/s", "cores": omp_threads(), "kind": "oracle",
+                               "sample": f"one interleave cycle ({cyc} decode steps) of 1 sequence at cache "
+                                         f"length {len(prompts[0]) - 1} (stand-in cache values), {dt:.1f} s"}
+    run.ctx.close()
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
