@@ -159,6 +159,30 @@ int sparsk_set_debug(sparsk_ctx *ctx, float *exit_hidden /*device or NULL*/,
  * "time_kernel" (see sparsk_kernel_time).  Returns SPARSK_EINVAL for an unknown name or value. */
 int sparsk_set_option(sparsk_ctx *ctx, const char *name /*host*/, int64_t value);
 
+/* Stand-alone split-KV grouped-query attention: the two kernels a decode step runs per layer
+ * (partials per KV split, then the merge), on caller-described rows.  Rows are grouped: group g
+ * is rows [grp_row0[g], grp_row0[g] + grp_nrows[g]) of ONE sequence at consecutive positions;
+ * row i of a group attends to cache positions 0..row_pos[i] of slot row_slot[i] (the causal
+ * block of Algorithm 1's full-depth branch on top of the earlier cache; a lower-pass row is a
+ * group of one).  All array pointers are DEVICE pointers.  Rows whose slot is outside
+ * [0, n_slots) or whose position is outside the cache read nothing and produce zeros.
+ * `scratch` (device, 256-byte aligned, >= sparsk_attention_scratch_bytes) is overwritten. */
+typedef struct {
+    const void *q;               /* bf16 [n_rows][n_q_heads*head_dim], rotated queries             */
+    const void *k_cache;         /* bf16 [n_slots][n_kv_heads][cache_len][head_dim], rotated keys  */
+    const void *v_cache;         /* bf16, same layout                                              */
+    void *out;                   /* bf16 [n_rows][n_q_heads*head_dim]                              */
+    const int32_t *row_slot, *row_pos;     /* [n_rows]                                             */
+    const int32_t *grp_row0, *grp_nrows;   /* [n_groups]                                           */
+    int32_t n_rows, n_groups;
+    int32_t max_grp_rows;        /* host-known bound on grp_nrows                                  */
+    int32_t max_len;             /* host-known bound on row_pos + 1                                */
+    int32_t n_q_heads, n_kv_heads, head_dim /* 64 or 128 */, cache_len, n_slots;
+} sparsk_attn_args;
+size_t sparsk_attention_scratch_bytes(int32_t n_rows, int32_t n_q_heads, int32_t head_dim);
+int sparsk_attention(const sparsk_attn_args *args /*host*/, void *scratch /*device*/, size_t scratch_bytes,
+                     void *cuda_stream);
+
 /* Per-kernel timing for roofline reports.  sparsk_set_option(ctx, "time_kernel", c) with c =
  * 1 QKV, 2 attention, 3 O-projection, 4 gate/up, 5 down-projection, 6 exit head brackets every
  * later launch of that class with CUDA events on the context's stream (up to 8192 launches; 0

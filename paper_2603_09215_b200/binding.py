@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libsparsk.so")
 EXPORTS = ("sparsk_workspace_bytes", "sparsk_create", "sparsk_prefill", "sparsk_decode_step",
            "sparsk_decode_step_host", "sparsk_reset_slot", "sparsk_import_kv", "sparsk_export_kv",
            "sparsk_set_len", "sparsk_slot_state", "sparsk_set_debug", "sparsk_set_option",
-           "sparsk_kernel_time", "sparsk_launch_count", "sparsk_last_error", "sparsk_destroy")
+           "sparsk_kernel_time", "sparsk_attention", "sparsk_attention_scratch_bytes", "sparsk_launch_count", "sparsk_last_error", "sparsk_destroy")
 
 OK, EINVAL, ECAPACITY, ENOHEAD, ECUDA, ESTATE, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
 
@@ -40,6 +40,13 @@ class Dims(C.Structure):
 _PP = C.POINTER(C.c_void_p)
 PER_LAYER = ("attn_norm", "wq", "wk", "wv", "wo", "mlp_norm", "w_gate", "w_up", "w_down",
              "head_norm", "head_proj")
+
+
+class AttnArgs(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("q", "k_cache", "v_cache", "out", "row_slot", "row_pos",
+                                          "grp_row0", "grp_nrows")] + [
+        (n, C.c_int32) for n in ("n_rows", "n_groups", "max_grp_rows", "max_len", "n_q_heads",
+                                 "n_kv_heads", "head_dim", "cache_len", "n_slots")]
 
 
 class Weights(C.Structure):
@@ -85,6 +92,10 @@ def load():
     L.sparsk_set_option.argtypes = [vp, C.c_char_p, C.c_int64]
     L.sparsk_kernel_time.restype = C.c_int
     L.sparsk_kernel_time.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+    L.sparsk_attention_scratch_bytes.restype = C.c_size_t
+    L.sparsk_attention_scratch_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32]
+    L.sparsk_attention.restype = C.c_int
+    L.sparsk_attention.argtypes = [C.POINTER(AttnArgs), vp, C.c_size_t, vp]
     L.sparsk_launch_count.restype = C.c_int64
     L.sparsk_launch_count.argtypes = [vp]
     L.sparsk_last_error.restype = C.c_char_p
@@ -121,6 +132,31 @@ def upload_weights(w: dict, device="cuda") -> dict:
 
 def _i32(a):
     return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def attn_args(q, k_cache, v_cache, out, row_slot, row_pos, grp_row0, grp_nrows, max_grp_rows, max_len,
+              n_q_heads) -> AttnArgs:
+    """Marshal torch CUDA tensors into the argument block of sparsk_attention.
+    k_cache / v_cache: [n_slots, n_kv_heads, cache_len, head_dim] bf16."""
+    a = AttnArgs()
+    a.q, a.k_cache, a.v_cache, a.out = q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), out.data_ptr()
+    a.row_slot, a.row_pos = row_slot.data_ptr(), row_pos.data_ptr()
+    a.grp_row0, a.grp_nrows = grp_row0.data_ptr(), grp_nrows.data_ptr()
+    a.n_rows, a.n_groups = q.shape[0], grp_row0.shape[0]
+    a.max_grp_rows, a.max_len = int(max_grp_rows), int(max_len)
+    a.n_slots, a.n_kv_heads, a.cache_len, a.head_dim = k_cache.shape
+    a.n_q_heads = n_q_heads
+    return a
+
+
+def attention(args: AttnArgs, scratch: torch.Tensor, stream=None) -> int:
+    """sparsk_attention on the current (or given) stream; returns the status code."""
+    st = (stream or torch.cuda.current_stream()).cuda_stream
+    return load().sparsk_attention(C.byref(args), scratch.data_ptr(), scratch.numel(), st)
+
+
+def attention_scratch_bytes(n_rows: int, n_q_heads: int, head_dim: int) -> int:
+    return load().sparsk_attention_scratch_bytes(n_rows, n_q_heads, head_dim)
 
 
 class Sparsk:

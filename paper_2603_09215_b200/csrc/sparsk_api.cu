@@ -18,8 +18,7 @@ using namespace sparsk;
 
 namespace {
 
-constexpr int MAX_SPLITS = 32;
-constexpr int MIN_SPLIT_LEN = 64;
+constexpr int MAX_SPLITS = AT_MAX_SPLITS;
 constexpr int STAGE_RING = 16;
 constexpr uint32_t CTX_MAGIC = 0x5350524bu;  // "SPRK"
 constexpr size_t TIME_POOL = 8192;           // event pairs available to the kernel timer
@@ -355,25 +354,13 @@ cudaError_t run_attn(sparsk_ctx *c, int layer, const RowSet &rs)
     a.n_groups = rs.n_groups;
     a.part_o = c->part_o; a.part_ml = c->part_ml; a.out = c->attn_o;
     a.Hq = d.n_q_heads; a.Hkv = d.n_kv_heads; a.S = d.max_seq_len;
-    a.n_qblk = (rs.max_grp_rows * G + AT_QB - 1) / AT_QB;
-    // enough splits to fill the machine, none shorter than MIN_SPLIT_LEN
-    int split = c->attn_split;
-    if (split <= 0) {
-        const long base = (long)rs.n_groups_h * a.n_qblk * d.n_kv_heads;
-        long want = std::max<long>(1, (2L * c->n_sm + base - 1) / base);
-        want = std::min<long>(want, MAX_SPLITS);
-        split = (int)((rs.max_len + want - 1) / want);
-        split = std::max(split, MIN_SPLIT_LEN);
-    }
-    split = (split + AT_TILE - 1) / AT_TILE * AT_TILE;
-    int n_splits = (rs.max_len + split - 1) / split;
-    if (n_splits > MAX_SPLITS) {
-        n_splits = MAX_SPLITS;
-        split = ((rs.max_len + n_splits - 1) / n_splits + AT_TILE - 1) / AT_TILE * AT_TILE;
-        n_splits = (rs.max_len + split - 1) / split;
-    }
-    a.split_len = split;
-    a.n_splits = n_splits;
+    const AttnPlan pl = attn_plan(c->n_sm, rs.n_groups_h, rs.max_grp_rows, G, d.n_kv_heads, rs.max_len, c->attn_split);
+    a.n_qblk = pl.n_qblk;
+    a.split_len = pl.split_len;
+    a.n_splits = pl.n_splits;
+    a.n_slots = d.max_seqs;
+    a.n_rows = rs.n_rows;
+    const int n_splits = pl.n_splits;
     dim3 grid(rs.n_groups_h * a.n_qblk, d.n_kv_heads, n_splits);
     cudaError_t e;
     if (d.head_dim == 128) {

@@ -18,6 +18,38 @@ namespace sparsk {
 constexpr int AT_THREADS = 128;
 constexpr int AT_QB = 32;    // query vectors per CTA
 constexpr int AT_TILE = 32;  // KV positions per tile
+constexpr int AT_MAX_SPLITS = 32;
+constexpr int AT_MIN_SPLIT = 64;
+
+// How a launch cuts the KV range: enough splits to fill the machine, none shorter than
+// AT_MIN_SPLIT positions (unless forced), at most AT_MAX_SPLITS.
+struct AttnPlan {
+    int n_qblk, split_len, n_splits;
+};
+inline AttnPlan attn_plan(int n_sm, int n_groups, int max_grp_rows, int G, int Hkv, int max_len, int forced_split)
+{
+    AttnPlan p;
+    p.n_qblk = (max_grp_rows * G + AT_QB - 1) / AT_QB;
+    int split = forced_split;
+    if (split <= 0) {
+        const long base = (long)n_groups * p.n_qblk * Hkv;
+        long want = (2L * n_sm + base - 1) / base;
+        want = want < 1 ? 1 : (want > AT_MAX_SPLITS ? AT_MAX_SPLITS : want);
+        split = (int)((max_len + want - 1) / want);
+        if (split < AT_MIN_SPLIT) split = AT_MIN_SPLIT;
+    }
+    split = (split + AT_TILE - 1) / AT_TILE * AT_TILE;
+    int n_splits = (max_len + split - 1) / split;
+    if (n_splits > AT_MAX_SPLITS) {
+        n_splits = AT_MAX_SPLITS;
+        split = ((max_len + n_splits - 1) / n_splits + AT_TILE - 1) / AT_TILE * AT_TILE;
+        n_splits = (max_len + split - 1) / split;
+    }
+    if (n_splits < 1) n_splits = 1;
+    p.split_len = split;
+    p.n_splits = n_splits;
+    return p;
+}
 
 struct AttnArgs {
     const bf16 *q;            // [rows][Hq*hd], already rotated
@@ -28,6 +60,8 @@ struct AttnArgs {
     float2 *part_ml;          // [rows*Hq][n_splits]  (max, sum)
     bf16 *out;                // [rows][Hq*hd]
     int Hq, Hkv, S, n_qblk, n_splits, split_len;
+    int n_slots;              // slots in the cache; rows naming another slot are skipped
+    int n_rows;               // rows in q/out; groups reaching beyond them are skipped
 };
 
 template <int HD>
@@ -46,6 +80,7 @@ __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(AttnArgs a)
     const int hk = blockIdx.y, sp = blockIdx.z;
     const int G = a.Hq / a.Hkv;
     const int row0 = a.grp_row0[g], nrows = a.grp_nrows[g];
+    if (row0 < 0 || nrows < 1 || row0 + nrows > a.n_rows) return;
     const int nq = nrows * G;
     const int q0 = qb * AT_QB;
     if (q0 >= nq) return;
@@ -54,8 +89,10 @@ __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(AttnArgs a)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     // positions this CTA may look at: its split, cut at the last query row's own position
+    // (and at the cache itself: a descriptor that points outside it reads nothing)
     const int last_row = (q0 + nq_here - 1) / G;
-    const int kv_end_all = pos0 + last_row + 1;
+    const bool sane = slot >= 0 && slot < a.n_slots && pos0 >= 0;
+    const int kv_end_all = sane ? min(pos0 + last_row + 1, a.S) : 0;
     const int s_beg = sp * a.split_len;
     const int s_end = min(s_beg + a.split_len, kv_end_all);
 
@@ -185,7 +222,7 @@ __global__ void __launch_bounds__(HD) attn_merge_kernel(AttnArgs a, const int *_
         den += ml.y * w;
         num += a.part_o[(cell0 + s) * HD + threadIdx.x] * w;
     }
-    a.out[(size_t)row * a.Hq * HD + head * HD + threadIdx.x] = __float2bfloat16(num / den);
+    a.out[(size_t)row * a.Hq * HD + head * HD + threadIdx.x] = __float2bfloat16(den > 0.f ? num / den : 0.f);
 }
 
 }  // namespace sparsk

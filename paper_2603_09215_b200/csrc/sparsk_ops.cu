@@ -1,0 +1,77 @@
+// Stand-alone entry points for single kernels of the decode path (C ABI in include/sparsk.h).
+// They run exactly the kernels a decode step runs, on caller-described inputs, so that one
+// stage can be driven, checked and profiled on its own.
+#include <cstdint>
+
+#include "../../include/sparsk.h"
+#include "sparsk_attn.cuh"
+#include "sparsk_step.cuh"
+
+using namespace sparsk;
+
+namespace {
+size_t up256(size_t v) { return (v + 255) / 256 * 256; }
+}  // namespace
+
+static bool attn_args_ok(const sparsk_attn_args *a)
+{
+    if (!a || !a->q || !a->k_cache || !a->v_cache || !a->out || !a->row_slot || !a->row_pos || !a->grp_row0 ||
+        !a->grp_nrows)
+        return false;
+    if (a->n_rows < 1 || a->n_groups < 1 || a->n_groups > a->n_rows || a->max_grp_rows < 1 ||
+        a->max_grp_rows > a->n_rows)
+        return false;
+    if (a->n_q_heads < 1 || a->n_kv_heads < 1 || a->n_q_heads % a->n_kv_heads) return false;
+    if (a->head_dim != 64 && a->head_dim != 128) return false;
+    if (a->cache_len < 1 || a->n_slots < 1 || a->max_len < 1 || a->max_len > a->cache_len) return false;
+    return true;
+}
+
+extern "C" size_t sparsk_attention_scratch_bytes(int32_t n_rows, int32_t n_q_heads, int32_t head_dim)
+{
+    if (n_rows < 1 || n_q_heads < 1 || (head_dim != 64 && head_dim != 128)) return 0;
+    const size_t cells = (size_t)n_rows * n_q_heads * AT_MAX_SPLITS;
+    return 256 + up256(cells * head_dim * sizeof(float)) + up256(cells * sizeof(float2));
+}
+
+// Shared by the entry points of this library that run the two attention kernels outside a
+// context: `scratch` holds two counters, then the split partials.
+int sparsk_attention_launch(const sparsk_attn_args *p, char *scratch, cudaStream_t st)
+{
+    int dev = 0, n_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return SPARSK_ECUDA;
+    const size_t cells = (size_t)p->n_rows * p->n_q_heads * AT_MAX_SPLITS;
+    int *counts = reinterpret_cast<int *>(scratch);
+    AttnArgs a{};
+    a.q = (const bf16 *)p->q; a.kc = (const bf16 *)p->k_cache; a.vc = (const bf16 *)p->v_cache;
+    a.grp_row0 = p->grp_row0; a.grp_nrows = p->grp_nrows; a.row_slot = p->row_slot; a.row_pos = p->row_pos;
+    a.n_groups = counts;
+    a.part_o = reinterpret_cast<float *>(scratch + 256);
+    a.part_ml = reinterpret_cast<float2 *>(scratch + 256 + up256(cells * p->head_dim * sizeof(float)));
+    a.out = (bf16 *)p->out;
+    a.Hq = p->n_q_heads; a.Hkv = p->n_kv_heads; a.S = p->cache_len; a.n_slots = p->n_slots; a.n_rows = p->n_rows;
+    const AttnPlan pl = attn_plan(n_sm, p->n_groups, p->max_grp_rows, p->n_q_heads / p->n_kv_heads,
+                                  p->n_kv_heads, p->max_len, 0);
+    a.n_qblk = pl.n_qblk; a.split_len = pl.split_len; a.n_splits = pl.n_splits;
+    set_int_kernel<<<1, 1, 0, st>>>(counts, p->n_groups);
+    set_int_kernel<<<1, 1, 0, st>>>(counts + 1, p->n_rows);
+    const dim3 grid(p->n_groups * pl.n_qblk, p->n_kv_heads, pl.n_splits);
+    if (p->head_dim == 128) {
+        attn_partial_kernel<128><<<grid, AT_THREADS, 0, st>>>(a);
+        attn_merge_kernel<128><<<dim3(p->n_rows, p->n_q_heads), 128, 0, st>>>(a, counts + 1);
+    } else {
+        attn_partial_kernel<64><<<grid, AT_THREADS, 0, st>>>(a);
+        attn_merge_kernel<64><<<dim3(p->n_rows, p->n_q_heads), 64, 0, st>>>(a, counts + 1);
+    }
+    return cudaGetLastError() == cudaSuccess ? SPARSK_OK : SPARSK_ECUDA;
+}
+
+extern "C" int sparsk_attention(const sparsk_attn_args *args, void *scratch, size_t scratch_bytes, void *cuda_stream)
+{
+    if (!attn_args_ok(args) || !scratch || ((uintptr_t)scratch % 256)) return SPARSK_EINVAL;
+    if (scratch_bytes < sparsk_attention_scratch_bytes(args->n_rows, args->n_q_heads, args->head_dim))
+        return SPARSK_EINVAL;
+    return sparsk_attention_launch(args, (char *)scratch, (cudaStream_t)cuda_stream);
+}

@@ -12,7 +12,7 @@ namespace sparsk {
 // input token (clamped into the vocabulary, with a status bit if it was outside) and clears
 // the sequence's argmax cell.
 // ---------------------------------------------------------------------------------------
-__global__ void schedule_kernel(StepDesc sd, int n, const int *__restrict__ staged /*[3][n]*/,
+static __global__ void schedule_kernel(StepDesc sd, int n, const int *__restrict__ staged /*[3][n]*/,
                                 const int *__restrict__ tokens_in, int vocab, int L, int e, int K,
                                 int r, int text_exit)
 {
@@ -71,7 +71,7 @@ __device__ __forceinline__ int block_exscan(int v, int *warp_tot /*[32] shared*/
 // "batch P u {t}").  Prefix sums give each sequence its offset in the upper row list; four
 // more give the per-(exit, modality) lists the head kernels read.  One block, n <= 1024.
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024) compact_kernel(StepDesc sd, int n, const int *__restrict__ kv_len,
+static __global__ void __launch_bounds__(1024) compact_kernel(StepDesc sd, int n, const int *__restrict__ kv_len,
                                                        const int *__restrict__ pend_cnt, int L, int e,
                                                        int list_stride)
 {
@@ -124,7 +124,7 @@ __global__ void __launch_bounds__(1024) compact_kernel(StepDesc sd, int n, const
 }
 
 // h^(0) = E[token]  (Sec. III), fp32 residual stream.
-__global__ void embed_kernel(const int *__restrict__ tokens, const bf16 *__restrict__ embed,
+static __global__ void embed_kernel(const int *__restrict__ tokens, const bf16 *__restrict__ embed,
                              float *__restrict__ h, int n, int d, int vocab, int *__restrict__ status)
 {
     griddep_wait();
@@ -146,7 +146,7 @@ __global__ void embed_kernel(const int *__restrict__ tokens, const bf16 *__restr
 }
 
 // Early-exit rows: store h^(e) in the pending store ("store h_t^(l_EE)", Algorithm 1).
-__global__ void stash_kernel(StepDesc sd, const float *__restrict__ h_lo, float *__restrict__ pend_h,
+static __global__ void stash_kernel(StepDesc sd, const float *__restrict__ h_lo, float *__restrict__ pend_h,
                              const int *__restrict__ pend_cnt, int n, int d, int L, int max_pending)
 {
     griddep_wait();
@@ -162,7 +162,7 @@ __global__ void stash_kernel(StepDesc sd, const float *__restrict__ h_lo, float 
 
 // Upper rows: h^(e) of pending positions comes from the pending store, of the current
 // position from the lower pass.
-__global__ void gather_upper_kernel(StepDesc sd, const float *__restrict__ h_lo,
+static __global__ void gather_upper_kernel(StepDesc sd, const float *__restrict__ h_lo,
                                     const float *__restrict__ pend_h, float *__restrict__ h_up, int d,
                                     int max_pending)
 {
@@ -178,7 +178,7 @@ __global__ void gather_upper_kernel(StepDesc sd, const float *__restrict__ h_lo,
 }
 
 // End of step: emit tokens and depths, advance lengths, grow or clear the pending sets.
-__global__ void finish_kernel(StepDesc sd, int n, int *__restrict__ kv_len, int *__restrict__ pend_cnt,
+static __global__ void finish_kernel(StepDesc sd, int n, int *__restrict__ kv_len, int *__restrict__ pend_cnt,
                               int *__restrict__ next_tokens, int *__restrict__ exit_depths, int L)
 {
     griddep_wait();
@@ -192,7 +192,7 @@ __global__ void finish_kernel(StepDesc sd, int n, int *__restrict__ kv_len, int 
 }
 
 // Parity hooks: copy the hidden state each head read; pre-fill the logits with -inf.
-__global__ void debug_hidden_kernel(StepDesc sd, const float *__restrict__ h_lo,
+static __global__ void debug_hidden_kernel(StepDesc sd, const float *__restrict__ h_lo,
                                     const float *__restrict__ h_up, float *__restrict__ out, int n, int d)
 {
     const int b = blockIdx.x;
@@ -201,14 +201,14 @@ __global__ void debug_hidden_kernel(StepDesc sd, const float *__restrict__ h_lo,
     const float *from = (cr >= 0) ? h_up + (size_t)cr * d : h_lo + (size_t)b * d;
     for (int i = threadIdx.x; i < d; i += blockDim.x) out[(size_t)b * d + i] = from[i];
 }
-__global__ void fill_kernel(float *__restrict__ p, size_t n, float v)
+static __global__ void fill_kernel(float *__restrict__ p, size_t n, float v)
 {
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
         p[i] = v;
 }
 
 // Prefill bookkeeping: rows of one chunk of one prompt.
-__global__ void prefill_rows_kernel(int *__restrict__ row_slot, int *__restrict__ row_pos,
+static __global__ void prefill_rows_kernel(int *__restrict__ row_slot, int *__restrict__ row_pos,
                                     int *__restrict__ grp_row0, int *__restrict__ grp_nrows, int slot,
                                     int pos0, int n)
 {
@@ -222,10 +222,10 @@ __global__ void prefill_rows_kernel(int *__restrict__ row_slot, int *__restrict_
         row_pos[i] = pos0 + i;
     }
 }
-__global__ void set_int_kernel(int *p, int v) { *p = v; }
+static __global__ void set_int_kernel(int *p, int v) { *p = v; }
 
 // Cache import/export: [n][Hkv*hd] <-> [Hkv][S][hd] of one (layer, slot).
-__global__ void kv_copy_kernel(bf16 *__restrict__ cache_k, bf16 *__restrict__ cache_v, bf16 *ext_k,
+static __global__ void kv_copy_kernel(bf16 *__restrict__ cache_k, bf16 *__restrict__ cache_v, bf16 *ext_k,
                                bf16 *ext_v, int first_pos, int n, int Hkv, int hd, int S, int to_cache)
 {
     const size_t total = (size_t)n * Hkv * hd;
