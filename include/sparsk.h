@@ -183,6 +183,26 @@ size_t sparsk_attention_scratch_bytes(int32_t n_rows, int32_t n_q_heads, int32_t
 int sparsk_attention(const sparsk_attn_args *args /*host*/, void *scratch /*device*/, size_t scratch_bytes,
                      void *cuda_stream);
 
+/* The same attention for callers that cannot allocate device memory (no counterpart in the
+ * paper: this exists for integration only).  Typical callers: a plug-in inside another engine
+ * whose memory plan leaves no allocator to call, code on a path where cudaMalloc is forbidden
+ * because it synchronises the device, a process whose device pool belongs to another runtime.
+ * The split partials go to a fixed area of SPARSK_STATIC_SCRATCH_BYTES that is part of the
+ * library image; every GPU that loads the library holds it until the process exits.  The call
+ * allocates nothing and frees nothing.
+ *   - A call whose partials do not fit (sparsk_attention_scratch_bytes(n_rows, n_q_heads,
+ *     head_dim) > SPARSK_STATIC_SCRATCH_BYTES) is refused with SPARSK_ECAPACITY before anything
+ *     is launched; `err` (host buffer, may be NULL) then says how much was needed.
+ *   - The first call on each device looks up the area's device address (with that device
+ *     current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one area, which keeps the previous call's contents;
+ *     nothing in it needs clearing between calls.  Two calls that overlap on the GPU (different
+ *     streams, no ordering between them) race on it: order them.
+ * Arguments, layouts and results are those of sparsk_attention. */
+#define SPARSK_STATIC_SCRATCH_BYTES (8u << 20)
+int sparsk_attention_static(const sparsk_attn_args *args /*host*/, void *cuda_stream, char *err /*host*/,
+                            size_t err_len);
+
 /* Per-kernel timing for roofline reports.  sparsk_set_option(ctx, "time_kernel", c) with c =
  * 1 QKV, 2 attention, 3 O-projection, 4 gate/up, 5 down-projection, 6 exit head brackets every
  * later launch of that class with CUDA events on the context's stream (up to 8192 launches; 0

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libsparsk.so")
 EXPORTS = ("sparsk_workspace_bytes", "sparsk_create", "sparsk_prefill", "sparsk_decode_step",
            "sparsk_decode_step_host", "sparsk_reset_slot", "sparsk_import_kv", "sparsk_export_kv",
            "sparsk_set_len", "sparsk_slot_state", "sparsk_set_debug", "sparsk_set_option",
-           "sparsk_kernel_time", "sparsk_attention", "sparsk_attention_scratch_bytes", "sparsk_launch_count", "sparsk_last_error", "sparsk_destroy")
+           "sparsk_kernel_time", "sparsk_attention", "sparsk_attention_scratch_bytes", "sparsk_attention_static", "sparsk_launch_count", "sparsk_last_error", "sparsk_destroy")
 
 OK, EINVAL, ECAPACITY, ENOHEAD, ECUDA, ESTATE, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
 
@@ -96,6 +96,8 @@ def load():
     L.sparsk_attention_scratch_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32]
     L.sparsk_attention.restype = C.c_int
     L.sparsk_attention.argtypes = [C.POINTER(AttnArgs), vp, C.c_size_t, vp]
+    L.sparsk_attention_static.restype = C.c_int
+    L.sparsk_attention_static.argtypes = [C.POINTER(AttnArgs), vp, C.c_char_p, C.c_size_t]
     L.sparsk_launch_count.restype = C.c_int64
     L.sparsk_launch_count.argtypes = [vp]
     L.sparsk_last_error.restype = C.c_char_p
@@ -153,6 +155,18 @@ def attention(args: AttnArgs, scratch: torch.Tensor, stream=None) -> int:
     """sparsk_attention on the current (or given) stream; returns the status code."""
     st = (stream or torch.cuda.current_stream()).cuda_stream
     return load().sparsk_attention(C.byref(args), scratch.data_ptr(), scratch.numel(), st)
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def attention_static(args: AttnArgs, stream=None):
+    """sparsk_attention_static: the attention kernels with the library's built-in scratch area,
+    for callers that cannot allocate.  Returns (status code, error text)."""
+    st = (stream or torch.cuda.current_stream()).cuda_stream
+    buf = C.create_string_buffer(256)
+    rc = load().sparsk_attention_static(C.byref(args), st, buf, len(buf))
+    return rc, buf.value.decode()
 
 
 def attention_scratch_bytes(n_rows: int, n_q_heads: int, head_dim: int) -> int:

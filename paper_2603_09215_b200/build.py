@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsparsk.so")
-SOURCES = ["sparsk_api.cu", "sparsk_ops.cu"]
+SOURCES = ["sparsk_api.cu", "sparsk_ops.cu", "sparsk_noalloc.cu"]
 
 
 def _stale() -> bool:
