@@ -29,6 +29,11 @@ SHAPES = {
                 d_ffn=13696, vocab_text=151552, vocab_speech=16384, rms_eps=1e-6,
                 rope_base=10000.0),
 }
+# Cut-down copies for profiler captures: the layers keep the full shapes (one layer's weights are
+# still several times the L2), but only four of them and a short text vocabulary, so that the
+# whole model stays near 2 GB on the device.
+SHAPES["step4"] = dict(SHAPES["step"], n_layers=4, vocab_text=8192)
+SHAPES["glm4"] = dict(SHAPES["glm"], n_layers=4, vocab_text=8192)
 
 # Workloads: (shape, batch, prompt length(s), decode steps, N_text, N_speech, e, K, r).
 WORKLOADS = {
@@ -46,6 +51,12 @@ WORKLOADS = {
     "cfg5_glm_b128": dict(shape="glm", batch=128, prompt=(8192, 8192), steps=256, n_text=13,
                           n_speech=26, exit_layer=30, refresh_period=4, refresh_phase=0,
                           random_phase=True),
+    # profiler-sized cases (not benchmark lines)
+    "prof_step4_b1": dict(shape="step4", batch=1, prompt=(512, 512), steps=64, n_text=1, n_speech=4,
+                          exit_layer=2, refresh_period=4, refresh_phase=0, random_phase=False),
+    "prof_glm4_b16": dict(shape="glm4", batch=16, prompt=(1024, 1024), steps=64, n_text=13,
+                          n_speech=26, exit_layer=3, refresh_period=4, refresh_phase=0,
+                          random_phase=False),
 }
 
 PER_LAYER = ("attn_norm", "wq", "wk", "wv", "wo", "mlp_norm", "w_gate", "w_up", "w_down",
