@@ -210,6 +210,12 @@ int sparsk_attention_static(const sparsk_attn_args *args /*host*/, void *cuda_st
  * bracketed launches and their number.  No counterpart in the paper: measurement only. */
 int sparsk_kernel_time(sparsk_ctx *ctx, double *total_ms /*host*/, int64_t *n_launches /*host*/);
 
+/* Synchronises the context's stream, then reads and clears the device status word that kernels
+ * raise instead of trapping: SPARSK_ETIMEOUT if a bounded in-kernel wait ran out, SPARSK_EINVAL
+ * if a token id had to be clamped into the vocabulary, else SPARSK_OK.  No counterpart in the
+ * paper: error reporting only. */
+int sparsk_check(sparsk_ctx *ctx);
+
 /* Number of kernels this library has launched on behalf of the context so far. */
 int64_t sparsk_launch_count(const sparsk_ctx *ctx);
 

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libsparsk.so")
 EXPORTS = ("sparsk_workspace_bytes", "sparsk_create", "sparsk_prefill", "sparsk_decode_step",
            "sparsk_decode_step_host", "sparsk_reset_slot", "sparsk_import_kv", "sparsk_export_kv",
            "sparsk_set_len", "sparsk_slot_state", "sparsk_set_debug", "sparsk_set_option",
-           "sparsk_kernel_time", "sparsk_attention", "sparsk_attention_scratch_bytes", "sparsk_attention_static", "sparsk_launch_count", "sparsk_last_error", "sparsk_destroy")
+           "sparsk_kernel_time", "sparsk_check", "sparsk_attention", "sparsk_attention_scratch_bytes", "sparsk_attention_static", "sparsk_launch_count", "sparsk_last_error", "sparsk_destroy")
 
 OK, EINVAL, ECAPACITY, ENOHEAD, ECUDA, ESTATE, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
 
@@ -98,6 +98,8 @@ def load():
     L.sparsk_attention.argtypes = [C.POINTER(AttnArgs), vp, C.c_size_t, vp]
     L.sparsk_attention_static.restype = C.c_int
     L.sparsk_attention_static.argtypes = [C.POINTER(AttnArgs), vp, C.c_char_p, C.c_size_t]
+    L.sparsk_check.restype = C.c_int
+    L.sparsk_check.argtypes = [vp]
     L.sparsk_launch_count.restype = C.c_int64
     L.sparsk_launch_count.argtypes = [vp]
     L.sparsk_last_error.restype = C.c_char_p
@@ -286,6 +288,10 @@ class Sparsk:
         ms, n = C.c_double(), C.c_int64()
         self._check(self.lib.sparsk_kernel_time(self.h, C.byref(ms), C.byref(n)))
         return ms.value, n.value
+
+    def check(self):
+        """Synchronise, then raise if a kernel reported a problem through the device status word."""
+        self._check(self.lib.sparsk_check(self.h))
 
     def launch_count(self) -> int:
         return self.lib.sparsk_launch_count(self.h)

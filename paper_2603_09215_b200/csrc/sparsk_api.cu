@@ -11,6 +11,7 @@
 #include "../../include/sparsk.h"
 #include "sparsk_attn.cuh"
 #include "sparsk_common.cuh"
+#include "sparsk_gemm.cuh"
 #include "sparsk_gemv.cuh"
 #include "sparsk_step.cuh"
 
@@ -58,7 +59,7 @@ struct sparsk_ctx {
     int *staged, *tok_dev, *out_tok_dev, *out_depth_dev;
     int *pf_slot, *pf_pos, *pf_grp_row0, *pf_grp_nrows, *pf_ngrp, *pf_nrows;
     float *h_lo, *h_up;
-    bf16 *qbuf, *attn_o, *act;
+    bf16 *qbuf, *attn_o, *act, *xnorm;
     float *part_o;
     float2 *part_ml;
     // pinned staging ring for the per-step host arrays
@@ -71,6 +72,11 @@ struct sparsk_ctx {
     int pdl, attn_split, gemm_min_rows, use_graph, gv_ks, gv_r, gv_grid_mult;
     float *dbg_hidden, *dbg_logits;
     int64_t launches;
+    // tensor-core path: TMA descriptors of every weight matrix and of the activation buffers
+    // (one per box height 16, 32, 64, 128, 256)
+    bool tc_ok;
+    std::vector<CUtensorMap> tm_wq, tm_wk, tm_wv, tm_wo, tm_wg, tm_wu, tm_wd, tm_head;
+    CUtensorMap tm_x[5], tm_ao[5], tm_act[5];
     // optional per-kernel-class timing (events around every launch of one class)
     int cur_class, time_class;
     std::vector<cudaEvent_t> tev;
@@ -149,6 +155,7 @@ size_t carve(sparsk_ctx *c, const sparsk_dims *d, char *base)
     int *pfng = w.take<int>(1), *pfnr = w.take<int>(1);
     float *hlo = w.take<float>(B * d->d_model), *hup = w.take<float>(R * d->d_model);
     bf16 *q = w.take<bf16>(R * qrow), *ao = w.take<bf16>(R * qrow), *act = w.take<bf16>(R * d->d_ffn);
+    bf16 *xn = w.take<bf16>(R * d->d_model);
     float *po = w.take<float>(R * d->n_q_heads * MAX_SPLITS * d->head_dim);
     float2 *pml = w.take<float2>(R * d->n_q_heads * MAX_SPLITS);
     if (c) {
@@ -156,7 +163,7 @@ size_t carve(sparsk_ctx *c, const sparsk_dims *d, char *base)
         c->sd = sd; c->staged = staged; c->tok_dev = tok; c->out_tok_dev = ot; c->out_depth_dev = od;
         c->pf_slot = pfs; c->pf_pos = pfp; c->pf_grp_row0 = pfg0; c->pf_grp_nrows = pfgn;
         c->pf_ngrp = pfng; c->pf_nrows = pfnr;
-        c->h_lo = hlo; c->h_up = hup; c->qbuf = q; c->attn_o = ao; c->act = act;
+        c->h_lo = hlo; c->h_up = hup; c->qbuf = q; c->attn_o = ao; c->act = act; c->xnorm = xn;
         c->part_o = po; c->part_ml = pml;
     }
     return align_up(w.off, 256);
@@ -312,6 +319,9 @@ cudaError_t run_gateup(sparsk_ctx *c, int layer, const float *h, int n_rows)
 #undef GU_CASE
 }
 
+bool use_tc(const sparsk_ctx *c, int n_rows);
+cudaError_t run_head_tc(sparsk_ctx *c, int layer, const float *h, int list, int n_rows);
+
 // Head of `layer` over list `l` (0 early/text, 1 early/speech, 2 full/text, 3 full/speech).
 cudaError_t run_head(sparsk_ctx *c, int layer, const float *h, int list, int n_rows)
 {
@@ -321,6 +331,7 @@ cudaError_t run_head(sparsk_ctx *c, int layer, const float *h, int list, int n_r
     in.h = h; in.gain = c->head_norm[li]; in.eps = d.rms_eps; in.K = d.d_model; in.n_rows = n_rows;
     in.row_idx = c->sd.list_row + (size_t)list * B;
     const int speech = list & 1;
+    if (use_tc(c, n_rows)) return run_head_tc(c, layer, h, list, n_rows);
     const int R = c->gv_r > 0 ? c->gv_r : 4;
     struct ClassScope {
         sparsk_ctx *c;
@@ -373,12 +384,183 @@ cudaError_t run_attn(sparsk_ctx *c, int layer, const RowSet &rs)
     return launch(c, attn_merge_kernel<64>, dim3(rs.n_rows, d.n_q_heads), dim3(64), 0, a, rs.n_rows_dev);
 }
 
+
+// ---------------------------------------------------------------- tensor-core dispatch
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// Descriptor of a row-major bf16 matrix [rows][cols] read in boxes of [box_rows][64] with the
+// 128-byte swizzle; out-of-range parts of a box read as zero.
+bool encode_map(EncodeTiledFn fn, CUtensorMap *m, const void *base, size_t rows, size_t cols, int box_rows)
+{
+    memset(m, 0, sizeof *m);
+    if (!base) return true;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)GM_BK, (cuuint32_t)box_rows};
+    const cuuint32_t es[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, es,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool build_maps(sparsk_ctx *c)
+{
+    const sparsk_dims &d = c->dm;
+    void *fp = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fp, cudaEnableDefault, &qr) != cudaSuccess || !fp ||
+        qr != cudaDriverEntryPointSuccess)
+        return false;
+    EncodeTiledFn fn = (EncodeTiledFn)fp;
+    const int L = d.n_layers, V = d.vocab_text + d.vocab_speech;
+    const size_t qd = (size_t)d.n_q_heads * d.head_dim, kd = (size_t)d.n_kv_heads * d.head_dim;
+    bool ok = true;
+    auto fill = [&](std::vector<CUtensorMap> &v, const std::vector<const bf16 *> &w, size_t rows, size_t cols) {
+        v.resize(L);
+        for (int l = 0; l < L; l++) ok = ok && encode_map(fn, &v[l], w[l], rows, cols, GM_BM);
+    };
+    fill(c->tm_wq, c->wq, qd, d.d_model); fill(c->tm_wk, c->wk, kd, d.d_model); fill(c->tm_wv, c->wv, kd, d.d_model);
+    fill(c->tm_wo, c->wo, d.d_model, qd); fill(c->tm_wg, c->w_gate, d.d_ffn, d.d_model);
+    fill(c->tm_wu, c->w_up, d.d_ffn, d.d_model); fill(c->tm_wd, c->w_down, d.d_model, d.d_ffn);
+    fill(c->tm_head, c->head_proj, V, d.d_model);
+    for (int b = 0; b < 5; b++) {
+        const int box = 16 << b;
+        ok = ok && encode_map(fn, &c->tm_x[b], c->xnorm, c->cap_rows, d.d_model, box);
+        ok = ok && encode_map(fn, &c->tm_ao[b], c->attn_o, c->cap_rows, qd, box);
+        ok = ok && encode_map(fn, &c->tm_act[b], c->act, c->cap_rows, d.d_ffn, box);
+    }
+    return ok;
+}
+
+int box_index(int m_rows)
+{
+    int b = 0;
+    while (b < 4 && (16 << b) < std::min(m_rows, GM_MAX_N)) b++;
+    return b;
+}
+
+template <class Epi>
+cudaError_t launch_gemm(sparsk_ctx *c, const CUtensorMap &a0, const CUtensorMap &a1, const CUtensorMap &a2,
+                        const CUtensorMap *b_maps, GemmArgs g, const Epi &epi)
+{
+    static bool attr_set = false;
+    constexpr int SMEM_BUDGET = 220 * 1024;
+    auto kern = wsgemm_kernel<Epi>;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    const int bi = box_index(g.m_rows);
+    g.box_n = 16 << bi;
+    const int stage_bytes = g.n_acc * GM_A_BYTES + g.box_n * GM_BK * 2;
+    g.stages = std::min(GM_MAX_STAGES, (SMEM_BUDGET - 1024 - GM_XCHG_BYTES) / stage_bytes);
+    if (g.stages < 2) return cudaErrorInvalidValue;
+    g.status = c->sd.counts + CNT_STATUS;
+    const int n_tiles = g.tiles[0] + (g.n_acc == 2 ? 0 : g.tiles[1] + g.tiles[2]);
+    const int k_iters = (g.K + GM_BK - 1) / GM_BK;
+    g.splits = std::max(1, std::min(g.splits, k_iters));
+    const int grid_x = std::max(1, std::min(c->n_sm, n_tiles * g.splits));
+    const int grid_y = (g.m_rows + GM_MAX_N - 1) / GM_MAX_N;
+    const size_t smem = 1024 + (size_t)g.stages * stage_bytes + GM_XCHG_BYTES;
+    return launch(c, kern, dim3(grid_x, grid_y), dim3(GM_THREADS), smem, a0, a1, a2, b_maps[bi], g, epi);
+}
+
+int div_up(int a, int b) { return (a + b - 1) / b; }
+
+cudaError_t run_norm(sparsk_ctx *c, const float *h, const bf16 *gain, const int *row_idx, int n_rows)
+{
+    return launch(c, rmsnorm_rows_kernel, dim3(n_rows), dim3(256), 0, h, gain, row_idx, c->xnorm, n_rows,
+                  c->dm.d_model, c->dm.rms_eps);
+}
+
+// One transformer layer over a row set on the tensor-core path.
+cudaError_t run_layer_tc(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
+{
+    const sparsk_dims &d = c->dm;
+    const int li = layer - 1, M = rs.n_rows;
+    const int qd = d.n_q_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim;
+    const size_t lstride = (size_t)d.max_seqs * d.n_kv_heads * d.max_seq_len * d.head_dim;
+    cudaError_t e;
+    c->cur_class = KC_MISC;
+    if ((e = run_norm(c, h, c->attn_norm[li], nullptr, M)) != cudaSuccess) return e;
+    {
+        c->cur_class = KC_QKV;
+        GemmArgs g{};
+        g.K = d.d_model; g.tiles[0] = div_up(qd, GM_BM); g.tiles[1] = g.tiles[2] = div_up(kd, GM_BM);
+        g.splits = 1; g.n_acc = 1; g.m_rows = M;
+        QkvEnd ep;
+        ep.q_out = c->qbuf; ep.kc = c->kcache + li * lstride; ep.vc = c->vcache + li * lstride; ep.rope = c->rope;
+        ep.row_slot = rs.slot; ep.row_pos = rs.pos; ep.Hq = d.n_q_heads; ep.Hkv = d.n_kv_heads; ep.hd = d.head_dim;
+        ep.S = d.max_seq_len;
+        if ((e = launch_gemm(c, c->tm_wq[li], c->tm_wk[li], c->tm_wv[li], c->tm_x, g, ep)) != cudaSuccess) return e;
+    }
+    c->cur_class = KC_ATTN;
+    if ((e = run_attn(c, layer, rs)) != cudaSuccess) return e;
+    {
+        c->cur_class = KC_OPROJ;
+        GemmArgs g{};
+        g.K = qd; g.tiles[0] = div_up(d.d_model, GM_BM); g.n_acc = 1; g.m_rows = M;
+        g.splits = c->n_sm / g.tiles[0];
+        ResidEnd ep;
+        ep.h = h; ep.n_out = d.d_model; ep.atomic = 1;
+        if ((e = launch_gemm(c, c->tm_wo[li], c->tm_wo[li], c->tm_wo[li], c->tm_ao, g, ep)) != cudaSuccess) return e;
+    }
+    c->cur_class = KC_MISC;
+    if ((e = run_norm(c, h, c->mlp_norm[li], nullptr, M)) != cudaSuccess) return e;
+    {
+        c->cur_class = KC_GATEUP;
+        GemmArgs g{};
+        g.K = d.d_model; g.tiles[0] = div_up(d.d_ffn, GM_BM); g.n_acc = 2; g.m_rows = M; g.splits = 1;
+        GateUpEnd ep;
+        ep.u = c->act; ep.F = d.d_ffn;
+        if ((e = launch_gemm(c, c->tm_wg[li], c->tm_wu[li], c->tm_wu[li], c->tm_x, g, ep)) != cudaSuccess) return e;
+    }
+    {
+        c->cur_class = KC_DOWN;
+        GemmArgs g{};
+        g.K = d.d_ffn; g.tiles[0] = div_up(d.d_model, GM_BM); g.n_acc = 1; g.m_rows = M;
+        g.splits = c->n_sm / g.tiles[0];
+        ResidEnd ep;
+        ep.h = h; ep.n_out = d.d_model; ep.atomic = 1;
+        e = launch_gemm(c, c->tm_wd[li], c->tm_wd[li], c->tm_wd[li], c->tm_act, g, ep);
+    }
+    c->cur_class = KC_MISC;
+    return e;
+}
+
+bool use_tc(const sparsk_ctx *c, int n_rows) { return c->tc_ok && n_rows >= c->gemm_min_rows && c->dm.d_model >= GM_BK; }
+
+// Head of `layer` over list `l` on the tensor-core path.
+cudaError_t run_head_tc(sparsk_ctx *c, int layer, const float *h, int list, int n_rows)
+{
+    const sparsk_dims &d = c->dm;
+    const int li = layer - 1, B = d.max_seqs, speech = list & 1;
+    cudaError_t e;
+    c->cur_class = KC_MISC;
+    if ((e = run_norm(c, h, c->head_norm[li], c->sd.list_row + (size_t)list * B, n_rows)) != cudaSuccess) return e;
+    c->cur_class = KC_HEAD;
+    HeadEnd ep;
+    ep.seq_of_row = c->sd.list_seq + (size_t)list * B; ep.argmax = c->sd.argmax; ep.logits = c->dbg_logits;
+    ep.lo = speech ? d.vocab_text : 0; ep.hi = speech ? d.vocab_text + d.vocab_speech : d.vocab_text;
+    ep.V = d.vocab_text + d.vocab_speech;
+    GemmArgs g{};
+    g.K = d.d_model; g.tiles[0] = div_up(ep.hi - ep.lo, GM_BM); g.row0[0] = ep.lo; g.n_acc = 1; g.m_rows = n_rows;
+    g.splits = 1;
+    e = launch_gemm(c, c->tm_head[li], c->tm_head[li], c->tm_head[li], c->tm_x, g, ep);
+    c->cur_class = KC_MISC;
+    return e;
+}
+
 // One transformer layer over a row set: h <- h^(layer).
 cudaError_t run_layer(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
 {
     const sparsk_dims &d = c->dm;
     const int li = layer - 1;
     cudaError_t e;
+    if (use_tc(c, rs.n_rows)) return run_layer_tc(c, layer, h, rs);
     c->cur_class = KC_QKV;
     if ((e = run_qkv(c, layer, h, rs)) != cudaSuccess) return e;
     c->cur_class = KC_ATTN;
@@ -447,7 +629,8 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
     carve(ctx, &ctx->dm, (char *)workspace);
     ctx->h_len.assign(dims->max_seqs, 0);
     ctx->h_pend.assign(dims->max_seqs, 0);
-    ctx->pdl = 0; ctx->attn_split = 0; ctx->gemm_min_rows = 1 << 30; ctx->use_graph = 0;
+    ctx->pdl = 0; ctx->attn_split = 0; ctx->gemm_min_rows = 5; ctx->use_graph = 0;
+    ctx->tc_ok = false;
     ctx->gv_ks = 0; ctx->gv_r = 0; ctx->gv_grid_mult = 1;
     ctx->dbg_hidden = nullptr; ctx->dbg_logits = nullptr;
     ctx->launches = 0;
@@ -470,6 +653,12 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
                 rc = fail(ctx, SPARSK_ECUDA, "staging setup failed: %s", cudaGetErrorString(ce));
         }
         if (rc) break;
+        // no silent change of path: without TMA descriptors the batched path cannot run
+        ctx->tc_ok = build_maps(ctx);
+        if (!ctx->tc_ok) {
+            rc = fail(ctx, SPARSK_ECUDA, "building the TMA descriptors failed");
+            break;
+        }
         // rotary table in double, stored as float (cos, sin)
         const int half = dims->head_dim / 2;
         std::vector<float2> tab((size_t)dims->max_seq_len * half);
@@ -557,6 +746,18 @@ extern "C" int sparsk_kernel_time(sparsk_ctx *ctx, double *total_ms, int64_t *n_
     }
     *total_ms = tot;
     *n_launches = (int64_t)(ctx->tev_used / 2);
+    return SPARSK_OK;
+}
+
+extern "C" int sparsk_check(sparsk_ctx *ctx)
+{
+    if (!good(ctx)) return SPARSK_ESTATE;
+    int status = 0;
+    CU(cudaMemcpyAsync(&status, ctx->sd.counts + CNT_STATUS, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+    CU(cudaStreamSynchronize(ctx->stream));
+    if (status) CU(cudaMemsetAsync(ctx->sd.counts + CNT_STATUS, 0, sizeof(int), ctx->stream));
+    if (status & ST_TIMEOUT) return fail(ctx, SPARSK_ETIMEOUT, "a bounded in-kernel wait ran out");
+    if (status & ST_BAD_TOKEN) return fail(ctx, SPARSK_EINVAL, "a token id was outside the vocabulary (clamped)");
     return SPARSK_OK;
 }
 

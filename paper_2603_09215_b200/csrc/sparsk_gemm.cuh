@@ -1,0 +1,499 @@
+// Batched weight-streaming path: Y^T = W X^T on the 5th-generation tensor cores.
+//
+// Once a pass has more than a handful of activation rows (a batch of sequences in the lower
+// pass, pending + current rows of all full-depth sequences in the upper pass, a prompt chunk in
+// prefill) every projection of a layer is a dense contraction whose weights must still be read
+// from HBM exactly once (Sec. IV-B.3: one batched pass loads each weight matrix once).  The
+// weights are therefore the M operand of tcgen05.mma (128 weight rows per tile, read through a
+// 2-D TMA tensor map straight from the caller's row-major matrices), the active rows are the N
+// operand (16..256, so a small batch still fills the instruction), accumulators live in TMEM.
+//
+// One persistent CTA per SM, three roles:
+//   warp 0      producer: TMA loads of [128 x 64] weight tiles and [N x 64] activation tiles
+//               (128-byte swizzle) into a ring of shared-memory stages
+//   warp 1      issues tcgen05.mma for every stage, commits stages back to the producer and
+//               finished accumulators to the epilogue; owns the TMEM allocation
+//   warps 2..5  epilogue: tcgen05.ld of the accumulator (thread = weight row), then the
+//               operation's own ending: rotary embedding + cache append, residual add,
+//               SiLU(gate) * up, or logits + restricted arg max
+// Accumulators are double buffered in TMEM so a tile's epilogue overlaps the next tile's MMAs.
+// Every wait is bounded: on a timeout the CTA raises ST_TIMEOUT, stops issuing work, drains its
+// own copies, frees its TMEM and returns.
+#pragma once
+
+#include <cuda.h>
+
+#include "sparsk_common.cuh"
+
+namespace sparsk {
+
+constexpr int GM_THREADS = 192;
+constexpr int GM_BM = 128;                     // weight rows per tile (UMMA M)
+constexpr int GM_BK = 64;                      // inner elements per stage: one 128-byte swizzle span
+constexpr int GM_MAX_N = 256;                  // activation rows per launch block (UMMA N limit)
+constexpr int GM_A_BYTES = GM_BM * GM_BK * 2;  // 16 KB
+constexpr int GM_MAX_STAGES = 12;
+constexpr int GM_CHUNK = 16;                   // accumulator columns per epilogue chunk
+constexpr int GM_XCHG_BYTES = GM_CHUNK * GM_BM * 4;
+constexpr unsigned long long GM_TIMEOUT_NS = 2000000000ull;
+
+struct GemmArgs {
+    int K;         // inner dimension
+    int tiles[3];  // 128-row tiles of weight matrix 0, 1, 2
+    int row0[3];   // first row of each matrix that belongs to this product (a head's id range)
+    int splits;    // cuts of the inner dimension per tile (> 1 only with an additive ending)
+    int n_acc;     // accumulators per tile: 2 when matrices 0 and 1 are streamed side by side
+    int m_rows;    // activation rows of the whole launch; block y owns rows [256 y, 256 y + 256)
+    int box_n;     // activation rows per TMA box (16, 32, 64, 128 or 256)
+    int stages;    // ring depth
+    int *status;   // device status word
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_test(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait for a phase of an mbarrier.  Returns false if the CTA is giving up (another
+// thread did, or this wait outlasted `limit_ns`); the caller then leaves its loop.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *giving_up, int *status,
+                                          unsigned long long limit_ns = GM_TIMEOUT_NS)
+{
+    unsigned long long t0 = 0;
+    for (uint32_t spin = 0;; ++spin) {
+        if (mbar_test(bar, parity)) return true;
+        if (spin > 32) __nanosleep(40);
+        if ((spin & 255u) == 255u) {
+            if (*giving_up) return false;
+            const unsigned long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > limit_ns) {
+                *giving_up = 1;
+                if (status) atomicOr(status, ST_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, uint64_t *bar, int x, int y)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// Shared-memory matrix descriptor of a K-major tile stored with the 128-byte swizzle: rows are
+// 128 bytes, groups of eight rows are 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr)
+{
+    return (uint64_t)((smem_addr & 0x3ffffu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
+           (2ull << 61);
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t umma_idesc_bf16(int n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(GM_BM >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, int accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16])
+{
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; i++) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// What an ending sees of one finished tile.
+struct TileCtx {
+    int matrix;      // which weight matrix the tile belongs to (0..2)
+    int tile;        // tile index inside that matrix
+    int split;       // which cut of the inner dimension
+    int row;         // this thread's weight row inside the tile (its TMEM lane), 0..127
+    int m0, m_end;   // activation rows of this launch block: [m0, m_end)
+    uint32_t taddr;  // TMEM address of accumulator 0, this thread's lane, column 0
+    int acc_stride;  // columns between accumulator 0 and accumulator 1
+    float *xchg;     // [GM_CHUNK][128] floats shared by the 128 epilogue threads
+};
+
+// ------------------------------------------------------------------ kernel
+template <class Epi>
+__global__ void __launch_bounds__(GM_THREADS, 1)
+    wsgemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
+                  const __grid_constant__ CUtensorMap map_a2, const __grid_constant__ CUtensorMap map_b,
+                  const GemmArgs g, const Epi epi)
+{
+    extern __shared__ __align__(1024) unsigned char gm_smem[];
+    __shared__ __align__(8) uint64_t full_bar[GM_MAX_STAGES], empty_bar[GM_MAX_STAGES], acc_full[2], acc_empty[2];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int giving_up_s;
+    volatile int *giving_up = &giving_up_s;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t ring = (smem_u32(gm_smem) + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
+    const int b_bytes = g.box_n * GM_BK * 2;
+    const int stage_bytes = g.n_acc * GM_A_BYTES + b_bytes;
+    unsigned char *ring_ptr = gm_smem + (ring - smem_u32(gm_smem));
+    float *xchg = reinterpret_cast<float *>(ring_ptr + (size_t)g.stages * stage_bytes);
+
+    const int m0 = blockIdx.y * GM_MAX_N;
+    const int m_end = min(g.m_rows, m0 + GM_MAX_N);
+    const int mma_n = ((m_end - m0) + 15) & ~15;
+    const int k_iters = (g.K + GM_BK - 1) / GM_BK;
+    const int n_tiles = g.tiles[0] + (g.n_acc == 2 ? 0 : g.tiles[1] + g.tiles[2]);
+    const int n_units = n_tiles * g.splits;
+    // accumulator buffers: 2 when they fit, else 1
+    const int acc_cols = g.n_acc * mma_n;
+    const int n_buf = (2 * acc_cols <= 512) ? 2 : 1;
+    uint32_t alloc_cols = 32;
+    while ((int)alloc_cols < n_buf * acc_cols) alloc_cols <<= 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < g.stages; s++) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 1);
+        }
+        for (int b = 0; b < 2; b++) {
+            mbar_init(&acc_full[b], 1);
+            mbar_init(&acc_empty[b], 4);
+        }
+        giving_up_s = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)),
+                     "r"(alloc_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+
+    // The weights do not depend on the previous kernel; everything else does.
+    griddep_wait();
+    griddep_launch();
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+                const int t = u / g.splits, sp = u % g.splits;
+                int mat = 0, tl = t;
+                if (g.n_acc == 1) {
+                    if (tl >= g.tiles[0]) { tl -= g.tiles[0]; mat = 1; }
+                    if (mat == 1 && tl >= g.tiles[1]) { tl -= g.tiles[1]; mat = 2; }
+                }
+                const CUtensorMap *ma = mat == 0 ? &map_a0 : (mat == 1 ? &map_a1 : &map_a2);
+                const int k_beg = (int)((long)k_iters * sp / g.splits), k_end = (int)((long)k_iters * (sp + 1) / g.splits);
+                for (int k = k_beg; k < k_end; k++, it++) {
+                    const int s = it % g.stages;
+                    const uint32_t ph = (it / g.stages) & 1;
+                    if (!(ok = mbar_wait(&empty_bar[s], ph ^ 1, giving_up, g.status))) break;
+                    unsigned char *st = ring_ptr + (size_t)s * stage_bytes;
+                    mbar_expect_tx(&full_bar[s], (uint32_t)stage_bytes);
+                    tma_load_2d(st, ma, &full_bar[s], k * GM_BK, g.row0[mat] + tl * GM_BM);
+                    if (g.n_acc == 2) tma_load_2d(st + GM_A_BYTES, &map_a1, &full_bar[s], k * GM_BK, g.row0[1] + tl * GM_BM);
+                    tma_load_2d(st + g.n_acc * GM_A_BYTES, &map_b, &full_bar[s], k * GM_BK, m0);
+                }
+            }
+            if (!ok) {
+                // giving up: let the copies already issued land (2 ms each at most) before the CTA
+                // goes away; stage s was last filled in round (it - 1 - s) / stages
+                __shared__ int never_s;
+                never_s = 0;
+                for (int s = 0; s < g.stages; s++)
+                    if (it > (uint32_t)s) mbar_wait(&full_bar[s], ((it - 1 - s) / g.stages) & 1, &never_s, nullptr, 2000000ull);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_bf16(mma_n);
+            uint32_t it = 0, tile_it = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, tile_it++) {
+                const int sp = u % g.splits;
+                const int k_beg = (int)((long)k_iters * sp / g.splits), k_end = (int)((long)k_iters * (sp + 1) / g.splits);
+                const int buf = tile_it % n_buf;
+                const uint32_t bph = (tile_it / n_buf) & 1;
+                if (!(ok = mbar_wait(&acc_empty[buf], bph ^ 1, giving_up, g.status))) break;
+                tc_fence_after();
+                const uint32_t d0 = tmem_base + (uint32_t)(buf * acc_cols);
+                for (int k = k_beg; k < k_end; k++, it++) {
+                    const int s = it % g.stages;
+                    const uint32_t ph = (it / g.stages) & 1;
+                    if (!(ok = mbar_wait(&full_bar[s], ph, giving_up, g.status))) break;
+                    tc_fence_after();
+                    const uint32_t a_addr = ring + (uint32_t)s * stage_bytes;
+                    const uint32_t b_addr = a_addr + g.n_acc * GM_A_BYTES;
+#pragma unroll
+                    for (int kk = 0; kk < GM_BK / 16; kk++) {
+                        const uint64_t db = umma_desc_sw128(b_addr + kk * 32);
+                        const int accum = (k > k_beg || kk > 0) ? 1 : 0;
+                        umma_bf16(d0, umma_desc_sw128(a_addr + kk * 32), db, idesc, accum);
+                        if (g.n_acc == 2) umma_bf16(d0 + mma_n, umma_desc_sw128(a_addr + GM_A_BYTES + kk * 32), db, idesc, accum);
+                    }
+                    umma_commit(&empty_bar[s]);  // the stage is free once these MMAs have read it
+                }
+                if (ok) umma_commit(&acc_full[buf]);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..5)
+        const int quad = warp & 3;  // TMEM lanes this warp may read: 32 quad .. 32 quad + 31
+        TileCtx tc;
+        tc.row = quad * 32 + lane;
+        tc.m0 = m0;
+        tc.m_end = m_end;
+        tc.acc_stride = mma_n;
+        tc.xchg = xchg;
+        uint32_t tile_it = 0;
+        bool ok = true;
+        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, tile_it++) {
+            const int t = u / g.splits;
+            tc.split = u % g.splits;
+            tc.matrix = 0;
+            tc.tile = t;
+            if (g.n_acc == 1) {
+                if (tc.tile >= g.tiles[0]) { tc.tile -= g.tiles[0]; tc.matrix = 1; }
+                if (tc.matrix == 1 && tc.tile >= g.tiles[1]) { tc.tile -= g.tiles[1]; tc.matrix = 2; }
+            }
+            const int buf = tile_it % n_buf;
+            const uint32_t bph = (tile_it / n_buf) & 1;
+            if (!(ok = mbar_wait(&acc_full[buf], bph, giving_up, g.status))) break;
+            tc_fence_after();
+            tc.taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * acc_cols);
+            epi.tile(tc);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[buf]);
+        }
+    }
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(alloc_cols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------ endings
+// All endings walk the accumulator in chunks of 16 columns (activation rows); thread = weight row.
+
+// q/k/v: rotary embedding of q and k (pairs i, i + hd/2 sit hd/2 lanes apart, so values are
+// exchanged through shared memory), q to the query buffer, k and v appended to the cache.
+struct QkvEnd {
+    bf16 *q_out;         // [rows][Hq*hd]
+    bf16 *kc, *vc;       // this layer's cache [slot][Hkv][S][hd]
+    const float2 *rope;  // [S][hd/2]
+    const int *row_slot, *row_pos;
+    int Hq, Hkv, hd, S;
+
+    __device__ void tile(const TileCtx &t) const
+    {
+        const int half = hd >> 1;
+        const int n = t.tile * GM_BM + t.row;  // row inside its matrix
+        const int n_rows_mat = (t.matrix == 0 ? Hq : Hkv) * hd;
+        const int head = n / hd, i = n % hd, j = i & (half - 1);
+        const bool hi = i >= half;
+        for (int c0 = 0; t.m0 + c0 < t.m_end; c0 += GM_CHUNK) {
+            float v[GM_CHUNK];
+            tmem_ld16(t.taddr + c0, v);
+            if (t.matrix < 2) {
+#pragma unroll
+                for (int c = 0; c < GM_CHUNK; c++) t.xchg[c * GM_BM + t.row] = v[c];
+                epi_barrier();
+            }
+            if (n < n_rows_mat) {
+#pragma unroll
+                for (int c = 0; c < GM_CHUNK; c++) {
+                    const int m = t.m0 + c0 + c;
+                    if (m >= t.m_end) break;
+                    const int slot = row_slot[m], pos = row_pos[m];
+                    if (t.matrix == 2) {
+                        vc[(((size_t)slot * Hkv + head) * S + pos) * hd + i] = __float2bfloat16(v[c]);
+                    } else {
+                        const float other = t.xchg[c * GM_BM + (t.row ^ half)];
+                        const float2 cs = rope[(size_t)pos * half + j];
+                        const float r = hi ? v[c] * cs.x + other * cs.y : v[c] * cs.x - other * cs.y;
+                        if (t.matrix == 0) q_out[(size_t)m * Hq * hd + n] = __float2bfloat16(r);
+                        else kc[(((size_t)slot * Hkv + head) * S + pos) * hd + i] = __float2bfloat16(r);
+                    }
+                }
+            }
+            if (t.matrix < 2) epi_barrier();
+        }
+    }
+};
+
+// h[m][n] += (W x_m)[n]; with the inner dimension cut across CTAs the partial sums meet in h.
+struct ResidEnd {
+    float *h;  // [rows][n_out]
+    int n_out, atomic;
+
+    __device__ void tile(const TileCtx &t) const
+    {
+        const int n = t.tile * GM_BM + t.row;
+        for (int c0 = 0; t.m0 + c0 < t.m_end; c0 += GM_CHUNK) {
+            float v[GM_CHUNK];
+            tmem_ld16(t.taddr + c0, v);
+            if (n >= n_out) continue;
+#pragma unroll
+            for (int c = 0; c < GM_CHUNK; c++) {
+                const int m = t.m0 + c0 + c;
+                if (m >= t.m_end) break;
+                float *dst = h + (size_t)m * n_out + n;
+                if (atomic) atomicAdd(dst, v[c]);
+                else *dst += v[c];
+            }
+        }
+    }
+};
+
+// u[m][f] = silu(gate) * up; accumulator 0 holds the gate rows, accumulator 1 the up rows.
+struct GateUpEnd {
+    bf16 *u;  // [rows][F]
+    int F;
+
+    __device__ void tile(const TileCtx &t) const
+    {
+        const int f = t.tile * GM_BM + t.row;
+        for (int c0 = 0; t.m0 + c0 < t.m_end; c0 += GM_CHUNK) {
+            float gt[GM_CHUNK], up[GM_CHUNK];
+            tmem_ld16(t.taddr + c0, gt);
+            tmem_ld16(t.taddr + t.acc_stride + c0, up);
+            if (f >= F) continue;
+#pragma unroll
+            for (int c = 0; c < GM_CHUNK; c++) {
+                const int m = t.m0 + c0 + c;
+                if (m >= t.m_end) break;
+                u[(size_t)m * F + f] = __float2bfloat16(gt[c] / (1.f + __expf(-gt[c])) * up[c]);
+            }
+        }
+    }
+};
+
+// Exit head over ids [lo, hi): per activation row the arg max (lowest id on ties) through the
+// same packed 64-bit key the small-batch path uses; optional dump of the logits.
+struct HeadEnd {
+    const int *seq_of_row;
+    unsigned long long *argmax;
+    float *logits;  // optional [n_seq][V]
+    int lo, hi, V;
+
+    __device__ void tile(const TileCtx &t) const
+    {
+        const int id = lo + t.tile * GM_BM + t.row;
+        const int lane = threadIdx.x & 31;
+        for (int c0 = 0; t.m0 + c0 < t.m_end; c0 += GM_CHUNK) {
+            float v[GM_CHUNK];
+            tmem_ld16(t.taddr + c0, v);
+#pragma unroll
+            for (int c = 0; c < GM_CHUNK; c++) {
+                const int m = t.m0 + c0 + c;
+                if (m >= t.m_end) break;  // uniform across the warp
+                unsigned long long key = id < hi ? argmax_key(v[c], id) : 0ull;
+                if (logits && id < hi) logits[(size_t)seq_of_row[m] * V + id] = v[c];
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
+                    key = other > key ? other : key;
+                }
+                if (lane == 0 && key) atomicMax(&argmax[seq_of_row[m]], key);
+            }
+        }
+    }
+};
+
+// RMSNorm of selected fp32 rows into the bf16 activation matrix the GEMM reads:
+// x[i] = h[row_idx ? row_idx[i] : i] / sqrt(mean(h^2) + eps) * gain.
+static __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const float *__restrict__ h, const bf16 *__restrict__ gain,
+                                                           const int *__restrict__ row_idx, bf16 *__restrict__ x,
+                                                           int n_rows, int K, float eps)
+{
+    __shared__ float red[8];
+    griddep_wait();
+    griddep_launch();
+    const int i = blockIdx.x;
+    if (i >= n_rows) return;
+    const float *src = h + (size_t)(row_idx ? row_idx[i] : i) * K;
+    float ss = 0.f;
+    for (int k = threadIdx.x * 4; k < K; k += 256 * 4) {
+        const float4 v = *reinterpret_cast<const float4 *>(src + k);
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    }
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; w++) tot += red[w];
+    const float inv = rsqrtf(tot / (float)K + eps);
+    for (int k = threadIdx.x * 8; k < K; k += 256 * 8) {
+        const float4 a = *reinterpret_cast<const float4 *>(src + k);
+        const float4 b = *reinterpret_cast<const float4 *>(src + k + 4);
+        float gn[8];
+        unpack8(*reinterpret_cast<const uint4 *>(gain + k), gn);
+        uint4 o;
+        o.x = pack_bf16x2(a.x * inv * gn[0], a.y * inv * gn[1]);
+        o.y = pack_bf16x2(a.z * inv * gn[2], a.w * inv * gn[3]);
+        o.z = pack_bf16x2(b.x * inv * gn[4], b.y * inv * gn[5]);
+        o.w = pack_bf16x2(b.z * inv * gn[6], b.w * inv * gn[7]);
+        *reinterpret_cast<uint4 *>(x + (size_t)i * K + k) = o;
+    }
+}
+
+}  // namespace sparsk

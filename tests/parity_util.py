@@ -44,6 +44,7 @@ class Pair:
     def prefill(self, prompts):
         """prompts: full prompts; the last token of each is kept as the first step's input."""
         self.g.prefill(list(range(self.n)), [p[:-1] for p in prompts])
+        self.g.check()
         for s, p in zip(self.os, prompts):
             s.prefill(p[:-1])
         self.next_in = [int(p[-1]) for p in prompts]
@@ -54,7 +55,7 @@ class Pair:
         ref = [self.os[s].decode_step(self.next_in[s], mods[i], ctrs[i]) for i, s in enumerate(slots)]
         self.tok[:k] = torch.tensor([self.next_in[s] for s in slots], dtype=torch.int32)
         self.g.decode_step(slots, self.tok, mods, ctrs, self.out_tok, self.out_dep)
-        torch.cuda.synchronize()
+        self.g.check()
         got_tok = self.out_tok[:k].cpu().numpy()
         got_dep = self.out_dep[:k].cpu().numpy()
         H = self.dbg_h[:k].cpu().numpy().astype(np.float64)

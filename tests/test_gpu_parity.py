@@ -42,15 +42,16 @@ def test_config1_tiny_full_run(util):
     P.close()
 
 
+@pytest.mark.parametrize("min_rows", [5, 1])
 @pytest.mark.parametrize("e,K,r,nt,ns", [(1, 2, 0, 1, 4), (2, 4, 1, 2, 7), (3, 2, 0, 1, 4), (2, 1, 0, 1, 4),
                                           (1, 5, 4, 0, 9)])
-def test_odd_shapes_and_schedules(util, e, K, r, nt, ns):
+def test_odd_shapes_and_schedules(util, e, K, r, nt, ns, min_rows):
     """head_dim 64, 3 query heads per kv head, dimensions that are not multiples of the 256-wide
     chunks, vocabulary ranges that are not multiples of the row groups; several (e, K, r)."""
     dims = synth.model_dims(MICRO64, e, K, r)
     w = synth.make_weights(dims, seed=5)
     prompt = synth.make_prompts(dims, 1, 37, 37, seed=7)[0]
-    P = util.Pair(dims, w, 1, 128, 2 * K, prefill_rows=16)
+    P = util.Pair(dims, w, 1, 128, 2 * K, prefill_rows=16, options={"gemm_min_rows": min_rows})
     P.prefill([prompt])
     for g in range(40):
         m, c = synth.interleave(g, nt, ns)
@@ -59,15 +60,18 @@ def test_odd_shapes_and_schedules(util, e, K, r, nt, ns):
     P.close()
 
 
-def test_heterogeneous_batch_matches_per_sequence_oracle(util):
+@pytest.mark.parametrize("min_rows", [5, 1, 1 << 30])
+def test_heterogeneous_batch_matches_per_sequence_oracle(util, min_rows):
     """Batch of 7 with random interleave phases and counter offsets and ragged prompts, so every
-    step mixes text, early-exit and refresh rows; sequences stay independent."""
+    step mixes text, early-exit and refresh rows; sequences stay independent.  Run with the
+    default hand-over between the small-batch and the tensor-core path (5 rows), with every
+    projection on the tensor cores, and with every projection on the small-batch path."""
     dims = synth.model_dims("tiny", 2, 4, 0)
     w = synth.make_weights(dims, seed=0)
     B = 7
     prompts = synth.make_prompts(dims, B, 9, 70, seed=4)
     phi, off = synth.make_phases(B, 1, 4, 4, True, seed=8)
-    P = util.Pair(dims, w, B, 70 + 64, 3, prefill_rows=24)
+    P = util.Pair(dims, w, B, 70 + 64, 3, prefill_rows=24, options={"gemm_min_rows": min_rows})
     P.prefill(prompts)
     mixed = 0
     for g in range(48):
