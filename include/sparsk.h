@@ -153,7 +153,8 @@ int sparsk_set_debug(sparsk_ctx *ctx, float *exit_hidden /*device or NULL*/,
                      float *exit_logits /*device or NULL*/);
 
 /* Tuning knobs, by name: "gemm_min_rows" (row count from which the tcgen05 path is used; a
- * large value keeps everything on the GEMV path), "use_graph" (0/1), "attn_split" (positions
+ * large value keeps everything on the GEMV path), "gemm_kb" (1: one 64-element block of the inner
+ * dimension per TMA copy instead of two; 0 = automatic), "use_graph" (0/1), "attn_split" (positions
  * per KV split), "pdl" (0/1, programmatic dependent launch between the kernels of a step),
  * "gemv_ks" / "gemv_r" (override the GEMV team width / rows per group; 0 = automatic),
  * "time_kernel" (see sparsk_kernel_time).  Returns SPARSK_EINVAL for an unknown name or value. */

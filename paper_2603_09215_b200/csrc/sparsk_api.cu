@@ -42,6 +42,10 @@ struct Carve {
 
 }  // namespace
 
+struct TmaPair {
+    CUtensorMap m2, m3;
+};
+
 struct sparsk_ctx {
     uint32_t magic;
     sparsk_dims dm;
@@ -75,8 +79,10 @@ struct sparsk_ctx {
     // tensor-core path: TMA descriptors of every weight matrix and of the activation buffers
     // (one per box height 16, 32, 64, 128, 256)
     bool tc_ok;
-    std::vector<CUtensorMap> tm_wq, tm_wk, tm_wv, tm_wo, tm_wg, tm_wu, tm_wd, tm_head;
-    CUtensorMap tm_x[5], tm_ao[5], tm_act[5];
+    std::vector<TmaPair> tm_wq, tm_wk, tm_wv, tm_wo, tm_wg, tm_wu, tm_wd, tm_head;
+    TmaPair tm_x[5], tm_ao[5], tm_act[5];
+    float *qkv_part;  // fp32 sums of a q/k/v product whose inner dimension is cut across CTAs
+    int tc_kb;        // 0: automatic; 1: force one k-block per copy (2-D descriptors)
     // optional per-kernel-class timing (events around every launch of one class)
     int cur_class, time_class;
     std::vector<cudaEvent_t> tev;
@@ -156,6 +162,7 @@ size_t carve(sparsk_ctx *c, const sparsk_dims *d, char *base)
     float *hlo = w.take<float>(B * d->d_model), *hup = w.take<float>(R * d->d_model);
     bf16 *q = w.take<bf16>(R * qrow), *ao = w.take<bf16>(R * qrow), *act = w.take<bf16>(R * d->d_ffn);
     bf16 *xn = w.take<bf16>(R * d->d_model);
+    float *qp = w.take<float>(R * (qrow + 2 * kvrow));
     float *po = w.take<float>(R * d->n_q_heads * MAX_SPLITS * d->head_dim);
     float2 *pml = w.take<float2>(R * d->n_q_heads * MAX_SPLITS);
     if (c) {
@@ -163,7 +170,7 @@ size_t carve(sparsk_ctx *c, const sparsk_dims *d, char *base)
         c->sd = sd; c->staged = staged; c->tok_dev = tok; c->out_tok_dev = ot; c->out_depth_dev = od;
         c->pf_slot = pfs; c->pf_pos = pfp; c->pf_grp_row0 = pfg0; c->pf_grp_nrows = pfgn;
         c->pf_ngrp = pfng; c->pf_nrows = pfnr;
-        c->h_lo = hlo; c->h_up = hup; c->qbuf = q; c->attn_o = ao; c->act = act; c->xnorm = xn;
+        c->h_lo = hlo; c->h_up = hup; c->qbuf = q; c->attn_o = ao; c->act = act; c->xnorm = xn; c->qkv_part = qp;
         c->part_o = po; c->part_ml = pml;
     }
     return align_up(w.off, 256);
@@ -373,36 +380,47 @@ cudaError_t run_attn(sparsk_ctx *c, int layer, const RowSet &rs)
     a.n_rows = rs.n_rows;
     const int n_splits = pl.n_splits;
     dim3 grid(rs.n_groups_h * a.n_qblk, d.n_kv_heads, n_splits);
-    cudaError_t e;
-    if (d.head_dim == 128) {
-        e = launch(c, attn_partial_kernel<128>, grid, dim3(AT_THREADS), 0, a);
-        if (e != cudaSuccess) return e;
-        return launch(c, attn_merge_kernel<128>, dim3(rs.n_rows, d.n_q_heads), dim3(128), 0, a, rs.n_rows_dev);
-    }
-    e = launch(c, attn_partial_kernel<64>, grid, dim3(AT_THREADS), 0, a);
+    AttnPartialFn fn;
+    cudaError_t e = attn_partial_fn(d.head_dim, pl.mt, &fn);
     if (e != cudaSuccess) return e;
+    e = launch(c, fn, grid, dim3(AT_THREADS), attn_smem_bytes(d.head_dim, pl.mt), a);
+    if (e != cudaSuccess) return e;
+    if (d.head_dim == 128) return launch(c, attn_merge_kernel<128>, dim3(rs.n_rows, d.n_q_heads), dim3(128), 0, a, rs.n_rows_dev);
     return launch(c, attn_merge_kernel<64>, dim3(rs.n_rows, d.n_q_heads), dim3(64), 0, a, rs.n_rows_dev);
 }
-
 
 // ---------------------------------------------------------------- tensor-core dispatch
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// Descriptor of a row-major bf16 matrix [rows][cols] read in boxes of [box_rows][64] with the
-// 128-byte swizzle; out-of-range parts of a box read as zero.
-bool encode_map(EncodeTiledFn fn, CUtensorMap *m, const void *base, size_t rows, size_t cols, int box_rows)
+// Descriptors of a row-major bf16 matrix [rows][cols], 128-byte swizzle, zero fill outside:
+// m2 reads boxes of [box_rows][64]; m3 (only when cols is a multiple of 64) views the matrix as
+// [64][rows][cols/64] and reads [box_rows] rows of two consecutive 64-element blocks at once.
+bool encode_maps(EncodeTiledFn fn, TmaPair *m, const void *base, size_t rows, size_t cols, int box_rows)
 {
     memset(m, 0, sizeof *m);
     if (!base) return true;
-    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)GM_BK, (cuuint32_t)box_rows};
-    const cuuint32_t es[2] = {1, 1};
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, es,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    const cuuint32_t es[3] = {1, 1, 1};
+    {
+        const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+        const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+        const cuuint32_t box[2] = {(cuuint32_t)GM_BK, (cuuint32_t)box_rows};
+        if (fn(&m->m2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, es,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return false;
+    }
+    if (cols % GM_BK == 0) {
+        const cuuint64_t dims[3] = {(cuuint64_t)GM_BK, (cuuint64_t)rows, (cuuint64_t)(cols / GM_BK)};
+        const cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)GM_BK * 2};
+        const cuuint32_t box[3] = {(cuuint32_t)GM_BK, (cuuint32_t)box_rows, 2};
+        if (fn(&m->m3, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, es,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return false;
+    }
+    return true;
 }
 
 bool build_maps(sparsk_ctx *c)
@@ -417,19 +435,19 @@ bool build_maps(sparsk_ctx *c)
     const int L = d.n_layers, V = d.vocab_text + d.vocab_speech;
     const size_t qd = (size_t)d.n_q_heads * d.head_dim, kd = (size_t)d.n_kv_heads * d.head_dim;
     bool ok = true;
-    auto fill = [&](std::vector<CUtensorMap> &v, const std::vector<const bf16 *> &w, size_t rows, size_t cols) {
+    auto fill = [&](std::vector<TmaPair> &v, const std::vector<const bf16 *> &w, size_t rows, size_t cols, int box) {
         v.resize(L);
-        for (int l = 0; l < L; l++) ok = ok && encode_map(fn, &v[l], w[l], rows, cols, GM_BM);
+        for (int l = 0; l < L; l++) ok = ok && encode_maps(fn, &v[l], w[l], rows, cols, box);
     };
-    fill(c->tm_wq, c->wq, qd, d.d_model); fill(c->tm_wk, c->wk, kd, d.d_model); fill(c->tm_wv, c->wv, kd, d.d_model);
-    fill(c->tm_wo, c->wo, d.d_model, qd); fill(c->tm_wg, c->w_gate, d.d_ffn, d.d_model);
-    fill(c->tm_wu, c->w_up, d.d_ffn, d.d_model); fill(c->tm_wd, c->w_down, d.d_model, d.d_ffn);
-    fill(c->tm_head, c->head_proj, V, d.d_model);
+    fill(c->tm_wq, c->wq, qd, d.d_model, 2 * GM_BM); fill(c->tm_wk, c->wk, kd, d.d_model, 2 * GM_BM);
+    fill(c->tm_wv, c->wv, kd, d.d_model, 2 * GM_BM); fill(c->tm_wo, c->wo, d.d_model, qd, 2 * GM_BM);
+    fill(c->tm_wg, c->w_gate, d.d_ffn, d.d_model, GM_BM); fill(c->tm_wu, c->w_up, d.d_ffn, d.d_model, GM_BM);
+    fill(c->tm_wd, c->w_down, d.d_model, d.d_ffn, 2 * GM_BM); fill(c->tm_head, c->head_proj, V, d.d_model, 2 * GM_BM);
     for (int b = 0; b < 5; b++) {
         const int box = 16 << b;
-        ok = ok && encode_map(fn, &c->tm_x[b], c->xnorm, c->cap_rows, d.d_model, box);
-        ok = ok && encode_map(fn, &c->tm_ao[b], c->attn_o, c->cap_rows, qd, box);
-        ok = ok && encode_map(fn, &c->tm_act[b], c->act, c->cap_rows, d.d_ffn, box);
+        ok = ok && encode_maps(fn, &c->tm_x[b], c->xnorm, c->cap_rows, d.d_model, box);
+        ok = ok && encode_maps(fn, &c->tm_ao[b], c->attn_o, c->cap_rows, qd, box);
+        ok = ok && encode_maps(fn, &c->tm_act[b], c->act, c->cap_rows, d.d_ffn, box);
     }
     return ok;
 }
@@ -442,8 +460,8 @@ int box_index(int m_rows)
 }
 
 template <class Epi>
-cudaError_t launch_gemm(sparsk_ctx *c, const CUtensorMap &a0, const CUtensorMap &a1, const CUtensorMap &a2,
-                        const CUtensorMap *b_maps, GemmArgs g, const Epi &epi)
+cudaError_t launch_gemm(sparsk_ctx *c, const TmaPair &a0, const TmaPair &a1, const TmaPair &a2, const TmaPair *b_maps,
+                        GemmArgs g, const Epi &epi)
 {
     static bool attr_set = false;
     constexpr int SMEM_BUDGET = 220 * 1024;
@@ -455,17 +473,23 @@ cudaError_t launch_gemm(sparsk_ctx *c, const CUtensorMap &a0, const CUtensorMap 
     }
     const int bi = box_index(g.m_rows);
     g.box_n = 16 << bi;
-    const int stage_bytes = g.n_acc * GM_A_BYTES + g.box_n * GM_BK * 2;
-    g.stages = std::min(GM_MAX_STAGES, (SMEM_BUDGET - 1024 - GM_XCHG_BYTES) / stage_bytes);
+    const int room = SMEM_BUDGET - 1024 - GM_XCHG_BYTES;
+    auto stage_bytes = [&](int kb) { return 2 * kb * GM_BLK_BYTES + kb * g.box_n * GM_BK * 2; };
+    // two k-blocks per copy whenever the inner dimension allows the 3-D view and two stages fit
+    g.three_d = (g.K % GM_BK == 0) && 2 * stage_bytes(2) <= room && c->tc_kb != 1;
+    g.kb = g.three_d ? 2 : 1;
+    g.stages = std::min(GM_MAX_STAGES, room / stage_bytes(g.kb));
     if (g.stages < 2) return cudaErrorInvalidValue;
     g.status = c->sd.counts + CNT_STATUS;
-    const int n_tiles = g.tiles[0] + (g.n_acc == 2 ? 0 : g.tiles[1] + g.tiles[2]);
-    const int k_iters = (g.K + GM_BK - 1) / GM_BK;
-    g.splits = std::max(1, std::min(g.splits, k_iters));
-    const int grid_x = std::max(1, std::min(c->n_sm, n_tiles * g.splits));
+    const int n_units = g.units[0] + (g.pair ? 0 : g.units[1] + g.units[2]);
+    const int k_stages = ((g.K + GM_BK - 1) / GM_BK + g.kb - 1) / g.kb;
+    g.splits = std::max(1, std::min(g.splits, k_stages));
+    const int grid_x = std::max(1, std::min(c->n_sm, n_units * g.splits));
     const int grid_y = (g.m_rows + GM_MAX_N - 1) / GM_MAX_N;
-    const size_t smem = 1024 + (size_t)g.stages * stage_bytes + GM_XCHG_BYTES;
-    return launch(c, kern, dim3(grid_x, grid_y), dim3(GM_THREADS), smem, a0, a1, a2, b_maps[bi], g, epi);
+    const size_t smem = 1024 + (size_t)g.stages * stage_bytes(g.kb) + GM_XCHG_BYTES;
+    if (g.three_d)
+        return launch(c, kern, dim3(grid_x, grid_y), dim3(GM_THREADS), smem, a0.m3, a1.m3, a2.m3, b_maps[bi].m3, g, epi);
+    return launch(c, kern, dim3(grid_x, grid_y), dim3(GM_THREADS), smem, a0.m2, a1.m2, a2.m2, b_maps[bi].m2, g, epi);
 }
 
 int div_up(int a, int b) { return (a + b - 1) / b; }
@@ -476,6 +500,9 @@ cudaError_t run_norm(sparsk_ctx *c, const float *h, const bf16 *gain, const int 
                   c->dm.d_model, c->dm.rms_eps);
 }
 
+// How many cuts of the inner dimension fill the machine when a product has `units` units.
+int splits_for(const sparsk_ctx *c, int units) { return units * 2 <= c->n_sm ? c->n_sm / units : 1; }
+
 // One transformer layer over a row set on the tensor-core path.
 cudaError_t run_layer_tc(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
 {
@@ -483,27 +510,33 @@ cudaError_t run_layer_tc(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
     const int li = layer - 1, M = rs.n_rows;
     const int qd = d.n_q_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim;
     const size_t lstride = (size_t)d.max_seqs * d.n_kv_heads * d.max_seq_len * d.head_dim;
+    bf16 *kc = c->kcache + li * lstride, *vc = c->vcache + li * lstride;
     cudaError_t e;
     c->cur_class = KC_MISC;
     if ((e = run_norm(c, h, c->attn_norm[li], nullptr, M)) != cudaSuccess) return e;
     {
         c->cur_class = KC_QKV;
         GemmArgs g{};
-        g.K = d.d_model; g.tiles[0] = div_up(qd, GM_BM); g.tiles[1] = g.tiles[2] = div_up(kd, GM_BM);
-        g.splits = 1; g.n_acc = 1; g.m_rows = M;
+        g.K = d.d_model; g.units[0] = div_up(qd, 2 * GM_BM); g.units[1] = g.units[2] = div_up(kd, 2 * GM_BM);
+        g.m_rows = M;
+        g.splits = splits_for(c, g.units[0] + g.units[1] + g.units[2]);
         QkvEnd ep;
-        ep.q_out = c->qbuf; ep.kc = c->kcache + li * lstride; ep.vc = c->vcache + li * lstride; ep.rope = c->rope;
+        ep.q_out = c->qbuf; ep.kc = kc; ep.vc = vc; ep.rope = c->rope;
         ep.row_slot = rs.slot; ep.row_pos = rs.pos; ep.Hq = d.n_q_heads; ep.Hkv = d.n_kv_heads; ep.hd = d.head_dim;
-        ep.S = d.max_seq_len;
+        ep.S = d.max_seq_len; ep.partial = g.splits > 1 ? c->qkv_part : nullptr;
         if ((e = launch_gemm(c, c->tm_wq[li], c->tm_wk[li], c->tm_wv[li], c->tm_x, g, ep)) != cudaSuccess) return e;
+        if (g.splits > 1 &&
+            (e = launch(c, qkv_finish_kernel, dim3(M), dim3(256), 0, c->qkv_part, c->qbuf, kc, vc, (const float2 *)c->rope,
+                        rs.slot, rs.pos, M, d.n_q_heads, d.n_kv_heads, d.head_dim, d.max_seq_len)) != cudaSuccess)
+            return e;
     }
     c->cur_class = KC_ATTN;
     if ((e = run_attn(c, layer, rs)) != cudaSuccess) return e;
     {
         c->cur_class = KC_OPROJ;
         GemmArgs g{};
-        g.K = qd; g.tiles[0] = div_up(d.d_model, GM_BM); g.n_acc = 1; g.m_rows = M;
-        g.splits = c->n_sm / g.tiles[0];
+        g.K = qd; g.units[0] = div_up(d.d_model, 2 * GM_BM); g.m_rows = M;
+        g.splits = splits_for(c, g.units[0]);
         ResidEnd ep;
         ep.h = h; ep.n_out = d.d_model; ep.atomic = 1;
         if ((e = launch_gemm(c, c->tm_wo[li], c->tm_wo[li], c->tm_wo[li], c->tm_ao, g, ep)) != cudaSuccess) return e;
@@ -513,7 +546,7 @@ cudaError_t run_layer_tc(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
     {
         c->cur_class = KC_GATEUP;
         GemmArgs g{};
-        g.K = d.d_model; g.tiles[0] = div_up(d.d_ffn, GM_BM); g.n_acc = 2; g.m_rows = M; g.splits = 1;
+        g.K = d.d_model; g.units[0] = div_up(d.d_ffn, GM_BM); g.pair = 1; g.m_rows = M; g.splits = 1;
         GateUpEnd ep;
         ep.u = c->act; ep.F = d.d_ffn;
         if ((e = launch_gemm(c, c->tm_wg[li], c->tm_wu[li], c->tm_wu[li], c->tm_x, g, ep)) != cudaSuccess) return e;
@@ -521,8 +554,8 @@ cudaError_t run_layer_tc(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
     {
         c->cur_class = KC_DOWN;
         GemmArgs g{};
-        g.K = d.d_ffn; g.tiles[0] = div_up(d.d_model, GM_BM); g.n_acc = 1; g.m_rows = M;
-        g.splits = c->n_sm / g.tiles[0];
+        g.K = d.d_ffn; g.units[0] = div_up(d.d_model, 2 * GM_BM); g.m_rows = M;
+        g.splits = splits_for(c, g.units[0]);
         ResidEnd ep;
         ep.h = h; ep.n_out = d.d_model; ep.atomic = 1;
         e = launch_gemm(c, c->tm_wd[li], c->tm_wd[li], c->tm_wd[li], c->tm_act, g, ep);
@@ -547,7 +580,7 @@ cudaError_t run_head_tc(sparsk_ctx *c, int layer, const float *h, int list, int 
     ep.lo = speech ? d.vocab_text : 0; ep.hi = speech ? d.vocab_text + d.vocab_speech : d.vocab_text;
     ep.V = d.vocab_text + d.vocab_speech;
     GemmArgs g{};
-    g.K = d.d_model; g.tiles[0] = div_up(ep.hi - ep.lo, GM_BM); g.row0[0] = ep.lo; g.n_acc = 1; g.m_rows = n_rows;
+    g.K = d.d_model; g.units[0] = div_up(ep.hi - ep.lo, 2 * GM_BM); g.row0[0] = ep.lo; g.m_rows = n_rows;
     g.splits = 1;
     e = launch_gemm(c, c->tm_head[li], c->tm_head[li], c->tm_head[li], c->tm_x, g, ep);
     c->cur_class = KC_MISC;
@@ -631,6 +664,7 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
     ctx->h_pend.assign(dims->max_seqs, 0);
     ctx->pdl = 0; ctx->attn_split = 0; ctx->gemm_min_rows = 5; ctx->use_graph = 0;
     ctx->tc_ok = false;
+    ctx->tc_kb = 0;
     ctx->gv_ks = 0; ctx->gv_r = 0; ctx->gv_grid_mult = 1;
     ctx->dbg_hidden = nullptr; ctx->dbg_logits = nullptr;
     ctx->launches = 0;
@@ -673,6 +707,7 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
             (ce = cudaMemsetAsync(ctx->kv_len, 0, sizeof(int) * dims->max_seqs, ctx->stream)) != cudaSuccess ||
             (ce = cudaMemsetAsync(ctx->pend_cnt, 0, sizeof(int) * dims->max_seqs, ctx->stream)) != cudaSuccess ||
             (ce = cudaMemsetAsync(ctx->sd.counts, 0, sizeof(int) * 8, ctx->stream)) != cudaSuccess ||
+            (ce = cudaMemsetAsync(ctx->qkv_part, 0, sizeof(float) * (size_t)ctx->cap_rows * (dims->n_q_heads + 2 * dims->n_kv_heads) * dims->head_dim, ctx->stream)) != cudaSuccess ||
             (ce = cudaStreamSynchronize(ctx->stream)) != cudaSuccess) {
             rc = fail(ctx, SPARSK_ECUDA, "table upload failed: %s", cudaGetErrorString(ce));
             break;
@@ -720,6 +755,7 @@ extern "C" int sparsk_set_option(sparsk_ctx *ctx, const char *name, int64_t valu
     else if (!strcmp(name, "pdl") && (value == 0 || value == 1)) ctx->pdl = (int)value;
     else if (!strcmp(name, "attn_split") && value >= 0 && value <= (1 << 24)) ctx->attn_split = (int)value;
     else if (!strcmp(name, "gemv_ks") && (value == 0 || value == 1 || value == 2 || value == 4 || value == 8 || value == 16)) ctx->gv_ks = (int)value;
+    else if (!strcmp(name, "gemm_kb") && (value == 0 || value == 1)) ctx->tc_kb = (int)value;
     else if (!strcmp(name, "gemv_r") && (value == 0 || value == 1 || value == 2 || value == 4)) ctx->gv_r = (int)value;
     else if (!strcmp(name, "time_kernel") && value >= 0 && value <= KC_HEAD) {
         // start (or stop, with 0) timing every launch of one kernel class; resets the totals

@@ -1,14 +1,20 @@
-// Split-KV grouped-query attention over the ragged KV cache (flash-decoding).
+// Split-KV grouped-query attention over the ragged KV cache (flash-decoding) on tensor cores.
 //
 // One CTA handles one (sequence group, block of query vectors, kv head, KV split).  A group is
 // the block of rows of ONE sequence that a pass processes together: a single row in the lower
 // pass, the pending positions plus the current one in the upper pass (Algorithm 1: "batch
 // P u {t} ... length-K mask"), a chunk of the prompt in prefill.  All query heads that share
-// the kv head, for all rows of the group, are served from one read of that head's K/V tile;
-// row r of the group may look at positions <= pos0 + r (the causal mask of the block on top
-// of the whole earlier cache).  K/V tiles are fetched with coalesced 16-byte loads; softmax
-// statistics are reduced with warp shuffles; each split writes an unnormalised partial
-// (acc, running max, running sum) and a second kernel merges the splits.
+// the kv head, for all rows of the group, form the M dimension of mma.sync m16n8k16 tiles, so one
+// read of that head's K/V serves them all; row r of the group may look at positions
+// <= pos0 + r (the causal mask of the block on top of the whole earlier cache).
+//
+// The split's positions are dealt to the CTA's four warps as contiguous sub-ranges.  Each warp
+// streams its own 16-position K/V tiles into a private three-stage shared-memory ring with
+// coalesced 16-byte cp.async copies (no CTA-wide barrier in the loop), computes S = Q K^T and
+// O += P V with bf16 MMAs and fp32 accumulators, and keeps an online softmax whose row maxima
+// and sums are reduced with shuffles inside the four-lane groups that share an accumulator row.
+// The four warps' states are merged through shared memory into one unnormalised partial
+// (acc, running max, running sum) per split; a second kernel merges the splits.
 #pragma once
 
 #include "sparsk_common.cuh"
@@ -16,20 +22,24 @@
 namespace sparsk {
 
 constexpr int AT_THREADS = 128;
-constexpr int AT_QB = 32;    // query vectors per CTA
-constexpr int AT_TILE = 32;  // KV positions per tile
+constexpr int AT_TP = 16;        // positions per warp tile
+constexpr int AT_NST = 3;        // ring stages per warp
 constexpr int AT_MAX_SPLITS = 32;
 constexpr int AT_MIN_SPLIT = 64;
 
-// How a launch cuts the KV range: enough splits to fill the machine, none shorter than
-// AT_MIN_SPLIT positions (unless forced), at most AT_MAX_SPLITS.
+// How a launch cuts the work: query vectors per CTA (16 or 32), and the KV range into enough
+// splits to fill the machine, none shorter than AT_MIN_SPLIT positions (unless forced), at most
+// AT_MAX_SPLITS.
 struct AttnPlan {
+    int mt;  // m16 tiles per CTA: 1 or 2
     int n_qblk, split_len, n_splits;
 };
 inline AttnPlan attn_plan(int n_sm, int n_groups, int max_grp_rows, int G, int Hkv, int max_len, int forced_split)
 {
     AttnPlan p;
-    p.n_qblk = (max_grp_rows * G + AT_QB - 1) / AT_QB;
+    const int nq = max_grp_rows * G;
+    p.mt = nq > 16 ? 2 : 1;
+    p.n_qblk = (nq + 16 * p.mt - 1) / (16 * p.mt);
     int split = forced_split;
     if (split <= 0) {
         const long base = (long)n_groups * p.n_qblk * Hkv;
@@ -38,17 +48,24 @@ inline AttnPlan attn_plan(int n_sm, int n_groups, int max_grp_rows, int G, int H
         split = (int)((max_len + want - 1) / want);
         if (split < AT_MIN_SPLIT) split = AT_MIN_SPLIT;
     }
-    split = (split + AT_TILE - 1) / AT_TILE * AT_TILE;
+    split = (split + AT_TP - 1) / AT_TP * AT_TP;
     int n_splits = (max_len + split - 1) / split;
     if (n_splits > AT_MAX_SPLITS) {
         n_splits = AT_MAX_SPLITS;
-        split = ((max_len + n_splits - 1) / n_splits + AT_TILE - 1) / AT_TILE * AT_TILE;
+        split = ((max_len + n_splits - 1) / n_splits + AT_TP - 1) / AT_TP * AT_TP;
         n_splits = (max_len + split - 1) / split;
     }
     if (n_splits < 1) n_splits = 1;
     p.split_len = split;
     p.n_splits = n_splits;
     return p;
+}
+inline size_t attn_smem_bytes(int head_dim, int mt)
+{
+    const size_t kp = head_dim + 8;
+    const size_t q = (size_t)16 * mt * kp * 2, ring = (size_t)4 * AT_NST * 2 * AT_TP * kp * 2;
+    const size_t merge = (size_t)4 * 16 * mt * (head_dim + 2) * 4;
+    return q + (ring > merge ? ring : merge);
 }
 
 struct AttnArgs {
@@ -64,14 +81,47 @@ struct AttnArgs {
     int n_rows;               // rows in q/out; groups reaching beyond them are skipped
 };
 
-template <int HD>
+__device__ __forceinline__ void cp_async16(void *dst, const void *src, int src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src),
+                 "r"(src_bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait()
+{
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], const void *p)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"((uint32_t)__cvta_generic_to_shared(p)));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t (&r)[4], const void *p)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"((uint32_t)__cvta_generic_to_shared(p)));
+}
+// D += A B, A 16x16 bf16 (row), B 16x8 bf16 (col), D 16x8 fp32.
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+template <int HD, int MT>
 __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(AttnArgs a)
 {
-    constexpr int KP = HD + 8;  // padded row, keeps 16-byte row reads conflict-free
-    __shared__ __align__(16) float qs[AT_QB][HD];
-    __shared__ __align__(16) bf16 Ks[AT_TILE][KP];
-    __shared__ __align__(16) bf16 Vs[AT_TILE][KP];
-    __shared__ float Ps[AT_QB][AT_TILE];
+    constexpr int QB = 16 * MT;     // query vectors per CTA
+    constexpr int KP = HD + 8;      // padded row: ldmatrix rows fall into distinct banks
+    constexpr int CH = HD / 8;      // 16-byte chunks per row
+    extern __shared__ __align__(16) unsigned char at_smem[];
+    bf16 *Qs = reinterpret_cast<bf16 *>(at_smem);  // [QB][KP]
+    bf16 *ring = Qs + QB * KP;                     // [4 warps][AT_NST][K,V][AT_TP][KP]
 
     griddep_wait();
     griddep_launch();
@@ -82,9 +132,9 @@ __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(AttnArgs a)
     const int row0 = a.grp_row0[g], nrows = a.grp_nrows[g];
     if (row0 < 0 || nrows < 1 || row0 + nrows > a.n_rows) return;
     const int nq = nrows * G;
-    const int q0 = qb * AT_QB;
+    const int q0 = qb * QB;
     if (q0 >= nq) return;
-    const int nq_here = min(AT_QB, nq - q0);
+    const int nq_here = min(QB, nq - q0);
     const int slot = a.row_slot[row0], pos0 = a.row_pos[row0];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
@@ -96,111 +146,215 @@ __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(AttnArgs a)
     const int s_beg = sp * a.split_len;
     const int s_end = min(s_beg + a.split_len, kv_end_all);
 
-    // queries -> shared, pre-scaled by 1/sqrt(hd)
-    const float scale = rsqrtf((float)HD);
-    for (int i = tid; i < AT_QB * (HD / 8); i += AT_THREADS) {
-        const int qi = i / (HD / 8), c = i % (HD / 8);
-        float f[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    for (int i = tid; i < QB * CH; i += AT_THREADS) {
+        const int qi = i / CH, c = i % CH;
+        uint4 v = make_uint4(0, 0, 0, 0);
         if (qi < nq_here) {
             const int qg = q0 + qi, r = qg / G, j = qg % G;
-            unpack8(*reinterpret_cast<const uint4 *>(a.q + (size_t)(row0 + r) * a.Hq * HD + (hk * G + j) * HD + c * 8), f);
+            v = *reinterpret_cast<const uint4 *>(a.q + (size_t)(row0 + r) * a.Hq * HD + (hk * G + j) * HD + c * 8);
         }
-#pragma unroll
-        for (int e = 0; e < 8; e++) qs[qi][c * 8 + e] = f[e] * scale;
+        *reinterpret_cast<uint4 *>(&Qs[qi * KP + c * 8]) = v;
     }
+    __syncthreads();
 
-    constexpr int QW = AT_QB / 4;   // query vectors per warp
-    constexpr int DL = HD / 32;     // output dims per lane
-    float m_run[QW], l_run[QW], acc[QW][DL];
+    // this warp's share of the split
+    const int span = max(s_end - s_beg, 0);
+    const int per = (((span + 3) >> 2) + AT_TP - 1) / AT_TP * AT_TP;
+    const int w_beg = s_beg + warp * per;
+    const int w_end = min(w_beg + per, s_end);
+    const int n_tiles = w_end > w_beg ? (w_end - w_beg + AT_TP - 1) / AT_TP : 0;
+    bf16 *wr = ring + (size_t)warp * AT_NST * 2 * AT_TP * KP;
+    const bf16 *kbase = a.kc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
+    const bf16 *vbase = a.vc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
+
+    auto issue = [&](int t) {
+        bf16 *kt = wr + (size_t)(t % AT_NST) * 2 * AT_TP * KP, *vt = kt + AT_TP * KP;
+        const int p0 = w_beg + t * AT_TP;
 #pragma unroll
-    for (int i = 0; i < QW; i++) {
-        m_run[i] = -INFINITY;
-        l_run[i] = 0.f;
+        for (int i = lane; i < AT_TP * CH; i += 32) {
+            const int r = i / CH, c = i % CH;
+            const bool ok = p0 + r < w_end;                  // rows past the end are zero-filled
+            const size_t off = (size_t)(ok ? p0 + r : w_beg) * HD + c * 8;
+            cp_async16(&kt[r * KP + c * 8], kbase + off, ok ? 16 : 0);
+            cp_async16(&vt[r * KP + c * 8], vbase + off, ok ? 16 : 0);
+        }
+    };
+
+    float o[MT][HD / 8][4], m_run[MT][2], l_run[MT][2];
 #pragma unroll
-        for (int e = 0; e < DL; e++) acc[i][e] = 0.f;
+    for (int mt = 0; mt < MT; mt++) {
+        m_run[mt][0] = m_run[mt][1] = -INFINITY;
+        l_run[mt][0] = l_run[mt][1] = 0.f;
+#pragma unroll
+        for (int nt = 0; nt < HD / 8; nt++)
+#pragma unroll
+            for (int e = 0; e < 4; e++) o[mt][nt][e] = 0.f;
     }
-    const bf16 *kbase = a.kc + ((size_t)slot * a.Hkv + hk) * a.S * HD;
-    const bf16 *vbase = a.vc + ((size_t)slot * a.Hkv + hk) * a.S * HD;
+    // last position each of this thread's accumulator rows may see
+    int limit[MT][2];
+#pragma unroll
+    for (int mt = 0; mt < MT; mt++)
+#pragma unroll
+        for (int hf = 0; hf < 2; hf++) {
+            const int qi = mt * 16 + (lane >> 2) + hf * 8;
+            limit[mt][hf] = qi < nq_here ? pos0 + (q0 + qi) / G : -1;
+        }
+    const float scale = rsqrtf((float)HD);
 
-    for (int t0 = s_beg; t0 < s_end; t0 += AT_TILE) {
-        __syncthreads();  // previous tile fully consumed (also orders the query stores)
-        for (int i = tid; i < AT_TILE * (HD / 8); i += AT_THREADS) {
-            const int t = i / (HD / 8), c = i % (HD / 8);
-            uint4 kv = make_uint4(0, 0, 0, 0), vv = make_uint4(0, 0, 0, 0);
-            if (t0 + t < s_end) {
-                kv = ld_stream16(kbase + (size_t)(t0 + t) * HD + c * 8);
-                vv = ld_stream16(vbase + (size_t)(t0 + t) * HD + c * 8);
-            }
-            *reinterpret_cast<uint4 *>(&Ks[t][c * 8]) = kv;
-            *reinterpret_cast<uint4 *>(&Vs[t][c * 8]) = vv;
-        }
-        __syncthreads();
-        // scores: lane = position, each warp walks its QW query vectors
-        const int tpos = t0 + lane;
-        float sc[QW];
 #pragma unroll
-        for (int i = 0; i < QW; i++) sc[i] = 0.f;
-#pragma unroll 4
-        for (int c = 0; c < HD / 8; c++) {
-            float kf[8];
-            unpack8(*reinterpret_cast<const uint4 *>(&Ks[lane][c * 8]), kf);
-#pragma unroll
-            for (int i = 0; i < QW; i++) {
-                const float4 qa = *reinterpret_cast<const float4 *>(&qs[warp * QW + i][c * 8]);
-                const float4 qb4 = *reinterpret_cast<const float4 *>(&qs[warp * QW + i][c * 8 + 4]);
-                sc[i] += kf[0] * qa.x + kf[1] * qa.y + kf[2] * qa.z + kf[3] * qa.w + kf[4] * qb4.x +
-                         kf[5] * qb4.y + kf[6] * qb4.z + kf[7] * qb4.w;
-            }
-        }
-#pragma unroll
-        for (int i = 0; i < QW; i++) {
-            const int qi = warp * QW + i;
-            const int r = (q0 + qi) / G;
-            const bool ok = qi < nq_here && tpos < s_end && tpos <= pos0 + r;
-            const float s = ok ? sc[i] : -INFINITY;
-            const float m_new = fmaxf(m_run[i], warp_max(s));
-            float alpha = 1.f, p = 0.f;
-            if (m_new != -INFINITY) {
-                alpha = __expf(m_run[i] - m_new);  // exp(-inf) = 0 on the first live tile
-                p = __expf(s - m_new);
-            }
-            l_run[i] = l_run[i] * alpha + warp_sum(p);
-            m_run[i] = m_new;
-            Ps[qi][lane] = p;
-#pragma unroll
-            for (int e = 0; e < DL; e++) acc[i][e] *= alpha;
-        }
+    for (int t = 0; t < AT_NST - 1; t++) {
+        if (t < n_tiles) issue(t);
+        cp_async_commit();
+    }
+    for (int t = 0; t < n_tiles; t++) {
+        cp_async_wait<AT_NST - 2>();
         __syncwarp();
-        // acc += P V : lane owns DL consecutive output dims
-        for (int t = 0; t < AT_TILE; t++) {
-            float vf[DL];
-            if constexpr (DL == 4) {
-                const uint2 v2 = *reinterpret_cast<const uint2 *>(&Vs[t][lane * 4]);
-                vf[0] = bf_lo(v2.x); vf[1] = bf_hi(v2.x); vf[2] = bf_lo(v2.y); vf[3] = bf_hi(v2.y);
-            } else {
-                const uint32_t v1 = *reinterpret_cast<const uint32_t *>(&Vs[t][lane * 2]);
-                vf[0] = bf_lo(v1); vf[1] = bf_hi(v1);
+        if (t + AT_NST - 1 < n_tiles) issue(t + AT_NST - 1);
+        cp_async_commit();
+        const bf16 *Kt = wr + (size_t)(t % AT_NST) * 2 * AT_TP * KP, *Vt = Kt + AT_TP * KP;
+        const int p0 = w_beg + t * AT_TP;
+
+        // S = Q K^T for 16 positions
+        float s[MT][2][4];
+#pragma unroll
+        for (int mt = 0; mt < MT; mt++)
+#pragma unroll
+            for (int nt = 0; nt < 2; nt++)
+#pragma unroll
+                for (int e = 0; e < 4; e++) s[mt][nt][e] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < HD / 16; ks++) {
+            uint32_t kb[4];
+            ldsm_x4(kb, &Kt[((lane & 7) + ((lane >> 4) << 3)) * KP + ks * 16 + ((lane >> 3) & 1) * 8]);
+#pragma unroll
+            for (int mt = 0; mt < MT; mt++) {
+                uint32_t qa[4];
+                ldsm_x4(qa, &Qs[(mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * KP + ks * 16 + (lane >> 4) * 8]);
+                mma_bf16(s[mt][0], qa, kb[0], kb[1]);
+                mma_bf16(s[mt][1], qa, kb[2], kb[3]);
             }
+        }
+        // online softmax; P as the A operand of the second product
+        uint32_t pa[MT][4];
 #pragma unroll
-            for (int i = 0; i < QW; i++) {
-                const float p = Ps[warp * QW + i][t];
+        for (int mt = 0; mt < MT; mt++) {
 #pragma unroll
-                for (int e = 0; e < DL; e++) acc[i][e] = fmaf(p, vf[e], acc[i][e]);
+            for (int hf = 0; hf < 2; hf++) {
+                float v[4];
+                float tmax = -INFINITY;
+#pragma unroll
+                for (int nt = 0; nt < 2; nt++)
+#pragma unroll
+                    for (int e = 0; e < 2; e++) {
+                        const int p = p0 + nt * 8 + (lane & 3) * 2 + e;
+                        const bool ok = p < w_end && p <= limit[mt][hf];
+                        v[nt * 2 + e] = ok ? s[mt][nt][hf * 2 + e] * scale : -INFINITY;
+                        tmax = fmaxf(tmax, v[nt * 2 + e]);
+                    }
+                tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
+                tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
+                const float m_new = fmaxf(m_run[mt][hf], tmax);
+                float alpha = 1.f, psum = 0.f;
+                if (m_new != -INFINITY) {
+                    alpha = __expf(m_run[mt][hf] - m_new);  // exp(-inf) = 0 on the first live tile
+#pragma unroll
+                    for (int i = 0; i < 4; i++) {
+                        v[i] = __expf(v[i] - m_new);
+                        psum += v[i];
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 4; i++) v[i] = 0.f;
+                }
+                l_run[mt][hf] = l_run[mt][hf] * alpha + psum;  // per-thread share; lanes are summed at the end
+                m_run[mt][hf] = m_new;
+                pa[mt][hf] = pack_bf16x2(v[0], v[1]);       // positions 0..7 of the tile
+                pa[mt][2 + hf] = pack_bf16x2(v[2], v[3]);   // positions 8..15
+#pragma unroll
+                for (int nt = 0; nt < HD / 8; nt++) {
+                    o[mt][nt][hf * 2] *= alpha;
+                    o[mt][nt][hf * 2 + 1] *= alpha;
+                }
+            }
+        }
+        // O += P V
+#pragma unroll
+        for (int np = 0; np < HD / 16; np++) {
+            uint32_t vb[4];
+            ldsm_x4_t(vb, &Vt[((lane & 7) + ((lane >> 3) & 1) * 8) * KP + np * 16 + (lane >> 4) * 8]);
+#pragma unroll
+            for (int mt = 0; mt < MT; mt++) {
+                mma_bf16(o[mt][2 * np], pa[mt], vb[0], vb[1]);
+                mma_bf16(o[mt][2 * np + 1], pa[mt], vb[2], vb[3]);
             }
         }
     }
-    // partials (an empty split leaves max = -inf, sum = 0, which the merge ignores)
+    cp_async_wait<0>();
+    __syncthreads();  // every warp is done with its ring: reuse it for the merge
+
+    // merge the four warps' states
+    float *Ow = reinterpret_cast<float *>(ring);   // [4][QB][HD]
+    float *mw = Ow + 4 * QB * HD, *lw = mw + 4 * QB;  // [4][QB] each
 #pragma unroll
-    for (int i = 0; i < QW; i++) {
-        const int qi = warp * QW + i;
-        if (qi >= nq_here) continue;
+    for (int mt = 0; mt < MT; mt++)
+#pragma unroll
+        for (int hf = 0; hf < 2; hf++) {
+            float l = l_run[mt][hf];
+            l += __shfl_xor_sync(0xffffffffu, l, 1);
+            l += __shfl_xor_sync(0xffffffffu, l, 2);
+            const int qi = mt * 16 + (lane >> 2) + hf * 8;
+            if ((lane & 3) == 0) {
+                mw[warp * QB + qi] = m_run[mt][hf];
+                lw[warp * QB + qi] = l;
+            }
+#pragma unroll
+            for (int nt = 0; nt < HD / 8; nt++) {
+                float2 v2 = make_float2(o[mt][nt][hf * 2], o[mt][nt][hf * 2 + 1]);
+                *reinterpret_cast<float2 *>(&Ow[((size_t)warp * QB + qi) * HD + nt * 8 + (lane & 3) * 2]) = v2;
+            }
+        }
+    __syncthreads();
+    // partials (an empty split leaves max = -inf, sum = 0, which the merge of the splits ignores)
+    for (int idx = tid; idx < nq_here * HD; idx += AT_THREADS) {
+        const int qi = idx / HD, d = idx % HD;
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < 4; w++) M = fmaxf(M, mw[w * QB + qi]);
+        float acc = 0.f, L = 0.f;
+#pragma unroll
+        for (int w = 0; w < 4; w++) {
+            const float mwv = mw[w * QB + qi];
+            if (mwv == -INFINITY) continue;
+            const float wgt = __expf(mwv - M);
+            acc += Ow[((size_t)w * QB + qi) * HD + d] * wgt;
+            L += lw[w * QB + qi] * wgt;
+        }
         const int qg = q0 + qi, r = qg / G, j = qg % G;
         const size_t cell = ((size_t)(row0 + r) * a.Hq + hk * G + j) * a.n_splits + sp;
-        float *po = a.part_o + cell * HD + lane * DL;
-#pragma unroll
-        for (int e = 0; e < DL; e++) po[e] = acc[i][e];
-        if (lane == 0) a.part_ml[cell] = make_float2(m_run[i], l_run[i]);
+        a.part_o[cell * HD + d] = acc;
+        if (d == 0) a.part_ml[cell] = make_float2(M, L);
     }
+}
+
+typedef void (*AttnPartialFn)(AttnArgs);
+// The instantiation for a head dimension (64 or 128) and a query block of 16 * mt vectors, with
+// its dynamic shared-memory limit raised on first use.
+inline cudaError_t attn_partial_fn(int head_dim, int mt, AttnPartialFn *fn)
+{
+    static bool ready[4] = {false, false, false, false};
+    const int idx = (head_dim == 128 ? 2 : 0) + (mt == 2 ? 1 : 0);
+    AttnPartialFn f = idx == 3 ? attn_partial_kernel<128, 2>
+                      : idx == 2 ? attn_partial_kernel<128, 1>
+                      : idx == 1 ? attn_partial_kernel<64, 2>
+                                 : attn_partial_kernel<64, 1>;
+    if (!ready[idx]) {
+        const cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   (int)attn_smem_bytes(head_dim, mt));
+        if (e != cudaSuccess) return e;
+        ready[idx] = true;
+    }
+    *fn = f;
+    return cudaSuccess;
 }
 
 // Merge the splits of every (row, query head): out = sum_s acc_s e^{m_s - M} / sum_s l_s e^{m_s - M}.

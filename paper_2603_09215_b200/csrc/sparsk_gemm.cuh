@@ -28,24 +28,32 @@
 namespace sparsk {
 
 constexpr int GM_THREADS = 192;
-constexpr int GM_BM = 128;                     // weight rows per tile (UMMA M)
-constexpr int GM_BK = 64;                      // inner elements per stage: one 128-byte swizzle span
+constexpr int GM_BM = 128;                     // weight rows per accumulator (UMMA M)
+constexpr int GM_BK = 64;                      // inner elements per k-block: one 128-byte swizzle span
 constexpr int GM_MAX_N = 256;                  // activation rows per launch block (UMMA N limit)
-constexpr int GM_A_BYTES = GM_BM * GM_BK * 2;  // 16 KB
-constexpr int GM_MAX_STAGES = 12;
+constexpr int GM_BLK_BYTES = GM_BM * GM_BK * 2;  // one accumulator's weights for one k-block: 16 KB
+constexpr int GM_MAX_STAGES = 6;
 constexpr int GM_CHUNK = 16;                   // accumulator columns per epilogue chunk
 constexpr int GM_XCHG_BYTES = GM_CHUNK * GM_BM * 4;
 constexpr unsigned long long GM_TIMEOUT_NS = 2000000000ull;
 
+// A unit of work is two accumulators of 128 weight rows each: either 256 consecutive rows of one
+// matrix (one TMA box), or 128 rows of matrix 0 and the same 128 rows of matrix 1 ("pair": gate
+// and up, whose results meet in the ending).  The TMA engine spends a fixed few hundred
+// nanoseconds per copy whatever its size, so a stage is made of few, large boxes: with a
+// three-dimensional view [64 elements][rows][K/64] of a row-major matrix one box carries two
+// k-blocks of every row.
 struct GemmArgs {
     int K;         // inner dimension
-    int tiles[3];  // 128-row tiles of weight matrix 0, 1, 2
+    int units[3];  // units of matrix 0, 1, 2 (pair: units[0] only)
     int row0[3];   // first row of each matrix that belongs to this product (a head's id range)
-    int splits;    // cuts of the inner dimension per tile (> 1 only with an additive ending)
-    int n_acc;     // accumulators per tile: 2 when matrices 0 and 1 are streamed side by side
+    int splits;    // cuts of the inner dimension per unit (> 1 only with an additive ending)
+    int pair;      // 1: accumulator 1 comes from matrix 1
     int m_rows;    // activation rows of the whole launch; block y owns rows [256 y, 256 y + 256)
     int box_n;     // activation rows per TMA box (16, 32, 64, 128 or 256)
     int stages;    // ring depth
+    int kb;        // k-blocks per stage (1 or 2)
+    int three_d;   // 1: the descriptors are the [64][rows][K/64] views (needs K % 64 == 0)
     int *status;   // device status word
 };
 
@@ -89,7 +97,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
     unsigned long long t0 = 0;
     for (uint32_t spin = 0;; ++spin) {
         if (mbar_test(bar, parity)) return true;
-        if (spin > 32) __nanosleep(40);
+        if (spin > 64) __nanosleep(32);
         if ((spin & 255u) == 255u) {
             if (*giving_up) return false;
             const unsigned long long now = global_ns();
@@ -102,11 +110,18 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
         }
     }
 }
-__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, uint64_t *bar, int x, int y)
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint64_t *bar, int x, int y)
 {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+        ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint64_t *bar, int x, int y, int z)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
         : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -152,12 +167,12 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16])
 }
 __device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-// What an ending sees of one finished tile.
+// What an ending sees of one finished unit.
 struct TileCtx {
-    int matrix;      // which weight matrix the tile belongs to (0..2)
-    int tile;        // tile index inside that matrix
+    int matrix;      // which weight matrix the unit belongs to (0..2)
+    int unit_row;    // first weight row of accumulator 0 inside that matrix (without GemmArgs::row0)
     int split;       // which cut of the inner dimension
-    int row;         // this thread's weight row inside the tile (its TMEM lane), 0..127
+    int row;         // this thread's row inside an accumulator (its TMEM lane), 0..127
     int m0, m_end;   // activation rows of this launch block: [m0, m_end)
     uint32_t taddr;  // TMEM address of accumulator 0, this thread's lane, column 0
     int acc_stride;  // columns between accumulator 0 and accumulator 1
@@ -174,24 +189,27 @@ __global__ void __launch_bounds__(GM_THREADS, 1)
     extern __shared__ __align__(1024) unsigned char gm_smem[];
     __shared__ __align__(8) uint64_t full_bar[GM_MAX_STAGES], empty_bar[GM_MAX_STAGES], acc_full[2], acc_empty[2];
     __shared__ uint32_t tmem_base_s;
-    __shared__ int giving_up_s;
+    __shared__ int giving_up_s, never_s;
     volatile int *giving_up = &giving_up_s;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t ring = (smem_u32(gm_smem) + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
-    const int b_bytes = g.box_n * GM_BK * 2;
-    const int stage_bytes = g.n_acc * GM_A_BYTES + b_bytes;
-    unsigned char *ring_ptr = gm_smem + (ring - smem_u32(gm_smem));
-    float *xchg = reinterpret_cast<float *>(ring_ptr + (size_t)g.stages * stage_bytes);
+    const int a_bytes = 2 * g.kb * GM_BLK_BYTES;                 // both accumulators' weights of a stage
+    const int b_blk = g.box_n * GM_BK * 2;
+    const int stage_bytes = a_bytes + g.kb * b_blk;
+    // where accumulator a's rows of k-block j sit inside a stage
+    const int a_blk_stride = g.pair ? GM_BLK_BYTES : 2 * GM_BLK_BYTES;
+    const int a_acc_off = g.pair ? g.kb * GM_BLK_BYTES : GM_BLK_BYTES;
+    float *xchg = reinterpret_cast<float *>(gm_smem + (ring - smem_u32(gm_smem)) + (size_t)g.stages * stage_bytes);
 
     const int m0 = blockIdx.y * GM_MAX_N;
     const int m_end = min(g.m_rows, m0 + GM_MAX_N);
     const int mma_n = ((m_end - m0) + 15) & ~15;
-    const int k_iters = (g.K + GM_BK - 1) / GM_BK;
-    const int n_tiles = g.tiles[0] + (g.n_acc == 2 ? 0 : g.tiles[1] + g.tiles[2]);
-    const int n_units = n_tiles * g.splits;
+    const int kb_total = (g.K + GM_BK - 1) / GM_BK;
+    const int k_stages = (kb_total + g.kb - 1) / g.kb;
+    const int n_units = (g.units[0] + (g.pair ? 0 : g.units[1] + g.units[2])) * g.splits;
     // accumulator buffers: 2 when they fit, else 1
-    const int acc_cols = g.n_acc * mma_n;
+    const int acc_cols = 2 * mma_n;
     const int n_buf = (2 * acc_cols <= 512) ? 2 : 1;
     uint32_t alloc_cols = 32;
     while ((int)alloc_cols < n_buf * acc_cols) alloc_cols <<= 1;
@@ -206,6 +224,7 @@ __global__ void __launch_bounds__(GM_THREADS, 1)
             mbar_init(&acc_empty[b], 4);
         }
         giving_up_s = 0;
+        never_s = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -219,9 +238,20 @@ __global__ void __launch_bounds__(GM_THREADS, 1)
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
 
-    // The weights do not depend on the previous kernel; everything else does.
     griddep_wait();
     griddep_launch();
+
+    // unit u -> (matrix, first row, split)
+    auto locate = [&](int u, int &mat, int &unit_row, int &sp) {
+        int t = u / g.splits;
+        sp = u % g.splits;
+        mat = 0;
+        if (!g.pair) {
+            if (t >= g.units[0]) { t -= g.units[0]; mat = 1; }
+            if (mat == 1 && t >= g.units[1]) { t -= g.units[1]; mat = 2; }
+        }
+        unit_row = t * (g.pair ? GM_BM : 2 * GM_BM);
+    };
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
@@ -229,30 +259,32 @@ __global__ void __launch_bounds__(GM_THREADS, 1)
             uint32_t it = 0;
             bool ok = true;
             for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-                const int t = u / g.splits, sp = u % g.splits;
-                int mat = 0, tl = t;
-                if (g.n_acc == 1) {
-                    if (tl >= g.tiles[0]) { tl -= g.tiles[0]; mat = 1; }
-                    if (mat == 1 && tl >= g.tiles[1]) { tl -= g.tiles[1]; mat = 2; }
-                }
+                int mat, unit_row, sp;
+                locate(u, mat, unit_row, sp);
                 const CUtensorMap *ma = mat == 0 ? &map_a0 : (mat == 1 ? &map_a1 : &map_a2);
-                const int k_beg = (int)((long)k_iters * sp / g.splits), k_end = (int)((long)k_iters * (sp + 1) / g.splits);
-                for (int k = k_beg; k < k_end; k++, it++) {
+                const int row = g.row0[mat] + unit_row;
+                const int ks_beg = (int)((long)k_stages * sp / g.splits), ks_end = (int)((long)k_stages * (sp + 1) / g.splits);
+                for (int ks = ks_beg; ks < ks_end; ks++, it++) {
                     const int s = it % g.stages;
                     const uint32_t ph = (it / g.stages) & 1;
                     if (!(ok = mbar_wait(&empty_bar[s], ph ^ 1, giving_up, g.status))) break;
-                    unsigned char *st = ring_ptr + (size_t)s * stage_bytes;
+                    const uint32_t st = ring + (uint32_t)s * stage_bytes;
                     mbar_expect_tx(&full_bar[s], (uint32_t)stage_bytes);
-                    tma_load_2d(st, ma, &full_bar[s], k * GM_BK, g.row0[mat] + tl * GM_BM);
-                    if (g.n_acc == 2) tma_load_2d(st + GM_A_BYTES, &map_a1, &full_bar[s], k * GM_BK, g.row0[1] + tl * GM_BM);
-                    tma_load_2d(st + g.n_acc * GM_A_BYTES, &map_b, &full_bar[s], k * GM_BK, m0);
+                    const int blk = ks * g.kb;
+                    if (g.three_d) {
+                        tma_load_3d(st, ma, &full_bar[s], 0, row, blk);
+                        if (g.pair) tma_load_3d(st + a_acc_off, &map_a1, &full_bar[s], 0, g.row0[1] + unit_row, blk);
+                        tma_load_3d(st + a_bytes, &map_b, &full_bar[s], 0, m0, blk);
+                    } else {
+                        tma_load_2d(st, ma, &full_bar[s], blk * GM_BK, row);
+                        if (g.pair) tma_load_2d(st + a_acc_off, &map_a1, &full_bar[s], blk * GM_BK, g.row0[1] + unit_row);
+                        tma_load_2d(st + a_bytes, &map_b, &full_bar[s], blk * GM_BK, m0);
+                    }
                 }
             }
             if (!ok) {
                 // giving up: let the copies already issued land (2 ms each at most) before the CTA
                 // goes away; stage s was last filled in round (it - 1 - s) / stages
-                __shared__ int never_s;
-                never_s = 0;
                 for (int s = 0; s < g.stages; s++)
                     if (it > (uint32_t)s) mbar_wait(&full_bar[s], ((it - 1 - s) / g.stages) & 1, &never_s, nullptr, 2000000ull);
             }
@@ -261,29 +293,34 @@ __global__ void __launch_bounds__(GM_THREADS, 1)
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_bf16(mma_n);
-            uint32_t it = 0, tile_it = 0;
+            uint32_t it = 0, unit_it = 0;
             bool ok = true;
-            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, tile_it++) {
+            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, unit_it++) {
                 const int sp = u % g.splits;
-                const int k_beg = (int)((long)k_iters * sp / g.splits), k_end = (int)((long)k_iters * (sp + 1) / g.splits);
-                const int buf = tile_it % n_buf;
-                const uint32_t bph = (tile_it / n_buf) & 1;
+                const int ks_beg = (int)((long)k_stages * sp / g.splits), ks_end = (int)((long)k_stages * (sp + 1) / g.splits);
+                const int buf = unit_it % n_buf;
+                const uint32_t bph = (unit_it / n_buf) & 1;
                 if (!(ok = mbar_wait(&acc_empty[buf], bph ^ 1, giving_up, g.status))) break;
                 tc_fence_after();
                 const uint32_t d0 = tmem_base + (uint32_t)(buf * acc_cols);
-                for (int k = k_beg; k < k_end; k++, it++) {
+                int accum = 0;
+                for (int ks = ks_beg; ks < ks_end; ks++, it++) {
                     const int s = it % g.stages;
                     const uint32_t ph = (it / g.stages) & 1;
                     if (!(ok = mbar_wait(&full_bar[s], ph, giving_up, g.status))) break;
                     tc_fence_after();
                     const uint32_t a_addr = ring + (uint32_t)s * stage_bytes;
-                    const uint32_t b_addr = a_addr + g.n_acc * GM_A_BYTES;
+                    const uint32_t b_addr = a_addr + a_bytes;
+                    for (int j = 0; j < g.kb; j++) {
+                        if (ks * g.kb + j >= kb_total) break;  // a box's last k-block may lie outside K
 #pragma unroll
-                    for (int kk = 0; kk < GM_BK / 16; kk++) {
-                        const uint64_t db = umma_desc_sw128(b_addr + kk * 32);
-                        const int accum = (k > k_beg || kk > 0) ? 1 : 0;
-                        umma_bf16(d0, umma_desc_sw128(a_addr + kk * 32), db, idesc, accum);
-                        if (g.n_acc == 2) umma_bf16(d0 + mma_n, umma_desc_sw128(a_addr + GM_A_BYTES + kk * 32), db, idesc, accum);
+                        for (int kk = 0; kk < GM_BK / 16; kk++) {
+                            const uint64_t db = umma_desc_sw128(b_addr + j * b_blk + kk * 32);
+                            const uint32_t a0 = a_addr + j * a_blk_stride + kk * 32;
+                            umma_bf16(d0, umma_desc_sw128(a0), db, idesc, accum);
+                            umma_bf16(d0 + mma_n, umma_desc_sw128(a0 + a_acc_off), db, idesc, accum);
+                            accum = 1;
+                        }
                     }
                     umma_commit(&empty_bar[s]);  // the stage is free once these MMAs have read it
                 }
@@ -299,19 +336,12 @@ __global__ void __launch_bounds__(GM_THREADS, 1)
         tc.m_end = m_end;
         tc.acc_stride = mma_n;
         tc.xchg = xchg;
-        uint32_t tile_it = 0;
+        uint32_t unit_it = 0;
         bool ok = true;
-        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, tile_it++) {
-            const int t = u / g.splits;
-            tc.split = u % g.splits;
-            tc.matrix = 0;
-            tc.tile = t;
-            if (g.n_acc == 1) {
-                if (tc.tile >= g.tiles[0]) { tc.tile -= g.tiles[0]; tc.matrix = 1; }
-                if (tc.matrix == 1 && tc.tile >= g.tiles[1]) { tc.tile -= g.tiles[1]; tc.matrix = 2; }
-            }
-            const int buf = tile_it % n_buf;
-            const uint32_t bph = (tile_it / n_buf) & 1;
+        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, unit_it++) {
+            locate(u, tc.matrix, tc.unit_row, tc.split);
+            const int buf = unit_it % n_buf;
+            const uint32_t bph = (unit_it / n_buf) & 1;
             if (!(ok = mbar_wait(&acc_full[buf], bph, giving_up, g.status))) break;
             tc_fence_after();
             tc.taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * acc_cols);
@@ -331,53 +361,104 @@ __global__ void __launch_bounds__(GM_THREADS, 1)
 }
 
 // ------------------------------------------------------------------ endings
-// All endings walk the accumulator in chunks of 16 columns (activation rows); thread = weight row.
+// All endings walk an accumulator in chunks of 16 columns (activation rows); thread = weight row.
 
-// q/k/v: rotary embedding of q and k (pairs i, i + hd/2 sit hd/2 lanes apart, so values are
-// exchanged through shared memory), q to the query buffer, k and v appended to the cache.
+// q/k/v.  With the whole inner dimension in one unit: rotary embedding of q and k (pairs i,
+// i + hd/2 sit hd/2 lanes apart, so values are exchanged through shared memory), q to the query
+// buffer, k and v appended to the cache.  With the inner dimension cut across CTAs the partial
+// sums are added into an fp32 scratch [rows][Hq*hd + 2*Hkv*hd] and qkv_finish_kernel does the rest.
 struct QkvEnd {
     bf16 *q_out;         // [rows][Hq*hd]
     bf16 *kc, *vc;       // this layer's cache [slot][Hkv][S][hd]
     const float2 *rope;  // [S][hd/2]
     const int *row_slot, *row_pos;
+    float *partial;      // scratch for split sums, or NULL
     int Hq, Hkv, hd, S;
 
     __device__ void tile(const TileCtx &t) const
     {
         const int half = hd >> 1;
-        const int n = t.tile * GM_BM + t.row;  // row inside its matrix
         const int n_rows_mat = (t.matrix == 0 ? Hq : Hkv) * hd;
-        const int head = n / hd, i = n % hd, j = i & (half - 1);
-        const bool hi = i >= half;
-        for (int c0 = 0; t.m0 + c0 < t.m_end; c0 += GM_CHUNK) {
-            float v[GM_CHUNK];
-            tmem_ld16(t.taddr + c0, v);
-            if (t.matrix < 2) {
+        const int width = (Hq + 2 * Hkv) * hd;
+        const int col0 = t.matrix == 0 ? 0 : (t.matrix == 1 ? Hq * hd : (Hq + Hkv) * hd);
+        for (int a = 0; a < 2; a++) {
+            const int n = t.unit_row + a * GM_BM + t.row;  // row inside its matrix
+            const int head = n / hd, i = n % hd, j = i & (half - 1);
+            const bool hi = i >= half;
+            for (int c0 = 0; t.m0 + c0 < t.m_end; c0 += GM_CHUNK) {
+                float v[GM_CHUNK];
+                tmem_ld16(t.taddr + a * t.acc_stride + c0, v);
+                if (partial) {
+                    if (n < n_rows_mat) {
 #pragma unroll
-                for (int c = 0; c < GM_CHUNK; c++) t.xchg[c * GM_BM + t.row] = v[c];
-                epi_barrier();
-            }
-            if (n < n_rows_mat) {
+                        for (int c = 0; c < GM_CHUNK; c++) {
+                            const int m = t.m0 + c0 + c;
+                            if (m < t.m_end) atomicAdd(partial + (size_t)m * width + col0 + n, v[c]);
+                        }
+                    }
+                    continue;
+                }
+                if (t.matrix < 2) {
 #pragma unroll
-                for (int c = 0; c < GM_CHUNK; c++) {
-                    const int m = t.m0 + c0 + c;
-                    if (m >= t.m_end) break;
-                    const int slot = row_slot[m], pos = row_pos[m];
-                    if (t.matrix == 2) {
-                        vc[(((size_t)slot * Hkv + head) * S + pos) * hd + i] = __float2bfloat16(v[c]);
-                    } else {
-                        const float other = t.xchg[c * GM_BM + (t.row ^ half)];
-                        const float2 cs = rope[(size_t)pos * half + j];
-                        const float r = hi ? v[c] * cs.x + other * cs.y : v[c] * cs.x - other * cs.y;
-                        if (t.matrix == 0) q_out[(size_t)m * Hq * hd + n] = __float2bfloat16(r);
-                        else kc[(((size_t)slot * Hkv + head) * S + pos) * hd + i] = __float2bfloat16(r);
+                    for (int c = 0; c < GM_CHUNK; c++) t.xchg[c * GM_BM + t.row] = v[c];
+                    epi_barrier();
+                }
+                if (n < n_rows_mat) {
+#pragma unroll
+                    for (int c = 0; c < GM_CHUNK; c++) {
+                        const int m = t.m0 + c0 + c;
+                        if (m >= t.m_end) break;
+                        const int slot = row_slot[m], pos = row_pos[m];
+                        if (t.matrix == 2) {
+                            vc[(((size_t)slot * Hkv + head) * S + pos) * hd + i] = __float2bfloat16(v[c]);
+                        } else {
+                            const float other = t.xchg[c * GM_BM + (t.row ^ half)];
+                            const float2 cs = rope[(size_t)pos * half + j];
+                            const float r = hi ? v[c] * cs.x + other * cs.y : v[c] * cs.x - other * cs.y;
+                            if (t.matrix == 0) q_out[(size_t)m * Hq * hd + n] = __float2bfloat16(r);
+                            else kc[(((size_t)slot * Hkv + head) * S + pos) * hd + i] = __float2bfloat16(r);
+                        }
                     }
                 }
+                if (t.matrix < 2) epi_barrier();
             }
-            if (t.matrix < 2) epi_barrier();
         }
     }
 };
+
+// Finishes a q/k/v product whose inner dimension was cut across CTAs: reads the summed row from
+// the scratch, applies the rotary embedding, writes q and appends k, v to the cache, and clears
+// the scratch for the next product.  One block per activation row.
+static __global__ void __launch_bounds__(256) qkv_finish_kernel(float *__restrict__ partial, bf16 *__restrict__ q_out,
+                                                         bf16 *__restrict__ kc, bf16 *__restrict__ vc,
+                                                         const float2 *__restrict__ rope,
+                                                         const int *__restrict__ row_slot,
+                                                         const int *__restrict__ row_pos, int n_rows, int Hq, int Hkv,
+                                                         int hd, int S)
+{
+    griddep_wait();
+    griddep_launch();
+    const int m = blockIdx.x;
+    if (m >= n_rows) return;
+    const int half = hd >> 1, width = (Hq + 2 * Hkv) * hd;
+    float *src = partial + (size_t)m * width;
+    const int slot = row_slot[m], pos = row_pos[m];
+    // q and k heads: one thread per rotary pair
+    for (int p = threadIdx.x; p < (Hq + Hkv) * half; p += blockDim.x) {
+        const int head = p / half, j = p % half;
+        const float a = src[head * hd + j], b = src[head * hd + j + half];
+        const float2 cs = rope[(size_t)pos * half + j];
+        const float ra = a * cs.x - b * cs.y, rb = b * cs.x + a * cs.y;
+        bf16 *dst = head < Hq ? q_out + (size_t)m * Hq * hd + head * hd + j
+                              : kc + (((size_t)slot * Hkv + (head - Hq)) * S + pos) * hd + j;
+        dst[0] = __float2bfloat16(ra);
+        dst[half] = __float2bfloat16(rb);
+    }
+    for (int i = threadIdx.x; i < Hkv * hd; i += blockDim.x)
+        vc[(((size_t)slot * Hkv + i / hd) * S + pos) * hd + i % hd] = __float2bfloat16(src[(Hq + Hkv) * hd + i]);
+    __syncthreads();
+    for (int i = threadIdx.x; i < width; i += blockDim.x) src[i] = 0.f;
+}
 
 // h[m][n] += (W x_m)[n]; with the inner dimension cut across CTAs the partial sums meet in h.
 struct ResidEnd {
@@ -386,18 +467,20 @@ struct ResidEnd {
 
     __device__ void tile(const TileCtx &t) const
     {
-        const int n = t.tile * GM_BM + t.row;
-        for (int c0 = 0; t.m0 + c0 < t.m_end; c0 += GM_CHUNK) {
-            float v[GM_CHUNK];
-            tmem_ld16(t.taddr + c0, v);
-            if (n >= n_out) continue;
+        for (int a = 0; a < 2; a++) {
+            const int n = t.unit_row + a * GM_BM + t.row;
+            for (int c0 = 0; t.m0 + c0 < t.m_end; c0 += GM_CHUNK) {
+                float v[GM_CHUNK];
+                tmem_ld16(t.taddr + a * t.acc_stride + c0, v);
+                if (n >= n_out) continue;
 #pragma unroll
-            for (int c = 0; c < GM_CHUNK; c++) {
-                const int m = t.m0 + c0 + c;
-                if (m >= t.m_end) break;
-                float *dst = h + (size_t)m * n_out + n;
-                if (atomic) atomicAdd(dst, v[c]);
-                else *dst += v[c];
+                for (int c = 0; c < GM_CHUNK; c++) {
+                    const int m = t.m0 + c0 + c;
+                    if (m >= t.m_end) break;
+                    float *dst = h + (size_t)m * n_out + n;
+                    if (atomic) atomicAdd(dst, v[c]);
+                    else *dst += v[c];
+                }
             }
         }
     }
@@ -410,7 +493,7 @@ struct GateUpEnd {
 
     __device__ void tile(const TileCtx &t) const
     {
-        const int f = t.tile * GM_BM + t.row;
+        const int f = t.unit_row + t.row;
         for (int c0 = 0; t.m0 + c0 < t.m_end; c0 += GM_CHUNK) {
             float gt[GM_CHUNK], up[GM_CHUNK];
             tmem_ld16(t.taddr + c0, gt);
@@ -436,23 +519,25 @@ struct HeadEnd {
 
     __device__ void tile(const TileCtx &t) const
     {
-        const int id = lo + t.tile * GM_BM + t.row;
         const int lane = threadIdx.x & 31;
-        for (int c0 = 0; t.m0 + c0 < t.m_end; c0 += GM_CHUNK) {
-            float v[GM_CHUNK];
-            tmem_ld16(t.taddr + c0, v);
+        for (int a = 0; a < 2; a++) {
+            const int id = lo + t.unit_row + a * GM_BM + t.row;
+            for (int c0 = 0; t.m0 + c0 < t.m_end; c0 += GM_CHUNK) {
+                float v[GM_CHUNK];
+                tmem_ld16(t.taddr + a * t.acc_stride + c0, v);
 #pragma unroll
-            for (int c = 0; c < GM_CHUNK; c++) {
-                const int m = t.m0 + c0 + c;
-                if (m >= t.m_end) break;  // uniform across the warp
-                unsigned long long key = id < hi ? argmax_key(v[c], id) : 0ull;
-                if (logits && id < hi) logits[(size_t)seq_of_row[m] * V + id] = v[c];
+                for (int c = 0; c < GM_CHUNK; c++) {
+                    const int m = t.m0 + c0 + c;
+                    if (m >= t.m_end) break;  // uniform across the warp
+                    unsigned long long key = id < hi ? argmax_key(v[c], id) : 0ull;
+                    if (logits && id < hi) logits[(size_t)seq_of_row[m] * V + id] = v[c];
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                    const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
-                    key = other > key ? other : key;
+                    for (int o = 16; o > 0; o >>= 1) {
+                        const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
+                        key = other > key ? other : key;
+                    }
+                    if (lane == 0 && key) atomicMax(&argmax[seq_of_row[m]], key);
                 }
-                if (lane == 0 && key) atomicMax(&argmax[seq_of_row[m]], key);
             }
         }
     }

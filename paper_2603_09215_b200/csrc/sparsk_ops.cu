@@ -58,13 +58,11 @@ int sparsk_attention_launch(const sparsk_attn_args *p, char *scratch, cudaStream
     set_int_kernel<<<1, 1, 0, st>>>(counts, p->n_groups);
     set_int_kernel<<<1, 1, 0, st>>>(counts + 1, p->n_rows);
     const dim3 grid(p->n_groups * pl.n_qblk, p->n_kv_heads, pl.n_splits);
-    if (p->head_dim == 128) {
-        attn_partial_kernel<128><<<grid, AT_THREADS, 0, st>>>(a);
-        attn_merge_kernel<128><<<dim3(p->n_rows, p->n_q_heads), 128, 0, st>>>(a, counts + 1);
-    } else {
-        attn_partial_kernel<64><<<grid, AT_THREADS, 0, st>>>(a);
-        attn_merge_kernel<64><<<dim3(p->n_rows, p->n_q_heads), 64, 0, st>>>(a, counts + 1);
-    }
+    AttnPartialFn fn;
+    if (attn_partial_fn(p->head_dim, pl.mt, &fn) != cudaSuccess) return SPARSK_ECUDA;
+    fn<<<grid, AT_THREADS, attn_smem_bytes(p->head_dim, pl.mt), st>>>(a);
+    if (p->head_dim == 128) attn_merge_kernel<128><<<dim3(p->n_rows, p->n_q_heads), 128, 0, st>>>(a, counts + 1);
+    else attn_merge_kernel<64><<<dim3(p->n_rows, p->n_q_heads), 64, 0, st>>>(a, counts + 1);
     return cudaGetLastError() == cudaSuccess ? SPARSK_OK : SPARSK_ECUDA;
 }
 
