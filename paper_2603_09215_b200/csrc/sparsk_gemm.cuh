@@ -255,39 +255,45 @@ __global__ void __launch_bounds__(GM_THREADS, 1)
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
-        if (lane == 0) {
-            uint32_t it = 0;
-            bool ok = true;
-            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-                int mat, unit_row, sp;
-                locate(u, mat, unit_row, sp);
-                const CUtensorMap *ma = mat == 0 ? &map_a0 : (mat == 1 ? &map_a1 : &map_a2);
-                const int row = g.row0[mat] + unit_row;
-                const int ks_beg = (int)((long)k_stages * sp / g.splits), ks_end = (int)((long)k_stages * (sp + 1) / g.splits);
-                for (int ks = ks_beg; ks < ks_end; ks++, it++) {
-                    const int s = it % g.stages;
-                    const uint32_t ph = (it / g.stages) & 1;
-                    if (!(ok = mbar_wait(&empty_bar[s], ph ^ 1, giving_up, g.status))) break;
-                    const uint32_t st = ring + (uint32_t)s * stage_bytes;
-                    mbar_expect_tx(&full_bar[s], (uint32_t)stage_bytes);
-                    const int blk = ks * g.kb;
-                    if (g.three_d) {
-                        tma_load_3d(st, ma, &full_bar[s], 0, row, blk);
-                        if (g.pair) tma_load_3d(st + a_acc_off, &map_a1, &full_bar[s], 0, g.row0[1] + unit_row, blk);
-                        tma_load_3d(st + a_bytes, &map_b, &full_bar[s], 0, m0, blk);
-                    } else {
-                        tma_load_2d(st, ma, &full_bar[s], blk * GM_BK, row);
-                        if (g.pair) tma_load_2d(st + a_acc_off, &map_a1, &full_bar[s], blk * GM_BK, g.row0[1] + unit_row);
-                        tma_load_2d(st + a_bytes, &map_b, &full_bar[s], blk * GM_BK, m0);
-                    }
+        // One thread needs a few hundred nanoseconds per TMA copy (barrier handshake included), so
+        // the copies of a stage are issued by different lanes side by side: lane 0 waits for the
+        // slot and posts the byte count, then lanes 0..2 each issue one box.
+        uint32_t it = 0;
+        bool ok = true;
+        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+            int mat, unit_row, sp;
+            locate(u, mat, unit_row, sp);
+            const CUtensorMap *ma = mat == 0 ? &map_a0 : (mat == 1 ? &map_a1 : &map_a2);
+            const int row = g.row0[mat] + unit_row;
+            const int ks_beg = (int)((long)k_stages * sp / g.splits), ks_end = (int)((long)k_stages * (sp + 1) / g.splits);
+            for (int ks = ks_beg; ks < ks_end; ks++, it++) {
+                const int s = it % g.stages;
+                const uint32_t ph = (it / g.stages) & 1;
+                int go = 1;
+                if (lane == 0) {
+                    go = mbar_wait(&empty_bar[s], ph ^ 1, giving_up, g.status) ? 1 : 0;
+                    if (go) mbar_expect_tx(&full_bar[s], (uint32_t)stage_bytes);
+                }
+                go = __shfl_sync(0xffffffffu, go, 0);
+                if (!(ok = go != 0)) break;
+                const uint32_t st = ring + (uint32_t)s * stage_bytes;
+                const int blk = ks * g.kb;
+                // lane 0: accumulator 0's weights (or the whole 256-row box); lane 1: accumulator 1's
+                // weights when they come from matrix 1; lane 2: the activations
+                const CUtensorMap *mp = lane == 0 ? ma : (lane == 1 ? &map_a1 : &map_b);
+                const uint32_t dst = lane == 0 ? st : (lane == 1 ? st + a_acc_off : st + a_bytes);
+                const int y = lane == 0 ? row : (lane == 1 ? g.row0[1] + unit_row : m0);
+                if (lane == 0 || lane == 2 || (lane == 1 && g.pair)) {
+                    if (g.three_d) tma_load_3d(dst, mp, &full_bar[s], 0, y, blk);
+                    else tma_load_2d(dst, mp, &full_bar[s], blk * GM_BK, y);
                 }
             }
-            if (!ok) {
-                // giving up: let the copies already issued land (2 ms each at most) before the CTA
-                // goes away; stage s was last filled in round (it - 1 - s) / stages
-                for (int s = 0; s < g.stages; s++)
-                    if (it > (uint32_t)s) mbar_wait(&full_bar[s], ((it - 1 - s) / g.stages) & 1, &never_s, nullptr, 2000000ull);
-            }
+        }
+        if (!ok && lane == 0) {
+            // giving up: let the copies already issued land (2 ms each at most) before the CTA
+            // goes away; stage s was last filled in round (it - 1 - s) / stages
+            for (int s = 0; s < g.stages; s++)
+                if (it > (uint32_t)s) mbar_wait(&full_bar[s], ((it - 1 - s) / g.stages) & 1, &never_s, nullptr, 2000000ull);
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
