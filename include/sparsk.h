@@ -153,7 +153,9 @@ int sparsk_set_debug(sparsk_ctx *ctx, float *exit_hidden /*device or NULL*/,
                      float *exit_logits /*device or NULL*/);
 
 /* Tuning knobs, by name: "gemm_min_rows" (row count from which the tcgen05 path is used; a
- * large value keeps everything on the GEMV path), "gemm_kb" (1: one 64-element block of the inner
+ * large value keeps everything on the GEMV path), "mega" (0/1: run passes of one
+ * or two rows as one persistent kernel per layer range; default 1), "mega_l2_ahead" (how many
+ * 16 KB weight items that kernel requests from the L2 ahead of its copies; 0 = none), "gemm_kb" (1: one 64-element block of the inner
  * dimension per TMA copy instead of two; 0 = automatic), "use_graph" (0/1), "attn_split" (positions
  * per KV split), "pdl" (0/1, programmatic dependent launch between the kernels of a step),
  * "gemv_ks" / "gemv_r" (override the GEMV team width / rows per group; 0 = automatic),
@@ -205,7 +207,7 @@ int sparsk_attention_static(const sparsk_attn_args *args /*host*/, void *cuda_st
                             size_t err_len);
 
 /* Per-kernel timing for roofline reports.  sparsk_set_option(ctx, "time_kernel", c) with c =
- * 1 QKV, 2 attention, 3 O-projection, 4 gate/up, 5 down-projection, 6 exit head brackets every
+ * 1 QKV, 2 attention, 3 O-projection, 4 gate/up, 5 down-projection, 6 exit head, 7 persistent layer-range kernel brackets every
  * later launch of that class with CUDA events on the context's stream (up to 8192 launches; 0
  * stops).  sparsk_kernel_time synchronises the stream and returns the summed device time of the
  * bracketed launches and their number.  No counterpart in the paper: measurement only. */
@@ -216,6 +218,13 @@ int sparsk_kernel_time(sparsk_ctx *ctx, double *total_ms /*host*/, int64_t *n_la
  * if a token id had to be clamped into the vocabulary, else SPARSK_OK.  No counterpart in the
  * paper: error reporting only. */
 int sparsk_check(sparsk_ctx *ctx);
+
+/* Phase clock of the persistent layer-range kernel: its first CTA records the GPU's nanosecond
+ * timer when it starts and after each of the six phases of every layer (q/k/v, attention,
+ * merge, O-projection, gate/up, down-projection).  Copies the entries of the most recent launch
+ * to out_ns (host), synchronising the stream; returns how many were written (at most
+ * `capacity`), or a negative code.  No counterpart in the paper: measurement only. */
+int sparsk_phase_trace(sparsk_ctx *ctx, int64_t *out_ns /*host*/, int32_t capacity);
 
 /* Number of kernels this library has launched on behalf of the context so far. */
 int64_t sparsk_launch_count(const sparsk_ctx *ctx);

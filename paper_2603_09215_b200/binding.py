@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libsparsk.so")
 EXPORTS = ("sparsk_workspace_bytes", "sparsk_create", "sparsk_prefill", "sparsk_decode_step",
            "sparsk_decode_step_host", "sparsk_reset_slot", "sparsk_import_kv", "sparsk_export_kv",
            "sparsk_set_len", "sparsk_slot_state", "sparsk_set_debug", "sparsk_set_option",
-           "sparsk_kernel_time", "sparsk_check", "sparsk_attention", "sparsk_attention_scratch_bytes", "sparsk_attention_static", "sparsk_launch_count", "sparsk_last_error", "sparsk_destroy")
+           "sparsk_kernel_time", "sparsk_check", "sparsk_phase_trace", "sparsk_attention", "sparsk_attention_scratch_bytes", "sparsk_attention_static", "sparsk_launch_count", "sparsk_last_error", "sparsk_destroy")
 
 OK, EINVAL, ECAPACITY, ENOHEAD, ECUDA, ESTATE, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
 
@@ -98,6 +98,8 @@ def load():
     L.sparsk_attention.argtypes = [C.POINTER(AttnArgs), vp, C.c_size_t, vp]
     L.sparsk_attention_static.restype = C.c_int
     L.sparsk_attention_static.argtypes = [C.POINTER(AttnArgs), vp, C.c_char_p, C.c_size_t]
+    L.sparsk_phase_trace.restype = C.c_int
+    L.sparsk_phase_trace.argtypes = [vp, C.POINTER(C.c_int64), C.c_int32]
     L.sparsk_check.restype = C.c_int
     L.sparsk_check.argtypes = [vp]
     L.sparsk_launch_count.restype = C.c_int64
@@ -288,6 +290,15 @@ class Sparsk:
         ms, n = C.c_double(), C.c_int64()
         self._check(self.lib.sparsk_kernel_time(self.h, C.byref(ms), C.byref(n)))
         return ms.value, n.value
+
+    def phase_trace(self, capacity: int = 4096) -> np.ndarray:
+        """Nanosecond clock of the persistent kernel's first CTA at its start and after each phase
+        of the most recent launch."""
+        buf = np.zeros(capacity, np.int64)
+        n = self.lib.sparsk_phase_trace(self.h, buf.ctypes.data_as(C.POINTER(C.c_int64)), capacity)
+        if n < 0:
+            self._check(n)
+        return buf[:n]
 
     def check(self):
         """Synchronise, then raise if a kernel reported a problem through the device status word."""

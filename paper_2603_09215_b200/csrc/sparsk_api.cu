@@ -13,6 +13,7 @@
 #include "sparsk_common.cuh"
 #include "sparsk_gemm.cuh"
 #include "sparsk_gemv.cuh"
+#include "sparsk_mega.cuh"
 #include "sparsk_step.cuh"
 
 using namespace sparsk;
@@ -23,7 +24,7 @@ constexpr int MAX_SPLITS = AT_MAX_SPLITS;
 constexpr int STAGE_RING = 16;
 constexpr uint32_t CTX_MAGIC = 0x5350524bu;  // "SPRK"
 constexpr size_t TIME_POOL = 8192;           // event pairs available to the kernel timer
-enum { KC_MISC = 0, KC_QKV = 1, KC_ATTN = 2, KC_OPROJ = 3, KC_GATEUP = 4, KC_DOWN = 5, KC_HEAD = 6 };
+enum { KC_MISC = 0, KC_QKV = 1, KC_ATTN = 2, KC_OPROJ = 3, KC_GATEUP = 4, KC_DOWN = 5, KC_HEAD = 6, KC_MEGA = 7 };
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -81,6 +82,15 @@ struct sparsk_ctx {
     bool tc_ok;
     std::vector<TmaPair> tm_wq, tm_wk, tm_wv, tm_wo, tm_wg, tm_wu, tm_wd, tm_head;
     TmaPair tm_x[5], tm_ao[5], tm_act[5];
+    // persistent layer-range kernel (one or two rows)
+    MkLayer *mk_layers;            // device [L]
+    unsigned long long *mk_bar;    // device: grid barrier counter; mk_bar_base mirrors its value
+    int *mk_abort;                 // device
+    unsigned long long *mk_trace;  // device [1 + 6 L]
+    int mk_trace_n;                // entries the last launch wrote
+    unsigned long long mk_bar_base;
+    int mega, mk_ok, mk_coop, mk_l2_ahead;
+    std::vector<MkLayer> mk_host;
     float *qkv_part;  // fp32 sums of a q/k/v product whose inner dimension is cut across CTAs
     int tc_kb;        // 0: automatic; 1: force one k-block per copy (2-D descriptors)
     // optional per-kernel-class timing (events around every launch of one class)
@@ -163,14 +173,20 @@ size_t carve(sparsk_ctx *c, const sparsk_dims *d, char *base)
     bf16 *q = w.take<bf16>(R * qrow), *ao = w.take<bf16>(R * qrow), *act = w.take<bf16>(R * d->d_ffn);
     bf16 *xn = w.take<bf16>(R * d->d_model);
     float *qp = w.take<float>(R * (qrow + 2 * kvrow));
-    float *po = w.take<float>(R * d->n_q_heads * MAX_SPLITS * d->head_dim);
-    float2 *pml = w.take<float2>(R * d->n_q_heads * MAX_SPLITS);
+    MkLayer *mkl = w.take<MkLayer>(L);
+    unsigned long long *mkb = w.take<unsigned long long>(1);
+    int *mka = w.take<int>(1);
+    unsigned long long *mkt = w.take<unsigned long long>(1 + 6 * L);
+    const size_t cells = std::max<size_t>(R * MAX_SPLITS, (size_t)MK_MAX_ROWS * MK_MAX_SPLITS) * d->n_q_heads;
+    float *po = w.take<float>(cells * d->head_dim);
+    float2 *pml = w.take<float2>(cells);
     if (c) {
         c->kcache = kc; c->vcache = vc; c->pend_h = ph; c->kv_len = kl; c->pend_cnt = pc; c->rope = rope;
         c->sd = sd; c->staged = staged; c->tok_dev = tok; c->out_tok_dev = ot; c->out_depth_dev = od;
         c->pf_slot = pfs; c->pf_pos = pfp; c->pf_grp_row0 = pfg0; c->pf_grp_nrows = pfgn;
         c->pf_ngrp = pfng; c->pf_nrows = pfnr;
         c->h_lo = hlo; c->h_up = hup; c->qbuf = q; c->attn_o = ao; c->act = act; c->xnorm = xn; c->qkv_part = qp;
+        c->mk_layers = mkl; c->mk_bar = mkb; c->mk_abort = mka; c->mk_trace = mkt;
         c->part_o = po; c->part_ml = pml;
     }
     return align_up(w.off, 256);
@@ -587,6 +603,136 @@ cudaError_t run_head_tc(sparsk_ctx *c, int layer, const float *h, int list, int 
     return e;
 }
 
+
+// ---------------------------------------------------------------- persistent layer-range kernel
+bool build_mega(sparsk_ctx *c)
+{
+    const sparsk_dims &d = c->dm;
+    void *fp = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fp, cudaEnableDefault, &qr) != cudaSuccess || !fp ||
+        qr != cudaDriverEntryPointSuccess)
+        return false;
+    EncodeTiledFn fn = (EncodeTiledFn)fp;
+    const size_t qd = (size_t)d.n_q_heads * d.head_dim, kd = (size_t)d.n_kv_heads * d.head_dim;
+    const size_t lstride = (size_t)d.max_seqs * d.n_kv_heads * d.max_seq_len * d.head_dim;
+    // [16 rows][256 columns] boxes of a row-major matrix, no swizzle, zero fill outside
+    auto enc = [&](CUtensorMap *m, const void *base, size_t rows, size_t cols) {
+        const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+        const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+        const cuuint32_t box[2] = {(cuuint32_t)MK_BOX_COLS, (cuuint32_t)MK_BOX_ROWS};
+        const cuuint32_t es[2] = {1, 1};
+        return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, es,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    };
+    c->mk_host.resize(d.n_layers);
+    bool ok = true;
+    for (int l = 0; l < d.n_layers; l++) {
+        MkLayer &m = c->mk_host[l];
+        memset(&m, 0, sizeof m);
+        ok = ok && enc(&m.map_q, c->wq[l], qd, d.d_model) && enc(&m.map_k, c->wk[l], kd, d.d_model) &&
+             enc(&m.map_v, c->wv[l], kd, d.d_model) && enc(&m.map_o, c->wo[l], d.d_model, qd) &&
+             enc(&m.map_g, c->w_gate[l], d.d_ffn, d.d_model) && enc(&m.map_u, c->w_up[l], d.d_ffn, d.d_model) &&
+             enc(&m.map_d, c->w_down[l], d.d_model, d.d_ffn);
+        m.attn_gain = c->attn_norm[l];
+        m.mlp_gain = c->mlp_norm[l];
+        m.kc = c->kcache + l * lstride;
+        m.vc = c->vcache + l * lstride;
+    }
+    if (!ok) return false;
+    if (cudaMemcpyAsync(c->mk_layers, c->mk_host.data(), sizeof(MkLayer) * d.n_layers, cudaMemcpyHostToDevice,
+                        c->stream) != cudaSuccess ||
+        cudaMemsetAsync(c->mk_bar, 0, sizeof(unsigned long long), c->stream) != cudaSuccess ||
+        cudaMemsetAsync(c->mk_abort, 0, sizeof(int), c->stream) != cudaSuccess)
+        return false;
+    c->mk_bar_base = 0;
+    int dev = 0, coop = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess)
+        return false;
+    c->mk_coop = coop;
+    return true;
+}
+
+size_t mega_smem(const sparsk_dims &d)
+{
+    const int inner = std::max(std::max(d.d_model, d.d_ffn), d.n_q_heads * d.head_dim);
+    return (size_t)MK_SLOTS * MK_SLOT_BYTES + mk_area_bytes(inner, d.head_dim);
+}
+
+// Can a pass of n_rows rows go through the persistent kernel?
+bool use_mega(const sparsk_ctx *c, int n_rows)
+{
+    return c->mega && c->mk_ok && c->mk_coop && n_rows >= 1 && n_rows <= MK_MAX_ROWS &&
+           mega_smem(c->dm) + 2048 <= 227 * 1024 && c->dm.head_dim % (2 * MK_BOX_ROWS) == 0;
+}
+
+template <int M, int HD>
+cudaError_t launch_mega_inst(sparsk_ctx *c, const MkArgs &a, size_t smem)
+{
+    static int grid_ok = -1;
+    auto kern = mega_kernel<M, HD>;
+    if (grid_ok < 0) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        int per_sm = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, MK_THREADS, smem);
+        if (e != cudaSuccess) return e;
+        grid_ok = per_sm >= 1 ? 1 : 0;
+    }
+    if (!grid_ok) return cudaErrorCooperativeLaunchTooLarge;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(c->n_sm);
+    cfg.blockDim = dim3(MK_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = c->stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    c->launches++;
+    const bool timed = c->time_class == KC_MEGA && c->tev_used + 2 <= c->tev.size();
+    if (timed) cudaEventRecord(c->tev[c->tev_used++], c->stream);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, a);
+    if (timed) cudaEventRecord(c->tev[c->tev_used++], c->stream);
+    return e;
+}
+
+// Layers [l_begin, l_end) (0-based) over a row set of one or two rows, in one launch.
+cudaError_t run_mega(sparsk_ctx *c, int l_begin, int l_end, float *h, const RowSet &rs)
+{
+    const sparsk_dims &d = c->dm;
+    MkArgs a{};
+    a.layers = c->mk_layers; a.layer_begin = l_begin; a.layer_end = l_end; a.h = h;
+    a.row_slot = rs.slot; a.row_pos = rs.pos; a.grp_row0 = rs.grp_row0; a.grp_nrows = rs.grp_nrows;
+    a.n_rows = rs.n_rows; a.n_groups = rs.n_groups_h;
+    a.q_buf = c->qbuf; a.attn_o = c->attn_o; a.act = c->act; a.part_o = c->part_o; a.part_ml = c->part_ml;
+    a.rope = c->rope;
+    a.d = d.d_model; a.Hq = d.n_q_heads; a.Hkv = d.n_kv_heads; a.hd = d.head_dim; a.F = d.d_ffn; a.S = d.max_seq_len;
+    a.n_slots = d.max_seqs; a.eps = d.rms_eps;
+    // KV cut: an item for every attention warp of the machine if there are that many 16-position tiles
+    const int G = d.n_q_heads / d.n_kv_heads;
+    const int n_qblk = (rs.max_grp_rows * G + 15) / 16;
+    const int base = std::max(1, rs.n_groups_h * n_qblk * d.n_kv_heads);
+    const int tiles = std::max(1, (rs.max_len + AT_TP - 1) / AT_TP);
+    int splits = c->attn_split > 0 ? (rs.max_len + c->attn_split - 1) / c->attn_split
+                                   : (c->n_sm * MK_ATT_WARPS + base - 1) / base;
+    splits = std::max(1, std::min(splits, std::min(MK_MAX_SPLITS, tiles)));
+    a.att_split_len = ((rs.max_len + splits - 1) / splits + AT_TP - 1) / AT_TP * AT_TP;
+    a.att_splits = std::max(1, (rs.max_len + a.att_split_len - 1) / a.att_split_len);
+    a.l2_ahead = c->mk_l2_ahead;
+    a.bar = c->mk_bar; a.bar_base = c->mk_bar_base; a.abort_word = c->mk_abort; a.status = c->sd.counts + CNT_STATUS;
+    a.trace = c->mk_trace;
+    c->mk_trace_n = 1 + 6 * (l_end - l_begin);
+    c->mk_bar_base += 6ull * (unsigned long long)(l_end - l_begin) * (unsigned long long)c->n_sm;
+    const size_t smem = mega_smem(d);
+    if (d.head_dim == 128)
+        return rs.n_rows == 1 ? launch_mega_inst<1, 128>(c, a, smem) : launch_mega_inst<2, 128>(c, a, smem);
+    return rs.n_rows == 1 ? launch_mega_inst<1, 64>(c, a, smem) : launch_mega_inst<2, 64>(c, a, smem);
+}
+
 // One transformer layer over a row set: h <- h^(layer).
 cudaError_t run_layer(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
 {
@@ -606,6 +752,18 @@ cudaError_t run_layer(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
     e = run_resid(c, c->w_down[li], c->act, h, d.d_ffn, d.d_model, rs.n_rows);
     c->cur_class = KC_MISC;
     return e;
+}
+
+// Layers l_first..l_last (1-based, inclusive) over a row set.
+cudaError_t run_layers(sparsk_ctx *c, int l_first, int l_last, float *h, const RowSet &rs)
+{
+    if (l_first > l_last) return cudaSuccess;
+    if (use_mega(c, rs.n_rows)) return run_mega(c, l_first - 1, l_last, h, rs);
+    for (int l = l_first; l <= l_last; l++) {
+        const cudaError_t e = run_layer(c, l, h, rs);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
 }
 
 bool good(const sparsk_ctx *c) { return c && c->magic == CTX_MAGIC; }
@@ -665,6 +823,8 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
     ctx->pdl = 0; ctx->attn_split = 0; ctx->gemm_min_rows = 5; ctx->use_graph = 0;
     ctx->tc_ok = false;
     ctx->tc_kb = 0;
+    ctx->mega = 1; ctx->mk_ok = 0; ctx->mk_coop = 0; ctx->mk_bar_base = 0; ctx->mk_trace_n = 0;
+    ctx->mk_l2_ahead = MK_L2_AHEAD;
     ctx->gv_ks = 0; ctx->gv_r = 0; ctx->gv_grid_mult = 1;
     ctx->dbg_hidden = nullptr; ctx->dbg_logits = nullptr;
     ctx->launches = 0;
@@ -691,6 +851,11 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
         ctx->tc_ok = build_maps(ctx);
         if (!ctx->tc_ok) {
             rc = fail(ctx, SPARSK_ECUDA, "building the TMA descriptors failed");
+            break;
+        }
+        ctx->mk_ok = build_mega(ctx) ? 1 : 0;
+        if (!ctx->mk_ok) {
+            rc = fail(ctx, SPARSK_ECUDA, "setting up the persistent layer kernel failed");
             break;
         }
         // rotary table in double, stored as float (cos, sin)
@@ -755,9 +920,11 @@ extern "C" int sparsk_set_option(sparsk_ctx *ctx, const char *name, int64_t valu
     else if (!strcmp(name, "pdl") && (value == 0 || value == 1)) ctx->pdl = (int)value;
     else if (!strcmp(name, "attn_split") && value >= 0 && value <= (1 << 24)) ctx->attn_split = (int)value;
     else if (!strcmp(name, "gemv_ks") && (value == 0 || value == 1 || value == 2 || value == 4 || value == 8 || value == 16)) ctx->gv_ks = (int)value;
+    else if (!strcmp(name, "mega") && (value == 0 || value == 1)) ctx->mega = (int)value;
+    else if (!strcmp(name, "mega_l2_ahead") && value >= 0 && value <= 4096) ctx->mk_l2_ahead = (int)value;
     else if (!strcmp(name, "gemm_kb") && (value == 0 || value == 1)) ctx->tc_kb = (int)value;
     else if (!strcmp(name, "gemv_r") && (value == 0 || value == 1 || value == 2 || value == 4)) ctx->gv_r = (int)value;
-    else if (!strcmp(name, "time_kernel") && value >= 0 && value <= KC_HEAD) {
+    else if (!strcmp(name, "time_kernel") && value >= 0 && value <= KC_MEGA) {
         // start (or stop, with 0) timing every launch of one kernel class; resets the totals
         if (value && ctx->tev.empty()) {
             ctx->tev.resize(2 * TIME_POOL);
@@ -792,9 +959,25 @@ extern "C" int sparsk_check(sparsk_ctx *ctx)
     CU(cudaMemcpyAsync(&status, ctx->sd.counts + CNT_STATUS, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
     CU(cudaStreamSynchronize(ctx->stream));
     if (status) CU(cudaMemsetAsync(ctx->sd.counts + CNT_STATUS, 0, sizeof(int), ctx->stream));
-    if (status & ST_TIMEOUT) return fail(ctx, SPARSK_ETIMEOUT, "a bounded in-kernel wait ran out");
+    if (status & ST_TIMEOUT) {
+        // the persistent kernel's barrier counter and abort word start over
+        CU(cudaMemsetAsync(ctx->mk_bar, 0, sizeof(unsigned long long), ctx->stream));
+        CU(cudaMemsetAsync(ctx->mk_abort, 0, sizeof(int), ctx->stream));
+        ctx->mk_bar_base = 0;
+        return fail(ctx, SPARSK_ETIMEOUT, "a bounded in-kernel wait ran out");
+    }
     if (status & ST_BAD_TOKEN) return fail(ctx, SPARSK_EINVAL, "a token id was outside the vocabulary (clamped)");
     return SPARSK_OK;
+}
+
+extern "C" int sparsk_phase_trace(sparsk_ctx *ctx, int64_t *out_ns, int32_t capacity)
+{
+    if (!good(ctx)) return SPARSK_ESTATE;
+    if (!out_ns || capacity < 0) return fail(ctx, SPARSK_EINVAL, "phase_trace: bad arguments");
+    const int n = std::min<int>(capacity, ctx->mk_trace_n);
+    if (n > 0) CU(cudaMemcpyAsync(out_ns, ctx->mk_trace, sizeof(int64_t) * n, cudaMemcpyDeviceToHost, ctx->stream));
+    CU(cudaStreamSynchronize(ctx->stream));
+    return n;
 }
 
 extern "C" int sparsk_reset_slot(sparsk_ctx *ctx, int32_t slot) { return sparsk_set_len(ctx, slot, 0); }
@@ -880,7 +1063,7 @@ extern "C" int sparsk_prefill(sparsk_ctx *ctx, int32_t n_seqs, const int32_t *sl
                       d.vocab_text + d.vocab_speech, ctx->sd.counts + CNT_STATUS));
             RowSet rs{ctx->pf_slot, ctx->pf_pos, ctx->pf_grp_row0, ctx->pf_grp_nrows, ctx->pf_ngrp, ctx->pf_nrows,
                       n, 1, n, pos0 + n};
-            for (int l = 1; l <= d.n_layers; l++) CU(run_layer(ctx, l, ctx->h_up, rs));
+            CU(run_layers(ctx, 1, d.n_layers, ctx->h_up, rs));
             CU(launch(ctx, set_int_kernel, dim3(1), dim3(1), 0, ctx->kv_len + s, pos0 + n));
             ctx->h_len[s] = pos0 + n;
         }
@@ -954,7 +1137,7 @@ extern "C" int sparsk_decode_step(sparsk_ctx *ctx, int32_t n, const int32_t *slo
     // ---- lower pass: layers 1..e over all sequences
     RowSet lo{ctx->sd.slot, ctx->sd.lo_pos, ctx->sd.lo_grp_row0, ctx->sd.lo_grp_nrows, ctx->sd.counts + CNT_NSEQ,
               ctx->sd.counts + CNT_NSEQ, n, n, 1, max_len_lo};
-    for (int l = 1; l <= e; l++) CU(run_layer(ctx, l, ctx->h_lo, lo));
+    CU(run_layers(ctx, 1, e, ctx->h_lo, lo));
     // ---- early exits: keep h^(e), read the token from g_e
     if (n_list[0] + n_list[1]) {
         CU(launch(ctx, stash_kernel, dim3(n), dim3(128), 0, ctx->sd, (const float *)ctx->h_lo, ctx->pend_h,
@@ -969,7 +1152,7 @@ extern "C" int sparsk_decode_step(sparsk_ctx *ctx, int32_t n, const int32_t *slo
                   (const float *)ctx->pend_h, ctx->h_up, d.d_model, d.max_pending));
         RowSet up{ctx->sd.up_slot, ctx->sd.up_pos, ctx->sd.up_grp_row0, ctx->sd.up_grp_nrows, ctx->sd.counts + CNT_NGRP,
                   ctx->sd.counts + CNT_MUP, m_up, n_grp, max_grp, max_len_up};
-        for (int l = e + 1; l <= L; l++) CU(run_layer(ctx, l, ctx->h_up, up));
+        CU(run_layers(ctx, e + 1, L, ctx->h_up, up));
         h_full = ctx->h_up;
     }
     for (int l = 2; l < 4; l++)

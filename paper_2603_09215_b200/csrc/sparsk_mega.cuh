@@ -1,0 +1,208 @@
+// Persistent layer-range kernel for passes of one or two rows.
+//
+// At one or two rows a decode step is nothing but a stream of weights from HBM (Sec. IV-B.3),
+// and one kernel per projection leaves HBM idle at every kernel boundary.  This kernel runs a
+// whole range of layers in ONE cooperative launch, one CTA per SM:
+//
+//   * warps 16..19 are producers.  They walk the same list of phases as everyone else but only
+//     ever look at weights, which depend on nothing, so they keep TMA copies of [16 rows x 256
+//     columns] weight boxes flowing into an 8-slot shared-memory ring across phase and layer
+//     boundaries.  Producer p owns the ring slots p and p + 4 and cycles them on its own (one
+//     thread needs a few hundred nanoseconds per copy, so four run side by side); while its
+//     slots are busy it asks the L2 for the boxes further ahead, so HBM keeps streaming while
+//     the consumers sit in a barrier or in the attention phases.
+//   * warps 0..15 are consumers.  Per layer they run six phases separated by grid-wide barriers:
+//     RMSNorm + q/k/v + rotary embedding + cache append; attention partials; merge of the
+//     splits; O-projection + residual; RMSNorm + gate/up + SiLU; down-projection + residual.
+//     In a projection phase a CTA owns "bands" of 32 weight rows; warp w owns row w of each of
+//     the band's two 16-row boxes (a rotary pair, a gate/up pair, or two plain rows), reads one
+//     16-byte unit per lane per box, keeps fp32 sums across the whole inner dimension and
+//     shuffles once per band.  Activations sit in shared memory as bf16.
+//
+// Every wait (ring slot, grid barrier) is bounded by a wall-clock limit; on a timeout the CTA
+// raises ST_TIMEOUT, tells the other CTAs through the abort word, lets its copies land and
+// returns.
+#pragma once
+
+#include "sparsk_attn.cuh"
+#include "sparsk_gemm.cuh"
+
+namespace sparsk {
+
+constexpr int MK_CW = 16;                       // consumer warps
+constexpr int MK_PW = 4;                        // producer warps
+constexpr int MK_THREADS = (MK_CW + MK_PW) * 32;
+constexpr int MK_BOX_ROWS = 16, MK_BOX_COLS = 256;
+constexpr int MK_BOX_BYTES = MK_BOX_ROWS * MK_BOX_COLS * 2;  // 8 KB
+constexpr int MK_SLOT_BYTES = 2 * MK_BOX_BYTES;              // two boxes per slot
+constexpr int MK_SLOTS = 8;
+constexpr int MK_MAX_ROWS = 2;
+constexpr int MK_L2_AHEAD = 0;                  // items (16 KB each) a producer requests from L2 ahead of its copies;
+                                                // measured slower than none on B200 (gate/up 61 us against 44), so off
+constexpr int MK_ATT_WARPS = 4;                 // consumer warps that run attention items
+constexpr int MK_ATT_NST = 2;
+constexpr int MK_MAX_SPLITS = 16;
+
+// Shared memory behind the ring: activations of a projection phase, or the attention warps'
+// query blocks and K/V rings.
+inline size_t mk_area_bytes(int max_inner, int head_dim)
+{
+    const size_t act = (size_t)MK_MAX_ROWS * ((max_inner + MK_BOX_COLS - 1) / MK_BOX_COLS * MK_BOX_COLS) * 2;
+    const size_t att = (size_t)MK_ATT_WARPS * (16 + MK_ATT_NST * 2 * AT_TP) * (head_dim + 8) * 2;
+    return act > att ? act : att;
+}
+
+enum { MK_QKV = 0, MK_ATTN = 1, MK_MERGE = 2, MK_OPROJ = 3, MK_GATEUP = 4, MK_DOWN = 5 };
+
+// One layer's worth of what the phases need (device array, one entry per layer).
+struct MkLayer {
+    CUtensorMap map_q, map_k, map_v, map_o, map_g, map_u, map_d;  // [256 x 16] boxes, no swizzle
+    const bf16 *attn_gain, *mlp_gain;
+    bf16 *kc, *vc;  // this layer's cache [slot][Hkv][S][hd]
+};
+
+struct MkArgs {
+    const MkLayer *layers;       // device
+    int layer_begin, layer_end;  // 0-based, [begin, end)
+    float *h;                    // residual stream of the pass [rows][d]
+    const int *row_slot, *row_pos, *grp_row0, *grp_nrows;
+    int n_rows, n_groups;
+    bf16 *q_buf, *attn_o, *act;  // [rows][Hq*hd], [rows][Hq*hd], [rows][F]
+    float *part_o;
+    float2 *part_ml;
+    const float2 *rope;
+    int d, Hq, Hkv, hd, F, S, n_slots;
+    float eps;
+    int att_splits, att_split_len;  // KV cut of the attention phase
+    int l2_ahead;                   // 0 switches the L2 requests off
+    unsigned long long *bar;        // grid barrier counter (monotonic)
+    unsigned long long bar_base;    // its value when this launch starts
+    int *abort_word;                // nonzero: some CTA gave up
+    int *status;
+    unsigned long long *trace;      // [1 + 6 * layers]: CTA 0's clock at the start and after every phase
+};
+
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long *p)
+{
+    unsigned long long v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ int ld_volatile_i32(const int *p)
+{
+    int v;
+    asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap *map, int x, int y)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void mk_consumer_sync() { asm volatile("bar.sync 2, %0;" ::"n"(MK_CW * 32) : "memory"); }
+
+// Bands and k-steps of a projection phase.
+struct MkShape {
+    int n_bands, k_steps;
+};
+__device__ __forceinline__ MkShape mk_shape(int type, const MkArgs &a)
+{
+    MkShape s;
+    const int half = a.hd >> 1;
+    switch (type) {
+    case MK_QKV:
+        s.n_bands = (a.Hq + a.Hkv) * (half / MK_BOX_ROWS) + (a.Hkv * a.hd + 2 * MK_BOX_ROWS - 1) / (2 * MK_BOX_ROWS);
+        s.k_steps = (a.d + MK_BOX_COLS - 1) / MK_BOX_COLS;
+        break;
+    case MK_OPROJ:
+        s.n_bands = (a.d + 2 * MK_BOX_ROWS - 1) / (2 * MK_BOX_ROWS);
+        s.k_steps = (a.Hq * a.hd + MK_BOX_COLS - 1) / MK_BOX_COLS;
+        break;
+    case MK_GATEUP:
+        s.n_bands = (a.F + MK_BOX_ROWS - 1) / MK_BOX_ROWS;
+        s.k_steps = (a.d + MK_BOX_COLS - 1) / MK_BOX_COLS;
+        break;
+    case MK_DOWN:
+        s.n_bands = (a.d + 2 * MK_BOX_ROWS - 1) / (2 * MK_BOX_ROWS);
+        s.k_steps = (a.F + MK_BOX_COLS - 1) / MK_BOX_COLS;
+        break;
+    default:
+        s.n_bands = 0;
+        s.k_steps = 0;
+    }
+    return s;
+}
+// Descriptor and first row of the two boxes of band b.
+__device__ __forceinline__ void mk_band(int type, const MkArgs &a, const MkLayer *L, int b, const CUtensorMap *(&map)[2],
+                                        int (&row)[2])
+{
+    const int half = a.hd >> 1, per_head = half / MK_BOX_ROWS;
+    switch (type) {
+    case MK_QKV: {
+        const int nq = a.Hq * per_head, nk = a.Hkv * per_head;
+        if (b < nq + nk) {
+            const bool isq = b < nq;
+            const int bb = isq ? b : b - nq;
+            map[0] = map[1] = isq ? &L->map_q : &L->map_k;
+            row[0] = (bb / per_head) * a.hd + (bb % per_head) * MK_BOX_ROWS;
+            row[1] = row[0] + half;
+        } else {
+            map[0] = map[1] = &L->map_v;
+            row[0] = (b - nq - nk) * 2 * MK_BOX_ROWS;
+            row[1] = row[0] + MK_BOX_ROWS;
+        }
+        break;
+    }
+    case MK_GATEUP:
+        map[0] = &L->map_g;
+        map[1] = &L->map_u;
+        row[0] = row[1] = b * MK_BOX_ROWS;
+        break;
+    default:
+        map[0] = map[1] = type == MK_OPROJ ? &L->map_o : &L->map_d;
+        row[0] = b * 2 * MK_BOX_ROWS;
+        row[1] = row[0] + MK_BOX_ROWS;
+    }
+}
+
+struct MkShared {
+    uint64_t full[MK_SLOTS], empty[MK_SLOTS];
+    int giving_up, never;
+    float red[MK_CW];
+};
+
+// Consumers only: wait until every CTA has arrived at this barrier.
+__device__ __forceinline__ bool mk_grid_barrier(const MkArgs &a, MkShared *sh, unsigned long long &epoch)
+{
+    mk_consumer_sync();
+    epoch += gridDim.x;
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(a.bar, 1ull);
+        unsigned long long t0 = 0;
+        for (uint32_t spin = 0;; ++spin) {
+            if (ld_acquire_u64(a.bar) >= epoch) break;
+            if ((spin & 63u) == 63u) {
+                if (ld_volatile_i32(a.abort_word) || sh->giving_up) {
+                    sh->giving_up = 1;
+                    break;
+                }
+                const unsigned long long now = global_ns();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > GM_TIMEOUT_NS) {
+                    sh->giving_up = 1;
+                    atomicOr(a.status, ST_TIMEOUT);
+                    atomicExch(a.abort_word, 1);
+                    break;
+                }
+            }
+        }
+        __threadfence();
+        if (blockIdx.x == 0 && a.trace) a.trace[(epoch - a.bar_base) / gridDim.x] = global_ns();
+    }
+    mk_consumer_sync();
+    return *(volatile int *)&sh->giving_up == 0;
+}
+
+}  // namespace sparsk
+
+#include "sparsk_mega_phases.cuh"

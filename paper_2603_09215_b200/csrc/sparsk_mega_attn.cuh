@@ -1,0 +1,202 @@
+// Attention and split-merge phases of the persistent layer-range kernel (see sparsk_mega.cuh).
+#pragma once
+
+namespace sparsk {
+
+// Items (group, query block, kv head, split) are dealt to MK_ATT_WARPS warps of every CTA; a warp
+// runs its item alone: 16 query vectors (query heads of the kv head, for the group's rows), its
+// own two-stage K/V ring inside the activation area, one partial per item.  The arithmetic is
+// that of attn_partial_kernel with one m16 tile.
+template <int HD>
+__device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, unsigned char *area)
+{
+    constexpr int KP = HD + 8, CH = HD / 8;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (warp >= MK_ATT_WARPS) return;
+    // per warp: its 16 query vectors, then the K/V ring
+    bf16 *Qs = reinterpret_cast<bf16 *>(area) + (size_t)warp * (16 + MK_ATT_NST * 2 * AT_TP) * KP;
+    bf16 *wr = Qs + 16 * KP;
+    const int G = a.Hq / a.Hkv;
+    const int n_workers = gridDim.x * MK_ATT_WARPS, worker = warp * gridDim.x + blockIdx.x;
+    int max_nq = 0;
+    for (int g = 0; g < a.n_groups; g++) max_nq = max(max_nq, a.grp_nrows[g] * G);
+    const int n_qblk = (max_nq + 15) / 16;
+    const int n_items = a.n_groups * n_qblk * a.Hkv * a.att_splits;
+    const float scale = rsqrtf((float)HD);
+    for (int item = worker; item < n_items; item += n_workers) {
+        int t = item;
+        const int sp = t % a.att_splits; t /= a.att_splits;
+        const int hk = t % a.Hkv; t /= a.Hkv;
+        const int qb = t % n_qblk, g = t / n_qblk;
+        const int row0 = a.grp_row0[g], nrows = a.grp_nrows[g];
+        const int nq = nrows * G, q0 = qb * 16;
+        if (row0 < 0 || nrows < 1 || row0 + nrows > a.n_rows || q0 >= nq) continue;
+        const int nq_here = min(16, nq - q0);
+        const int slot = a.row_slot[row0], pos0 = a.row_pos[row0];
+        const bool sane = slot >= 0 && slot < a.n_slots && pos0 >= 0;
+        const int last_row = (q0 + nq_here - 1) / G;
+        const int kv_end_all = sane ? min(pos0 + last_row + 1, a.S) : 0;
+        const int w_beg = sp * a.att_split_len;
+        const int w_end = min(w_beg + a.att_split_len, kv_end_all);
+        const int n_tiles = w_end > w_beg ? (w_end - w_beg + AT_TP - 1) / AT_TP : 0;
+        const bf16 *kbase = L->kc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
+        const bf16 *vbase = L->vc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
+
+        __syncwarp();
+        for (int i = lane; i < 16 * CH; i += 32) {
+            const int qi = i / CH, c = i % CH;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (qi < nq_here) {
+                const int qg = q0 + qi, r = qg / G, j = qg % G;
+                v = *reinterpret_cast<const uint4 *>(a.q_buf + (size_t)(row0 + r) * a.Hq * HD + (hk * G + j) * HD + c * 8);
+            }
+            *reinterpret_cast<uint4 *>(&Qs[qi * KP + c * 8]) = v;
+        }
+        __syncwarp();
+
+        auto issue = [&](int tt) {
+            bf16 *kt = wr + (size_t)(tt % MK_ATT_NST) * 2 * AT_TP * KP, *vt = kt + AT_TP * KP;
+            const int p0 = w_beg + tt * AT_TP;
+#pragma unroll
+            for (int i = lane; i < AT_TP * CH; i += 32) {
+                const int r = i / CH, c = i % CH;
+                const bool ok = p0 + r < w_end;  // rows past the end are zero-filled
+                const size_t off = (size_t)(ok ? p0 + r : w_beg) * HD + c * 8;
+                cp_async16(&kt[r * KP + c * 8], kbase + off, ok ? 16 : 0);
+                cp_async16(&vt[r * KP + c * 8], vbase + off, ok ? 16 : 0);
+            }
+        };
+        float o[HD / 8][4], m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+#pragma unroll
+        for (int nt = 0; nt < HD / 8; nt++)
+#pragma unroll
+            for (int e = 0; e < 4; e++) o[nt][e] = 0.f;
+        int limit[2];
+#pragma unroll
+        for (int hf = 0; hf < 2; hf++) {
+            const int qi = (lane >> 2) + hf * 8;
+            limit[hf] = qi < nq_here ? pos0 + (q0 + qi) / G : -1;
+        }
+        if (n_tiles > 0) issue(0);
+        cp_async_commit();
+        for (int tt = 0; tt < n_tiles; tt++) {
+            if (tt + 1 < n_tiles) issue(tt + 1);
+            cp_async_commit();
+            cp_async_wait<1>();
+            __syncwarp();
+            const bf16 *Kt = wr + (size_t)(tt % MK_ATT_NST) * 2 * AT_TP * KP, *Vt = Kt + AT_TP * KP;
+            const int p0 = w_beg + tt * AT_TP;
+            float s[2][4];
+#pragma unroll
+            for (int nt = 0; nt < 2; nt++)
+#pragma unroll
+                for (int e = 0; e < 4; e++) s[nt][e] = 0.f;
+#pragma unroll
+            for (int ks = 0; ks < HD / 16; ks++) {
+                uint32_t kb[4], qa[4];
+                ldsm_x4(kb, &Kt[((lane & 7) + ((lane >> 4) << 3)) * KP + ks * 16 + ((lane >> 3) & 1) * 8]);
+                ldsm_x4(qa, &Qs[((lane & 7) + ((lane >> 3) & 1) * 8) * KP + ks * 16 + (lane >> 4) * 8]);
+                mma_bf16(s[0], qa, kb[0], kb[1]);
+                mma_bf16(s[1], qa, kb[2], kb[3]);
+            }
+            uint32_t pa[4];
+#pragma unroll
+            for (int hf = 0; hf < 2; hf++) {
+                float v[4];
+                float tmax = -INFINITY;
+#pragma unroll
+                for (int nt = 0; nt < 2; nt++)
+#pragma unroll
+                    for (int e = 0; e < 2; e++) {
+                        const int p = p0 + nt * 8 + (lane & 3) * 2 + e;
+                        const bool ok = p < w_end && p <= limit[hf];
+                        v[nt * 2 + e] = ok ? s[nt][hf * 2 + e] * scale : -INFINITY;
+                        tmax = fmaxf(tmax, v[nt * 2 + e]);
+                    }
+                tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
+                tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
+                const float m_new = fmaxf(m_run[hf], tmax);
+                float alpha = 1.f, psum = 0.f;
+                if (m_new != -INFINITY) {
+                    alpha = __expf(m_run[hf] - m_new);
+#pragma unroll
+                    for (int i = 0; i < 4; i++) {
+                        v[i] = __expf(v[i] - m_new);
+                        psum += v[i];
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 4; i++) v[i] = 0.f;
+                }
+                l_run[hf] = l_run[hf] * alpha + psum;
+                m_run[hf] = m_new;
+                pa[hf] = pack_bf16x2(v[0], v[1]);
+                pa[2 + hf] = pack_bf16x2(v[2], v[3]);
+#pragma unroll
+                for (int nt = 0; nt < HD / 8; nt++) {
+                    o[nt][hf * 2] *= alpha;
+                    o[nt][hf * 2 + 1] *= alpha;
+                }
+            }
+#pragma unroll
+            for (int np = 0; np < HD / 16; np++) {
+                uint32_t vb[4];
+                ldsm_x4_t(vb, &Vt[((lane & 7) + ((lane >> 3) & 1) * 8) * KP + np * 16 + (lane >> 4) * 8]);
+                mma_bf16(o[2 * np], pa, vb[0], vb[1]);
+                mma_bf16(o[2 * np + 1], pa, vb[2], vb[3]);
+            }
+            __syncwarp();  // the stage may be refilled by the next iteration's copies
+        }
+        cp_async_wait<0>();
+        // this item's partial
+#pragma unroll
+        for (int hf = 0; hf < 2; hf++) {
+            float l = l_run[hf];
+            l += __shfl_xor_sync(0xffffffffu, l, 1);
+            l += __shfl_xor_sync(0xffffffffu, l, 2);
+            const int qi = (lane >> 2) + hf * 8;
+            if (qi < nq_here) {
+                const int qg = q0 + qi, r = qg / G, j = qg % G;
+                const size_t cell = ((size_t)(row0 + r) * a.Hq + hk * G + j) * a.att_splits + sp;
+                if ((lane & 3) == 0) a.part_ml[cell] = make_float2(m_run[hf], l);
+#pragma unroll
+                for (int nt = 0; nt < HD / 8; nt++)
+                    *reinterpret_cast<float2 *>(a.part_o + cell * HD + nt * 8 + (lane & 3) * 2) =
+                        make_float2(o[nt][hf * 2], o[nt][hf * 2 + 1]);
+            }
+        }
+    }
+}
+
+// Merge of the splits: one warp per (row, query head); lane s holds split s's weight, lanes own
+// HD/32 output dims.  att_splits <= 32.
+template <int HD>
+__device__ __forceinline__ void mk_merge(const MkArgs &a)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr int DL = HD / 32;
+    const int n_items = a.n_rows * a.Hq;
+    for (int item = warp * gridDim.x + blockIdx.x; item < n_items; item += gridDim.x * MK_CW) {
+        const size_t cell0 = (size_t)item * a.att_splits;
+        float2 ml = make_float2(-INFINITY, 0.f);
+        if (lane < a.att_splits) ml = a.part_ml[cell0 + lane];
+        const float M = warp_max(ml.x);
+        const float w_mine = ml.x == -INFINITY ? 0.f : __expf(ml.x - M);
+        const float den = warp_sum(ml.y * w_mine);
+        float num[DL];
+#pragma unroll
+        for (int e = 0; e < DL; e++) num[e] = 0.f;
+#pragma unroll 4
+        for (int s = 0; s < a.att_splits; s++) {
+            const float w = __shfl_sync(0xffffffffu, w_mine, s);
+            const float *po = a.part_o + (cell0 + s) * HD + lane * DL;
+#pragma unroll
+            for (int e = 0; e < DL; e++) num[e] += po[e] * w;
+        }
+        bf16 *dst = a.attn_o + (size_t)item * HD + lane * DL;
+#pragma unroll
+        for (int e = 0; e < DL; e++) dst[e] = __float2bfloat16(den > 0.f ? num[e] / den : 0.f);
+    }
+}
+
+}  // namespace sparsk

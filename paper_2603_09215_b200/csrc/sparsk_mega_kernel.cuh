@@ -1,0 +1,156 @@
+// The persistent layer-range kernel itself (see sparsk_mega.cuh).
+#pragma once
+
+namespace sparsk {
+
+// Walks this CTA's ring items in consumption order: for every layer, for the four projection
+// phases, for every band the CTA owns, for every k-step.
+struct MkCursor {
+    int l, type, j, ks, my_bands, k_steps;
+    uint32_t idx;
+    bool done;
+
+    __device__ void settle(const MkArgs &a)
+    {
+        // move to the next phase that has bands for this CTA
+        for (;;) {
+            if (l >= a.layer_end) {
+                done = true;
+                return;
+            }
+            const MkShape shp = mk_shape(type, a);
+            my_bands = (int)blockIdx.x < shp.n_bands ? (shp.n_bands - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+            k_steps = shp.k_steps;
+            if (my_bands > 0 && k_steps > 0) return;
+            next_phase();
+        }
+    }
+    __device__ void next_phase()
+    {
+        type = type == MK_QKV ? MK_OPROJ : (type == MK_OPROJ ? MK_GATEUP : (type == MK_GATEUP ? MK_DOWN : MK_QKV));
+        if (type == MK_QKV) l++;
+        j = 0;
+        ks = 0;
+    }
+    __device__ void init(const MkArgs &a)
+    {
+        l = a.layer_begin;
+        type = MK_QKV;
+        j = ks = 0;
+        idx = 0;
+        done = false;
+        settle(a);
+    }
+    __device__ void advance(const MkArgs &a)
+    {
+        idx++;
+        if (++ks < k_steps) return;
+        ks = 0;
+        if (++j < my_bands) return;
+        next_phase();
+        settle(a);
+    }
+    __device__ int band() const { return (int)blockIdx.x + j * (int)gridDim.x; }
+};
+
+template <int M, int HD>
+__global__ void __launch_bounds__(MK_THREADS, 1) mega_kernel(const MkArgs a)
+{
+    extern __shared__ __align__(1024) unsigned char mk_smem[];
+    __shared__ MkShared sh;
+    unsigned char *ring = mk_smem;                                     // MK_SLOTS x 16 KB
+    unsigned char *area = mk_smem + (size_t)MK_SLOTS * MK_SLOT_BYTES;  // activations / attention rings
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < MK_SLOTS; s++) {
+            mbar_init(&sh.full[s], 1);
+            mbar_init(&sh.empty[s], MK_CW);
+        }
+        sh.giving_up = 0;
+        sh.never = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp >= MK_CW) {
+        // ------------------------------------------------------------ producers
+        const int p = warp - MK_CW;  // owns items p, p + 4, ... and with them ring slots p and p + 4
+        MkCursor ld, pf;
+        ld.init(a);
+        pf.init(a);
+        bool ok = true;
+        while (!ld.done && ok) {
+            // requests to the L2 for this producer's boxes up to l2_ahead items ahead
+            while (!pf.done && pf.idx < ld.idx + (uint32_t)a.l2_ahead) {
+                if ((int)(pf.idx % MK_PW) == p && lane < 2) {
+                    const CUtensorMap *map[2];
+                    int row[2];
+                    mk_band(pf.type, a, a.layers + pf.l, pf.band(), map, row);
+                    tma_prefetch_2d(map[lane], pf.ks * MK_BOX_COLS, row[lane]);
+                }
+                pf.advance(a);
+            }
+            if ((int)(ld.idx % MK_PW) == p) {
+                const int s = ld.idx % MK_SLOTS;
+                int go = 1;
+                if (lane == 0) {
+                    go = mbar_wait(&sh.empty[s], ((ld.idx / MK_SLOTS) & 1) ^ 1, &sh.giving_up, a.status) ? 1 : 0;
+                    if (go) mbar_expect_tx(&sh.full[s], MK_SLOT_BYTES);
+                }
+                go = __shfl_sync(0xffffffffu, go, 0);
+                if (!(ok = go != 0)) break;
+                if (lane < 2) {
+                    const CUtensorMap *map[2];
+                    int row[2];
+                    mk_band(ld.type, a, a.layers + ld.l, ld.band(), map, row);
+                    tma_load_2d(smem_u32(ring) + s * MK_SLOT_BYTES + lane * MK_BOX_BYTES, map[lane], &sh.full[s],
+                                ld.ks * MK_BOX_COLS, row[lane]);
+                }
+            }
+            ld.advance(a);
+        }
+        // never leave with copies in flight: every slot this producer filled must have landed
+        // (consumers that gave up no longer free slots, so wait on the full barriers, 2 ms each)
+        if (lane == 0) {
+            const uint32_t total = ld.idx;  // items before the point where this producer stopped
+            for (int s = p; s < MK_SLOTS; s += MK_PW)
+                if (total > (uint32_t)s) mbar_wait(&sh.full[s], ((total - 1 - s) / MK_SLOTS) & 1, &sh.never, nullptr, 2000000ull);
+        }
+    } else {
+        // ------------------------------------------------------------ consumers
+        uint32_t it = 0;
+        unsigned long long epoch = a.bar_base;
+        if (blockIdx.x == 0 && threadIdx.x == 0 && a.trace) a.trace[0] = global_ns();
+        bf16 *act = reinterpret_cast<bf16 *>(area);
+        bool ok = true;
+        const int qd = a.Hq * a.hd;
+        auto pad256 = [](int k) { return (k + MK_BOX_COLS - 1) / MK_BOX_COLS * MK_BOX_COLS; };
+        for (int l = a.layer_begin; l < a.layer_end && ok; l++) {
+            const MkLayer *L = a.layers + l;
+            // q/k/v
+            mk_load_act<M>(act, pad256(a.d), a.d, a.h, nullptr, L->attn_gain, a.eps, &sh);
+            if (!(ok = mk_project<M>(MK_QKV, a, L, act, pad256(a.d), ring, &sh, it))) break;
+            if (!(ok = mk_grid_barrier(a, &sh, epoch))) break;
+            // attention and the merge of its splits
+            mk_attention<HD>(a, L, area);
+            if (!(ok = mk_grid_barrier(a, &sh, epoch))) break;
+            mk_merge<HD>(a);
+            if (!(ok = mk_grid_barrier(a, &sh, epoch))) break;
+            // O-projection
+            mk_load_act<M>(act, pad256(qd), qd, nullptr, a.attn_o, nullptr, 0.f, &sh);
+            if (!(ok = mk_project<M>(MK_OPROJ, a, L, act, pad256(qd), ring, &sh, it))) break;
+            if (!(ok = mk_grid_barrier(a, &sh, epoch))) break;
+            // MLP
+            mk_load_act<M>(act, pad256(a.d), a.d, a.h, nullptr, L->mlp_gain, a.eps, &sh);
+            if (!(ok = mk_project<M>(MK_GATEUP, a, L, act, pad256(a.d), ring, &sh, it))) break;
+            if (!(ok = mk_grid_barrier(a, &sh, epoch))) break;
+            mk_load_act<M>(act, pad256(a.F), a.F, nullptr, a.act, nullptr, 0.f, &sh);
+            if (!(ok = mk_project<M>(MK_DOWN, a, L, act, pad256(a.F), ring, &sh, it))) break;
+            if (!(ok = mk_grid_barrier(a, &sh, epoch))) break;
+        }
+        if (!ok && threadIdx.x == 0) sh.giving_up = 1;
+    }
+    __syncthreads();
+}
+
+}  // namespace sparsk

@@ -1,0 +1,145 @@
+// Phases of the persistent layer-range kernel (see sparsk_mega.cuh) and the kernel itself.
+#pragma once
+
+namespace sparsk {
+
+// ------------------------------------------------------------------ activations -> shared memory
+// With h: x = h / sqrt(mean(h^2) + eps) * gain as bf16; otherwise a copy of bf16 rows.  Rows are
+// padded with zeros to a multiple of 256 columns (the last weight box is zero-filled there too).
+template <int M>
+__device__ __forceinline__ void mk_load_act(bf16 *act, int kpad, int K, const float *h, const bf16 *x, const bf16 *gain,
+                                            float eps, MkShared *sh)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int T = MK_CW * 32;
+#pragma unroll
+    for (int m = 0; m < M; m++) {
+        bf16 *dst = act + (size_t)m * kpad;
+        if (h) {
+            const float *src = h + (size_t)m * K;
+            float ss = 0.f;
+            for (int i = tid * 4; i < K; i += T * 4) {
+                const float4 v = *reinterpret_cast<const float4 *>(src + i);
+                ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+            }
+            ss = warp_sum(ss);
+            if (lane == 0) sh->red[warp] = ss;
+            mk_consumer_sync();
+            float tot = 0.f;
+#pragma unroll
+            for (int w = 0; w < MK_CW; w++) tot += sh->red[w];
+            mk_consumer_sync();
+            const float inv = rsqrtf(tot / (float)K + eps);
+            for (int i = tid * 8; i < kpad; i += T * 8) {
+                uint4 o = make_uint4(0, 0, 0, 0);
+                if (i < K) {
+                    const float4 p = *reinterpret_cast<const float4 *>(src + i);
+                    const float4 q = *reinterpret_cast<const float4 *>(src + i + 4);
+                    float g[8];
+                    unpack8(*reinterpret_cast<const uint4 *>(gain + i), g);
+                    o.x = pack_bf16x2(p.x * inv * g[0], p.y * inv * g[1]);
+                    o.y = pack_bf16x2(p.z * inv * g[2], p.w * inv * g[3]);
+                    o.z = pack_bf16x2(q.x * inv * g[4], q.y * inv * g[5]);
+                    o.w = pack_bf16x2(q.z * inv * g[6], q.w * inv * g[7]);
+                }
+                *reinterpret_cast<uint4 *>(dst + i) = o;
+            }
+        } else {
+            const bf16 *src = x + (size_t)m * K;
+            for (int i = tid * 8; i < kpad; i += T * 8)
+                *reinterpret_cast<uint4 *>(dst + i) = i < K ? *reinterpret_cast<const uint4 *>(src + i) : make_uint4(0, 0, 0, 0);
+        }
+    }
+    mk_consumer_sync();
+}
+
+// ------------------------------------------------------------------ projection phase (consumers)
+template <int M>
+__device__ __forceinline__ bool mk_project(int type, const MkArgs &a, const MkLayer *L, const bf16 *act, int kpad,
+                                           unsigned char *ring, MkShared *sh, uint32_t &it)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const MkShape shp = mk_shape(type, a);
+    const int half = a.hd >> 1, per_head = half / MK_BOX_ROWS;
+    for (int b = blockIdx.x; b < shp.n_bands; b += gridDim.x) {
+        float acc[2][M];
+#pragma unroll
+        for (int r = 0; r < 2; r++)
+#pragma unroll
+            for (int m = 0; m < M; m++) acc[r][m] = 0.f;
+        for (int ks = 0; ks < shp.k_steps; ks++, it++) {
+            const int s = it % MK_SLOTS;
+            if (!mbar_wait(&sh->full[s], (it / MK_SLOTS) & 1, &sh->giving_up, a.status)) return false;
+            const unsigned char *slot = ring + (size_t)s * MK_SLOT_BYTES + (size_t)warp * MK_BOX_COLS * 2 + lane * 16;
+            float w0[8], w1[8];
+            unpack8(*reinterpret_cast<const uint4 *>(slot), w0);
+            unpack8(*reinterpret_cast<const uint4 *>(slot + MK_BOX_BYTES), w1);
+#pragma unroll
+            for (int m = 0; m < M; m++) {
+                float x[8];
+                unpack8(*reinterpret_cast<const uint4 *>(act + (size_t)m * kpad + ks * MK_BOX_COLS + lane * 8), x);
+#pragma unroll
+                for (int j = 0; j < 8; j++) {
+                    acc[0][m] = fmaf(w0[j], x[j], acc[0][m]);
+                    acc[1][m] = fmaf(w1[j], x[j], acc[1][m]);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh->empty[s]);
+        }
+#pragma unroll
+        for (int r = 0; r < 2; r++)
+#pragma unroll
+            for (int m = 0; m < M; m++) acc[r][m] = warp_sum(acc[r][m]);
+        // lane m finishes activation row m
+        float v0 = acc[0][0], v1 = acc[1][0];
+#pragma unroll
+        for (int m = 1; m < M; m++)
+            if (lane == m) {
+                v0 = acc[0][m];
+                v1 = acc[1][m];
+            }
+        if (lane < M) {
+            const int m = lane;
+            switch (type) {
+            case MK_QKV: {
+                const int nq = a.Hq * per_head, nk = a.Hkv * per_head;
+                const int slot_id = a.row_slot[m], pos = a.row_pos[m];
+                if (b < nq + nk) {
+                    const bool isq = b < nq;
+                    const int bb = isq ? b : b - nq;
+                    const int head = bb / per_head, i = (bb % per_head) * MK_BOX_ROWS + warp;
+                    const float2 cs = a.rope[(size_t)pos * half + i];
+                    const float ra = v0 * cs.x - v1 * cs.y, rb = v1 * cs.x + v0 * cs.y;
+                    bf16 *dst = isq ? a.q_buf + (size_t)m * a.Hq * a.hd + head * a.hd + i
+                                    : L->kc + (((size_t)slot_id * a.Hkv + head) * a.S + pos) * a.hd + i;
+                    dst[0] = __float2bfloat16(ra);
+                    dst[half] = __float2bfloat16(rb);
+                } else {
+                    const int n0 = (b - nq - nk) * 2 * MK_BOX_ROWS + warp, n1 = n0 + MK_BOX_ROWS;
+                    const int kvd = a.Hkv * a.hd;
+                    if (n0 < kvd) L->vc[(((size_t)slot_id * a.Hkv + n0 / a.hd) * a.S + pos) * a.hd + n0 % a.hd] = __float2bfloat16(v0);
+                    if (n1 < kvd) L->vc[(((size_t)slot_id * a.Hkv + n1 / a.hd) * a.S + pos) * a.hd + n1 % a.hd] = __float2bfloat16(v1);
+                }
+                break;
+            }
+            case MK_GATEUP: {
+                const int f = b * MK_BOX_ROWS + warp;
+                if (f < a.F) a.act[(size_t)m * a.F + f] = __float2bfloat16(v0 / (1.f + __expf(-v0)) * v1);
+                break;
+            }
+            default: {
+                const int n0 = b * 2 * MK_BOX_ROWS + warp, n1 = n0 + MK_BOX_ROWS;
+                if (n0 < a.d) a.h[(size_t)m * a.d + n0] += v0;
+                if (n1 < a.d) a.h[(size_t)m * a.d + n1] += v1;
+            }
+            }
+        }
+    }
+    return true;
+}
+
+}  // namespace sparsk
+
+#include "sparsk_mega_attn.cuh"
+#include "sparsk_mega_kernel.cuh"
