@@ -164,6 +164,48 @@ __device__ __forceinline__ void mk_band(int type, const MkArgs &a, const MkLayer
     }
 }
 
+// This CTA's share of a projection phase, as segments (band, k-steps [ks0, ks1)).  q/k/v and
+// gate/up deal whole bands round-robin (144 and F/16 bands fill 148 SMs well).  The two residual
+// projections have d/32 bands, fewer than there are SMs, and an additive ending, so their
+// (band, k-step) pairs are laid end to end and cut into equal contiguous shares; a share that
+// ends inside a band adds its partial sums into the residual stream with atomics.
+struct MkSeg {
+    int band, ks0, ks1;
+};
+struct MkWalk {
+    int k_steps, n_bands, j;
+    bool stream;
+    long pos, hi;
+    __device__ void init(int type, const MkArgs &a)
+    {
+        const MkShape shp = mk_shape(type, a);
+        k_steps = shp.k_steps;
+        n_bands = shp.n_bands;
+        stream = type == MK_OPROJ || type == MK_DOWN;
+        j = blockIdx.x;
+        const long T = (long)n_bands * k_steps;
+        pos = (long)blockIdx.x * T / gridDim.x;
+        hi = (long)(blockIdx.x + 1) * T / gridDim.x;
+    }
+    __device__ bool next(MkSeg &s)
+    {
+        if (stream) {
+            if (pos >= hi) return false;
+            s.band = (int)(pos / k_steps);
+            s.ks0 = (int)(pos % k_steps);
+            s.ks1 = (int)min((long)k_steps, s.ks0 + (hi - pos));
+            pos += s.ks1 - s.ks0;
+            return true;
+        }
+        if (j >= n_bands || k_steps < 1) return false;
+        s.band = j;
+        s.ks0 = 0;
+        s.ks1 = k_steps;
+        j += gridDim.x;
+        return true;
+    }
+};
+
 struct MkShared {
     uint64_t full[MK_SLOTS], empty[MK_SLOTS];
     int giving_up, never;

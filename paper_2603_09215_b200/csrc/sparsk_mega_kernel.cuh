@@ -4,24 +4,27 @@
 namespace sparsk {
 
 // Walks this CTA's ring items in consumption order: for every layer, for the four projection
-// phases, for every band the CTA owns, for every k-step.
+// phases, for every segment the CTA owns, for every k-step.
 struct MkCursor {
-    int l, type, j, ks, my_bands, k_steps;
+    int l, type, ks;
+    MkWalk walk;
+    MkSeg seg;
     uint32_t idx;
     bool done;
 
     __device__ void settle(const MkArgs &a)
     {
-        // move to the next phase that has bands for this CTA
+        // move to the next phase that has work for this CTA
         for (;;) {
             if (l >= a.layer_end) {
                 done = true;
                 return;
             }
-            const MkShape shp = mk_shape(type, a);
-            my_bands = (int)blockIdx.x < shp.n_bands ? (shp.n_bands - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
-            k_steps = shp.k_steps;
-            if (my_bands > 0 && k_steps > 0) return;
+            walk.init(type, a);
+            if (walk.next(seg)) {
+                ks = seg.ks0;
+                return;
+            }
             next_phase();
         }
     }
@@ -29,14 +32,11 @@ struct MkCursor {
     {
         type = type == MK_QKV ? MK_OPROJ : (type == MK_OPROJ ? MK_GATEUP : (type == MK_GATEUP ? MK_DOWN : MK_QKV));
         if (type == MK_QKV) l++;
-        j = 0;
-        ks = 0;
     }
     __device__ void init(const MkArgs &a)
     {
         l = a.layer_begin;
         type = MK_QKV;
-        j = ks = 0;
         idx = 0;
         done = false;
         settle(a);
@@ -44,13 +44,15 @@ struct MkCursor {
     __device__ void advance(const MkArgs &a)
     {
         idx++;
-        if (++ks < k_steps) return;
-        ks = 0;
-        if (++j < my_bands) return;
+        if (++ks < seg.ks1) return;
+        if (walk.next(seg)) {
+            ks = seg.ks0;
+            return;
+        }
         next_phase();
         settle(a);
     }
-    __device__ int band() const { return (int)blockIdx.x + j * (int)gridDim.x; }
+    __device__ int band() const { return seg.band; }
 };
 
 template <int M, int HD>

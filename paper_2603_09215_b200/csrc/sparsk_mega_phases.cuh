@@ -59,15 +59,18 @@ __device__ __forceinline__ bool mk_project(int type, const MkArgs &a, const MkLa
                                            unsigned char *ring, MkShared *sh, uint32_t &it)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const MkShape shp = mk_shape(type, a);
     const int half = a.hd >> 1, per_head = half / MK_BOX_ROWS;
-    for (int b = blockIdx.x; b < shp.n_bands; b += gridDim.x) {
+    MkWalk walk;
+    walk.init(type, a);
+    MkSeg seg;
+    while (walk.next(seg)) {
+        const int b = seg.band;
         float acc[2][M];
 #pragma unroll
         for (int r = 0; r < 2; r++)
 #pragma unroll
             for (int m = 0; m < M; m++) acc[r][m] = 0.f;
-        for (int ks = 0; ks < shp.k_steps; ks++, it++) {
+        for (int ks = seg.ks0; ks < seg.ks1; ks++, it++) {
             const int s = it % MK_SLOTS;
             if (!mbar_wait(&sh->full[s], (it / MK_SLOTS) & 1, &sh->giving_up, a.status)) return false;
             const unsigned char *slot = ring + (size_t)s * MK_SLOT_BYTES + (size_t)warp * MK_BOX_COLS * 2 + lane * 16;
@@ -130,8 +133,9 @@ __device__ __forceinline__ bool mk_project(int type, const MkArgs &a, const MkLa
             }
             default: {
                 const int n0 = b * 2 * MK_BOX_ROWS + warp, n1 = n0 + MK_BOX_ROWS;
-                if (n0 < a.d) a.h[(size_t)m * a.d + n0] += v0;
-                if (n1 < a.d) a.h[(size_t)m * a.d + n1] += v1;
+                // shares of a band held by different CTAs meet in the residual stream
+                if (n0 < a.d) atomicAdd(a.h + (size_t)m * a.d + n0, v0);
+                if (n1 < a.d) atomicAdd(a.h + (size_t)m * a.d + n1, v1);
             }
             }
         }
