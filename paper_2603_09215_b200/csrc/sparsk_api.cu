@@ -89,7 +89,7 @@ struct sparsk_ctx {
     unsigned long long *mk_trace;  // device [1 + 6 L]
     int mk_trace_n;                // entries the last launch wrote
     unsigned long long mk_bar_base;
-    int mega, mk_ok, mk_coop, mk_l2_ahead;
+    int mega, mk_ok, mk_coop;
     std::vector<MkLayer> mk_host;
     float *qkv_part;  // fp32 sums of a q/k/v product whose inner dimension is cut across CTAs
     int tc_kb;        // 0: automatic; 1: force one k-block per copy (2-D descriptors)
@@ -722,7 +722,6 @@ cudaError_t run_mega(sparsk_ctx *c, int l_begin, int l_end, float *h, const RowS
     splits = std::max(1, std::min(splits, std::min(MK_MAX_SPLITS, tiles)));
     a.att_split_len = ((rs.max_len + splits - 1) / splits + AT_TP - 1) / AT_TP * AT_TP;
     a.att_splits = std::max(1, (rs.max_len + a.att_split_len - 1) / a.att_split_len);
-    a.l2_ahead = c->mk_l2_ahead;
     a.bar = c->mk_bar; a.bar_base = c->mk_bar_base; a.abort_word = c->mk_abort; a.status = c->sd.counts + CNT_STATUS;
     a.trace = c->mk_trace;
     c->mk_trace_n = 1 + 6 * (l_end - l_begin);
@@ -824,7 +823,6 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
     ctx->tc_ok = false;
     ctx->tc_kb = 0;
     ctx->mega = 1; ctx->mk_ok = 0; ctx->mk_coop = 0; ctx->mk_bar_base = 0; ctx->mk_trace_n = 0;
-    ctx->mk_l2_ahead = MK_L2_AHEAD;
     ctx->gv_ks = 0; ctx->gv_r = 0; ctx->gv_grid_mult = 1;
     ctx->dbg_hidden = nullptr; ctx->dbg_logits = nullptr;
     ctx->launches = 0;
@@ -921,7 +919,6 @@ extern "C" int sparsk_set_option(sparsk_ctx *ctx, const char *name, int64_t valu
     else if (!strcmp(name, "attn_split") && value >= 0 && value <= (1 << 24)) ctx->attn_split = (int)value;
     else if (!strcmp(name, "gemv_ks") && (value == 0 || value == 1 || value == 2 || value == 4 || value == 8 || value == 16)) ctx->gv_ks = (int)value;
     else if (!strcmp(name, "mega") && (value == 0 || value == 1)) ctx->mega = (int)value;
-    else if (!strcmp(name, "mega_l2_ahead") && value >= 0 && value <= 4096) ctx->mk_l2_ahead = (int)value;
     else if (!strcmp(name, "gemm_kb") && (value == 0 || value == 1)) ctx->tc_kb = (int)value;
     else if (!strcmp(name, "gemv_r") && (value == 0 || value == 1 || value == 2 || value == 4)) ctx->gv_r = (int)value;
     else if (!strcmp(name, "time_kernel") && value >= 0 && value <= KC_MEGA) {

@@ -8,9 +8,10 @@
 //     ever look at weights, which depend on nothing, so they keep TMA copies of [16 rows x 256
 //     columns] weight boxes flowing into an 8-slot shared-memory ring across phase and layer
 //     boundaries.  Producer p owns the ring slots p and p + 4 and cycles them on its own (one
-//     thread needs a few hundred nanoseconds per copy, so four run side by side); while its
-//     slots are busy it asks the L2 for the boxes further ahead, so HBM keeps streaming while
-//     the consumers sit in a barrier or in the attention phases.
+//     thread needs a few hundred nanoseconds per copy, so four run side by side).  The ring is
+//     what keeps HBM streaming while the consumers sit in a barrier or in the attention phases.
+//     (Asking the L2 for boxes further ahead, with tensor or bulk prefetches, from the producers
+//     or from a warp of its own, was measured and made every phase slower, gate/up by 30-80 %.)
 //   * warps 0..15 are consumers.  Per layer they run six phases separated by grid-wide barriers:
 //     RMSNorm + q/k/v + rotary embedding + cache append; attention partials; merge of the
 //     splits; O-projection + residual; RMSNorm + gate/up + SiLU; down-projection + residual.
@@ -37,8 +38,6 @@ constexpr int MK_BOX_BYTES = MK_BOX_ROWS * MK_BOX_COLS * 2;  // 8 KB
 constexpr int MK_SLOT_BYTES = 2 * MK_BOX_BYTES;              // two boxes per slot
 constexpr int MK_SLOTS = 8;
 constexpr int MK_MAX_ROWS = 2;
-constexpr int MK_L2_AHEAD = 0;                  // items (16 KB each) a producer requests from L2 ahead of its copies;
-                                                // measured slower than none on B200 (gate/up 61 us against 44), so off
 constexpr int MK_ATT_WARPS = 4;                 // consumer warps that run attention items
 constexpr int MK_ATT_NST = 2;
 constexpr int MK_MAX_SPLITS = 16;
@@ -74,7 +73,6 @@ struct MkArgs {
     int d, Hq, Hkv, hd, F, S, n_slots;
     float eps;
     int att_splits, att_split_len;  // KV cut of the attention phase
-    int l2_ahead;                   // 0 switches the L2 requests off
     unsigned long long *bar;        // grid barrier counter (monotonic)
     unsigned long long bar_base;    // its value when this launch starts
     int *abort_word;                // nonzero: some CTA gave up
@@ -93,10 +91,6 @@ __device__ __forceinline__ int ld_volatile_i32(const int *p)
     int v;
     asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
-}
-__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap *map, int x, int y)
-{
-    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(x), "r"(y) : "memory");
 }
 __device__ __forceinline__ void mk_consumer_sync() { asm volatile("bar.sync 2, %0;" ::"n"(MK_CW * 32) : "memory"); }
 

@@ -77,21 +77,10 @@ __global__ void __launch_bounds__(MK_THREADS, 1) mega_kernel(const MkArgs a)
     if (warp >= MK_CW) {
         // ------------------------------------------------------------ producers
         const int p = warp - MK_CW;  // owns items p, p + 4, ... and with them ring slots p and p + 4
-        MkCursor ld, pf;
+        MkCursor ld;
         ld.init(a);
-        pf.init(a);
         bool ok = true;
         while (!ld.done && ok) {
-            // requests to the L2 for this producer's boxes up to l2_ahead items ahead
-            while (!pf.done && pf.idx < ld.idx + (uint32_t)a.l2_ahead) {
-                if ((int)(pf.idx % MK_PW) == p && lane < 2) {
-                    const CUtensorMap *map[2];
-                    int row[2];
-                    mk_band(pf.type, a, a.layers + pf.l, pf.band(), map, row);
-                    tma_prefetch_2d(map[lane], pf.ks * MK_BOX_COLS, row[lane]);
-                }
-                pf.advance(a);
-            }
             if ((int)(ld.idx % MK_PW) == p) {
                 const int s = ld.idx % MK_SLOTS;
                 int go = 1;
