@@ -654,17 +654,13 @@ bool build_mega(sparsk_ctx *c)
     return true;
 }
 
-size_t mega_smem(const sparsk_dims &d)
-{
-    const int inner = std::max(std::max(d.d_model, d.d_ffn), d.n_q_heads * d.head_dim);
-    return (size_t)MK_SLOTS * MK_SLOT_BYTES + mk_area_bytes(inner, d.head_dim);
-}
+size_t mega_smem(const sparsk_dims &) { return (size_t)MK_SLOTS * MK_SLOT_BYTES + MK_AREA_BYTES; }
 
 // Can a pass of n_rows rows go through the persistent kernel?
 bool use_mega(const sparsk_ctx *c, int n_rows)
 {
     return c->mega && c->mk_ok && c->mk_coop && n_rows >= 1 && n_rows <= MK_MAX_ROWS &&
-           mega_smem(c->dm) + 2048 <= 227 * 1024 && c->dm.head_dim % (2 * MK_BOX_ROWS) == 0;
+           mk_attn_bytes(c->dm.head_dim) <= MK_AREA_BYTES && c->dm.head_dim % (2 * MK_BOX_ROWS) == 0;
 }
 
 template <int M, int HD>
@@ -727,9 +723,20 @@ cudaError_t run_mega(sparsk_ctx *c, int l_begin, int l_end, float *h, const RowS
     c->mk_trace_n = 1 + 6 * (l_end - l_begin);
     c->mk_bar_base += 6ull * (unsigned long long)(l_end - l_begin) * (unsigned long long)c->n_sm;
     const size_t smem = mega_smem(d);
-    if (d.head_dim == 128)
-        return rs.n_rows == 1 ? launch_mega_inst<1, 128>(c, a, smem) : launch_mega_inst<2, 128>(c, a, smem);
-    return rs.n_rows == 1 ? launch_mega_inst<1, 64>(c, a, smem) : launch_mega_inst<2, 64>(c, a, smem);
+    if (d.head_dim == 128) {
+        switch (rs.n_rows) {
+        case 1: return launch_mega_inst<1, 128>(c, a, smem);
+        case 2: return launch_mega_inst<2, 128>(c, a, smem);
+        case 3: return launch_mega_inst<3, 128>(c, a, smem);
+        default: return launch_mega_inst<4, 128>(c, a, smem);
+        }
+    }
+    switch (rs.n_rows) {
+    case 1: return launch_mega_inst<1, 64>(c, a, smem);
+    case 2: return launch_mega_inst<2, 64>(c, a, smem);
+    case 3: return launch_mega_inst<3, 64>(c, a, smem);
+    default: return launch_mega_inst<4, 64>(c, a, smem);
+    }
 }
 
 // One transformer layer over a row set: h <- h^(layer).

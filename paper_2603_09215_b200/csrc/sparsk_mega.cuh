@@ -37,19 +37,21 @@ constexpr int MK_BOX_ROWS = 16, MK_BOX_COLS = 256;
 constexpr int MK_BOX_BYTES = MK_BOX_ROWS * MK_BOX_COLS * 2;  // 8 KB
 constexpr int MK_SLOT_BYTES = 2 * MK_BOX_BYTES;              // two boxes per slot
 constexpr int MK_SLOTS = 8;
-constexpr int MK_MAX_ROWS = 2;
+constexpr int MK_MAX_ROWS = 4;
+constexpr int MK_AREA_BYTES = 88 * 1024;        // shared memory behind the ring
 constexpr int MK_ATT_WARPS = 4;                 // consumer warps that run attention items
 constexpr int MK_ATT_NST = 2;
 constexpr int MK_MAX_SPLITS = 16;
 
-// Shared memory behind the ring: activations of a projection phase, or the attention warps'
-// query blocks and K/V rings.
-inline size_t mk_area_bytes(int max_inner, int head_dim)
+// The area behind the ring holds the activations of a projection phase (M rows of bf16; when
+// M rows of the whole inner dimension do not fit, a window of k-steps that is reloaded as the
+// phase moves along), or the attention warps' query blocks and K/V rings.
+inline size_t mk_attn_bytes(int head_dim)
 {
-    const size_t act = (size_t)MK_MAX_ROWS * ((max_inner + MK_BOX_COLS - 1) / MK_BOX_COLS * MK_BOX_COLS) * 2;
-    const size_t att = (size_t)MK_ATT_WARPS * (16 + MK_ATT_NST * 2 * AT_TP) * (head_dim + 8) * 2;
-    return act > att ? act : att;
+    return (size_t)MK_ATT_WARPS * (16 + MK_ATT_NST * 2 * AT_TP) * (head_dim + 8) * 2;
 }
+// k-steps of M activation rows that fit the area
+__host__ __device__ inline int mk_act_window(int M) { return MK_AREA_BYTES / (M * MK_BOX_COLS * 2); }
 
 enum { MK_QKV = 0, MK_ATTN = 1, MK_MERGE = 2, MK_OPROJ = 3, MK_GATEUP = 4, MK_DOWN = 5 };
 

@@ -115,12 +115,10 @@ __global__ void __launch_bounds__(MK_THREADS, 1) mega_kernel(const MkArgs a)
         bf16 *act = reinterpret_cast<bf16 *>(area);
         bool ok = true;
         const int qd = a.Hq * a.hd;
-        auto pad256 = [](int k) { return (k + MK_BOX_COLS - 1) / MK_BOX_COLS * MK_BOX_COLS; };
         for (int l = a.layer_begin; l < a.layer_end && ok; l++) {
             const MkLayer *L = a.layers + l;
             // q/k/v
-            mk_load_act<M>(act, pad256(a.d), a.d, a.h, nullptr, L->attn_gain, a.eps, &sh);
-            if (!(ok = mk_project<M>(MK_QKV, a, L, act, pad256(a.d), ring, &sh, it))) break;
+            if (!(ok = mk_project<M>(MK_QKV, a, L, act, a.d, a.h, nullptr, L->attn_gain, ring, &sh, it))) break;
             if (!(ok = mk_grid_barrier(a, &sh, epoch))) break;
             // attention and the merge of its splits
             mk_attention<HD>(a, L, area);
@@ -128,15 +126,12 @@ __global__ void __launch_bounds__(MK_THREADS, 1) mega_kernel(const MkArgs a)
             mk_merge<HD>(a);
             if (!(ok = mk_grid_barrier(a, &sh, epoch))) break;
             // O-projection
-            mk_load_act<M>(act, pad256(qd), qd, nullptr, a.attn_o, nullptr, 0.f, &sh);
-            if (!(ok = mk_project<M>(MK_OPROJ, a, L, act, pad256(qd), ring, &sh, it))) break;
+            if (!(ok = mk_project<M>(MK_OPROJ, a, L, act, qd, nullptr, a.attn_o, nullptr, ring, &sh, it))) break;
             if (!(ok = mk_grid_barrier(a, &sh, epoch))) break;
             // MLP
-            mk_load_act<M>(act, pad256(a.d), a.d, a.h, nullptr, L->mlp_gain, a.eps, &sh);
-            if (!(ok = mk_project<M>(MK_GATEUP, a, L, act, pad256(a.d), ring, &sh, it))) break;
+            if (!(ok = mk_project<M>(MK_GATEUP, a, L, act, a.d, a.h, nullptr, L->mlp_gain, ring, &sh, it))) break;
             if (!(ok = mk_grid_barrier(a, &sh, epoch))) break;
-            mk_load_act<M>(act, pad256(a.F), a.F, nullptr, a.act, nullptr, 0.f, &sh);
-            if (!(ok = mk_project<M>(MK_DOWN, a, L, act, pad256(a.F), ring, &sh, it))) break;
+            if (!(ok = mk_project<M>(MK_DOWN, a, L, act, a.F, nullptr, a.act, nullptr, ring, &sh, it))) break;
             if (!(ok = mk_grid_barrier(a, &sh, epoch))) break;
         }
         if (!ok && threadIdx.x == 0) sh.giving_up = 1;

@@ -4,17 +4,19 @@
 namespace sparsk {
 
 // ------------------------------------------------------------------ activations -> shared memory
-// With h: x = h / sqrt(mean(h^2) + eps) * gain as bf16; otherwise a copy of bf16 rows.  Rows are
-// padded with zeros to a multiple of 256 columns (the last weight box is zero-filled there too).
+// Columns [c0, c0 + ncols) of the M activation rows, as bf16, row m at act + m * ncols.  With h:
+// x = h / sqrt(mean(h^2) + eps) * gain; otherwise a copy of bf16 rows.  Columns at or beyond K
+// are zeros (the last weight box is zero-filled there too).  ncols is a multiple of 256.
 template <int M>
-__device__ __forceinline__ void mk_load_act(bf16 *act, int kpad, int K, const float *h, const bf16 *x, const bf16 *gain,
-                                            float eps, MkShared *sh)
+__device__ __forceinline__ void mk_load_act(bf16 *act, int c0, int ncols, int K, const float *h, const bf16 *x,
+                                            const bf16 *gain, float eps, MkShared *sh)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int T = MK_CW * 32;
+    mk_consumer_sync();  // everyone is done with what the area held
 #pragma unroll
     for (int m = 0; m < M; m++) {
-        bf16 *dst = act + (size_t)m * kpad;
+        bf16 *dst = act + (size_t)m * ncols;
         if (h) {
             const float *src = h + (size_t)m * K;
             float ss = 0.f;
@@ -30,13 +32,14 @@ __device__ __forceinline__ void mk_load_act(bf16 *act, int kpad, int K, const fl
             for (int w = 0; w < MK_CW; w++) tot += sh->red[w];
             mk_consumer_sync();
             const float inv = rsqrtf(tot / (float)K + eps);
-            for (int i = tid * 8; i < kpad; i += T * 8) {
+            for (int i = tid * 8; i < ncols; i += T * 8) {
                 uint4 o = make_uint4(0, 0, 0, 0);
-                if (i < K) {
-                    const float4 p = *reinterpret_cast<const float4 *>(src + i);
-                    const float4 q = *reinterpret_cast<const float4 *>(src + i + 4);
+                const int k = c0 + i;
+                if (k < K) {
+                    const float4 p = *reinterpret_cast<const float4 *>(src + k);
+                    const float4 q = *reinterpret_cast<const float4 *>(src + k + 4);
                     float g[8];
-                    unpack8(*reinterpret_cast<const uint4 *>(gain + i), g);
+                    unpack8(*reinterpret_cast<const uint4 *>(gain + k), g);
                     o.x = pack_bf16x2(p.x * inv * g[0], p.y * inv * g[1]);
                     o.y = pack_bf16x2(p.z * inv * g[2], p.w * inv * g[3]);
                     o.z = pack_bf16x2(q.x * inv * g[4], q.y * inv * g[5]);
@@ -46,22 +49,35 @@ __device__ __forceinline__ void mk_load_act(bf16 *act, int kpad, int K, const fl
             }
         } else {
             const bf16 *src = x + (size_t)m * K;
-            for (int i = tid * 8; i < kpad; i += T * 8)
-                *reinterpret_cast<uint4 *>(dst + i) = i < K ? *reinterpret_cast<const uint4 *>(src + i) : make_uint4(0, 0, 0, 0);
+            for (int i = tid * 8; i < ncols; i += T * 8)
+                *reinterpret_cast<uint4 *>(dst + i) =
+                    c0 + i < K ? *reinterpret_cast<const uint4 *>(src + c0 + i) : make_uint4(0, 0, 0, 0);
         }
     }
     mk_consumer_sync();
 }
 
 // ------------------------------------------------------------------ projection phase (consumers)
+// The activations of the phase come from `h` (normalised with `gain`) or from the bf16 rows `x`,
+// K columns each.  If M rows of the whole inner dimension fit the area they are loaded once;
+// otherwise the area holds a window of k-steps that follows the CTA's segments.
 template <int M>
-__device__ __forceinline__ bool mk_project(int type, const MkArgs &a, const MkLayer *L, const bf16 *act, int kpad,
-                                           unsigned char *ring, MkShared *sh, uint32_t &it)
+__device__ __forceinline__ bool mk_project(int type, const MkArgs &a, const MkLayer *L, bf16 *act, int K,
+                                           const float *h, const bf16 *x, const bf16 *gain, unsigned char *ring,
+                                           MkShared *sh, uint32_t &it)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int half = a.hd >> 1, per_head = half / MK_BOX_ROWS;
     MkWalk walk;
     walk.init(type, a);
+    const int window = mk_act_window(M);
+    const bool whole = walk.k_steps <= window;
+    int win0 = 0, win1 = 0;  // k-steps the area holds: [win0, win1)
+    if (whole) {
+        win1 = walk.k_steps;
+        mk_load_act<M>(act, 0, win1 * MK_BOX_COLS, K, h, x, gain, a.eps, sh);
+    }
+    const int ncols = whole ? walk.k_steps * MK_BOX_COLS : window * MK_BOX_COLS;
     MkSeg seg;
     while (walk.next(seg)) {
         const int b = seg.band;
@@ -71,6 +87,11 @@ __device__ __forceinline__ bool mk_project(int type, const MkArgs &a, const MkLa
 #pragma unroll
             for (int m = 0; m < M; m++) acc[r][m] = 0.f;
         for (int ks = seg.ks0; ks < seg.ks1; ks++, it++) {
+            if (ks < win0 || ks >= win1) {  // uniform across the CTA: move the window
+                win0 = ks;
+                win1 = min(walk.k_steps, ks + window);
+                mk_load_act<M>(act, win0 * MK_BOX_COLS, ncols, K, h, x, gain, a.eps, sh);
+            }
             const int s = it % MK_SLOTS;
             if (!mbar_wait(&sh->full[s], (it / MK_SLOTS) & 1, &sh->giving_up, a.status)) return false;
             const unsigned char *slot = ring + (size_t)s * MK_SLOT_BYTES + (size_t)warp * MK_BOX_COLS * 2 + lane * 16;
@@ -79,12 +100,12 @@ __device__ __forceinline__ bool mk_project(int type, const MkArgs &a, const MkLa
             unpack8(*reinterpret_cast<const uint4 *>(slot + MK_BOX_BYTES), w1);
 #pragma unroll
             for (int m = 0; m < M; m++) {
-                float x[8];
-                unpack8(*reinterpret_cast<const uint4 *>(act + (size_t)m * kpad + ks * MK_BOX_COLS + lane * 8), x);
+                float xv[8];
+                unpack8(*reinterpret_cast<const uint4 *>(act + (size_t)m * ncols + (ks - win0) * MK_BOX_COLS + lane * 8), xv);
 #pragma unroll
                 for (int j = 0; j < 8; j++) {
-                    acc[0][m] = fmaf(w0[j], x[j], acc[0][m]);
-                    acc[1][m] = fmaf(w1[j], x[j], acc[1][m]);
+                    acc[0][m] = fmaf(w0[j], xv[j], acc[0][m]);
+                    acc[1][m] = fmaf(w1[j], xv[j], acc[1][m]);
                 }
             }
             __syncwarp();
