@@ -1,0 +1,142 @@
+"""GPU parity at the full model shapes of the five workloads (launch configuration of bench.py).
+
+The oracle cannot afford a prompt of hundreds of tokens at these shapes, so every sequence
+starts from a cache of stand-in values (synth.synth_kv) loaded into both sides; from there the
+library and the oracle run the same interleaved steps, teacher-forced on the oracle's tokens.
+With a batch the oracle follows a seeded subset of the sequences (sequences are independent,
+which the small-shape tests establish); the other sequences run free and are held to the exit
+schedule only.  Acceptance rules are those of parity_util: depths bit-exact, hidden states and
+logits within 2e-2, tokens identical where the oracle's top-2 margin exceeds 5e-2."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2603_09215_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _need_gpu():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+
+
+class Model:
+    """Random weights of a shape, once per module, on the host and on the device."""
+
+    def __init__(self, shape, head_layers):
+        from paper_2603_09215_b200 import binding
+        self.shape = shape
+        self.dims0 = synth.model_dims(shape, head_layers[0], 1, 0)
+        self.w = synth.make_weights(self.dims0, seed=0, head_layers=head_layers)
+        self.gw = binding.upload_weights(self.w)
+
+
+@pytest.fixture(scope="module")
+def step_model():
+    _need_gpu()
+    m = Model("step", [20, 28])
+    yield m
+    del m.gw
+    torch.cuda.empty_cache()
+
+
+@pytest.fixture(scope="module")
+def glm_model():
+    _need_gpu()
+    m = Model("glm", [20, 30, 40])
+    yield m
+    del m.gw
+    torch.cuda.empty_cache()
+
+
+def _load_cache(P, lens, checked, dims, shared_seed=77):
+    """Stand-in cache of lens[s] positions for every slot; the checked slots get their own
+    values (also given to their oracle), the others share one set."""
+    from oracle.bruteforce import bf16_to_f64
+    L = dims["n_layers"]
+    n_max = max(lens)
+    shared_k, shared_v = synth.synth_kv(dims, n_max, seed=shared_seed)
+    dev = lambda a: torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+    for layer in range(1, L + 1):
+        kt, vt = dev(shared_k[layer - 1]), dev(shared_v[layer - 1])
+        for s, n in enumerate(lens):
+            if s not in checked:
+                P.g.import_kv(s, layer, 0, kt[:n], vt[:n])
+    for s in checked:
+        k, v = synth.synth_kv(dims, lens[s], seed=1000 + s)
+        for layer in range(1, L + 1):
+            P.g.import_kv(s, layer, 0, dev(k[layer - 1]), dev(v[layer - 1]))
+            kf, vf = bf16_to_f64(k[layer - 1]), bf16_to_f64(v[layer - 1])
+            for p in range(lens[s]):
+                P.os[s].set_kv(layer, p, kf[p], vf[p])
+        P.os[s].set_len(lens[s])
+    for s, n in enumerate(lens):
+        P.g.set_len(s, n)
+    torch.cuda.synchronize()
+
+
+def _run(model, wl_name, steps, g0, n_checked, lens=None, exit_layer=None, period=None, batch=None):
+    from tests import parity_util as pu
+    wl = dict(synth.WORKLOADS[wl_name])
+    e = wl["exit_layer"] if exit_layer is None else exit_layer
+    K = wl["refresh_period"] if period is None else period
+    dims = synth.model_dims(model.shape, e, K, wl["refresh_phase"])
+    B = wl["batch"] if batch is None else batch
+    rng = np.random.Generator(np.random.PCG64(5))
+    if lens is None:
+        lens = [int(x) for x in rng.integers(wl["prompt"][0], wl["prompt"][1] + 1, size=B)] if wl["prompt"][0] != wl["prompt"][1] \
+            else [wl["prompt"][0] - 1] * B
+    phi, off = synth.make_phases(B, wl["n_text"], wl["n_speech"], K, wl["random_phase"], seed=3)
+    checked = sorted(int(x) for x in rng.choice(B, size=min(n_checked, B), replace=False))
+    P = pu.Pair(dims, model.w, B, max(lens) + steps + 2, max(K - 1, 1), oracle_slots=checked, gw=model.gw)
+    _load_cache(P, lens, set(checked), dims)
+    V = dims["vocab_text"] + dims["vocab_speech"]
+    P.next_in = [int(x) for x in rng.integers(0, V, size=B)]
+    mixed = 0
+    for g in range(g0, g0 + steps):
+        mc = [synth.interleave(g, wl["n_text"], wl["n_speech"], int(p), int(o)) for p, o in zip(phi, off)]
+        _, _, dep = P.step([m for m, _ in mc], [c for _, c in mc])
+        mixed += len(set(int(x) for x in dep)) > 1
+    stats = dict(P.stats, mixed_steps=mixed, checked=checked)
+    P.close()
+    return stats
+
+
+def test_config2_step_shape_batch1(step_model):
+    """Workload 2: Step-shaped, batch 1, cache of 511 positions, two interleave cycles
+    (text, refresh, three early exits; the second cycle's text step flushes three pending rows)."""
+    st = _run(step_model, "cfg2_step_b1", steps=10, g0=0, n_checked=1)
+    print("cfg2", st)
+    assert st["tok_checked"] >= 5
+
+
+def test_config3_step_shape_batch64(step_model):
+    """Workload 3: batch 64, ragged caches of 256..2048 positions, random interleave phases and
+    counter offsets so every step mixes depths; the oracle follows two of the sequences."""
+    st = _run(step_model, "cfg3_step_b64", steps=10, g0=0, n_checked=2)
+    print("cfg3", st)
+    assert st["mixed_steps"] >= 8
+
+
+def test_config4_glm_shape_batch16(glm_model):
+    """Workload 4: GLM-shaped, batch 16, caches of 1023 positions, phase-aligned 13:26 interleave;
+    steps 11..20 cover the end of a text chunk, two refreshes and a flush of three pending rows."""
+    st = _run(glm_model, "cfg4_glm_b16", steps=10, g0=11, n_checked=2)
+    print("cfg4", st)
+
+
+def test_config5_glm_shape_long_context(glm_model):
+    """Workload 5 (long-context stress): caches of 8191 positions; batch 128 with the oracle on
+    two sequences, for the e=30, K=4 cell."""
+    st = _run(glm_model, "cfg5_glm_b128", steps=6, g0=12, n_checked=2, lens=[8191] * 128)
+    print("cfg5", st)
+
+
+@pytest.mark.parametrize("e", [20, 30, 40])
+@pytest.mark.parametrize("K", [2, 4, 8])
+def test_config5_sweep_depths(glm_model, e, K):
+    """Every (e, K) cell of workload 5's sweep: exit depths of all 128 sequences over one
+    interleave cycle are exactly the schedule's (checked inside the driver for every step)."""
+    st = _run(glm_model, "cfg5_glm_b128", steps=39, g0=0, n_checked=0, lens=[64] * 128, exit_layer=e, period=K)
+    assert st["steps"] == 39
