@@ -86,6 +86,7 @@ struct sparsk_ctx {
     MkLayer *mk_layers;            // device [L]
     unsigned long long *mk_bar;    // device: grid barrier counter; mk_bar_base mirrors its value
     int *mk_abort;                 // device
+    float *mk_attn_o, *mk_act;     // device fp32 [MK_MAX_ROWS][Hq*hd], [MK_MAX_ROWS][F]
     unsigned long long *mk_trace;  // device [1 + 6 L]
     int mk_trace_n;                // entries the last launch wrote
     unsigned long long mk_bar_base;
@@ -176,6 +177,7 @@ size_t carve(sparsk_ctx *c, const sparsk_dims *d, char *base)
     MkLayer *mkl = w.take<MkLayer>(L);
     unsigned long long *mkb = w.take<unsigned long long>(1);
     int *mka = w.take<int>(1);
+    float *mkao = w.take<float>((size_t)MK_MAX_ROWS * qrow), *mkact = w.take<float>((size_t)MK_MAX_ROWS * d->d_ffn);
     unsigned long long *mkt = w.take<unsigned long long>(1 + 6 * L);
     const size_t cells = std::max<size_t>(R * MAX_SPLITS, (size_t)MK_MAX_ROWS * MK_MAX_SPLITS) * d->n_q_heads;
     float *po = w.take<float>(cells * d->head_dim);
@@ -186,7 +188,7 @@ size_t carve(sparsk_ctx *c, const sparsk_dims *d, char *base)
         c->pf_slot = pfs; c->pf_pos = pfp; c->pf_grp_row0 = pfg0; c->pf_grp_nrows = pfgn;
         c->pf_ngrp = pfng; c->pf_nrows = pfnr;
         c->h_lo = hlo; c->h_up = hup; c->qbuf = q; c->attn_o = ao; c->act = act; c->xnorm = xn; c->qkv_part = qp;
-        c->mk_layers = mkl; c->mk_bar = mkb; c->mk_abort = mka; c->mk_trace = mkt;
+        c->mk_layers = mkl; c->mk_bar = mkb; c->mk_abort = mka; c->mk_attn_o = mkao; c->mk_act = mkact; c->mk_trace = mkt;
         c->part_o = po; c->part_ml = pml;
     }
     return align_up(w.off, 256);
@@ -704,7 +706,7 @@ cudaError_t run_mega(sparsk_ctx *c, int l_begin, int l_end, float *h, const RowS
     a.layers = c->mk_layers; a.layer_begin = l_begin; a.layer_end = l_end; a.h = h;
     a.row_slot = rs.slot; a.row_pos = rs.pos; a.grp_row0 = rs.grp_row0; a.grp_nrows = rs.grp_nrows;
     a.n_rows = rs.n_rows; a.n_groups = rs.n_groups_h;
-    a.q_buf = c->qbuf; a.attn_o = c->attn_o; a.act = c->act; a.part_o = c->part_o; a.part_ml = c->part_ml;
+    a.q_buf = c->qbuf; a.attn_o = c->mk_attn_o; a.act = c->mk_act; a.part_o = c->part_o; a.part_ml = c->part_ml;
     a.rope = c->rope;
     a.d = d.d_model; a.Hq = d.n_q_heads; a.Hkv = d.n_kv_heads; a.hd = d.head_dim; a.F = d.d_ffn; a.S = d.max_seq_len;
     a.n_slots = d.max_seqs; a.eps = d.rms_eps;

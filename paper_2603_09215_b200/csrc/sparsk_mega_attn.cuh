@@ -193,9 +193,9 @@ __device__ __forceinline__ void mk_merge(const MkArgs &a)
 #pragma unroll
             for (int e = 0; e < DL; e++) num[e] += po[e] * w;
         }
-        bf16 *dst = a.attn_o + (size_t)item * HD + lane * DL;
+        float *dst = a.attn_o + (size_t)item * HD + lane * DL;
 #pragma unroll
-        for (int e = 0; e < DL; e++) dst[e] = __float2bfloat16(den > 0.f ? num[e] / den : 0.f);
+        for (int e = 0; e < DL; e++) dst[e] = den > 0.f ? num[e] / den : 0.f;
     }
 }
 

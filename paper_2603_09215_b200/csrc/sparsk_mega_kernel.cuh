@@ -112,7 +112,7 @@ __global__ void __launch_bounds__(MK_THREADS, 1) mega_kernel(const MkArgs a)
         uint32_t it = 0;
         unsigned long long epoch = a.bar_base;
         if (blockIdx.x == 0 && threadIdx.x == 0 && a.trace) a.trace[0] = global_ns();
-        bf16 *act = reinterpret_cast<bf16 *>(area);
+        float *act = reinterpret_cast<float *>(area);
         bool ok = true;
         const int qd = a.Hq * a.hd;
         for (int l = a.layer_begin; l < a.layer_end && ok; l++) {

@@ -4,11 +4,11 @@
 namespace sparsk {
 
 // ------------------------------------------------------------------ activations -> shared memory
-// Columns [c0, c0 + ncols) of the M activation rows, as bf16, row m at act + m * ncols.  With h:
-// x = h / sqrt(mean(h^2) + eps) * gain; otherwise a copy of bf16 rows.  Columns at or beyond K
-// are zeros (the last weight box is zero-filled there too).  ncols is a multiple of 256.
+// Columns [c0, c0 + ncols) of the M activation rows, as fp32, row m at act + m * ncols.  With h:
+// x = h / sqrt(mean(h^2) + eps) * gain; otherwise a copy of the fp32 rows x.  Columns at or
+// beyond K are zeros (the last weight box is zero-filled there too).  ncols is a multiple of 256.
 template <int M>
-__device__ __forceinline__ void mk_load_act(bf16 *act, int c0, int ncols, int K, const float *h, const bf16 *x,
+__device__ __forceinline__ void mk_load_act(float *act, int c0, int ncols, int K, const float *h, const float *x,
                                             const bf16 *gain, float eps, MkShared *sh)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -16,7 +16,7 @@ __device__ __forceinline__ void mk_load_act(bf16 *act, int c0, int ncols, int K,
     mk_consumer_sync();  // everyone is done with what the area held
 #pragma unroll
     for (int m = 0; m < M; m++) {
-        bf16 *dst = act + (size_t)m * ncols;
+        float *dst = act + (size_t)m * ncols;
         if (h) {
             const float *src = h + (size_t)m * K;
             float ss = 0.f;
@@ -32,38 +32,34 @@ __device__ __forceinline__ void mk_load_act(bf16 *act, int c0, int ncols, int K,
             for (int w = 0; w < MK_CW; w++) tot += sh->red[w];
             mk_consumer_sync();
             const float inv = rsqrtf(tot / (float)K + eps);
-            for (int i = tid * 8; i < ncols; i += T * 8) {
-                uint4 o = make_uint4(0, 0, 0, 0);
+            for (int i = tid * 4; i < ncols; i += T * 4) {
+                float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
                 const int k = c0 + i;
                 if (k < K) {
                     const float4 p = *reinterpret_cast<const float4 *>(src + k);
-                    const float4 q = *reinterpret_cast<const float4 *>(src + k + 4);
-                    float g[8];
-                    unpack8(*reinterpret_cast<const uint4 *>(gain + k), g);
-                    o.x = pack_bf16x2(p.x * inv * g[0], p.y * inv * g[1]);
-                    o.y = pack_bf16x2(p.z * inv * g[2], p.w * inv * g[3]);
-                    o.z = pack_bf16x2(q.x * inv * g[4], q.y * inv * g[5]);
-                    o.w = pack_bf16x2(q.z * inv * g[6], q.w * inv * g[7]);
+                    const uint2 g2 = *reinterpret_cast<const uint2 *>(gain + k);
+                    o = make_float4(p.x * inv * bf_lo(g2.x), p.y * inv * bf_hi(g2.x), p.z * inv * bf_lo(g2.y),
+                                    p.w * inv * bf_hi(g2.y));
                 }
-                *reinterpret_cast<uint4 *>(dst + i) = o;
+                *reinterpret_cast<float4 *>(dst + i) = o;
             }
         } else {
-            const bf16 *src = x + (size_t)m * K;
-            for (int i = tid * 8; i < ncols; i += T * 8)
-                *reinterpret_cast<uint4 *>(dst + i) =
-                    c0 + i < K ? *reinterpret_cast<const uint4 *>(src + c0 + i) : make_uint4(0, 0, 0, 0);
+            const float *src = x + (size_t)m * K;
+            for (int i = tid * 4; i < ncols; i += T * 4)
+                *reinterpret_cast<float4 *>(dst + i) =
+                    c0 + i < K ? *reinterpret_cast<const float4 *>(src + c0 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
     }
     mk_consumer_sync();
 }
 
 // ------------------------------------------------------------------ projection phase (consumers)
-// The activations of the phase come from `h` (normalised with `gain`) or from the bf16 rows `x`,
+// The activations of the phase come from `h` (normalised with `gain`) or from the fp32 rows `x`,
 // K columns each.  If M rows of the whole inner dimension fit the area they are loaded once;
 // otherwise the area holds a window of k-steps that follows the CTA's segments.
 template <int M>
-__device__ __forceinline__ bool mk_project(int type, const MkArgs &a, const MkLayer *L, bf16 *act, int K,
-                                           const float *h, const bf16 *x, const bf16 *gain, unsigned char *ring,
+__device__ __forceinline__ bool mk_project(int type, const MkArgs &a, const MkLayer *L, float *act, int K,
+                                           const float *h, const float *x, const bf16 *gain, unsigned char *ring,
                                            MkShared *sh, uint32_t &it)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -100,8 +96,9 @@ __device__ __forceinline__ bool mk_project(int type, const MkArgs &a, const MkLa
             unpack8(*reinterpret_cast<const uint4 *>(slot + MK_BOX_BYTES), w1);
 #pragma unroll
             for (int m = 0; m < M; m++) {
-                float xv[8];
-                unpack8(*reinterpret_cast<const uint4 *>(act + (size_t)m * ncols + (ks - win0) * MK_BOX_COLS + lane * 8), xv);
+                const float *xp = act + (size_t)m * ncols + (ks - win0) * MK_BOX_COLS + lane * 8;
+                const float4 xa = *reinterpret_cast<const float4 *>(xp), xb = *reinterpret_cast<const float4 *>(xp + 4);
+                const float xv[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
 #pragma unroll
                 for (int j = 0; j < 8; j++) {
                     acc[0][m] = fmaf(w0[j], xv[j], acc[0][m]);
@@ -149,7 +146,7 @@ __device__ __forceinline__ bool mk_project(int type, const MkArgs &a, const MkLa
             }
             case MK_GATEUP: {
                 const int f = b * MK_BOX_ROWS + warp;
-                if (f < a.F) a.act[(size_t)m * a.F + f] = __float2bfloat16(v0 / (1.f + __expf(-v0)) * v1);
+                if (f < a.F) a.act[(size_t)m * a.F + f] = v0 / (1.f + __expf(-v0)) * v1;
                 break;
             }
             default: {
