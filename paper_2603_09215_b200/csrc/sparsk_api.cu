@@ -64,7 +64,9 @@ struct sparsk_ctx {
     int *staged, *tok_dev, *out_tok_dev, *out_depth_dev;
     int *pf_slot, *pf_pos, *pf_grp_row0, *pf_grp_nrows, *pf_ngrp, *pf_nrows;
     float *h_lo, *h_up;
-    bf16 *qbuf, *attn_o, *act, *xnorm;
+    float *qbuf;
+    bf16 *attn_o, *act, *xnorm;
+    bf16 *attn_o_lo, *act_lo, *xnorm_lo;  // second bf16 term of the tensor-core path's activations
     float *part_o;
     float2 *part_ml;
     // pinned staging ring for the per-step host arrays
@@ -81,7 +83,7 @@ struct sparsk_ctx {
     // (one per box height 16, 32, 64, 128, 256)
     bool tc_ok;
     std::vector<TmaPair> tm_wq, tm_wk, tm_wv, tm_wo, tm_wg, tm_wu, tm_wd, tm_head;
-    TmaPair tm_x[5], tm_ao[5], tm_act[5];
+    TmaPair tm_x[5], tm_ao[5], tm_act[5], tm_x_lo[5], tm_ao_lo[5], tm_act_lo[5];
     // persistent layer-range kernel (one or two rows)
     MkLayer *mk_layers;            // device [L]
     unsigned long long *mk_bar;    // device: grid barrier counter; mk_bar_base mirrors its value
@@ -171,8 +173,10 @@ size_t carve(sparsk_ctx *c, const sparsk_dims *d, char *base)
     int *pfs = w.take<int>(R), *pfp = w.take<int>(R), *pfg0 = w.take<int>(1), *pfgn = w.take<int>(1);
     int *pfng = w.take<int>(1), *pfnr = w.take<int>(1);
     float *hlo = w.take<float>(B * d->d_model), *hup = w.take<float>(R * d->d_model);
-    bf16 *q = w.take<bf16>(R * qrow), *ao = w.take<bf16>(R * qrow), *act = w.take<bf16>(R * d->d_ffn);
+    float *q = w.take<float>(R * qrow);
+    bf16 *ao = w.take<bf16>(R * qrow), *act = w.take<bf16>(R * d->d_ffn);
     bf16 *xn = w.take<bf16>(R * d->d_model);
+    bf16 *aol = w.take<bf16>(R * qrow), *actl = w.take<bf16>(R * d->d_ffn), *xnl = w.take<bf16>(R * d->d_model);
     float *qp = w.take<float>(R * (qrow + 2 * kvrow));
     MkLayer *mkl = w.take<MkLayer>(L);
     unsigned long long *mkb = w.take<unsigned long long>(1);
@@ -188,6 +192,7 @@ size_t carve(sparsk_ctx *c, const sparsk_dims *d, char *base)
         c->pf_slot = pfs; c->pf_pos = pfp; c->pf_grp_row0 = pfg0; c->pf_grp_nrows = pfgn;
         c->pf_ngrp = pfng; c->pf_nrows = pfnr;
         c->h_lo = hlo; c->h_up = hup; c->qbuf = q; c->attn_o = ao; c->act = act; c->xnorm = xn; c->qkv_part = qp;
+        c->attn_o_lo = aol; c->act_lo = actl; c->xnorm_lo = xnl;
         c->mk_layers = mkl; c->mk_bar = mkb; c->mk_abort = mka; c->mk_attn_o = mkao; c->mk_act = mkact; c->mk_trace = mkt;
         c->part_o = po; c->part_ml = pml;
     }
@@ -383,12 +388,13 @@ cudaError_t run_attn(sparsk_ctx *c, int layer, const RowSet &rs)
     const int G = d.n_q_heads / d.n_kv_heads;
     const size_t lstride = (size_t)d.max_seqs * d.n_kv_heads * d.max_seq_len * d.head_dim;
     AttnArgs a{};
-    a.q = c->qbuf;
+    a.q = nullptr;
+    a.q32 = c->qbuf;
     a.kc = c->kcache + (layer - 1) * lstride;
     a.vc = c->vcache + (layer - 1) * lstride;
     a.grp_row0 = rs.grp_row0; a.grp_nrows = rs.grp_nrows; a.row_slot = rs.slot; a.row_pos = rs.pos;
     a.n_groups = rs.n_groups;
-    a.part_o = c->part_o; a.part_ml = c->part_ml; a.out = c->attn_o;
+    a.part_o = c->part_o; a.part_ml = c->part_ml; a.out = c->attn_o; a.out_lo = c->attn_o_lo;
     a.Hq = d.n_q_heads; a.Hkv = d.n_kv_heads; a.S = d.max_seq_len;
     const AttnPlan pl = attn_plan(c->n_sm, rs.n_groups_h, rs.max_grp_rows, G, d.n_kv_heads, rs.max_len, c->attn_split);
     a.n_qblk = pl.n_qblk;
@@ -466,6 +472,9 @@ bool build_maps(sparsk_ctx *c)
         ok = ok && encode_maps(fn, &c->tm_x[b], c->xnorm, c->cap_rows, d.d_model, box);
         ok = ok && encode_maps(fn, &c->tm_ao[b], c->attn_o, c->cap_rows, qd, box);
         ok = ok && encode_maps(fn, &c->tm_act[b], c->act, c->cap_rows, d.d_ffn, box);
+        ok = ok && encode_maps(fn, &c->tm_x_lo[b], c->xnorm_lo, c->cap_rows, d.d_model, box);
+        ok = ok && encode_maps(fn, &c->tm_ao_lo[b], c->attn_o_lo, c->cap_rows, qd, box);
+        ok = ok && encode_maps(fn, &c->tm_act_lo[b], c->act_lo, c->cap_rows, d.d_ffn, box);
     }
     return ok;
 }
@@ -479,7 +488,7 @@ int box_index(int m_rows)
 
 template <class Epi>
 cudaError_t launch_gemm(sparsk_ctx *c, const TmaPair &a0, const TmaPair &a1, const TmaPair &a2, const TmaPair *b_maps,
-                        GemmArgs g, const Epi &epi)
+                        const TmaPair *b_lo_maps, GemmArgs g, const Epi &epi)
 {
     static bool attr_set = false;
     constexpr int SMEM_BUDGET = 220 * 1024;
@@ -492,7 +501,7 @@ cudaError_t launch_gemm(sparsk_ctx *c, const TmaPair &a0, const TmaPair &a1, con
     const int bi = box_index(g.m_rows);
     g.box_n = 16 << bi;
     const int room = SMEM_BUDGET - 1024 - GM_XCHG_BYTES;
-    auto stage_bytes = [&](int kb) { return 2 * kb * GM_BLK_BYTES + kb * g.box_n * GM_BK * 2; };
+    auto stage_bytes = [&](int kb) { return 2 * kb * GM_BLK_BYTES + 2 * kb * g.box_n * GM_BK * 2; };
     // two k-blocks per copy whenever the inner dimension allows the 3-D view and two stages fit
     g.three_d = (g.K % GM_BK == 0) && 2 * stage_bytes(2) <= room && c->tc_kb != 1;
     g.kb = g.three_d ? 2 : 1;
@@ -506,15 +515,17 @@ cudaError_t launch_gemm(sparsk_ctx *c, const TmaPair &a0, const TmaPair &a1, con
     const int grid_y = (g.m_rows + GM_MAX_N - 1) / GM_MAX_N;
     const size_t smem = 1024 + (size_t)g.stages * stage_bytes(g.kb) + GM_XCHG_BYTES;
     if (g.three_d)
-        return launch(c, kern, dim3(grid_x, grid_y), dim3(GM_THREADS), smem, a0.m3, a1.m3, a2.m3, b_maps[bi].m3, g, epi);
-    return launch(c, kern, dim3(grid_x, grid_y), dim3(GM_THREADS), smem, a0.m2, a1.m2, a2.m2, b_maps[bi].m2, g, epi);
+        return launch(c, kern, dim3(grid_x, grid_y), dim3(GM_THREADS), smem, a0.m3, a1.m3, a2.m3, b_maps[bi].m3,
+                      b_lo_maps[bi].m3, g, epi);
+    return launch(c, kern, dim3(grid_x, grid_y), dim3(GM_THREADS), smem, a0.m2, a1.m2, a2.m2, b_maps[bi].m2,
+                  b_lo_maps[bi].m2, g, epi);
 }
 
 int div_up(int a, int b) { return (a + b - 1) / b; }
 
 cudaError_t run_norm(sparsk_ctx *c, const float *h, const bf16 *gain, const int *row_idx, int n_rows)
 {
-    return launch(c, rmsnorm_rows_kernel, dim3(n_rows), dim3(256), 0, h, gain, row_idx, c->xnorm, n_rows,
+    return launch(c, rmsnorm_rows_kernel, dim3(n_rows), dim3(256), 0, h, gain, row_idx, c->xnorm, c->xnorm_lo, n_rows,
                   c->dm.d_model, c->dm.rms_eps);
 }
 
@@ -542,7 +553,7 @@ cudaError_t run_layer_tc(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
         ep.q_out = c->qbuf; ep.kc = kc; ep.vc = vc; ep.rope = c->rope;
         ep.row_slot = rs.slot; ep.row_pos = rs.pos; ep.Hq = d.n_q_heads; ep.Hkv = d.n_kv_heads; ep.hd = d.head_dim;
         ep.S = d.max_seq_len; ep.partial = g.splits > 1 ? c->qkv_part : nullptr;
-        if ((e = launch_gemm(c, c->tm_wq[li], c->tm_wk[li], c->tm_wv[li], c->tm_x, g, ep)) != cudaSuccess) return e;
+        if ((e = launch_gemm(c, c->tm_wq[li], c->tm_wk[li], c->tm_wv[li], c->tm_x, c->tm_x_lo, g, ep)) != cudaSuccess) return e;
         if (g.splits > 1 &&
             (e = launch(c, qkv_finish_kernel, dim3(M), dim3(256), 0, c->qkv_part, c->qbuf, kc, vc, (const float2 *)c->rope,
                         rs.slot, rs.pos, M, d.n_q_heads, d.n_kv_heads, d.head_dim, d.max_seq_len)) != cudaSuccess)
@@ -557,7 +568,7 @@ cudaError_t run_layer_tc(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
         g.splits = splits_for(c, g.units[0]);
         ResidEnd ep;
         ep.h = h; ep.n_out = d.d_model; ep.atomic = 1;
-        if ((e = launch_gemm(c, c->tm_wo[li], c->tm_wo[li], c->tm_wo[li], c->tm_ao, g, ep)) != cudaSuccess) return e;
+        if ((e = launch_gemm(c, c->tm_wo[li], c->tm_wo[li], c->tm_wo[li], c->tm_ao, c->tm_ao_lo, g, ep)) != cudaSuccess) return e;
     }
     c->cur_class = KC_MISC;
     if ((e = run_norm(c, h, c->mlp_norm[li], nullptr, M)) != cudaSuccess) return e;
@@ -566,8 +577,8 @@ cudaError_t run_layer_tc(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
         GemmArgs g{};
         g.K = d.d_model; g.units[0] = div_up(d.d_ffn, GM_BM); g.pair = 1; g.m_rows = M; g.splits = 1;
         GateUpEnd ep;
-        ep.u = c->act; ep.F = d.d_ffn;
-        if ((e = launch_gemm(c, c->tm_wg[li], c->tm_wu[li], c->tm_wu[li], c->tm_x, g, ep)) != cudaSuccess) return e;
+        ep.u = c->act; ep.u_lo = c->act_lo; ep.F = d.d_ffn;
+        if ((e = launch_gemm(c, c->tm_wg[li], c->tm_wu[li], c->tm_wu[li], c->tm_x, c->tm_x_lo, g, ep)) != cudaSuccess) return e;
     }
     {
         c->cur_class = KC_DOWN;
@@ -576,7 +587,7 @@ cudaError_t run_layer_tc(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
         g.splits = splits_for(c, g.units[0]);
         ResidEnd ep;
         ep.h = h; ep.n_out = d.d_model; ep.atomic = 1;
-        e = launch_gemm(c, c->tm_wd[li], c->tm_wd[li], c->tm_wd[li], c->tm_act, g, ep);
+        e = launch_gemm(c, c->tm_wd[li], c->tm_wd[li], c->tm_wd[li], c->tm_act, c->tm_act_lo, g, ep);
     }
     c->cur_class = KC_MISC;
     return e;
@@ -600,7 +611,7 @@ cudaError_t run_head_tc(sparsk_ctx *c, int layer, const float *h, int list, int 
     GemmArgs g{};
     g.K = d.d_model; g.units[0] = div_up(ep.hi - ep.lo, 2 * GM_BM); g.row0[0] = ep.lo; g.m_rows = n_rows;
     g.splits = 1;
-    e = launch_gemm(c, c->tm_head[li], c->tm_head[li], c->tm_head[li], c->tm_x, g, ep);
+    e = launch_gemm(c, c->tm_head[li], c->tm_head[li], c->tm_head[li], c->tm_x, c->tm_x_lo, g, ep);
     c->cur_class = KC_MISC;
     return e;
 }

@@ -11,7 +11,8 @@
 // The split's positions are dealt to the CTA's four warps as contiguous sub-ranges.  Each warp
 // streams its own 16-position K/V tiles into a private three-stage shared-memory ring with
 // coalesced 16-byte cp.async copies (no CTA-wide barrier in the loop), computes S = Q K^T and
-// O += P V with bf16 MMAs and fp32 accumulators, and keeps an online softmax whose row maxima
+// O += P V with bf16 MMAs and fp32 accumulators (queries and softmax weights enter as two bf16
+// terms, hi + lo, so that only the cache itself is rounded to bf16), and keeps an online softmax whose row maxima
 // and sums are reduced with shuffles inside the four-lane groups that share an accumulator row.
 // The four warps' states are merged through shared memory into one unnormalised partial
 // (acc, running max, running sum) per split; a second kernel merges the splits.
@@ -23,7 +24,7 @@ namespace sparsk {
 
 constexpr int AT_THREADS = 128;
 constexpr int AT_TP = 16;        // positions per warp tile
-constexpr int AT_NST = 3;        // ring stages per warp
+constexpr int AT_NST = 3;        // ring stages per warp (two when the CTA holds 32 query vectors)
 constexpr int AT_MAX_SPLITS = 32;
 constexpr int AT_MIN_SPLIT = 64;
 
@@ -63,19 +64,21 @@ inline AttnPlan attn_plan(int n_sm, int n_groups, int max_grp_rows, int G, int H
 inline size_t attn_smem_bytes(int head_dim, int mt)
 {
     const size_t kp = head_dim + 8;
-    const size_t q = (size_t)16 * mt * kp * 2, ring = (size_t)4 * AT_NST * 2 * AT_TP * kp * 2;
+    const size_t q = (size_t)2 * 16 * mt * kp * 2, ring = (size_t)4 * (mt == 2 ? 2 : AT_NST) * 2 * AT_TP * kp * 2;
     const size_t merge = (size_t)4 * 16 * mt * (head_dim + 2) * 4;
     return q + (ring > merge ? ring : merge);
 }
 
 struct AttnArgs {
     const bf16 *q;            // [rows][Hq*hd], already rotated
+    const float *q32;         // the same in fp32; used instead of q when not NULL
     const bf16 *kc, *vc;      // this layer: [slot][Hkv][S][hd]
     const int *grp_row0, *grp_nrows, *row_slot, *row_pos;
     const int *n_groups;      // device count
     float *part_o;            // [rows*Hq][n_splits][hd]
     float2 *part_ml;          // [rows*Hq][n_splits]  (max, sum)
     bf16 *out;                // [rows][Hq*hd]
+    bf16 *out_lo;             // optional second bf16 term: out + out_lo carries 16 significant bits
     int Hq, Hkv, S, n_qblk, n_splits, split_len;
     int n_slots;              // slots in the cache; rows naming another slot are skipped
     int n_rows;               // rows in q/out; groups reaching beyond them are skipped
@@ -119,9 +122,11 @@ __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(AttnArgs a)
     constexpr int QB = 16 * MT;     // query vectors per CTA
     constexpr int KP = HD + 8;      // padded row: ldmatrix rows fall into distinct banks
     constexpr int CH = HD / 8;      // 16-byte chunks per row
+    constexpr int NS = MT == 2 ? 2 : AT_NST;
     extern __shared__ __align__(16) unsigned char at_smem[];
-    bf16 *Qs = reinterpret_cast<bf16 *>(at_smem);  // [QB][KP]
-    bf16 *ring = Qs + QB * KP;                     // [4 warps][AT_NST][K,V][AT_TP][KP]
+    bf16 *Qs = reinterpret_cast<bf16 *>(at_smem);  // [QB][KP] hi terms
+    bf16 *Ql = Qs + QB * KP;                       // [QB][KP] lo terms
+    bf16 *ring = Ql + QB * KP;                     // [4 warps][NS][K,V][AT_TP][KP]
 
     griddep_wait();
     griddep_launch();
@@ -148,12 +153,21 @@ __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(AttnArgs a)
 
     for (int i = tid; i < QB * CH; i += AT_THREADS) {
         const int qi = i / CH, c = i % CH;
-        uint4 v = make_uint4(0, 0, 0, 0);
+        uint4 hi = make_uint4(0, 0, 0, 0), lo = hi;
         if (qi < nq_here) {
             const int qg = q0 + qi, r = qg / G, j = qg % G;
-            v = *reinterpret_cast<const uint4 *>(a.q + (size_t)(row0 + r) * a.Hq * HD + (hk * G + j) * HD + c * 8);
+            const size_t off = (size_t)(row0 + r) * a.Hq * HD + (hk * G + j) * HD + c * 8;
+            if (a.q32) {
+                const float4 x0 = *reinterpret_cast<const float4 *>(a.q32 + off);
+                const float4 x1 = *reinterpret_cast<const float4 *>(a.q32 + off + 4);
+                const float v[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+                split8(v, hi, lo);
+            } else {
+                hi = *reinterpret_cast<const uint4 *>(a.q + off);
+            }
         }
-        *reinterpret_cast<uint4 *>(&Qs[qi * KP + c * 8]) = v;
+        *reinterpret_cast<uint4 *>(&Qs[qi * KP + c * 8]) = hi;
+        *reinterpret_cast<uint4 *>(&Ql[qi * KP + c * 8]) = lo;
     }
     __syncthreads();
 
@@ -163,12 +177,12 @@ __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(AttnArgs a)
     const int w_beg = s_beg + warp * per;
     const int w_end = min(w_beg + per, s_end);
     const int n_tiles = w_end > w_beg ? (w_end - w_beg + AT_TP - 1) / AT_TP : 0;
-    bf16 *wr = ring + (size_t)warp * AT_NST * 2 * AT_TP * KP;
+    bf16 *wr = ring + (size_t)warp * NS * 2 * AT_TP * KP;
     const bf16 *kbase = a.kc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
     const bf16 *vbase = a.vc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
 
     auto issue = [&](int t) {
-        bf16 *kt = wr + (size_t)(t % AT_NST) * 2 * AT_TP * KP, *vt = kt + AT_TP * KP;
+        bf16 *kt = wr + (size_t)(t % NS) * 2 * AT_TP * KP, *vt = kt + AT_TP * KP;
         const int p0 = w_beg + t * AT_TP;
 #pragma unroll
         for (int i = lane; i < AT_TP * CH; i += 32) {
@@ -202,16 +216,16 @@ __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(AttnArgs a)
     const float scale = rsqrtf((float)HD);
 
 #pragma unroll
-    for (int t = 0; t < AT_NST - 1; t++) {
+    for (int t = 0; t < NS - 1; t++) {
         if (t < n_tiles) issue(t);
         cp_async_commit();
     }
     for (int t = 0; t < n_tiles; t++) {
-        cp_async_wait<AT_NST - 2>();
+        cp_async_wait<NS - 2>();
         __syncwarp();
-        if (t + AT_NST - 1 < n_tiles) issue(t + AT_NST - 1);
+        if (t + NS - 1 < n_tiles) issue(t + NS - 1);
         cp_async_commit();
-        const bf16 *Kt = wr + (size_t)(t % AT_NST) * 2 * AT_TP * KP, *Vt = Kt + AT_TP * KP;
+        const bf16 *Kt = wr + (size_t)(t % NS) * 2 * AT_TP * KP, *Vt = Kt + AT_TP * KP;
         const int p0 = w_beg + t * AT_TP;
 
         // S = Q K^T for 16 positions
@@ -228,14 +242,18 @@ __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(AttnArgs a)
             ldsm_x4(kb, &Kt[((lane & 7) + ((lane >> 4) << 3)) * KP + ks * 16 + ((lane >> 3) & 1) * 8]);
 #pragma unroll
             for (int mt = 0; mt < MT; mt++) {
-                uint32_t qa[4];
-                ldsm_x4(qa, &Qs[(mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * KP + ks * 16 + (lane >> 4) * 8]);
+                uint32_t qa[4], ql[4];
+                const int qoff = (mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * KP + ks * 16 + (lane >> 4) * 8;
+                ldsm_x4(qa, &Qs[qoff]);
+                ldsm_x4(ql, &Ql[qoff]);
                 mma_bf16(s[mt][0], qa, kb[0], kb[1]);
                 mma_bf16(s[mt][1], qa, kb[2], kb[3]);
+                mma_bf16(s[mt][0], ql, kb[0], kb[1]);
+                mma_bf16(s[mt][1], ql, kb[2], kb[3]);
             }
         }
         // online softmax; P as the A operand of the second product
-        uint32_t pa[MT][4];
+        uint32_t pa[MT][4], pl[MT][4];
 #pragma unroll
         for (int mt = 0; mt < MT; mt++) {
 #pragma unroll
@@ -268,8 +286,8 @@ __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(AttnArgs a)
                 }
                 l_run[mt][hf] = l_run[mt][hf] * alpha + psum;  // per-thread share; lanes are summed at the end
                 m_run[mt][hf] = m_new;
-                pa[mt][hf] = pack_bf16x2(v[0], v[1]);       // positions 0..7 of the tile
-                pa[mt][2 + hf] = pack_bf16x2(v[2], v[3]);   // positions 8..15
+                split_pair(v[0], v[1], pa[mt][hf], pl[mt][hf]);          // positions 0..7 of the tile
+                split_pair(v[2], v[3], pa[mt][2 + hf], pl[mt][2 + hf]);  // positions 8..15
 #pragma unroll
                 for (int nt = 0; nt < HD / 8; nt++) {
                     o[mt][nt][hf * 2] *= alpha;
@@ -286,6 +304,8 @@ __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(AttnArgs a)
             for (int mt = 0; mt < MT; mt++) {
                 mma_bf16(o[mt][2 * np], pa[mt], vb[0], vb[1]);
                 mma_bf16(o[mt][2 * np + 1], pa[mt], vb[2], vb[3]);
+                mma_bf16(o[mt][2 * np], pl[mt], vb[0], vb[1]);
+                mma_bf16(o[mt][2 * np + 1], pl[mt], vb[2], vb[3]);
             }
         }
     }
@@ -376,7 +396,10 @@ __global__ void __launch_bounds__(HD) attn_merge_kernel(AttnArgs a, const int *_
         den += ml.y * w;
         num += a.part_o[(cell0 + s) * HD + threadIdx.x] * w;
     }
-    a.out[(size_t)row * a.Hq * HD + head * HD + threadIdx.x] = __float2bfloat16(den > 0.f ? num / den : 0.f);
+    const float val = den > 0.f ? num / den : 0.f;
+    const bf16 hi = __float2bfloat16(val);
+    a.out[(size_t)row * a.Hq * HD + head * HD + threadIdx.x] = hi;
+    if (a.out_lo) a.out_lo[(size_t)row * a.Hq * HD + head * HD + threadIdx.x] = __float2bfloat16(val - __bfloat162float(hi));
 }
 
 }  // namespace sparsk

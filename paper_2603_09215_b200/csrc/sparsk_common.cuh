@@ -58,6 +58,22 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b)
     return *reinterpret_cast<uint32_t *>(&t);
 }
 
+// x = hi + lo with hi = bf16(x), lo = bf16(x - hi): two bf16 terms that carry 16 significant
+// bits through a bf16 tensor-core product.
+__device__ __forceinline__ void split_pair(float a, float b, uint32_t &hi, uint32_t &lo)
+{
+    const bf16 ha = __float2bfloat16(a), hb = __float2bfloat16(b);
+    hi = pack_bf16x2(__bfloat162float(ha), __bfloat162float(hb));
+    lo = pack_bf16x2(a - __bfloat162float(ha), b - __bfloat162float(hb));
+}
+__device__ __forceinline__ void split8(const float (&v)[8], uint4 &hi, uint4 &lo)
+{
+    split_pair(v[0], v[1], hi.x, lo.x);
+    split_pair(v[2], v[3], hi.y, lo.y);
+    split_pair(v[4], v[5], hi.z, lo.z);
+    split_pair(v[6], v[7], hi.w, lo.w);
+}
+
 __device__ __forceinline__ float warp_sum(float v)
 {
 #pragma unroll

@@ -16,6 +16,11 @@
 //   warps 2..5  epilogue: tcgen05.ld of the accumulator (thread = weight row), then the
 //               operation's own ending: rotary embedding + cache append, residual add,
 //               SiLU(gate) * up, or logits + restricted arg max
+// The activation operand is carried as two bf16 terms, x = hi + lo with lo = bf16(x - hi), and
+// every weight tile is multiplied by both into the same accumulator: tcgen05 takes bf16 operands
+// only, and at random initialisation a single bf16 rounding of the activations early in the
+// stack is amplified by every later layer to 2-3 % at the exit of a 28-layer stack.  The second
+// product costs tensor time and L2 traffic, not HBM bytes.
 // Accumulators are double buffered in TMEM so a tile's epilogue overlaps the next tile's MMAs.
 // Every wait is bounded: on a timeout the CTA raises ST_TIMEOUT, stops issuing work, drains its
 // own copies, frees its TMEM and returns.
@@ -184,6 +189,7 @@ template <class Epi>
 __global__ void __launch_bounds__(GM_THREADS, 1)
     wsgemm_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
                   const __grid_constant__ CUtensorMap map_a2, const __grid_constant__ CUtensorMap map_b,
+                  const __grid_constant__ CUtensorMap map_b_lo,
                   const GemmArgs g, const Epi epi)
 {
     extern __shared__ __align__(1024) unsigned char gm_smem[];
@@ -196,7 +202,8 @@ __global__ void __launch_bounds__(GM_THREADS, 1)
     const uint32_t ring = (smem_u32(gm_smem) + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
     const int a_bytes = 2 * g.kb * GM_BLK_BYTES;                 // both accumulators' weights of a stage
     const int b_blk = g.box_n * GM_BK * 2;
-    const int stage_bytes = a_bytes + g.kb * b_blk;
+    const int b_half = g.kb * b_blk;                              // the hi tiles; the lo tiles follow
+    const int stage_bytes = a_bytes + 2 * b_half;
     // where accumulator a's rows of k-block j sit inside a stage
     const int a_blk_stride = g.pair ? GM_BLK_BYTES : 2 * GM_BLK_BYTES;
     const int a_acc_off = g.pair ? g.kb * GM_BLK_BYTES : GM_BLK_BYTES;
@@ -279,11 +286,11 @@ __global__ void __launch_bounds__(GM_THREADS, 1)
                 const uint32_t st = ring + (uint32_t)s * stage_bytes;
                 const int blk = ks * g.kb;
                 // lane 0: accumulator 0's weights (or the whole 256-row box); lane 1: accumulator 1's
-                // weights when they come from matrix 1; lane 2: the activations
-                const CUtensorMap *mp = lane == 0 ? ma : (lane == 1 ? &map_a1 : &map_b);
-                const uint32_t dst = lane == 0 ? st : (lane == 1 ? st + a_acc_off : st + a_bytes);
+                // weights when they come from matrix 1; lanes 2 and 3: the two terms of the activations
+                const CUtensorMap *mp = lane == 0 ? ma : (lane == 1 ? &map_a1 : (lane == 2 ? &map_b : &map_b_lo));
+                const uint32_t dst = lane == 0 ? st : (lane == 1 ? st + a_acc_off : st + a_bytes + (lane == 3 ? b_half : 0));
                 const int y = lane == 0 ? row : (lane == 1 ? g.row0[1] + unit_row : m0);
-                if (lane == 0 || lane == 2 || (lane == 1 && g.pair)) {
+                if (lane == 0 || lane == 2 || lane == 3 || (lane == 1 && g.pair)) {
                     if (g.three_d) tma_load_3d(dst, mp, &full_bar[s], 0, y, blk);
                     else tma_load_2d(dst, mp, &full_bar[s], blk * GM_BK, y);
                 }
@@ -322,9 +329,13 @@ __global__ void __launch_bounds__(GM_THREADS, 1)
 #pragma unroll
                         for (int kk = 0; kk < GM_BK / 16; kk++) {
                             const uint64_t db = umma_desc_sw128(b_addr + j * b_blk + kk * 32);
-                            const uint32_t a0 = a_addr + j * a_blk_stride + kk * 32;
-                            umma_bf16(d0, umma_desc_sw128(a0), db, idesc, accum);
-                            umma_bf16(d0 + mma_n, umma_desc_sw128(a0 + a_acc_off), db, idesc, accum);
+                            const uint64_t dl = umma_desc_sw128(b_addr + b_half + j * b_blk + kk * 32);
+                            const uint64_t da0 = umma_desc_sw128(a_addr + j * a_blk_stride + kk * 32);
+                            const uint64_t da1 = umma_desc_sw128(a_addr + j * a_blk_stride + kk * 32 + a_acc_off);
+                            umma_bf16(d0, da0, db, idesc, accum);
+                            umma_bf16(d0, da0, dl, idesc, 1);
+                            umma_bf16(d0 + mma_n, da1, db, idesc, accum);
+                            umma_bf16(d0 + mma_n, da1, dl, idesc, 1);
                             accum = 1;
                         }
                     }
@@ -374,7 +385,7 @@ __global__ void __launch_bounds__(GM_THREADS, 1)
 // buffer, k and v appended to the cache.  With the inner dimension cut across CTAs the partial
 // sums are added into an fp32 scratch [rows][Hq*hd + 2*Hkv*hd] and qkv_finish_kernel does the rest.
 struct QkvEnd {
-    bf16 *q_out;         // [rows][Hq*hd]
+    float *q_out;        // [rows][Hq*hd] fp32 (the attention kernels split it into two bf16 terms)
     bf16 *kc, *vc;       // this layer's cache [slot][Hkv][S][hd]
     const float2 *rope;  // [S][hd/2]
     const int *row_slot, *row_pos;
@@ -421,7 +432,7 @@ struct QkvEnd {
                             const float other = t.xchg[c * GM_BM + (t.row ^ half)];
                             const float2 cs = rope[(size_t)pos * half + j];
                             const float r = hi ? v[c] * cs.x + other * cs.y : v[c] * cs.x - other * cs.y;
-                            if (t.matrix == 0) q_out[(size_t)m * Hq * hd + n] = __float2bfloat16(r);
+                            if (t.matrix == 0) q_out[(size_t)m * Hq * hd + n] = r;
                             else kc[(((size_t)slot * Hkv + head) * S + pos) * hd + i] = __float2bfloat16(r);
                         }
                     }
@@ -435,7 +446,7 @@ struct QkvEnd {
 // Finishes a q/k/v product whose inner dimension was cut across CTAs: reads the summed row from
 // the scratch, applies the rotary embedding, writes q and appends k, v to the cache, and clears
 // the scratch for the next product.  One block per activation row.
-static __global__ void __launch_bounds__(256) qkv_finish_kernel(float *__restrict__ partial, bf16 *__restrict__ q_out,
+static __global__ void __launch_bounds__(256) qkv_finish_kernel(float *__restrict__ partial, float *__restrict__ q_out,
                                                          bf16 *__restrict__ kc, bf16 *__restrict__ vc,
                                                          const float2 *__restrict__ rope,
                                                          const int *__restrict__ row_slot,
@@ -455,10 +466,15 @@ static __global__ void __launch_bounds__(256) qkv_finish_kernel(float *__restric
         const float a = src[head * hd + j], b = src[head * hd + j + half];
         const float2 cs = rope[(size_t)pos * half + j];
         const float ra = a * cs.x - b * cs.y, rb = b * cs.x + a * cs.y;
-        bf16 *dst = head < Hq ? q_out + (size_t)m * Hq * hd + head * hd + j
-                              : kc + (((size_t)slot * Hkv + (head - Hq)) * S + pos) * hd + j;
-        dst[0] = __float2bfloat16(ra);
-        dst[half] = __float2bfloat16(rb);
+        if (head < Hq) {
+            float *dst = q_out + (size_t)m * Hq * hd + head * hd + j;
+            dst[0] = ra;
+            dst[half] = rb;
+        } else {
+            bf16 *dst = kc + (((size_t)slot * Hkv + (head - Hq)) * S + pos) * hd + j;
+            dst[0] = __float2bfloat16(ra);
+            dst[half] = __float2bfloat16(rb);
+        }
     }
     for (int i = threadIdx.x; i < Hkv * hd; i += blockDim.x)
         vc[(((size_t)slot * Hkv + i / hd) * S + pos) * hd + i % hd] = __float2bfloat16(src[(Hq + Hkv) * hd + i]);
@@ -494,7 +510,7 @@ struct ResidEnd {
 
 // u[m][f] = silu(gate) * up; accumulator 0 holds the gate rows, accumulator 1 the up rows.
 struct GateUpEnd {
-    bf16 *u;  // [rows][F]
+    bf16 *u, *u_lo;  // [rows][F]: u + u_lo carries the activation to 16 significant bits
     int F;
 
     __device__ void tile(const TileCtx &t) const
@@ -509,7 +525,10 @@ struct GateUpEnd {
             for (int c = 0; c < GM_CHUNK; c++) {
                 const int m = t.m0 + c0 + c;
                 if (m >= t.m_end) break;
-                u[(size_t)m * F + f] = __float2bfloat16(gt[c] / (1.f + __expf(-gt[c])) * up[c]);
+                const float val = gt[c] / (1.f + __expf(-gt[c])) * up[c];
+                const bf16 hi = __float2bfloat16(val);
+                u[(size_t)m * F + f] = hi;
+                u_lo[(size_t)m * F + f] = __float2bfloat16(val - __bfloat162float(hi));
             }
         }
     }
@@ -549,11 +568,11 @@ struct HeadEnd {
     }
 };
 
-// RMSNorm of selected fp32 rows into the bf16 activation matrix the GEMM reads:
-// x[i] = h[row_idx ? row_idx[i] : i] / sqrt(mean(h^2) + eps) * gain.
+// RMSNorm of selected fp32 rows into the activation matrices the GEMM reads, as two bf16 terms:
+// x + x_lo = h[row_idx ? row_idx[i] : i] / sqrt(mean(h^2) + eps) * gain.
 static __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const float *__restrict__ h, const bf16 *__restrict__ gain,
                                                            const int *__restrict__ row_idx, bf16 *__restrict__ x,
-                                                           int n_rows, int K, float eps)
+                                                           bf16 *__restrict__ x_lo, int n_rows, int K, float eps)
 {
     __shared__ float red[8];
     griddep_wait();
@@ -578,12 +597,12 @@ static __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const float *_
         const float4 b = *reinterpret_cast<const float4 *>(src + k + 4);
         float gn[8];
         unpack8(*reinterpret_cast<const uint4 *>(gain + k), gn);
-        uint4 o;
-        o.x = pack_bf16x2(a.x * inv * gn[0], a.y * inv * gn[1]);
-        o.y = pack_bf16x2(a.z * inv * gn[2], a.w * inv * gn[3]);
-        o.z = pack_bf16x2(b.x * inv * gn[4], b.y * inv * gn[5]);
-        o.w = pack_bf16x2(b.z * inv * gn[6], b.w * inv * gn[7]);
-        *reinterpret_cast<uint4 *>(x + (size_t)i * K + k) = o;
+        const float v[8] = {a.x * inv * gn[0], a.y * inv * gn[1], a.z * inv * gn[2], a.w * inv * gn[3],
+                            b.x * inv * gn[4], b.y * inv * gn[5], b.z * inv * gn[6], b.w * inv * gn[7]};
+        uint4 hi, lo;
+        split8(v, hi, lo);
+        *reinterpret_cast<uint4 *>(x + (size_t)i * K + k) = hi;
+        *reinterpret_cast<uint4 *>(x_lo + (size_t)i * K + k) = lo;
     }
 }
 

@@ -225,7 +225,7 @@ template <int R>
 struct QkvOp {
     struct State {};
     const bf16 *wq, *wk, *wv;
-    bf16 *q_out;              // [rows][Hq*hd]
+    float *q_out;             // [rows][Hq*hd] fp32
     bf16 *kc, *vc;            // this layer's cache: [slot][Hkv][S][hd]
     const float2 *rope;       // [S][hd/2] (cos, sin)
     const int *row_slot, *row_pos;
@@ -263,9 +263,9 @@ struct QkvOp {
                 const float a = v[p], b = v[P + p];
                 const float ra = a * cs.x - b * cs.y, rb = b * cs.x + a * cs.y;
                 if (isq) {
-                    bf16 *dst = q_out + (size_t)m * Hq * hd + head * hd + i0 + p;
-                    dst[0] = __float2bfloat16(ra);
-                    dst[half] = __float2bfloat16(rb);
+                    float *dst = q_out + (size_t)m * Hq * hd + head * hd + i0 + p;
+                    dst[0] = ra;
+                    dst[half] = rb;
                 } else {
                     bf16 *dst = kc + (((size_t)slot * Hkv + head) * S + pos) * hd + i0 + p;
                     dst[0] = __float2bfloat16(ra);

@@ -42,7 +42,7 @@ constexpr int MK_SLOT_BYTES = 2 * MK_BOX_BYTES;              // two boxes per sl
 constexpr int MK_SLOTS = 8;
 constexpr int MK_MAX_ROWS = 4;
 constexpr int MK_AREA_BYTES = 88 * 1024;        // shared memory behind the ring
-constexpr int MK_ATT_WARPS = 4;                 // consumer warps that run attention items
+constexpr int MK_ATT_WARPS = 3;                 // consumer warps that run attention items
 constexpr int MK_ATT_NST = 2;
 constexpr int MK_MAX_SPLITS = 16;
 
@@ -51,7 +51,7 @@ constexpr int MK_MAX_SPLITS = 16;
 // phase moves along), or the attention warps' query blocks and K/V rings.
 inline size_t mk_attn_bytes(int head_dim)
 {
-    return (size_t)MK_ATT_WARPS * (16 + MK_ATT_NST * 2 * AT_TP) * (head_dim + 8) * 2;
+    return (size_t)MK_ATT_WARPS * (2 * 16 + MK_ATT_NST * 2 * AT_TP) * (head_dim + 8) * 2;
 }
 // k-steps of M fp32 activation rows that fit the area
 __host__ __device__ inline int mk_act_window(int M) { return MK_AREA_BYTES / (M * MK_BOX_COLS * 4); }
@@ -71,7 +71,7 @@ struct MkArgs {
     float *h;                    // residual stream of the pass [rows][d]
     const int *row_slot, *row_pos, *grp_row0, *grp_nrows;
     int n_rows, n_groups;
-    bf16 *q_buf;                 // [rows][Hq*hd]
+    float *q_buf;                // [rows][Hq*hd]
     float *attn_o, *act;         // [rows][Hq*hd], [rows][F]
     float *part_o;
     float2 *part_ml;

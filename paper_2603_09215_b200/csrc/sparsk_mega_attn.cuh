@@ -6,16 +6,17 @@ namespace sparsk {
 // Items (group, query block, kv head, split) are dealt to MK_ATT_WARPS warps of every CTA; a warp
 // runs its item alone: 16 query vectors (query heads of the kv head, for the group's rows), its
 // own two-stage K/V ring inside the activation area, one partial per item.  The arithmetic is
-// that of attn_partial_kernel with one m16 tile.
+// that of attn_partial_kernel with one m16 tile (queries and softmax weights as two bf16 terms).
 template <int HD>
 __device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, unsigned char *area)
 {
     constexpr int KP = HD + 8, CH = HD / 8;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (warp >= MK_ATT_WARPS) return;
-    // per warp: its 16 query vectors, then the K/V ring
-    bf16 *Qs = reinterpret_cast<bf16 *>(area) + (size_t)warp * (16 + MK_ATT_NST * 2 * AT_TP) * KP;
-    bf16 *wr = Qs + 16 * KP;
+    // per warp: its 16 query vectors (hi and lo term), then the K/V ring
+    bf16 *Qs = reinterpret_cast<bf16 *>(area) + (size_t)warp * (2 * 16 + MK_ATT_NST * 2 * AT_TP) * KP;
+    bf16 *Ql = Qs + 16 * KP;
+    bf16 *wr = Ql + 16 * KP;
     const int G = a.Hq / a.Hkv;
     const int n_workers = gridDim.x * MK_ATT_WARPS, worker = warp * gridDim.x + blockIdx.x;
     int max_nq = 0;
@@ -45,12 +46,16 @@ __device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, 
         __syncwarp();
         for (int i = lane; i < 16 * CH; i += 32) {
             const int qi = i / CH, c = i % CH;
-            uint4 v = make_uint4(0, 0, 0, 0);
+            uint4 hi = make_uint4(0, 0, 0, 0), lo = hi;
             if (qi < nq_here) {
                 const int qg = q0 + qi, r = qg / G, j = qg % G;
-                v = *reinterpret_cast<const uint4 *>(a.q_buf + (size_t)(row0 + r) * a.Hq * HD + (hk * G + j) * HD + c * 8);
+                const float *src = a.q_buf + (size_t)(row0 + r) * a.Hq * HD + (hk * G + j) * HD + c * 8;
+                const float4 x0 = *reinterpret_cast<const float4 *>(src), x1 = *reinterpret_cast<const float4 *>(src + 4);
+                const float v[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+                split8(v, hi, lo);
             }
-            *reinterpret_cast<uint4 *>(&Qs[qi * KP + c * 8]) = v;
+            *reinterpret_cast<uint4 *>(&Qs[qi * KP + c * 8]) = hi;
+            *reinterpret_cast<uint4 *>(&Ql[qi * KP + c * 8]) = lo;
         }
         __syncwarp();
 
@@ -93,13 +98,16 @@ __device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, 
                 for (int e = 0; e < 4; e++) s[nt][e] = 0.f;
 #pragma unroll
             for (int ks = 0; ks < HD / 16; ks++) {
-                uint32_t kb[4], qa[4];
+                uint32_t kb[4], qa[4], ql[4];
                 ldsm_x4(kb, &Kt[((lane & 7) + ((lane >> 4) << 3)) * KP + ks * 16 + ((lane >> 3) & 1) * 8]);
                 ldsm_x4(qa, &Qs[((lane & 7) + ((lane >> 3) & 1) * 8) * KP + ks * 16 + (lane >> 4) * 8]);
+                ldsm_x4(ql, &Ql[((lane & 7) + ((lane >> 3) & 1) * 8) * KP + ks * 16 + (lane >> 4) * 8]);
                 mma_bf16(s[0], qa, kb[0], kb[1]);
                 mma_bf16(s[1], qa, kb[2], kb[3]);
+                mma_bf16(s[0], ql, kb[0], kb[1]);
+                mma_bf16(s[1], ql, kb[2], kb[3]);
             }
-            uint32_t pa[4];
+            uint32_t pa[4], pl[4];
 #pragma unroll
             for (int hf = 0; hf < 2; hf++) {
                 float v[4];
@@ -130,8 +138,8 @@ __device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, 
                 }
                 l_run[hf] = l_run[hf] * alpha + psum;
                 m_run[hf] = m_new;
-                pa[hf] = pack_bf16x2(v[0], v[1]);
-                pa[2 + hf] = pack_bf16x2(v[2], v[3]);
+                split_pair(v[0], v[1], pa[hf], pl[hf]);
+                split_pair(v[2], v[3], pa[2 + hf], pl[2 + hf]);
 #pragma unroll
                 for (int nt = 0; nt < HD / 8; nt++) {
                     o[nt][hf * 2] *= alpha;
@@ -144,6 +152,8 @@ __device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, 
                 ldsm_x4_t(vb, &Vt[((lane & 7) + ((lane >> 3) & 1) * 8) * KP + np * 16 + (lane >> 4) * 8]);
                 mma_bf16(o[2 * np], pa, vb[0], vb[1]);
                 mma_bf16(o[2 * np + 1], pa, vb[2], vb[3]);
+                mma_bf16(o[2 * np], pl, vb[0], vb[1]);
+                mma_bf16(o[2 * np + 1], pl, vb[2], vb[3]);
             }
             __syncwarp();  // the stage may be refilled by the next iteration's copies
         }

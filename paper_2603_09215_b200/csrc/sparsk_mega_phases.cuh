@@ -132,10 +132,15 @@ __device__ __forceinline__ bool mk_project(int type, const MkArgs &a, const MkLa
                     const int head = bb / per_head, i = (bb % per_head) * MK_BOX_ROWS + warp;
                     const float2 cs = a.rope[(size_t)pos * half + i];
                     const float ra = v0 * cs.x - v1 * cs.y, rb = v1 * cs.x + v0 * cs.y;
-                    bf16 *dst = isq ? a.q_buf + (size_t)m * a.Hq * a.hd + head * a.hd + i
-                                    : L->kc + (((size_t)slot_id * a.Hkv + head) * a.S + pos) * a.hd + i;
-                    dst[0] = __float2bfloat16(ra);
-                    dst[half] = __float2bfloat16(rb);
+                    if (isq) {
+                        float *dst = a.q_buf + (size_t)m * a.Hq * a.hd + head * a.hd + i;
+                        dst[0] = ra;
+                        dst[half] = rb;
+                    } else {
+                        bf16 *dst = L->kc + (((size_t)slot_id * a.Hkv + head) * a.S + pos) * a.hd + i;
+                        dst[0] = __float2bfloat16(ra);
+                        dst[half] = __float2bfloat16(rb);
+                    }
                 } else {
                     const int n0 = (b - nq - nk) * 2 * MK_BOX_ROWS + warp, n1 = n0 + MK_BOX_ROWS;
                     const int kvd = a.Hkv * a.hd;
