@@ -729,6 +729,7 @@ cudaError_t run_mega(sparsk_ctx *c, int l_begin, int l_end, float *h, const RowS
     int splits = c->attn_split > 0 ? (rs.max_len + c->attn_split - 1) / c->attn_split
                                    : (c->n_sm * MK_ATT_WARPS + base - 1) / base;
     splits = std::max(1, std::min(splits, std::min(MK_MAX_SPLITS, tiles)));
+    a.att_qblk = n_qblk;
     a.att_split_len = ((rs.max_len + splits - 1) / splits + AT_TP - 1) / AT_TP * AT_TP;
     a.att_splits = std::max(1, (rs.max_len + a.att_split_len - 1) / a.att_split_len);
     a.bar = c->mk_bar; a.bar_base = c->mk_bar_base; a.abort_word = c->mk_abort; a.status = c->sd.counts + CNT_STATUS;

@@ -44,7 +44,7 @@ constexpr int MK_MAX_ROWS = 4;
 constexpr int MK_AREA_BYTES = 88 * 1024;        // shared memory behind the ring
 constexpr int MK_ATT_WARPS = 3;                 // consumer warps that run attention items
 constexpr int MK_ATT_NST = 2;
-constexpr int MK_MAX_SPLITS = 16;
+constexpr int MK_MAX_SPLITS = 32;             // the merge keeps one split per lane
 
 // The area behind the ring holds the activations of a projection phase (M rows of bf16; when
 // M rows of the whole inner dimension do not fit, a window of k-steps that is reloaded as the
@@ -79,6 +79,7 @@ struct MkArgs {
     int d, Hq, Hkv, hd, F, S, n_slots;
     float eps;
     int att_splits, att_split_len;  // KV cut of the attention phase
+    int att_qblk;                   // blocks of 16 query vectors per group
     unsigned long long *bar;        // grid barrier counter (monotonic)
     unsigned long long bar_base;    // its value when this launch starts
     int *abort_word;                // nonzero: some CTA gave up
@@ -209,6 +210,7 @@ struct MkWalk {
 struct MkShared {
     uint64_t full[MK_SLOTS], empty[MK_SLOTS];
     int giving_up, never;
+    int row_slot[MK_MAX_ROWS], row_pos[MK_MAX_ROWS], grp_row0[MK_MAX_ROWS], grp_nrows[MK_MAX_ROWS];  // copies of the row set
     float red[MK_CW];
 };
 
@@ -218,8 +220,9 @@ __device__ __forceinline__ bool mk_grid_barrier(const MkArgs &a, MkShared *sh, u
     mk_consumer_sync();
     epoch += gridDim.x;
     if (threadIdx.x == 0) {
-        __threadfence();
-        atomicAdd(a.bar, 1ull);
+        // release: everything this CTA wrote (ordered before by the CTA barrier) is visible to
+        // whoever acquires the counter; no value comes back, so nothing waits on the round trip
+        asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(a.bar), "l"(1ull) : "memory");
         unsigned long long t0 = 0;
         for (uint32_t spin = 0;; ++spin) {
             if (ld_acquire_u64(a.bar) >= epoch) break;
@@ -238,7 +241,6 @@ __device__ __forceinline__ bool mk_grid_barrier(const MkArgs &a, MkShared *sh, u
                 }
             }
         }
-        __threadfence();
         if (blockIdx.x == 0 && a.trace) a.trace[(epoch - a.bar_base) / gridDim.x] = global_ns();
     }
     mk_consumer_sync();

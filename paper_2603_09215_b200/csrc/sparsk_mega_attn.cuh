@@ -8,7 +8,7 @@ namespace sparsk {
 // own two-stage K/V ring inside the activation area, one partial per item.  The arithmetic is
 // that of attn_partial_kernel with one m16 tile (queries and softmax weights as two bf16 terms).
 template <int HD>
-__device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, unsigned char *area)
+__device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, unsigned char *area, const MkShared *sh)
 {
     constexpr int KP = HD + 8, CH = HD / 8;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -19,9 +19,7 @@ __device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, 
     bf16 *wr = Ql + 16 * KP;
     const int G = a.Hq / a.Hkv;
     const int n_workers = gridDim.x * MK_ATT_WARPS, worker = warp * gridDim.x + blockIdx.x;
-    int max_nq = 0;
-    for (int g = 0; g < a.n_groups; g++) max_nq = max(max_nq, a.grp_nrows[g] * G);
-    const int n_qblk = (max_nq + 15) / 16;
+    const int n_qblk = a.att_qblk;
     const int n_items = a.n_groups * n_qblk * a.Hkv * a.att_splits;
     const float scale = rsqrtf((float)HD);
     for (int item = worker; item < n_items; item += n_workers) {
@@ -29,11 +27,11 @@ __device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, 
         const int sp = t % a.att_splits; t /= a.att_splits;
         const int hk = t % a.Hkv; t /= a.Hkv;
         const int qb = t % n_qblk, g = t / n_qblk;
-        const int row0 = a.grp_row0[g], nrows = a.grp_nrows[g];
+        const int row0 = sh->grp_row0[g], nrows = sh->grp_nrows[g];
         const int nq = nrows * G, q0 = qb * 16;
         if (row0 < 0 || nrows < 1 || row0 + nrows > a.n_rows || q0 >= nq) continue;
         const int nq_here = min(16, nq - q0);
-        const int slot = a.row_slot[row0], pos0 = a.row_pos[row0];
+        const int slot = sh->row_slot[row0], pos0 = sh->row_pos[row0];
         const bool sane = slot >= 0 && slot < a.n_slots && pos0 >= 0;
         const int last_row = (q0 + nq_here - 1) / G;
         const int kv_end_all = sane ? min(pos0 + last_row + 1, a.S) : 0;
@@ -42,22 +40,6 @@ __device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, 
         const int n_tiles = w_end > w_beg ? (w_end - w_beg + AT_TP - 1) / AT_TP : 0;
         const bf16 *kbase = L->kc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
         const bf16 *vbase = L->vc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
-
-        __syncwarp();
-        for (int i = lane; i < 16 * CH; i += 32) {
-            const int qi = i / CH, c = i % CH;
-            uint4 hi = make_uint4(0, 0, 0, 0), lo = hi;
-            if (qi < nq_here) {
-                const int qg = q0 + qi, r = qg / G, j = qg % G;
-                const float *src = a.q_buf + (size_t)(row0 + r) * a.Hq * HD + (hk * G + j) * HD + c * 8;
-                const float4 x0 = *reinterpret_cast<const float4 *>(src), x1 = *reinterpret_cast<const float4 *>(src + 4);
-                const float v[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-                split8(v, hi, lo);
-            }
-            *reinterpret_cast<uint4 *>(&Qs[qi * KP + c * 8]) = hi;
-            *reinterpret_cast<uint4 *>(&Ql[qi * KP + c * 8]) = lo;
-        }
-        __syncwarp();
 
         auto issue = [&](int tt) {
             bf16 *kt = wr + (size_t)(tt % MK_ATT_NST) * 2 * AT_TP * KP, *vt = kt + AT_TP * KP;
@@ -84,10 +66,27 @@ __device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, 
         }
         if (n_tiles > 0) issue(0);
         cp_async_commit();
+        if (n_tiles > 1) issue(1);
+        cp_async_commit();
+        // the queries, while the first tiles are on their way
+        __syncwarp();
+        for (int i = lane; i < 16 * CH; i += 32) {
+            const int qi = i / CH, c = i % CH;
+            uint4 hi = make_uint4(0, 0, 0, 0), lo = hi;
+            if (qi < nq_here) {
+                const int qg = q0 + qi, r = qg / G, j = qg % G;
+                const float *src = a.q_buf + (size_t)(row0 + r) * a.Hq * HD + (hk * G + j) * HD + c * 8;
+                const float4 x0 = *reinterpret_cast<const float4 *>(src), x1 = *reinterpret_cast<const float4 *>(src + 4);
+                const float v[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+                split8(v, hi, lo);
+            }
+            *reinterpret_cast<uint4 *>(&Qs[qi * KP + c * 8]) = hi;
+            *reinterpret_cast<uint4 *>(&Ql[qi * KP + c * 8]) = lo;
+        }
+        __syncwarp();
+
         for (int tt = 0; tt < n_tiles; tt++) {
-            if (tt + 1 < n_tiles) issue(tt + 1);
-            cp_async_commit();
-            cp_async_wait<1>();
+            cp_async_wait<1>();  // all but the newest group: tile tt has landed
             __syncwarp();
             const bf16 *Kt = wr + (size_t)(tt % MK_ATT_NST) * 2 * AT_TP * KP, *Vt = Kt + AT_TP * KP;
             const int p0 = w_beg + tt * AT_TP;
@@ -155,7 +154,9 @@ __device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, 
                 mma_bf16(o[2 * np], pl, vb[0], vb[1]);
                 mma_bf16(o[2 * np + 1], pl, vb[2], vb[3]);
             }
-            __syncwarp();  // the stage may be refilled by the next iteration's copies
+            __syncwarp();  // everyone is done with this stage: refill it with the tile after next
+            if (tt + 2 < n_tiles) issue(tt + 2);
+            cp_async_commit();
         }
         cp_async_wait<0>();
         // this item's partial
@@ -178,34 +179,29 @@ __device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, 
     }
 }
 
-// Merge of the splits: one warp per (row, query head); lane s holds split s's weight, lanes own
-// HD/32 output dims.  att_splits <= 32.
+// Merge of the splits: one warp per (row, query head, 32 output dims).  Lane s holds split s's
+// weight (att_splits <= 32); every lane owns one output dim and has all its loads in flight at once.
 template <int HD>
 __device__ __forceinline__ void mk_merge(const MkArgs &a)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    constexpr int DL = HD / 32;
-    const int n_items = a.n_rows * a.Hq;
+    constexpr int PARTS = HD / 32;
+    const int n_items = a.n_rows * a.Hq * PARTS;
     for (int item = warp * gridDim.x + blockIdx.x; item < n_items; item += gridDim.x * MK_CW) {
-        const size_t cell0 = (size_t)item * a.att_splits;
+        const int cell = item / PARTS, d = (item % PARTS) * 32 + lane;
+        const size_t cell0 = (size_t)cell * a.att_splits;
         float2 ml = make_float2(-INFINITY, 0.f);
         if (lane < a.att_splits) ml = a.part_ml[cell0 + lane];
+        float v[MK_MAX_SPLITS];
+#pragma unroll
+        for (int s = 0; s < MK_MAX_SPLITS; s++) v[s] = s < a.att_splits ? a.part_o[(cell0 + s) * HD + d] : 0.f;
         const float M = warp_max(ml.x);
         const float w_mine = ml.x == -INFINITY ? 0.f : __expf(ml.x - M);
         const float den = warp_sum(ml.y * w_mine);
-        float num[DL];
+        float num = 0.f;
 #pragma unroll
-        for (int e = 0; e < DL; e++) num[e] = 0.f;
-#pragma unroll 4
-        for (int s = 0; s < a.att_splits; s++) {
-            const float w = __shfl_sync(0xffffffffu, w_mine, s);
-            const float *po = a.part_o + (cell0 + s) * HD + lane * DL;
-#pragma unroll
-            for (int e = 0; e < DL; e++) num[e] += po[e] * w;
-        }
-        float *dst = a.attn_o + (size_t)item * HD + lane * DL;
-#pragma unroll
-        for (int e = 0; e < DL; e++) dst[e] = den > 0.f ? num[e] / den : 0.f;
+        for (int s = 0; s < MK_MAX_SPLITS; s++) num += v[s] * __shfl_sync(0xffffffffu, w_mine, s);
+        a.attn_o[(size_t)cell * HD + d] = den > 0.f ? num / den : 0.f;
     }
 }
 

@@ -70,6 +70,12 @@ __global__ void __launch_bounds__(MK_THREADS, 1) mega_kernel(const MkArgs a)
         }
         sh.giving_up = 0;
         sh.never = 0;
+        for (int i = 0; i < MK_MAX_ROWS; i++) {
+            sh.row_slot[i] = i < a.n_rows ? a.row_slot[i] : -1;
+            sh.row_pos[i] = i < a.n_rows ? a.row_pos[i] : -1;
+            sh.grp_row0[i] = i < a.n_groups ? a.grp_row0[i] : -1;
+            sh.grp_nrows[i] = i < a.n_groups ? a.grp_nrows[i] : 0;
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -121,7 +127,7 @@ __global__ void __launch_bounds__(MK_THREADS, 1) mega_kernel(const MkArgs a)
             if (!(ok = mk_project<M>(MK_QKV, a, L, act, a.d, a.h, nullptr, L->attn_gain, ring, &sh, it))) break;
             if (!(ok = mk_grid_barrier(a, &sh, epoch))) break;
             // attention and the merge of its splits
-            mk_attention<HD>(a, L, area);
+            mk_attention<HD>(a, L, area, &sh);
             if (!(ok = mk_grid_barrier(a, &sh, epoch))) break;
             mk_merge<HD>(a);
             if (!(ok = mk_grid_barrier(a, &sh, epoch))) break;

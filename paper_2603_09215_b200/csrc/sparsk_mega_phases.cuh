@@ -125,7 +125,7 @@ __device__ __forceinline__ bool mk_project(int type, const MkArgs &a, const MkLa
             switch (type) {
             case MK_QKV: {
                 const int nq = a.Hq * per_head, nk = a.Hkv * per_head;
-                const int slot_id = a.row_slot[m], pos = a.row_pos[m];
+                const int slot_id = sh->row_slot[m], pos = sh->row_pos[m];
                 if (b < nq + nk) {
                     const bool isq = b < nq;
                     const int bb = isq ? b : b - nq;
