@@ -157,7 +157,7 @@ class Runner:
         self.pend = [0] * B
         self.depth_log = []     # (modality, depth) per emitted token
         self.bytes = 0
-        self.mega_layers = 0    # layer passes that ran inside the persistent kernel (passes of <= 4 rows)
+        self.mega_layers = 0    # layer passes that ran inside the persistent kernel (passes of <= 2 rows)
         self.mega_bytes = 0     # their weight and cache bytes
 
     def _fill_synthetic(self, prompts):
@@ -179,11 +179,11 @@ class Runner:
         self.bytes += step_bytes(d, depths, mods, self.lens, self.pend)
         kvb = 2 * d["n_kv_heads"] * d["head_dim"] * 2
         wl = layer_weight_bytes(d)
-        if len(depths) <= 4:
+        if len(depths) <= 2:
             self.mega_layers += e
             self.mega_bytes += e * (wl + sum((ln + 2) * kvb for ln in self.lens))
         up = [(ln, pn) for dep, ln, pn in zip(depths, self.lens, self.pend) if dep == L and e < L]
-        if up and sum(pn + 1 for _, pn in up) <= 4:
+        if up and sum(pn + 1 for _, pn in up) <= 2:
             self.mega_layers += L - e
             self.mega_bytes += (L - e) * (wl + sum((ln + 1) * kvb + (pn + 1) * kvb for ln, pn in up))
         for i, dep in enumerate(depths):

@@ -92,7 +92,7 @@ struct sparsk_ctx {
     unsigned long long *mk_trace;  // device [1 + 6 L]
     int mk_trace_n;                // entries the last launch wrote
     unsigned long long mk_bar_base;
-    int mega, mk_ok, mk_coop;
+    int mega, mk_ok, mk_coop, mk_max_rows;
     std::vector<MkLayer> mk_host;
     float *qkv_part;  // fp32 sums of a q/k/v product whose inner dimension is cut across CTAs
     int tc_kb;        // 0: automatic; 1: force one k-block per copy (2-D descriptors)
@@ -595,6 +595,7 @@ cudaError_t run_layer_tc(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
 
 bool use_tc(const sparsk_ctx *c, int n_rows) { return c->tc_ok && n_rows >= c->gemm_min_rows && c->dm.d_model >= GM_BK; }
 
+
 // Head of `layer` over list `l` on the tensor-core path.
 cudaError_t run_head_tc(sparsk_ctx *c, int layer, const float *h, int list, int n_rows)
 {
@@ -672,7 +673,7 @@ size_t mega_smem(const sparsk_dims &) { return (size_t)MK_SLOTS * MK_SLOT_BYTES 
 // Can a pass of n_rows rows go through the persistent kernel?
 bool use_mega(const sparsk_ctx *c, int n_rows)
 {
-    return c->mega && c->mk_ok && c->mk_coop && n_rows >= 1 && n_rows <= MK_MAX_ROWS &&
+    return c->mega && c->mk_ok && c->mk_coop && n_rows >= 1 && n_rows <= c->mk_max_rows &&
            mk_attn_bytes(c->dm.head_dim) <= MK_AREA_BYTES && c->dm.head_dim % (2 * MK_BOX_ROWS) == 0;
 }
 
@@ -840,9 +841,10 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
     carve(ctx, &ctx->dm, (char *)workspace);
     ctx->h_len.assign(dims->max_seqs, 0);
     ctx->h_pend.assign(dims->max_seqs, 0);
-    ctx->pdl = 0; ctx->attn_split = 0; ctx->gemm_min_rows = 5; ctx->use_graph = 0;
+    ctx->pdl = 0; ctx->attn_split = 0; ctx->gemm_min_rows = 3; ctx->use_graph = 0;
     ctx->tc_ok = false;
     ctx->tc_kb = 0;
+    ctx->mk_max_rows = 2;
     ctx->mega = 1; ctx->mk_ok = 0; ctx->mk_coop = 0; ctx->mk_bar_base = 0; ctx->mk_trace_n = 0;
     ctx->gv_ks = 0; ctx->gv_r = 0; ctx->gv_grid_mult = 1;
     ctx->dbg_hidden = nullptr; ctx->dbg_logits = nullptr;
@@ -940,6 +942,7 @@ extern "C" int sparsk_set_option(sparsk_ctx *ctx, const char *name, int64_t valu
     else if (!strcmp(name, "attn_split") && value >= 0 && value <= (1 << 24)) ctx->attn_split = (int)value;
     else if (!strcmp(name, "gemv_ks") && (value == 0 || value == 1 || value == 2 || value == 4 || value == 8 || value == 16)) ctx->gv_ks = (int)value;
     else if (!strcmp(name, "mega") && (value == 0 || value == 1)) ctx->mega = (int)value;
+    else if (!strcmp(name, "mega_max_rows") && value >= 1 && value <= MK_MAX_ROWS) ctx->mk_max_rows = (int)value;
     else if (!strcmp(name, "gemm_kb") && (value == 0 || value == 1)) ctx->tc_kb = (int)value;
     else if (!strcmp(name, "gemv_r") && (value == 0 || value == 1 || value == 2 || value == 4)) ctx->gv_r = (int)value;
     else if (!strcmp(name, "time_kernel") && value >= 0 && value <= KC_MEGA) {

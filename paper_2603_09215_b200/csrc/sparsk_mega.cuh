@@ -10,8 +10,10 @@
 //     boundaries.  Producer p owns the ring slots p and p + 4 and cycles them on its own (one
 //     thread needs a few hundred nanoseconds per copy, so four run side by side).  The ring is
 //     what keeps HBM streaming while the consumers sit in a barrier or in the attention phases.
-//     (Asking the L2 for boxes further ahead, with tensor or bulk prefetches, from the producers
-//     or from a warp of its own, was measured and made every phase slower, gate/up by 30-80 %.)
+//     (Asking the L2 for weights further ahead was measured in three forms and lost each time:
+//     tensor or bulk prefetches running ahead of the copies made every phase slower, gate/up by
+//     30-80 %; a burst for the next gate/up bands during the attention phases delayed the
+//     attention's own cache reads by as much as it later saved.)
 //   * warps 0..15 are consumers.  Per layer they run six phases separated by grid-wide barriers:
 //     RMSNorm + q/k/v + rotary embedding + cache append; attention partials; merge of the
 //     splits; O-projection + residual; RMSNorm + gate/up + SiLU; down-projection + residual.

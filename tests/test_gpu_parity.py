@@ -42,7 +42,7 @@ def test_config1_tiny_full_run(util):
     P.close()
 
 
-@pytest.mark.parametrize("min_rows", [5, 1])
+@pytest.mark.parametrize("min_rows", [3, 1])
 @pytest.mark.parametrize("e,K,r,nt,ns", [(1, 2, 0, 1, 4), (2, 4, 1, 2, 7), (3, 2, 0, 1, 4), (2, 1, 0, 1, 4),
                                           (1, 5, 4, 0, 9)])
 def test_odd_shapes_and_schedules(util, e, K, r, nt, ns, min_rows):
@@ -60,11 +60,11 @@ def test_odd_shapes_and_schedules(util, e, K, r, nt, ns, min_rows):
     P.close()
 
 
-@pytest.mark.parametrize("min_rows", [5, 1, 1 << 30])
+@pytest.mark.parametrize("min_rows", [3, 1, 1 << 30])
 def test_heterogeneous_batch_matches_per_sequence_oracle(util, min_rows):
     """Batch of 7 with random interleave phases and counter offsets and ragged prompts, so every
     step mixes text, early-exit and refresh rows; sequences stay independent.  Run with the
-    default hand-over between the small-batch and the tensor-core path (5 rows), with every
+    default hand-over between the small-batch and the tensor-core path (3 rows), with every
     projection on the tensor cores, and with every projection on the small-batch path."""
     dims = synth.model_dims("tiny", 2, 4, 0)
     w = synth.make_weights(dims, seed=0)
