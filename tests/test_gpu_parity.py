@@ -173,3 +173,22 @@ def test_host_step_and_error_codes(util):
     with pytest.raises(binding.SparskError) as ei:
         binding.Sparsk(d2, gw, 1, 16, 2)
     assert ei.value.code == binding.ENOHEAD
+
+
+@pytest.mark.parametrize("options", [{"mega": 0}, {"mega_max_rows": 4}, {"mega_max_rows": 1, "gemm_min_rows": 2},
+                                     {"mega": 0, "gemm_min_rows": 1 << 30}, {"gemm_kb": 1, "mega": 0, "gemm_min_rows": 1}])
+def test_every_route_for_small_passes(util, options):
+    """Passes of 1..4 rows (K = 4: flushes of up to three pending rows) through each of the three
+    implementations: the persistent kernel (also with its moving activation window at 3-4 rows),
+    the tensor-core path (with 2-D descriptors too) and the small-batch kernels."""
+    dims = synth.model_dims("tiny", 2, 4, 0)
+    w = synth.make_weights(dims, seed=0)
+    prompt = synth.make_prompts(dims, 1, 21, 21, seed=11)[0]
+    P = util.Pair(dims, w, 1, 96, 3, prefill_rows=16, options=options)
+    P.prefill([prompt])
+    for g in range(25):
+        m, c = synth.interleave(g, 1, 4)
+        P.step([m], [c])
+    ln, pend = P.g.slot_state(0)
+    P.check_cache(0, range(1, 5), ln - pend)
+    P.close()
