@@ -158,7 +158,7 @@ int sparsk_set_debug(sparsk_ctx *ctx, float *exit_hidden /*device or NULL*/,
  * largest pass that kernel takes; default 2, above which its CUDA-core inner loop falls behind
  * HBM), "gemm_kb" (1: one 64-element block of the inner
  * dimension per TMA copy instead of two; 0 = automatic), "use_graph" (0/1), "attn_split" (positions
- * per KV split), "pdl" (0/1, programmatic dependent launch between the kernels of a step),
+ * per KV split), "pdl" (0/1, programmatic dependent launch between the kernels of a step; default 1),
  * "gemv_ks" / "gemv_r" (override the GEMV team width / rows per group; 0 = automatic),
  * "time_kernel" (see sparsk_kernel_time).  Returns SPARSK_EINVAL for an unknown name or value. */
 int sparsk_set_option(sparsk_ctx *ctx, const char *name /*host*/, int64_t value);

@@ -841,7 +841,7 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
     carve(ctx, &ctx->dm, (char *)workspace);
     ctx->h_len.assign(dims->max_seqs, 0);
     ctx->h_pend.assign(dims->max_seqs, 0);
-    ctx->pdl = 0; ctx->attn_split = 0; ctx->gemm_min_rows = 3; ctx->use_graph = 0;
+    ctx->pdl = 1; ctx->attn_split = 0; ctx->gemm_min_rows = 3; ctx->use_graph = 0;
     ctx->tc_ok = false;
     ctx->tc_kb = 0;
     ctx->mk_max_rows = 2;

@@ -195,6 +195,7 @@ static __global__ void finish_kernel(StepDesc sd, int n, int *__restrict__ kv_le
 static __global__ void debug_hidden_kernel(StepDesc sd, const float *__restrict__ h_lo,
                                     const float *__restrict__ h_up, float *__restrict__ out, int n, int d)
 {
+    griddep_wait();
     const int b = blockIdx.x;
     if (b >= n) return;
     const int cr = sd.cur_row[b];
@@ -203,6 +204,7 @@ static __global__ void debug_hidden_kernel(StepDesc sd, const float *__restrict_
 }
 static __global__ void fill_kernel(float *__restrict__ p, size_t n, float v)
 {
+    griddep_wait();
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
         p[i] = v;
 }
@@ -212,6 +214,7 @@ static __global__ void prefill_rows_kernel(int *__restrict__ row_slot, int *__re
                                     int *__restrict__ grp_row0, int *__restrict__ grp_nrows, int slot,
                                     int pos0, int n)
 {
+    griddep_wait();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i == 0) {
         grp_row0[0] = 0;
@@ -222,12 +225,17 @@ static __global__ void prefill_rows_kernel(int *__restrict__ row_slot, int *__re
         row_pos[i] = pos0 + i;
     }
 }
-static __global__ void set_int_kernel(int *p, int v) { *p = v; }
+static __global__ void set_int_kernel(int *p, int v)
+{
+    griddep_wait();
+    *p = v;
+}
 
 // Cache import/export: [n][Hkv*hd] <-> [Hkv][S][hd] of one (layer, slot).
 static __global__ void kv_copy_kernel(bf16 *__restrict__ cache_k, bf16 *__restrict__ cache_v, bf16 *ext_k,
                                bf16 *ext_v, int first_pos, int n, int Hkv, int hd, int S, int to_cache)
 {
+    griddep_wait();
     const size_t total = (size_t)n * Hkv * hd;
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total;
          i += (size_t)gridDim.x * blockDim.x) {
