@@ -245,7 +245,9 @@ __global__ void __launch_bounds__(GM_THREADS, 1)
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_s;
 
-    griddep_wait();
+    // Weights depend on no earlier kernel, activations and outputs do: the producer starts the
+    // first weight copies before it waits for the grid dependency, the epilogue waits before it
+    // touches anything, the MMA warp touches no global memory.
     griddep_launch();
 
     // unit u -> (matrix, first row, split)
@@ -267,6 +269,10 @@ __global__ void __launch_bounds__(GM_THREADS, 1)
         // slot and posts the byte count, then lanes 0..2 each issue one box.
         uint32_t it = 0;
         bool ok = true;
+        // pass 0 fills the ring's first round with weights only, then waits for the grid
+        // dependency; pass 1 is the whole loop, adding only the activations to those stages
+        for (int pass = 0; pass < 2 && ok; pass++) {
+        it = 0;
         for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
             int mat, unit_row, sp;
             locate(u, mat, unit_row, sp);
@@ -274,10 +280,12 @@ __global__ void __launch_bounds__(GM_THREADS, 1)
             const int row = g.row0[mat] + unit_row;
             const int ks_beg = (int)((long)k_stages * sp / g.splits), ks_end = (int)((long)k_stages * (sp + 1) / g.splits);
             for (int ks = ks_beg; ks < ks_end; ks++, it++) {
+                if (pass == 0 && it >= (uint32_t)g.stages) break;
+                const bool early = it < (uint32_t)g.stages;  // its weights went out in pass 0
                 const int s = it % g.stages;
                 const uint32_t ph = (it / g.stages) & 1;
                 int go = 1;
-                if (lane == 0) {
+                if (lane == 0 && !(pass == 1 && early)) {
                     go = mbar_wait(&empty_bar[s], ph ^ 1, giving_up, g.status) ? 1 : 0;
                     if (go) mbar_expect_tx(&full_bar[s], (uint32_t)stage_bytes);
                 }
@@ -290,11 +298,15 @@ __global__ void __launch_bounds__(GM_THREADS, 1)
                 const CUtensorMap *mp = lane == 0 ? ma : (lane == 1 ? &map_a1 : (lane == 2 ? &map_b : &map_b_lo));
                 const uint32_t dst = lane == 0 ? st : (lane == 1 ? st + a_acc_off : st + a_bytes + (lane == 3 ? b_half : 0));
                 const int y = lane == 0 ? row : (lane == 1 ? g.row0[1] + unit_row : m0);
-                if (lane == 0 || lane == 2 || lane == 3 || (lane == 1 && g.pair)) {
+                const bool weights = lane == 0 || (lane == 1 && g.pair), acts = lane == 2 || lane == 3;
+                if ((weights && !(pass == 1 && early)) || (acts && pass == 1)) {
                     if (g.three_d) tma_load_3d(dst, mp, &full_bar[s], 0, y, blk);
                     else tma_load_2d(dst, mp, &full_bar[s], blk * GM_BK, y);
                 }
             }
+            if (pass == 0 && it >= (uint32_t)g.stages) break;
+        }
+        if (pass == 0) griddep_wait();
         }
         if (!ok && lane == 0) {
             // giving up: let the copies already issued land (2 ms each at most) before the CTA
@@ -346,6 +358,7 @@ __global__ void __launch_bounds__(GM_THREADS, 1)
         }
     } else {
         // ------------------------------------------------------------ epilogue (warps 2..5)
+        griddep_wait();
         const int quad = warp & 3;  // TMEM lanes this warp may read: 32 quad .. 32 quad + 31
         TileCtx tc;
         tc.row = quad * 32 + lane;
