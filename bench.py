@@ -28,7 +28,7 @@ if ROOT not in sys.path:
 
 from paper_2603_09215_b200 import synth  # noqa: E402
 
-KC = {"qkv": 1, "attn": 2, "oproj": 3, "gateup": 4, "down": 5, "head": 6, "mega": 7}
+KC = {"qkv": 1, "attn": 2, "oproj": 3, "gateup": 4, "down": 5, "head": 6, "mega": 7, "all": 8}
 
 
 # --------------------------------------------------------------------------- byte model
@@ -108,8 +108,12 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------- workload
-def workload_setup(name, rank):
+def workload_setup(name, rank, exit_layer=None, period=None):
     wl = dict(synth.WORKLOADS[name])
+    if exit_layer is not None:
+        wl["exit_layer"] = exit_layer
+    if period is not None:
+        wl["refresh_period"] = period
     dims = synth.model_dims(wl["shape"], wl["exit_layer"], wl["refresh_period"], wl["refresh_phase"])
     B = wl["batch"]
     prompts = synth.make_prompts(dims, B, wl["prompt"][0], wl["prompt"][1], seed=1 + 1000 * rank,
@@ -268,11 +272,13 @@ def main():
     ap.add_argument("--no-full-depth", action="store_true")
     ap.add_argument("--option", action="append", default=[], help="library option name=value")
     ap.add_argument("--time-kernel", default="mega", choices=sorted(KC))
+    ap.add_argument("--exit-layer", type=int, default=None, help="override the workload's exit layer e (sweep cells)")
+    ap.add_argument("--period", type=int, default=None, help="override the workload's refresh period K (sweep cells)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     W = max(args.warmup, 3)
-    wl, dims, prompts, phi, off = workload_setup(args.workload, rank)
+    wl, dims, prompts, phi, off = workload_setup(args.workload, rank, args.exit_layer, args.period)
     cyc = wl["n_text"] + wl["n_speech"]
     L = dims["n_layers"]
     cfg = {"workload": args.workload, "shape": wl["shape"], "batch_per_gpu": wl["batch"],
@@ -383,6 +389,11 @@ def main():
     ml0, mb0 = run.mega_layers, run.mega_bytes
     run.run_cycles(min(args.steps, 8))
     kms, kn = run.ctx.kernel_time()
+    classes = None
+    if kname == "all":
+        n_steps = min(args.steps, 8) * cyc
+        classes = {k: {"ms_per_decode_step": v[0] / n_steps, "launches_per_decode_step": v[1] / n_steps}
+                   for k, v in run.ctx.kernel_time_by_class().items() if v[1]}
     run.ctx.set_option("time_kernel", 0)
     d = dims
     kbytes = {"gateup": 2 * d["d_ffn"] * d["d_model"] * 2, "down": d["d_ffn"] * d["d_model"] * 2,
@@ -429,6 +440,8 @@ def main():
                         "frac_of_measured_copy": step_b / (ms * 1e-3) / 1e9 / hbm_peak,
                         "frac_of_nominal_8tbs": step_b / (ms * 1e-3) / 1e9 / 8000.0},
            "layer_saving": sav, "setup_s": setup_s}
+    if classes:
+        out["kernel_classes"] = classes
     if full:
         out["full_depth"] = full
         out["reduction"] = {"wall_time_pct": (1 - (ms / args.steps) / full["ms_per_step"]) * 100,

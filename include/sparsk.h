@@ -208,11 +208,15 @@ int sparsk_attention_static(const sparsk_attn_args *args /*host*/, void *cuda_st
                             size_t err_len);
 
 /* Per-kernel timing for roofline reports.  sparsk_set_option(ctx, "time_kernel", c) with c =
- * 1 QKV, 2 attention, 3 O-projection, 4 gate/up, 5 down-projection, 6 exit head, 7 persistent layer-range kernel brackets every
- * later launch of that class with CUDA events on the context's stream (up to 8192 launches; 0
+ * 1 QKV, 2 attention, 3 O-projection, 4 gate/up, 5 down-projection, 6 exit head, 7 persistent layer-range kernel (8: all of them, see sparsk_kernel_time_by_class) brackets every
+ * later launch of that class with CUDA events on the context's stream (up to 16384 launches; 0
  * stops).  sparsk_kernel_time synchronises the stream and returns the summed device time of the
  * bracketed launches and their number.  No counterpart in the paper: measurement only. */
 int sparsk_kernel_time(sparsk_ctx *ctx, double *total_ms /*host*/, int64_t *n_launches /*host*/);
+/* With "time_kernel" = 8 every launch is bracketed and remembered with its class; this returns
+ * the summed device time and the launch count of each class, indexed 0 bookkeeping (schedule,
+ * compaction, embedding, norms, stash, gather, finish), 1..7 as above.  Arrays of 8. */
+int sparsk_kernel_time_by_class(sparsk_ctx *ctx, double *total_ms /*host [8]*/, int64_t *n_launches /*host [8]*/);
 
 /* Synchronises the context's stream, then reads and clears the device status word that kernels
  * raise instead of trapping: SPARSK_ETIMEOUT if a bounded in-kernel wait ran out, SPARSK_EINVAL

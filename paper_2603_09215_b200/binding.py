@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libsparsk.so")
 EXPORTS = ("sparsk_workspace_bytes", "sparsk_create", "sparsk_prefill", "sparsk_decode_step",
            "sparsk_decode_step_host", "sparsk_reset_slot", "sparsk_import_kv", "sparsk_export_kv",
            "sparsk_set_len", "sparsk_slot_state", "sparsk_set_debug", "sparsk_set_option",
-           "sparsk_kernel_time", "sparsk_check", "sparsk_phase_trace", "sparsk_attention", "sparsk_attention_scratch_bytes", "sparsk_attention_static", "sparsk_launch_count", "sparsk_last_error", "sparsk_destroy")
+           "sparsk_kernel_time", "sparsk_kernel_time_by_class", "sparsk_check", "sparsk_phase_trace", "sparsk_attention", "sparsk_attention_scratch_bytes", "sparsk_attention_static", "sparsk_launch_count", "sparsk_last_error", "sparsk_destroy")
 
 OK, EINVAL, ECAPACITY, ENOHEAD, ECUDA, ESTATE, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
 
@@ -100,6 +100,8 @@ def load():
     L.sparsk_attention_static.argtypes = [C.POINTER(AttnArgs), vp, C.c_char_p, C.c_size_t]
     L.sparsk_phase_trace.restype = C.c_int
     L.sparsk_phase_trace.argtypes = [vp, C.POINTER(C.c_int64), C.c_int32]
+    L.sparsk_kernel_time_by_class.restype = C.c_int
+    L.sparsk_kernel_time_by_class.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     L.sparsk_check.restype = C.c_int
     L.sparsk_check.argtypes = [vp]
     L.sparsk_launch_count.restype = C.c_int64
@@ -303,6 +305,13 @@ class Sparsk:
     def check(self):
         """Synchronise, then raise if a kernel reported a problem through the device status word."""
         self._check(self.lib.sparsk_check(self.h))
+
+    def kernel_time_by_class(self):
+        """{class name: (summed ms, launches)} of the launches bracketed since time_kernel was set to 8."""
+        ms, n = (C.c_double * 8)(), (C.c_int64 * 8)()
+        self._check(self.lib.sparsk_kernel_time_by_class(self.h, ms, n))
+        names = ("bookkeeping", "qkv", "attn", "oproj", "gateup", "down", "head", "mega")
+        return {k: (ms[i], n[i]) for i, k in enumerate(names)}
 
     def launch_count(self) -> int:
         return self.lib.sparsk_launch_count(self.h)

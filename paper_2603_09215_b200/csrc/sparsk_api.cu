@@ -23,8 +23,8 @@ namespace {
 constexpr int MAX_SPLITS = AT_MAX_SPLITS;
 constexpr int STAGE_RING = 16;
 constexpr uint32_t CTX_MAGIC = 0x5350524bu;  // "SPRK"
-constexpr size_t TIME_POOL = 8192;           // event pairs available to the kernel timer
-enum { KC_MISC = 0, KC_QKV = 1, KC_ATTN = 2, KC_OPROJ = 3, KC_GATEUP = 4, KC_DOWN = 5, KC_HEAD = 6, KC_MEGA = 7 };
+constexpr size_t TIME_POOL = 16384;           // event pairs available to the kernel timer
+enum { KC_MISC = 0, KC_QKV = 1, KC_ATTN = 2, KC_OPROJ = 3, KC_GATEUP = 4, KC_DOWN = 5, KC_HEAD = 6, KC_MEGA = 7, KC_ALL = 8 };
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -99,6 +99,7 @@ struct sparsk_ctx {
     // optional per-kernel-class timing (events around every launch of one class)
     int cur_class, time_class;
     std::vector<cudaEvent_t> tev;
+    std::vector<unsigned char> tev_class;  // class of each bracketed launch
     size_t tev_used;
     char err[512];
 };
@@ -216,8 +217,12 @@ cudaError_t launch(sparsk_ctx *c, void (*kern)(KArgs...), dim3 grid, dim3 block,
         cfg.numAttrs = 1;
     }
     c->launches++;
-    const bool timed = c->time_class == c->cur_class && c->time_class != KC_MISC && c->tev_used + 2 <= c->tev.size();
-    if (timed) cudaEventRecord(c->tev[c->tev_used++], c->stream);
+    const bool timed = ((c->time_class == c->cur_class && c->time_class != KC_MISC) || c->time_class == KC_ALL) &&
+                       c->tev_used + 2 <= c->tev.size();
+    if (timed) {
+        c->tev_class[c->tev_used / 2] = (unsigned char)c->cur_class;
+        cudaEventRecord(c->tev[c->tev_used++], c->stream);
+    }
     const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
     if (timed) cudaEventRecord(c->tev[c->tev_used++], c->stream);
     return e;
@@ -703,8 +708,11 @@ cudaError_t launch_mega_inst(sparsk_ctx *c, const MkArgs &a, size_t smem)
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     c->launches++;
-    const bool timed = c->time_class == KC_MEGA && c->tev_used + 2 <= c->tev.size();
-    if (timed) cudaEventRecord(c->tev[c->tev_used++], c->stream);
+    const bool timed = (c->time_class == KC_MEGA || c->time_class == KC_ALL) && c->tev_used + 2 <= c->tev.size();
+    if (timed) {
+        c->tev_class[c->tev_used / 2] = KC_MEGA;
+        cudaEventRecord(c->tev[c->tev_used++], c->stream);
+    }
     const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, a);
     if (timed) cudaEventRecord(c->tev[c->tev_used++], c->stream);
     return e;
@@ -945,10 +953,11 @@ extern "C" int sparsk_set_option(sparsk_ctx *ctx, const char *name, int64_t valu
     else if (!strcmp(name, "mega_max_rows") && value >= 1 && value <= MK_MAX_ROWS) ctx->mk_max_rows = (int)value;
     else if (!strcmp(name, "gemm_kb") && (value == 0 || value == 1)) ctx->tc_kb = (int)value;
     else if (!strcmp(name, "gemv_r") && (value == 0 || value == 1 || value == 2 || value == 4)) ctx->gv_r = (int)value;
-    else if (!strcmp(name, "time_kernel") && value >= 0 && value <= KC_MEGA) {
+    else if (!strcmp(name, "time_kernel") && value >= 0 && value <= KC_ALL) {
         // start (or stop, with 0) timing every launch of one kernel class; resets the totals
         if (value && ctx->tev.empty()) {
             ctx->tev.resize(2 * TIME_POOL);
+            ctx->tev_class.assign(TIME_POOL, 0);
             for (auto &ev : ctx->tev) CU(cudaEventCreate(&ev));
         }
         ctx->time_class = (int)value;
@@ -988,6 +997,25 @@ extern "C" int sparsk_check(sparsk_ctx *ctx)
         return fail(ctx, SPARSK_ETIMEOUT, "a bounded in-kernel wait ran out");
     }
     if (status & ST_BAD_TOKEN) return fail(ctx, SPARSK_EINVAL, "a token id was outside the vocabulary (clamped)");
+    return SPARSK_OK;
+}
+
+extern "C" int sparsk_kernel_time_by_class(sparsk_ctx *ctx, double *total_ms, int64_t *n_launches)
+{
+    if (!good(ctx)) return SPARSK_ESTATE;
+    if (!total_ms || !n_launches) return fail(ctx, SPARSK_EINVAL, "kernel_time_by_class: NULL output");
+    CU(cudaStreamSynchronize(ctx->stream));
+    for (int k = 0; k < 8; k++) {
+        total_ms[k] = 0.0;
+        n_launches[k] = 0;
+    }
+    for (size_t i = 0; i + 1 < ctx->tev_used; i += 2) {
+        float ms = 0.f;
+        CU(cudaEventElapsedTime(&ms, ctx->tev[i], ctx->tev[i + 1]));
+        const int k = ctx->tev_class[i / 2] & 7;
+        total_ms[k] += ms;
+        n_launches[k]++;
+    }
     return SPARSK_OK;
 }
 
