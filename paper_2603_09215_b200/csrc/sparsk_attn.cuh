@@ -43,10 +43,27 @@ inline AttnPlan attn_plan(int n_sm, int n_groups, int max_grp_rows, int G, int H
     p.n_qblk = (nq + 16 * p.mt - 1) / (16 * p.mt);
     int split = forced_split;
     if (split <= 0) {
-        const long base = (long)n_groups * p.n_qblk * Hkv;
-        long want = (2L * n_sm + base - 1) / base;
-        want = want < 1 ? 1 : (want > AT_MAX_SPLITS ? AT_MAX_SPLITS : want);
-        split = (int)((max_len + want - 1) / want);
+        // Two CTAs fit an SM.  Cut the KV range so that the CTAs fill whole waves of 2 * n_sm and,
+        // when the work allows, at least four of them (sequences are ragged and the causal cut
+        // makes CTAs unequal: many short CTAs even that out); never below AT_MIN_SPLIT positions.
+        const long slots = 2L * n_sm, base = (long)n_groups * p.n_qblk * Hkv;
+        const int max_s = (int)(max_len / AT_MIN_SPLIT < 1 ? 1 : (max_len / AT_MIN_SPLIT > AT_MAX_SPLITS ? AT_MAX_SPLITS : max_len / AT_MIN_SPLIT));
+        int best_s = 1;
+        double best = -1.0;
+        for (int s = 1; s <= max_s; s++) {
+            const long n = base * s, waves = (n + slots - 1) / slots;
+            const double eff = (double)n / (double)(waves * slots);
+            if (waves >= 4 && eff >= 0.92) {
+                best_s = s;
+                break;
+            }
+            const double score = eff * (double)(waves < 4 ? waves : 4);
+            if (score > best + 1e-9) {
+                best = score;
+                best_s = s;
+            }
+        }
+        split = (max_len + best_s - 1) / best_s;
         if (split < AT_MIN_SPLIT) split = AT_MIN_SPLIT;
     }
     split = (split + AT_TP - 1) / AT_TP * AT_TP;

@@ -62,9 +62,8 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b)
 // bits through a bf16 tensor-core product.
 __device__ __forceinline__ void split_pair(float a, float b, uint32_t &hi, uint32_t &lo)
 {
-    const bf16 ha = __float2bfloat16(a), hb = __float2bfloat16(b);
-    hi = pack_bf16x2(__bfloat162float(ha), __bfloat162float(hb));
-    lo = pack_bf16x2(a - __bfloat162float(ha), b - __bfloat162float(hb));
+    hi = pack_bf16x2(a, b);  // one packed conversion, widened back with shifts
+    lo = pack_bf16x2(a - bf_lo(hi), b - bf_hi(hi));
 }
 __device__ __forceinline__ void split8(const float (&v)[8], uint4 &hi, uint4 &lo)
 {
