@@ -260,6 +260,24 @@ def omp_threads():
     return int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
 
 
+# --------------------------------------------------------------------------- ranks
+def max_over_ranks(ms: float, world: int, device: str) -> float:
+    """Replicas share nothing on the data path; the only exchange is this one: the job's time is
+    the slowest rank's."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_tokens_per_s(tokens_per_rank: int, ms: float, world: int) -> float:
+    """Whole-job throughput of `world` replicas that each emitted tokens_per_rank in ms."""
+    return world * tokens_per_rank / (ms / 1e3)
+
+
 # --------------------------------------------------------------------------- main
 def main():
     ap = argparse.ArgumentParser()
@@ -348,11 +366,7 @@ def main():
         n = runner.run_cycles(cycles, host=host)
         ev1.record()
         barrier()
-        ms = ev0.elapsed_time(ev1)
-        if world > 1:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = max_over_ranks(ev0.elapsed_time(ev1), world, "cuda")
         return ms, n, runner.ctx.launch_count() - l0
 
     # ---- SPAR-K schedule, tokens on the device
@@ -366,7 +380,7 @@ def main():
     ms, ntok, launches = timed(run, args.steps)
     clocks = sampler.stop()
     step_b = (run.bytes - b0)
-    value = world * ntok / (ms / 1e3)
+    value = job_tokens_per_s(ntok, ms, world)
     peaks = {}
     pk_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(pk_path):
