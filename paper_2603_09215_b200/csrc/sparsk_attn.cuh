@@ -133,23 +133,25 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], 
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-template <int HD, int MT>
-__global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(AttnArgs a)
+// The work of one CTA (group * n_qblk + query block, kv head, split) by 128 threads; `sync` is the
+// barrier of those threads.  Also the attention phase of the persistent layer kernel, which runs
+// it on four-warp groups over virtual block indices.
+struct AttnCtaSync {
+    __device__ void operator()() const { __syncthreads(); }
+};
+template <int HD, int MT, int NS, class Sync>
+__device__ __forceinline__ void attn_partial_body(const AttnArgs &a, int bx, int hk, int sp, unsigned char *at_smem, int tid,
+                                                  Sync sync)
 {
     constexpr int QB = 16 * MT;     // query vectors per CTA
     constexpr int KP = HD + 8;      // padded row: ldmatrix rows fall into distinct banks
     constexpr int CH = HD / 8;      // 16-byte chunks per row
-    constexpr int NS = MT == 2 ? 2 : AT_NST;
-    extern __shared__ __align__(16) unsigned char at_smem[];
     bf16 *Qs = reinterpret_cast<bf16 *>(at_smem);  // [QB][KP] hi terms
     bf16 *Ql = Qs + QB * KP;                       // [QB][KP] lo terms
     bf16 *ring = Ql + QB * KP;                     // [4 warps][NS][K,V][AT_TP][KP]
 
-    griddep_wait();
-    griddep_launch();
-    const int g = blockIdx.x / a.n_qblk, qb = blockIdx.x % a.n_qblk;
+    const int g = bx / a.n_qblk, qb = bx % a.n_qblk;
     if (g >= *a.n_groups) return;
-    const int hk = blockIdx.y, sp = blockIdx.z;
     const int G = a.Hq / a.Hkv;
     const int row0 = a.grp_row0[g], nrows = a.grp_nrows[g];
     if (row0 < 0 || nrows < 1 || row0 + nrows > a.n_rows) return;
@@ -158,7 +160,7 @@ __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(AttnArgs a)
     if (q0 >= nq) return;
     const int nq_here = min(QB, nq - q0);
     const int slot = a.row_slot[row0], pos0 = a.row_pos[row0];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int lane = tid & 31, warp = tid >> 5;
 
     // positions this CTA may look at: its split, cut at the last query row's own position
     // (and at the cache itself: a descriptor that points outside it reads nothing)
@@ -186,7 +188,7 @@ __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(AttnArgs a)
         *reinterpret_cast<uint4 *>(&Qs[qi * KP + c * 8]) = hi;
         *reinterpret_cast<uint4 *>(&Ql[qi * KP + c * 8]) = lo;
     }
-    __syncthreads();
+    sync();
 
     // this warp's share of the split
     const int span = max(s_end - s_beg, 0);
@@ -327,7 +329,7 @@ __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(AttnArgs a)
         }
     }
     cp_async_wait<0>();
-    __syncthreads();  // every warp is done with its ring: reuse it for the merge
+    sync();  // every warp is done with its ring: reuse it for the merge
 
     // merge the four warps' states
     float *Ow = reinterpret_cast<float *>(ring);   // [4][QB][HD]
@@ -350,7 +352,7 @@ __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(AttnArgs a)
                 *reinterpret_cast<float2 *>(&Ow[((size_t)warp * QB + qi) * HD + nt * 8 + (lane & 3) * 2]) = v2;
             }
         }
-    __syncthreads();
+    sync();
     // partials (an empty split leaves max = -inf, sum = 0, which the merge of the splits ignores)
     for (int idx = tid; idx < nq_here * HD; idx += AT_THREADS) {
         const int qi = idx / HD, d = idx % HD;
@@ -371,6 +373,16 @@ __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(AttnArgs a)
         a.part_o[cell * HD + d] = acc;
         if (d == 0) a.part_ml[cell] = make_float2(M, L);
     }
+}
+
+template <int HD, int MT>
+__global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(AttnArgs a)
+{
+    extern __shared__ __align__(16) unsigned char at_smem_dyn[];
+    griddep_wait();
+    griddep_launch();
+    attn_partial_body<HD, MT, (MT == 2 ? 2 : AT_NST)>(a, blockIdx.x, blockIdx.y, blockIdx.z, at_smem_dyn, threadIdx.x,
+                                                      AttnCtaSync());
 }
 
 typedef void (*AttnPartialFn)(AttnArgs);
