@@ -15,6 +15,7 @@
 #include "sparsk_gemv.cuh"
 #include "sparsk_mega.cuh"
 #include "sparsk_step.cuh"
+#include "sparsk_tcmega.cuh"
 
 using namespace sparsk;
 
@@ -89,13 +90,16 @@ struct sparsk_ctx {
     unsigned long long *mk_bar;    // device: grid barrier counter; mk_bar_base mirrors its value
     int *mk_abort;                 // device
     float *mk_attn_o, *mk_act;     // device fp32 [MK_MAX_ROWS][Hq*hd], [MK_MAX_ROWS][F]
-    unsigned long long *mk_trace;  // device [1 + 6 L]
+    unsigned long long *mk_trace;  // device [1 + 9 L]
     int mk_trace_n;                // entries the last launch wrote
     unsigned long long mk_bar_base;
     int mega, mk_ok, mk_coop, mk_max_rows;
     std::vector<MkLayer> mk_host;
     float *qkv_part;  // fp32 sums of a q/k/v product whose inner dimension is cut across CTAs
     int tc_kb;        // 0: automatic; 1: force one k-block per copy (2-D descriptors)
+    // persistent tcgen05 layer-range kernel (3..TK_MAX_N rows)
+    TkLayer *tk_layers;  // device [L]
+    int tcmega, tk_ok;
     // optional per-kernel-class timing (events around every launch of one class)
     int cur_class, time_class;
     std::vector<cudaEvent_t> tev;
@@ -180,10 +184,11 @@ size_t carve(sparsk_ctx *c, const sparsk_dims *d, char *base)
     bf16 *aol = w.take<bf16>(R * qrow), *actl = w.take<bf16>(R * d->d_ffn), *xnl = w.take<bf16>(R * d->d_model);
     float *qp = w.take<float>(R * (qrow + 2 * kvrow));
     MkLayer *mkl = w.take<MkLayer>(L);
+    TkLayer *tkl = w.take<TkLayer>(L);
     unsigned long long *mkb = w.take<unsigned long long>(1);
     int *mka = w.take<int>(1);
     float *mkao = w.take<float>((size_t)MK_MAX_ROWS * qrow), *mkact = w.take<float>((size_t)MK_MAX_ROWS * d->d_ffn);
-    unsigned long long *mkt = w.take<unsigned long long>(1 + 6 * L);
+    unsigned long long *mkt = w.take<unsigned long long>(1 + 9 * L);
     const size_t cells = std::max<size_t>(R * MAX_SPLITS, (size_t)MK_MAX_ROWS * MK_MAX_SPLITS) * d->n_q_heads;
     float *po = w.take<float>(cells * d->head_dim);
     float2 *pml = w.take<float2>(cells);
@@ -194,7 +199,7 @@ size_t carve(sparsk_ctx *c, const sparsk_dims *d, char *base)
         c->pf_ngrp = pfng; c->pf_nrows = pfnr;
         c->h_lo = hlo; c->h_up = hup; c->qbuf = q; c->attn_o = ao; c->act = act; c->xnorm = xn; c->qkv_part = qp;
         c->attn_o_lo = aol; c->act_lo = actl; c->xnorm_lo = xnl;
-        c->mk_layers = mkl; c->mk_bar = mkb; c->mk_abort = mka; c->mk_attn_o = mkao; c->mk_act = mkact; c->mk_trace = mkt;
+        c->mk_layers = mkl; c->tk_layers = tkl; c->mk_bar = mkb; c->mk_abort = mka; c->mk_attn_o = mkao; c->mk_act = mkact; c->mk_trace = mkt;
         c->part_o = po; c->part_ml = pml;
     }
     return align_up(w.off, 256);
@@ -762,6 +767,115 @@ cudaError_t run_mega(sparsk_ctx *c, int l_begin, int l_end, float *h, const RowS
     }
 }
 
+// ---------------------------------------------------------------- persistent tcgen05 layer-range kernel
+bool build_tcmega(sparsk_ctx *c)
+{
+    const sparsk_dims &d = c->dm;
+    const size_t lstride = (size_t)d.max_seqs * d.n_kv_heads * d.max_seq_len * d.head_dim;
+    std::vector<TkLayer> host(d.n_layers);
+    for (int l = 0; l < d.n_layers; l++) {
+        TkLayer &t = host[l];
+        memset(&t, 0, sizeof t);
+        t.wq = c->tm_wq[l].m2; t.wk = c->tm_wk[l].m2; t.wv = c->tm_wv[l].m2; t.wo = c->tm_wo[l].m2;
+        t.wg = c->tm_wg[l].m2; t.wu = c->tm_wu[l].m2; t.wd = c->tm_wd[l].m2;
+        t.attn_gain = c->attn_norm[l];
+        t.mlp_gain = c->mlp_norm[l];
+        t.kc = c->kcache + l * lstride;
+        t.vc = c->vcache + l * lstride;
+    }
+    // pageable source: the copy has left the host buffer when the call returns
+    return cudaMemcpyAsync(c->tk_layers, host.data(), sizeof(TkLayer) * d.n_layers, cudaMemcpyHostToDevice, c->stream) ==
+           cudaSuccess;
+}
+
+size_t tk_attn_bytes(int head_dim, int mt)
+{
+    const size_t kp = head_dim + 8;
+    const size_t q = (size_t)2 * 16 * mt * kp * 2, ring = (size_t)4 * 2 * 2 * AT_TP * kp * 2;
+    const size_t merge = (size_t)4 * 16 * mt * (head_dim + 2) * 4;
+    return q + std::max(ring, merge);
+}
+
+// Can a pass over this row set go through the persistent tcgen05 kernel?
+bool use_tcmega(const sparsk_ctx *c, const RowSet &rs)
+{
+    const sparsk_dims &d = c->dm;
+    return c->tcmega && c->tk_ok && c->tc_ok && c->mk_coop && rs.n_rows >= c->gemm_min_rows && rs.n_rows <= TK_MAX_N &&
+           d.d_model >= GM_BK && tk_attn_bytes(d.head_dim, 2) <= (size_t)TK_ATT_BYTES;
+}
+
+template <int HD>
+cudaError_t launch_tcmega_inst(sparsk_ctx *c, const TkArgs &a)
+{
+    static int grid_ok = -1;
+    auto kern = tcmega_kernel<HD>;
+    if (grid_ok < 0) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TK_SMEM);
+        if (e != cudaSuccess) return e;
+        int per_sm = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, TK_THREADS, TK_SMEM);
+        if (e != cudaSuccess) return e;
+        grid_ok = per_sm >= 1 ? 1 : 0;
+    }
+    if (!grid_ok) return cudaErrorCooperativeLaunchTooLarge;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(c->n_sm);
+    cfg.blockDim = dim3(TK_THREADS);
+    cfg.dynamicSmemBytes = TK_SMEM;
+    cfg.stream = c->stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    c->launches++;
+    const bool timed = (c->time_class == KC_MEGA || c->time_class == KC_ALL) && c->tev_used + 2 <= c->tev.size();
+    if (timed) {
+        c->tev_class[c->tev_used / 2] = KC_MEGA;
+        cudaEventRecord(c->tev[c->tev_used++], c->stream);
+    }
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, a);
+    if (timed) cudaEventRecord(c->tev[c->tev_used++], c->stream);
+    return e;
+}
+
+// Layers [l_begin, l_end) (0-based) over a row set of 3..TK_MAX_N rows, in one launch.
+cudaError_t run_tcmega(sparsk_ctx *c, int l_begin, int l_end, float *h, const RowSet &rs)
+{
+    const sparsk_dims &d = c->dm;
+    const int qd = d.n_q_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, G = d.n_q_heads / d.n_kv_heads;
+    TkArgs a;
+    memset(&a, 0, sizeof a);
+    const int bi = box_index(rs.n_rows);
+    a.box_n = 16 << bi;
+    a.x_hi = c->tm_x[bi].m2; a.x_lo = c->tm_x_lo[bi].m2; a.ao_hi = c->tm_ao[bi].m2; a.ao_lo = c->tm_ao_lo[bi].m2;
+    a.act_hi = c->tm_act[bi].m2; a.act_lo = c->tm_act_lo[bi].m2;
+    a.layers = c->tk_layers; a.layer_begin = l_begin; a.layer_end = l_end; a.h = h;
+    a.row_slot = rs.slot; a.row_pos = rs.pos; a.grp_row0 = rs.grp_row0; a.grp_nrows = rs.grp_nrows;
+    a.n_groups_dev = rs.n_groups;
+    a.m_rows = rs.n_rows;
+    a.q32 = c->qbuf; a.qkv_part = c->qkv_part;
+    a.x_hi_p = c->xnorm; a.x_lo_p = c->xnorm_lo; a.ao_hi_p = c->attn_o; a.ao_lo_p = c->attn_o_lo;
+    a.act_hi_p = c->act; a.act_lo_p = c->act_lo;
+    a.part_o = c->part_o; a.part_ml = c->part_ml; a.rope = c->rope;
+    a.d = d.d_model; a.Hq = d.n_q_heads; a.Hkv = d.n_kv_heads; a.hd = d.head_dim; a.F = d.d_ffn; a.S = d.max_seq_len;
+    a.n_slots = d.max_seqs; a.eps = d.rms_eps;
+    // every cut of an inner dimension holds at least one k-block
+    auto cuts = [&](int units, int K) { return std::max(1, std::min(splits_for(c, units), div_up(K, GM_BK))); };
+    a.splits_qkv = cuts(div_up(qd, 2 * GM_BM) + 2 * div_up(kd, 2 * GM_BM), d.d_model);
+    a.splits_o = cuts(div_up(d.d_model, 2 * GM_BM), qd);
+    a.splits_down = cuts(div_up(d.d_model, 2 * GM_BM), d.d_ffn);
+    const AttnPlan pl = attn_plan(c->n_sm, rs.n_groups_h, rs.max_grp_rows, G, d.n_kv_heads, rs.max_len, c->attn_split);
+    a.att_groups = rs.n_groups_h; a.att_qblk = pl.n_qblk; a.att_splits = pl.n_splits; a.att_split_len = pl.split_len;
+    a.att_mt = pl.mt;
+    a.bar = c->mk_bar; a.bar_base = c->mk_bar_base; a.abort_word = c->mk_abort; a.status = c->sd.counts + CNT_STATUS;
+    c->mk_bar_base += (unsigned long long)TK_PHASES * (unsigned long long)(l_end - l_begin) * (unsigned long long)c->n_sm;
+    a.trace = c->mk_trace;
+    c->mk_trace_n = 1 + TK_PHASES * (l_end - l_begin);
+    return d.head_dim == 128 ? launch_tcmega_inst<128>(c, a) : launch_tcmega_inst<64>(c, a);
+}
+
 // One transformer layer over a row set: h <- h^(layer).
 cudaError_t run_layer(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
 {
@@ -788,6 +902,7 @@ cudaError_t run_layers(sparsk_ctx *c, int l_first, int l_last, float *h, const R
 {
     if (l_first > l_last) return cudaSuccess;
     if (use_mega(c, rs.n_rows)) return run_mega(c, l_first - 1, l_last, h, rs);
+    if (use_tcmega(c, rs)) return run_tcmega(c, l_first - 1, l_last, h, rs);
     for (int l = l_first; l <= l_last; l++) {
         const cudaError_t e = run_layer(c, l, h, rs);
         if (e != cudaSuccess) return e;
@@ -853,6 +968,7 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
     ctx->tc_ok = false;
     ctx->tc_kb = 0;
     ctx->mk_max_rows = 2;
+    ctx->tcmega = 0; ctx->tk_ok = 0;
     ctx->mega = 1; ctx->mk_ok = 0; ctx->mk_coop = 0; ctx->mk_bar_base = 0; ctx->mk_trace_n = 0;
     ctx->gv_ks = 0; ctx->gv_r = 0; ctx->gv_grid_mult = 1;
     ctx->dbg_hidden = nullptr; ctx->dbg_logits = nullptr;
@@ -885,6 +1001,11 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
         ctx->mk_ok = build_mega(ctx) ? 1 : 0;
         if (!ctx->mk_ok) {
             rc = fail(ctx, SPARSK_ECUDA, "setting up the persistent layer kernel failed");
+            break;
+        }
+        ctx->tk_ok = build_tcmega(ctx) ? 1 : 0;
+        if (!ctx->tk_ok) {
+            rc = fail(ctx, SPARSK_ECUDA, "setting up the persistent tensor-core layer kernel failed");
             break;
         }
         // rotary table in double, stored as float (cos, sin)
@@ -950,6 +1071,7 @@ extern "C" int sparsk_set_option(sparsk_ctx *ctx, const char *name, int64_t valu
     else if (!strcmp(name, "attn_split") && value >= 0 && value <= (1 << 24)) ctx->attn_split = (int)value;
     else if (!strcmp(name, "gemv_ks") && (value == 0 || value == 1 || value == 2 || value == 4 || value == 8 || value == 16)) ctx->gv_ks = (int)value;
     else if (!strcmp(name, "mega") && (value == 0 || value == 1)) ctx->mega = (int)value;
+    else if (!strcmp(name, "tcmega") && (value == 0 || value == 1)) ctx->tcmega = (int)value;
     else if (!strcmp(name, "mega_max_rows") && value >= 1 && value <= MK_MAX_ROWS) ctx->mk_max_rows = (int)value;
     else if (!strcmp(name, "gemm_kb") && (value == 0 || value == 1)) ctx->tc_kb = (int)value;
     else if (!strcmp(name, "gemv_r") && (value == 0 || value == 1 || value == 2 || value == 4)) ctx->gv_r = (int)value;

@@ -60,18 +60,34 @@ def test_odd_shapes_and_schedules(util, e, K, r, nt, ns, min_rows):
     P.close()
 
 
-@pytest.mark.parametrize("min_rows", [3, 1, 1 << 30])
-def test_heterogeneous_batch_matches_per_sequence_oracle(util, min_rows):
+def test_odd_shapes_persistent_tensor_core_kernel(util):
+    """head_dim 64, three query heads per kv head, inner dimensions that are not multiples of 64:
+    every pass (1..5 rows, 16-row prefill chunks) through the persistent tensor-core kernel."""
+    dims = synth.model_dims(MICRO64, 2, 4, 1)
+    w = synth.make_weights(dims, seed=5)
+    prompt = synth.make_prompts(dims, 1, 37, 37, seed=7)[0]
+    P = util.Pair(dims, w, 1, 128, 8, prefill_rows=16, options={"tcmega": 1, "mega": 0, "gemm_min_rows": 1})
+    P.prefill([prompt])
+    for g in range(40):
+        m, c = synth.interleave(g, 2, 7)
+        P.step([m], [c])
+    P.check_cache(0, range(1, 4), P.g.slot_state(0)[0] - P.g.slot_state(0)[1])
+    P.close()
+
+
+@pytest.mark.parametrize("min_rows,tcmega", [(3, 0), (1, 0), (1 << 30, 0), (3, 1)])
+def test_heterogeneous_batch_matches_per_sequence_oracle(util, min_rows, tcmega):
     """Batch of 7 with random interleave phases and counter offsets and ragged prompts, so every
     step mixes text, early-exit and refresh rows; sequences stay independent.  Run with the
     default hand-over between the small-batch and the tensor-core path (3 rows), with every
-    projection on the tensor cores, and with every projection on the small-batch path."""
+    projection on the tensor cores, with every projection on the small-batch path, and with the
+    tensor-core layers as one persistent kernel per layer range."""
     dims = synth.model_dims("tiny", 2, 4, 0)
     w = synth.make_weights(dims, seed=0)
     B = 7
     prompts = synth.make_prompts(dims, B, 9, 70, seed=4)
     phi, off = synth.make_phases(B, 1, 4, 4, True, seed=8)
-    P = util.Pair(dims, w, B, 70 + 64, 3, prefill_rows=24, options={"gemm_min_rows": min_rows})
+    P = util.Pair(dims, w, B, 70 + 64, 3, prefill_rows=24, options={"gemm_min_rows": min_rows, "tcmega": tcmega})
     P.prefill(prompts)
     mixed = 0
     for g in range(48):
@@ -176,11 +192,13 @@ def test_host_step_and_error_codes(util):
 
 
 @pytest.mark.parametrize("options", [{"mega": 0}, {"mega_max_rows": 4}, {"mega_max_rows": 1, "gemm_min_rows": 2},
-                                     {"mega": 0, "gemm_min_rows": 1 << 30}, {"gemm_kb": 1, "mega": 0, "gemm_min_rows": 1}])
+                                     {"mega": 0, "gemm_min_rows": 1 << 30}, {"gemm_kb": 1, "mega": 0, "gemm_min_rows": 1},
+                                     {"tcmega": 1}, {"tcmega": 1, "mega": 0, "gemm_min_rows": 1}])
 def test_every_route_for_small_passes(util, options):
-    """Passes of 1..4 rows (K = 4: flushes of up to three pending rows) through each of the three
+    """Passes of 1..4 rows (K = 4: flushes of up to three pending rows) through each of the
     implementations: the persistent kernel (also with its moving activation window at 3-4 rows),
-    the tensor-core path (with 2-D descriptors too) and the small-batch kernels."""
+    the tensor-core path (with 2-D descriptors too, and as one persistent kernel per layer range)
+    and the small-batch kernels."""
     dims = synth.model_dims("tiny", 2, 4, 0)
     w = synth.make_weights(dims, seed=0)
     prompt = synth.make_prompts(dims, 1, 21, 21, seed=11)[0]
