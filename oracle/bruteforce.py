@@ -82,9 +82,10 @@ def head_logits(dims: dict, w: dict, layer: int, h: np.ndarray) -> np.ndarray:
 
 def scheduled_depth(dims: dict, modality: int, c: int) -> int:
     """Sec. IV-B.1: in-chunk index c runs all L layers iff c mod K == r; text always does
-    unless text_exit is set."""
+    unless text_exit is set (1: text too; 2: text only, speech always full, Sec. V-E row G10)."""
     L, e = dims["n_layers"], dims["exit_layer"]
-    if modality == 0 and not dims.get("text_exit", 0):
+    te = dims.get("text_exit", 0)
+    if (modality == 0 and te == 0) or (modality == 1 and te == 2):
         return L
     return L if c % dims["refresh_period"] == dims["refresh_phase"] else e
 

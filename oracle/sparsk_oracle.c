@@ -53,7 +53,9 @@ typedef struct {
     int32_t refresh_period; /* K >= 1                                             */
     int32_t refresh_phase;  /* r in [0,K): in-chunk index c is full iff c%K == r  */
     int32_t text_exit;      /* 0: text always full depth (paper's main rows);
-                               1: text follows the same schedule (rows G10)       */
+                               1: text follows the same schedule as speech;
+                               2: only text follows it, speech always runs L
+                                  layers (Sec. V-E, row G10: text Even, speech --) */
     int32_t max_len;        /* positions a sequence can hold                      */
 } ora_dims;
 
@@ -102,7 +104,8 @@ static double bf16_to_double(uint16_t b)
 int32_t ora_depth(int32_t modality, int32_t c, int32_t K, int32_t r, int32_t e, int32_t L,
                   int32_t text_exit)
 {
-    if (modality == 0 && !text_exit) return L;
+    if (modality == 0 && text_exit == 0) return L;
+    if (modality == 1 && text_exit == 2) return L;
     return (c % K == r) ? L : e;
 }
 

@@ -51,6 +51,37 @@ def test_matches_cache_free_recomputation(e, K, r, nt, ns, phase):
         assert abs(g["margin"] - x["margin"]) < 1e-9
 
 
+@pytest.mark.parametrize("text_exit,K,r,nt,ns,running", [
+    (1, 2, 0, 3, 4, False),    # text and speech both follow Even
+    (2, 2, 0, 5, 3, False),    # text only (Sec. V-E row G10); speech flushes the pending text rows
+    (0, 6, 5, 1, 5, False),    # fixed-layer exit: no refresh inside a chunk, the text step flushes 5 rows
+    (0, 3, 0, 1, 4, True),     # counter running across chunks instead of restarting
+    (0, 2, 1, 1, 4, False)])   # Odd
+def test_schedule_variants_match_cache_free_recomputation(text_exit, K, r, nt, ns, running):
+    """The schedule variants of Sec. IV-B.1 / V-B / V-E: whatever the caller's counters make of the
+    depths, pending rows persist until the next full-depth step of either modality and the stream
+    equals cache-free recomputation."""
+    dims = synth.model_dims(MICRO, 2, K, r, text_exit=text_exit)
+    w = synth.make_weights(dims, seed=13)
+    prompt = synth.make_prompts(dims, 1, 6, 6, seed=3)[0]
+    mc = [synth.interleave(g, nt, ns, running=running) for g in range(26)]
+    mods, ctrs = [m for m, _ in mc], [c for _, c in mc]
+    _, _, got = _run_oracle(dims, w, prompt, mods, ctrs)
+    ref = bf.decode_stream(dims, w, prompt, mods, ctrs)
+    assert [g["depth"] for g in got] == [x["depth"] for x in ref]
+    assert [g["token"] for g in got] == [x["token"] for x in ref]
+    for g, x in zip(got, ref):
+        np.testing.assert_allclose(g["hidden"], x["hidden"], rtol=1e-9, atol=1e-11)
+    depths = [g["depth"] for g in got]
+    assert 2 in depths and 3 in depths
+    if text_exit == 2:
+        assert all(d == 3 for d, m in zip(depths, mods) if m == 1)
+        assert any(d == 2 for d, m in zip(depths, mods) if m == 0)
+    if K == 6:   # fixed-layer: every speech step leaves early, pending reaches the chunk length
+        assert all(d == 2 for d, m in zip(depths, mods) if m == 1)
+        assert max(len(g["pending_after"]) for g in got) == ns
+
+
 def test_config1_full_run_matches_cache_free_recomputation():
     wl = synth.WORKLOADS["cfg1_tiny_b1"]
     dims = synth.model_dims("tiny", wl["exit_layer"], wl["refresh_period"], wl["refresh_phase"])

@@ -53,6 +53,30 @@ def test_schedule_patterns_from_the_text():
         assert d.count(L) == 2 and d.count(e) == 2
 
 
+def test_text_only_schedule_row_G10():
+    """Sec. V-E row G10: the periodic rule on text tokens only; speech stays at full depth."""
+    path = os.path.join(os.path.dirname(__file__), "golden", "table2_text_schedule.txt")
+    rows = [l.split() for l in open(path) if l.strip() and not l.startswith("#")]
+    assert rows
+    for name, L, Nt, Ns, sched, e, avg_t, avg_s, tol in rows:
+        L, Nt, Ns, e = int(L), int(Nt), int(Ns), int(e)
+        K, r = _kr(sched, Nt)
+        text = [ora.depth(0, c, K, r, e, L, 2) for c in range(Nt)]
+        speech = [ora.depth(1, c, K, r, e, L, 2) for c in range(Ns)]
+        assert abs(sum(text) / Nt - float(avg_t)) <= float(tol), (name, text)
+        assert sum(speech) / Ns == float(avg_s), (name, speech)
+        # on whole periods the printed value is exact
+        whole = [ora.depth(0, c, K, r, e, L, 2) for c in range(K * 6)]
+        assert sum(whole) / len(whole) == float(avg_t)
+    # the three modes side by side (L = 4, e = 2, Even)
+    assert [ora.depth(0, c, 2, 0, 2, 4, 0) for c in range(4)] == [4, 4, 4, 4]
+    assert [ora.depth(1, c, 2, 0, 2, 4, 0) for c in range(4)] == [4, 2, 4, 2]
+    assert [ora.depth(0, c, 2, 0, 2, 4, 1) for c in range(4)] == [4, 2, 4, 2]
+    assert [ora.depth(1, c, 2, 0, 2, 4, 1) for c in range(4)] == [4, 2, 4, 2]
+    assert [ora.depth(0, c, 2, 0, 2, 4, 2) for c in range(4)] == [4, 2, 4, 2]
+    assert [ora.depth(1, c, 2, 0, 2, 4, 2) for c in range(4)] == [4, 4, 4, 4]
+
+
 def test_full_count_closed_form_against_enumeration():
     # number of full-depth positions in a chunk of N: floor((N - r + K - 1) / K)
     L, e = 40, 30
