@@ -65,7 +65,9 @@ typedef struct {
     int32_t refresh_period; /* K >= 1; K == 1 makes every step full depth */
     int32_t refresh_phase;  /* r in [0, K): in-chunk index c is full depth iff c % K == r */
     int32_t text_exit;      /* 0: text steps always run L layers (the paper's main rows);
-                               1: text steps follow the same (K, r, e) rule (Sec. V-E) */
+                               1: text steps follow the same (K, r, e) rule as speech steps;
+                               2: only text steps follow it and speech steps always run L
+                                  layers (Sec. V-E, row G10) */
     int32_t max_seqs;       /* number of sequence slots */
     int32_t max_seq_len;    /* positions per slot */
     int32_t max_pending;    /* pending positions per slot; >= K-1 for the periodic schedule */

@@ -140,7 +140,7 @@ bool dims_ok(const sparsk_dims *d)
     if (!(d->rms_eps >= 0.f) || !(d->rope_base > 0.f)) return false;
     if (d->exit_layer < 1 || d->exit_layer > d->n_layers) return false;
     if (d->refresh_period < 1 || d->refresh_phase < 0 || d->refresh_phase >= d->refresh_period) return false;
-    if (d->text_exit != 0 && d->text_exit != 1) return false;
+    if (d->text_exit < 0 || d->text_exit > 2) return false;
     if (d->max_seqs < 1 || d->max_seqs > 1024 || d->max_seq_len < 1) return false;
     if (d->max_pending < 0 || d->prefill_rows < 0) return false;
     return true;
@@ -1263,7 +1263,7 @@ extern "C" int sparsk_decode_step(sparsk_ctx *ctx, int32_t n, const int32_t *slo
         if (modality[i] > 1) return fail(ctx, SPARSK_EINVAL, "decode_step: modality[%d]=%d", i, modality[i]);
         if (counters[i] < 0) return fail(ctx, SPARSK_EINVAL, "decode_step: counter[%d]=%d", i, counters[i]);
         if (ctx->h_len[s] + 1 > d.max_seq_len) return fail(ctx, SPARSK_ECAPACITY, "decode_step: slot %d is full (%d positions)", s, ctx->h_len[s]);
-        const int depth = (modality[i] == 0 && !d.text_exit) ? L : ((counters[i] % K == r) ? L : e);
+        const int depth = scheduled_depth(modality[i], counters[i], K, r, e, L, d.text_exit);
         const bool full = depth == L;
         if (!full && ctx->h_pend[s] + 1 > d.max_pending)
             return fail(ctx, SPARSK_ECAPACITY, "decode_step: slot %d would hold %d pending positions (max_pending %d)", s, ctx->h_pend[s] + 1, d.max_pending);
@@ -1336,7 +1336,7 @@ extern "C" int sparsk_decode_step(sparsk_ctx *ctx, int32_t n, const int32_t *slo
     // ---- host mirror follows
     for (int i = 0; i < n; i++) {
         const int s = slots[i];
-        const int depth = (modality[i] == 0 && !d.text_exit) ? L : ((counters[i] % K == r) ? L : e);
+        const int depth = scheduled_depth(modality[i], counters[i], K, r, e, L, d.text_exit);
         ctx->h_len[s] += 1;
         ctx->h_pend[s] = (depth == L) ? 0 : ctx->h_pend[s] + 1;
     }

@@ -6,11 +6,20 @@
 
 namespace sparsk {
 
+// Layers a step runs (Sec. IV-B.1): in-chunk index c runs L layers iff c mod K == r, else e.
+// text_exit 0: text (modality 0) always runs L; 1: text follows the rule too; 2: only text follows
+// it and speech always runs L (Sec. V-E, row G10).  The host's mirror of the pending counts uses
+// the same function.
+__host__ __device__ inline int scheduled_depth(int modality, int c, int K, int r, int e, int L, int text_exit)
+{
+    if (modality == 0 && text_exit == 0) return L;
+    if (modality != 0 && text_exit == 2) return L;
+    return (c % K == r) ? L : e;
+}
+
 // ---------------------------------------------------------------------------------------
-// Exit schedule (Sec. IV-B.1).  One thread per sequence: text runs L layers unless the text
-// schedule is on; in-chunk index c runs L layers iff c mod K == r, else e.  Also latches the
-// input token (clamped into the vocabulary, with a status bit if it was outside) and clears
-// the sequence's argmax cell.
+// Exit schedule (Sec. IV-B.1).  One thread per sequence.  Also latches the input token (clamped
+// into the vocabulary, with a status bit if it was outside) and clears the sequence's argmax cell.
 // ---------------------------------------------------------------------------------------
 static __global__ void schedule_kernel(StepDesc sd, int n, const int *__restrict__ staged /*[3][n]*/,
                                 const int *__restrict__ tokens_in, int vocab, int L, int e, int K,
@@ -21,7 +30,7 @@ static __global__ void schedule_kernel(StepDesc sd, int n, const int *__restrict
     if (b == 0) sd.counts[CNT_NSEQ] = n;
     if (b >= n) return;
     int slot = staged[b], mod = staged[n + b], c = staged[2 * n + b];
-    int depth = (mod == 0 && !text_exit) ? L : ((c % K == r) ? L : e);
+    int depth = scheduled_depth(mod, c, K, r, e, L, text_exit);
     int tok = tokens_in[b];
     if (tok < 0 || tok >= vocab) {
         atomicOr(&sd.counts[CNT_STATUS], ST_BAD_TOKEN);

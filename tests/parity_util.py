@@ -76,7 +76,8 @@ class Pair:
             if r is None:
                 # unchecked sequence: its depth still has to follow the schedule; it runs on
                 # the token the library produced
-                want = L if (mods[i] == 0 and not self.dims.get("text_exit", 0)) else (L if ctrs[i] % K == r_ else e)
+                te = self.dims.get("text_exit", 0)
+                want = L if ((mods[i] == 0 and te == 0) or (mods[i] == 1 and te == 2)) else (L if ctrs[i] % K == r_ else e)
                 assert got_dep[i] == want, (i, got_dep[i], want)
                 self.next_in[s] = int(got_tok[i])
                 continue
