@@ -58,7 +58,8 @@ def test_ties_go_to_the_lower_id_and_range_is_respected():
     assert list(s["ids"]) == [2, 3, 4, 5, 6, 7]
     assert [smp.nucleus_sample(z, 2, 8, 0.7, 1.0, u)["token"] for u in (0.0, 0.17, 0.55, 0.99)] == [2, 3, 5, 7]
     # landing_error: zero inside the token's interval, the distance outside, inf outside the kept set
-    s = smp.nucleus_sample(z, 2, 8, 0.7, 1.0, 0.5)
-    assert smp.landing_error(s, 5, 0.5) == 0.0
-    assert abs(smp.landing_error(s, 2, 0.5) - (0.5 - 1 / 6)) < 1e-12
-    assert smp.landing_error(s, 9, 0.5) == float("inf")
+    s = smp.nucleus_sample(z, 2, 8, 0.7, 1.0, 0.55)
+    assert smp.landing_error(s, 5, 0.55) == 0.0
+    assert abs(smp.landing_error(s, 2, 0.55) - (0.55 - 1 / 6)) < 1e-12
+    assert abs(smp.landing_error(s, 7, 0.55) - (5 / 6 - 0.55)) < 1e-12
+    assert smp.landing_error(s, 9, 0.55) == float("inf")
