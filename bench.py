@@ -134,7 +134,7 @@ def cycle_schedule(wl, phi, off, g0, n):
 class Runner:
     """Drives one library context through decode steps with tokens kept on the device."""
 
-    def __init__(self, dims, gw, wl, prompts, phi, off, total_steps, options=None, synthetic_kv=False):
+    def __init__(self, dims, gw, wl, prompts, phi, off, total_steps, options=None, synthetic_kv=False, sampling=None):
         import torch
         from paper_2603_09215_b200 import binding
         self.torch = torch
@@ -147,6 +147,12 @@ class Runner:
                                   prefill_rows=64)
         for k, v in (options or {}).items():
             self.ctx.set_option(k, v)
+        # nucleus sampling (Sec. V-A decodes the 28-layer backbone with it): a table of uniform
+        # numbers on the device, one row per decode step
+        self.sampling = sampling
+        if sampling:
+            self.uni = torch.from_numpy(synth.make_uniforms(1024 * B, seed=7)).cuda().view(1024, B)
+            self.uni_row = 0
         self.slots = list(range(B))
         if synthetic_kv:
             self._fill_synthetic(prompts)
@@ -201,16 +207,23 @@ class Runner:
         if host:
             nt, dp = np.zeros(self.B, np.int32), np.zeros(self.B, np.int32)
             for mods, ctrs in sched:
+                self._next_uniforms()
                 self.ctx.decode_step_host(self.slots, self.host_tok, mods, ctrs, nt, dp)
                 self.host_tok[:] = nt
                 self._account(mods, ctrs)
         else:
             for mods, ctrs in sched:
+                self._next_uniforms()
                 self.ctx.decode_step(self.slots, self.tok[0], mods, ctrs, self.tok[1], self.dep)
                 self.tok.reverse()
                 self._account(mods, ctrs)
         self.g += n_cycles * cyc
         return n_cycles * cyc * self.B
+
+    def _next_uniforms(self):
+        if self.sampling:
+            self.ctx.set_sampling(self.sampling[0], self.sampling[1], self.uni[self.uni_row % 1024])
+            self.uni_row += 1
 
     def sync_host_tokens(self):
         self.host_tok[:] = self.tok[0].cpu().numpy()
@@ -290,6 +303,8 @@ def main():
     ap.add_argument("--no-full-depth", action="store_true")
     ap.add_argument("--option", action="append", default=[], help="library option name=value")
     ap.add_argument("--time-kernel", default="mega", choices=sorted(KC))
+    ap.add_argument("--sampling", default=None, metavar="T,P",
+                    help="nucleus sampling with temperature T and top_p P (the paper's 0.7,0.9) instead of the arg max")
     ap.add_argument("--exit-layer", type=int, default=None, help="override the workload's exit layer e (sweep cells)")
     ap.add_argument("--period", type=int, default=None, help="override the workload's refresh period K (sweep cells)")
     args = ap.parse_args()
@@ -351,10 +366,12 @@ def main():
     for o in args.option:
         k, v = o.split("=")
         opts[k] = int(v)
+    sampling = tuple(float(x) for x in args.sampling.split(",")) if args.sampling else None
+    cfg["decoding"] = f"nucleus T={sampling[0]} top_p={sampling[1]}" if sampling else "greedy (restricted arg max)"
     synthetic_kv = max(wl["prompt"]) > 4096      # long prompts: cache contents are stand-ins
     extra = (W + args.steps) * 2 + 8
     total_steps = extra * cyc
-    run = Runner(dims, gw, wl, prompts, phi, off, total_steps, opts, synthetic_kv)
+    run = Runner(dims, gw, wl, prompts, phi, off, total_steps, opts, synthetic_kv, sampling)
     cfg["cache_fill"] = "stand-in values (imported)" if synthetic_kv else "real prefill of random prompts"
     setup_s = time.time() - t_setup
 
@@ -435,7 +452,7 @@ def main():
     if not args.no_full_depth:
         wl_f = dict(wl, refresh_period=1, refresh_phase=0)
         dims_f = synth.model_dims(wl["shape"], wl["exit_layer"], 1, 0)
-        rf = Runner(dims_f, gw, wl_f, prompts, phi, off, total_steps, opts, synthetic_kv)
+        rf = Runner(dims_f, gw, wl_f, prompts, phi, off, total_steps, opts, synthetic_kv, sampling)
         rf.run_cycles(W)
         fb0 = rf.bytes
         ms_f, ntok_f, _ = timed(rf, args.steps)

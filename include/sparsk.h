@@ -165,6 +165,34 @@ int sparsk_set_debug(sparsk_ctx *ctx, float *exit_hidden /*device or NULL*/,
  * "time_kernel" (see sparsk_kernel_time).  Returns SPARSK_EINVAL for an unknown name or value. */
 int sparsk_set_option(sparsk_ctx *ctx, const char *name /*host*/, int64_t value);
 
+/* Nucleus sampling (Sec. V-A: the 28-layer backbone is decoded with temperature 0.7 and top_p 0.9;
+ * the 40-layer one greedily).  After this call every decode step draws each sequence's token from
+ * the nucleus of its exit head's logits instead of taking their arg max: over the ids of the step's
+ * modality, p = softmax(z / temperature); ids in decreasing p (equal p: lower id first); the
+ * shortest prefix whose mass reaches top_p is kept; the token is the first id whose cumulative
+ * mass exceeds u * (kept mass).  u comes from `uniforms` (DEVICE float [max_seqs], borrowed until
+ * the next call of this function): the step reads uniforms[i] in [0, 1) for the i-th sequence of
+ * its `slots` argument, so the caller refills the array before each step on the same stream; no
+ * random numbers are generated inside the library.  `scratch` (DEVICE, 16-byte aligned, at least
+ * sparsk_sampling_scratch_bytes(dims), borrowed) holds the logits of a step.  Exit depths, the
+ * pending sets and the cache are unaffected by how the token is chosen.
+ * uniforms == NULL switches back to greedy decoding.  SPARSK_EINVAL for temperature <= 0 or not
+ * finite, top_p outside (0, 1], a missing, misaligned or short scratch; SPARSK_ECAPACITY if a
+ * modality has more than 196,608 ids (what one cluster of the sampling kernel holds in registers). */
+size_t sparsk_sampling_scratch_bytes(const sparsk_dims *dims /*host*/);
+int sparsk_set_sampling(sparsk_ctx *ctx, float temperature, float top_p, const float *uniforms /*device*/,
+                        void *scratch /*device*/, size_t scratch_bytes);
+
+/* The sampling kernel on its own: row i of `logits` (DEVICE float [n][vocab_text + vocab_speech])
+ * is sampled over ids [0, vocab_text) if modality[i] == 0, else over [vocab_text, vocab_text +
+ * vocab_speech), with uniforms[i]; tokens[i] receives the id (-1 if the range is empty).  All
+ * array arguments are DEVICE pointers; nothing else is written.  Enqueued on `cuda_stream`;
+ * SPARSK_EINVAL for NULL pointers, n < 1, vocab_text < 1, vocab_speech < 0, a range of more than
+ * 196,608 ids, temperature <= 0 or top_p outside (0, 1]. */
+int sparsk_nucleus_sample(const float *logits, const float *uniforms, const int32_t *modality, int32_t n,
+                          int32_t vocab_text, int32_t vocab_speech, float temperature, float top_p,
+                          int32_t *tokens, void *cuda_stream);
+
 /* Stand-alone split-KV grouped-query attention: the two kernels a decode step runs per layer
  * (partials per KV split, then the merge), on caller-described rows.  Rows are grouped: group g
  * is rows [grp_row0[g], grp_row0[g] + grp_nrows[g]) of ONE sequence at consecutive positions;

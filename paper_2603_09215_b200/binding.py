@@ -18,7 +18,8 @@ LIB_PATH = os.path.join(_HERE, "libsparsk.so")
 EXPORTS = ("sparsk_workspace_bytes", "sparsk_create", "sparsk_prefill", "sparsk_decode_step",
            "sparsk_decode_step_host", "sparsk_reset_slot", "sparsk_import_kv", "sparsk_export_kv",
            "sparsk_set_len", "sparsk_slot_state", "sparsk_set_debug", "sparsk_set_option",
-           "sparsk_kernel_time", "sparsk_kernel_time_by_class", "sparsk_check", "sparsk_phase_trace", "sparsk_attention", "sparsk_attention_scratch_bytes", "sparsk_attention_static", "sparsk_launch_count", "sparsk_last_error", "sparsk_destroy")
+           "sparsk_kernel_time", "sparsk_kernel_time_by_class", "sparsk_check", "sparsk_phase_trace", "sparsk_attention", "sparsk_attention_scratch_bytes", "sparsk_attention_static", "sparsk_sampling_scratch_bytes", "sparsk_set_sampling", "sparsk_nucleus_sample",
+           "sparsk_launch_count", "sparsk_last_error", "sparsk_destroy")
 
 OK, EINVAL, ECAPACITY, ENOHEAD, ECUDA, ESTATE, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
 
@@ -98,6 +99,12 @@ def load():
     L.sparsk_attention.argtypes = [C.POINTER(AttnArgs), vp, C.c_size_t, vp]
     L.sparsk_attention_static.restype = C.c_int
     L.sparsk_attention_static.argtypes = [C.POINTER(AttnArgs), vp, C.c_char_p, C.c_size_t]
+    L.sparsk_sampling_scratch_bytes.restype = C.c_size_t
+    L.sparsk_sampling_scratch_bytes.argtypes = [C.POINTER(Dims)]
+    L.sparsk_set_sampling.restype = C.c_int
+    L.sparsk_set_sampling.argtypes = [vp, C.c_float, C.c_float, vp, vp, C.c_size_t]
+    L.sparsk_nucleus_sample.restype = C.c_int
+    L.sparsk_nucleus_sample.argtypes = [vp, vp, vp, C.c_int32, C.c_int32, C.c_int32, C.c_float, C.c_float, vp, vp]
     L.sparsk_phase_trace.restype = C.c_int
     L.sparsk_phase_trace.argtypes = [vp, C.POINTER(C.c_int64), C.c_int32]
     L.sparsk_kernel_time_by_class.restype = C.c_int
@@ -173,6 +180,22 @@ def attention_static(args: AttnArgs, stream=None):
     buf = C.create_string_buffer(256)
     rc = load().sparsk_attention_static(C.byref(args), st, buf, len(buf))
     return rc, buf.value.decode()
+
+
+def nucleus_sample(logits: torch.Tensor, uniforms: torch.Tensor, modality: torch.Tensor, vocab_text: int,
+                   vocab_speech: int, temperature: float, top_p: float, stream=None) -> torch.Tensor:
+    """Tokens [n] (int32, device) drawn from rows of `logits` [n, vocab_text + vocab_speech] (float32)."""
+    L = load()
+    n = logits.shape[0]
+    assert logits.dtype == torch.float32 and logits.is_contiguous() and logits.shape[1] == vocab_text + vocab_speech
+    assert uniforms.dtype == torch.float32 and modality.dtype == torch.int32
+    out = torch.empty(n, dtype=torch.int32, device=logits.device)
+    st = torch.cuda.current_stream().cuda_stream if stream is None else stream
+    rc = L.sparsk_nucleus_sample(logits.data_ptr(), uniforms.data_ptr(), modality.data_ptr(), n,
+                                 vocab_text, vocab_speech, float(temperature), float(top_p), out.data_ptr(), st)
+    if rc != OK:
+        raise SparskError(rc, "sparsk_nucleus_sample")
+    return out
 
 
 def attention_scratch_bytes(n_rows: int, n_q_heads: int, head_dim: int) -> int:
@@ -284,6 +307,21 @@ class Sparsk:
         self._dbg = (hidden, logits)
         self._check(self.lib.sparsk_set_debug(self.h, None if hidden is None else hidden.data_ptr(),
                                               None if logits is None else logits.data_ptr()))
+
+    def set_sampling(self, temperature: float, top_p: float, uniforms: torch.Tensor | None):
+        """Nucleus sampling from now on, with uniforms[i] (float32, device, one per sequence of a
+        step) as the random numbers; None goes back to greedy decoding."""
+        if uniforms is None:
+            self._samp = None
+            self._check(self.lib.sparsk_set_sampling(self.h, 0.0, 1.0, None, None, 0))
+            return
+        assert uniforms.dtype == torch.float32 and uniforms.is_cuda and uniforms.numel() >= self.cd.max_seqs
+        nbytes = self.lib.sparsk_sampling_scratch_bytes(C.byref(self.cd))
+        old = getattr(self, "_samp", None)
+        scratch = old[1] if old else torch.empty(nbytes, dtype=torch.uint8, device=uniforms.device)
+        self._samp = (uniforms, scratch)
+        self._check(self.lib.sparsk_set_sampling(self.h, float(temperature), float(top_p), uniforms.data_ptr(),
+                                                 scratch.data_ptr(), nbytes))
 
     def set_option(self, name: str, value: int):
         self._check(self.lib.sparsk_set_option(self.h, name.encode(), int(value)))

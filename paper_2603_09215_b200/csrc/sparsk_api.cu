@@ -14,6 +14,7 @@
 #include "sparsk_gemm.cuh"
 #include "sparsk_gemv.cuh"
 #include "sparsk_mega.cuh"
+#include "sparsk_sample.cuh"
 #include "sparsk_step.cuh"
 #include "sparsk_tcmega.cuh"
 
@@ -79,6 +80,10 @@ struct sparsk_ctx {
     // options
     int pdl, attn_split, gemm_min_rows, use_graph, gv_ks, gv_r, gv_grid_mult;
     float *dbg_hidden, *dbg_logits;
+    // nucleus sampling (off while samp_uniforms is NULL)
+    float samp_temperature, samp_top_p;
+    const float *samp_uniforms;  // device [max_seqs], read by every decode step
+    float *samp_scratch;         // device [max_seqs][Vt + Vs]
     int64_t launches;
     // tensor-core path: TMA descriptors of every weight matrix and of the activation buffers
     // (one per box height 16, 32, 64, 128, 256)
@@ -359,6 +364,9 @@ cudaError_t run_gateup(sparsk_ctx *c, int layer, const float *h, int n_rows)
 #undef GU_CASE
 }
 
+// Where the heads leave their logits: the parity hook's buffer, else the sampler's, else nowhere.
+float *head_logits(const sparsk_ctx *c) { return c->dbg_logits ? c->dbg_logits : (c->samp_uniforms ? c->samp_scratch : nullptr); }
+
 bool use_tc(const sparsk_ctx *c, int n_rows);
 cudaError_t run_head_tc(sparsk_ctx *c, int layer, const float *h, int list, int n_rows);
 
@@ -382,7 +390,7 @@ cudaError_t run_head(sparsk_ctx *c, int layer, const float *h, int list, int n_r
     {                                                                                            \
         HeadOp<RR> op;                                                                           \
         op.w = c->head_proj[li]; op.seq_of_row = c->sd.list_seq + (size_t)list * B;              \
-        op.argmax = c->sd.argmax; op.logits = c->dbg_logits; op.d = d.d_model;                   \
+        op.argmax = c->sd.argmax; op.logits = head_logits(c); op.d = d.d_model;                   \
         op.lo = speech ? d.vocab_text : 0; op.hi = speech ? d.vocab_text + d.vocab_speech : d.vocab_text; \
         op.V = d.vocab_text + d.vocab_speech;                                                    \
         const int ng = (op.hi - op.lo + RR - 1) / RR;                                            \
@@ -616,7 +624,7 @@ cudaError_t run_head_tc(sparsk_ctx *c, int layer, const float *h, int list, int 
     if ((e = run_norm(c, h, c->head_norm[li], c->sd.list_row + (size_t)list * B, n_rows)) != cudaSuccess) return e;
     c->cur_class = KC_HEAD;
     HeadEnd ep;
-    ep.seq_of_row = c->sd.list_seq + (size_t)list * B; ep.argmax = c->sd.argmax; ep.logits = c->dbg_logits;
+    ep.seq_of_row = c->sd.list_seq + (size_t)list * B; ep.argmax = c->sd.argmax; ep.logits = head_logits(c);
     ep.lo = speech ? d.vocab_text : 0; ep.hi = speech ? d.vocab_text + d.vocab_speech : d.vocab_text;
     ep.V = d.vocab_text + d.vocab_speech;
     GemmArgs g{};
@@ -972,6 +980,7 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
     ctx->mega = 1; ctx->mk_ok = 0; ctx->mk_coop = 0; ctx->mk_bar_base = 0; ctx->mk_trace_n = 0;
     ctx->gv_ks = 0; ctx->gv_r = 0; ctx->gv_grid_mult = 1;
     ctx->dbg_hidden = nullptr; ctx->dbg_logits = nullptr;
+    ctx->samp_temperature = 0.f; ctx->samp_top_p = 1.f; ctx->samp_uniforms = nullptr; ctx->samp_scratch = nullptr;
     ctx->launches = 0;
     ctx->cur_class = KC_MISC; ctx->time_class = KC_MISC; ctx->tev_used = 0;
     ctx->stage_next = 0;
@@ -1058,6 +1067,35 @@ extern "C" int sparsk_set_debug(sparsk_ctx *ctx, float *exit_hidden, float *exit
     if (!good(ctx)) return SPARSK_ESTATE;
     ctx->dbg_hidden = exit_hidden;
     ctx->dbg_logits = exit_logits;
+    return SPARSK_OK;
+}
+
+extern "C" size_t sparsk_sampling_scratch_bytes(const sparsk_dims *dims)
+{
+    if (!dims_ok(dims)) return 0;
+    return (size_t)dims->max_seqs * ((size_t)dims->vocab_text + dims->vocab_speech) * sizeof(float);
+}
+
+extern "C" int sparsk_set_sampling(sparsk_ctx *ctx, float temperature, float top_p, const float *uniforms, void *scratch,
+                                   size_t scratch_bytes)
+{
+    if (!good(ctx)) return SPARSK_ESTATE;
+    if (!uniforms) {  // back to greedy decoding
+        ctx->samp_uniforms = nullptr;
+        ctx->samp_scratch = nullptr;
+        return SPARSK_OK;
+    }
+    if (!(temperature > 0.f) || !(temperature < INFINITY) || !(top_p > 0.f) || !(top_p <= 1.f))
+        return fail(ctx, SPARSK_EINVAL, "set_sampling: temperature %g, top_p %g", (double)temperature, (double)top_p);
+    if (ctx->dm.vocab_text > SP_MAX_RANGE || ctx->dm.vocab_speech > SP_MAX_RANGE)
+        return fail(ctx, SPARSK_ECAPACITY, "set_sampling: a modality has more than %d ids", SP_MAX_RANGE);
+    if (!scratch || ((uintptr_t)scratch % 16) || scratch_bytes < sparsk_sampling_scratch_bytes(&ctx->dm))
+        return fail(ctx, SPARSK_EINVAL, "set_sampling: scratch of %zu bytes, need %zu (16-byte aligned)", scratch_bytes,
+                    sparsk_sampling_scratch_bytes(&ctx->dm));
+    ctx->samp_temperature = temperature;
+    ctx->samp_top_p = top_p;
+    ctx->samp_uniforms = uniforms;
+    ctx->samp_scratch = (float *)scratch;
     return SPARSK_OK;
 }
 
@@ -1328,6 +1366,22 @@ extern "C" int sparsk_decode_step(sparsk_ctx *ctx, int32_t n, const int32_t *slo
     }
     for (int l = 2; l < 4; l++)
         if (n_list[l]) CU(run_head(ctx, L, h_full, l, n_list[l]));
+    if (ctx->samp_uniforms) {
+        // replace the arg max by a draw from the nucleus of the same logits (Sec. V-A)
+        SampleArgs sa{};
+        sa.logits = head_logits(ctx); sa.uniforms = ctx->samp_uniforms;
+        sa.modality = ctx->sd.modality; sa.key_out = ctx->sd.argmax; sa.token_out = nullptr;
+        sa.V = V; sa.Vt = d.vocab_text; sa.Vs = d.vocab_speech;
+        sa.inv_temperature = 1.f / ctx->samp_temperature; sa.top_p = ctx->samp_top_p;
+        const bool timed = (ctx->time_class == KC_HEAD || ctx->time_class == KC_ALL) && ctx->tev_used + 2 <= ctx->tev.size();
+        if (timed) {
+            ctx->tev_class[ctx->tev_used / 2] = KC_HEAD;
+            cudaEventRecord(ctx->tev[ctx->tev_used++], ctx->stream);
+        }
+        CU(launch_nucleus_sample(sa, n, n_list[0] + n_list[2] > 0, n_list[1] + n_list[3] > 0, ctx->stream, ctx->pdl != 0,
+                                 &ctx->launches));
+        if (timed) cudaEventRecord(ctx->tev[ctx->tev_used++], ctx->stream);
+    }
     if (ctx->dbg_hidden)
         CU(launch(ctx, debug_hidden_kernel, dim3(n), dim3(128), 0, ctx->sd, (const float *)ctx->h_lo,
                   (const float *)ctx->h_up, ctx->dbg_hidden, (int)n, d.d_model));

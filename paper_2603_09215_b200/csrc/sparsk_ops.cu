@@ -5,6 +5,7 @@
 
 #include "../../include/sparsk.h"
 #include "sparsk_attn.cuh"
+#include "sparsk_sample.cuh"
 #include "sparsk_step.cuh"
 
 using namespace sparsk;
@@ -72,4 +73,22 @@ extern "C" int sparsk_attention(const sparsk_attn_args *args, void *scratch, siz
     if (scratch_bytes < sparsk_attention_scratch_bytes(args->n_rows, args->n_q_heads, args->head_dim))
         return SPARSK_EINVAL;
     return sparsk_attention_launch(args, (char *)scratch, (cudaStream_t)cuda_stream);
+}
+
+extern "C" int sparsk_nucleus_sample(const float *logits, const float *uniforms, const int32_t *modality, int32_t n,
+                                     int32_t vocab_text, int32_t vocab_speech, float temperature, float top_p,
+                                     int32_t *tokens, void *cuda_stream)
+{
+    if (!logits || !uniforms || !modality || !tokens) return SPARSK_EINVAL;
+    if (n < 1 || vocab_text < 1 || vocab_speech < 0 || vocab_text > SP_MAX_RANGE || vocab_speech > SP_MAX_RANGE)
+        return SPARSK_EINVAL;
+    if (!(temperature > 0.f) || !(temperature < INFINITY) || !(top_p > 0.f) || !(top_p <= 1.f)) return SPARSK_EINVAL;
+    SampleArgs a{};
+    a.logits = logits; a.uniforms = uniforms; a.modality = modality;
+    a.key_out = nullptr; a.token_out = tokens;
+    a.V = vocab_text + vocab_speech; a.Vt = vocab_text; a.Vs = vocab_speech;
+    a.inv_temperature = 1.f / temperature; a.top_p = top_p;
+    return launch_nucleus_sample(a, n, true, vocab_speech > 0, (cudaStream_t)cuda_stream, false, nullptr) == cudaSuccess
+               ? SPARSK_OK
+               : SPARSK_ECUDA;
 }

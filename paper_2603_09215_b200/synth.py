@@ -157,6 +157,21 @@ def interleave(step: int, n_text: int, n_speech: int, phase: int = 0, offset: in
     return 1, before - first + offset
 
 
+def make_uniforms(n: int, seed: int) -> np.ndarray:
+    """n uniform numbers in [0, 1) as float32 (PCG64): the draws a sampling decoder consumes."""
+    g = np.random.Generator(np.random.PCG64(seed))
+    u = g.random(n, dtype=np.float32)
+    return np.minimum(u, np.float32(0.99999994))
+
+
+def make_logits(n: int, vocab: int, scale: float, seed: int) -> np.ndarray:
+    """[n, vocab] float32 logits ~ N(0, scale): flat distributions for small scales (random heads
+    give about 0.3 to 1.3), a few dominant ids for large ones."""
+    g = torch.Generator("cpu")
+    g.manual_seed(seed)
+    return torch.empty((n, vocab), dtype=torch.float32).normal_(0, scale, generator=g).numpy()
+
+
 def synth_kv(dims: dict, n: int, seed: int) -> tuple:
     """Stand-in cache contents for long-context cases where a real prefill is not affordable on
     the CPU: keys and values ~ N(0, 1) rounded to bfloat16, [L, n, Hkv*hd] uint16 each."""
