@@ -28,6 +28,12 @@ if ROOT not in sys.path:
 
 from paper_2603_09215_b200 import synth  # noqa: E402
 
+# DRAM bytes (read + write) per algorithmic byte of the persistent kernel, from its ncu capture on a
+# two-layer launch (profiles/mega_kernel_step4_b1.md: 935.38 MB read + 10.3 MB written against
+# 934.3 MB algorithmic); a launch's traffic is its layers' weights and cache, so it grows in
+# proportion to the layer passes and the ratio carries over to the full-size launches timed here.
+MEGA_DRAM_PER_ALGORITHMIC_BYTE = (935.38 + 10.3) / 934.3
+
 KC = {"qkv": 1, "attn": 2, "oproj": 3, "gateup": 4, "down": 5, "head": 6, "mega": 7, "all": 8}
 
 
@@ -438,7 +444,9 @@ def main():
         lb = run.mega_bytes - mb0
         ach = lb / (kms * 1e-3) / 1e9
         roof.update(achieved=ach, frac=ach / hbm_peak, launches_timed=kn, avg_launch_us=1e3 * kms / kn,
-                    bytes_per_launch=lb / kn, layer_passes=run.mega_layers - ml0,
+                    bytes_per_launch=lb / kn, traffic=lb / kn * MEGA_DRAM_PER_ALGORITHMIC_BYTE,
+                    traffic_source="ncu capture of a two-layer launch, scaled by layer passes",
+                    layer_passes=run.mega_layers - ml0,
                     us_per_layer=1e3 * kms / max(1, run.mega_layers - ml0))
     elif kbytes and kn:
         ach = kbytes / (kms / kn * 1e-3) / 1e9
