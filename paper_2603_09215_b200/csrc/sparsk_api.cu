@@ -10,6 +10,7 @@
 
 #include "../../include/sparsk.h"
 #include "sparsk_attn.cuh"
+#include "sparsk_attn_tc.cuh"
 #include "sparsk_common.cuh"
 #include "sparsk_gemm.cuh"
 #include "sparsk_gemv.cuh"
@@ -90,6 +91,8 @@ struct sparsk_ctx {
     bool tc_ok;
     std::vector<TmaPair> tm_wq, tm_wk, tm_wv, tm_wo, tm_wg, tm_wu, tm_wd, tm_head;
     TmaPair tm_x[5], tm_ao[5], tm_act[5], tm_x_lo[5], tm_ao_lo[5], tm_act_lo[5];
+    std::vector<CUtensorMap> tm_kc, tm_vc;  // per layer: the cache viewed as [64][slots * Hkv * S rows][hd / 64], boxes of [64][64][2]
+    int attn_tc, attn_tc_min_q;             // tcgen05 attention for blocks of at least this many query vectors
     // persistent layer-range kernel (one or two rows)
     MkLayer *mk_layers;            // device [L]
     unsigned long long *mk_bar;    // device: grid barrier counter; mk_bar_base mirrors its value
@@ -303,6 +306,7 @@ struct RowSet {
     int n_groups_h; // host count
     int max_grp_rows;
     int max_len;    // longest prefix any row attends to (host)
+    int n_big;      // groups with at least attn_tc_min_q query vectors per kv head (0: not counted, assume all)
 };
 
 cudaError_t run_qkv(sparsk_ctx *c, int layer, const float *h, const RowSet &rs)
@@ -400,6 +404,8 @@ cudaError_t run_head(sparsk_ctx *c, int layer, const float *h, int list, int n_r
 #undef HD_CASE
 }
 
+int div_up(int a, int b);
+
 cudaError_t run_attn(sparsk_ctx *c, int layer, const RowSet &rs)
 {
     const sparsk_dims &d = c->dm;
@@ -414,19 +420,75 @@ cudaError_t run_attn(sparsk_ctx *c, int layer, const RowSet &rs)
     a.n_groups = rs.n_groups;
     a.part_o = c->part_o; a.part_ml = c->part_ml; a.out = c->attn_o; a.out_lo = c->attn_o_lo;
     a.Hq = d.n_q_heads; a.Hkv = d.n_kv_heads; a.S = d.max_seq_len;
-    const AttnPlan pl = attn_plan(c->n_sm, rs.n_groups_h, rs.max_grp_rows, G, d.n_kv_heads, rs.max_len, c->attn_split);
-    a.n_qblk = pl.n_qblk;
-    a.split_len = pl.split_len;
-    a.n_splits = pl.n_splits;
     a.n_slots = d.max_seqs;
     a.n_rows = rs.n_rows;
-    const int n_splits = pl.n_splits;
-    dim3 grid(rs.n_groups_h * a.n_qblk, d.n_kv_heads, n_splits);
-    AttnPartialFn fn;
-    cudaError_t e = attn_partial_fn(d.head_dim, pl.mt, &fn);
-    if (e != cudaSuccess) return e;
-    e = launch(c, fn, grid, dim3(AT_THREADS), attn_smem_bytes(d.head_dim, pl.mt), a);
-    if (e != cudaSuccess) return e;
+    a.nq_min = 0;
+    a.nq_max = 1 << 30;
+    cudaError_t e;
+    const bool blocks_tc = c->attn_tc && c->tc_ok && d.head_dim == TA_HD && rs.max_grp_rows * G >= c->attn_tc_min_q;
+    AttnPlan pl = attn_plan(c->n_sm, rs.n_groups_h, blocks_tc ? 1 : rs.max_grp_rows, G, d.n_kv_heads, rs.max_len, c->attn_split);
+    if (blocks_tc) {
+        // Groups with many query vectors per kv head go to the tcgen05 kernel (one CTA per SM, tiles
+        // of 64 positions), the others to the mma.sync kernel; both launches cover all groups, a CTA
+        // leaves at once if its group belongs to the other, and both use one split plan so that the
+        // merge finds every partial where it expects it.
+        static bool ready = false;
+        if (!ready) {
+            if ((e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TA_SMEM)) != cudaSuccess) return e;
+            ready = true;
+        }
+        // The tcgen05 kernel wants few, long splits (about one CTA per SM from the big groups alone,
+        // its set-up is worth a few tiles), the other kernel many short ones: the first kernel's
+        // split is `mult` of the second's, and it marks the partial slots in between as empty.
+        const int n_big = rs.n_big > 0 ? rs.n_big : rs.n_groups_h;
+        const int big_ctas = std::max(1, n_big * div_up(rs.max_grp_rows * G, TA_QB) * d.n_kv_heads);
+        const int tiles = std::max(1, div_up(rs.max_len, TA_NT));
+        int s_tc = 1;
+        {   // the split count whose CTAs fill whole waves of one CTA per SM best (at least 8 tiles each)
+            double best = -1.0;
+            const int s_max = std::max(1, std::min(AT_MAX_SPLITS, tiles / 8));
+            for (int sc = 1; sc <= s_max; sc++) {
+                const long n = (long)big_ctas * sc, waves = (n + c->n_sm - 1) / c->n_sm;
+                const double eff = (double)n / (double)(waves * c->n_sm);
+                const double score = eff * (waves >= 2 ? 1.0 : 0.9);  // a second wave evens out ragged lengths
+                if (score > best + 1e-9) {
+                    best = score;
+                    s_tc = sc;
+                }
+                if (waves >= 2 && eff >= 0.9) break;
+            }
+        }
+        if (c->attn_split > 0) s_tc = pl.n_splits;
+        s_tc = std::min(s_tc, AT_MAX_SPLITS);
+        const int mult = std::max(1, std::min(AT_MAX_SPLITS / s_tc, div_up(pl.n_splits, s_tc)));
+        const int small_len = div_up(div_up(rs.max_len, s_tc * mult), TA_NT) * TA_NT;
+        pl.split_len = small_len;
+        pl.n_splits = std::max(1, div_up(rs.max_len, small_len));
+        AttnTcArgs ta;
+        ta.a = a;
+        ta.a.n_qblk = div_up(rs.max_grp_rows * G, TA_QB);
+        ta.a.split_len = small_len * mult;
+        ta.a.n_splits = pl.n_splits;
+        ta.a.nq_min = c->attn_tc_min_q;
+        ta.split_mult = mult;
+        ta.status = c->sd.counts + CNT_STATUS;
+        const int n_splits_tc = std::max(1, div_up(rs.max_len, small_len * mult));
+        dim3 grid(rs.n_groups_h * ta.a.n_qblk, d.n_kv_heads, n_splits_tc);
+        e = launch(c, attn_tc_kernel, grid, dim3(TA_THREADS), (size_t)TA_SMEM, c->tm_kc[layer - 1], c->tm_vc[layer - 1], ta);
+        if (e != cudaSuccess) return e;
+        a.nq_max = c->attn_tc_min_q - 1;
+    }
+    a.n_qblk = blocks_tc ? div_up(std::min(rs.max_grp_rows * G, c->attn_tc_min_q - 1), 16 * pl.mt) : pl.n_qblk;
+    a.split_len = pl.split_len;
+    a.n_splits = pl.n_splits;
+    if (!blocks_tc || c->attn_tc_min_q > 1) {
+        dim3 grid(rs.n_groups_h * a.n_qblk, d.n_kv_heads, a.n_splits);
+        AttnPartialFn fn;
+        e = attn_partial_fn(d.head_dim, pl.mt, &fn);
+        if (e != cudaSuccess) return e;
+        e = launch(c, fn, grid, dim3(AT_THREADS), attn_smem_bytes(d.head_dim, pl.mt), a);
+        if (e != cudaSuccess) return e;
+    }
     if (d.head_dim == 128) return launch(c, attn_merge_kernel<128>, dim3(rs.n_rows, d.n_q_heads), dim3(128), 0, a, rs.n_rows_dev);
     return launch(c, attn_merge_kernel<64>, dim3(rs.n_rows, d.n_q_heads), dim3(64), 0, a, rs.n_rows_dev);
 }
@@ -485,6 +547,18 @@ bool build_maps(sparsk_ctx *c)
     fill(c->tm_wv, c->wv, kd, d.d_model, 2 * GM_BM); fill(c->tm_wo, c->wo, d.d_model, qd, 2 * GM_BM);
     fill(c->tm_wg, c->w_gate, d.d_ffn, d.d_model, GM_BM); fill(c->tm_wu, c->w_up, d.d_ffn, d.d_model, GM_BM);
     fill(c->tm_wd, c->w_down, d.d_model, d.d_ffn, 2 * GM_BM); fill(c->tm_head, c->head_proj, V, d.d_model, 2 * GM_BM);
+    if (d.head_dim == TA_HD) {
+        const size_t lstride = (size_t)d.max_seqs * d.n_kv_heads * d.max_seq_len * d.head_dim;
+        c->tm_kc.resize(L);
+        c->tm_vc.resize(L);
+        for (int l = 0; l < L && ok; l++) {
+            TmaPair t;
+            ok = ok && encode_maps(fn, &t, c->kcache + l * lstride, (size_t)d.max_seqs * d.n_kv_heads * d.max_seq_len, d.head_dim, TA_NT);
+            c->tm_kc[l] = t.m3;
+            ok = ok && encode_maps(fn, &t, c->vcache + l * lstride, (size_t)d.max_seqs * d.n_kv_heads * d.max_seq_len, d.head_dim, TA_NT);
+            c->tm_vc[l] = t.m3;
+        }
+    }
     for (int b = 0; b < 5; b++) {
         const int box = 16 << b;
         ok = ok && encode_maps(fn, &c->tm_x[b], c->xnorm, c->cap_rows, d.d_model, box);
@@ -977,6 +1051,7 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
     ctx->tc_kb = 0;
     ctx->mk_max_rows = 2;
     ctx->tcmega = 0; ctx->tk_ok = 0;
+    ctx->attn_tc = 1; ctx->attn_tc_min_q = 33;
     ctx->mega = 1; ctx->mk_ok = 0; ctx->mk_coop = 0; ctx->mk_bar_base = 0; ctx->mk_trace_n = 0;
     ctx->gv_ks = 0; ctx->gv_r = 0; ctx->gv_grid_mult = 1;
     ctx->dbg_hidden = nullptr; ctx->dbg_logits = nullptr;
@@ -1028,6 +1103,10 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
             }
         }
         if ((ce = cudaMemcpyAsync(ctx->rope, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess ||
+            // the cache starts out as zeros: the tcgen05 attention kernel multiplies whole 64-position
+            // tiles, and a masked weight of zero times an unwritten NaN pattern would still be NaN
+            (ce = cudaMemsetAsync(ctx->kcache, 0, sizeof(bf16) * (size_t)dims->n_layers * dims->max_seqs * dims->n_kv_heads * dims->max_seq_len * dims->head_dim, ctx->stream)) != cudaSuccess ||
+            (ce = cudaMemsetAsync(ctx->vcache, 0, sizeof(bf16) * (size_t)dims->n_layers * dims->max_seqs * dims->n_kv_heads * dims->max_seq_len * dims->head_dim, ctx->stream)) != cudaSuccess ||
             (ce = cudaMemsetAsync(ctx->kv_len, 0, sizeof(int) * dims->max_seqs, ctx->stream)) != cudaSuccess ||
             (ce = cudaMemsetAsync(ctx->pend_cnt, 0, sizeof(int) * dims->max_seqs, ctx->stream)) != cudaSuccess ||
             (ce = cudaMemsetAsync(ctx->sd.counts, 0, sizeof(int) * 8, ctx->stream)) != cudaSuccess ||
@@ -1110,6 +1189,8 @@ extern "C" int sparsk_set_option(sparsk_ctx *ctx, const char *name, int64_t valu
     else if (!strcmp(name, "gemv_ks") && (value == 0 || value == 1 || value == 2 || value == 4 || value == 8 || value == 16)) ctx->gv_ks = (int)value;
     else if (!strcmp(name, "mega") && (value == 0 || value == 1)) ctx->mega = (int)value;
     else if (!strcmp(name, "tcmega") && (value == 0 || value == 1)) ctx->tcmega = (int)value;
+    else if (!strcmp(name, "attn_tc") && (value == 0 || value == 1)) ctx->attn_tc = (int)value;
+    else if (!strcmp(name, "attn_tc_min_q") && value >= 1 && value <= (1 << 20)) ctx->attn_tc_min_q = (int)value;
     else if (!strcmp(name, "mega_max_rows") && value >= 1 && value <= MK_MAX_ROWS) ctx->mk_max_rows = (int)value;
     else if (!strcmp(name, "gemm_kb") && (value == 0 || value == 1)) ctx->tc_kb = (int)value;
     else if (!strcmp(name, "gemv_r") && (value == 0 || value == 1 || value == 2 || value == 4)) ctx->gv_r = (int)value;
@@ -1293,7 +1374,8 @@ extern "C" int sparsk_decode_step(sparsk_ctx *ctx, int32_t n, const int32_t *slo
     // ---- host mirror of the schedule: validates, and sizes the launches
     std::vector<char> seen(B, 0);
     int n_list[4] = {0, 0, 0, 0};
-    int m_up = 0, n_grp = 0, max_grp = 1, max_len_lo = 0, max_len_up = 0;
+    int m_up = 0, n_grp = 0, max_grp = 1, max_len_lo = 0, max_len_up = 0, n_big = 0;
+    const int G_heads = d.n_q_heads / d.n_kv_heads;
     for (int i = 0; i < n; i++) {
         const int s = slots[i];
         if (s < 0 || s >= B || seen[s]) return fail(ctx, SPARSK_EINVAL, "decode_step: slot %d invalid or repeated", s);
@@ -1311,6 +1393,7 @@ extern "C" int sparsk_decode_step(sparsk_ctx *ctx, int32_t n, const int32_t *slo
             m_up += ctx->h_pend[s] + 1;
             n_grp++;
             max_grp = std::max(max_grp, ctx->h_pend[s] + 1);
+            n_big += (ctx->h_pend[s] + 1) * G_heads >= ctx->attn_tc_min_q;
             max_len_up = std::max(max_len_up, ctx->h_len[s] + 1);
         }
     }
@@ -1360,7 +1443,7 @@ extern "C" int sparsk_decode_step(sparsk_ctx *ctx, int32_t n, const int32_t *slo
         CU(launch(ctx, gather_upper_kernel, dim3(m_up), dim3(128), 0, ctx->sd, (const float *)ctx->h_lo,
                   (const float *)ctx->pend_h, ctx->h_up, d.d_model, d.max_pending));
         RowSet up{ctx->sd.up_slot, ctx->sd.up_pos, ctx->sd.up_grp_row0, ctx->sd.up_grp_nrows, ctx->sd.counts + CNT_NGRP,
-                  ctx->sd.counts + CNT_MUP, m_up, n_grp, max_grp, max_len_up};
+                  ctx->sd.counts + CNT_MUP, m_up, n_grp, max_grp, max_len_up, n_big};
         CU(run_layers(ctx, e + 1, L, ctx->h_up, up));
         h_full = ctx->h_up;
     }

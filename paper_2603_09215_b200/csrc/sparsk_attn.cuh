@@ -99,6 +99,7 @@ struct AttnArgs {
     int Hq, Hkv, S, n_qblk, n_splits, split_len;
     int n_slots;              // slots in the cache; rows naming another slot are skipped
     int n_rows;               // rows in q/out; groups reaching beyond them are skipped
+    int nq_min, nq_max;       // only groups with this many query vectors per kv head (another launch takes the rest)
 };
 
 __device__ __forceinline__ void cp_async16(void *dst, const void *src, int src_bytes)
@@ -157,7 +158,7 @@ __device__ __forceinline__ void attn_partial_body(const AttnArgs &a, int bx, int
     if (row0 < 0 || nrows < 1 || row0 + nrows > a.n_rows) return;
     const int nq = nrows * G;
     const int q0 = qb * QB;
-    if (q0 >= nq) return;
+    if (q0 >= nq || nq < a.nq_min || nq > a.nq_max) return;
     const int nq_here = min(QB, nq - q0);
     const int slot = a.row_slot[row0], pos0 = a.row_pos[row0];
     const int lane = tid & 31, warp = tid >> 5;

@@ -1,0 +1,411 @@
+// Split-KV attention for blocks of many query vectors on the 5th-generation tensor cores.
+//
+// A refresh step of a sequence with 16 query heads per kv head and three pending positions has
+// 64 query vectors that share one K/V stream (Algorithm 1: the pending positions and the current
+// one go through the upper layers as one causal block).  With two-term bf16 operands that is 128
+// flop per cache byte: beyond what mma.sync delivers, so the block kernel of sparsk_attn.cuh is
+// tensor-bound there.  This kernel runs the same arithmetic on tcgen05:
+//
+//   S = Q K^T : A = the block's query vectors (up to 128 rows, hi and lo planes, K-major, written
+//               once into swizzled shared memory), B = a [64 positions x 128] K tile exactly as
+//               TMA delivers it from the cache (K-major), accumulator [128 x 64] fp32 in TMEM
+//   O_t = P V : A = the tile's softmax weights (hi and lo planes, written by the softmax warps
+//               into swizzled shared memory), B = the V tile as delivered (positions x head dim =
+//               MN-major), accumulated over all tiles in a [128 x 128] fp32 TMEM accumulator that
+//               the softmax warps rescale in place (tcgen05.ld / st) when a tile raises a row's
+//               running maximum
+//
+// CTA = (group, block of 128 query vectors, kv head, KV split); warp 0 issues the TMA copies of a
+// three-stage K/V ring, warp 1 issues the MMAs and owns the TMEM allocation, warps 2..5 (thread =
+// query vector = TMEM lane) do the softmax and keep the output row.  S is double buffered so that
+// the next tile's scores are computed while this tile's weights are being formed.  The partials
+// (unnormalised output, running max, running sum per split) have the layout of the other
+// attention kernel, and attn_merge_kernel merges them.  Every wait is bounded.
+#pragma once
+
+#include "sparsk_attn.cuh"
+#include "sparsk_gemm.cuh"
+
+namespace sparsk {
+
+constexpr int TA_THREADS = 192;
+constexpr int TA_QB = 128;      // query vectors per CTA (UMMA M)
+constexpr int TA_NT = 64;       // positions per tile
+constexpr int TA_HD = 128;      // head dimension this kernel is built for
+constexpr int TA_STAGES = 3;
+constexpr float TA_RAISE = 11.f;  // a row's reference maximum (in units of log2 e) moves only when a tile exceeds it by this much
+constexpr int TA_Q_BYTES = 2 * TA_QB * TA_HD * 2;    // hi and lo planes: 64 KB
+constexpr int TA_P_BYTES = 2 * TA_QB * TA_NT * 2;    // hi and lo planes: 32 KB
+constexpr int TA_KV_BYTES = 2 * TA_NT * TA_HD * 2;   // K and V tile of a stage: 32 KB
+constexpr int TA_SMEM = 1024 + TA_Q_BYTES + TA_P_BYTES + TA_STAGES * TA_KV_BYTES;
+
+struct AttnTcArgs {
+    AttnArgs a;        // q32, row and group arrays, partial buffers, shapes, the split plan
+    int split_mult;    // this kernel's split s fills partial slot s * split_mult of the a.n_splits slots a
+                       // row has (the slots in between are marked empty): its splits are split_mult times
+                       // as long as those of the kernel that takes the small groups of the same launch set
+    int *status;       // device status word (ST_TIMEOUT on a wait that ran out)
+};
+
+// MN-major operand with the 128-byte swizzle: 64 contiguous elements per row of 128 bytes, groups
+// of eight rows 1024 bytes apart (stride offset), the next 64 elements `lbo` bytes on (leading offset).
+__device__ __forceinline__ uint64_t umma_desc_sw128_mn(uint32_t smem_addr, uint32_t lbo_bytes)
+{
+    return (uint64_t)((smem_addr & 0x3ffffu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+// bf16 x bf16 -> fp32, M = 128, N = n, A K-major; B K-major or (b_mn) MN-major.
+__device__ __forceinline__ uint32_t umma_idesc_bf16_ex(int n, bool b_mn)
+{
+    return umma_idesc_bf16(n) | (b_mn ? (1u << 16) : 0u);
+}
+__device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+
+__global__ void __launch_bounds__(TA_THREADS, 1)
+    attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const AttnTcArgs args)
+{
+    extern __shared__ __align__(1024) unsigned char ta_smem[];
+    __shared__ __align__(8) uint64_t kv_full[TA_STAGES], kv_empty[TA_STAGES], s_full[2], s_empty[2], p_full, o_full;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int giving_up_s, never_s;
+    volatile int *giving_up = &giving_up_s;
+    const AttnArgs &a = args.a;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t base = (smem_u32(ta_smem) + 1023u) & ~1023u;
+    unsigned char *base_p = ta_smem + (base - smem_u32(ta_smem));
+    const uint32_t q_hi = base, q_lo = base + TA_Q_BYTES / 2;
+    const uint32_t p_hi = base + TA_Q_BYTES, p_lo = p_hi + TA_P_BYTES / 2;
+    const uint32_t kv0 = base + TA_Q_BYTES + TA_P_BYTES;
+
+    // ---- what this CTA works on (every thread computes the same); a CTA whose group belongs to
+    // the other kernel, or does not exist, leaves before it sets anything up
+    griddep_wait();
+    griddep_launch();
+    const int bx = blockIdx.x, hk = blockIdx.y, sp = blockIdx.z;
+    const int g = bx / a.n_qblk, qb = bx % a.n_qblk;
+    const int G = a.Hq / a.Hkv;
+    bool live = g < *a.n_groups;
+    int row0 = 0, nrows = 0;
+    if (live) {
+        row0 = a.grp_row0[g];
+        nrows = a.grp_nrows[g];
+        live = row0 >= 0 && nrows >= 1 && row0 + nrows <= a.n_rows;
+    }
+    const int nq = nrows * G, q0 = qb * TA_QB;
+    live = live && q0 < nq && nq >= a.nq_min && nq <= a.nq_max;
+    if (!live) return;
+    const int nq_here = min(TA_QB, nq - q0);
+    const int slot = a.row_slot[row0], pos0 = a.row_pos[row0];
+    const bool sane = slot >= 0 && slot < a.n_slots && pos0 >= 0;
+    const int last_row = (q0 + nq_here - 1) / G;
+    const int kv_end_all = sane ? min(pos0 + last_row + 1, a.S) : 0;
+    const int s_beg = sp * a.split_len;
+    const int s_end = min(s_beg + a.split_len, kv_end_all);
+    const int n_tiles = s_end > s_beg ? (s_end - s_beg + TA_NT - 1) / TA_NT : 0;
+    const int cache_row0 = ((sane ? slot : 0) * a.Hkv + hk) * a.S;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < TA_STAGES; s++) {
+            mbar_init(&kv_full[s], 1);
+            mbar_init(&kv_empty[s], 1);
+        }
+        for (int b = 0; b < 2; b++) {
+            mbar_init(&s_full[b], 1);
+            mbar_init(&s_empty[b], 128);
+        }
+        mbar_init(&p_full, 128);
+        mbar_init(&o_full, 1);
+        giving_up_s = 0;
+        never_s = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(256)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+
+    // ---- the queries, as two bf16 planes in the swizzled K-major layout (thread = query vector)
+    if (warp >= 2 && n_tiles > 0) {
+        const int qi = (warp & 3) * 32 + lane;
+        const bool have = qi < nq_here;
+        const int qg = q0 + qi, r = qg / G, j = qg % G;
+        const float *src = a.q32 + (size_t)(row0 + (have ? r : 0)) * a.Hq * TA_HD + (hk * G + (have ? j : 0)) * TA_HD;
+#pragma unroll
+        for (int c = 0; c < TA_HD / 8; c++) {
+            uint4 hi = make_uint4(0, 0, 0, 0), lo = hi;
+            if (have) {
+                const float4 x0 = *reinterpret_cast<const float4 *>(src + c * 8);
+                const float4 x1 = *reinterpret_cast<const float4 *>(src + c * 8 + 4);
+                const float v[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+                split8(v, hi, lo);
+            }
+            const uint32_t off = (uint32_t)(c >> 3) * (TA_QB * 128) + (uint32_t)qi * 128 + (uint32_t)(((c & 7) ^ (qi & 7)) << 4);
+            *reinterpret_cast<uint4 *>(base_p + off) = hi;
+            *reinterpret_cast<uint4 *>(base_p + TA_Q_BYTES / 2 + off) = lo;
+        }
+        asm volatile("fence.proxy.async;" ::: "memory");  // the MMAs read these through the async proxy
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+    const uint32_t t_s0 = tmem_base, t_o = tmem_base + 128;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ producer
+        // One thread needs a few hundred nanoseconds per TMA copy, so a tile is two copies (the
+        // [64][rows][2] view of the cache brings both 64-column halves of K, or of V, at once)
+        // issued by two lanes side by side.
+        uint32_t issued = 0;
+        bool ok = true;
+        for (int t = 0; t < n_tiles && ok; t++) {
+            const int st = t % TA_STAGES;
+            int go = 1;
+            if (lane == 0) {
+                go = mbar_wait(&kv_empty[st], ((t / TA_STAGES) & 1) ^ 1, giving_up, args.status) ? 1 : 0;
+                if (go) mbar_expect_tx(&kv_full[st], TA_KV_BYTES);
+            }
+            go = __shfl_sync(0xffffffffu, go, 0);
+            if (!(ok = go != 0)) break;
+            const uint32_t dst = kv0 + (uint32_t)st * TA_KV_BYTES;
+            const int y = cache_row0 + s_beg + t * TA_NT;
+            if (lane == 0) tma_load_3d(dst, &map_k, &kv_full[st], 0, y, 0);
+            if (lane == 1) tma_load_3d(dst + 16384, &map_v, &kv_full[st], 0, y, 0);
+            issued++;
+        }
+        // never leave with copies in flight
+        if (lane == 0)
+            for (int st = 0; st < TA_STAGES; st++)
+                if (issued > (uint32_t)st)
+                    mbar_wait(&kv_full[st], ((issued - 1 - st) / TA_STAGES) & 1, &never_s, nullptr, 2000000ull);
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0 && n_tiles > 0) {
+            const uint32_t idesc_s = umma_idesc_bf16_ex(TA_NT, false), idesc_o = umma_idesc_bf16_ex(TA_HD, true);
+            bool ok = true;
+            auto issue_s = [&](int t) {
+                const int st = t % TA_STAGES, b = t & 1;
+                if (!(ok = mbar_wait(&kv_full[st], (t / TA_STAGES) & 1, giving_up, args.status))) return;
+                if (!(ok = mbar_wait(&s_empty[b], ((t >> 1) & 1) ^ 1, giving_up, args.status))) return;
+                tc_fence_after();
+                const uint32_t kt = kv0 + (uint32_t)st * TA_KV_BYTES, d = t_s0 + (uint32_t)b * TA_NT;
+#pragma unroll
+                for (int kk = 0; kk < TA_HD / 16; kk++) {
+                    const uint32_t qoff = (uint32_t)(kk >> 2) * (TA_QB * 128) + (uint32_t)(kk & 3) * 32;
+                    const uint64_t db = umma_desc_sw128(kt + (uint32_t)(kk >> 2) * 8192 + (uint32_t)(kk & 3) * 32);
+                    umma_bf16(d, umma_desc_sw128(q_hi + qoff), db, idesc_s, kk > 0);
+                    umma_bf16(d, umma_desc_sw128(q_lo + qoff), db, idesc_s, 1);
+                }
+                umma_commit(&s_full[b]);
+            };
+            issue_s(0);
+            for (int t = 0; t < n_tiles && ok; t++) {
+                if (t + 1 < n_tiles) issue_s(t + 1);
+                if (!ok) break;
+                const int st = t % TA_STAGES;
+                if (!(ok = mbar_wait(&p_full, t & 1, giving_up, args.status))) break;
+                tc_fence_after();
+                const uint32_t vt = kv0 + (uint32_t)st * TA_KV_BYTES + 16384;
+#pragma unroll
+                for (int kk = 0; kk < TA_NT / 16; kk++) {
+                    const uint64_t dv = umma_desc_sw128_mn(vt + (uint32_t)kk * 2048, 8192);
+                    umma_bf16(t_o, umma_desc_sw128(p_hi + (uint32_t)kk * 32), dv, idesc_o, t > 0 || kk > 0);
+                    umma_bf16(t_o, umma_desc_sw128(p_lo + (uint32_t)kk * 32), dv, idesc_o, 1);
+                }
+                umma_commit(&kv_empty[st]);  // the stage and the weights are free once these have read them
+                umma_commit(&o_full);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ softmax and output (thread = query vector)
+        const int quad = warp & 3, qi = quad * 32 + lane;
+        const bool have = qi < nq_here;
+        const int limit = have ? pos0 + (q0 + qi) / G : -1;
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        const float scale = rsqrtf((float)TA_HD);
+        float m_run = -INFINITY, l_run = 0.f;
+        bool ok = true;
+        // The choice below is per WARP: tcgen05.ld/st are warp-wide (.sync.aligned) instructions, so
+        // a warp either runs the whole softmax path with all its lanes (lanes without a query
+        // vector see everything masked) or none of it.
+        const bool warp_idle = quad * 32 >= nq_here;
+        if (warp_idle && n_tiles > 0) {
+            // a warp without query vectors: its rows of the weight planes stay zero, and it only
+            // keeps the barriers' arrival counts whole
+            for (int c = 0; c < 8; c++) {
+                *reinterpret_cast<uint4 *>(base_p + TA_Q_BYTES + (uint32_t)qi * 128 + (c << 4)) = make_uint4(0, 0, 0, 0);
+                *reinterpret_cast<uint4 *>(base_p + TA_Q_BYTES + TA_P_BYTES / 2 + (uint32_t)qi * 128 + (c << 4)) = make_uint4(0, 0, 0, 0);
+            }
+            asm volatile("fence.proxy.async;" ::: "memory");
+            for (int t = 0; t < n_tiles && ok; t++) {
+                if (!(ok = mbar_wait(&s_full[t & 1], (t >> 1) & 1, giving_up, args.status))) break;
+                if (t > 0 && !(ok = mbar_wait(&o_full, (t - 1) & 1, giving_up, args.status))) break;
+                mbar_arrive(&s_empty[t & 1]);
+                mbar_arrive(&p_full);
+            }
+        } else if (n_tiles > 0) {
+            // The output row accumulates in TMEM over all tiles (the MMAs add into it), relative to
+            // the running maximum m_run; when a tile raises a row's maximum the warp rescales its
+            // rows of the accumulator in place before the tile's product is issued.
+            for (int t = 0; t < n_tiles && ok; t++) {
+                const int b = t & 1;
+                ok = mbar_wait(&s_full[b], (t >> 1) & 1, giving_up, args.status);
+                if (!(ok = __all_sync(0xffffffffu, ok))) break;  // the loads below are warp-wide
+                tc_fence_after();
+                const uint32_t ts = t_s0 + lane_addr + (uint32_t)b * TA_NT;
+                const int p0 = s_beg + t * TA_NT;
+                uint32_t sr[4][16];
+#pragma unroll
+                for (int c = 0; c < 4; c++) tmem_ld16_nowait(ts + c * 16, sr[c]);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                tc_fence_before();
+                mbar_arrive(&s_empty[b]);  // the scores are in registers
+                // scores in units of log2(e): one multiply-add and one ex2 per weight.  A tile that
+                // lies wholly inside what every row of the warp may see (the common case: only a
+                // split's last tiles touch the causal edge or the split's end) needs no masking.
+                const float c2 = scale * 1.4426950408889634f;
+                const int min_limit = __reduce_min_sync(0xffffffffu, have ? limit : 0x7fffffff);
+                const bool full_tile = p0 + TA_NT <= s_end && p0 + TA_NT - 1 <= min_limit &&
+                                       __all_sync(0xffffffffu, have);
+                float tmax = -INFINITY;
+                if (full_tile) {
+#pragma unroll
+                    for (int c = 0; c < 4; c++)
+#pragma unroll
+                        for (int i = 0; i < 16; i++) {
+                            const float x = __uint_as_float(sr[c][i]) * c2;
+                            sr[c][i] = __float_as_uint(x);
+                            tmax = fmaxf(tmax, x);
+                        }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 4; c++)
+#pragma unroll
+                        for (int i = 0; i < 16; i++) {
+                            const int p = p0 + c * 16 + i;
+                            const float x = (p < s_end && p <= limit) ? __uint_as_float(sr[c][i]) * c2 : -INFINITY;
+                            sr[c][i] = __float_as_uint(x);
+                            tmax = fmaxf(tmax, x);
+                        }
+                }
+                // The reference maximum is allowed to lag the true one by TA_RAISE (weights then reach
+                // 2^11, which two bf16 terms and fp32 sums carry without loss): otherwise some lane of
+                // the warp would see a new maximum in most tiles and the accumulator would be
+                // rescaled nearly every time.  Partials stay exact: (o, l) are relative to m_run.
+                const bool raise = tmax > m_run + TA_RAISE;
+                const float m_new = raise ? tmax : m_run;
+                const float factor = raise ? exp2f(m_run - m_new) : 1.f;  // 2^(-inf) = 0 on the first live tile
+                const float m_ref = m_new == -INFINITY ? 0.f : m_new;  // a row that has seen nothing yet: all weights 0
+                float psum = 0.f;
+                uint4 whi[8], wlo[8];
+#pragma unroll
+                for (int c = 0; c < 8; c++) {
+                    float w[8];
+#pragma unroll
+                    for (int i = 0; i < 8; i++) {
+                        w[i] = exp2f(__uint_as_float(sr[c >> 1][(c & 1) * 8 + i]) - m_ref);  // 2^(-inf) = 0 for masked positions
+                        psum += w[i];
+                    }
+                    split8(w, whi[c], wlo[c]);
+                }
+                // the previous product has read the weight planes and is in the accumulator
+                if (t > 0) {
+                    ok = mbar_wait(&o_full, (t - 1) & 1, giving_up, args.status);
+                    if (!(ok = __all_sync(0xffffffffu, ok))) break;
+                    tc_fence_after();
+                    if (__any_sync(0xffffffffu, raise)) {
+#pragma unroll
+                        for (int c0 = 0; c0 < TA_HD; c0 += 32) {
+                            uint32_t r0[16], r1[16];
+                            tmem_ld16_nowait(t_o + lane_addr + c0, r0);
+                            tmem_ld16_nowait(t_o + lane_addr + c0 + 16, r1);
+                            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                            for (int i = 0; i < 16; i++) {
+                                r0[i] = __float_as_uint(__uint_as_float(r0[i]) * factor);
+                                r1[i] = __float_as_uint(__uint_as_float(r1[i]) * factor);
+                            }
+                            tmem_st16(t_o + lane_addr + c0, r0);
+                            tmem_st16(t_o + lane_addr + c0 + 16, r1);
+                        }
+                        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < 8; c++) {
+                    const uint32_t off = (uint32_t)qi * 128 + (uint32_t)((c ^ (qi & 7)) << 4);
+                    *reinterpret_cast<uint4 *>(base_p + TA_Q_BYTES + off) = whi[c];
+                    *reinterpret_cast<uint4 *>(base_p + TA_Q_BYTES + TA_P_BYTES / 2 + off) = wlo[c];
+                }
+                tc_fence_before();
+                asm volatile("fence.proxy.async;" ::: "memory");
+                mbar_arrive(&p_full);
+                l_run = l_run * factor + psum;
+                m_run = m_new;
+            }
+        }
+        float o[TA_HD];
+        if (!warp_idle && n_tiles > 0 && ok) {
+            ok = mbar_wait(&o_full, (n_tiles - 1) & 1, giving_up, args.status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (ok) {
+                tc_fence_after();
+#pragma unroll
+                for (int c0 = 0; c0 < TA_HD; c0 += 64) {
+                    uint32_t r[4][16];
+#pragma unroll
+                    for (int c = 0; c < 4; c++) tmem_ld16_nowait(t_o + lane_addr + c0 + c * 16, r[c]);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                    for (int c = 0; c < 4; c++)
+#pragma unroll
+                        for (int i = 0; i < 16; i++) o[c0 + c * 16 + i] = __uint_as_float(r[c][i]);
+                }
+                tc_fence_before();
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < TA_HD; i++) o[i] = 0.f;
+        }
+        if (have && ok) {
+            const int qg = q0 + qi, r = qg / G, j = qg % G;
+            const size_t cell0 = ((size_t)(row0 + r) * a.Hq + hk * G + j) * a.n_splits;
+            const int first = sp * args.split_mult;
+            if (first < a.n_splits) {
+                float *dst = a.part_o + (cell0 + first) * TA_HD;
+#pragma unroll
+                for (int i = 0; i < TA_HD; i += 4) *reinterpret_cast<float4 *>(dst + i) = make_float4(o[i], o[i + 1], o[i + 2], o[i + 3]);
+                a.part_ml[cell0 + first] = make_float2(m_run * 0.6931471805599453f, l_run);  // back to natural-log units
+            }
+            for (int e = first + 1; e < min(first + args.split_mult, a.n_splits); e++)
+                a.part_ml[cell0 + e] = make_float2(-INFINITY, 0.f);
+        }
+    }
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256) : "memory");
+    }
+}
+
+}  // namespace sparsk

@@ -53,6 +53,7 @@ int sparsk_attention_launch(const sparsk_attn_args *p, char *scratch, cudaStream
     a.part_ml = reinterpret_cast<float2 *>(scratch + 256 + up256(cells * p->head_dim * sizeof(float)));
     a.out = (bf16 *)p->out;
     a.Hq = p->n_q_heads; a.Hkv = p->n_kv_heads; a.S = p->cache_len; a.n_slots = p->n_slots; a.n_rows = p->n_rows;
+    a.nq_min = 0; a.nq_max = 1 << 30;
     const AttnPlan pl = attn_plan(n_sm, p->n_groups, p->max_grp_rows, p->n_q_heads / p->n_kv_heads,
                                   p->n_kv_heads, p->max_len, 0);
     a.n_qblk = pl.n_qblk; a.split_len = pl.split_len; a.n_splits = pl.n_splits;

@@ -86,6 +86,7 @@ __device__ __forceinline__ void tk_attention(const TkArgs &a, const TkLayer *L, 
     at.part_o = a.part_o; at.part_ml = a.part_ml; at.out = a.ao_hi_p; at.out_lo = a.ao_lo_p;
     at.Hq = a.Hq; at.Hkv = a.Hkv; at.S = a.S; at.n_qblk = a.att_qblk; at.n_splits = a.att_splits;
     at.split_len = a.att_split_len; at.n_slots = a.n_slots; at.n_rows = a.m_rows;
+    at.nq_min = 0; at.nq_max = 1 << 30;
     const int grp = threadIdx.x >> 7, tid = threadIdx.x & 127;
     unsigned char *my = smem + (size_t)grp * TK_ATT_BYTES;
     const TkGroupSync sync{4 + grp};

@@ -103,6 +103,37 @@ def test_heterogeneous_batch_matches_per_sequence_oracle(util, min_rows, tcmega)
     P.close()
 
 
+MICRO128 = dict(n_layers=3, d_model=192, n_q_heads=8, n_kv_heads=1, head_dim=128, d_ffn=320,
+                vocab_text=211, vocab_speech=77, rms_eps=1e-6, rope_base=10000.0)
+
+
+@pytest.mark.parametrize("min_q,split", [(33, 0), (1, 0), (1, 64)])
+def test_tensor_core_attention_for_blocks_of_query_vectors(util, min_q, split):
+    """head_dim 128 with eight query heads per kv head: flushes of five pending rows + current
+    (48 query vectors), prefill chunks of 24 rows (192 query vectors = two blocks of 128) and,
+    with min_q = 1, single rows too go through the tcgen05 attention kernel; with 64-position
+    splits a pass has several KV splits and ragged last tiles."""
+    dims = synth.model_dims(MICRO128, 1, 6, 0)
+    w = synth.make_weights(dims, seed=3)
+    B = 3
+    prompts = synth.make_prompts(dims, B, 70, 150, seed=12)
+    P = util.Pair(dims, w, B, 150 + 64, 5, prefill_rows=24,
+                  options={"attn_tc_min_q": min_q, "attn_split": split})
+    P.prefill(prompts)
+    for s in range(B):
+        P.check_cache(s, range(1, 4), len(prompts[s]) - 1)
+    phases = [0, 3, 5]
+    for g in range(30):
+        mc = [synth.interleave(g, 1, 6, ph) for ph in phases]
+        P.step([m for m, _ in mc], [c for _, c in mc])
+    for s in range(B):
+        ln, pend = P.g.slot_state(s)
+        P.check_cache(s, range(1, 2), ln)
+        P.check_cache(s, range(2, 4), ln - pend)
+    print("tc attention", P.stats)
+    P.close()
+
+
 def test_subset_of_slots_and_slot_reuse(util):
     """Steps may name any subset of slots in any order; a reset slot starts over."""
     dims = synth.model_dims("tiny", 2, 3, 0)
