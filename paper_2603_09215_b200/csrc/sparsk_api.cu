@@ -426,7 +426,11 @@ cudaError_t run_attn(sparsk_ctx *c, int layer, const RowSet &rs)
     a.nq_max = 1 << 30;
     cudaError_t e;
     const bool blocks_tc = c->attn_tc && c->tc_ok && d.head_dim == TA_HD && rs.max_grp_rows * G >= c->attn_tc_min_q;
-    AttnPlan pl = attn_plan(c->n_sm, rs.n_groups_h, blocks_tc ? 1 : rs.max_grp_rows, G, d.n_kv_heads, rs.max_len, c->attn_split);
+    // groups the tcgen05 kernel takes (the host knows every group's row count) and the rest
+    const int n_big = blocks_tc ? (rs.n_big > 0 ? rs.n_big : rs.n_groups_h) : 0;
+    const int n_small = rs.n_groups_h - n_big;
+    AttnPlan pl = attn_plan(c->n_sm, blocks_tc ? std::max(1, n_small) : rs.n_groups_h, blocks_tc ? 1 : rs.max_grp_rows, G,
+                            d.n_kv_heads, rs.max_len, c->attn_split);
     if (blocks_tc) {
         // Groups with many query vectors per kv head go to the tcgen05 kernel (one CTA per SM, tiles
         // of 64 positions), the others to the mma.sync kernel; both launches cover all groups, a CTA
@@ -440,7 +444,6 @@ cudaError_t run_attn(sparsk_ctx *c, int layer, const RowSet &rs)
         // The tcgen05 kernel wants few, long splits (about one CTA per SM from the big groups alone,
         // its set-up is worth a few tiles), the other kernel many short ones: the first kernel's
         // split is `mult` of the second's, and it marks the partial slots in between as empty.
-        const int n_big = rs.n_big > 0 ? rs.n_big : rs.n_groups_h;
         const int big_ctas = std::max(1, n_big * div_up(rs.max_grp_rows * G, TA_QB) * d.n_kv_heads);
         const int tiles = std::max(1, div_up(rs.max_len, TA_NT));
         int s_tc = 1;
@@ -481,7 +484,7 @@ cudaError_t run_attn(sparsk_ctx *c, int layer, const RowSet &rs)
     a.n_qblk = blocks_tc ? div_up(std::min(rs.max_grp_rows * G, c->attn_tc_min_q - 1), 16 * pl.mt) : pl.n_qblk;
     a.split_len = pl.split_len;
     a.n_splits = pl.n_splits;
-    if (!blocks_tc || c->attn_tc_min_q > 1) {
+    if (!blocks_tc || (c->attn_tc_min_q > 1 && n_small > 0)) {
         dim3 grid(rs.n_groups_h * a.n_qblk, d.n_kv_heads, a.n_splits);
         AttnPartialFn fn;
         e = attn_partial_fn(d.head_dim, pl.mt, &fn);
