@@ -16,8 +16,8 @@
 //               running maximum
 //
 // CTA = (group, block of 128 query vectors, kv head, KV split); warp 0 issues the TMA copies of a
-// three-stage K/V ring, warp 1 issues the MMAs and owns the TMEM allocation, warps 2..5 (thread =
-// query vector = TMEM lane) do the softmax and keep the output row.  S is double buffered so that
+// three-stage K/V ring, warp 1 issues the MMAs and owns the TMEM allocation, warps 2..9 do the
+// softmax (thread = query vector = TMEM lane, two warps per lane quadrant with half the columns each).  S is double buffered so that
 // the next tile's scores are computed while this tile's weights are being formed.  The partials
 // (unnormalised output, running max, running sum per split) have the layout of the other
 // attention kernel, and attn_merge_kernel merges them.  Every wait is bounded.
@@ -28,7 +28,7 @@
 
 namespace sparsk {
 
-constexpr int TA_THREADS = 192;
+constexpr int TA_THREADS = 320;   // TMA warp, MMA warp, eight softmax warps
 constexpr int TA_QB = 128;      // query vectors per CTA (UMMA M)
 constexpr int TA_NT = 64;       // positions per tile
 constexpr int TA_HD = 128;      // head dimension this kernel is built for
@@ -85,6 +85,7 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
     __shared__ __align__(8) uint64_t kv_full[TA_STAGES], kv_empty[TA_STAGES], s_full[2], s_empty[2], p_full, o_full;
     __shared__ uint32_t tmem_base_s;
     __shared__ int giving_up_s, never_s;
+    __shared__ float xch[3][2][TA_QB];  // [tile parity, or 2 for the final sums][column half][query vector]: what the two warps of a row exchange
     volatile int *giving_up = &giving_up_s;
     const AttnArgs &a = args.a;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -128,9 +129,9 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
         }
         for (int b = 0; b < 2; b++) {
             mbar_init(&s_full[b], 1);
-            mbar_init(&s_empty[b], 128);
+            mbar_init(&s_empty[b], 256);
         }
-        mbar_init(&p_full, 128);
+        mbar_init(&p_full, 256);
         mbar_init(&o_full, 1);
         giving_up_s = 0;
         never_s = 0;
@@ -144,12 +145,13 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
 
     // ---- the queries, as two bf16 planes in the swizzled K-major layout (thread = query vector)
     if (warp >= 2 && n_tiles > 0) {
-        const int qi = (warp & 3) * 32 + lane;
+        const int qi = (warp & 3) * 32 + lane, half = (warp - 2) >> 2;  // the two warps of a row take 8 chunks each
         const bool have = qi < nq_here;
         const int qg = q0 + qi, r = qg / G, j = qg % G;
         const float *src = a.q32 + (size_t)(row0 + (have ? r : 0)) * a.Hq * TA_HD + (hk * G + (have ? j : 0)) * TA_HD;
 #pragma unroll
-        for (int c = 0; c < TA_HD / 8; c++) {
+        for (int cc = 0; cc < TA_HD / 16; cc++) {
+            const int c = half * (TA_HD / 16) + cc;
             uint4 hi = make_uint4(0, 0, 0, 0), lo = hi;
             if (have) {
                 const float4 x0 = *reinterpret_cast<const float4 *>(src + c * 8);
@@ -236,21 +238,27 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
         }
     } else {
         // ------------------------------------------------------------ softmax and output (thread = query vector)
-        const int quad = warp & 3, qi = quad * 32 + lane;
+        // Two warps per TMEM lane quadrant: both own the same 32 query vectors (thread = query
+        // vector), warp `half` takes score columns [32 half, 32 half + 32) and output columns
+        // [64 half, 64 half + 64); they exchange their tile maxima (and at the end their sums)
+        // through shared memory behind a 64-thread named barrier.
+        const int quad = warp & 3, half = (warp - 2) >> 2, qi = quad * 32 + lane;
         const bool have = qi < nq_here;
         const int limit = have ? pos0 + (q0 + qi) / G : -1;
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
         const float scale = rsqrtf((float)TA_HD);
-        float m_run = -INFINITY, l_run = 0.f;
+        float m_run = -INFINITY, l_run = 0.f;  // l_run: this warp's columns only
         bool ok = true;
-        // The choice below is per WARP: tcgen05.ld/st are warp-wide (.sync.aligned) instructions, so
-        // a warp either runs the whole softmax path with all its lanes (lanes without a query
+        auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(8 + quad) : "memory"); };
+        // The choice below is per quadrant: tcgen05.ld/st are warp-wide (.sync.aligned) instructions,
+        // so a warp either runs the whole softmax path with all its lanes (lanes without a query
         // vector see everything masked) or none of it.
         const bool warp_idle = quad * 32 >= nq_here;
         if (warp_idle && n_tiles > 0) {
-            // a warp without query vectors: its rows of the weight planes stay zero, and it only
-            // keeps the barriers' arrival counts whole
-            for (int c = 0; c < 8; c++) {
+            // warps without query vectors: their rows of the weight planes stay zero, and they only
+            // keep the barriers' arrival counts whole
+            for (int cc = 0; cc < 4; cc++) {
+                const int c = half * 4 + cc;
                 *reinterpret_cast<uint4 *>(base_p + TA_Q_BYTES + (uint32_t)qi * 128 + (c << 4)) = make_uint4(0, 0, 0, 0);
                 *reinterpret_cast<uint4 *>(base_p + TA_Q_BYTES + TA_P_BYTES / 2 + (uint32_t)qi * 128 + (c << 4)) = make_uint4(0, 0, 0, 0);
             }
@@ -263,32 +271,36 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
             }
         } else if (n_tiles > 0) {
             // The output row accumulates in TMEM over all tiles (the MMAs add into it), relative to
-            // the running maximum m_run; when a tile raises a row's maximum the warp rescales its
-            // rows of the accumulator in place before the tile's product is issued.
-            for (int t = 0; t < n_tiles && ok; t++) {
+            // the running maximum m_run; when a tile raises a row's maximum the warps rescale their
+            // columns of the accumulator in place before the tile's product is issued.
+            const float c2 = scale * 1.4426950408889634f;  // scores in units of log2(e)
+            const int min_limit = __reduce_min_sync(0xffffffffu, have ? limit : 0x7fffffff);
+            const bool all_have = __all_sync(0xffffffffu, have);
+            for (int t = 0; t < n_tiles; t++) {
                 const int b = t & 1;
-                ok = mbar_wait(&s_full[b], (t >> 1) & 1, giving_up, args.status);
-                if (!(ok = __all_sync(0xffffffffu, ok))) break;  // the loads below are warp-wide
-                tc_fence_after();
-                const uint32_t ts = t_s0 + lane_addr + (uint32_t)b * TA_NT;
-                const int p0 = s_beg + t * TA_NT;
-                uint32_t sr[4][16];
+                ok = ok && mbar_wait(&s_full[b], (t >> 1) & 1, giving_up, args.status);
+                ok = __all_sync(0xffffffffu, ok);  // the loads below are warp-wide
+                const uint32_t ts = t_s0 + lane_addr + (uint32_t)b * TA_NT + (uint32_t)half * 32;
+                const int p0 = s_beg + t * TA_NT + half * 32;
+                uint32_t sr[2][16];
+                if (ok) {
+                    tc_fence_after();
+                    tmem_ld16_nowait(ts, sr[0]);
+                    tmem_ld16_nowait(ts + 16, sr[1]);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    tc_fence_before();
+                    mbar_arrive(&s_empty[b]);  // the scores are in registers
+                } else {
 #pragma unroll
-                for (int c = 0; c < 4; c++) tmem_ld16_nowait(ts + c * 16, sr[c]);
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                tc_fence_before();
-                mbar_arrive(&s_empty[b]);  // the scores are in registers
-                // scores in units of log2(e): one multiply-add and one ex2 per weight.  A tile that
-                // lies wholly inside what every row of the warp may see (the common case: only a
-                // split's last tiles touch the causal edge or the split's end) needs no masking.
-                const float c2 = scale * 1.4426950408889634f;
-                const int min_limit = __reduce_min_sync(0xffffffffu, have ? limit : 0x7fffffff);
-                const bool full_tile = p0 + TA_NT <= s_end && p0 + TA_NT - 1 <= min_limit &&
-                                       __all_sync(0xffffffffu, have);
+                    for (int i = 0; i < 16; i++) sr[0][i] = sr[1][i] = 0xff800000u;  // -inf: keep going to the barriers below
+                }
+                // A tile that lies wholly inside what every row of the warp may see (the common case:
+                // only a split's last tiles touch the causal edge or the split's end) needs no masking.
+                const bool full_tile = p0 + 32 <= s_end && p0 + 31 <= min_limit && all_have;
                 float tmax = -INFINITY;
                 if (full_tile) {
 #pragma unroll
-                    for (int c = 0; c < 4; c++)
+                    for (int c = 0; c < 2; c++)
 #pragma unroll
                         for (int i = 0; i < 16; i++) {
                             const float x = __uint_as_float(sr[c][i]) * c2;
@@ -297,7 +309,7 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
                         }
                 } else {
 #pragma unroll
-                    for (int c = 0; c < 4; c++)
+                    for (int c = 0; c < 2; c++)
 #pragma unroll
                         for (int i = 0; i < 16; i++) {
                             const int p = p0 + c * 16 + i;
@@ -306,6 +318,15 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
                             tmax = fmaxf(tmax, x);
                         }
                 }
+                // the row's maximum over both halves (both warps always reach this barrier, also when giving up)
+                xch[b][half][qi] = tmax;
+                pair_sync();
+                tmax = fmaxf(tmax, xch[b][half ^ 1][qi]);
+                ok = ok && *giving_up == 0;
+                if (!(ok = __all_sync(0xffffffffu, ok))) {
+                    // leave together: the partner warp reads the same flag after the same barrier
+                    break;
+                }
                 // The reference maximum is allowed to lag the true one by TA_RAISE (weights then reach
                 // 2^11, which two bf16 terms and fp32 sums carry without loss): otherwise some lane of
                 // the warp would see a new maximum in most tiles and the accumulator would be
@@ -313,11 +334,11 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
                 const bool raise = tmax > m_run + TA_RAISE;
                 const float m_new = raise ? tmax : m_run;
                 const float factor = raise ? exp2f(m_run - m_new) : 1.f;  // 2^(-inf) = 0 on the first live tile
-                const float m_ref = m_new == -INFINITY ? 0.f : m_new;  // a row that has seen nothing yet: all weights 0
+                const float m_ref = m_new == -INFINITY ? 0.f : m_new;    // a row that has seen nothing yet: all weights 0
                 float psum = 0.f;
-                uint4 whi[8], wlo[8];
+                uint4 whi[4], wlo[4];
 #pragma unroll
-                for (int c = 0; c < 8; c++) {
+                for (int c = 0; c < 4; c++) {
                     float w[8];
 #pragma unroll
                     for (int i = 0; i < 8; i++) {
@@ -326,77 +347,87 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
                     }
                     split8(w, whi[c], wlo[c]);
                 }
-                // the previous product has read the weight planes and is in the accumulator
+                // the previous product has read the weight planes and is in the accumulator.  A wait
+                // that fails here does not leave the loop on its own: the two warps of a row only
+                // leave together, after the next named barrier (which has no time limit).
                 if (t > 0) {
                     ok = mbar_wait(&o_full, (t - 1) & 1, giving_up, args.status);
-                    if (!(ok = __all_sync(0xffffffffu, ok))) break;
+                    ok = __all_sync(0xffffffffu, ok);
+                }
+                if (ok) {
                     tc_fence_after();
-                    if (__any_sync(0xffffffffu, raise)) {
+                    if (t > 0 && __any_sync(0xffffffffu, raise)) {
+                        const uint32_t to = t_o + lane_addr + (uint32_t)half * 64;
 #pragma unroll
-                        for (int c0 = 0; c0 < TA_HD; c0 += 32) {
+                        for (int c0 = 0; c0 < 64; c0 += 32) {
                             uint32_t r0[16], r1[16];
-                            tmem_ld16_nowait(t_o + lane_addr + c0, r0);
-                            tmem_ld16_nowait(t_o + lane_addr + c0 + 16, r1);
+                            tmem_ld16_nowait(to + c0, r0);
+                            tmem_ld16_nowait(to + c0 + 16, r1);
                             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
                             for (int i = 0; i < 16; i++) {
                                 r0[i] = __float_as_uint(__uint_as_float(r0[i]) * factor);
                                 r1[i] = __float_as_uint(__uint_as_float(r1[i]) * factor);
                             }
-                            tmem_st16(t_o + lane_addr + c0, r0);
-                            tmem_st16(t_o + lane_addr + c0 + 16, r1);
+                            tmem_st16(to + c0, r0);
+                            tmem_st16(to + c0 + 16, r1);
                         }
                         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                     }
-                }
 #pragma unroll
-                for (int c = 0; c < 8; c++) {
-                    const uint32_t off = (uint32_t)qi * 128 + (uint32_t)((c ^ (qi & 7)) << 4);
-                    *reinterpret_cast<uint4 *>(base_p + TA_Q_BYTES + off) = whi[c];
-                    *reinterpret_cast<uint4 *>(base_p + TA_Q_BYTES + TA_P_BYTES / 2 + off) = wlo[c];
+                    for (int cc = 0; cc < 4; cc++) {
+                        const int c = half * 4 + cc;
+                        const uint32_t off = (uint32_t)qi * 128 + (uint32_t)((c ^ (qi & 7)) << 4);
+                        *reinterpret_cast<uint4 *>(base_p + TA_Q_BYTES + off) = whi[cc];
+                        *reinterpret_cast<uint4 *>(base_p + TA_Q_BYTES + TA_P_BYTES / 2 + off) = wlo[cc];
+                    }
+                    tc_fence_before();
+                    asm volatile("fence.proxy.async;" ::: "memory");
+                    mbar_arrive(&p_full);
                 }
-                tc_fence_before();
-                asm volatile("fence.proxy.async;" ::: "memory");
-                mbar_arrive(&p_full);
                 l_run = l_run * factor + psum;
                 m_run = m_new;
             }
         }
-        float o[TA_HD];
+        float o[64];
         if (!warp_idle && n_tiles > 0 && ok) {
             ok = mbar_wait(&o_full, (n_tiles - 1) & 1, giving_up, args.status);
             ok = __all_sync(0xffffffffu, ok);
             if (ok) {
                 tc_fence_after();
+                uint32_t r[4][16];
 #pragma unroll
-                for (int c0 = 0; c0 < TA_HD; c0 += 64) {
-                    uint32_t r[4][16];
+                for (int c = 0; c < 4; c++) tmem_ld16_nowait(t_o + lane_addr + (uint32_t)half * 64 + c * 16, r[c]);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-                    for (int c = 0; c < 4; c++) tmem_ld16_nowait(t_o + lane_addr + c0 + c * 16, r[c]);
-                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                for (int c = 0; c < 4; c++)
 #pragma unroll
-                    for (int c = 0; c < 4; c++)
-#pragma unroll
-                        for (int i = 0; i < 16; i++) o[c0 + c * 16 + i] = __uint_as_float(r[c][i]);
-                }
+                    for (int i = 0; i < 16; i++) o[c * 16 + i] = __uint_as_float(r[c][i]);
                 tc_fence_before();
             }
         } else {
 #pragma unroll
-            for (int i = 0; i < TA_HD; i++) o[i] = 0.f;
+            for (int i = 0; i < 64; i++) o[i] = 0.f;
+        }
+        // the row's sum over both halves (quadrants that ran the softmax path: both warps get here)
+        if (!warp_idle && n_tiles > 0) {
+            xch[2][half][qi] = l_run;
+            pair_sync();
+            l_run += xch[2][half ^ 1][qi];
         }
         if (have && ok) {
             const int qg = q0 + qi, r = qg / G, j = qg % G;
             const size_t cell0 = ((size_t)(row0 + r) * a.Hq + hk * G + j) * a.n_splits;
             const int first = sp * args.split_mult;
             if (first < a.n_splits) {
-                float *dst = a.part_o + (cell0 + first) * TA_HD;
+                float *dst = a.part_o + (cell0 + first) * TA_HD + half * 64;
 #pragma unroll
-                for (int i = 0; i < TA_HD; i += 4) *reinterpret_cast<float4 *>(dst + i) = make_float4(o[i], o[i + 1], o[i + 2], o[i + 3]);
-                a.part_ml[cell0 + first] = make_float2(m_run * 0.6931471805599453f, l_run);  // back to natural-log units
+                for (int i = 0; i < 64; i += 4) *reinterpret_cast<float4 *>(dst + i) = make_float4(o[i], o[i + 1], o[i + 2], o[i + 3]);
+                if (half == 0) a.part_ml[cell0 + first] = make_float2(m_run * 0.6931471805599453f, l_run);  // back to natural-log units
             }
-            for (int e = first + 1; e < min(first + args.split_mult, a.n_splits); e++)
-                a.part_ml[cell0 + e] = make_float2(-INFINITY, 0.f);
+            if (half == 0)
+                for (int e = first + 1; e < min(first + args.split_mult, a.n_splits); e++)
+                    a.part_ml[cell0 + e] = make_float2(-INFINITY, 0.f);
         }
     }
     // ---------------------------------------------------------------- teardown
