@@ -16,8 +16,10 @@
 //               running maximum
 //
 // CTA = (group, block of 128 query vectors, kv head, KV split); warp 0 issues the TMA copies of a
-// three-stage K/V ring, warp 1 issues the MMAs and owns the TMEM allocation, warps 2..9 do the
-// softmax (thread = query vector = TMEM lane, two warps per lane quadrant with half the columns each).  S is double buffered so that
+// K ring (three tiles) and a V ring (two), warp 1 issues the MMAs and owns the TMEM allocation, warps 2..9 do the
+// softmax (thread = query vector = TMEM lane, two warps per lane quadrant with half the columns each).
+// S and the weight planes are double buffered: a tile's scores and weights are formed while the
+// product of the tile before it is still running.  S is double buffered so that
 // the next tile's scores are computed while this tile's weights are being formed.  The partials
 // (unnormalised output, running max, running sum per split) have the layout of the other
 // attention kernel, and attn_merge_kernel merges them.  Every wait is bounded.
@@ -32,12 +34,13 @@ constexpr int TA_THREADS = 320;   // TMA warp, MMA warp, eight softmax warps
 constexpr int TA_QB = 128;      // query vectors per CTA (UMMA M)
 constexpr int TA_NT = 64;       // positions per tile
 constexpr int TA_HD = 128;      // head dimension this kernel is built for
-constexpr int TA_STAGES = 3;
+constexpr int TA_KST = 3;        // K tiles in flight: tile t + 3 is requested when the scores of tile t are done
+constexpr int TA_VST = 2;        // V tiles in flight: tile t + 2 is requested when the product of tile t is done
 constexpr float TA_RAISE = 11.f;  // a row's reference maximum (in units of log2 e) moves only when a tile exceeds it by this much
 constexpr int TA_Q_BYTES = 2 * TA_QB * TA_HD * 2;    // hi and lo planes: 64 KB
-constexpr int TA_P_BYTES = 2 * TA_QB * TA_NT * 2;    // hi and lo planes: 32 KB
-constexpr int TA_KV_BYTES = 2 * TA_NT * TA_HD * 2;   // K and V tile of a stage: 32 KB
-constexpr int TA_SMEM = 1024 + TA_Q_BYTES + TA_P_BYTES + TA_STAGES * TA_KV_BYTES;
+constexpr int TA_P_BYTES = 2 * TA_QB * TA_NT * 2;    // hi and lo planes of one tile's weights: 32 KB (two buffers)
+constexpr int TA_T_BYTES = TA_NT * TA_HD * 2;        // one K or V tile: 16 KB
+constexpr int TA_SMEM = 1024 + TA_Q_BYTES + 2 * TA_P_BYTES + (TA_KST + TA_VST) * TA_T_BYTES;
 
 struct AttnTcArgs {
     AttnArgs a;        // q32, row and group arrays, partial buffers, shapes, the split plan
@@ -82,7 +85,8 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
     attn_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const AttnTcArgs args)
 {
     extern __shared__ __align__(1024) unsigned char ta_smem[];
-    __shared__ __align__(8) uint64_t kv_full[TA_STAGES], kv_empty[TA_STAGES], s_full[2], s_empty[2], p_full, o_full;
+    __shared__ __align__(8) uint64_t k_full[TA_KST], k_empty[TA_KST], v_full[TA_VST], v_empty[TA_VST], s_full[2], s_empty[2],
+        p_full[2], o_full[2];
     __shared__ uint32_t tmem_base_s;
     __shared__ int giving_up_s, never_s;
     __shared__ float xch[3][2][TA_QB];  // [tile parity, or 2 for the final sums][column half][query vector]: what the two warps of a row exchange
@@ -92,8 +96,8 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
     const uint32_t base = (smem_u32(ta_smem) + 1023u) & ~1023u;
     unsigned char *base_p = ta_smem + (base - smem_u32(ta_smem));
     const uint32_t q_hi = base, q_lo = base + TA_Q_BYTES / 2;
-    const uint32_t p_hi = base + TA_Q_BYTES, p_lo = p_hi + TA_P_BYTES / 2;
-    const uint32_t kv0 = base + TA_Q_BYTES + TA_P_BYTES;
+    const uint32_t p0_hi = base + TA_Q_BYTES;  // buffer b: hi plane at p0_hi + b * TA_P_BYTES, lo plane TA_P_BYTES / 2 on
+    const uint32_t k0 = base + TA_Q_BYTES + 2 * TA_P_BYTES, v0 = k0 + TA_KST * TA_T_BYTES;
 
     // ---- what this CTA works on (every thread computes the same); a CTA whose group belongs to
     // the other kernel, or does not exist, leaves before it sets anything up
@@ -123,16 +127,20 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
     const int cache_row0 = ((sane ? slot : 0) * a.Hkv + hk) * a.S;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < TA_STAGES; s++) {
-            mbar_init(&kv_full[s], 1);
-            mbar_init(&kv_empty[s], 1);
+        for (int s = 0; s < TA_KST; s++) {
+            mbar_init(&k_full[s], 1);
+            mbar_init(&k_empty[s], 1);
+        }
+        for (int s = 0; s < TA_VST; s++) {
+            mbar_init(&v_full[s], 1);
+            mbar_init(&v_empty[s], 1);
         }
         for (int b = 0; b < 2; b++) {
             mbar_init(&s_full[b], 1);
             mbar_init(&s_empty[b], 256);
+            mbar_init(&p_full[b], 256);
+            mbar_init(&o_full[b], 1);
         }
-        mbar_init(&p_full, 256);
-        mbar_init(&o_full, 1);
         giving_up_s = 0;
         never_s = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -163,7 +171,7 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
             *reinterpret_cast<uint4 *>(base_p + off) = hi;
             *reinterpret_cast<uint4 *>(base_p + TA_Q_BYTES / 2 + off) = lo;
         }
-        asm volatile("fence.proxy.async;" ::: "memory");  // the MMAs read these through the async proxy
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the MMAs read these through the async proxy
     }
     tc_fence_before();
     __syncthreads();
@@ -174,66 +182,72 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
     if (warp == 0) {
         // ------------------------------------------------------------ producer
         // One thread needs a few hundred nanoseconds per TMA copy, so a tile is two copies (the
-        // [64][rows][2] view of the cache brings both 64-column halves of K, or of V, at once)
-        // issued by two lanes side by side.
-        uint32_t issued = 0;
-        bool ok = true;
-        for (int t = 0; t < n_tiles && ok; t++) {
-            const int st = t % TA_STAGES;
-            int go = 1;
-            if (lane == 0) {
-                go = mbar_wait(&kv_empty[st], ((t / TA_STAGES) & 1) ^ 1, giving_up, args.status) ? 1 : 0;
-                if (go) mbar_expect_tx(&kv_full[st], TA_KV_BYTES);
+        // [64][rows][2] view of the cache brings both 64-column halves of K, or of V, at once):
+        // lane 0 runs the K ring, lane 1 the V ring, each at its own pace.
+        if (lane < 2) {
+            const bool is_v = lane == 1;
+            const int depth = is_v ? TA_VST : TA_KST;
+            uint64_t *full = is_v ? v_full : k_full, *empty = is_v ? v_empty : k_empty;
+            const uint32_t ring0 = is_v ? v0 : k0;
+            const CUtensorMap *map = is_v ? &map_v : &map_k;
+            uint32_t issued = 0;
+            for (int t = 0; t < n_tiles; t++) {
+                const int st = t % depth;
+                if (!mbar_wait(&empty[st], ((t / depth) & 1) ^ 1, giving_up, args.status)) break;
+                mbar_expect_tx(&full[st], TA_T_BYTES);
+                tma_load_3d(ring0 + (uint32_t)st * TA_T_BYTES, map, &full[st], 0, cache_row0 + s_beg + t * TA_NT, 0);
+                issued++;
             }
-            go = __shfl_sync(0xffffffffu, go, 0);
-            if (!(ok = go != 0)) break;
-            const uint32_t dst = kv0 + (uint32_t)st * TA_KV_BYTES;
-            const int y = cache_row0 + s_beg + t * TA_NT;
-            if (lane == 0) tma_load_3d(dst, &map_k, &kv_full[st], 0, y, 0);
-            if (lane == 1) tma_load_3d(dst + 16384, &map_v, &kv_full[st], 0, y, 0);
-            issued++;
-        }
-        // never leave with copies in flight
-        if (lane == 0)
-            for (int st = 0; st < TA_STAGES; st++)
+            // never leave with copies in flight
+            for (int st = 0; st < depth; st++)
                 if (issued > (uint32_t)st)
-                    mbar_wait(&kv_full[st], ((issued - 1 - st) / TA_STAGES) & 1, &never_s, nullptr, 2000000ull);
+                    mbar_wait(&full[st], ((issued - 1 - st) / depth) & 1, &never_s, nullptr, 2000000ull);
+        }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0 && n_tiles > 0) {
             const uint32_t idesc_s = umma_idesc_bf16_ex(TA_NT, false), idesc_o = umma_idesc_bf16_ex(TA_HD, true);
             bool ok = true;
+            const uint64_t dq_hi = umma_desc_sw128(q_hi), dq_lo = umma_desc_sw128(q_lo);
             auto issue_s = [&](int t) {
-                const int st = t % TA_STAGES, b = t & 1;
-                if (!(ok = mbar_wait(&kv_full[st], (t / TA_STAGES) & 1, giving_up, args.status))) return;
+                const int st = t % TA_KST, b = t & 1;
+                if (!(ok = mbar_wait(&k_full[st], (t / TA_KST) & 1, giving_up, args.status))) return;
                 if (!(ok = mbar_wait(&s_empty[b], ((t >> 1) & 1) ^ 1, giving_up, args.status))) return;
                 tc_fence_after();
-                const uint32_t kt = kv0 + (uint32_t)st * TA_KV_BYTES, d = t_s0 + (uint32_t)b * TA_NT;
+                // one thread issues every MMA, so the descriptors are built once and only advanced:
+                // the address field (16-byte units, low 14 bits) takes the constant offsets by addition
+                const uint64_t dk0 = umma_desc_sw128(k0 + (uint32_t)st * TA_T_BYTES);
+                const uint32_t d = t_s0 + (uint32_t)b * TA_NT;
 #pragma unroll
                 for (int kk = 0; kk < TA_HD / 16; kk++) {
-                    const uint32_t qoff = (uint32_t)(kk >> 2) * (TA_QB * 128) + (uint32_t)(kk & 3) * 32;
-                    const uint64_t db = umma_desc_sw128(kt + (uint32_t)(kk >> 2) * 8192 + (uint32_t)(kk & 3) * 32);
-                    umma_bf16(d, umma_desc_sw128(q_hi + qoff), db, idesc_s, kk > 0);
-                    umma_bf16(d, umma_desc_sw128(q_lo + qoff), db, idesc_s, 1);
+                    const uint64_t qadv = (uint64_t)(((kk >> 2) * (TA_QB * 128) + (kk & 3) * 32) >> 4);
+                    const uint64_t db = dk0 + (uint64_t)(((kk >> 2) * 8192 + (kk & 3) * 32) >> 4);
+                    umma_bf16(d, dq_hi + qadv, db, idesc_s, kk > 0);
+                    umma_bf16(d, dq_lo + qadv, db, idesc_s, 1);
                 }
+                umma_commit(&k_empty[st]);  // the K tile is free once the scores are computed
                 umma_commit(&s_full[b]);
             };
+            // order of issue: S(0), S(1), P.V(0), S(2), P.V(1), ...: a tile's scores never wait for
+            // the weights of the tile before it
             issue_s(0);
             for (int t = 0; t < n_tiles && ok; t++) {
                 if (t + 1 < n_tiles) issue_s(t + 1);
                 if (!ok) break;
-                const int st = t % TA_STAGES;
-                if (!(ok = mbar_wait(&p_full, t & 1, giving_up, args.status))) break;
+                const int st = t % TA_VST, b = t & 1;
+                if (!(ok = mbar_wait(&v_full[st], (t / TA_VST) & 1, giving_up, args.status))) break;
+                if (!(ok = mbar_wait(&p_full[b], (t >> 1) & 1, giving_up, args.status))) break;
                 tc_fence_after();
-                const uint32_t vt = kv0 + (uint32_t)st * TA_KV_BYTES + 16384;
+                const uint64_t dv0 = umma_desc_sw128_mn(v0 + (uint32_t)st * TA_T_BYTES, 8192);
+                const uint64_t dp_hi = umma_desc_sw128(p0_hi + (uint32_t)b * TA_P_BYTES), dp_lo = dp_hi + (uint64_t)((TA_P_BYTES / 2) >> 4);
 #pragma unroll
                 for (int kk = 0; kk < TA_NT / 16; kk++) {
-                    const uint64_t dv = umma_desc_sw128_mn(vt + (uint32_t)kk * 2048, 8192);
-                    umma_bf16(t_o, umma_desc_sw128(p_hi + (uint32_t)kk * 32), dv, idesc_o, t > 0 || kk > 0);
-                    umma_bf16(t_o, umma_desc_sw128(p_lo + (uint32_t)kk * 32), dv, idesc_o, 1);
+                    const uint64_t dv = dv0 + (uint64_t)((kk * 2048) >> 4);
+                    umma_bf16(t_o, dp_hi + (uint64_t)((kk * 32) >> 4), dv, idesc_o, t > 0 || kk > 0);
+                    umma_bf16(t_o, dp_lo + (uint64_t)((kk * 32) >> 4), dv, idesc_o, 1);
                 }
-                umma_commit(&kv_empty[st]);  // the stage and the weights are free once these have read them
-                umma_commit(&o_full);
+                umma_commit(&v_empty[st]);  // the V tile and this buffer of weights are free once these have read them
+                umma_commit(&o_full[b]);
             }
         }
     } else {
@@ -257,17 +271,17 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
         if (warp_idle && n_tiles > 0) {
             // warps without query vectors: their rows of the weight planes stay zero, and they only
             // keep the barriers' arrival counts whole
-            for (int cc = 0; cc < 4; cc++) {
-                const int c = half * 4 + cc;
-                *reinterpret_cast<uint4 *>(base_p + TA_Q_BYTES + (uint32_t)qi * 128 + (c << 4)) = make_uint4(0, 0, 0, 0);
-                *reinterpret_cast<uint4 *>(base_p + TA_Q_BYTES + TA_P_BYTES / 2 + (uint32_t)qi * 128 + (c << 4)) = make_uint4(0, 0, 0, 0);
+            for (int cc = 0; cc < 16; cc++) {  // both buffers, both planes, this warp's four chunks of the row
+                const int c = half * 4 + (cc & 3);
+                *reinterpret_cast<uint4 *>(base_p + TA_Q_BYTES + (cc >> 2) * (TA_P_BYTES / 2) + (uint32_t)qi * 128 + (c << 4)) =
+                    make_uint4(0, 0, 0, 0);
             }
-            asm volatile("fence.proxy.async;" ::: "memory");
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             for (int t = 0; t < n_tiles && ok; t++) {
                 if (!(ok = mbar_wait(&s_full[t & 1], (t >> 1) & 1, giving_up, args.status))) break;
-                if (t > 0 && !(ok = mbar_wait(&o_full, (t - 1) & 1, giving_up, args.status))) break;
+                if (t >= 2 && !(ok = mbar_wait(&o_full[t & 1], ((t >> 1) - 1) & 1, giving_up, args.status))) break;
                 mbar_arrive(&s_empty[t & 1]);
-                mbar_arrive(&p_full);
+                mbar_arrive(&p_full[t & 1]);
             }
         } else if (n_tiles > 0) {
             // The output row accumulates in TMEM over all tiles (the MMAs add into it), relative to
@@ -347,16 +361,19 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
                     }
                     split8(w, whi[c], wlo[c]);
                 }
-                // the previous product has read the weight planes and is in the accumulator.  A wait
-                // that fails here does not leave the loop on its own: the two warps of a row only
+                // The weights go to buffer b, which the product of tile t - 2 has read by the time
+                // o_full[b] completes; a rescaling needs every product so far in the accumulator.  A
+                // wait that fails here does not leave the loop on its own: the two warps of a row only
                 // leave together, after the next named barrier (which has no time limit).
-                if (t > 0) {
-                    ok = mbar_wait(&o_full, (t - 1) & 1, giving_up, args.status);
+                if (t >= 2) {
+                    ok = mbar_wait(&o_full[b], ((t >> 1) - 1) & 1, giving_up, args.status);
                     ok = __all_sync(0xffffffffu, ok);
                 }
-                if (ok) {
-                    tc_fence_after();
-                    if (t > 0 && __any_sync(0xffffffffu, raise)) {
+                if (ok && t > 0 && __any_sync(0xffffffffu, raise)) {
+                    ok = mbar_wait(&o_full[(t - 1) & 1], ((t - 1) >> 1) & 1, giving_up, args.status);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (ok) {
+                        tc_fence_after();
                         const uint32_t to = t_o + lane_addr + (uint32_t)half * 64;
 #pragma unroll
                         for (int c0 = 0; c0 < 64; c0 += 32) {
@@ -374,16 +391,18 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
                         }
                         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                     }
+                }
+                if (ok) {
 #pragma unroll
                     for (int cc = 0; cc < 4; cc++) {
                         const int c = half * 4 + cc;
-                        const uint32_t off = (uint32_t)qi * 128 + (uint32_t)((c ^ (qi & 7)) << 4);
+                        const uint32_t off = (uint32_t)b * TA_P_BYTES + (uint32_t)qi * 128 + (uint32_t)((c ^ (qi & 7)) << 4);
                         *reinterpret_cast<uint4 *>(base_p + TA_Q_BYTES + off) = whi[cc];
                         *reinterpret_cast<uint4 *>(base_p + TA_Q_BYTES + TA_P_BYTES / 2 + off) = wlo[cc];
                     }
                     tc_fence_before();
-                    asm volatile("fence.proxy.async;" ::: "memory");
-                    mbar_arrive(&p_full);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    mbar_arrive(&p_full[b]);
                 }
                 l_run = l_run * factor + psum;
                 m_run = m_new;
@@ -391,7 +410,7 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
         }
         float o[64];
         if (!warp_idle && n_tiles > 0 && ok) {
-            ok = mbar_wait(&o_full, (n_tiles - 1) & 1, giving_up, args.status);
+            ok = mbar_wait(&o_full[(n_tiles - 1) & 1], ((n_tiles - 1) >> 1) & 1, giving_up, args.status);
             ok = __all_sync(0xffffffffu, ok);
             if (ok) {
                 tc_fence_after();
