@@ -6,14 +6,18 @@
 // flop per cache byte: beyond what mma.sync delivers, so the block kernel of sparsk_attn.cuh is
 // tensor-bound there.  This kernel runs the same arithmetic on tcgen05:
 //
-//   S = Q K^T : A = the block's query vectors (up to 128 rows, hi and lo planes, K-major, written
-//               once into swizzled shared memory), B = a [64 positions x 128] K tile exactly as
-//               TMA delivers it from the cache (K-major), accumulator [128 x 64] fp32 in TMEM
-//   O_t = P V : A = the tile's softmax weights (hi and lo planes, written by the softmax warps
-//               into swizzled shared memory), B = the V tile as delivered (positions x head dim =
-//               MN-major), accumulated over all tiles in a [128 x 128] fp32 TMEM accumulator that
-//               the softmax warps rescale in place (tcgen05.ld / st) when a tile raises a row's
-//               running maximum
+//   S = Q K^T : A = the block's query vectors (up to 128 rows, hi and lo bf16 planes) held in TMEM,
+//               stored there once with tcgen05.st (lane = query vector, elements packed two per
+//               column); B = a [64 positions x 128] K tile exactly as TMA delivers it from the
+//               cache (K-major); accumulator [128 x 64] fp32 in TMEM
+//   O += P V  : A = the tile's softmax weights (hi and lo planes), written by the softmax warps
+//               straight into TMEM; B = the V tile as delivered (positions x head dim = MN-major);
+//               accumulated over all tiles in a [128 x 128] fp32 TMEM accumulator that the softmax
+//               warps rescale in place (tcgen05.ld / st) when a tile raises a row's reference maximum
+// With both A operands in TMEM an MMA reads only its K or V slice from shared memory (2 or 4 KB
+// instead of 6 or 8): with the operands in shared memory the MMAs ran at 80 and 120 cycles each
+// against 32 and 64 at the tensor rate.  All 512 TMEM columns are used: scores 2 x 64, output
+// 128, weights 2 x 64, queries 128.
 //
 // CTA = (group, block of 128 query vectors, kv head, KV split); warp 0 issues the TMA copies of a
 // K ring (three tiles) and a V ring (two), warp 1 issues the MMAs and owns the TMEM allocation, warps 2..9 do the
@@ -34,13 +38,13 @@ constexpr int TA_THREADS = 320;   // TMA warp, MMA warp, eight softmax warps
 constexpr int TA_QB = 128;      // query vectors per CTA (UMMA M)
 constexpr int TA_NT = 64;       // positions per tile
 constexpr int TA_HD = 128;      // head dimension this kernel is built for
-constexpr int TA_KST = 3;        // K tiles in flight: tile t + 3 is requested when the scores of tile t are done
-constexpr int TA_VST = 2;        // V tiles in flight: tile t + 2 is requested when the product of tile t is done
+constexpr int TA_KST = 4;        // K tiles in flight: tile t + 4 is requested when the scores of tile t are done
+constexpr int TA_VST = 3;        // V tiles in flight: tile t + 3 is requested when the product of tile t is done
 constexpr float TA_RAISE = 11.f;  // a row's reference maximum (in units of log2 e) moves only when a tile exceeds it by this much
-constexpr int TA_Q_BYTES = 2 * TA_QB * TA_HD * 2;    // hi and lo planes: 64 KB
-constexpr int TA_P_BYTES = 2 * TA_QB * TA_NT * 2;    // hi and lo planes of one tile's weights: 32 KB (two buffers)
 constexpr int TA_T_BYTES = TA_NT * TA_HD * 2;        // one K or V tile: 16 KB
-constexpr int TA_SMEM = 1024 + TA_Q_BYTES + 2 * TA_P_BYTES + (TA_KST + TA_VST) * TA_T_BYTES;
+constexpr int TA_SMEM = 1024 + (TA_KST + TA_VST) * TA_T_BYTES;
+// TMEM columns (all 512): scores 2 x 64, output 128, weights 2 x (hi 32 + lo 32), queries hi 64 + lo 64
+constexpr int TA_C_S = 0, TA_C_O = 128, TA_C_P = 256, TA_C_Q = 384;
 
 struct AttnTcArgs {
     AttnArgs a;        // q32, row and group arrays, partial buffers, shapes, the split plan
@@ -72,6 +76,16 @@ __device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, uint32_t (&r)[1
         : "memory");
 }
 
+// D (+)= A B with the A operand in TMEM (lane = row, 16-bit elements packed two per column) and B in shared memory.
+__device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc, int accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16])
 {
     asm volatile(
@@ -94,10 +108,7 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
     const AttnArgs &a = args.a;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t base = (smem_u32(ta_smem) + 1023u) & ~1023u;
-    unsigned char *base_p = ta_smem + (base - smem_u32(ta_smem));
-    const uint32_t q_hi = base, q_lo = base + TA_Q_BYTES / 2;
-    const uint32_t p0_hi = base + TA_Q_BYTES;  // buffer b: hi plane at p0_hi + b * TA_P_BYTES, lo plane TA_P_BYTES / 2 on
-    const uint32_t k0 = base + TA_Q_BYTES + 2 * TA_P_BYTES, v0 = k0 + TA_KST * TA_T_BYTES;
+    const uint32_t k0 = base, v0 = k0 + TA_KST * TA_T_BYTES;
 
     // ---- what this CTA works on (every thread computes the same); a CTA whose group belongs to
     // the other kernel, or does not exist, leaves before it sets anything up
@@ -146,38 +157,49 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(256)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
 
-    // ---- the queries, as two bf16 planes in the swizzled K-major layout (thread = query vector)
+    tc_fence_before();
+    __syncthreads();  // the TMEM base address is known
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+    const uint32_t t_s0 = tmem_base + TA_C_S, t_o = tmem_base + TA_C_O, t_p = tmem_base + TA_C_P, t_q = tmem_base + TA_C_Q;
+
+    // ---- the queries, as two bf16 planes in TMEM (thread = query vector = lane; 16-bit elements
+    // packed two per column): the A operand of every score MMA, stored once.  The two warps of a
+    // lane quadrant take 64 of the 128 head dimensions each.
     if (warp >= 2 && n_tiles > 0) {
-        const int qi = (warp & 3) * 32 + lane, half = (warp - 2) >> 2;  // the two warps of a row take 8 chunks each
+        const int qi = (warp & 3) * 32 + lane, half = (warp - 2) >> 2;
         const bool have = qi < nq_here;
         const int qg = q0 + qi, r = qg / G, j = qg % G;
-        const float *src = a.q32 + (size_t)(row0 + (have ? r : 0)) * a.Hq * TA_HD + (hk * G + (have ? j : 0)) * TA_HD;
+        const float *src = a.q32 + (size_t)(row0 + (have ? r : 0)) * a.Hq * TA_HD + (hk * G + (have ? j : 0)) * TA_HD + half * 64;
+        const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
 #pragma unroll
-        for (int cc = 0; cc < TA_HD / 16; cc++) {
-            const int c = half * (TA_HD / 16) + cc;
-            uint4 hi = make_uint4(0, 0, 0, 0), lo = hi;
-            if (have) {
-                const float4 x0 = *reinterpret_cast<const float4 *>(src + c * 8);
-                const float4 x1 = *reinterpret_cast<const float4 *>(src + c * 8 + 4);
-                const float v[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-                split8(v, hi, lo);
+        for (int blk = 0; blk < 2; blk++) {  // 32 elements = 16 packed columns per store
+            uint32_t hi[16], lo[16];
+#pragma unroll
+            for (int c = 0; c < 4; c++) {
+                uint4 h4 = make_uint4(0, 0, 0, 0), l4 = h4;
+                if (have) {
+                    const float4 x0 = *reinterpret_cast<const float4 *>(src + blk * 32 + c * 8);
+                    const float4 x1 = *reinterpret_cast<const float4 *>(src + blk * 32 + c * 8 + 4);
+                    const float v[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+                    split8(v, h4, l4);
+                }
+                hi[c * 4] = h4.x; hi[c * 4 + 1] = h4.y; hi[c * 4 + 2] = h4.z; hi[c * 4 + 3] = h4.w;
+                lo[c * 4] = l4.x; lo[c * 4 + 1] = l4.y; lo[c * 4 + 2] = l4.z; lo[c * 4 + 3] = l4.w;
             }
-            const uint32_t off = (uint32_t)(c >> 3) * (TA_QB * 128) + (uint32_t)qi * 128 + (uint32_t)(((c & 7) ^ (qi & 7)) << 4);
-            *reinterpret_cast<uint4 *>(base_p + off) = hi;
-            *reinterpret_cast<uint4 *>(base_p + TA_Q_BYTES / 2 + off) = lo;
+            tmem_st16(t_q + lane_addr + (uint32_t)(half * 32 + blk * 16), hi);
+            tmem_st16(t_q + lane_addr + 64 + (uint32_t)(half * 32 + blk * 16), lo);
         }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the MMAs read these through the async proxy
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base = tmem_base_s;
-    const uint32_t t_s0 = tmem_base, t_o = tmem_base + 128;
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
@@ -208,7 +230,6 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
         if (lane == 0 && n_tiles > 0) {
             const uint32_t idesc_s = umma_idesc_bf16_ex(TA_NT, false), idesc_o = umma_idesc_bf16_ex(TA_HD, true);
             bool ok = true;
-            const uint64_t dq_hi = umma_desc_sw128(q_hi), dq_lo = umma_desc_sw128(q_lo);
             auto issue_s = [&](int t) {
                 const int st = t % TA_KST, b = t & 1;
                 if (!(ok = mbar_wait(&k_full[st], (t / TA_KST) & 1, giving_up, args.status))) return;
@@ -219,11 +240,10 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
                 const uint64_t dk0 = umma_desc_sw128(k0 + (uint32_t)st * TA_T_BYTES);
                 const uint32_t d = t_s0 + (uint32_t)b * TA_NT;
 #pragma unroll
-                for (int kk = 0; kk < TA_HD / 16; kk++) {
-                    const uint64_t qadv = (uint64_t)(((kk >> 2) * (TA_QB * 128) + (kk & 3) * 32) >> 4);
+                for (int kk = 0; kk < TA_HD / 16; kk++) {  // 16 head dimensions = 8 packed TMEM columns of the queries
                     const uint64_t db = dk0 + (uint64_t)(((kk >> 2) * 8192 + (kk & 3) * 32) >> 4);
-                    umma_bf16(d, dq_hi + qadv, db, idesc_s, kk > 0);
-                    umma_bf16(d, dq_lo + qadv, db, idesc_s, 1);
+                    umma_bf16_ts(d, t_q + (uint32_t)kk * 8, db, idesc_s, kk > 0);
+                    umma_bf16_ts(d, t_q + 64 + (uint32_t)kk * 8, db, idesc_s, 1);
                 }
                 umma_commit(&k_empty[st]);  // the K tile is free once the scores are computed
                 umma_commit(&s_full[b]);
@@ -239,12 +259,12 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
                 if (!(ok = mbar_wait(&p_full[b], (t >> 1) & 1, giving_up, args.status))) break;
                 tc_fence_after();
                 const uint64_t dv0 = umma_desc_sw128_mn(v0 + (uint32_t)st * TA_T_BYTES, 8192);
-                const uint64_t dp_hi = umma_desc_sw128(p0_hi + (uint32_t)b * TA_P_BYTES), dp_lo = dp_hi + (uint64_t)((TA_P_BYTES / 2) >> 4);
+                const uint32_t tp = t_p + (uint32_t)b * 64;  // this tile's weights: hi plane, lo plane 32 columns on
 #pragma unroll
-                for (int kk = 0; kk < TA_NT / 16; kk++) {
+                for (int kk = 0; kk < TA_NT / 16; kk++) {  // 16 positions = 8 packed columns
                     const uint64_t dv = dv0 + (uint64_t)((kk * 2048) >> 4);
-                    umma_bf16(t_o, dp_hi + (uint64_t)((kk * 32) >> 4), dv, idesc_o, t > 0 || kk > 0);
-                    umma_bf16(t_o, dp_lo + (uint64_t)((kk * 32) >> 4), dv, idesc_o, 1);
+                    umma_bf16_ts(t_o, tp + (uint32_t)kk * 8, dv, idesc_o, t > 0 || kk > 0);
+                    umma_bf16_ts(t_o, tp + 32 + (uint32_t)kk * 8, dv, idesc_o, 1);
                 }
                 umma_commit(&v_empty[st]);  // the V tile and this buffer of weights are free once these have read them
                 umma_commit(&o_full[b]);
@@ -271,12 +291,15 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
         if (warp_idle && n_tiles > 0) {
             // warps without query vectors: their rows of the weight planes stay zero, and they only
             // keep the barriers' arrival counts whole
-            for (int cc = 0; cc < 16; cc++) {  // both buffers, both planes, this warp's four chunks of the row
-                const int c = half * 4 + (cc & 3);
-                *reinterpret_cast<uint4 *>(base_p + TA_Q_BYTES + (cc >> 2) * (TA_P_BYTES / 2) + (uint32_t)qi * 128 + (c << 4)) =
-                    make_uint4(0, 0, 0, 0);
+            {   // both buffers, both planes, this warp's 16 columns of each
+                uint32_t z[16];
+#pragma unroll
+                for (int i = 0; i < 16; i++) z[i] = 0u;
+#pragma unroll
+                for (int pl = 0; pl < 4; pl++) tmem_st16(t_p + lane_addr + (uint32_t)(pl * 32 + half * 16), z);
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                tc_fence_before();
             }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             for (int t = 0; t < n_tiles && ok; t++) {
                 if (!(ok = mbar_wait(&s_full[t & 1], (t >> 1) & 1, giving_up, args.status))) break;
                 if (t >= 2 && !(ok = mbar_wait(&o_full[t & 1], ((t >> 1) - 1) & 1, giving_up, args.status))) break;
@@ -393,15 +416,17 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
                     }
                 }
                 if (ok) {
+                    uint32_t ph[16], pl[16];
 #pragma unroll
-                    for (int cc = 0; cc < 4; cc++) {
-                        const int c = half * 4 + cc;
-                        const uint32_t off = (uint32_t)b * TA_P_BYTES + (uint32_t)qi * 128 + (uint32_t)((c ^ (qi & 7)) << 4);
-                        *reinterpret_cast<uint4 *>(base_p + TA_Q_BYTES + off) = whi[cc];
-                        *reinterpret_cast<uint4 *>(base_p + TA_Q_BYTES + TA_P_BYTES / 2 + off) = wlo[cc];
+                    for (int c = 0; c < 4; c++) {
+                        ph[c * 4] = whi[c].x; ph[c * 4 + 1] = whi[c].y; ph[c * 4 + 2] = whi[c].z; ph[c * 4 + 3] = whi[c].w;
+                        pl[c * 4] = wlo[c].x; pl[c * 4 + 1] = wlo[c].y; pl[c * 4 + 2] = wlo[c].z; pl[c * 4 + 3] = wlo[c].w;
                     }
+                    const uint32_t tp = t_p + lane_addr + (uint32_t)(b * 64 + half * 16);
+                    tmem_st16(tp, ph);
+                    tmem_st16(tp + 32, pl);
+                    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                     tc_fence_before();
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     mbar_arrive(&p_full[b]);
                 }
                 l_run = l_run * factor + psum;
@@ -454,7 +479,7 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
     }
 }
 
