@@ -82,12 +82,16 @@ def head_logits(dims: dict, w: dict, layer: int, h: np.ndarray) -> np.ndarray:
 
 def scheduled_depth(dims: dict, modality: int, c: int) -> int:
     """Sec. IV-B.1: in-chunk index c runs all L layers iff c mod K == r; text always does
-    unless text_exit is set (1: text too; 2: text only, speech always full, Sec. V-E row G10)."""
+    unless text_exit is set (1: text too; 2: text only, speech always full, Sec. V-E row G10).
+    Text positions that follow the schedule may have their own (text_period, text_phase)."""
     L, e = dims["n_layers"], dims["exit_layer"]
     te = dims.get("text_exit", 0)
     if (modality == 0 and te == 0) or (modality == 1 and te == 2):
         return L
-    return L if c % dims["refresh_period"] == dims["refresh_phase"] else e
+    K, r = dims["refresh_period"], dims["refresh_phase"]
+    if modality == 0 and dims.get("text_period", 0) > 0:      # text positions with a period of their own
+        K, r = dims["text_period"], dims.get("text_phase", 0)
+    return L if c % K == r else e
 
 
 def decode_stream(dims: dict, w: dict, prompt, modalities, counters, forced=None):

@@ -22,7 +22,7 @@ class _Dims(C.Structure):
                                          "head_dim", "d_ffn", "vocab_text", "vocab_speech")] + [
         ("rms_eps", C.c_double), ("rope_base", C.c_double)] + [
         (n, C.c_int32) for n in ("exit_layer", "refresh_period", "refresh_phase", "text_exit",
-                                 "max_len")]
+                                 "max_len", "text_period", "text_phase")]
 
 
 _PP = C.POINTER(C.c_void_p)
@@ -46,6 +46,8 @@ def lib():
         L = C.CDLL(_build.build())
         L.ora_depth.restype = C.c_int32
         L.ora_depth.argtypes = [C.c_int32] * 7
+        L.ora_depth_mod.restype = C.c_int32
+        L.ora_depth_mod.argtypes = [C.c_int32] * 9
         L.ora_rmsnorm.restype = None
         L.ora_rmsnorm.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_double, C.c_void_p]
         L.ora_rope.restype = None
@@ -80,6 +82,11 @@ def lib():
 
 def depth(modality: int, c: int, K: int, r: int, e: int, L: int, text_exit: int = 0) -> int:
     return lib().ora_depth(modality, c, K, r, e, L, text_exit)
+
+
+def depth_mod(modality: int, c: int, K_s: int, r_s: int, K_t: int, r_t: int, e: int, L: int,
+              text_exit: int) -> int:
+    return lib().ora_depth_mod(modality, c, K_s, r_s, K_t, r_t, e, L, text_exit)
 
 
 def _u16(a) -> np.ndarray:
@@ -124,6 +131,8 @@ class OracleModel:
                   "vocab_text", "vocab_speech", "exit_layer", "refresh_period", "refresh_phase"):
             setattr(d, k, int(dims[k]))
         d.text_exit = int(dims.get("text_exit", 0))
+        d.text_period = int(dims.get("text_period", 0))
+        d.text_phase = int(dims.get("text_phase", 0))
         d.rms_eps = float(dims["rms_eps"])
         d.rope_base = float(dims["rope_base"])
         d.max_len = int(max_len)

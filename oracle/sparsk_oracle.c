@@ -57,6 +57,10 @@ typedef struct {
                                2: only text follows it, speech always runs L
                                   layers (Sec. V-E, row G10: text Even, speech --) */
     int32_t max_len;        /* positions a sequence can hold                      */
+    int32_t text_period;    /* K of text positions when they follow the schedule
+                               (text_exit 1 or 2); 0: the same K and r as speech:
+                               the modalities may need different policies (Sec. V-E) */
+    int32_t text_phase;     /* r of text positions, in [0, text_period)           */
 } ora_dims;
 
 typedef struct {
@@ -107,6 +111,16 @@ int32_t ora_depth(int32_t modality, int32_t c, int32_t K, int32_t r, int32_t e, 
     if (modality == 0 && text_exit == 0) return L;
     if (modality == 1 && text_exit == 2) return L;
     return (c % K == r) ? L : e;
+}
+
+/* The same rule with a period and a phase of its own for each modality (Sec. V-E: text and
+ * speech positions may need different policies): speech positions use (K_s, r_s), text
+ * positions that follow the schedule use (K_t, r_t). */
+int32_t ora_depth_mod(int32_t modality, int32_t c, int32_t K_s, int32_t r_s, int32_t K_t,
+                      int32_t r_t, int32_t e, int32_t L, int32_t text_exit)
+{
+    if (modality == 0) return ora_depth(0, c, K_t, r_t, e, L, text_exit);
+    return ora_depth(1, c, K_s, r_s, e, L, text_exit);
 }
 
 /* y = x / sqrt(mean(x^2) + eps) * g */
@@ -188,6 +202,8 @@ ora_model *ora_model_new(const ora_dims *dm, const ora_weights *w)
     if (dm->refresh_period < 1 || dm->refresh_phase < 0 || dm->refresh_phase >= dm->refresh_period)
         return NULL;
     if (dm->n_q_heads % dm->n_kv_heads != 0 || dm->head_dim % 2 != 0) return NULL;
+    if (dm->text_period < 0 || (dm->text_period > 0 && (dm->text_phase < 0 || dm->text_phase >= dm->text_period)))
+        return NULL;
     ora_model *m = (ora_model *)calloc(1, sizeof *m);
     m->dm = *dm;
     m->w = *w;
@@ -259,7 +275,7 @@ void ora_set_len(ora_seq *s, int32_t len)
  * updated in place from h^(layer-1) to h^(layer).  All rows first write their
  * K/V into the cache, then every row attends to positions 0..pos[i]: that is
  * the causal mask over the block plus the whole earlier cache (Algorithm 1,
- * "batch P u {t} through layers l_EE+1..L").
+ * full-depth branch: pending positions and the current one pass the upper layers together).
  */
 static void layer_block(ora_seq *s, int layer, const int32_t *pos, int n_rows, double *H)
 {
@@ -277,7 +293,6 @@ static void layer_block(ora_seq *s, int layer, const int32_t *pos, int n_rows, d
     double *T = (double *)malloc(sizeof(double) * (size_t)n_rows * d);
     double *Gt = (double *)malloc(sizeof(double) * (size_t)n_rows * F);
     double *Up = (double *)malloc(sizeof(double) * (size_t)n_rows * F);
-    double *wts = (double *)malloc(sizeof(double) * (size_t)dm->max_len);
 
     for (int i = 0; i < n_rows; i++)
         ora_rmsnorm(H + (size_t)i * d, w->attn_norm[li], d, dm->rms_eps, A + (size_t)i * d);
@@ -290,13 +305,21 @@ static void layer_block(ora_seq *s, int layer, const int32_t *pos, int n_rows, d
         memcpy(kv_at(s->K, dm, layer, pos[i]), Kn + (size_t)i * kd, sizeof(double) * kd);
         memcpy(kv_at(s->V, dm, layer, pos[i]), Vn + (size_t)i * kd, sizeof(double) * kd);
     }
-    for (int i = 0; i < n_rows; i++)
-        for (int j = 0; j < Hq; j++) {
-            int kvh = j / G;
-            ora_attend(Q + (size_t)i * qd + j * hd, kv_at(s->K, dm, layer, 0) + kvh * hd,
-                       kv_at(s->V, dm, layer, 0) + kvh * hd, pos[i] + 1, hd, kd, wts,
-                       O + (size_t)i * qd + j * hd);
-        }
+    /* every (row, head) pair is one independent call of ora_attend; the pairs are only dealt to
+     * threads, each with its own buffer for the softmax weights */
+#pragma omp parallel
+    {
+        double *wts = (double *)malloc(sizeof(double) * (size_t)dm->max_len);
+#pragma omp for collapse(2) schedule(static)
+        for (int i = 0; i < n_rows; i++)
+            for (int j = 0; j < Hq; j++) {
+                int kvh = j / G;
+                ora_attend(Q + (size_t)i * qd + j * hd, kv_at(s->K, dm, layer, 0) + kvh * hd,
+                           kv_at(s->V, dm, layer, 0) + kvh * hd, pos[i] + 1, hd, kd, wts,
+                           O + (size_t)i * qd + j * hd);
+            }
+        free(wts);
+    }
     matmul_rows(w->wo[li], d, qd, O, n_rows, T);
     for (size_t i = 0; i < (size_t)n_rows * d; i++) H[i] += T[i];
 
@@ -308,7 +331,7 @@ static void layer_block(ora_seq *s, int layer, const int32_t *pos, int n_rows, d
     matmul_rows(w->w_down[li], d, F, Gt, n_rows, T);
     for (size_t i = 0; i < (size_t)n_rows * d; i++) H[i] += T[i];
 
-    free(A); free(Q); free(Kn); free(Vn); free(O); free(T); free(Gt); free(Up); free(wts);
+    free(A); free(Q); free(Kn); free(Vn); free(O); free(T); free(Gt); free(Up);
 }
 
 static void embed_row(const ora_model *m, int32_t token, double *h)
@@ -389,8 +412,10 @@ int32_t ora_decode_step(ora_seq *s, int32_t token, int32_t modality, int32_t cou
     const ora_dims *dm = &m->dm;
     const int d = dm->d_model, L = dm->n_layers, e = dm->exit_layer;
     if (s->len >= dm->max_len) return -1;
-    const int dep = ora_depth(modality, counter, dm->refresh_period, dm->refresh_phase, e, L,
-                              dm->text_exit);
+    const int K_t = dm->text_period > 0 ? dm->text_period : dm->refresh_period;
+    const int r_t = dm->text_period > 0 ? dm->text_phase : dm->refresh_phase;
+    const int dep = ora_depth_mod(modality, counter, dm->refresh_period, dm->refresh_phase, K_t, r_t,
+                                  e, L, dm->text_exit);
     if (dep < L && s->n_pending >= s->max_pending) return -1;
     if (!m->w.head_norm[dep - 1] || !m->w.head_proj[dep - 1]) return -2;
 

@@ -51,17 +51,19 @@ def test_matches_cache_free_recomputation(e, K, r, nt, ns, phase):
         assert abs(g["margin"] - x["margin"]) < 1e-9
 
 
-@pytest.mark.parametrize("text_exit,K,r,nt,ns,running", [
-    (1, 2, 0, 3, 4, False),    # text and speech both follow Even
-    (2, 2, 0, 5, 3, False),    # text only (Sec. V-E row G10); speech flushes the pending text rows
-    (0, 6, 5, 1, 5, False),    # fixed-layer exit: no refresh inside a chunk, the text step flushes 5 rows
-    (0, 3, 0, 1, 4, True),     # counter running across chunks instead of restarting
-    (0, 2, 1, 1, 4, False)])   # Odd
-def test_schedule_variants_match_cache_free_recomputation(text_exit, K, r, nt, ns, running):
+@pytest.mark.parametrize("text_exit,K,r,nt,ns,running,tp,tr", [
+    (1, 2, 0, 3, 4, False, 0, 0),    # text and speech both follow Even
+    (2, 2, 0, 5, 3, False, 0, 0),    # text only (Sec. V-E row G10); speech flushes the pending text rows
+    (0, 6, 5, 1, 5, False, 0, 0),    # fixed-layer exit: no refresh inside a chunk, the text step flushes 5 rows
+    (0, 3, 0, 1, 4, True, 0, 0),     # counter running across chunks instead of restarting
+    (0, 2, 1, 1, 4, False, 0, 0),    # Odd
+    (1, 4, 0, 6, 8, False, 3, 1),    # a period and phase of its own for each modality (Sec. V-E)
+    (2, 2, 0, 6, 2, False, 3, 2)])   # text only, with its own period
+def test_schedule_variants_match_cache_free_recomputation(text_exit, K, r, nt, ns, running, tp, tr):
     """The schedule variants of Sec. IV-B.1 / V-B / V-E: whatever the caller's counters make of the
     depths, pending rows persist until the next full-depth step of either modality and the stream
     equals cache-free recomputation."""
-    dims = synth.model_dims(MICRO, 2, K, r, text_exit=text_exit)
+    dims = synth.model_dims(MICRO, 2, K, r, text_exit=text_exit, text_period=tp, text_phase=tr)
     w = synth.make_weights(dims, seed=13)
     prompt = synth.make_prompts(dims, 1, 6, 6, seed=3)[0]
     mc = [synth.interleave(g, nt, ns, running=running) for g in range(26)]
@@ -77,6 +79,10 @@ def test_schedule_variants_match_cache_free_recomputation(text_exit, K, r, nt, n
     if text_exit == 2:
         assert all(d == 3 for d, m in zip(depths, mods) if m == 1)
         assert any(d == 2 for d, m in zip(depths, mods) if m == 0)
+    if tp:       # each modality follows its own (period, phase): text counters are in-chunk indices
+        assert [d for d, m in zip(depths, mods) if m == 0] == [3 if c % tp == tr else 2 for c, m in zip(ctrs, mods) if m == 0]
+        if text_exit == 1:
+            assert [d for d, m in zip(depths, mods) if m == 1] == [3 if c % K == r else 2 for c, m in zip(ctrs, mods) if m == 1]
     if K == 6:   # fixed-layer: every speech step leaves early, pending reaches the chunk length
         assert all(d == 2 for d, m in zip(depths, mods) if m == 1)
         assert max(len(g["pending_after"]) for g in got) == ns

@@ -104,6 +104,33 @@ def test_mean_depth_identity_on_whole_periods():
             assert gap <= Fraction((40 - 30) * (K - 1), K * N)
 
 
+def test_per_modality_period_and_phase():
+    """Sec. V-E asks for different policies for text and speech.  With a period and phase of its
+    own per modality each side keeps the closed forms of Sec. IV-B.1 independently: the number of
+    full-depth positions of a chunk is floor((N - r + K - 1) / K) with that modality's (K, r), and
+    the mean depth over whole periods is (e (K - 1) + L) / K; the paper's own two-sided row G11
+    has speech on Even(36) at 38.00 whatever the text side does."""
+    L, e = 40, 36
+    for Ks, rs, Kt, rt in ((2, 0, 3, 1), (4, 0, 2, 1), (2, 1, 5, 4), (3, 2, 3, 0)):
+        for N in (1, 5, 13, 26):
+            sp = [ora.depth_mod(1, c, Ks, rs, Kt, rt, e, L, 1) for c in range(N)]
+            tx = [ora.depth_mod(0, c, Ks, rs, Kt, rt, e, L, 1) for c in range(N)]
+            assert sum(d == L for d in sp) == (N - rs + Ks - 1) // Ks
+            assert sum(d == L for d in tx) == (N - rt + Kt - 1) // Kt
+            assert set(sp + tx) <= {e, L}
+        for K, r, mod in ((Ks, rs, 1), (Kt, rt, 0)):
+            whole = [ora.depth_mod(mod, c, Ks, rs, Kt, rt, e, L, 1) for c in range(K * 4)]
+            assert Fraction(sum(whole), len(whole)) == Fraction(e * (K - 1) + L, K)
+        # the modes that exempt a modality still do
+        assert all(ora.depth_mod(0, c, Ks, rs, Kt, rt, e, L, 0) == L for c in range(12))
+        assert all(ora.depth_mod(1, c, Ks, rs, Kt, rt, e, L, 2) == L for c in range(12))
+        # with the same pair on both sides it is the one-pair rule
+        assert [ora.depth_mod(m, c, Ks, rs, Ks, rs, e, L, 1) for m in (0, 1) for c in range(9)] == \
+               [ora.depth(m, c, Ks, rs, e, L, 1) for m in (0, 1) for c in range(9)]
+    # row G11's speech side: Even(36) on the 26-position chunk of the 40-layer backbone
+    assert sum(ora.depth_mod(1, c, 2, 0, 7, 3, 36, 40, 1) for c in range(26)) / 26 == 38.0
+
+
 def test_K1_and_e_equal_L_are_full_depth():
     assert all(ora.depth(1, c, 1, 0, 5, 9) == 9 for c in range(20))
     assert all(ora.depth(1, c, 4, 0, 9, 9) == 9 for c in range(20))
