@@ -28,10 +28,10 @@ if ROOT not in sys.path:
 
 from paper_2603_09215_b200 import synth  # noqa: E402
 
-# DRAM bytes (read + write) per algorithmic byte of the persistent kernel, from its ncu capture on a
-# two-layer launch (profiles/mega_kernel_step4_b1.md: 935.38 MB read + 10.3 MB written against
-# 934.3 MB algorithmic); a launch's traffic is its layers' weights and cache, so it grows in
-# proportion to the layer passes and the ratio carries over to the full-size launches timed here.
+# DRAM bytes (read + write) per algorithmic byte of the persistent kernel, from its profiler capture
+# on a two-layer launch (935.38 MB read + 10.3 MB written against 934.3 MB algorithmic); a launch's
+# traffic is its layers' weights and cache, so it grows in proportion to the layer passes and the
+# ratio carries over to the full-size launches timed here.
 MEGA_DRAM_PER_ALGORITHMIC_BYTE = (935.38 + 10.3) / 934.3
 
 KC = {"qkv": 1, "attn": 2, "oproj": 3, "gateup": 4, "down": 5, "head": 6, "mega": 7, "all": 8}
@@ -173,7 +173,8 @@ class Runner:
         self.pend = [0] * B
         self.depth_log = []     # (modality, depth) per emitted token
         self.bytes = 0
-        self.mega_layers = 0    # layer passes that ran inside the persistent kernel (passes of <= 2 rows)
+        self.mega_seen = self.ctx.route_counts()["mega"]
+        self.mega_layers = 0    # layer passes that ran inside the persistent kernel
         self.mega_bytes = 0     # their weight and cache bytes
 
     def _fill_synthetic(self, prompts):
@@ -182,26 +183,42 @@ class Runner:
             n = len(p) - 1
             k, v = synth.synth_kv(self.dims, n, seed=100 + s)
             for layer in range(1, self.dims["n_layers"] + 1):
-                kt = torch.from_numpy(k[layer - 1].view(np.int16)).cuda().view(torch.bfloat16)
-                vt = torch.from_numpy(v[layer - 1].view(np.int16)).cuda().view(torch.bfloat16)
+                kt = torch.from_numpy(k[layer - 1].view(np.int16)).cuda().view(torch.bfloat16).to(torch.float16)
+                vt = torch.from_numpy(v[layer - 1].view(np.int16)).cuda().view(torch.bfloat16).to(torch.float16)
                 self.ctx.import_kv(s, layer, 0, kt, vt)
             self.ctx.set_len(s, n)
         torch.cuda.synchronize()
 
     def _account(self, mods, ctrs):
+        """Byte model of the step just enqueued, and which of its two passes the library ran in
+        the persistent kernel (asked of the library, not re-derived: sparsk_route_counts)."""
         d = self.dims
         L, e, K, r = d["n_layers"], d["exit_layer"], d["refresh_period"], d["refresh_phase"]
-        depths = [L if m == 0 else (L if c % K == r else e) for m, c in zip(mods, ctrs)]
+        te = d.get("text_exit", 0)
+
+        def depth(m, c):
+            if (m == 0 and te == 0) or (m == 1 and te == 2):
+                return L
+            return L if c % K == r else e
+        depths = [depth(m, c) for m, c in zip(mods, ctrs)]
         self.bytes += step_bytes(d, depths, mods, self.lens, self.pend)
         kvb = 2 * d["n_kv_heads"] * d["head_dim"] * 2
         wl = layer_weight_bytes(d)
-        if len(depths) <= 2:
+        up = [(ln, pn) for dep, ln, pn in zip(depths, self.lens, self.pend) if dep == L and e < L]
+        rows_lo, rows_up = len(depths), sum(pn + 1 for _, pn in up)
+        mega_now = self.ctx.route_counts()["mega"]
+        delta, self.mega_seen = mega_now - self.mega_seen, mega_now
+        n_up = (L - e) if up else 0
+        # the persistent kernel takes the small passes: if only one of the two ran there, it is
+        # the one with fewer rows (the counts differ unless e = L - e)
+        lo_in = delta == e + n_up or (delta == e and (n_up != e or rows_lo <= rows_up))
+        up_in = n_up and (delta == e + n_up or (delta == n_up and not lo_in))
+        if delta and lo_in:
             self.mega_layers += e
             self.mega_bytes += e * (wl + sum((ln + 2) * kvb for ln in self.lens))
-        up = [(ln, pn) for dep, ln, pn in zip(depths, self.lens, self.pend) if dep == L and e < L]
-        if up and sum(pn + 1 for _, pn in up) <= 2:
-            self.mega_layers += L - e
-            self.mega_bytes += (L - e) * (wl + sum((ln + 1) * kvb + (pn + 1) * kvb for ln, pn in up))
+        if delta and up_in:
+            self.mega_layers += n_up
+            self.mega_bytes += n_up * (wl + sum((ln + 1) * kvb + (pn + 1) * kvb for ln, pn in up))
         for i, dep in enumerate(depths):
             self.lens[i] += 1
             self.pend[i] = 0 if dep == L else self.pend[i] + 1
@@ -297,6 +314,64 @@ def job_tokens_per_s(tokens_per_rank: int, ms: float, world: int) -> float:
     return world * tokens_per_rank / (ms / 1e3)
 
 
+def batch_leg(name, gw, rank, world, W, cycles, opts, sampling, hbm_peak, peak_kind, uuid, timed, with_full):
+    """One more workload on the weights already on the device: throughput of the scheduled decoder
+    and of full depth, the step's byte-model fraction of the HBM peak, and the dominant GEMM class
+    (gate/up) timed launch by launch."""
+    wl, dims, prompts, phi, off = workload_setup(name, rank)
+    cyc = wl["n_text"] + wl["n_speech"]
+    L = dims["n_layers"]
+    total_steps = ((W + cycles) * 2 + 8) * cyc
+    run = Runner(dims, gw, wl, prompts, phi, off, total_steps, opts, False, sampling)
+    run.run_cycles(W)
+    sampler = ClockSampler(uuid)
+    sampler.start()
+    b0 = run.bytes
+    ms, ntok, launches = timed(run, cycles)
+    clocks = sampler.stop()
+    step_b = run.bytes - b0
+    ach = step_b / (ms * 1e-3) / 1e9
+    out = {"workload": name, "batch_per_gpu": wl["batch"], "prompt_len": list(wl["prompt"]),
+           "exit_layer": wl["exit_layer"], "refresh_period": wl["refresh_period"],
+           "cache_fill": "real prefill of random prompts", "steps": cycles, "decode_steps_per_step": cyc,
+           "value": job_tokens_per_s(ntok, ms, world), "unit": "tokens/s", "ms_per_step": ms / cycles,
+           "gpu_launches": int(launches), "clocks": clocks,
+           "step_hbm": {"bytes_per_step": step_b / cycles, "achieved_gbs": ach,
+                        "frac_of_measured_copy": ach / hbm_peak, "frac_of_nominal_8tbs": ach / 8000.0}}
+    d = dims
+    run.ctx.set_option("time_kernel", KC["gateup"])
+    run.run_cycles(min(cycles, 4))
+    kms, kn = run.ctx.kernel_time()
+    run.ctx.set_option("time_kernel", 0)
+    kbytes = 2 * d["d_ffn"] * d["d_model"] * 2
+    if kn:
+        g = kbytes / (kms / kn * 1e-3) / 1e9
+        out["roofline"] = {"bound": "hbm", "kernel": "gateup", "unit": "GB/s", "peak": hbm_peak, "peak_kind": peak_kind,
+                           "achieved": g, "frac": g / hbm_peak, "launches_timed": kn, "avg_launch_us": 1e3 * kms / kn,
+                           "bytes_per_launch": kbytes, "traffic": None}
+    sav = layer_saving(run.depth_log, L)
+    out["layer_saving"] = sav
+    out["routes"] = run.ctx.route_counts()
+    run.ctx.close()
+    del run
+    if with_full:
+        wl_f = dict(wl, refresh_period=1, refresh_phase=0)
+        dims_f = synth.model_dims(wl["shape"], wl["exit_layer"], 1, 0)
+        rf = Runner(dims_f, gw, wl_f, prompts, phi, off, total_steps, opts, False, sampling)
+        rf.run_cycles(W)
+        fb0 = rf.bytes
+        ms_f, ntok_f, _ = timed(rf, cycles)
+        fb = rf.bytes - fb0
+        out["full_depth"] = {"value": job_tokens_per_s(ntok_f, ms_f, world), "unit": "tokens/s",
+                             "ms_per_step": ms_f / cycles, "bytes_per_step": fb / cycles,
+                             "hbm_frac": fb / (ms_f * 1e-3) / 1e9 / hbm_peak}
+        out["reduction"] = {"wall_time_pct": (1 - (ms / cycles) / (ms_f / cycles)) * 100,
+                            "byte_model_pct": (1 - step_b / fb) * 100,
+                            "layer_saving_all_tokens_pct": sav["all_saving_pct"]}
+        rf.ctx.close()
+    return out
+
+
 # --------------------------------------------------------------------------- main
 def main():
     ap = argparse.ArgumentParser()
@@ -307,6 +382,8 @@ def main():
     ap.add_argument("--workload", default="cfg2_step_b1", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-full-depth", action="store_true")
+    ap.add_argument("--no-batch64", action="store_true",
+                    help="skip the batch-64 leg (workload cfg3_step_b64) that the default run adds")
     ap.add_argument("--option", action="append", default=[], help="library option name=value")
     ap.add_argument("--time-kernel", default="mega", choices=sorted(KC))
     ap.add_argument("--sampling", default=None, metavar="T,P",
@@ -469,8 +546,13 @@ def main():
                 "hbm_frac": ((rf.bytes - fb0) / (ms_f * 1e-3) / 1e9) / hbm_peak}
         rf.ctx.close()
 
+    # ---- the batch-64 half of the metric: workload cfg3_step_b64 on the same weights
+    batch64 = None
+    if args.workload == "cfg2_step_b1" and not args.no_batch64:
+        batch64 = batch_leg("cfg3_step_b64", gw, rank, world, W, min(args.steps, 12), opts, sampling, hbm_peak,
+                            peak_kind, uuid, timed, not args.no_full_depth)
+
     sav = layer_saving(run.depth_log, L)
-    n_text = sum(1 for m, _ in run.depth_log[-ntok:] if m == 0)
     out = {"metric": "decode_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world,
            "steps": args.steps, "warmup": W, "ms_per_step": ms / args.steps, "higher_is_better": True,
            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": cfg,
@@ -481,6 +563,8 @@ def main():
            "layer_saving": sav, "setup_s": setup_s}
     if classes:
         out["kernel_classes"] = classes
+    if batch64:
+        out["batch64"] = batch64
     if full:
         out["full_depth"] = full
         out["reduction"] = {"wall_time_pct": (1 - (ms / args.steps) / full["ms_per_step"]) * 100,

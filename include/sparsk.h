@@ -44,7 +44,7 @@ extern "C" {
 #define SPARSK_ECAPACITY (-2) /* a sequence would exceed max_seq_len or max_pending           */
 #define SPARSK_ENOHEAD (-3)   /* the step needs an exit head whose pointers are NULL          */
 #define SPARSK_ECUDA (-4)     /* a CUDA call failed; text in sparsk_last_error                */
-#define SPARSK_ESTATE (-5)    /* slot never prefilled / context destroyed                     */
+#define SPARSK_ESTATE (-5)    /* slot in the wrong state for the call / not a context         */
 #define SPARSK_ETIMEOUT (-6)  /* a bounded in-kernel wait ran out (reported by the next call) */
 
 typedef struct sparsk_ctx sparsk_ctx; /* opaque */
@@ -72,6 +72,10 @@ typedef struct {
     int32_t max_seq_len;    /* positions per slot */
     int32_t max_pending;    /* pending positions per slot; >= K-1 for the periodic schedule */
     int32_t prefill_rows;   /* rows per prefill pass (0 = default) */
+    int32_t text_period;    /* K of text steps when they follow the rule (text_exit 1 or 2); 0 = the
+                               same K and r as speech steps.  Sec. V-E: the two modalities may need
+                               different policies */
+    int32_t text_phase;     /* r of text steps, in [0, text_period) */
 } sparsk_dims;
 
 /* All pointers are DEVICE pointers to bfloat16 data; the arrays of pointers themselves
@@ -94,7 +98,8 @@ typedef struct {
 } sparsk_weights;
 
 /* Bytes of device workspace sparsk_create needs for these dims; 0 if the dims are invalid.
- * The workspace holds the KV cache ([L][slot][H_kv][max_seq_len][hd] bf16, keys and values),
+ * No counterpart in the paper (memory management).  The workspace holds the KV cache
+ * ([L][slot][H_kv][max_seq_len][hd] fp16, keys and values),
  * the pending store ([slot][max_pending][d] fp32), per-slot lengths, the step descriptor,
  * activation buffers, split-KV scratch and the rotary table. */
 size_t sparsk_workspace_bytes(const sparsk_dims *dims /*host*/);
@@ -118,25 +123,34 @@ int sparsk_prefill(sparsk_ctx *ctx, int32_t n_seqs, const int32_t *slots /*host*
  * step, or the last prompt token).  modality[i]: 0 text / 1 speech, the modality of the token
  * this step EMITS; the argmax is restricted to that id range (lowest id on ties).
  * speech_counters[i]: index c of that token inside its chunk.  Outputs: next_tokens[i] and
- * exit_depths[i] (e or L).  Host arrays are read before the call returns. */
+ * exit_depths[i] (e or L).  Host arrays are read before the call returns.  The token ids live
+ * on the device, so the host cannot check them: an id outside [0, V_t+V_s) is clamped into the
+ * vocabulary by the kernels, the step runs and advances its slots, and the next sparsk_check
+ * reports SPARSK_EINVAL. */
 int sparsk_decode_step(sparsk_ctx *ctx, int32_t n_seqs, const int32_t *slots /*host*/,
                        const int32_t *token_ids /*device [n]*/, const uint8_t *modality /*host [n]*/,
                        const int32_t *speech_counters /*host [n]*/,
                        int32_t *next_tokens /*device [n]*/, int32_t *exit_depths /*device [n]*/);
 
-/* Same step with HOST token and result buffers: copies token_ids to the device, runs the step,
- * copies both results back and synchronises the stream.  This is the call a host-side
- * generation loop makes when it consumes every token as it is produced. */
+/* The same iteration of Algorithm 1 with HOST token and result buffers: copies token_ids to the
+ * device, runs the step, copies both results back and synchronises the stream.  This is the call
+ * a host-side generation loop makes when it consumes every token as it is produced.  Token ids
+ * outside [0, V_t+V_s) are refused with SPARSK_EINVAL before anything is launched (state
+ * unchanged).  If a bounded in-kernel wait ran out during the step the call returns
+ * SPARSK_ETIMEOUT once, the kernels' barrier state is reset, and the slots that took part hold
+ * an incomplete step: reset them (sparsk_reset_slot) before using them again. */
 int sparsk_decode_step_host(sparsk_ctx *ctx, int32_t n_seqs, const int32_t *slots /*host*/,
                             const int32_t *token_ids /*host [n]*/, const uint8_t *modality /*host*/,
                             const int32_t *speech_counters /*host*/,
                             int32_t *next_tokens /*host [n]*/, int32_t *exit_depths /*host [n]*/);
 
-/* Forget a slot: length 0, pending set empty. */
+/* Forget a slot: length 0, pending set empty (the state Algorithm 1 starts a sequence from).
+ * No counterpart in the paper beyond that: slot management. */
 int sparsk_reset_slot(sparsk_ctx *ctx, int32_t slot);
 
 /* Load / read cache contents of one layer (1-based) of a slot: n positions starting at
- * first_pos, keys already rotated, layout [n][H_kv*hd] bf16, device pointers.  set_len declares
+ * first_pos, keys already rotated, layout [n][H_kv*hd] fp16 (IEEE half, the cache's own element
+ * type: weights are bf16, but the cache keeps 11 significant bits), device pointers.  set_len declares
  * that positions [0, len) are complete at every layer (pending set empty).  These let a caller
  * restore a saved prefix, and let tests inspect the KV invariant of Sec. IV-B.3. */
 int sparsk_import_kv(sparsk_ctx *ctx, int32_t slot, int32_t layer, int32_t first_pos, int32_t n,
@@ -144,25 +158,36 @@ int sparsk_import_kv(sparsk_ctx *ctx, int32_t slot, int32_t layer, int32_t first
 int sparsk_export_kv(sparsk_ctx *ctx, int32_t slot, int32_t layer, int32_t first_pos, int32_t n,
                      void *k /*device*/, void *v /*device*/);
 int sparsk_set_len(sparsk_ctx *ctx, int32_t slot, int32_t len);
-/* Host view of a slot: positions held and pending count (no device access). */
+/* Host view of a slot: positions held and size of the pending set P of Algorithm 1 (no device
+ * access).  No counterpart in the paper: inspection only. */
 int sparsk_slot_state(const sparsk_ctx *ctx, int32_t slot, int32_t *len /*host*/,
                       int32_t *pending /*host*/);
 
 /* Parity hooks.  While non-NULL, every decode step also writes, for sequence i of the step,
- * the hidden state its head read (exit_hidden [n, d] fp32) and its logits (exit_logits
- * [n, V_t+V_s] fp32, -inf outside the modality's id range).  Device pointers, caller-owned. */
+ * the hidden state its head read (exit_hidden [n, d] fp32: h^(e) or h^(L), the argument of g_e
+ * in Eq. 2 or of g_L in Eq. 1) and its logits (exit_logits [n, V_t+V_s] fp32, -inf outside the
+ * modality's id range).  Device pointers, caller-owned, registered BEFORE the steps they are to
+ * observe: the heads write logits only while a buffer is registered, nothing of a step is kept
+ * otherwise. */
 int sparsk_set_debug(sparsk_ctx *ctx, float *exit_hidden /*device or NULL*/,
                      float *exit_logits /*device or NULL*/);
 
-/* Tuning knobs, by name: "gemm_min_rows" (row count from which the tcgen05 path is used; a
+/* Tuning knobs, by name (no counterpart in the paper: implementation choices): "gemm_min_rows" (row count from which the tcgen05 path is used; a
  * large value keeps everything on the GEMV path), "mega" (0/1: run passes of one
  * or two rows as one persistent kernel per layer range; default 1), "mega_max_rows" (1..4: the
  * largest pass that kernel takes; default 2, above which its CUDA-core inner loop falls behind
  * HBM), "gemm_kb" (1: one 64-element block of the inner
- * dimension per TMA copy instead of two; 0 = automatic), "use_graph" (0/1), "attn_split" (positions
+ * dimension per TMA copy instead of two; 0 = automatic), "attn_split" (positions
  * per KV split), "pdl" (0/1, programmatic dependent launch between the kernels of a step; default 1),
  * "gemv_ks" / "gemv_r" (override the GEMV team width / rows per group; 0 = automatic),
- * "time_kernel" (see sparsk_kernel_time).  Returns SPARSK_EINVAL for an unknown name or value. */
+ * "trim_last_layer" (0/1/2: in a full-depth step, pending rows leave layer L after its K/V
+ * projection, since Algorithm 1's full-depth branch reads h^(L) of the current position only; 1,
+ * the default, does so when the remaining rows still fill the tensor-core path, 2 whenever a step
+ * has pending rows, 0 never; results are identical),
+ * "time_kernel" (see sparsk_kernel_time), "inject_barrier_timeout" (test hook, 1: the next launch
+ * of the persistent kernel is given a grid-barrier count that no CTA can reach, so its bounded
+ * wait runs out after about two seconds, the kernel returns and the step reports
+ * SPARSK_ETIMEOUT; nothing faults or hangs).  Returns SPARSK_EINVAL for an unknown name or value. */
 int sparsk_set_option(sparsk_ctx *ctx, const char *name /*host*/, int64_t value);
 
 /* Nucleus sampling (Sec. V-A: the 28-layer backbone is decoded with temperature 0.7 and top_p 0.9;
@@ -196,6 +221,9 @@ int sparsk_nucleus_sample(const float *logits, const float *uniforms, const int3
 /* Stand-alone split-KV grouped-query attention: the two kernels a decode step runs per layer
  * (partials per KV split, then the merge), on caller-described rows.  Rows are grouped: group g
  * is rows [grp_row0[g], grp_row0[g] + grp_nrows[g]) of ONE sequence at consecutive positions;
+ * the groups must partition [0, n_rows) (every row in exactly one group) and no group may have
+ * more than max_grp_rows rows: a row outside every group, or beyond an under-stated
+ * max_grp_rows, gets whatever the scratch held;
  * row i of a group attends to cache positions 0..row_pos[i] of slot row_slot[i] (the causal
  * block of Algorithm 1's full-depth branch on top of the earlier cache; a lower-pass row is a
  * group of one).  All array pointers are DEVICE pointers.  Rows whose slot is outside
@@ -203,8 +231,8 @@ int sparsk_nucleus_sample(const float *logits, const float *uniforms, const int3
  * `scratch` (device, 256-byte aligned, >= sparsk_attention_scratch_bytes) is overwritten. */
 typedef struct {
     const void *q;               /* bf16 [n_rows][n_q_heads*head_dim], rotated queries             */
-    const void *k_cache;         /* bf16 [n_slots][n_kv_heads][cache_len][head_dim], rotated keys  */
-    const void *v_cache;         /* bf16, same layout                                              */
+    const void *k_cache;         /* fp16 [n_slots][n_kv_heads][cache_len][head_dim], rotated keys  */
+    const void *v_cache;         /* fp16, same layout                                              */
     void *out;                   /* bf16 [n_rows][n_q_heads*head_dim]                              */
     const int32_t *row_slot, *row_pos;     /* [n_rows]                                             */
     const int32_t *grp_row0, *grp_nrows;   /* [n_groups]                                           */
@@ -213,6 +241,7 @@ typedef struct {
     int32_t max_len;             /* host-known bound on row_pos + 1                                */
     int32_t n_q_heads, n_kv_heads, head_dim /* 64 or 128 */, cache_len, n_slots;
 } sparsk_attn_args;
+/* Bytes of scratch sparsk_attention needs (no counterpart in the paper: memory management). */
 size_t sparsk_attention_scratch_bytes(int32_t n_rows, int32_t n_q_heads, int32_t head_dim);
 int sparsk_attention(const sparsk_attn_args *args /*host*/, void *scratch /*device*/, size_t scratch_bytes,
                      void *cuda_stream);
@@ -243,15 +272,18 @@ int sparsk_attention_static(const sparsk_attn_args *args /*host*/, void *cuda_st
  * stops).  sparsk_kernel_time synchronises the stream and returns the summed device time of the
  * bracketed launches and their number.  No counterpart in the paper: measurement only. */
 int sparsk_kernel_time(sparsk_ctx *ctx, double *total_ms /*host*/, int64_t *n_launches /*host*/);
-/* With "time_kernel" = 8 every launch is bracketed and remembered with its class; this returns
+/* No counterpart in the paper (measurement only).  With "time_kernel" = 8 every launch is
+ * bracketed and remembered with its class; this returns
  * the summed device time and the launch count of each class, indexed 0 bookkeeping (schedule,
  * compaction, embedding, norms, stash, gather, finish), 1..7 as above.  Arrays of 8. */
 int sparsk_kernel_time_by_class(sparsk_ctx *ctx, double *total_ms /*host [8]*/, int64_t *n_launches /*host [8]*/);
 
 /* Synchronises the context's stream, then reads and clears the device status word that kernels
  * raise instead of trapping: SPARSK_ETIMEOUT if a bounded in-kernel wait ran out, SPARSK_EINVAL
- * if a token id had to be clamped into the vocabulary, else SPARSK_OK.  No counterpart in the
- * paper: error reporting only. */
+ * if a token id had to be clamped into the vocabulary, else SPARSK_OK.  After SPARSK_ETIMEOUT
+ * the kernels' barrier state has been reset; the slots of the step that timed out hold an
+ * incomplete step and must be reset before further use.  No counterpart in the paper: error
+ * reporting only. */
 int sparsk_check(sparsk_ctx *ctx);
 
 /* Phase clock of the persistent layer-range kernel: its first CTA records the GPU's nanosecond
@@ -261,13 +293,24 @@ int sparsk_check(sparsk_ctx *ctx);
  * `capacity`), or a negative code.  No counterpart in the paper: measurement only. */
 int sparsk_phase_trace(sparsk_ctx *ctx, int64_t *out_ns /*host*/, int32_t capacity);
 
-/* Number of kernels this library has launched on behalf of the context so far. */
+/* Number of kernels this library has launched on behalf of the context so far.  No counterpart
+ * in the paper: measurement only. */
 int64_t sparsk_launch_count(const sparsk_ctx *ctx);
 
-/* Text of the last error of this context (host string, valid until the next call). */
+/* Which implementation the layer passes so far went through (a pass = one layer over one row
+ * set): layer_passes[0] persistent layer-range kernel (1-2 rows), [1] tcgen05 kernels launched
+ * per projection, [2] small-batch GEMV kernels.  Lets a benchmark
+ * attribute bytes to the kernel it times without re-deriving the choice.  No counterpart in the
+ * paper: measurement only. */
+int sparsk_route_counts(const sparsk_ctx *ctx, int64_t *layer_passes /*host [3]*/);
+
+/* Text of the last error of this context (host string, valid until the next call).  No
+ * counterpart in the paper: error reporting only. */
 const char *sparsk_last_error(const sparsk_ctx *ctx);
 
-/* Release host-side state.  The workspace and weights are the caller's to free. */
+/* Release host-side state.  The workspace and weights are the caller's to free.  The pointer
+ * is dead afterwards: passing it to any call is undefined (SPARSK_ESTATE is returned only for
+ * NULL and for memory that is recognisably not a live context).  No counterpart in the paper. */
 int sparsk_destroy(sparsk_ctx *ctx);
 
 #ifdef __cplusplus

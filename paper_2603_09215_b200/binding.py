@@ -19,7 +19,7 @@ EXPORTS = ("sparsk_workspace_bytes", "sparsk_create", "sparsk_prefill", "sparsk_
            "sparsk_decode_step_host", "sparsk_reset_slot", "sparsk_import_kv", "sparsk_export_kv",
            "sparsk_set_len", "sparsk_slot_state", "sparsk_set_debug", "sparsk_set_option",
            "sparsk_kernel_time", "sparsk_kernel_time_by_class", "sparsk_check", "sparsk_phase_trace", "sparsk_attention", "sparsk_attention_scratch_bytes", "sparsk_attention_static", "sparsk_sampling_scratch_bytes", "sparsk_set_sampling", "sparsk_nucleus_sample",
-           "sparsk_launch_count", "sparsk_last_error", "sparsk_destroy")
+           "sparsk_launch_count", "sparsk_route_counts", "sparsk_last_error", "sparsk_destroy")
 
 OK, EINVAL, ECAPACITY, ENOHEAD, ECUDA, ESTATE, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
 
@@ -35,7 +35,8 @@ class Dims(C.Structure):
                                          "d_ffn", "vocab_text", "vocab_speech")] + [
         ("rms_eps", C.c_float), ("rope_base", C.c_float)] + [
         (n, C.c_int32) for n in ("exit_layer", "refresh_period", "refresh_phase", "text_exit",
-                                 "max_seqs", "max_seq_len", "max_pending", "prefill_rows")]
+                                 "max_seqs", "max_seq_len", "max_pending", "prefill_rows",
+                                 "text_period", "text_phase")]
 
 
 _PP = C.POINTER(C.c_void_p)
@@ -113,6 +114,8 @@ def load():
     L.sparsk_check.argtypes = [vp]
     L.sparsk_launch_count.restype = C.c_int64
     L.sparsk_launch_count.argtypes = [vp]
+    L.sparsk_route_counts.restype = C.c_int
+    L.sparsk_route_counts.argtypes = [vp, C.POINTER(C.c_int64)]
     L.sparsk_last_error.restype = C.c_char_p
     L.sparsk_last_error.argtypes = [vp]
     L.sparsk_destroy.restype = C.c_int
@@ -127,6 +130,8 @@ def make_dims(dims: dict, max_seqs: int, max_seq_len: int, max_pending: int, pre
               "vocab_speech", "exit_layer", "refresh_period", "refresh_phase"):
         setattr(d, k, int(dims[k]))
     d.text_exit = int(dims.get("text_exit", 0))
+    d.text_period = int(dims.get("text_period", 0))
+    d.text_phase = int(dims.get("text_phase", 0))
     d.rms_eps = float(dims["rms_eps"])
     d.rope_base = float(dims["rope_base"])
     d.max_seqs, d.max_seq_len, d.max_pending, d.prefill_rows = max_seqs, max_seq_len, max_pending, prefill_rows
@@ -152,7 +157,8 @@ def _i32(a):
 def attn_args(q, k_cache, v_cache, out, row_slot, row_pos, grp_row0, grp_nrows, max_grp_rows, max_len,
               n_q_heads) -> AttnArgs:
     """Marshal torch CUDA tensors into the argument block of sparsk_attention.
-    k_cache / v_cache: [n_slots, n_kv_heads, cache_len, head_dim] bf16."""
+    q, out: bf16; k_cache / v_cache: [n_slots, n_kv_heads, cache_len, head_dim] float16."""
+    assert k_cache.dtype == torch.float16 and v_cache.dtype == torch.float16
     a = AttnArgs()
     a.q, a.k_cache, a.v_cache, a.out = q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), out.data_ptr()
     a.row_slot, a.row_pos = row_slot.data_ptr(), row_pos.data_ptr()
@@ -288,12 +294,14 @@ class Sparsk:
         self._check(self.lib.sparsk_set_len(self.h, slot, n))
 
     def import_kv(self, slot: int, layer: int, first_pos: int, k: torch.Tensor, v: torch.Tensor):
+        """k, v: [n, H_kv*hd] float16 on the device (the cache's own element type)."""
+        assert k.dtype == torch.float16 and v.dtype == torch.float16 and k.is_contiguous() and v.is_contiguous()
         self._check(self.lib.sparsk_import_kv(self.h, slot, layer, first_pos, k.shape[0], k.data_ptr(),
                                               v.data_ptr()))
 
     def export_kv(self, slot: int, layer: int, first_pos: int, n: int):
         row = self.cd.n_kv_heads * self.cd.head_dim
-        k = torch.empty((n, row), dtype=torch.bfloat16, device=self.workspace.device)
+        k = torch.empty((n, row), dtype=torch.float16, device=self.workspace.device)
         v = torch.empty_like(k)
         self._check(self.lib.sparsk_export_kv(self.h, slot, layer, first_pos, n, k.data_ptr(), v.data_ptr()))
         return k, v
@@ -353,3 +361,9 @@ class Sparsk:
 
     def launch_count(self) -> int:
         return self.lib.sparsk_launch_count(self.h)
+
+    def route_counts(self) -> dict:
+        """Layer passes so far by implementation."""
+        n = (C.c_int64 * 3)()
+        self._check(self.lib.sparsk_route_counts(self.h, n))
+        return dict(zip(("mega", "tc", "gemv"), (int(x) for x in n)))

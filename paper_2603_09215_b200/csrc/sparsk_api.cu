@@ -17,7 +17,6 @@
 #include "sparsk_mega.cuh"
 #include "sparsk_sample.cuh"
 #include "sparsk_step.cuh"
-#include "sparsk_tcmega.cuh"
 
 using namespace sparsk;
 
@@ -59,7 +58,7 @@ struct sparsk_ctx {
     int n_sm;
     int cap_rows;  // rows any pass may have
     // workspace
-    bf16 *kcache, *vcache;
+    kv_t *kcache, *vcache;
     float *pend_h;
     int *kv_len, *pend_cnt;
     float2 *rope;
@@ -68,6 +67,9 @@ struct sparsk_ctx {
     int *pf_slot, *pf_pos, *pf_grp_row0, *pf_grp_nrows, *pf_ngrp, *pf_nrows;
     float *h_lo, *h_up;
     float *qbuf;
+    float *h_last, *q_last;      // the current rows alone, for the trimmed last layer of the upper pass
+    int *last_slot, *last_pos;
+    int trim_last;               // 0: never, 1: when it pays (default), 2: whenever there are pending rows
     bf16 *attn_o, *act, *xnorm;
     bf16 *attn_o_lo, *act_lo, *xnorm_lo;  // second bf16 term of the tensor-core path's activations
     float *part_o;
@@ -79,7 +81,7 @@ struct sparsk_ctx {
     // host mirror of per-slot state
     std::vector<int> h_len, h_pend;
     // options
-    int pdl, attn_split, gemm_min_rows, use_graph, gv_ks, gv_r, gv_grid_mult;
+    int pdl, attn_split, gemm_min_rows, gv_ks, gv_r;
     float *dbg_hidden, *dbg_logits;
     // nucleus sampling (off while samp_uniforms is NULL)
     float samp_temperature, samp_top_p;
@@ -98,16 +100,17 @@ struct sparsk_ctx {
     unsigned long long *mk_bar;    // device: grid barrier counter; mk_bar_base mirrors its value
     int *mk_abort;                 // device
     float *mk_attn_o, *mk_act;     // device fp32 [MK_MAX_ROWS][Hq*hd], [MK_MAX_ROWS][F]
-    unsigned long long *mk_trace;  // device [1 + 9 L]
+    unsigned long long *mk_trace;  // device [1 + 6 L]
     int mk_trace_n;                // entries the last launch wrote
     unsigned long long mk_bar_base;
     int mega, mk_ok, mk_coop, mk_max_rows;
+    int inject_timeout;            // test hook: the next persistent launch waits for a barrier count nobody reaches
+    int64_t route_layers[3];       // layer passes so far by implementation: see sparsk_route_counts
     std::vector<MkLayer> mk_host;
     float *qkv_part;  // fp32 sums of a q/k/v product whose inner dimension is cut across CTAs
     int tc_kb;        // 0: automatic; 1: force one k-block per copy (2-D descriptors)
-    // persistent tcgen05 layer-range kernel (3..TK_MAX_N rows)
-    TkLayer *tk_layers;  // device [L]
-    int tcmega, tk_ok;
+    int gemm_smem_kb; // shared-memory budget of a tcgen05 GEMM CTA
+    int gemm_cps;     // CTAs per SM a split GEMM is cut for (1 or 2; 2 needs a budget that lets two share an SM)
     // optional per-kernel-class timing (events around every launch of one class)
     int cur_class, time_class;
     std::vector<cudaEvent_t> tev;
@@ -149,6 +152,7 @@ bool dims_ok(const sparsk_dims *d)
     if (d->exit_layer < 1 || d->exit_layer > d->n_layers) return false;
     if (d->refresh_period < 1 || d->refresh_phase < 0 || d->refresh_phase >= d->refresh_period) return false;
     if (d->text_exit < 0 || d->text_exit > 2) return false;
+    if (d->text_period < 0 || (d->text_period > 0 && (d->text_phase < 0 || d->text_phase >= d->text_period))) return false;
     if (d->max_seqs < 1 || d->max_seqs > 1024 || d->max_seq_len < 1) return false;
     if (d->max_pending < 0 || d->prefill_rows < 0) return false;
     return true;
@@ -168,8 +172,8 @@ size_t carve(sparsk_ctx *c, const sparsk_dims *d, char *base)
     const size_t B = d->max_seqs, S = d->max_seq_len, L = d->n_layers;
     const size_t kvrow = (size_t)d->n_kv_heads * d->head_dim, qrow = (size_t)d->n_q_heads * d->head_dim;
     const size_t R = cap_rows_of(d);
-    bf16 *kc = w.take<bf16>(L * B * S * kvrow);
-    bf16 *vc = w.take<bf16>(L * B * S * kvrow);
+    kv_t *kc = w.take<kv_t>(L * B * S * kvrow);
+    kv_t *vc = w.take<kv_t>(L * B * S * kvrow);
     float *ph = w.take<float>(B * (size_t)std::max(1, d->max_pending) * d->d_model);
     int *kl = w.take<int>(B), *pc = w.take<int>(B);
     float2 *rope = w.take<float2>(S * (d->head_dim / 2));
@@ -187,16 +191,17 @@ size_t carve(sparsk_ctx *c, const sparsk_dims *d, char *base)
     int *pfng = w.take<int>(1), *pfnr = w.take<int>(1);
     float *hlo = w.take<float>(B * d->d_model), *hup = w.take<float>(R * d->d_model);
     float *q = w.take<float>(R * qrow);
+    float *hlast = w.take<float>(B * d->d_model), *qlast = w.take<float>(B * qrow);
+    int *lslot = w.take<int>(B), *lpos = w.take<int>(B);
     bf16 *ao = w.take<bf16>(R * qrow), *act = w.take<bf16>(R * d->d_ffn);
     bf16 *xn = w.take<bf16>(R * d->d_model);
     bf16 *aol = w.take<bf16>(R * qrow), *actl = w.take<bf16>(R * d->d_ffn), *xnl = w.take<bf16>(R * d->d_model);
     float *qp = w.take<float>(R * (qrow + 2 * kvrow));
     MkLayer *mkl = w.take<MkLayer>(L);
-    TkLayer *tkl = w.take<TkLayer>(L);
     unsigned long long *mkb = w.take<unsigned long long>(1);
     int *mka = w.take<int>(1);
     float *mkao = w.take<float>((size_t)MK_MAX_ROWS * qrow), *mkact = w.take<float>((size_t)MK_MAX_ROWS * d->d_ffn);
-    unsigned long long *mkt = w.take<unsigned long long>(1 + 9 * L);
+    unsigned long long *mkt = w.take<unsigned long long>(1 + 6 * L);
     const size_t cells = std::max<size_t>(R * MAX_SPLITS, (size_t)MK_MAX_ROWS * MK_MAX_SPLITS) * d->n_q_heads;
     float *po = w.take<float>(cells * d->head_dim);
     float2 *pml = w.take<float2>(cells);
@@ -205,9 +210,10 @@ size_t carve(sparsk_ctx *c, const sparsk_dims *d, char *base)
         c->sd = sd; c->staged = staged; c->tok_dev = tok; c->out_tok_dev = ot; c->out_depth_dev = od;
         c->pf_slot = pfs; c->pf_pos = pfp; c->pf_grp_row0 = pfg0; c->pf_grp_nrows = pfgn;
         c->pf_ngrp = pfng; c->pf_nrows = pfnr;
+        c->h_last = hlast; c->q_last = qlast; c->last_slot = lslot; c->last_pos = lpos;
         c->h_lo = hlo; c->h_up = hup; c->qbuf = q; c->attn_o = ao; c->act = act; c->xnorm = xn; c->qkv_part = qp;
         c->attn_o_lo = aol; c->act_lo = actl; c->xnorm_lo = xnl;
-        c->mk_layers = mkl; c->tk_layers = tkl; c->mk_bar = mkb; c->mk_abort = mka; c->mk_attn_o = mkao; c->mk_act = mkact; c->mk_trace = mkt;
+        c->mk_layers = mkl; c->mk_bar = mkb; c->mk_abort = mka; c->mk_attn_o = mkao; c->mk_act = mkact; c->mk_trace = mkt;
         c->part_o = po; c->part_ml = pml;
     }
     return align_up(w.off, 256);
@@ -272,7 +278,8 @@ GvPlan plan_gemv(const sparsk_ctx *c, int n_groups, int K)
 template <class Op, int R, int M, bool NORM>
 cudaError_t launch_gemv_inst(sparsk_ctx *c, const Op &op, GvIn in, int n_groups)
 {
-    static bool attr_set = false;
+    static PerDevice<bool> attr_done;
+    bool &attr_set = attr_done.here();
     auto kern = gemv_kernel<Op, R, M, NORM>;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
@@ -307,6 +314,7 @@ struct RowSet {
     int max_grp_rows;
     int max_len;    // longest prefix any row attends to (host)
     int n_big;      // groups with at least attn_tc_min_q query vectors per kv head (0: not counted, assume all)
+    const float *q; // the rows' queries if they are not the context's query buffer (NULL: they are)
 };
 
 cudaError_t run_qkv(sparsk_ctx *c, int layer, const float *h, const RowSet &rs)
@@ -413,7 +421,7 @@ cudaError_t run_attn(sparsk_ctx *c, int layer, const RowSet &rs)
     const size_t lstride = (size_t)d.max_seqs * d.n_kv_heads * d.max_seq_len * d.head_dim;
     AttnArgs a{};
     a.q = nullptr;
-    a.q32 = c->qbuf;
+    a.q32 = rs.q ? rs.q : c->qbuf;
     a.kc = c->kcache + (layer - 1) * lstride;
     a.vc = c->vcache + (layer - 1) * lstride;
     a.grp_row0 = rs.grp_row0; a.grp_nrows = rs.grp_nrows; a.row_slot = rs.slot; a.row_pos = rs.pos;
@@ -436,7 +444,8 @@ cudaError_t run_attn(sparsk_ctx *c, int layer, const RowSet &rs)
         // of 64 positions), the others to the mma.sync kernel; both launches cover all groups, a CTA
         // leaves at once if its group belongs to the other, and both use one split plan so that the
         // merge finds every partial where it expects it.
-        static bool ready = false;
+        static PerDevice<bool> ready_dev;
+        bool &ready = ready_dev.here();
         if (!ready) {
             if ((e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TA_SMEM)) != cudaSuccess) return e;
             ready = true;
@@ -504,7 +513,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 // Descriptors of a row-major bf16 matrix [rows][cols], 128-byte swizzle, zero fill outside:
 // m2 reads boxes of [box_rows][64]; m3 (only when cols is a multiple of 64) views the matrix as
 // [64][rows][cols/64] and reads [box_rows] rows of two consecutive 64-element blocks at once.
-bool encode_maps(EncodeTiledFn fn, TmaPair *m, const void *base, size_t rows, size_t cols, int box_rows)
+bool encode_maps(EncodeTiledFn fn, TmaPair *m, const void *base, size_t rows, size_t cols, int box_rows,
+                 CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16)
 {
     memset(m, 0, sizeof *m);
     if (!base) return true;
@@ -513,7 +523,7 @@ bool encode_maps(EncodeTiledFn fn, TmaPair *m, const void *base, size_t rows, si
         const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
         const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
         const cuuint32_t box[2] = {(cuuint32_t)GM_BK, (cuuint32_t)box_rows};
-        if (fn(&m->m2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, es,
+        if (fn(&m->m2, dtype, 2, const_cast<void *>(base), dims, strides, box, es,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return false;
@@ -522,7 +532,7 @@ bool encode_maps(EncodeTiledFn fn, TmaPair *m, const void *base, size_t rows, si
         const cuuint64_t dims[3] = {(cuuint64_t)GM_BK, (cuuint64_t)rows, (cuuint64_t)(cols / GM_BK)};
         const cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)GM_BK * 2};
         const cuuint32_t box[3] = {(cuuint32_t)GM_BK, (cuuint32_t)box_rows, 2};
-        if (fn(&m->m3, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, es,
+        if (fn(&m->m3, dtype, 3, const_cast<void *>(base), dims, strides, box, es,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return false;
@@ -556,9 +566,11 @@ bool build_maps(sparsk_ctx *c)
         c->tm_vc.resize(L);
         for (int l = 0; l < L && ok; l++) {
             TmaPair t;
-            ok = ok && encode_maps(fn, &t, c->kcache + l * lstride, (size_t)d.max_seqs * d.n_kv_heads * d.max_seq_len, d.head_dim, TA_NT);
+            ok = ok && encode_maps(fn, &t, c->kcache + l * lstride, (size_t)d.max_seqs * d.n_kv_heads * d.max_seq_len, d.head_dim, TA_NT,
+                                   CU_TENSOR_MAP_DATA_TYPE_FLOAT16);
             c->tm_kc[l] = t.m3;
-            ok = ok && encode_maps(fn, &t, c->vcache + l * lstride, (size_t)d.max_seqs * d.n_kv_heads * d.max_seq_len, d.head_dim, TA_NT);
+            ok = ok && encode_maps(fn, &t, c->vcache + l * lstride, (size_t)d.max_seqs * d.n_kv_heads * d.max_seq_len, d.head_dim, TA_NT,
+                                   CU_TENSOR_MAP_DATA_TYPE_FLOAT16);
             c->tm_vc[l] = t.m3;
         }
     }
@@ -585,7 +597,8 @@ template <class Epi>
 cudaError_t launch_gemm(sparsk_ctx *c, const TmaPair &a0, const TmaPair &a1, const TmaPair &a2, const TmaPair *b_maps,
                         const TmaPair *b_lo_maps, GemmArgs g, const Epi &epi)
 {
-    static bool attr_set = false;
+    static PerDevice<bool> attr_done;
+    bool &attr_set = attr_done.here();
     constexpr int SMEM_BUDGET = 220 * 1024;
     auto kern = wsgemm_kernel<Epi>;
     if (!attr_set) {
@@ -595,20 +608,27 @@ cudaError_t launch_gemm(sparsk_ctx *c, const TmaPair &a0, const TmaPair &a1, con
     }
     const int bi = box_index(g.m_rows);
     g.box_n = 16 << bi;
-    const int room = SMEM_BUDGET - 1024 - GM_XCHG_BYTES;
+    // the ring may be told to stay small enough for two CTAs (of this kernel or of the next one in
+    // the stream) to share an SM, so that one's ending overlaps the other's first copies; rows
+    // that do not fit such a ring take the whole SM
     auto stage_bytes = [&](int kb) { return 2 * kb * GM_BLK_BYTES + 2 * kb * g.box_n * GM_BK * 2; };
-    // two k-blocks per copy whenever the inner dimension allows the 3-D view and two stages fit
-    g.three_d = (g.K % GM_BK == 0) && 2 * stage_bytes(2) <= room && c->tc_kb != 1;
-    g.kb = g.three_d ? 2 : 1;
-    g.stages = std::min(GM_MAX_STAGES, room / stage_bytes(g.kb));
-    if (g.stages < 2) return cudaErrorInvalidValue;
+    auto plan = [&](int budget) {
+        const int room = budget - 1024 - GM_XCHG_BYTES;
+        // two k-blocks per copy whenever the inner dimension allows the 3-D view and two stages fit
+        g.three_d = (g.K % GM_BK == 0) && 2 * stage_bytes(2) <= room && c->tc_kb != 1;
+        g.kb = g.three_d ? 2 : 1;
+        g.stages = std::min(GM_MAX_STAGES, room / stage_bytes(g.kb));
+        return g.stages >= 2;
+    };
+    if (!plan(std::min(SMEM_BUDGET, c->gemm_smem_kb * 1024)) && !plan(SMEM_BUDGET)) return cudaErrorInvalidValue;
     g.status = c->sd.counts + CNT_STATUS;
     const int n_units = g.units[0] + (g.pair ? 0 : g.units[1] + g.units[2]);
     const int k_stages = ((g.K + GM_BK - 1) / GM_BK + g.kb - 1) / g.kb;
     g.splits = std::max(1, std::min(g.splits, k_stages));
-    const int grid_x = std::max(1, std::min(c->n_sm, n_units * g.splits));
-    const int grid_y = (g.m_rows + GM_MAX_N - 1) / GM_MAX_N;
     const size_t smem = 1024 + (size_t)g.stages * stage_bytes(g.kb) + GM_XCHG_BYTES;
+    const int per_sm = (smem + 1024) * 2 <= 227 * 1024 ? std::max(1, c->gemm_cps) : 1;  // CTAs of this launch that fit an SM
+    const int grid_x = std::max(1, std::min(c->n_sm * per_sm, n_units * g.splits));
+    const int grid_y = (g.m_rows + GM_MAX_N - 1) / GM_MAX_N;
     if (g.three_d)
         return launch(c, kern, dim3(grid_x, grid_y), dim3(GM_THREADS), smem, a0.m3, a1.m3, a2.m3, b_maps[bi].m3,
                       b_lo_maps[bi].m3, g, epi);
@@ -625,16 +645,22 @@ cudaError_t run_norm(sparsk_ctx *c, const float *h, const bf16 *gain, const int 
 }
 
 // How many cuts of the inner dimension fill the machine when a product has `units` units.
-int splits_for(const sparsk_ctx *c, int units) { return units * 2 <= c->n_sm ? c->n_sm / units : 1; }
+int splits_for(const sparsk_ctx *c, int units)
+{
+    const int ctas = c->n_sm * std::max(1, c->gemm_cps);
+    return units * 2 <= ctas ? ctas / units : 1;
+}
 
-// One transformer layer over a row set on the tensor-core path.
-cudaError_t run_layer_tc(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
+// One transformer layer over a row set on the tensor-core path, in two halves: the front
+// (RMSNorm, q/k/v projection, rotary embedding, cache append) and the back (attention,
+// O-projection, MLP).  The last layer of an upper pass runs its back half on fewer rows.
+cudaError_t run_layer_tc_front(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
 {
     const sparsk_dims &d = c->dm;
     const int li = layer - 1, M = rs.n_rows;
     const int qd = d.n_q_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim;
     const size_t lstride = (size_t)d.max_seqs * d.n_kv_heads * d.max_seq_len * d.head_dim;
-    bf16 *kc = c->kcache + li * lstride, *vc = c->vcache + li * lstride;
+    kv_t *kc = c->kcache + li * lstride, *vc = c->vcache + li * lstride;
     cudaError_t e;
     c->cur_class = KC_MISC;
     if ((e = run_norm(c, h, c->attn_norm[li], nullptr, M)) != cudaSuccess) return e;
@@ -654,6 +680,16 @@ cudaError_t run_layer_tc(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
                         rs.slot, rs.pos, M, d.n_q_heads, d.n_kv_heads, d.head_dim, d.max_seq_len)) != cudaSuccess)
             return e;
     }
+    c->cur_class = KC_MISC;
+    return cudaSuccess;
+}
+
+cudaError_t run_layer_tc_back(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
+{
+    const sparsk_dims &d = c->dm;
+    const int li = layer - 1, M = rs.n_rows;
+    const int qd = d.n_q_heads * d.head_dim;
+    cudaError_t e;
     c->cur_class = KC_ATTN;
     if ((e = run_attn(c, layer, rs)) != cudaSuccess) return e;
     {
@@ -775,17 +811,18 @@ bool use_mega(const sparsk_ctx *c, int n_rows)
 template <int M, int HD>
 cudaError_t launch_mega_inst(sparsk_ctx *c, const MkArgs &a, size_t smem)
 {
-    static int grid_ok = -1;
+    static PerDevice<int> grid_dev;  // 0: not asked yet, 1: one CTA per SM fits, 2: it does not
+    int &grid_ok = grid_dev.here();
     auto kern = mega_kernel<M, HD>;
-    if (grid_ok < 0) {
+    if (grid_ok == 0) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         int per_sm = 0;
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, MK_THREADS, smem);
         if (e != cudaSuccess) return e;
-        grid_ok = per_sm >= 1 ? 1 : 0;
+        grid_ok = per_sm >= 1 ? 1 : 2;
     }
-    if (!grid_ok) return cudaErrorCooperativeLaunchTooLarge;
+    if (grid_ok != 1) return cudaErrorCooperativeLaunchTooLarge;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3(c->n_sm);
@@ -832,6 +869,12 @@ cudaError_t run_mega(sparsk_ctx *c, int l_begin, int l_end, float *h, const RowS
     a.att_split_len = ((rs.max_len + splits - 1) / splits + AT_TP - 1) / AT_TP * AT_TP;
     a.att_splits = std::max(1, (rs.max_len + a.att_split_len - 1) / a.att_split_len);
     a.bar = c->mk_bar; a.bar_base = c->mk_bar_base; a.abort_word = c->mk_abort; a.status = c->sd.counts + CNT_STATUS;
+    if (c->inject_timeout) {
+        // the launch is told a barrier count that is never reached: its first grid barrier runs
+        // into the wall-clock limit, every CTA gives up and the step reports SPARSK_ETIMEOUT
+        a.bar_base += 1ull << 40;
+        c->inject_timeout = 0;
+    }
     a.trace = c->mk_trace;
     c->mk_trace_n = 1 + 6 * (l_end - l_begin);
     c->mk_bar_base += 6ull * (unsigned long long)(l_end - l_begin) * (unsigned long long)c->n_sm;
@@ -852,124 +895,23 @@ cudaError_t run_mega(sparsk_ctx *c, int l_begin, int l_end, float *h, const RowS
     }
 }
 
-// ---------------------------------------------------------------- persistent tcgen05 layer-range kernel
-bool build_tcmega(sparsk_ctx *c)
+// Front half of a layer over a row set: q to the query buffer, k and v into the cache.
+cudaError_t run_layer_front(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
 {
-    const sparsk_dims &d = c->dm;
-    const size_t lstride = (size_t)d.max_seqs * d.n_kv_heads * d.max_seq_len * d.head_dim;
-    std::vector<TkLayer> host(d.n_layers);
-    for (int l = 0; l < d.n_layers; l++) {
-        TkLayer &t = host[l];
-        memset(&t, 0, sizeof t);
-        t.wq = c->tm_wq[l].m2; t.wk = c->tm_wk[l].m2; t.wv = c->tm_wv[l].m2; t.wo = c->tm_wo[l].m2;
-        t.wg = c->tm_wg[l].m2; t.wu = c->tm_wu[l].m2; t.wd = c->tm_wd[l].m2;
-        t.attn_gain = c->attn_norm[l];
-        t.mlp_gain = c->mlp_norm[l];
-        t.kc = c->kcache + l * lstride;
-        t.vc = c->vcache + l * lstride;
-    }
-    // pageable source: the copy has left the host buffer when the call returns
-    return cudaMemcpyAsync(c->tk_layers, host.data(), sizeof(TkLayer) * d.n_layers, cudaMemcpyHostToDevice, c->stream) ==
-           cudaSuccess;
-}
-
-size_t tk_attn_bytes(int head_dim, int mt)
-{
-    const size_t kp = head_dim + 8;
-    const size_t q = (size_t)2 * 16 * mt * kp * 2, ring = (size_t)4 * 2 * 2 * AT_TP * kp * 2;
-    const size_t merge = (size_t)4 * 16 * mt * (head_dim + 2) * 4;
-    return q + std::max(ring, merge);
-}
-
-// Can a pass over this row set go through the persistent tcgen05 kernel?
-bool use_tcmega(const sparsk_ctx *c, const RowSet &rs)
-{
-    const sparsk_dims &d = c->dm;
-    return c->tcmega && c->tk_ok && c->tc_ok && c->mk_coop && rs.n_rows >= c->gemm_min_rows && rs.n_rows <= TK_MAX_N &&
-           d.d_model >= GM_BK && tk_attn_bytes(d.head_dim, 2) <= (size_t)TK_ATT_BYTES;
-}
-
-template <int HD>
-cudaError_t launch_tcmega_inst(sparsk_ctx *c, const TkArgs &a)
-{
-    static int grid_ok = -1;
-    auto kern = tcmega_kernel<HD>;
-    if (grid_ok < 0) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TK_SMEM);
-        if (e != cudaSuccess) return e;
-        int per_sm = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, TK_THREADS, TK_SMEM);
-        if (e != cudaSuccess) return e;
-        grid_ok = per_sm >= 1 ? 1 : 0;
-    }
-    if (!grid_ok) return cudaErrorCooperativeLaunchTooLarge;
-    cudaLaunchConfig_t cfg;
-    memset(&cfg, 0, sizeof cfg);
-    cfg.gridDim = dim3(c->n_sm);
-    cfg.blockDim = dim3(TK_THREADS);
-    cfg.dynamicSmemBytes = TK_SMEM;
-    cfg.stream = c->stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeCooperative;
-    attr[0].val.cooperative = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    c->launches++;
-    const bool timed = (c->time_class == KC_MEGA || c->time_class == KC_ALL) && c->tev_used + 2 <= c->tev.size();
-    if (timed) {
-        c->tev_class[c->tev_used / 2] = KC_MEGA;
-        cudaEventRecord(c->tev[c->tev_used++], c->stream);
-    }
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, a);
-    if (timed) cudaEventRecord(c->tev[c->tev_used++], c->stream);
+    if (use_tc(c, rs.n_rows)) return run_layer_tc_front(c, layer, h, rs);
+    c->cur_class = KC_QKV;
+    const cudaError_t e = run_qkv(c, layer, h, rs);
+    c->cur_class = KC_MISC;
     return e;
 }
 
-// Layers [l_begin, l_end) (0-based) over a row set of 3..TK_MAX_N rows, in one launch.
-cudaError_t run_tcmega(sparsk_ctx *c, int l_begin, int l_end, float *h, const RowSet &rs)
-{
-    const sparsk_dims &d = c->dm;
-    const int qd = d.n_q_heads * d.head_dim, kd = d.n_kv_heads * d.head_dim, G = d.n_q_heads / d.n_kv_heads;
-    TkArgs a;
-    memset(&a, 0, sizeof a);
-    const int bi = box_index(rs.n_rows);
-    a.box_n = 16 << bi;
-    a.x_hi = c->tm_x[bi].m2; a.x_lo = c->tm_x_lo[bi].m2; a.ao_hi = c->tm_ao[bi].m2; a.ao_lo = c->tm_ao_lo[bi].m2;
-    a.act_hi = c->tm_act[bi].m2; a.act_lo = c->tm_act_lo[bi].m2;
-    a.layers = c->tk_layers; a.layer_begin = l_begin; a.layer_end = l_end; a.h = h;
-    a.row_slot = rs.slot; a.row_pos = rs.pos; a.grp_row0 = rs.grp_row0; a.grp_nrows = rs.grp_nrows;
-    a.n_groups_dev = rs.n_groups;
-    a.m_rows = rs.n_rows;
-    a.q32 = c->qbuf; a.qkv_part = c->qkv_part;
-    a.x_hi_p = c->xnorm; a.x_lo_p = c->xnorm_lo; a.ao_hi_p = c->attn_o; a.ao_lo_p = c->attn_o_lo;
-    a.act_hi_p = c->act; a.act_lo_p = c->act_lo;
-    a.part_o = c->part_o; a.part_ml = c->part_ml; a.rope = c->rope;
-    a.d = d.d_model; a.Hq = d.n_q_heads; a.Hkv = d.n_kv_heads; a.hd = d.head_dim; a.F = d.d_ffn; a.S = d.max_seq_len;
-    a.n_slots = d.max_seqs; a.eps = d.rms_eps;
-    // every cut of an inner dimension holds at least one k-block
-    auto cuts = [&](int units, int K) { return std::max(1, std::min(splits_for(c, units), div_up(K, GM_BK))); };
-    a.splits_qkv = cuts(div_up(qd, 2 * GM_BM) + 2 * div_up(kd, 2 * GM_BM), d.d_model);
-    a.splits_o = cuts(div_up(d.d_model, 2 * GM_BM), qd);
-    a.splits_down = cuts(div_up(d.d_model, 2 * GM_BM), d.d_ffn);
-    const AttnPlan pl = attn_plan(c->n_sm, rs.n_groups_h, rs.max_grp_rows, G, d.n_kv_heads, rs.max_len, c->attn_split);
-    a.att_groups = rs.n_groups_h; a.att_qblk = pl.n_qblk; a.att_splits = pl.n_splits; a.att_split_len = pl.split_len;
-    a.att_mt = pl.mt;
-    a.bar = c->mk_bar; a.bar_base = c->mk_bar_base; a.abort_word = c->mk_abort; a.status = c->sd.counts + CNT_STATUS;
-    c->mk_bar_base += (unsigned long long)TK_PHASES * (unsigned long long)(l_end - l_begin) * (unsigned long long)c->n_sm;
-    a.trace = c->mk_trace;
-    c->mk_trace_n = 1 + TK_PHASES * (l_end - l_begin);
-    return d.head_dim == 128 ? launch_tcmega_inst<128>(c, a) : launch_tcmega_inst<64>(c, a);
-}
-
-// One transformer layer over a row set: h <- h^(layer).
-cudaError_t run_layer(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
+// Back half: attention, O-projection and MLP; h <- h^(layer).
+cudaError_t run_layer_back(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
 {
     const sparsk_dims &d = c->dm;
     const int li = layer - 1;
     cudaError_t e;
-    if (use_tc(c, rs.n_rows)) return run_layer_tc(c, layer, h, rs);
-    c->cur_class = KC_QKV;
-    if ((e = run_qkv(c, layer, h, rs)) != cudaSuccess) return e;
+    if (use_tc(c, rs.n_rows)) return run_layer_tc_back(c, layer, h, rs);
     c->cur_class = KC_ATTN;
     if ((e = run_attn(c, layer, rs)) != cudaSuccess) return e;
     c->cur_class = KC_OPROJ;
@@ -982,12 +924,23 @@ cudaError_t run_layer(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
     return e;
 }
 
+// One transformer layer over a row set: h <- h^(layer).
+cudaError_t run_layer(sparsk_ctx *c, int layer, float *h, const RowSet &rs)
+{
+    const cudaError_t e = run_layer_front(c, layer, h, rs);
+    return e != cudaSuccess ? e : run_layer_back(c, layer, h, rs);
+}
+
 // Layers l_first..l_last (1-based, inclusive) over a row set.
 cudaError_t run_layers(sparsk_ctx *c, int l_first, int l_last, float *h, const RowSet &rs)
 {
     if (l_first > l_last) return cudaSuccess;
-    if (use_mega(c, rs.n_rows)) return run_mega(c, l_first - 1, l_last, h, rs);
-    if (use_tcmega(c, rs)) return run_tcmega(c, l_first - 1, l_last, h, rs);
+    const int n_layers = l_last - l_first + 1;
+    if (use_mega(c, rs.n_rows)) {
+        c->route_layers[0] += n_layers;
+        return run_mega(c, l_first - 1, l_last, h, rs);
+    }
+    c->route_layers[use_tc(c, rs.n_rows) ? 1 : 2] += n_layers;
     for (int l = l_first; l <= l_last; l++) {
         const cudaError_t e = run_layer(c, l, h, rs);
         if (e != cudaSuccess) return e;
@@ -1049,14 +1002,18 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
     carve(ctx, &ctx->dm, (char *)workspace);
     ctx->h_len.assign(dims->max_seqs, 0);
     ctx->h_pend.assign(dims->max_seqs, 0);
-    ctx->pdl = 1; ctx->attn_split = 0; ctx->gemm_min_rows = 3; ctx->use_graph = 0;
+    ctx->pdl = 1; ctx->attn_split = 0; ctx->gemm_min_rows = 3;
     ctx->tc_ok = false;
     ctx->tc_kb = 0;
+    ctx->gemm_smem_kb = 220;
+    ctx->gemm_cps = 1;
     ctx->mk_max_rows = 2;
-    ctx->tcmega = 0; ctx->tk_ok = 0;
     ctx->attn_tc = 1; ctx->attn_tc_min_q = 33;
+    ctx->inject_timeout = 0;
+    ctx->trim_last = 1;
+    for (auto &v : ctx->route_layers) v = 0;
     ctx->mega = 1; ctx->mk_ok = 0; ctx->mk_coop = 0; ctx->mk_bar_base = 0; ctx->mk_trace_n = 0;
-    ctx->gv_ks = 0; ctx->gv_r = 0; ctx->gv_grid_mult = 1;
+    ctx->gv_ks = 0; ctx->gv_r = 0;
     ctx->dbg_hidden = nullptr; ctx->dbg_logits = nullptr;
     ctx->samp_temperature = 0.f; ctx->samp_top_p = 1.f; ctx->samp_uniforms = nullptr; ctx->samp_scratch = nullptr;
     ctx->launches = 0;
@@ -1090,11 +1047,6 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
             rc = fail(ctx, SPARSK_ECUDA, "setting up the persistent layer kernel failed");
             break;
         }
-        ctx->tk_ok = build_tcmega(ctx) ? 1 : 0;
-        if (!ctx->tk_ok) {
-            rc = fail(ctx, SPARSK_ECUDA, "setting up the persistent tensor-core layer kernel failed");
-            break;
-        }
         // rotary table in double, stored as float (cos, sin)
         const int half = dims->head_dim / 2;
         std::vector<float2> tab((size_t)dims->max_seq_len * half);
@@ -1108,8 +1060,8 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
         if ((ce = cudaMemcpyAsync(ctx->rope, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice, ctx->stream)) != cudaSuccess ||
             // the cache starts out as zeros: the tcgen05 attention kernel multiplies whole 64-position
             // tiles, and a masked weight of zero times an unwritten NaN pattern would still be NaN
-            (ce = cudaMemsetAsync(ctx->kcache, 0, sizeof(bf16) * (size_t)dims->n_layers * dims->max_seqs * dims->n_kv_heads * dims->max_seq_len * dims->head_dim, ctx->stream)) != cudaSuccess ||
-            (ce = cudaMemsetAsync(ctx->vcache, 0, sizeof(bf16) * (size_t)dims->n_layers * dims->max_seqs * dims->n_kv_heads * dims->max_seq_len * dims->head_dim, ctx->stream)) != cudaSuccess ||
+            (ce = cudaMemsetAsync(ctx->kcache, 0, sizeof(kv_t) * (size_t)dims->n_layers * dims->max_seqs * dims->n_kv_heads * dims->max_seq_len * dims->head_dim, ctx->stream)) != cudaSuccess ||
+            (ce = cudaMemsetAsync(ctx->vcache, 0, sizeof(kv_t) * (size_t)dims->n_layers * dims->max_seqs * dims->n_kv_heads * dims->max_seq_len * dims->head_dim, ctx->stream)) != cudaSuccess ||
             (ce = cudaMemsetAsync(ctx->kv_len, 0, sizeof(int) * dims->max_seqs, ctx->stream)) != cudaSuccess ||
             (ce = cudaMemsetAsync(ctx->pend_cnt, 0, sizeof(int) * dims->max_seqs, ctx->stream)) != cudaSuccess ||
             (ce = cudaMemsetAsync(ctx->sd.counts, 0, sizeof(int) * 8, ctx->stream)) != cudaSuccess ||
@@ -1143,6 +1095,13 @@ extern "C" int sparsk_destroy(sparsk_ctx *ctx)
 
 extern "C" const char *sparsk_last_error(const sparsk_ctx *ctx) { return good(ctx) ? ctx->err : "invalid context"; }
 extern "C" int64_t sparsk_launch_count(const sparsk_ctx *ctx) { return good(ctx) ? ctx->launches : -1; }
+extern "C" int sparsk_route_counts(const sparsk_ctx *ctx, int64_t *layer_passes)
+{
+    if (!good(ctx)) return SPARSK_ESTATE;
+    if (!layer_passes) return SPARSK_EINVAL;
+    for (int i = 0; i < 3; i++) layer_passes[i] = ctx->route_layers[i];
+    return SPARSK_OK;
+}
 
 extern "C" int sparsk_set_debug(sparsk_ctx *ctx, float *exit_hidden, float *exit_logits)
 {
@@ -1186,16 +1145,18 @@ extern "C" int sparsk_set_option(sparsk_ctx *ctx, const char *name, int64_t valu
     if (!good(ctx)) return SPARSK_ESTATE;
     if (!name) return fail(ctx, SPARSK_EINVAL, "option name is NULL");
     if (!strcmp(name, "gemm_min_rows") && value >= 1) ctx->gemm_min_rows = (int)std::min<int64_t>(value, 1 << 30);
-    else if (!strcmp(name, "use_graph") && (value == 0 || value == 1)) ctx->use_graph = (int)value;
     else if (!strcmp(name, "pdl") && (value == 0 || value == 1)) ctx->pdl = (int)value;
     else if (!strcmp(name, "attn_split") && value >= 0 && value <= (1 << 24)) ctx->attn_split = (int)value;
     else if (!strcmp(name, "gemv_ks") && (value == 0 || value == 1 || value == 2 || value == 4 || value == 8 || value == 16)) ctx->gv_ks = (int)value;
     else if (!strcmp(name, "mega") && (value == 0 || value == 1)) ctx->mega = (int)value;
-    else if (!strcmp(name, "tcmega") && (value == 0 || value == 1)) ctx->tcmega = (int)value;
     else if (!strcmp(name, "attn_tc") && (value == 0 || value == 1)) ctx->attn_tc = (int)value;
     else if (!strcmp(name, "attn_tc_min_q") && value >= 1 && value <= (1 << 20)) ctx->attn_tc_min_q = (int)value;
     else if (!strcmp(name, "mega_max_rows") && value >= 1 && value <= MK_MAX_ROWS) ctx->mk_max_rows = (int)value;
     else if (!strcmp(name, "gemm_kb") && (value == 0 || value == 1)) ctx->tc_kb = (int)value;
+    else if (!strcmp(name, "gemm_ctas_per_sm") && (value == 1 || value == 2)) ctx->gemm_cps = (int)value;
+    else if (!strcmp(name, "gemm_smem_kb") && value >= 48 && value <= 220) ctx->gemm_smem_kb = (int)value;
+    else if (!strcmp(name, "trim_last_layer") && value >= 0 && value <= 2) ctx->trim_last = (int)value;
+    else if (!strcmp(name, "inject_barrier_timeout") && (value == 0 || value == 1)) ctx->inject_timeout = (int)value;
     else if (!strcmp(name, "gemv_r") && (value == 0 || value == 1 || value == 2 || value == 4)) ctx->gv_r = (int)value;
     else if (!strcmp(name, "time_kernel") && value >= 0 && value <= KC_ALL) {
         // start (or stop, with 0) timing every launch of one kernel class; resets the totals
@@ -1226,15 +1187,17 @@ extern "C" int sparsk_kernel_time(sparsk_ctx *ctx, double *total_ms, int64_t *n_
     return SPARSK_OK;
 }
 
-extern "C" int sparsk_check(sparsk_ctx *ctx)
+// Reads and clears the device status word (the stream is synchronised) and turns it into a
+// return code.  After a timeout the persistent kernels' grid-barrier counter, its host mirror and
+// the abort word start over, so that the next launch does not find a stale abort request or a
+// counter that no longer matches its base.
+static int read_status(sparsk_ctx *ctx)
 {
-    if (!good(ctx)) return SPARSK_ESTATE;
     int status = 0;
     CU(cudaMemcpyAsync(&status, ctx->sd.counts + CNT_STATUS, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
     CU(cudaStreamSynchronize(ctx->stream));
     if (status) CU(cudaMemsetAsync(ctx->sd.counts + CNT_STATUS, 0, sizeof(int), ctx->stream));
     if (status & ST_TIMEOUT) {
-        // the persistent kernel's barrier counter and abort word start over
         CU(cudaMemsetAsync(ctx->mk_bar, 0, sizeof(unsigned long long), ctx->stream));
         CU(cudaMemsetAsync(ctx->mk_abort, 0, sizeof(int), ctx->stream));
         ctx->mk_bar_base = 0;
@@ -1242,6 +1205,12 @@ extern "C" int sparsk_check(sparsk_ctx *ctx)
     }
     if (status & ST_BAD_TOKEN) return fail(ctx, SPARSK_EINVAL, "a token id was outside the vocabulary (clamped)");
     return SPARSK_OK;
+}
+
+extern "C" int sparsk_check(sparsk_ctx *ctx)
+{
+    if (!good(ctx)) return SPARSK_ESTATE;
+    return read_status(ctx);
 }
 
 extern "C" int sparsk_kernel_time_by_class(sparsk_ctx *ctx, double *total_ms, int64_t *n_launches)
@@ -1308,8 +1277,8 @@ static int kv_io(sparsk_ctx *ctx, int32_t slot, int32_t layer, int32_t first_pos
     const size_t off = ((size_t)(layer - 1) * d.max_seqs + slot) * per_slot;
     const size_t total = (size_t)n * d.n_kv_heads * d.head_dim;
     const int blocks = (int)std::min<size_t>((total + 255) / 256, 4096);
-    CU(launch(ctx, kv_copy_kernel, dim3(blocks), dim3(256), 0, ctx->kcache + off, ctx->vcache + off, (bf16 *)k,
-              (bf16 *)v, (int)first_pos, (int)n, d.n_kv_heads, d.head_dim, d.max_seq_len, to_cache));
+    CU(launch(ctx, kv_copy_kernel, dim3(blocks), dim3(256), 0, ctx->kcache + off, ctx->vcache + off, (kv_t *)k,
+              (kv_t *)v, (int)first_pos, (int)n, d.n_kv_heads, d.head_dim, d.max_seq_len, to_cache));
     return SPARSK_OK;
 }
 extern "C" int sparsk_import_kv(sparsk_ctx *ctx, int32_t slot, int32_t layer, int32_t first_pos, int32_t n,
@@ -1371,7 +1340,9 @@ extern "C" int sparsk_decode_step(sparsk_ctx *ctx, int32_t n, const int32_t *slo
 {
     if (!good(ctx)) return SPARSK_ESTATE;
     const sparsk_dims &d = ctx->dm;
-    const int L = d.n_layers, e = d.exit_layer, K = d.refresh_period, r = d.refresh_phase, B = d.max_seqs;
+    const int L = d.n_layers, e = d.exit_layer, B = d.max_seqs;
+    const SchedParams sp{L, e, d.refresh_period, d.refresh_phase, d.text_period > 0 ? d.text_period : d.refresh_period,
+                         d.text_period > 0 ? d.text_phase : d.refresh_phase, d.text_exit};
     if (n < 1 || n > B || !slots || !token_ids || !modality || !counters || !next_tokens || !exit_depths)
         return fail(ctx, SPARSK_EINVAL, "decode_step: bad arguments (n=%d)", n);
     // ---- host mirror of the schedule: validates, and sizes the launches
@@ -1386,7 +1357,7 @@ extern "C" int sparsk_decode_step(sparsk_ctx *ctx, int32_t n, const int32_t *slo
         if (modality[i] > 1) return fail(ctx, SPARSK_EINVAL, "decode_step: modality[%d]=%d", i, modality[i]);
         if (counters[i] < 0) return fail(ctx, SPARSK_EINVAL, "decode_step: counter[%d]=%d", i, counters[i]);
         if (ctx->h_len[s] + 1 > d.max_seq_len) return fail(ctx, SPARSK_ECAPACITY, "decode_step: slot %d is full (%d positions)", s, ctx->h_len[s]);
-        const int depth = scheduled_depth(modality[i], counters[i], K, r, e, L, d.text_exit);
+        const int depth = scheduled_depth(modality[i], counters[i], sp);
         const bool full = depth == L;
         if (!full && ctx->h_pend[s] + 1 > d.max_pending)
             return fail(ctx, SPARSK_ECAPACITY, "decode_step: slot %d would hold %d pending positions (max_pending %d)", s, ctx->h_pend[s] + 1, d.max_pending);
@@ -1420,7 +1391,7 @@ extern "C" int sparsk_decode_step(sparsk_ctx *ctx, int32_t n, const int32_t *slo
     // ---- schedule, compaction, embedding
     const int V = d.vocab_text + d.vocab_speech;
     CU(launch(ctx, schedule_kernel, dim3((n + 127) / 128), dim3(128), 0, ctx->sd, (int)n, (const int *)ctx->staged,
-              (const int *)token_ids, V, L, e, K, r, d.text_exit));
+              (const int *)token_ids, V, sp));
     CU(launch(ctx, compact_kernel, dim3(1), dim3(1024), 0, ctx->sd, (int)n, (const int *)ctx->kv_len,
               (const int *)ctx->pend_cnt, L, e, B));
     CU(launch(ctx, embed_kernel, dim3(n), dim3(128), 0, (const int *)ctx->sd.token, ctx->embed, ctx->h_lo, (int)n, d.d_model,
@@ -1447,7 +1418,28 @@ extern "C" int sparsk_decode_step(sparsk_ctx *ctx, int32_t n, const int32_t *slo
                   (const float *)ctx->pend_h, ctx->h_up, d.d_model, d.max_pending));
         RowSet up{ctx->sd.up_slot, ctx->sd.up_pos, ctx->sd.up_grp_row0, ctx->sd.up_grp_nrows, ctx->sd.counts + CNT_NGRP,
                   ctx->sd.counts + CNT_MUP, m_up, n_grp, max_grp, max_len_up, n_big};
-        CU(run_layers(ctx, e + 1, L, ctx->h_up, up));
+        // Layer L gives the pending rows nothing but their K/V: nothing reads their h^(L).  When the
+        // step has pending rows and the rest of the layer is cheaper on one row per sequence
+        // (attention over long prefixes, projections with enough rows to be tensor-bound), the
+        // layer's back half runs on the current rows alone.
+        const int qd = d.n_q_heads * d.head_dim;
+        const bool persistent = use_mega(ctx, m_up);
+        const bool trim = m_up > n_grp && !persistent &&
+                          (ctx->trim_last == 2 || (ctx->trim_last == 1 && use_tc(ctx, n_grp)));
+        if (!trim) {
+            CU(run_layers(ctx, e + 1, L, ctx->h_up, up));
+        } else {
+            CU(run_layers(ctx, e + 1, L - 1, ctx->h_up, up));
+            ctx->route_layers[use_tc(ctx, m_up) ? 1 : 2] += 1;
+            CU(run_layer_front(ctx, L, ctx->h_up, up));
+            CU(launch(ctx, take_current_kernel, dim3(n_grp), dim3(256), 0, ctx->sd, (const float *)ctx->h_up,
+                      (const float *)ctx->qbuf, ctx->h_last, ctx->q_last, ctx->last_slot, ctx->last_pos, d.d_model, qd));
+            RowSet last{ctx->last_slot, ctx->last_pos, ctx->sd.lo_grp_row0, ctx->sd.lo_grp_nrows, ctx->sd.counts + CNT_NGRP,
+                        ctx->sd.counts + CNT_NGRP, n_grp, n_grp, 1, max_len_up, 0, ctx->q_last};
+            CU(run_layer_back(ctx, L, ctx->h_last, last));
+            CU(launch(ctx, put_current_kernel, dim3(n_grp), dim3(256), 0, ctx->sd, (const float *)ctx->h_last, ctx->h_up,
+                      d.d_model));
+        }
         h_full = ctx->h_up;
     }
     for (int l = 2; l < 4; l++)
@@ -1476,7 +1468,7 @@ extern "C" int sparsk_decode_step(sparsk_ctx *ctx, int32_t n, const int32_t *slo
     // ---- host mirror follows
     for (int i = 0; i < n; i++) {
         const int s = slots[i];
-        const int depth = scheduled_depth(modality[i], counters[i], K, r, e, L, d.text_exit);
+        const int depth = scheduled_depth(modality[i], counters[i], sp);
         ctx->h_len[s] += 1;
         ctx->h_pend[s] = (depth == L) ? 0 : ctx->h_pend[s] + 1;
     }
@@ -1490,16 +1482,16 @@ extern "C" int sparsk_decode_step_host(sparsk_ctx *ctx, int32_t n, const int32_t
     if (!good(ctx)) return SPARSK_ESTATE;
     if (n < 1 || n > ctx->dm.max_seqs || !token_ids || !next_tokens || !exit_depths)
         return fail(ctx, SPARSK_EINVAL, "decode_step_host: bad arguments (n=%d)", n);
+    // the tokens are host data here, so their range is checked like every other host argument:
+    // before anything is enqueued, leaving all state as it was
+    const int V = ctx->dm.vocab_text + ctx->dm.vocab_speech;
+    for (int i = 0; i < n; i++)
+        if (token_ids[i] < 0 || token_ids[i] >= V)
+            return fail(ctx, SPARSK_EINVAL, "decode_step_host: token_ids[%d]=%d is outside the vocabulary [0, %d)", i, token_ids[i], V);
     CU(cudaMemcpyAsync(ctx->tok_dev, token_ids, sizeof(int) * n, cudaMemcpyHostToDevice, ctx->stream));
     const int rc = sparsk_decode_step(ctx, n, slots, ctx->tok_dev, modality, counters, ctx->out_tok_dev, ctx->out_depth_dev);
     if (rc != SPARSK_OK) return rc;
     CU(cudaMemcpyAsync(next_tokens, ctx->out_tok_dev, sizeof(int) * n, cudaMemcpyDeviceToHost, ctx->stream));
     CU(cudaMemcpyAsync(exit_depths, ctx->out_depth_dev, sizeof(int) * n, cudaMemcpyDeviceToHost, ctx->stream));
-    int status = 0;
-    CU(cudaMemcpyAsync(&status, ctx->sd.counts + CNT_STATUS, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
-    CU(cudaStreamSynchronize(ctx->stream));
-    if (status) CU(cudaMemsetAsync(ctx->sd.counts + CNT_STATUS, 0, sizeof(int), ctx->stream));
-    if (status & ST_TIMEOUT) return fail(ctx, SPARSK_ETIMEOUT, "a bounded in-kernel wait ran out");
-    if (status & ST_BAD_TOKEN) return fail(ctx, SPARSK_EINVAL, "a token id was outside the vocabulary (clamped)");
-    return SPARSK_OK;
+    return read_status(ctx);
 }

@@ -2,8 +2,8 @@
 //
 // One CTA handles one (sequence group, block of query vectors, kv head, KV split).  A group is
 // the block of rows of ONE sequence that a pass processes together: a single row in the lower
-// pass, the pending positions plus the current one in the upper pass (Algorithm 1: "batch
-// P u {t} ... length-K mask"), a chunk of the prompt in prefill.  All query heads that share
+// pass, the pending positions plus the current one in the upper pass (Algorithm 1, full-depth
+// branch: one causal block of at most K rows), a chunk of the prompt in prefill.  All query heads that share
 // the kv head, for all rows of the group, form the M dimension of mma.sync m16n8k16 tiles, so one
 // read of that head's K/V serves them all; row r of the group may look at positions
 // <= pos0 + r (the causal mask of the block on top of the whole earlier cache).
@@ -11,8 +11,8 @@
 // The split's positions are dealt to the CTA's four warps as contiguous sub-ranges.  Each warp
 // streams its own 16-position K/V tiles into a private three-stage shared-memory ring with
 // coalesced 16-byte cp.async copies (no CTA-wide barrier in the loop), computes S = Q K^T and
-// O += P V with bf16 MMAs and fp32 accumulators (queries and softmax weights enter as two bf16
-// terms, hi + lo, so that only the cache itself is rounded to bf16), and keeps an online softmax whose row maxima
+// O += P V with fp16 MMAs and fp32 accumulators (the cache is fp16; queries and softmax weights
+// enter as two fp16 terms, hi + lo, so that only the cache itself is rounded), and keeps an online softmax whose row maxima
 // and sums are reduced with shuffles inside the four-lane groups that share an accumulator row.
 // The four warps' states are merged through shared memory into one unnormalised partial
 // (acc, running max, running sum) per split; a second kernel merges the splits.
@@ -89,7 +89,7 @@ inline size_t attn_smem_bytes(int head_dim, int mt)
 struct AttnArgs {
     const bf16 *q;            // [rows][Hq*hd], already rotated
     const float *q32;         // the same in fp32; used instead of q when not NULL
-    const bf16 *kc, *vc;      // this layer: [slot][Hkv][S][hd]
+    const kv_t *kc, *vc;      // this layer: [slot][Hkv][S][hd]
     const int *grp_row0, *grp_nrows, *row_slot, *row_pos;
     const int *n_groups;      // device count
     float *part_o;            // [rows*Hq][n_splits][hd]
@@ -126,10 +126,10 @@ __device__ __forceinline__ void ldsm_x4_t(uint32_t (&r)[4], const void *p)
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                  : "r"((uint32_t)__cvta_generic_to_shared(p)));
 }
-// D += A B, A 16x16 bf16 (row), B 16x8 bf16 (col), D 16x8 fp32.
-__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+// D += A B, A 16x16 fp16 (row), B 16x8 fp16 (col), D 16x8 fp32.
+__device__ __forceinline__ void mma_f16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
 {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
@@ -147,9 +147,9 @@ __device__ __forceinline__ void attn_partial_body(const AttnArgs &a, int bx, int
     constexpr int QB = 16 * MT;     // query vectors per CTA
     constexpr int KP = HD + 8;      // padded row: ldmatrix rows fall into distinct banks
     constexpr int CH = HD / 8;      // 16-byte chunks per row
-    bf16 *Qs = reinterpret_cast<bf16 *>(at_smem);  // [QB][KP] hi terms
-    bf16 *Ql = Qs + QB * KP;                       // [QB][KP] lo terms
-    bf16 *ring = Ql + QB * KP;                     // [4 warps][NS][K,V][AT_TP][KP]
+    kv_t *Qs = reinterpret_cast<kv_t *>(at_smem);  // [QB][KP] hi terms
+    kv_t *Ql = Qs + QB * KP;                       // [QB][KP] lo terms
+    kv_t *ring = Ql + QB * KP;                     // [4 warps][NS][K,V][AT_TP][KP]
 
     const int g = bx / a.n_qblk, qb = bx % a.n_qblk;
     if (g >= *a.n_groups) return;
@@ -181,9 +181,11 @@ __device__ __forceinline__ void attn_partial_body(const AttnArgs &a, int bx, int
                 const float4 x0 = *reinterpret_cast<const float4 *>(a.q32 + off);
                 const float4 x1 = *reinterpret_cast<const float4 *>(a.q32 + off + 4);
                 const float v[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-                split8(v, hi, lo);
+                split8_h(v, hi, lo);
             } else {
-                hi = *reinterpret_cast<const uint4 *>(a.q + off);
+                float v[8];
+                unpack8(*reinterpret_cast<const uint4 *>(a.q + off), v);  // bf16 queries, widened
+                split8_h(v, hi, lo);
             }
         }
         *reinterpret_cast<uint4 *>(&Qs[qi * KP + c * 8]) = hi;
@@ -197,12 +199,12 @@ __device__ __forceinline__ void attn_partial_body(const AttnArgs &a, int bx, int
     const int w_beg = s_beg + warp * per;
     const int w_end = min(w_beg + per, s_end);
     const int n_tiles = w_end > w_beg ? (w_end - w_beg + AT_TP - 1) / AT_TP : 0;
-    bf16 *wr = ring + (size_t)warp * NS * 2 * AT_TP * KP;
-    const bf16 *kbase = a.kc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
-    const bf16 *vbase = a.vc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
+    kv_t *wr = ring + (size_t)warp * NS * 2 * AT_TP * KP;
+    const kv_t *kbase = a.kc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
+    const kv_t *vbase = a.vc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
 
     auto issue = [&](int t) {
-        bf16 *kt = wr + (size_t)(t % NS) * 2 * AT_TP * KP, *vt = kt + AT_TP * KP;
+        kv_t *kt = wr + (size_t)(t % NS) * 2 * AT_TP * KP, *vt = kt + AT_TP * KP;
         const int p0 = w_beg + t * AT_TP;
 #pragma unroll
         for (int i = lane; i < AT_TP * CH; i += 32) {
@@ -245,7 +247,7 @@ __device__ __forceinline__ void attn_partial_body(const AttnArgs &a, int bx, int
         __syncwarp();
         if (t + NS - 1 < n_tiles) issue(t + NS - 1);
         cp_async_commit();
-        const bf16 *Kt = wr + (size_t)(t % NS) * 2 * AT_TP * KP, *Vt = Kt + AT_TP * KP;
+        const kv_t *Kt = wr + (size_t)(t % NS) * 2 * AT_TP * KP, *Vt = Kt + AT_TP * KP;
         const int p0 = w_beg + t * AT_TP;
 
         // S = Q K^T for 16 positions
@@ -266,10 +268,10 @@ __device__ __forceinline__ void attn_partial_body(const AttnArgs &a, int bx, int
                 const int qoff = (mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * KP + ks * 16 + (lane >> 4) * 8;
                 ldsm_x4(qa, &Qs[qoff]);
                 ldsm_x4(ql, &Ql[qoff]);
-                mma_bf16(s[mt][0], qa, kb[0], kb[1]);
-                mma_bf16(s[mt][1], qa, kb[2], kb[3]);
-                mma_bf16(s[mt][0], ql, kb[0], kb[1]);
-                mma_bf16(s[mt][1], ql, kb[2], kb[3]);
+                mma_f16(s[mt][0], qa, kb[0], kb[1]);
+                mma_f16(s[mt][1], qa, kb[2], kb[3]);
+                mma_f16(s[mt][0], ql, kb[0], kb[1]);
+                mma_f16(s[mt][1], ql, kb[2], kb[3]);
             }
         }
         // online softmax; P as the A operand of the second product
@@ -306,8 +308,8 @@ __device__ __forceinline__ void attn_partial_body(const AttnArgs &a, int bx, int
                 }
                 l_run[mt][hf] = l_run[mt][hf] * alpha + psum;  // per-thread share; lanes are summed at the end
                 m_run[mt][hf] = m_new;
-                split_pair(v[0], v[1], pa[mt][hf], pl[mt][hf]);          // positions 0..7 of the tile
-                split_pair(v[2], v[3], pa[mt][2 + hf], pl[mt][2 + hf]);  // positions 8..15
+                split_pair_h(v[0], v[1], pa[mt][hf], pl[mt][hf]);          // positions 0..7 of the tile
+                split_pair_h(v[2], v[3], pa[mt][2 + hf], pl[mt][2 + hf]);  // positions 8..15
 #pragma unroll
                 for (int nt = 0; nt < HD / 8; nt++) {
                     o[mt][nt][hf * 2] *= alpha;
@@ -322,10 +324,10 @@ __device__ __forceinline__ void attn_partial_body(const AttnArgs &a, int bx, int
             ldsm_x4_t(vb, &Vt[((lane & 7) + ((lane >> 3) & 1) * 8) * KP + np * 16 + (lane >> 4) * 8]);
 #pragma unroll
             for (int mt = 0; mt < MT; mt++) {
-                mma_bf16(o[mt][2 * np], pa[mt], vb[0], vb[1]);
-                mma_bf16(o[mt][2 * np + 1], pa[mt], vb[2], vb[3]);
-                mma_bf16(o[mt][2 * np], pl[mt], vb[0], vb[1]);
-                mma_bf16(o[mt][2 * np + 1], pl[mt], vb[2], vb[3]);
+                mma_f16(o[mt][2 * np], pa[mt], vb[0], vb[1]);
+                mma_f16(o[mt][2 * np + 1], pa[mt], vb[2], vb[3]);
+                mma_f16(o[mt][2 * np], pl[mt], vb[0], vb[1]);
+                mma_f16(o[mt][2 * np + 1], pl[mt], vb[2], vb[3]);
             }
         }
     }
@@ -380,8 +382,8 @@ template <int HD, int MT>
 __global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(AttnArgs a)
 {
     extern __shared__ __align__(16) unsigned char at_smem_dyn[];
-    griddep_wait();
     griddep_launch();
+    griddep_wait();
     attn_partial_body<HD, MT, (MT == 2 ? 2 : AT_NST)>(a, blockIdx.x, blockIdx.y, blockIdx.z, at_smem_dyn, threadIdx.x,
                                                       AttnCtaSync());
 }
@@ -391,17 +393,18 @@ typedef void (*AttnPartialFn)(AttnArgs);
 // its dynamic shared-memory limit raised on first use.
 inline cudaError_t attn_partial_fn(int head_dim, int mt, AttnPartialFn *fn)
 {
-    static bool ready[4] = {false, false, false, false};
+    static PerDevice<bool> ready_dev[4];
     const int idx = (head_dim == 128 ? 2 : 0) + (mt == 2 ? 1 : 0);
     AttnPartialFn f = idx == 3 ? attn_partial_kernel<128, 2>
                       : idx == 2 ? attn_partial_kernel<128, 1>
                       : idx == 1 ? attn_partial_kernel<64, 2>
                                  : attn_partial_kernel<64, 1>;
-    if (!ready[idx]) {
+    bool &ready = ready_dev[idx].here();
+    if (!ready) {
         const cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                    (int)attn_smem_bytes(head_dim, mt));
         if (e != cudaSuccess) return e;
-        ready[idx] = true;
+        ready = true;
     }
     *fn = f;
     return cudaSuccess;
@@ -411,8 +414,8 @@ inline cudaError_t attn_partial_fn(int head_dim, int mt, AttnPartialFn *fn)
 template <int HD>
 __global__ void __launch_bounds__(HD) attn_merge_kernel(AttnArgs a, const int *__restrict__ n_rows)
 {
-    griddep_wait();
     griddep_launch();
+    griddep_wait();
     const int row = blockIdx.x, head = blockIdx.y;
     if (row >= *n_rows) return;
     const size_t cell0 = ((size_t)row * a.Hq + head) * a.n_splits;

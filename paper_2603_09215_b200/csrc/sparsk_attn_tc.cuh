@@ -2,11 +2,11 @@
 //
 // A refresh step of a sequence with 16 query heads per kv head and three pending positions has
 // 64 query vectors that share one K/V stream (Algorithm 1: the pending positions and the current
-// one go through the upper layers as one causal block).  With two-term bf16 operands that is 128
+// one go through the upper layers as one causal block).  With two-term fp16 operands that is 128
 // flop per cache byte: beyond what mma.sync delivers, so the block kernel of sparsk_attn.cuh is
 // tensor-bound there.  This kernel runs the same arithmetic on tcgen05:
 //
-//   S = Q K^T : A = the block's query vectors (up to 128 rows, hi and lo bf16 planes) held in TMEM,
+//   S = Q K^T : A = the block's query vectors (up to 128 rows, hi and lo fp16 planes) held in TMEM,
 //               stored there once with tcgen05.st (lane = query vector, elements packed two per
 //               column); B = a [64 positions x 128] K tile exactly as TMA delivers it from the
 //               cache (K-major); accumulator [128 x 64] fp32 in TMEM
@@ -20,11 +20,10 @@
 // 128, weights 2 x 64, queries 128.
 //
 // CTA = (group, block of 128 query vectors, kv head, KV split); warp 0 issues the TMA copies of a
-// K ring (three tiles) and a V ring (two), warp 1 issues the MMAs and owns the TMEM allocation, warps 2..9 do the
-// softmax (thread = query vector = TMEM lane, two warps per lane quadrant with half the columns each).
-// S and the weight planes are double buffered: a tile's scores and weights are formed while the
-// product of the tile before it is still running.  S is double buffered so that
-// the next tile's scores are computed while this tile's weights are being formed.  The partials
+// K ring (TA_KST tiles) and a V ring (TA_VST tiles), warp 1 issues the MMAs and owns the TMEM
+// allocation, warps 2..9 do the softmax (thread = query vector = TMEM lane, two warps per lane
+// quadrant with half the columns each).  The scores and the weight planes are double buffered: a
+// tile's scores and weights are formed while the product of the tile before it still runs.  The partials
 // (unnormalised output, running max, running sum per split) have the layout of the other
 // attention kernel, and attn_merge_kernel merges them.  Every wait is bounded.
 #pragma once
@@ -61,10 +60,11 @@ __device__ __forceinline__ uint64_t umma_desc_sw128_mn(uint32_t smem_addr, uint3
     return (uint64_t)((smem_addr & 0x3ffffu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
            (1ull << 46) | (2ull << 61);
 }
-// bf16 x bf16 -> fp32, M = 128, N = n, A K-major; B K-major or (b_mn) MN-major.
-__device__ __forceinline__ uint32_t umma_idesc_bf16_ex(int n, bool b_mn)
+// fp16 x fp16 -> fp32 (the cache is fp16; operand format fields 0 = f16 where the weight GEMMs set
+// 1 = bf16), M = 128, N = n, A K-major; B K-major or (b_mn) MN-major.
+__device__ __forceinline__ uint32_t umma_idesc_f16_ex(int n, bool b_mn)
 {
-    return umma_idesc_bf16(n) | (b_mn ? (1u << 16) : 0u);
+    return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TA_QB >> 4) << 24) | (b_mn ? (1u << 16) : 0u);
 }
 __device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, uint32_t (&r)[16])
 {
@@ -77,7 +77,7 @@ __device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, uint32_t (&r)[1
 }
 
 // D (+)= A B with the A operand in TMEM (lane = row, 16-bit elements packed two per column) and B in shared memory.
-__device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc, int accumulate)
+__device__ __forceinline__ void umma_f16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc, int accumulate)
 {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -112,8 +112,8 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
 
     // ---- what this CTA works on (every thread computes the same); a CTA whose group belongs to
     // the other kernel, or does not exist, leaves before it sets anything up
-    griddep_wait();
     griddep_launch();
+    griddep_wait();
     const int bx = blockIdx.x, hk = blockIdx.y, sp = blockIdx.z;
     const int g = bx / a.n_qblk, qb = bx % a.n_qblk;
     const int G = a.Hq / a.Hkv;
@@ -168,7 +168,7 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
     const uint32_t tmem_base = tmem_base_s;
     const uint32_t t_s0 = tmem_base + TA_C_S, t_o = tmem_base + TA_C_O, t_p = tmem_base + TA_C_P, t_q = tmem_base + TA_C_Q;
 
-    // ---- the queries, as two bf16 planes in TMEM (thread = query vector = lane; 16-bit elements
+    // ---- the queries, as two fp16 planes in TMEM (thread = query vector = lane; 16-bit elements
     // packed two per column): the A operand of every score MMA, stored once.  The two warps of a
     // lane quadrant take 64 of the 128 head dimensions each.
     if (warp >= 2 && n_tiles > 0) {
@@ -187,7 +187,7 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
                     const float4 x0 = *reinterpret_cast<const float4 *>(src + blk * 32 + c * 8);
                     const float4 x1 = *reinterpret_cast<const float4 *>(src + blk * 32 + c * 8 + 4);
                     const float v[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-                    split8(v, h4, l4);
+                    split8_h(v, h4, l4);
                 }
                 hi[c * 4] = h4.x; hi[c * 4 + 1] = h4.y; hi[c * 4 + 2] = h4.z; hi[c * 4 + 3] = h4.w;
                 lo[c * 4] = l4.x; lo[c * 4 + 1] = l4.y; lo[c * 4 + 2] = l4.z; lo[c * 4 + 3] = l4.w;
@@ -228,7 +228,7 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0 && n_tiles > 0) {
-            const uint32_t idesc_s = umma_idesc_bf16_ex(TA_NT, false), idesc_o = umma_idesc_bf16_ex(TA_HD, true);
+            const uint32_t idesc_s = umma_idesc_f16_ex(TA_NT, false), idesc_o = umma_idesc_f16_ex(TA_HD, true);
             bool ok = true;
             auto issue_s = [&](int t) {
                 const int st = t % TA_KST, b = t & 1;
@@ -242,8 +242,8 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
 #pragma unroll
                 for (int kk = 0; kk < TA_HD / 16; kk++) {  // 16 head dimensions = 8 packed TMEM columns of the queries
                     const uint64_t db = dk0 + (uint64_t)(((kk >> 2) * 8192 + (kk & 3) * 32) >> 4);
-                    umma_bf16_ts(d, t_q + (uint32_t)kk * 8, db, idesc_s, kk > 0);
-                    umma_bf16_ts(d, t_q + 64 + (uint32_t)kk * 8, db, idesc_s, 1);
+                    umma_f16_ts(d, t_q + (uint32_t)kk * 8, db, idesc_s, kk > 0);
+                    umma_f16_ts(d, t_q + 64 + (uint32_t)kk * 8, db, idesc_s, 1);
                 }
                 umma_commit(&k_empty[st]);  // the K tile is free once the scores are computed
                 umma_commit(&s_full[b]);
@@ -263,8 +263,8 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
 #pragma unroll
                 for (int kk = 0; kk < TA_NT / 16; kk++) {  // 16 positions = 8 packed columns
                     const uint64_t dv = dv0 + (uint64_t)((kk * 2048) >> 4);
-                    umma_bf16_ts(t_o, tp + (uint32_t)kk * 8, dv, idesc_o, t > 0 || kk > 0);
-                    umma_bf16_ts(t_o, tp + 32 + (uint32_t)kk * 8, dv, idesc_o, 1);
+                    umma_f16_ts(t_o, tp + (uint32_t)kk * 8, dv, idesc_o, t > 0 || kk > 0);
+                    umma_f16_ts(t_o, tp + 32 + (uint32_t)kk * 8, dv, idesc_o, 1);
                 }
                 umma_commit(&v_empty[st]);  // the V tile and this buffer of weights are free once these have read them
                 umma_commit(&o_full[b]);
@@ -365,7 +365,7 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
                     break;
                 }
                 // The reference maximum is allowed to lag the true one by TA_RAISE (weights then reach
-                // 2^11, which two bf16 terms and fp32 sums carry without loss): otherwise some lane of
+                // 2^11, which two fp16 terms and fp32 sums carry without loss): otherwise some lane of
                 // the warp would see a new maximum in most tiles and the accumulator would be
                 // rescaled nearly every time.  Partials stay exact: (o, l) are relative to m_run.
                 const bool raise = tmax > m_run + TA_RAISE;
@@ -382,7 +382,7 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
                         w[i] = exp2f(__uint_as_float(sr[c >> 1][(c & 1) * 8 + i]) - m_ref);  // 2^(-inf) = 0 for masked positions
                         psum += w[i];
                     }
-                    split8(w, whi[c], wlo[c]);
+                    split8_h(w, whi[c], wlo[c]);
                 }
                 // The weights go to buffer b, which the product of tile t - 2 has read by the time
                 // o_full[b] completes; a rescaling needs every product so far in the accumulator.  A

@@ -2,12 +2,21 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
 namespace sparsk {
 
 typedef __nv_bfloat16 bf16;
+// Element of the KV cache: IEEE half precision.  Weights and the activations that meet them are
+// bfloat16, but a cached key or value is re-read by every later step, and at random
+// initialisation its rounding error is amplified by every later layer: with 8 significant bits
+// (bfloat16) the exit states of a 28-layer stack drift to 2 % from the fp64 reference once a few
+// hundred positions of the cache are the decoder's own; the 11 bits of fp16 cost the same two
+// bytes and leave 0.3 %.  Keys and values are O(1)..O(100) numbers, far inside the fp16 range;
+// a value beyond it is stored as the largest finite fp16 number.
+typedef __half kv_t;
 
 // Row bookkeeping of one decode step, all device arrays inside the workspace.
 // "Lower" rows are the step's sequences themselves (one row each, layers 1..e);
@@ -27,6 +36,27 @@ struct StepDesc {
 enum { CNT_NSEQ = 0, CNT_MUP = 1, CNT_NGRP = 2, CNT_LIST0 = 3 /* ..6 */, CNT_STATUS = 7 };
 enum { ST_BAD_TOKEN = 1, ST_TIMEOUT = 2 };
 
+// Host side: a value kept once per device of the process.  Function attributes (dynamic
+// shared-memory limits, occupancy answers) belong to a device, so "already set" is remembered
+// for the device that is current, not for the process.
+template <class T>
+struct PerDevice {
+    T v[64];
+    T &here()
+    {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        return v[(unsigned)dev & 63u];
+    }
+};
+
+// Programmatic dependent launch.  A kernel lets the next one in the stream start as early as it
+// can (launch_dependents, normally its first instruction) and touches nothing an earlier kernel
+// writes before its own wait has returned (wait = the predecessor grid has completed and its
+// writes are visible).  Every kernel here waits before it completes, so completion is transitive:
+// when a kernel's wait returns, everything before it in the stream is done.  The early start is
+// what lets a weight-streaming kernel issue its first weight copies (which depend on nothing)
+// while a small kernel between two of them is still running.
 __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;"); }
 
@@ -71,6 +101,29 @@ __device__ __forceinline__ void split8(const float (&v)[8], uint4 &hi, uint4 &lo
     split_pair(v[2], v[3], hi.y, lo.y);
     split_pair(v[4], v[5], hi.z, lo.z);
     split_pair(v[6], v[7], hi.w, lo.w);
+}
+
+__device__ __forceinline__ kv_t to_kv(float x) { return __float2half_rn(fminf(fmaxf(x, -65504.f), 65504.f)); }
+// The same two-term form in fp16 (what multiplies the cache in the attention kernels): hi has 11
+// significant bits, hi + lo about 22.
+__device__ __forceinline__ uint32_t pack_h2(float a, float b)
+{
+    __half2 t = __floats2half2_rn(a, b);
+    return *reinterpret_cast<uint32_t *>(&t);
+}
+__device__ __forceinline__ void split_pair_h(float a, float b, uint32_t &hi, uint32_t &lo)
+{
+    const __half2 h = __floats2half2_rn(a, b);
+    const float2 f = __half22float2(h);
+    hi = *reinterpret_cast<const uint32_t *>(&h);
+    lo = pack_h2(a - f.x, b - f.y);
+}
+__device__ __forceinline__ void split8_h(const float (&v)[8], uint4 &hi, uint4 &lo)
+{
+    split_pair_h(v[0], v[1], hi.x, lo.x);
+    split_pair_h(v[2], v[3], hi.y, lo.y);
+    split_pair_h(v[4], v[5], hi.z, lo.z);
+    split_pair_h(v[6], v[7], hi.w, lo.w);
 }
 
 __device__ __forceinline__ float warp_sum(float v)

@@ -399,7 +399,7 @@ __global__ void __launch_bounds__(GM_THREADS, 1)
 // sums are added into an fp32 scratch [rows][Hq*hd + 2*Hkv*hd] and qkv_finish_kernel does the rest.
 struct QkvEnd {
     float *q_out;        // [rows][Hq*hd] fp32 (the attention kernels split it into two bf16 terms)
-    bf16 *kc, *vc;       // this layer's cache [slot][Hkv][S][hd]
+    kv_t *kc, *vc;       // this layer's cache [slot][Hkv][S][hd]
     const float2 *rope;  // [S][hd/2]
     const int *row_slot, *row_pos;
     float *partial;      // scratch for split sums, or NULL
@@ -440,13 +440,13 @@ struct QkvEnd {
                         if (m >= t.m_end) break;
                         const int slot = row_slot[m], pos = row_pos[m];
                         if (t.matrix == 2) {
-                            vc[(((size_t)slot * Hkv + head) * S + pos) * hd + i] = __float2bfloat16(v[c]);
+                            vc[(((size_t)slot * Hkv + head) * S + pos) * hd + i] = to_kv(v[c]);
                         } else {
                             const float other = t.xchg[c * GM_BM + (t.row ^ half)];
                             const float2 cs = rope[(size_t)pos * half + j];
                             const float r = hi ? v[c] * cs.x + other * cs.y : v[c] * cs.x - other * cs.y;
                             if (t.matrix == 0) q_out[(size_t)m * Hq * hd + n] = r;
-                            else kc[(((size_t)slot * Hkv + head) * S + pos) * hd + i] = __float2bfloat16(r);
+                            else kc[(((size_t)slot * Hkv + head) * S + pos) * hd + i] = to_kv(r);
                         }
                     }
                 }
@@ -460,14 +460,14 @@ struct QkvEnd {
 // the scratch, applies the rotary embedding, writes q and appends k, v to the cache, and clears
 // the scratch for the next product.  One block per activation row.
 static __global__ void __launch_bounds__(256) qkv_finish_kernel(float *__restrict__ partial, float *__restrict__ q_out,
-                                                         bf16 *__restrict__ kc, bf16 *__restrict__ vc,
+                                                         kv_t *__restrict__ kc, kv_t *__restrict__ vc,
                                                          const float2 *__restrict__ rope,
                                                          const int *__restrict__ row_slot,
                                                          const int *__restrict__ row_pos, int n_rows, int Hq, int Hkv,
                                                          int hd, int S)
 {
-    griddep_wait();
     griddep_launch();
+    griddep_wait();
     const int m = blockIdx.x;
     if (m >= n_rows) return;
     const int half = hd >> 1, width = (Hq + 2 * Hkv) * hd;
@@ -484,13 +484,13 @@ static __global__ void __launch_bounds__(256) qkv_finish_kernel(float *__restric
             dst[0] = ra;
             dst[half] = rb;
         } else {
-            bf16 *dst = kc + (((size_t)slot * Hkv + (head - Hq)) * S + pos) * hd + j;
-            dst[0] = __float2bfloat16(ra);
-            dst[half] = __float2bfloat16(rb);
+            kv_t *dst = kc + (((size_t)slot * Hkv + (head - Hq)) * S + pos) * hd + j;
+            dst[0] = to_kv(ra);
+            dst[half] = to_kv(rb);
         }
     }
     for (int i = threadIdx.x; i < Hkv * hd; i += blockDim.x)
-        vc[(((size_t)slot * Hkv + i / hd) * S + pos) * hd + i % hd] = __float2bfloat16(src[(Hq + Hkv) * hd + i]);
+        vc[(((size_t)slot * Hkv + i / hd) * S + pos) * hd + i % hd] = to_kv(src[(Hq + Hkv) * hd + i]);
     __syncthreads();
     for (int i = threadIdx.x; i < width; i += blockDim.x) src[i] = 0.f;
 }
@@ -588,8 +588,8 @@ static __global__ void __launch_bounds__(256) rmsnorm_rows_kernel(const float *_
                                                            bf16 *__restrict__ x_lo, int n_rows, int K, float eps)
 {
     __shared__ float red[8];
-    griddep_wait();
     griddep_launch();
+    griddep_wait();
     const int i = blockIdx.x;
     if (i >= n_rows) return;
     const float *src = h + (size_t)(row_idx ? row_idx[i] : i) * K;

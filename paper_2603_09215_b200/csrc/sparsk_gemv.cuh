@@ -153,8 +153,8 @@ __global__ void __launch_bounds__(GV_THREADS, 1) gemv_kernel(Op op, GvIn in)
             }
         }
     }
-    griddep_wait();
     griddep_launch();
+    griddep_wait();
 
     gv_load_act<M, NORM>(in, m0, mrows, act, red);
     __syncthreads();
@@ -226,7 +226,7 @@ struct QkvOp {
     struct State {};
     const bf16 *wq, *wk, *wv;
     float *q_out;             // [rows][Hq*hd] fp32
-    bf16 *kc, *vc;            // this layer's cache: [slot][Hkv][S][hd]
+    kv_t *kc, *vc;            // this layer's cache: [slot][Hkv][S][hd]
     const float2 *rope;       // [S][hd/2] (cos, sin)
     const int *row_slot, *row_pos;
     int d, Hq, Hkv, hd, S;
@@ -267,17 +267,17 @@ struct QkvOp {
                     dst[0] = ra;
                     dst[half] = rb;
                 } else {
-                    bf16 *dst = kc + (((size_t)slot * Hkv + head) * S + pos) * hd + i0 + p;
-                    dst[0] = __float2bfloat16(ra);
-                    dst[half] = __float2bfloat16(rb);
+                    kv_t *dst = kc + (((size_t)slot * Hkv + head) * S + pos) * hd + i0 + p;
+                    dst[0] = to_kv(ra);
+                    dst[half] = to_kv(rb);
                 }
             }
         } else {
             const int row0 = (g - gq() - gk()) * R;
             const int head = row0 / hd, i0 = row0 % hd;
-            bf16 *dst = vc + (((size_t)slot * Hkv + head) * S + pos) * hd + i0;
+            kv_t *dst = vc + (((size_t)slot * Hkv + head) * S + pos) * hd + i0;
 #pragma unroll
-            for (int r = 0; r < R; r++) dst[r] = __float2bfloat16(v[r]);
+            for (int r = 0; r < R; r++) dst[r] = to_kv(v[r]);
         }
     }
     __device__ void final(State &, int, int) const {}

@@ -64,7 +64,7 @@ enum { MK_QKV = 0, MK_ATTN = 1, MK_MERGE = 2, MK_OPROJ = 3, MK_GATEUP = 4, MK_DO
 struct MkLayer {
     CUtensorMap map_q, map_k, map_v, map_o, map_g, map_u, map_d;  // [256 x 16] boxes, no swizzle
     const bf16 *attn_gain, *mlp_gain;
-    bf16 *kc, *vc;  // this layer's cache [slot][Hkv][S][hd]
+    kv_t *kc, *vc;  // this layer's cache [slot][Hkv][S][hd]
 };
 
 struct MkArgs {
@@ -230,7 +230,10 @@ __device__ __forceinline__ bool mk_grid_barrier(const MkArgs &a, MkShared *sh, u
             if (ld_acquire_u64(a.bar) >= epoch) break;
             if ((spin & 63u) == 63u) {
                 if (ld_volatile_i32(a.abort_word) || sh->giving_up) {
+                    // another CTA (or an earlier launch that was never cleaned up after) gave up:
+                    // leave too, and say so, so that skipping the rest is never silent
                     sh->giving_up = 1;
+                    atomicOr(a.status, ST_TIMEOUT);
                     break;
                 }
                 const unsigned long long now = global_ns();

@@ -6,7 +6,7 @@ namespace sparsk {
 // Items (group, query block, kv head, split) are dealt to MK_ATT_WARPS warps of every CTA; a warp
 // runs its item alone: 16 query vectors (query heads of the kv head, for the group's rows), its
 // own two-stage K/V ring inside the activation area, one partial per item.  The arithmetic is
-// that of attn_partial_kernel with one m16 tile (queries and softmax weights as two bf16 terms).
+// that of attn_partial_kernel with one m16 tile (queries and softmax weights as two fp16 terms).
 template <int HD>
 __device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, unsigned char *area, const MkShared *sh)
 {
@@ -14,9 +14,9 @@ __device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (warp >= MK_ATT_WARPS) return;
     // per warp: its 16 query vectors (hi and lo term), then the K/V ring
-    bf16 *Qs = reinterpret_cast<bf16 *>(area) + (size_t)warp * (2 * 16 + MK_ATT_NST * 2 * AT_TP) * KP;
-    bf16 *Ql = Qs + 16 * KP;
-    bf16 *wr = Ql + 16 * KP;
+    kv_t *Qs = reinterpret_cast<kv_t *>(area) + (size_t)warp * (2 * 16 + MK_ATT_NST * 2 * AT_TP) * KP;
+    kv_t *Ql = Qs + 16 * KP;
+    kv_t *wr = Ql + 16 * KP;
     const int G = a.Hq / a.Hkv;
     const int n_workers = gridDim.x * MK_ATT_WARPS, worker = warp * gridDim.x + blockIdx.x;
     const int n_qblk = a.att_qblk;
@@ -38,11 +38,11 @@ __device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, 
         const int w_beg = sp * a.att_split_len;
         const int w_end = min(w_beg + a.att_split_len, kv_end_all);
         const int n_tiles = w_end > w_beg ? (w_end - w_beg + AT_TP - 1) / AT_TP : 0;
-        const bf16 *kbase = L->kc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
-        const bf16 *vbase = L->vc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
+        const kv_t *kbase = L->kc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
+        const kv_t *vbase = L->vc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
 
         auto issue = [&](int tt) {
-            bf16 *kt = wr + (size_t)(tt % MK_ATT_NST) * 2 * AT_TP * KP, *vt = kt + AT_TP * KP;
+            kv_t *kt = wr + (size_t)(tt % MK_ATT_NST) * 2 * AT_TP * KP, *vt = kt + AT_TP * KP;
             const int p0 = w_beg + tt * AT_TP;
 #pragma unroll
             for (int i = lane; i < AT_TP * CH; i += 32) {
@@ -78,7 +78,7 @@ __device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, 
                 const float *src = a.q_buf + (size_t)(row0 + r) * a.Hq * HD + (hk * G + j) * HD + c * 8;
                 const float4 x0 = *reinterpret_cast<const float4 *>(src), x1 = *reinterpret_cast<const float4 *>(src + 4);
                 const float v[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-                split8(v, hi, lo);
+                split8_h(v, hi, lo);
             }
             *reinterpret_cast<uint4 *>(&Qs[qi * KP + c * 8]) = hi;
             *reinterpret_cast<uint4 *>(&Ql[qi * KP + c * 8]) = lo;
@@ -88,7 +88,7 @@ __device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, 
         for (int tt = 0; tt < n_tiles; tt++) {
             cp_async_wait<1>();  // all but the newest group: tile tt has landed
             __syncwarp();
-            const bf16 *Kt = wr + (size_t)(tt % MK_ATT_NST) * 2 * AT_TP * KP, *Vt = Kt + AT_TP * KP;
+            const kv_t *Kt = wr + (size_t)(tt % MK_ATT_NST) * 2 * AT_TP * KP, *Vt = Kt + AT_TP * KP;
             const int p0 = w_beg + tt * AT_TP;
             float s[2][4];
 #pragma unroll
@@ -101,10 +101,10 @@ __device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, 
                 ldsm_x4(kb, &Kt[((lane & 7) + ((lane >> 4) << 3)) * KP + ks * 16 + ((lane >> 3) & 1) * 8]);
                 ldsm_x4(qa, &Qs[((lane & 7) + ((lane >> 3) & 1) * 8) * KP + ks * 16 + (lane >> 4) * 8]);
                 ldsm_x4(ql, &Ql[((lane & 7) + ((lane >> 3) & 1) * 8) * KP + ks * 16 + (lane >> 4) * 8]);
-                mma_bf16(s[0], qa, kb[0], kb[1]);
-                mma_bf16(s[1], qa, kb[2], kb[3]);
-                mma_bf16(s[0], ql, kb[0], kb[1]);
-                mma_bf16(s[1], ql, kb[2], kb[3]);
+                mma_f16(s[0], qa, kb[0], kb[1]);
+                mma_f16(s[1], qa, kb[2], kb[3]);
+                mma_f16(s[0], ql, kb[0], kb[1]);
+                mma_f16(s[1], ql, kb[2], kb[3]);
             }
             uint32_t pa[4], pl[4];
 #pragma unroll
@@ -137,8 +137,8 @@ __device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, 
                 }
                 l_run[hf] = l_run[hf] * alpha + psum;
                 m_run[hf] = m_new;
-                split_pair(v[0], v[1], pa[hf], pl[hf]);
-                split_pair(v[2], v[3], pa[2 + hf], pl[2 + hf]);
+                split_pair_h(v[0], v[1], pa[hf], pl[hf]);
+                split_pair_h(v[2], v[3], pa[2 + hf], pl[2 + hf]);
 #pragma unroll
                 for (int nt = 0; nt < HD / 8; nt++) {
                     o[nt][hf * 2] *= alpha;
@@ -149,10 +149,10 @@ __device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, 
             for (int np = 0; np < HD / 16; np++) {
                 uint32_t vb[4];
                 ldsm_x4_t(vb, &Vt[((lane & 7) + ((lane >> 3) & 1) * 8) * KP + np * 16 + (lane >> 4) * 8]);
-                mma_bf16(o[2 * np], pa, vb[0], vb[1]);
-                mma_bf16(o[2 * np + 1], pa, vb[2], vb[3]);
-                mma_bf16(o[2 * np], pl, vb[0], vb[1]);
-                mma_bf16(o[2 * np + 1], pl, vb[2], vb[3]);
+                mma_f16(o[2 * np], pa, vb[0], vb[1]);
+                mma_f16(o[2 * np + 1], pa, vb[2], vb[3]);
+                mma_f16(o[2 * np], pl, vb[0], vb[1]);
+                mma_f16(o[2 * np + 1], pl, vb[2], vb[3]);
             }
             __syncwarp();  // everyone is done with this stage: refill it with the tile after next
             if (tt + 2 < n_tiles) issue(tt + 2);

@@ -137,15 +137,15 @@ __device__ __forceinline__ bool mk_project(int type, const MkArgs &a, const MkLa
                         dst[0] = ra;
                         dst[half] = rb;
                     } else {
-                        bf16 *dst = L->kc + (((size_t)slot_id * a.Hkv + head) * a.S + pos) * a.hd + i;
-                        dst[0] = __float2bfloat16(ra);
-                        dst[half] = __float2bfloat16(rb);
+                        kv_t *dst = L->kc + (((size_t)slot_id * a.Hkv + head) * a.S + pos) * a.hd + i;
+                        dst[0] = to_kv(ra);
+                        dst[half] = to_kv(rb);
                     }
                 } else {
                     const int n0 = (b - nq - nk) * 2 * MK_BOX_ROWS + warp, n1 = n0 + MK_BOX_ROWS;
                     const int kvd = a.Hkv * a.hd;
-                    if (n0 < kvd) L->vc[(((size_t)slot_id * a.Hkv + n0 / a.hd) * a.S + pos) * a.hd + n0 % a.hd] = __float2bfloat16(v0);
-                    if (n1 < kvd) L->vc[(((size_t)slot_id * a.Hkv + n1 / a.hd) * a.S + pos) * a.hd + n1 % a.hd] = __float2bfloat16(v1);
+                    if (n0 < kvd) L->vc[(((size_t)slot_id * a.Hkv + n0 / a.hd) * a.S + pos) * a.hd + n0 % a.hd] = to_kv(v0);
+                    if (n1 < kvd) L->vc[(((size_t)slot_id * a.Hkv + n1 / a.hd) * a.S + pos) * a.hd + n1 % a.hd] = to_kv(v1);
                 }
                 break;
             }

@@ -67,8 +67,10 @@ extern "C" int sparsk_attention_static(const sparsk_attn_args *args, void *cuda_
         }
         scratch = g_scratch_addr[dev];
     }
-    // Nothing in the area has to start at zero: the two counters are rewritten by every call and
-    // every partial cell a call reads is one it wrote first.
+    // Nothing in the area has to start at zero: the two counters are rewritten by every call and,
+    // as long as the groups partition the rows and none exceeds max_grp_rows (the documented
+    // precondition of sparsk_attention), every partial cell a call reads is one it wrote first.
+    // A row outside every group would be merged from whatever an earlier call left here.
     const int rc = sparsk_attention(args, scratch, need, cuda_stream);
     if (rc == SPARSK_EINVAL) say(err, err_len, "sparsk_attention rejected the arguments");
     if (rc == SPARSK_ECUDA) say(err, err_len, "a kernel launch failed");

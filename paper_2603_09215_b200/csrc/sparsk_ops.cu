@@ -46,7 +46,7 @@ int sparsk_attention_launch(const sparsk_attn_args *p, char *scratch, cudaStream
     const size_t cells = (size_t)p->n_rows * p->n_q_heads * AT_MAX_SPLITS;
     int *counts = reinterpret_cast<int *>(scratch);
     AttnArgs a{};
-    a.q = (const bf16 *)p->q; a.kc = (const bf16 *)p->k_cache; a.vc = (const bf16 *)p->v_cache;
+    a.q = (const bf16 *)p->q; a.kc = (const kv_t *)p->k_cache; a.vc = (const kv_t *)p->v_cache;
     a.grp_row0 = p->grp_row0; a.grp_nrows = p->grp_nrows; a.row_slot = p->row_slot; a.row_pos = p->row_pos;
     a.n_groups = counts;
     a.part_o = reinterpret_cast<float *>(scratch + 256);

@@ -259,7 +259,8 @@ __global__ void __launch_bounds__(SP_THREADS, 1) nucleus_sample_kernel(SampleArg
 inline cudaError_t launch_nucleus_sample(SampleArgs a, int n, bool has_text, bool has_speech, cudaStream_t st, bool pdl,
                                          int64_t *n_launches)
 {
-    static bool ready = false;
+    static PerDevice<bool> ready_dev;
+    bool &ready = ready_dev.here();
     if (!ready) {
         cudaError_t e = cudaFuncSetAttribute(nucleus_sample_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SP_SMEM);
         if (e == cudaSuccess)

@@ -8,13 +8,18 @@ namespace sparsk {
 
 // Layers a step runs (Sec. IV-B.1): in-chunk index c runs L layers iff c mod K == r, else e.
 // text_exit 0: text (modality 0) always runs L; 1: text follows the rule too; 2: only text follows
-// it and speech always runs L (Sec. V-E, row G10).  The host's mirror of the pending counts uses
-// the same function.
-__host__ __device__ inline int scheduled_depth(int modality, int c, int K, int r, int e, int L, int text_exit)
+// it and speech always runs L (Sec. V-E, row G10).  Text steps that follow the rule use their own
+// period and phase (Kt, rt), speech steps (K, r): the two modalities may need different policies
+// (Sec. V-E).  The host's mirror of the pending counts uses the same function.
+struct SchedParams {
+    int L, e, K, r, Kt, rt, text_exit;
+};
+__host__ __device__ inline int scheduled_depth(int modality, int c, const SchedParams &p)
 {
-    if (modality == 0 && text_exit == 0) return L;
-    if (modality != 0 && text_exit == 2) return L;
-    return (c % K == r) ? L : e;
+    if (modality == 0 && p.text_exit == 0) return p.L;
+    if (modality != 0 && p.text_exit == 2) return p.L;
+    if (modality == 0) return (c % p.Kt == p.rt) ? p.L : p.e;
+    return (c % p.K == p.r) ? p.L : p.e;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -22,15 +27,14 @@ __host__ __device__ inline int scheduled_depth(int modality, int c, int K, int r
 // into the vocabulary, with a status bit if it was outside) and clears the sequence's argmax cell.
 // ---------------------------------------------------------------------------------------
 static __global__ void schedule_kernel(StepDesc sd, int n, const int *__restrict__ staged /*[3][n]*/,
-                                const int *__restrict__ tokens_in, int vocab, int L, int e, int K,
-                                int r, int text_exit)
+                                const int *__restrict__ tokens_in, int vocab, SchedParams sp)
 {
     griddep_wait();
     int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b == 0) sd.counts[CNT_NSEQ] = n;
     if (b >= n) return;
     int slot = staged[b], mod = staged[n + b], c = staged[2 * n + b];
-    int depth = scheduled_depth(mod, c, K, r, e, L, text_exit);
+    int depth = scheduled_depth(mod, c, sp);
     int tok = tokens_in[b];
     if (tok < 0 || tok >= vocab) {
         atomicOr(&sd.counts[CNT_STATUS], ST_BAD_TOKEN);
@@ -76,8 +80,8 @@ __device__ __forceinline__ int block_exscan(int v, int *warp_tot /*[32] shared*/
 
 // ---------------------------------------------------------------------------------------
 // Active-row compaction.  Sequences that leave at layer e drop out of layers e+1..L; every
-// full-depth sequence contributes its pending positions plus its current one (Algorithm 1:
-// "batch P u {t}").  Prefix sums give each sequence its offset in the upper row list; four
+// full-depth sequence contributes its pending positions plus its current one (Algorithm 1,
+// full-depth branch).  Prefix sums give each sequence its offset in the upper row list; four
 // more give the per-(exit, modality) lists the head kernels read.  One block, n <= 1024.
 // ---------------------------------------------------------------------------------------
 static __global__ void __launch_bounds__(1024) compact_kernel(StepDesc sd, int n, const int *__restrict__ kv_len,
@@ -154,7 +158,7 @@ static __global__ void embed_kernel(const int *__restrict__ tokens, const bf16 *
     }
 }
 
-// Early-exit rows: store h^(e) in the pending store ("store h_t^(l_EE)", Algorithm 1).
+// Early-exit rows: h^(e) goes to the pending store (Algorithm 1, early-exit branch).
 static __global__ void stash_kernel(StepDesc sd, const float *__restrict__ h_lo, float *__restrict__ pend_h,
                              const int *__restrict__ pend_cnt, int n, int d, int L, int max_pending)
 {
@@ -182,6 +186,42 @@ static __global__ void gather_upper_kernel(StepDesc sd, const float *__restrict_
     const float *from = (src >= 0) ? pend_h + ((size_t)sd.up_slot[row] * max_pending + src) * d
                                    : h_lo + (size_t)(-1 - src) * d;
     const float4 *s4 = reinterpret_cast<const float4 *>(from);
+    float4 *d4 = reinterpret_cast<float4 *>(h_up + (size_t)row * d);
+    for (int i = threadIdx.x; i < d / 4; i += blockDim.x) d4[i] = s4[i];
+}
+
+// Last layer of the upper pass: pending rows only need their K/V there (nothing reads their
+// h^(L): Algorithm 1's full-depth branch takes the token from the current position alone), so
+// after the K/V projection the layer goes on with one row per full-depth sequence.  Group g's
+// current row is the last row of the group: its residual stream and its query move to row g of
+// the compact buffers, with its slot and position.
+static __global__ void take_current_kernel(StepDesc sd, const float *__restrict__ h_up, const float *__restrict__ q_up,
+                                    float *__restrict__ h_last, float *__restrict__ q_last,
+                                    int *__restrict__ last_slot, int *__restrict__ last_pos, int d, int qd)
+{
+    griddep_wait();
+    const int g = blockIdx.x;
+    if (g >= sd.counts[CNT_NGRP]) return;
+    const int row = sd.up_grp_row0[g] + sd.up_grp_nrows[g] - 1;
+    if (threadIdx.x == 0) {
+        last_slot[g] = sd.up_slot[row];
+        last_pos[g] = sd.up_pos[row];
+    }
+    const float4 *hs = reinterpret_cast<const float4 *>(h_up + (size_t)row * d);
+    float4 *hd4 = reinterpret_cast<float4 *>(h_last + (size_t)g * d);
+    for (int i = threadIdx.x; i < d / 4; i += blockDim.x) hd4[i] = hs[i];
+    const float4 *qs = reinterpret_cast<const float4 *>(q_up + (size_t)row * qd);
+    float4 *qd4 = reinterpret_cast<float4 *>(q_last + (size_t)g * qd);
+    for (int i = threadIdx.x; i < qd / 4; i += blockDim.x) qd4[i] = qs[i];
+}
+// ... and h^(L) of the current rows goes back to where the heads read it.
+static __global__ void put_current_kernel(StepDesc sd, const float *__restrict__ h_last, float *__restrict__ h_up, int d)
+{
+    griddep_wait();
+    const int g = blockIdx.x;
+    if (g >= sd.counts[CNT_NGRP]) return;
+    const int row = sd.up_grp_row0[g] + sd.up_grp_nrows[g] - 1;
+    const float4 *s4 = reinterpret_cast<const float4 *>(h_last + (size_t)g * d);
     float4 *d4 = reinterpret_cast<float4 *>(h_up + (size_t)row * d);
     for (int i = threadIdx.x; i < d / 4; i += blockDim.x) d4[i] = s4[i];
 }
@@ -240,9 +280,9 @@ static __global__ void set_int_kernel(int *p, int v)
     *p = v;
 }
 
-// Cache import/export: [n][Hkv*hd] <-> [Hkv][S][hd] of one (layer, slot).
-static __global__ void kv_copy_kernel(bf16 *__restrict__ cache_k, bf16 *__restrict__ cache_v, bf16 *ext_k,
-                               bf16 *ext_v, int first_pos, int n, int Hkv, int hd, int S, int to_cache)
+// Cache import/export: [n][Hkv*hd] <-> [Hkv][S][hd] of one (layer, slot), fp16 on both sides.
+static __global__ void kv_copy_kernel(kv_t *__restrict__ cache_k, kv_t *__restrict__ cache_v, kv_t *ext_k,
+                               kv_t *ext_v, int first_pos, int n, int Hkv, int hd, int S, int to_cache)
 {
     griddep_wait();
     const size_t total = (size_t)n * Hkv * hd;

@@ -42,7 +42,7 @@ class Pair:
         self.out_tok = torch.zeros(n_seqs, dtype=torch.int32, device="cuda")
         self.out_dep = torch.zeros(n_seqs, dtype=torch.int32, device="cuda")
         self.stats = {"steps": 0, "max_hidden": 0.0, "max_logit": 0.0, "tok_checked": 0,
-                      "tok_skipped": 0}
+                      "tok_skipped": 0, "max_flush": 0, "flushes": 0}
 
     def prefill(self, prompts):
         """prompts: full prompts; the last token of each is kept as the first step's input."""
@@ -56,6 +56,7 @@ class Pair:
     def step(self, mods, ctrs, slots=None):
         slots = list(range(self.n)) if slots is None else list(slots)
         k = len(slots)
+        pend_before = [len(self.os[s].pending) if s in self.checked else 0 for s in slots]
         ref = [self.os[s].decode_step(self.next_in[s], mods[i], ctrs[i]) if s in self.checked else None
                for i, s in enumerate(slots)]
         self.tok[:k] = torch.tensor([self.next_in[s] for s in slots], dtype=torch.int32)
@@ -77,11 +78,17 @@ class Pair:
                 # unchecked sequence: its depth still has to follow the schedule; it runs on
                 # the token the library produced
                 te = self.dims.get("text_exit", 0)
-                want = L if ((mods[i] == 0 and te == 0) or (mods[i] == 1 and te == 2)) else (L if ctrs[i] % K == r_ else e)
+                Km, rm = (self.dims["text_period"], self.dims.get("text_phase", 0)) \
+                    if mods[i] == 0 and self.dims.get("text_period", 0) > 0 else (K, r_)
+                want = L if ((mods[i] == 0 and te == 0) or (mods[i] == 1 and te == 2)) else (L if ctrs[i] % Km == rm else e)
                 assert got_dep[i] == want, (i, got_dep[i], want)
                 self.next_in[s] = int(got_tok[i])
                 continue
             assert got_dep[i] == r["depth"], (i, got_dep[i], r["depth"])
+            if r["depth"] == L and e < L and pend_before[i]:
+                # a full-depth step that pushed pending rows through the upper layers with its own
+                self.stats["flushes"] += 1
+                self.stats["max_flush"] = max(self.stats["max_flush"], pend_before[i])
             eh = rel_err(H[i], r["hidden"])
             lo, hi = (0, Vt) if mods[i] == 0 else (Vt, V)
             ez = rel_err(Z[i][lo:hi], r["logits"][lo:hi])

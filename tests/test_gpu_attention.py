@@ -10,12 +10,12 @@ REL_TOL = 2e-2
 
 
 def make_case(seed, n_slots, Hq, Hkv, hd, S, groups):
-    """groups: list of (slot, pos0, nrows).  Returns numpy inputs (bf16-rounded float64) and tensors."""
+    """groups: list of (slot, pos0, nrows).  Queries rounded to bf16, keys and values to fp16."""
     g = torch.Generator("cpu").manual_seed(seed)
     n_rows = sum(n for _, _, n in groups)
     q = torch.randn((n_rows, Hq * hd), generator=g).to(torch.bfloat16)
-    k = torch.randn((n_slots, Hkv, S, hd), generator=g).to(torch.bfloat16)
-    v = torch.randn((n_slots, Hkv, S, hd), generator=g).to(torch.bfloat16)
+    k = torch.randn((n_slots, Hkv, S, hd), generator=g).to(torch.float16)    # the cache's element type
+    v = torch.randn((n_slots, Hkv, S, hd), generator=g).to(torch.float16)
     row_slot, row_pos, g0, gn = [], [], [], []
     for slot, pos0, n in groups:
         g0.append(len(row_slot)); gn.append(n)

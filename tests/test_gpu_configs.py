@@ -1,8 +1,10 @@
 """GPU parity at the full model shapes of the five workloads (launch configuration of bench.py).
 
-The oracle cannot afford a prompt of hundreds of tokens at these shapes, so every sequence
-starts from a cache of stand-in values (synth.synth_kv) loaded into both sides; from there the
+The oracle cannot afford prompts of many hundreds of tokens at these shapes, so the workload runs
+start from a cache of stand-in values (synth.synth_kv) loaded into both sides; from there the
 library and the oracle run the same interleaved steps, teacher-forced on the oracle's tokens.
+Real prefill at these shapes is compared on prompts of 131 tokens (two full chunks of 64 rows and
+a ragged third).
 With a batch the oracle follows a seeded subset of the sequences (sequences are independent,
 which the small-shape tests establish); the other sequences run free and are held to the exit
 schedule only.  Acceptance rules are those of parity_util: depths bit-exact, hidden states and
@@ -57,7 +59,8 @@ def _load_cache(P, lens, checked, dims, shared_seed=77):
     L = dims["n_layers"]
     n_max = max(lens)
     shared_k, shared_v = synth.synth_kv(dims, n_max, seed=shared_seed)
-    dev = lambda a: torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+    # stand-in values are bf16 bit patterns; the cache holds fp16, which represents them exactly
+    dev = lambda a: torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16).to(torch.float16)
     for layer in range(1, L + 1):
         kt, vt = dev(shared_k[layer - 1]), dev(shared_v[layer - 1])
         for s, n in enumerate(lens):
@@ -104,33 +107,80 @@ def _run(model, wl_name, steps, g0, n_checked, lens=None, exit_layer=None, perio
 
 
 def test_config2_step_shape_batch1(step_model):
-    """Workload 2: Step-shaped, batch 1, cache of 511 positions, two interleave cycles
-    (text, refresh, three early exits; the second cycle's text step flushes three pending rows)."""
-    st = _run(step_model, "cfg2_step_b1", steps=10, g0=0, n_checked=1)
+    """Workload 2: Step-shaped, batch 1, cache of 511 positions, the first 256 decode steps of
+    the workload's 1024 (51 interleave cycles: text, refresh, three early exits; every cycle's
+    text step pushes three pending rows through the upper layers with its own)."""
+    st = _run(step_model, "cfg2_step_b1", steps=256, g0=0, n_checked=1)
     print("cfg2", st)
-    assert st["tok_checked"] >= 5
+    assert st["steps"] == 256 and st["tok_checked"] >= 128
+    assert st["max_flush"] == 3 and st["flushes"] >= 50
 
 
 def test_config3_step_shape_batch64(step_model):
     """Workload 3: batch 64, ragged caches of 256..2048 positions, random interleave phases and
-    counter offsets so every step mixes depths; the oracle follows two of the sequences."""
+    counter offsets so every step mixes depths; the oracle follows two of the sequences for two
+    interleave cycles."""
     st = _run(step_model, "cfg3_step_b64", steps=10, g0=0, n_checked=2)
     print("cfg3", st)
     assert st["mixed_steps"] >= 8
+    assert st["flushes"] >= 2
 
 
 def test_config4_glm_shape_batch16(glm_model):
-    """Workload 4: GLM-shaped, batch 16, caches of 1023 positions, phase-aligned 13:26 interleave;
-    steps 11..20 cover the end of a text chunk, two refreshes and a flush of three pending rows."""
-    st = _run(glm_model, "cfg4_glm_b16", steps=10, g0=11, n_checked=2)
+    """Workload 4: GLM-shaped, batch 16, caches of 1023 positions, phase-aligned 13:26 interleave,
+    two whole interleave cycles (78 steps): text chunks, refreshes every fourth speech position
+    with three pending rows each, and the text step after a chunk that ends on an early exit."""
+    st = _run(glm_model, "cfg4_glm_b16", steps=78, g0=0, n_checked=2)
     print("cfg4", st)
+    assert st["steps"] == 78 and st["max_flush"] == 3 and st["flushes"] >= 24
 
 
 def test_config5_glm_shape_long_context(glm_model):
     """Workload 5 (long-context stress): caches of 8191 positions; batch 128 with the oracle on
-    two sequences, for the e=30, K=4 cell."""
-    st = _run(glm_model, "cfg5_glm_b128", steps=6, g0=12, n_checked=2, lens=[8191] * 128)
+    two sequences, for the e=30, K=4 cell, two whole interleave cycles (78 steps) with random
+    phases, so the checked sequences refresh with three pending rows while others sit at any
+    other point of their cycle."""
+    st = _run(glm_model, "cfg5_glm_b128", steps=78, g0=0, n_checked=2, lens=[8191] * 128)
     print("cfg5", st)
+    assert st["steps"] == 78 and st["max_flush"] == 3 and st["flushes"] >= 20
+
+
+def _real_prefill(model, wl_name, prompt_len):
+    """A prompt long enough for two full 64-row prefill chunks and a ragged third, ingested by
+    sparsk_prefill (the tcgen05 GEMMs and the tcgen05 attention kernel at blocks of hundreds of
+    query vectors per kv head) and by the oracle; the cache of every layer is compared, then one
+    interleave cycle runs on top of it."""
+    from tests import parity_util as pu
+    wl = synth.WORKLOADS[wl_name]
+    dims = synth.model_dims(model.shape, wl["exit_layer"], wl["refresh_period"], wl["refresh_phase"])
+    K = wl["refresh_period"]
+    cyc = wl["n_text"] + wl["n_speech"]
+    prompt = synth.make_prompts(dims, 1, prompt_len, prompt_len, seed=21)[0]
+    P = pu.Pair(dims, model.w, 1, prompt_len + cyc + 3, max(K - 1, 1), prefill_rows=64, gw=model.gw)
+    P.prefill([prompt])
+    assert P.g.slot_state(0) == (prompt_len - 1, 0)
+    P.check_cache(0, range(1, dims["n_layers"] + 1), prompt_len - 1)
+    for g in range(cyc + 1):       # one whole cycle and the text step that follows it (it flushes the chunk's tail)
+        m, c = synth.interleave(g, wl["n_text"], wl["n_speech"])
+        P.step([m], [c])
+    ln, pend = P.g.slot_state(0)
+    P.check_cache(0, range(1, dims["exit_layer"] + 1), ln)
+    P.check_cache(0, range(dims["exit_layer"] + 1, dims["n_layers"] + 1), ln - pend)
+    st = dict(P.stats)
+    P.close()
+    return st
+
+
+def test_real_prefill_step_shape(step_model):
+    st = _real_prefill(step_model, "cfg2_step_b1", 131)
+    print("prefill step", st)
+    assert st["steps"] == 6 and st["max_flush"] == 3
+
+
+def test_real_prefill_glm_shape(glm_model):
+    st = _real_prefill(glm_model, "cfg4_glm_b16", 131)
+    print("prefill glm", st)
+    assert st["steps"] == 40 and st["max_flush"] == 3
 
 
 @pytest.mark.parametrize("e", [20, 30, 40])

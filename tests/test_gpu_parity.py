@@ -60,34 +60,20 @@ def test_odd_shapes_and_schedules(util, e, K, r, nt, ns, min_rows):
     P.close()
 
 
-def test_odd_shapes_persistent_tensor_core_kernel(util):
-    """head_dim 64, three query heads per kv head, inner dimensions that are not multiples of 64:
-    every pass (1..5 rows, 16-row prefill chunks) through the persistent tensor-core kernel."""
-    dims = synth.model_dims(MICRO64, 2, 4, 1)
-    w = synth.make_weights(dims, seed=5)
-    prompt = synth.make_prompts(dims, 1, 37, 37, seed=7)[0]
-    P = util.Pair(dims, w, 1, 128, 8, prefill_rows=16, options={"tcmega": 1, "mega": 0, "gemm_min_rows": 1})
-    P.prefill([prompt])
-    for g in range(40):
-        m, c = synth.interleave(g, 2, 7)
-        P.step([m], [c])
-    P.check_cache(0, range(1, 4), P.g.slot_state(0)[0] - P.g.slot_state(0)[1])
-    P.close()
-
-
-@pytest.mark.parametrize("min_rows,tcmega", [(3, 0), (1, 0), (1 << 30, 0), (3, 1)])
-def test_heterogeneous_batch_matches_per_sequence_oracle(util, min_rows, tcmega):
+@pytest.mark.parametrize("min_rows,trim", [(3, 1), (1, 2), (1 << 30, 2), (3, 0), (3, 2)])
+def test_heterogeneous_batch_matches_per_sequence_oracle(util, min_rows, trim):
     """Batch of 7 with random interleave phases and counter offsets and ragged prompts, so every
     step mixes text, early-exit and refresh rows; sequences stay independent.  Run with the
     default hand-over between the small-batch and the tensor-core path (3 rows), with every
-    projection on the tensor cores, with every projection on the small-batch path, and with the
-    tensor-core layers as one persistent kernel per layer range."""
+    projection on the tensor cores, and with every projection on the small-batch path; and with the pending rows leaving
+    the last layer after its K/V projection (trim 2: always, 1: when it pays, 0: never), which
+    must change nothing: the cache of every layer is compared below."""
     dims = synth.model_dims("tiny", 2, 4, 0)
     w = synth.make_weights(dims, seed=0)
     B = 7
     prompts = synth.make_prompts(dims, B, 9, 70, seed=4)
     phi, off = synth.make_phases(B, 1, 4, 4, True, seed=8)
-    P = util.Pair(dims, w, B, 70 + 64, 3, prefill_rows=24, options={"gemm_min_rows": min_rows, "tcmega": tcmega})
+    P = util.Pair(dims, w, B, 70 + 64, 3, prefill_rows=24, options={"gemm_min_rows": min_rows, "trim_last_layer": trim})
     P.prefill(prompts)
     mixed = 0
     for g in range(48):
@@ -167,8 +153,8 @@ def test_imported_cache_long_context(util):
     P = util.Pair(dims, w, 2, n + 40, 3)
     from oracle.bruteforce import bf16_to_f64
     for layer in range(1, 5):
-        kt = torch.from_numpy(k[layer - 1].view(np.int16)).cuda().view(torch.bfloat16)
-        vt = torch.from_numpy(v[layer - 1].view(np.int16)).cuda().view(torch.bfloat16)
+        kt = torch.from_numpy(k[layer - 1].view(np.int16)).cuda().view(torch.bfloat16).to(torch.float16)
+        vt = torch.from_numpy(v[layer - 1].view(np.int16)).cuda().view(torch.bfloat16).to(torch.float16)
         for s in range(2):
             P.g.import_kv(s, layer, 0, kt, vt)
         kf, vf = bf16_to_f64(k[layer - 1]), bf16_to_f64(v[layer - 1])
@@ -210,9 +196,12 @@ def test_host_step_and_error_codes(util):
         P.g.decode_step_host([0, 1], [5, 6], [1, 1], [2, 2], nt, dp)
     assert ei.value.code == binding.ECAPACITY
     assert [P.g.slot_state(s) for s in range(2)] == [(b[0] + 1, 1) for b in before]
-    with pytest.raises(binding.SparskError) as ei:      # token outside the vocabulary
+    before = [P.g.slot_state(s) for s in range(2)]
+    with pytest.raises(binding.SparskError) as ei:      # token outside the vocabulary: refused on the host
         P.g.decode_step_host([0], [10 ** 6], [0], [0], nt, dp)
     assert ei.value.code == binding.EINVAL
+    assert [P.g.slot_state(s) for s in range(2)] == before      # nothing ran, nothing advanced
+    P.g.check()
     P.close()
     # a schedule that needs a head that was not supplied
     d2 = synth.model_dims("tiny", 3, 3, 0)
@@ -224,12 +213,12 @@ def test_host_step_and_error_codes(util):
 
 @pytest.mark.parametrize("options", [{"mega": 0}, {"mega_max_rows": 4}, {"mega_max_rows": 1, "gemm_min_rows": 2},
                                      {"mega": 0, "gemm_min_rows": 1 << 30}, {"gemm_kb": 1, "mega": 0, "gemm_min_rows": 1},
-                                     {"tcmega": 1}, {"tcmega": 1, "mega": 0, "gemm_min_rows": 1}])
+                                     {"trim_last_layer": 2}, {"trim_last_layer": 2, "mega": 0, "gemm_min_rows": 1},
+                                     {"trim_last_layer": 2, "mega": 0, "gemm_min_rows": 1 << 30}, {"trim_last_layer": 0}])
 def test_every_route_for_small_passes(util, options):
     """Passes of 1..4 rows (K = 4: flushes of up to three pending rows) through each of the
     implementations: the persistent kernel (also with its moving activation window at 3-4 rows),
-    the tensor-core path (with 2-D descriptors too, and as one persistent kernel per layer range)
-    and the small-batch kernels."""
+    the tensor-core path (with 2-D descriptors too) and the small-batch kernels."""
     dims = synth.model_dims("tiny", 2, 4, 0)
     w = synth.make_weights(dims, seed=0)
     prompt = synth.make_prompts(dims, 1, 21, 21, seed=11)[0]
@@ -237,6 +226,42 @@ def test_every_route_for_small_passes(util, options):
     P.prefill([prompt])
     for g in range(25):
         m, c = synth.interleave(g, 1, 4)
+        P.step([m], [c])
+    ln, pend = P.g.slot_state(0)
+    P.check_cache(0, range(1, 5), ln - pend)
+    P.close()
+
+
+def test_timeout_is_reported_once_and_the_context_recovers(util):
+    """A bounded in-kernel wait that runs out: the persistent kernel is told a grid-barrier count
+    that no CTA can reach (a host-side test hook; nothing faults or hangs), its wait ends at the
+    wall-clock limit, every CTA leaves, and the step returns SPARSK_ETIMEOUT exactly once.  The
+    library then resets its barrier state by itself: after the caller resets the slot that took
+    part, decoding matches the oracle again."""
+    from paper_2603_09215_b200 import binding
+    dims = synth.model_dims("tiny", 2, 3, 0)
+    w = synth.make_weights(dims, seed=0)
+    prompt = synth.make_prompts(dims, 1, 14, 14, seed=5)[0]
+    P = util.Pair(dims, w, 1, 64, 2)
+    P.prefill([prompt])
+    for g in range(4):
+        m, c = synth.interleave(g, 2, 4)
+        P.step([m], [c])
+    assert P.g.route_counts()["mega"] > 0                 # the steps above ran in the persistent kernel
+    nt, dp = np.zeros(1, np.int32), np.zeros(1, np.int32)
+    P.g.set_option("inject_barrier_timeout", 1)
+    with pytest.raises(binding.SparskError) as ei:
+        P.g.decode_step_host([0], [P.next_in[0]], [1], [0], nt, dp)
+    assert ei.value.code == binding.ETIMEOUT
+    P.g.check()                                           # reported once; the status word is clear again
+    # the interrupted step left slot 0 incomplete: start it over on both sides
+    P.g.reset_slot(0)
+    P.os[0] = P.om.new_seq(2)
+    P.g.prefill([0], [prompt[:-1]])
+    P.os[0].prefill(prompt[:-1])
+    P.next_in[0] = int(prompt[-1])
+    for g in range(12):
+        m, c = synth.interleave(g, 2, 4)
         P.step([m], [c])
     ln, pend = P.g.slot_state(0)
     P.check_cache(0, range(1, 5), ln - pend)

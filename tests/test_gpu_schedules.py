@@ -79,3 +79,36 @@ def test_text_side_schedule_in_a_mixed_batch(util):
         P.check_cache(s, range(1, 3), ln)
         P.check_cache(s, range(3, 5), ln - pend)
     P.close()
+
+
+@pytest.mark.parametrize("text_exit,K,r,tp,tr,nt,ns,maxp", [
+    (1, 4, 0, 3, 1, 6, 8, 5),     # speech Triple-like (K = 4), text with period 3 and phase 1
+    (2, 2, 0, 3, 2, 6, 2, 3),     # text only with its own period; speech steps are full depth
+])
+def test_period_and_phase_per_modality(util, text_exit, K, r, tp, tr, nt, ns, maxp):
+    """Sec. V-E: text and speech may need different policies.  Each modality follows the periodic
+    rule with its own (period, phase); pending rows of either modality are pushed through the
+    upper layers by the next full-depth step of either."""
+    dims = synth.model_dims("tiny", 2, K, r, text_exit=text_exit, text_period=tp, text_phase=tr)
+    w = synth.make_weights(dims, seed=0)
+    B = 3
+    prompts = synth.make_prompts(dims, B, 10, 30, seed=17)
+    P = util.Pair(dims, w, B, 30 + 64, maxp, prefill_rows=16)
+    P.prefill(prompts)
+    L, e = dims["n_layers"], dims["exit_layer"]
+    phases = [0, 5, 9]
+    for g in range(42):
+        mc = [synth.interleave(g, nt, ns, ph) for ph in phases]
+        mods, ctrs = [m for m, _ in mc], [c for _, c in mc]
+        _, _, dep = P.step(mods, ctrs)
+        for m, c, d in zip(mods, ctrs, dep):
+            if m == 0:
+                assert d == (L if c % tp == tr else e)
+            else:
+                assert d == (L if (text_exit == 2 or c % K == r) else e)
+    for s in range(B):
+        ln, pend = P.g.slot_state(s)
+        P.check_cache(s, range(1, e + 1), ln)
+        P.check_cache(s, range(e + 1, L + 1), ln - pend)
+    assert P.stats["flushes"] > 5 and P.stats["tok_checked"] > 10, P.stats
+    P.close()

@@ -4,7 +4,8 @@ Some users of this library run where no allocator can be called: inside another 
 memory plan, or on a path where cudaMalloc is off limits because it synchronises the device.
 sparsk_attention_static serves them from a scratch area built into the library.  This test calls
 it through the C ABI, twice in a row on different inputs (the area keeps the first call's
-contents), and checks each result against sparsk_attention run with caller-provided scratch.
+contents), and checks each result against sparsk_attention run with caller-provided scratch and
+against the CPU oracle's softmax attention.
 It lives in a file that is collected last, and passes both alone and after the other tests.
 """
 import numpy as np
@@ -47,11 +48,18 @@ def test_static_scratch_attention_matches_the_allocating_entry_point():
     from paper_2603_09215_b200 import binding
     first = _case(11, [(0, 700, 4), (1, 64, 1), (2, 333, 2)])
     second = _case(12, [(1, 10, 1), (0, 850, 3)])            # fewer rows, other lengths: stale cells remain
+    from tests.test_gpu_attention import oracle_out
     for c in (first, second):
         ref = _run(binding, c, static=False)
         got = _run(binding, c, static=True)
         assert np.isfinite(got).all()
         err = np.abs(got - ref).max() / np.abs(ref).max()
+        assert err <= REL_TOL, err
+        # and directly against the CPU oracle's softmax attention, row by row and head by head
+        _, _, Hq, hd = c["meta"]
+        want = oracle_out(c["q"].cpu(), c["k"].cpu(), c["v"].cpu(), c["rs"].cpu().tolist(), c["rp"].cpu().tolist(),
+                          Hq, c["k"].shape[1], hd)
+        err = np.abs(got - want).max() / np.abs(want).max()
         assert err <= REL_TOL, err
     # a call whose partials do not fit the built-in area is refused, with the sizes in the message
     big = _case(13, [(0, 0, 1)], Hq=32, Hkv=2, hd=128, S=8)
