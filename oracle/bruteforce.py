@@ -94,24 +94,47 @@ def scheduled_depth(dims: dict, modality: int, c: int) -> int:
     return L if c % K == r else e
 
 
-def decode_stream(dims: dict, w: dict, prompt, modalities, counters, forced=None):
+def entropy(z: np.ndarray) -> float:
+    """Entropy (nats) of softmax(z) (Sec. V-B: the confidence signal of the compared method)."""
+    lp = z - z.max()
+    lp = lp - np.log(np.exp(lp).sum())
+    p = np.exp(lp)
+    return float(-(p[p > 0] * lp[p > 0]).sum())
+
+
+def decode_stream(dims: dict, w: dict, prompt, modalities, counters, forced=None, depths=None):
     """Greedy SPAR-K generation by full recomputation.  `prompt` is the whole prompt (the last
     prompt token is the first step's input).  If `forced` is given its tokens are fed back
-    instead of the computed ones (teacher forcing).  Returns a list of per-step dicts."""
+    instead of the computed ones (teacher forcing).  Returns a list of per-step dicts.
+
+    The depth of a step is `depths[s]` if given; else, for a modality in dims["conf_modalities"]
+    (bit 0 text, bit 1 speech), the first layer l >= conf_start whose head's prediction over the
+    modality's ids has entropy < conf_threshold (L if none; Sec. V-B); else the schedule's."""
     toks = list(np.asarray(prompt))
     Vt = dims["vocab_text"]
     V = Vt + dims["vocab_speech"]
     out = []
     for s, (mod, c) in enumerate(zip(modalities, counters)):
-        dep = scheduled_depth(dims, int(mod), int(c))
         fw = forward_all(dims, w, toks)
         p = len(toks) - 1
+        lo, hi = (0, Vt) if mod == 0 else (Vt, V)
+        ents = {}
+        if depths is not None:
+            dep = int(depths[s])
+        elif (dims.get("conf_modalities", 0) >> (1 if mod else 0)) & 1:
+            dep = dims["n_layers"]
+            for l in range(dims["conf_start"], dims["n_layers"]):
+                ents[l] = entropy(head_logits(dims, w, l, fw["H"][l, p])[lo:hi])
+                if ents[l] < dims["conf_threshold"]:
+                    dep = l
+                    break
+        else:
+            dep = scheduled_depth(dims, int(mod), int(c))
         hid = fw["H"][dep, p]
         z = head_logits(dims, w, dep, hid)
-        lo, hi = (0, Vt) if mod == 0 else (Vt, V)
         y = lo + int(np.argmax(z[lo:hi]))
         zs = np.sort(z[lo:hi])
         out.append({"token": y, "depth": dep, "hidden": hid, "logits": z, "pos": p,
-                    "margin": float(zs[-1] - zs[-2])})
+                    "margin": float(zs[-1] - zs[-2]), "entropies": ents})
         toks.append(int(forced[s]) if forced is not None else y)
     return out

@@ -22,7 +22,8 @@ class _Dims(C.Structure):
                                          "head_dim", "d_ffn", "vocab_text", "vocab_speech")] + [
         ("rms_eps", C.c_double), ("rope_base", C.c_double)] + [
         (n, C.c_int32) for n in ("exit_layer", "refresh_period", "refresh_phase", "text_exit",
-                                 "max_len", "text_period", "text_phase")]
+                                 "max_len", "text_period", "text_phase", "conf_modalities",
+                                 "conf_start")] + [("conf_threshold", C.c_double)]
 
 
 _PP = C.POINTER(C.c_void_p)
@@ -76,6 +77,14 @@ def lib():
         L.ora_decode_step.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                       C.POINTER(C.c_int32), C.POINTER(C.c_int32),
                                       C.POINTER(C.c_double), C.c_void_p, C.c_void_p]
+        L.ora_seq_pending_fill.restype = C.c_int32
+        L.ora_seq_pending_fill.argtypes = [C.c_void_p, C.c_int32]
+        L.ora_entropy.restype = C.c_double
+        L.ora_entropy.argtypes = [C.c_void_p, C.c_int32]
+        L.ora_decode_step_dyn.restype = C.c_int32
+        L.ora_decode_step_dyn.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                          C.POINTER(C.c_int32), C.POINTER(C.c_int32),
+                                          C.POINTER(C.c_double), C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -87,6 +96,12 @@ def depth(modality: int, c: int, K: int, r: int, e: int, L: int, text_exit: int 
 def depth_mod(modality: int, c: int, K_s: int, r_s: int, K_t: int, r_t: int, e: int, L: int,
               text_exit: int) -> int:
     return lib().ora_depth_mod(modality, c, K_s, r_s, K_t, r_t, e, L, text_exit)
+
+
+def entropy(z) -> float:
+    """Entropy (nats) of softmax(z)."""
+    z = np.ascontiguousarray(z, dtype=np.float64)
+    return lib().ora_entropy(z.ctypes.data, z.size)
 
 
 def _u16(a) -> np.ndarray:
@@ -133,6 +148,9 @@ class OracleModel:
         d.text_exit = int(dims.get("text_exit", 0))
         d.text_period = int(dims.get("text_period", 0))
         d.text_phase = int(dims.get("text_phase", 0))
+        d.conf_modalities = int(dims.get("conf_modalities", 0))
+        d.conf_start = int(dims.get("conf_start", 0))
+        d.conf_threshold = float(dims.get("conf_threshold", 0.0))
         d.rms_eps = float(dims["rms_eps"])
         d.rope_base = float(dims["rope_base"])
         d.max_len = int(max_len)
@@ -192,6 +210,12 @@ class OracleSeq:
         n = lib().ora_seq_pending(self._h)
         return [lib().ora_seq_pending_pos(self._h, j) for j in range(n)]
 
+    @property
+    def pending_fill(self) -> list:
+        """For each pending position, the layer its K/V is complete up to."""
+        n = lib().ora_seq_pending(self._h)
+        return [lib().ora_seq_pending_fill(self._h, j) for j in range(n)]
+
     def get_kv(self, layer: int, pos: int):
         k = np.empty(self.model.kv_row)
         v = np.empty(self.model.kv_row)
@@ -224,3 +248,19 @@ class OracleSeq:
             raise RuntimeError(f"oracle decode_step failed ({rc})")
         return {"token": nt.value, "depth": dp.value, "margin": mg.value, "hidden": hid,
                 "logits": lg}
+
+    def decode_step_dyn(self, token: int, modality: int, counter: int, forced_depth: int = 0,
+                        want_logits: bool = True):
+        """A step whose depth is dictated (forced_depth in 1..L) or decided on the way by the
+        confidence rule of the dims (forced_depth = 0)."""
+        nt, dp, mg = C.c_int32(), C.c_int32(), C.c_double()
+        hid = np.empty(self.model.d_model)
+        lg = np.empty(self.model.V) if want_logits else None
+        ent = np.empty(max(1, self.model.dims["n_layers"] - 1))
+        rc = lib().ora_decode_step_dyn(self._h, int(token), int(modality), int(counter), int(forced_depth),
+                                       C.byref(nt), C.byref(dp), C.byref(mg), hid.ctypes.data,
+                                       lg.ctypes.data if want_logits else None, ent.ctypes.data)
+        if rc:
+            raise RuntimeError(f"oracle decode_step_dyn failed ({rc})")
+        return {"token": nt.value, "depth": dp.value, "margin": mg.value, "hidden": hid,
+                "logits": lg, "entropies": ent}

@@ -61,6 +61,15 @@ typedef struct {
                                (text_exit 1 or 2); 0: the same K and r as speech:
                                the modalities may need different policies (Sec. V-E) */
     int32_t text_phase;     /* r of text positions, in [0, text_period)           */
+    /* Confidence-based early exit (Sec. V-B, compared method 3; thresholds in Sec. VI):
+     * positions of the modalities in conf_modalities (bit 0 text, bit 1 speech) ignore the
+     * schedule; from layer conf_start on, the head of each layer is applied to the position's
+     * hidden state, and the position exits at the first layer whose prediction has an
+     * entropy below conf_threshold (natural logarithm, over the ids of the modality being
+     * emitted); if none does, it runs all L layers. */
+    int32_t conf_modalities;
+    int32_t conf_start;     /* first layer whose head is consulted, 1..L-1        */
+    double conf_threshold;
 } ora_dims;
 
 typedef struct {
@@ -89,6 +98,9 @@ typedef struct {
     int32_t n_pending; /* |P|                                                     */
     int32_t *pend_pos; /* positions in P, ascending                               */
     double *pend_h;    /* h^(l_EE) of each pending position, [max_pending][d]     */
+    int32_t *pend_fill; /* layers whose K/V the pending position already has (the
+                           layer it left at, or a later one it was carried to); the
+                           scheduled decoder only ever stores l_EE here           */
     int32_t max_pending;
     double *K, *V;     /* [L][max_len][Hkv*hd], keys stored after rotation        */
 } ora_seq;
@@ -220,10 +232,11 @@ ora_seq *ora_seq_new(const ora_model *m, int32_t max_pending)
     s->max_pending = max_pending < 1 ? 1 : max_pending;
     s->pend_pos = (int32_t *)calloc((size_t)s->max_pending, sizeof(int32_t));
     s->pend_h = (double *)calloc((size_t)s->max_pending * dm->d_model, sizeof(double));
+    s->pend_fill = (int32_t *)calloc((size_t)s->max_pending, sizeof(int32_t));
     size_t kv = (size_t)dm->n_layers * dm->max_len * dm->n_kv_heads * dm->head_dim;
     s->K = (double *)calloc(kv, sizeof(double));
     s->V = (double *)calloc(kv, sizeof(double));
-    if (!s->pend_pos || !s->pend_h || !s->K || !s->V) return NULL;
+    if (!s->pend_pos || !s->pend_h || !s->pend_fill || !s->K || !s->V) return NULL;
     return s;
 }
 
@@ -232,6 +245,7 @@ void ora_seq_free(ora_seq *s)
     if (!s) return;
     free(s->pend_pos);
     free(s->pend_h);
+    free(s->pend_fill);
     free(s->K);
     free(s->V);
     free(s);
@@ -240,6 +254,7 @@ void ora_seq_free(ora_seq *s)
 int32_t ora_seq_len(const ora_seq *s) { return s->len; }
 int32_t ora_seq_pending(const ora_seq *s) { return s->n_pending; }
 int32_t ora_seq_pending_pos(const ora_seq *s, int32_t j) { return s->pend_pos[j]; }
+int32_t ora_seq_pending_fill(const ora_seq *s, int32_t j) { return s->pend_fill[j]; }
 
 static double *kv_at(double *base, const ora_dims *dm, int layer /*1-based*/, int pos)
 {
@@ -428,6 +443,7 @@ int32_t ora_decode_step(ora_seq *s, int32_t token, int32_t modality, int32_t cou
     if (dep < L) {
         /* early exit: keep h^(l_EE), defer the upper K/V, read the token from g_{l_EE} */
         s->pend_pos[s->n_pending] = p;
+        s->pend_fill[s->n_pending] = e;
         memcpy(s->pend_h + (size_t)s->n_pending * d, h, sizeof(double) * d);
         s->n_pending++;
         *next_token = head_argmax(m, e, h, modality, logits, margin);
@@ -454,5 +470,131 @@ int32_t ora_decode_step(ora_seq *s, int32_t token, int32_t modality, int32_t cou
     *depth = dep;
     s->len = p + 1;
     free(h);
+    return 0;
+}
+
+/* ---------------------------------------------------------------- exits at any layer */
+
+/* Entropy (natural logarithm) of softmax(z[0..n)).  Sec. V-B: the confidence signal of the
+ * compared method is the entropy of the layer's next-token distribution. */
+double ora_entropy(const double *z, int32_t n)
+{
+    double mx = -INFINITY;
+    for (int i = 0; i < n; i++)
+        if (z[i] > mx) mx = z[i];
+    double sum = 0.0;
+    for (int i = 0; i < n; i++) sum += exp(z[i] - mx);
+    double h = 0.0;
+    for (int i = 0; i < n; i++) {
+        double p = exp(z[i] - mx) / sum;
+        if (p > 0.0) h -= p * log(p);
+    }
+    return h;
+}
+
+/*
+ * One decoding step whose depth is not known beforehand: either dictated by the caller
+ * (forced_depth in 1..L: any layer that has a head) or decided on the way by the confidence
+ * rule of the dims (forced_depth = 0; positions of a modality outside conf_modalities follow
+ * the schedule as in ora_decode_step).
+ *
+ * Deferred filling, stated for exits at arbitrary layers (Sec. IV-B.3 states it for one exit
+ * layer; the rule is the same): a position that left at layer f lacks K/V above f.  Whenever a
+ * later position is about to run a layer l > f, the earlier one is taken along through l in
+ * the same causal block, so that every position attends to complete K/V at every layer it
+ * runs.  A pending position therefore records how far it has been carried (pend_fill) and the
+ * hidden state at that layer; a step that runs all L layers completes and drops them all.
+ * With a single exit layer this is exactly Algorithm 1.
+ *
+ * entropies (may be NULL) receives, for layer l = 1..L-1, the entropy computed at that layer
+ * or -1 where no head was consulted.
+ */
+int32_t ora_decode_step_dyn(ora_seq *s, int32_t token, int32_t modality, int32_t counter,
+                            int32_t forced_depth, int32_t *next_token, int32_t *depth,
+                            double *margin, double *hidden, double *logits, double *entropies)
+{
+    const ora_model *m = s->m;
+    const ora_dims *dm = &m->dm;
+    const int d = dm->d_model, L = dm->n_layers;
+    const int V = dm->vocab_text + dm->vocab_speech;
+    if (s->len >= dm->max_len) return -1;
+    if (forced_depth < 0 || forced_depth > L) return -3;
+    const int by_conf = forced_depth == 0 && ((dm->conf_modalities >> (modality ? 1 : 0)) & 1);
+    int target = forced_depth;   /* 0: decided by confidence */
+    if (forced_depth == 0 && !by_conf) {
+        const int K_t = dm->text_period > 0 ? dm->text_period : dm->refresh_period;
+        const int r_t = dm->text_period > 0 ? dm->text_phase : dm->refresh_phase;
+        target = ora_depth_mod(modality, counter, dm->refresh_period, dm->refresh_phase, K_t, r_t,
+                               dm->exit_layer, L, dm->text_exit);
+    }
+    if (target && (!m->w.head_norm[target - 1] || !m->w.head_proj[target - 1])) return -2;
+    if (by_conf && (dm->conf_start < 1 || dm->conf_start >= L)) return -3;
+    if (s->n_pending >= s->max_pending) return -1;   /* the step may add one */
+    if (entropies)
+        for (int l = 1; l < L; l++) entropies[l - 1] = -1.0;
+
+    const int32_t p = s->len;
+    const int n_max = s->n_pending + 1;
+    double *H = (double *)malloc(sizeof(double) * (size_t)n_max * d);
+    double *Hb = (double *)malloc(sizeof(double) * (size_t)n_max * d);
+    int32_t *pos = (int32_t *)malloc(sizeof(int32_t) * (size_t)n_max);
+    int32_t *who = (int32_t *)malloc(sizeof(int32_t) * (size_t)n_max);
+    double *z = (double *)malloc(sizeof(double) * (size_t)V);
+    /* row j < n_pending: pending position j at the layer it has been carried to; last row: the
+     * new position */
+    for (int j = 0; j < s->n_pending; j++) memcpy(H + (size_t)j * d, s->pend_h + (size_t)j * d, sizeof(double) * d);
+    double *hc = H + (size_t)s->n_pending * d;
+    embed_row(m, token, hc);
+
+    int dep = 0;
+    for (int l = 1; l <= L; l++) {
+        /* the block of this layer: pending positions not yet carried through l, then the new one */
+        int n = 0;
+        for (int j = 0; j < s->n_pending; j++)
+            if (s->pend_fill[j] < l) {
+                pos[n] = s->pend_pos[j];
+                who[n] = j;
+                memcpy(Hb + (size_t)n * d, H + (size_t)j * d, sizeof(double) * d);
+                n++;
+            }
+        pos[n] = p;
+        who[n] = s->n_pending;
+        memcpy(Hb + (size_t)n * d, hc, sizeof(double) * d);
+        n++;
+        layer_block(s, l, pos, n, Hb);
+        for (int i = 0; i < n; i++) memcpy(H + (size_t)who[i] * d, Hb + (size_t)i * d, sizeof(double) * d);
+        for (int j = 0; j < s->n_pending; j++)
+            if (s->pend_fill[j] < l) s->pend_fill[j] = l;
+        dep = l;
+        if (target) {
+            if (l == target) break;
+        } else if (l >= dm->conf_start && l < L) {
+            if (!m->w.head_norm[l - 1] || !m->w.head_proj[l - 1]) {
+                free(H); free(Hb); free(pos); free(who); free(z);
+                return -2;
+            }
+            head_argmax(m, l, hc, modality, z, NULL);
+            const int lo = modality == 0 ? 0 : dm->vocab_text;
+            const int hi = modality == 0 ? dm->vocab_text : V;
+            const double ent = ora_entropy(z + lo, hi - lo);
+            if (entropies) entropies[l - 1] = ent;
+            if (ent < dm->conf_threshold) break;
+        }
+    }
+    *next_token = head_argmax(m, dep, hc, modality, logits, margin);
+    if (hidden) memcpy(hidden, hc, sizeof(double) * d);
+    if (dep == L) {
+        s->n_pending = 0;
+    } else {
+        /* every pending position has been carried to layer dep (or was beyond it already) */
+        for (int j = 0; j < s->n_pending; j++) memcpy(s->pend_h + (size_t)j * d, H + (size_t)j * d, sizeof(double) * d);
+        s->pend_pos[s->n_pending] = p;
+        s->pend_fill[s->n_pending] = dep;
+        memcpy(s->pend_h + (size_t)s->n_pending * d, hc, sizeof(double) * d);
+        s->n_pending++;
+    }
+    *depth = dep;
+    s->len = p + 1;
+    free(H); free(Hb); free(pos); free(who); free(z);
     return 0;
 }
