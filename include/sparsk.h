@@ -76,6 +76,19 @@ typedef struct {
                                same K and r as speech steps.  Sec. V-E: the two modalities may need
                                different policies */
     int32_t text_phase;     /* r of text steps, in [0, text_period) */
+    /* Confidence-based early exit, the compared method of Sec. V-B (thresholds of Sec. VI: 0.1
+     * for the 28-layer backbone, 0.5 for the 40-layer one).  Steps that emit a token of a
+     * modality in conf_modalities (bit 0 text, bit 1 speech; 0 = off) ignore the schedule: after
+     * every layer l in [conf_start, L) the head g_l is applied to the position's hidden state and
+     * the step leaves at the first layer whose prediction, over the ids of the modality, has an
+     * entropy (natural logarithm) below conf_threshold; otherwise it runs all L layers.  Such a
+     * position is pending exactly like a scheduled early exit: later steps carry it upwards as
+     * far as they go themselves.  Needs heads for the layers conf_start .. L.  A context in
+     * this mode synchronises its stream inside every decode step (the host learns each depth
+     * when the kernels do) and does not offer nucleus sampling. */
+    int32_t conf_modalities;
+    int32_t conf_start;
+    float conf_threshold;
 } sparsk_dims;
 
 /* All pointers are DEVICE pointers to bfloat16 data; the arrays of pointers themselves

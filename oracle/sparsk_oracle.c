@@ -507,7 +507,9 @@ double ora_entropy(const double *z, int32_t n)
  * With a single exit layer this is exactly Algorithm 1.
  *
  * entropies (may be NULL) receives, for layer l = 1..L-1, the entropy computed at that layer
- * or -1 where no head was consulted.
+ * or -1 where no head was consulted.  With a dictated depth the rule decides nothing, but for a
+ * position of a confidence modality the entropies of the layers conf_start .. depth are still
+ * reported (a checker can then judge a depth chosen elsewhere against them).
  */
 int32_t ora_decode_step_dyn(ora_seq *s, int32_t token, int32_t modality, int32_t counter,
                             int32_t forced_depth, int32_t *next_token, int32_t *depth,
@@ -519,7 +521,8 @@ int32_t ora_decode_step_dyn(ora_seq *s, int32_t token, int32_t modality, int32_t
     const int V = dm->vocab_text + dm->vocab_speech;
     if (s->len >= dm->max_len) return -1;
     if (forced_depth < 0 || forced_depth > L) return -3;
-    const int by_conf = forced_depth == 0 && ((dm->conf_modalities >> (modality ? 1 : 0)) & 1);
+    const int conf_mod = (dm->conf_modalities >> (modality ? 1 : 0)) & 1;
+    const int by_conf = forced_depth == 0 && conf_mod;
     int target = forced_depth;   /* 0: decided by confidence */
     if (forced_depth == 0 && !by_conf) {
         const int K_t = dm->text_period > 0 ? dm->text_period : dm->refresh_period;
@@ -566,20 +569,22 @@ int32_t ora_decode_step_dyn(ora_seq *s, int32_t token, int32_t modality, int32_t
         for (int j = 0; j < s->n_pending; j++)
             if (s->pend_fill[j] < l) s->pend_fill[j] = l;
         dep = l;
-        if (target) {
-            if (l == target) break;
-        } else if (l >= dm->conf_start && l < L) {
+        if (conf_mod && dm->conf_start >= 1 && l >= dm->conf_start && l < L && (by_conf || entropies)) {
             if (!m->w.head_norm[l - 1] || !m->w.head_proj[l - 1]) {
-                free(H); free(Hb); free(pos); free(who); free(z);
-                return -2;
+                if (by_conf) {
+                    free(H); free(Hb); free(pos); free(who); free(z);
+                    return -2;
+                }
+            } else {
+                head_argmax(m, l, hc, modality, z, NULL);
+                const int lo = modality == 0 ? 0 : dm->vocab_text;
+                const int hi = modality == 0 ? dm->vocab_text : V;
+                const double ent = ora_entropy(z + lo, hi - lo);
+                if (entropies) entropies[l - 1] = ent;
+                if (by_conf && ent < dm->conf_threshold) break;
             }
-            head_argmax(m, l, hc, modality, z, NULL);
-            const int lo = modality == 0 ? 0 : dm->vocab_text;
-            const int hi = modality == 0 ? dm->vocab_text : V;
-            const double ent = ora_entropy(z + lo, hi - lo);
-            if (entropies) entropies[l - 1] = ent;
-            if (ent < dm->conf_threshold) break;
         }
+        if (target && l == target) break;
     }
     *next_token = head_argmax(m, dep, hc, modality, logits, margin);
     if (hidden) memcpy(hidden, hc, sizeof(double) * d);

@@ -36,7 +36,8 @@ class Dims(C.Structure):
         ("rms_eps", C.c_float), ("rope_base", C.c_float)] + [
         (n, C.c_int32) for n in ("exit_layer", "refresh_period", "refresh_phase", "text_exit",
                                  "max_seqs", "max_seq_len", "max_pending", "prefill_rows",
-                                 "text_period", "text_phase")]
+                                 "text_period", "text_phase", "conf_modalities", "conf_start")] + [
+        ("conf_threshold", C.c_float)]
 
 
 _PP = C.POINTER(C.c_void_p)
@@ -132,6 +133,9 @@ def make_dims(dims: dict, max_seqs: int, max_seq_len: int, max_pending: int, pre
     d.text_exit = int(dims.get("text_exit", 0))
     d.text_period = int(dims.get("text_period", 0))
     d.text_phase = int(dims.get("text_phase", 0))
+    d.conf_modalities = int(dims.get("conf_modalities", 0))
+    d.conf_start = int(dims.get("conf_start", 0))
+    d.conf_threshold = float(dims.get("conf_threshold", 0.0))
     d.rms_eps = float(dims["rms_eps"])
     d.rope_base = float(dims["rope_base"])
     d.max_seqs, d.max_seq_len, d.max_pending, d.prefill_rows = max_seqs, max_seq_len, max_pending, prefill_rows

@@ -1,6 +1,7 @@
 // Host side of the SPAR-K decode library: argument checks, the host mirror of the exit
 // schedule (which only sizes launches; the device kernels are authoritative), workspace
 // carving and the launch sequence of a step.  C ABI declared in include/sparsk.h.
+#include <algorithm>
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
@@ -94,6 +95,7 @@ struct sparsk_ctx {
     std::vector<TmaPair> tm_wq, tm_wk, tm_wv, tm_wo, tm_wg, tm_wu, tm_wd, tm_head;
     TmaPair tm_x[5], tm_ao[5], tm_act[5], tm_x_lo[5], tm_ao_lo[5], tm_act_lo[5];
     std::vector<CUtensorMap> tm_kc, tm_vc;  // per layer: the cache viewed as [64][slots * Hkv * S rows][hd / 64], boxes of [64][64][2]
+    int attn_stages;                        // K/V ring depth of the warp-per-item attention kernel (2 or 3)
     int attn_tc, attn_tc_min_q;             // tcgen05 attention for blocks of at least this many query vectors
     // persistent layer-range kernel (one or two rows)
     MkLayer *mk_layers;            // device [L]
@@ -104,6 +106,14 @@ struct sparsk_ctx {
     int mk_trace_n;                // entries the last launch wrote
     unsigned long long mk_bar_base;
     int mega, mk_ok, mk_coop, mk_max_rows;
+    // confidence-based exit (dims.conf_modalities != 0): the host drives the step layer by layer
+    std::vector<std::vector<int>> h_fill;  // per slot: layer each pending position has been carried to
+    int *conf_host;                // pinned arena for the row sets of a step's segments
+    size_t conf_host_ints, conf_seg_ints;
+    int *conf_rows_dev;            // device: [slot R][pos R][src R][seq R][grp_row0 B][grp_nrows B][n_groups][n_rows]
+    int *conf_list_dev;            // device: [rows B][modality B]
+    float *conf_ent_dev, *conf_ent_host;  // entropies of a layer's candidates (device, pinned host)
+    float *conf_logits;            // device [B][V] when neither the parity hook nor a sampler lends a buffer
     int inject_timeout;            // test hook: the next persistent launch waits for a barrier count nobody reaches
     int64_t route_layers[3];       // layer passes so far by implementation: see sparsk_route_counts
     std::vector<MkLayer> mk_host;
@@ -152,6 +162,8 @@ bool dims_ok(const sparsk_dims *d)
     if (d->exit_layer < 1 || d->exit_layer > d->n_layers) return false;
     if (d->refresh_period < 1 || d->refresh_phase < 0 || d->refresh_phase >= d->refresh_period) return false;
     if (d->text_exit < 0 || d->text_exit > 2) return false;
+    if (d->conf_modalities < 0 || d->conf_modalities > 3) return false;
+    if (d->conf_modalities && (d->conf_start < 1 || d->conf_start >= d->n_layers || !(d->conf_threshold >= 0.f))) return false;
     if (d->text_period < 0 || (d->text_period > 0 && (d->text_phase < 0 || d->text_phase >= d->text_period))) return false;
     if (d->max_seqs < 1 || d->max_seqs > 1024 || d->max_seq_len < 1) return false;
     if (d->max_pending < 0 || d->prefill_rows < 0) return false;
@@ -191,6 +203,14 @@ size_t carve(sparsk_ctx *c, const sparsk_dims *d, char *base)
     int *pfng = w.take<int>(1), *pfnr = w.take<int>(1);
     float *hlo = w.take<float>(B * d->d_model), *hup = w.take<float>(R * d->d_model);
     float *q = w.take<float>(R * qrow);
+    int *crows = nullptr, *clist = nullptr;
+    float *cent = nullptr, *clog = nullptr;
+    if (d->conf_modalities) {
+        crows = w.take<int>(4 * R + 2 * B + 2);
+        clist = w.take<int>(2 * B);
+        cent = w.take<float>(B);
+        clog = w.take<float>(B * ((size_t)d->vocab_text + d->vocab_speech));
+    }
     float *hlast = w.take<float>(B * d->d_model), *qlast = w.take<float>(B * qrow);
     int *lslot = w.take<int>(B), *lpos = w.take<int>(B);
     bf16 *ao = w.take<bf16>(R * qrow), *act = w.take<bf16>(R * d->d_ffn);
@@ -210,6 +230,7 @@ size_t carve(sparsk_ctx *c, const sparsk_dims *d, char *base)
         c->sd = sd; c->staged = staged; c->tok_dev = tok; c->out_tok_dev = ot; c->out_depth_dev = od;
         c->pf_slot = pfs; c->pf_pos = pfp; c->pf_grp_row0 = pfg0; c->pf_grp_nrows = pfgn;
         c->pf_ngrp = pfng; c->pf_nrows = pfnr;
+        c->conf_rows_dev = crows; c->conf_list_dev = clist; c->conf_ent_dev = cent; c->conf_logits = clog;
         c->h_last = hlast; c->q_last = qlast; c->last_slot = lslot; c->last_pos = lpos;
         c->h_lo = hlo; c->h_up = hup; c->qbuf = q; c->attn_o = ao; c->act = act; c->xnorm = xn; c->qkv_part = qp;
         c->attn_o_lo = aol; c->act_lo = actl; c->xnorm_lo = xnl;
@@ -377,7 +398,10 @@ cudaError_t run_gateup(sparsk_ctx *c, int layer, const float *h, int n_rows)
 }
 
 // Where the heads leave their logits: the parity hook's buffer, else the sampler's, else nowhere.
-float *head_logits(const sparsk_ctx *c) { return c->dbg_logits ? c->dbg_logits : (c->samp_uniforms ? c->samp_scratch : nullptr); }
+float *head_logits(const sparsk_ctx *c)
+{
+    return c->dbg_logits ? c->dbg_logits : (c->samp_uniforms ? c->samp_scratch : c->conf_logits);
+}
 
 bool use_tc(const sparsk_ctx *c, int n_rows);
 cudaError_t run_head_tc(sparsk_ctx *c, int layer, const float *h, int list, int n_rows);
@@ -437,7 +461,9 @@ cudaError_t run_attn(sparsk_ctx *c, int layer, const RowSet &rs)
     // groups the tcgen05 kernel takes (the host knows every group's row count) and the rest
     const int n_big = blocks_tc ? (rs.n_big > 0 ? rs.n_big : rs.n_groups_h) : 0;
     const int n_small = rs.n_groups_h - n_big;
-    AttnPlan pl = attn_plan(c->n_sm, blocks_tc ? std::max(1, n_small) : rs.n_groups_h, blocks_tc ? 1 : rs.max_grp_rows, G,
+    const int warp_ctas = c->n_sm * attn_warp_ctas_per_sm(d.head_dim, c->attn_stages);
+    const int small_rows = blocks_tc ? std::max(1, std::min(rs.max_grp_rows, (c->attn_tc_min_q - 1) / G)) : rs.max_grp_rows;
+    AttnPlan pl = attn_plan(warp_ctas * AW_WARPS, blocks_tc ? std::max(1, n_small) : rs.n_groups_h, small_rows, G,
                             d.n_kv_heads, rs.max_len, c->attn_split);
     if (blocks_tc) {
         // Groups with many query vectors per kv head go to the tcgen05 kernel (one CTA per SM, tiles
@@ -490,15 +516,18 @@ cudaError_t run_attn(sparsk_ctx *c, int layer, const RowSet &rs)
         if (e != cudaSuccess) return e;
         a.nq_max = c->attn_tc_min_q - 1;
     }
-    a.n_qblk = blocks_tc ? div_up(std::min(rs.max_grp_rows * G, c->attn_tc_min_q - 1), 16 * pl.mt) : pl.n_qblk;
+    a.n_qblk = blocks_tc ? div_up(std::min(rs.max_grp_rows * G, c->attn_tc_min_q - 1), 16) : pl.n_qblk;
     a.split_len = pl.split_len;
     a.n_splits = pl.n_splits;
+    a.max_groups = rs.n_groups_h;
     if (!blocks_tc || (c->attn_tc_min_q > 1 && n_small > 0)) {
-        dim3 grid(rs.n_groups_h * a.n_qblk, d.n_kv_heads, a.n_splits);
-        AttnPartialFn fn;
-        e = attn_partial_fn(d.head_dim, pl.mt, &fn);
+        // every group is in the item space (the kernel skips those the other kernel takes)
+        const long n_items = (long)rs.n_groups_h * a.n_qblk * d.n_kv_heads * a.n_splits;
+        const int grid = (int)std::max<long>(1, std::min<long>(warp_ctas, (n_items + AW_WARPS - 1) / AW_WARPS));
+        AttnWarpFn fn;
+        e = attn_warp_fn(d.head_dim, c->attn_stages, &fn);
         if (e != cudaSuccess) return e;
-        e = launch(c, fn, grid, dim3(AT_THREADS), attn_smem_bytes(d.head_dim, pl.mt), a);
+        e = launch(c, fn, dim3(grid), dim3(AW_WARPS * 32), AW_WARPS * attn_warp_bytes(d.head_dim, c->attn_stages), a);
         if (e != cudaSuccess) return e;
     }
     if (d.head_dim == 128) return launch(c, attn_merge_kernel<128>, dim3(rs.n_rows, d.n_q_heads), dim3(128), 0, a, rs.n_rows_dev);
@@ -982,6 +1011,9 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
     // the heads of layers e and L are what the periodic schedule reads
     if (!w->head_norm[L - 1] || !w->head_proj[L - 1]) return SPARSK_ENOHEAD;
     if (dims->refresh_period > 1 && e < L && (!w->head_norm[e - 1] || !w->head_proj[e - 1])) return SPARSK_ENOHEAD;
+    if (dims->conf_modalities)   // the confidence rule consults the head of every layer from conf_start on
+        for (int l = dims->conf_start; l < L; l++)
+            if (!w->head_norm[l - 1] || !w->head_proj[l - 1]) return SPARSK_ENOHEAD;
 
     sparsk_ctx *ctx = new (std::nothrow) sparsk_ctx();
     if (!ctx) return SPARSK_EINVAL;
@@ -1008,9 +1040,11 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
     ctx->gemm_smem_kb = 220;
     ctx->gemm_cps = 1;
     ctx->mk_max_rows = 2;
-    ctx->attn_tc = 1; ctx->attn_tc_min_q = 33;
+    ctx->attn_tc = 1; ctx->attn_tc_min_q = 33; ctx->attn_stages = AW_NST;
     ctx->inject_timeout = 0;
     ctx->trim_last = 1;
+    ctx->conf_host = nullptr; ctx->conf_ent_host = nullptr;
+    ctx->h_fill.assign(dims->max_seqs, std::vector<int>());
     for (auto &v : ctx->route_layers) v = 0;
     ctx->mega = 1; ctx->mk_ok = 0; ctx->mk_coop = 0; ctx->mk_bar_base = 0; ctx->mk_trace_n = 0;
     ctx->gv_ks = 0; ctx->gv_r = 0;
@@ -1036,6 +1070,16 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
                 rc = fail(ctx, SPARSK_ECUDA, "staging setup failed: %s", cudaGetErrorString(ce));
         }
         if (rc) break;
+        if (dims->conf_modalities) {
+            // one region per segment of a step (at most one per layer, plus lists per consulted layer)
+            ctx->conf_seg_ints = 4 * (size_t)ctx->cap_rows + 4 * (size_t)dims->max_seqs + 8;
+            ctx->conf_host_ints = ctx->conf_seg_ints * (2 * (size_t)L + 4);
+            if ((ce = cudaHostAlloc((void **)&ctx->conf_host, ctx->conf_host_ints * sizeof(int), cudaHostAllocDefault)) != cudaSuccess ||
+                (ce = cudaHostAlloc((void **)&ctx->conf_ent_host, sizeof(float) * dims->max_seqs, cudaHostAllocDefault)) != cudaSuccess) {
+                rc = fail(ctx, SPARSK_ECUDA, "staging setup failed: %s", cudaGetErrorString(ce));
+                break;
+            }
+        }
         // no silent change of path: without TMA descriptors the batched path cannot run
         ctx->tc_ok = build_maps(ctx);
         if (!ctx->tc_ok) {
@@ -1088,6 +1132,8 @@ extern "C" int sparsk_destroy(sparsk_ctx *ctx)
         if (ctx->stage_ev[i]) cudaEventDestroy(ctx->stage_ev[i]);
     }
     for (cudaEvent_t ev : ctx->tev) cudaEventDestroy(ev);
+    if (ctx->conf_host) cudaFreeHost(ctx->conf_host);
+    if (ctx->conf_ent_host) cudaFreeHost(ctx->conf_ent_host);
     ctx->magic = 0;
     delete ctx;
     return SPARSK_OK;
@@ -1126,6 +1172,8 @@ extern "C" int sparsk_set_sampling(sparsk_ctx *ctx, float temperature, float top
         ctx->samp_scratch = nullptr;
         return SPARSK_OK;
     }
+    if (ctx->dm.conf_modalities)
+        return fail(ctx, SPARSK_EINVAL, "set_sampling: a context with confidence-based exit decodes greedily");
     if (!(temperature > 0.f) || !(temperature < INFINITY) || !(top_p > 0.f) || !(top_p <= 1.f))
         return fail(ctx, SPARSK_EINVAL, "set_sampling: temperature %g, top_p %g", (double)temperature, (double)top_p);
     if (ctx->dm.vocab_text > SP_MAX_RANGE || ctx->dm.vocab_speech > SP_MAX_RANGE)
@@ -1149,6 +1197,7 @@ extern "C" int sparsk_set_option(sparsk_ctx *ctx, const char *name, int64_t valu
     else if (!strcmp(name, "attn_split") && value >= 0 && value <= (1 << 24)) ctx->attn_split = (int)value;
     else if (!strcmp(name, "gemv_ks") && (value == 0 || value == 1 || value == 2 || value == 4 || value == 8 || value == 16)) ctx->gv_ks = (int)value;
     else if (!strcmp(name, "mega") && (value == 0 || value == 1)) ctx->mega = (int)value;
+    else if (!strcmp(name, "attn_stages") && (value == 2 || value == 3)) ctx->attn_stages = (int)value;
     else if (!strcmp(name, "attn_tc") && (value == 0 || value == 1)) ctx->attn_tc = (int)value;
     else if (!strcmp(name, "attn_tc_min_q") && value >= 1 && value <= (1 << 20)) ctx->attn_tc_min_q = (int)value;
     else if (!strcmp(name, "mega_max_rows") && value >= 1 && value <= MK_MAX_ROWS) ctx->mk_max_rows = (int)value;
@@ -1253,6 +1302,7 @@ extern "C" int sparsk_set_len(sparsk_ctx *ctx, int32_t slot, int32_t len)
     CU(launch(ctx, set_int_kernel, dim3(1), dim3(1), 0, ctx->pend_cnt + slot, 0));
     ctx->h_len[slot] = len;
     ctx->h_pend[slot] = 0;
+    ctx->h_fill[slot].clear();
     return SPARSK_OK;
 }
 
@@ -1333,6 +1383,225 @@ extern "C" int sparsk_prefill(sparsk_ctx *ctx, int32_t n_seqs, const int32_t *sl
     return SPARSK_OK;
 }
 
+// --------------------------------------------------------------------------- decode step, confidence-based exit
+// The step of a context whose dims name a confidence modality (Sec. V-B, compared method 3).
+// Depths are not known beforehand, so the host walks the layers in segments: a segment is a run
+// of layers over one row set; it ends where a pending position joins (the layer after the one it
+// has been carried to), where a scheduled sequence leaves, and after every layer from
+// conf_start on while a confidence sequence is still running, because there its head is
+// consulted: head, entropy kernel, copy of the entropies to the host, stream synchronisation,
+// decision.  Pending positions carry the layer they have been filled to; a sequence's rows in a
+// segment are the pending positions not yet carried through its first layer (always the newest
+// ones: an older position has been carried at least as far as a newer one) followed by the
+// current position, i.e. consecutive positions, one attention group.
+static int decode_step_conf(sparsk_ctx *ctx, int32_t n, const int32_t *slots, const int32_t *token_ids,
+                            const uint8_t *modality, const int32_t *counters, int32_t *next_tokens, int32_t *exit_depths)
+{
+    const sparsk_dims &d = ctx->dm;
+    const int L = d.n_layers, e = d.exit_layer, B = d.max_seqs, cs = d.conf_start;
+    const int V = d.vocab_text + d.vocab_speech, G_heads = d.n_q_heads / d.n_kv_heads;
+    const SchedParams sp{L, e, d.refresh_period, d.refresh_phase, d.text_period > 0 ? d.text_period : d.refresh_period,
+                         d.text_period > 0 ? d.text_phase : d.refresh_phase, d.text_exit};
+    std::vector<char> seen(B, 0);
+    std::vector<int> target(n), depth(n, 0);
+    int max_len = 0;
+    for (int i = 0; i < n; i++) {
+        const int s = slots[i];
+        if (s < 0 || s >= B || seen[s]) return fail(ctx, SPARSK_EINVAL, "decode_step: slot %d invalid or repeated", s);
+        seen[s] = 1;
+        if (modality[i] > 1) return fail(ctx, SPARSK_EINVAL, "decode_step: modality[%d]=%d", i, modality[i]);
+        if (counters[i] < 0) return fail(ctx, SPARSK_EINVAL, "decode_step: counter[%d]=%d", i, counters[i]);
+        if (ctx->h_len[s] + 1 > d.max_seq_len) return fail(ctx, SPARSK_ECAPACITY, "decode_step: slot %d is full (%d positions)", s, ctx->h_len[s]);
+        const bool by_conf = (d.conf_modalities >> (modality[i] ? 1 : 0)) & 1;
+        target[i] = by_conf ? 0 : scheduled_depth(modality[i], counters[i], sp);
+        if (target[i] != L && (int)ctx->h_fill[s].size() + 1 > d.max_pending)
+            return fail(ctx, SPARSK_ECAPACITY, "decode_step: slot %d may hold %d pending positions (max_pending %d)", s,
+                        (int)ctx->h_fill[s].size() + 1, d.max_pending);
+        if (target[i] && (!ctx->head_norm[target[i] - 1] || !ctx->head_proj[target[i] - 1]))
+            return fail(ctx, SPARSK_ENOHEAD, "decode_step: layer %d has no exit head", target[i]);
+        max_len = std::max(max_len, ctx->h_len[s] + 1);
+    }
+    // ---- stage the host arrays; latch tokens; embed
+    const int ring = ctx->stage_next;
+    ctx->stage_next = (ring + 1) % STAGE_RING;
+    CU(cudaEventSynchronize(ctx->stage_ev[ring]));
+    int *st = ctx->stage_host[ring];
+    for (int i = 0; i < n; i++) {
+        st[i] = slots[i];
+        st[n + i] = modality[i];
+        st[2 * n + i] = counters[i];
+    }
+    CU(cudaMemcpyAsync(ctx->staged, st, sizeof(int) * 3 * n, cudaMemcpyHostToDevice, ctx->stream));
+    CU(cudaEventRecord(ctx->stage_ev[ring], ctx->stream));
+    CU(launch(ctx, schedule_kernel, dim3((n + 127) / 128), dim3(128), 0, ctx->sd, (int)n, (const int *)ctx->staged,
+              (const int *)token_ids, V, sp));
+    // the lower-row arrays (positions, one-row groups); "e = L" keeps every head on the lower rows
+    CU(launch(ctx, compact_kernel, dim3(1), dim3(1024), 0, ctx->sd, (int)n, (const int *)ctx->kv_len,
+              (const int *)ctx->pend_cnt, L, L, B));
+    CU(launch(ctx, embed_kernel, dim3(n), dim3(128), 0, (const int *)ctx->sd.token, ctx->embed, ctx->h_lo, (int)n, d.d_model,
+              V, ctx->sd.counts + CNT_STATUS));
+    if (ctx->dbg_logits) {
+        const size_t cnt = (size_t)n * V;
+        CU(launch(ctx, fill_kernel, dim3((unsigned)std::min<size_t>((cnt + 255) / 256, 2048)), dim3(256), 0, ctx->dbg_logits, cnt, -INFINITY));
+    }
+    const int R = ctx->cap_rows;
+    size_t arena = 0;  // ints of the pinned arena used so far in this step
+    auto region = [&](size_t ints) -> int * {
+        if (arena + ints > ctx->conf_host_ints) return nullptr;
+        int *p = ctx->conf_host + arena;
+        arena += ints;
+        return p;
+    };
+    // heads of `layer` for the listed sequences (indices into the step), text and speech apart
+    auto heads = [&](int layer, const std::vector<int> &who) -> int {
+        for (int mod = 0; mod < 2; mod++) {
+            std::vector<int> rows;
+            for (int i : who)
+                if ((modality[i] ? 1 : 0) == mod) rows.push_back(i);
+            if (rows.empty()) continue;
+            int *hb = region(rows.size());
+            if (!hb) return fail(ctx, SPARSK_ECAPACITY, "decode_step: staging arena exhausted");
+            std::copy(rows.begin(), rows.end(), hb);
+            CU(cudaMemcpyAsync(ctx->sd.list_row + (size_t)mod * B, hb, sizeof(int) * rows.size(), cudaMemcpyHostToDevice, ctx->stream));
+            CU(cudaMemcpyAsync(ctx->sd.list_seq + (size_t)mod * B, hb, sizeof(int) * rows.size(), cudaMemcpyHostToDevice, ctx->stream));
+            CU(launch(ctx, clear_keys_kernel, dim3(((int)rows.size() + 127) / 128), dim3(128), 0, ctx->sd.argmax,
+                      (const int *)(ctx->sd.list_row + (size_t)mod * B), (int)rows.size()));
+            CU(run_head(ctx, layer, ctx->h_lo, mod, (int)rows.size()));
+        }
+        return SPARSK_OK;
+    };
+    auto leave = [&](int i, int at) -> int {   // sequence i leaves at layer `at`
+        const int s = slots[i];
+        depth[i] = at;
+        std::vector<int> &fill = ctx->h_fill[s];
+        if (at == L) {
+            fill.clear();
+        } else {
+            CU(cudaMemcpyAsync(ctx->pend_h + ((size_t)s * d.max_pending + fill.size()) * d.d_model, ctx->h_lo + (size_t)i * d.d_model,
+                               sizeof(float) * d.d_model, cudaMemcpyDeviceToDevice, ctx->stream));
+            fill.push_back(at);
+        }
+        return SPARSK_OK;
+    };
+
+    std::vector<int> active(n);
+    for (int i = 0; i < n; i++) active[i] = i;
+    int l = 1;
+    while (!active.empty()) {
+        // ---- where this segment ends
+        int seg_end = L;
+        for (int i : active) {
+            seg_end = std::min(seg_end, target[i] ? target[i] : std::max(l, cs));
+            for (int f : ctx->h_fill[slots[i]])
+                if (f >= l) seg_end = std::min(seg_end, f);
+        }
+        // ---- its rows
+        struct Row { int slot, pos, src, seq; };
+        std::vector<Row> rows;
+        std::vector<int> g_row0, g_nrows;
+        int max_grp = 1, n_big = 0, seg_len = 0;
+        for (int i : active) {
+            const int s = slots[i];
+            const std::vector<int> &fill = ctx->h_fill[s];
+            const int P = (int)fill.size();
+            int j0 = 0;
+            while (j0 < P && fill[j0] >= l) j0++;   // carried through layer l already
+            g_row0.push_back((int)rows.size());
+            g_nrows.push_back(P - j0 + 1);
+            for (int j = j0; j < P; j++) rows.push_back({s, ctx->h_len[s] - P + j, j, i});
+            rows.push_back({s, ctx->h_len[s], -1, i});
+            max_grp = std::max(max_grp, P - j0 + 1);
+            n_big += (P - j0 + 1) * G_heads >= ctx->attn_tc_min_q;
+            seg_len = std::max(seg_len, ctx->h_len[s] + 1);
+        }
+        const int m = (int)rows.size(), ng = (int)active.size();
+        if (m > R) return fail(ctx, SPARSK_ECAPACITY, "decode_step: %d rows exceed capacity %d", m, R);
+        if (m == n && ng == n) {
+            // nothing but the step's own positions, in order: the lower rows as they stand
+            RowSet lo{ctx->sd.slot, ctx->sd.lo_pos, ctx->sd.lo_grp_row0, ctx->sd.lo_grp_nrows, ctx->sd.counts + CNT_NSEQ,
+                      ctx->sd.counts + CNT_NSEQ, n, n, 1, seg_len};
+            CU(run_layers(ctx, l, seg_end, ctx->h_lo, lo));
+        } else {
+            int *hb = region(4 * (size_t)R + 2 * (size_t)B + 2);
+            if (!hb) return fail(ctx, SPARSK_ECAPACITY, "decode_step: staging arena exhausted");
+            int *h_slot = hb, *h_pos = hb + R, *h_src = hb + 2 * R, *h_seq = hb + 3 * R, *h_g0 = hb + 4 * R, *h_gn = h_g0 + B,
+                *h_cnt = h_gn + B;
+            for (int k = 0; k < m; k++) {
+                h_slot[k] = rows[k].slot; h_pos[k] = rows[k].pos; h_src[k] = rows[k].src; h_seq[k] = rows[k].seq;
+            }
+            for (int k = 0; k < ng; k++) {
+                h_g0[k] = g_row0[k];
+                h_gn[k] = g_nrows[k];
+            }
+            h_cnt[0] = ng;
+            h_cnt[1] = m;
+            int *dv = ctx->conf_rows_dev;
+            CU(cudaMemcpyAsync(dv, hb, sizeof(int) * (4 * (size_t)R + 2 * (size_t)B + 2), cudaMemcpyHostToDevice, ctx->stream));
+            int *d_slot = dv, *d_pos = dv + R, *d_src = dv + 2 * R, *d_seq = dv + 3 * R, *d_g0 = dv + 4 * R, *d_gn = d_g0 + B,
+                *d_cnt = d_gn + B;
+            CU(launch(ctx, rows_move_kernel, dim3(m), dim3(128), 0, ctx->h_up, ctx->h_lo, ctx->pend_h, (const int *)d_slot,
+                      (const int *)d_seq, (const int *)d_src, m, d.d_model, d.max_pending, 1));
+            RowSet up{d_slot, d_pos, d_g0, d_gn, d_cnt, d_cnt + 1, m, ng, max_grp, seg_len, n_big};
+            CU(run_layers(ctx, l, seg_end, ctx->h_up, up));
+            CU(launch(ctx, rows_move_kernel, dim3(m), dim3(128), 0, ctx->h_up, ctx->h_lo, ctx->pend_h, (const int *)d_slot,
+                      (const int *)d_seq, (const int *)d_src, m, d.d_model, d.max_pending, 0));
+        }
+        for (int i : active)   // the pending positions that took part have been carried to seg_end
+            for (int &f : ctx->h_fill[slots[i]])
+                if (f < seg_end) f = seg_end;
+        // ---- who leaves after layer seg_end
+        std::vector<int> leaving, asking;
+        for (int i : active) {
+            if (seg_end == L || target[i] == seg_end) leaving.push_back(i);
+            else if (!target[i] && seg_end >= cs) asking.push_back(i);
+        }
+        if (!leaving.empty()) {
+            const int rc = heads(seg_end, leaving);
+            if (rc != SPARSK_OK) return rc;
+        }
+        if (!asking.empty()) {
+            int rc = heads(seg_end, asking);
+            if (rc != SPARSK_OK) return rc;
+            int *hb = region(2 * asking.size());
+            if (!hb) return fail(ctx, SPARSK_ECAPACITY, "decode_step: staging arena exhausted");
+            for (size_t k = 0; k < asking.size(); k++) {
+                hb[k] = asking[k];
+                hb[asking.size() + k] = modality[asking[k]] ? 1 : 0;
+            }
+            CU(cudaMemcpyAsync(ctx->conf_list_dev, hb, sizeof(int) * 2 * asking.size(), cudaMemcpyHostToDevice, ctx->stream));
+            CU(launch(ctx, entropy_kernel, dim3((unsigned)asking.size()), dim3(1024), 0, (const float *)head_logits(ctx),
+                      (const int *)ctx->conf_list_dev, (const int *)(ctx->conf_list_dev + asking.size()), (int)asking.size(), V,
+                      d.vocab_text, ctx->conf_ent_dev));
+            CU(cudaMemcpyAsync(ctx->conf_ent_host, ctx->conf_ent_dev, sizeof(float) * asking.size(), cudaMemcpyDeviceToHost, ctx->stream));
+            CU(cudaStreamSynchronize(ctx->stream));
+            for (size_t k = 0; k < asking.size(); k++)
+                if (ctx->conf_ent_host[k] < d.conf_threshold) leaving.push_back(asking[k]);
+        }
+        for (int i : leaving) {
+            const int rc = leave(i, seg_end);
+            if (rc != SPARSK_OK) return rc;
+            active.erase(std::find(active.begin(), active.end(), i));
+        }
+        l = seg_end + 1;
+    }
+    // ---- outputs and state
+    int *hb = region(n);
+    if (!hb) return fail(ctx, SPARSK_ECAPACITY, "decode_step: staging arena exhausted");
+    std::copy(depth.begin(), depth.end(), hb);
+    CU(cudaMemcpyAsync(ctx->sd.depth, hb, sizeof(int) * n, cudaMemcpyHostToDevice, ctx->stream));
+    if (ctx->dbg_hidden)
+        CU(launch(ctx, debug_hidden_kernel, dim3(n), dim3(128), 0, ctx->sd, (const float *)ctx->h_lo,
+                  (const float *)ctx->h_up, ctx->dbg_hidden, (int)n, d.d_model));
+    CU(launch(ctx, finish_kernel, dim3((n + 127) / 128), dim3(128), 0, ctx->sd, (int)n, ctx->kv_len, ctx->pend_cnt,
+              next_tokens, exit_depths, L));
+    for (int i = 0; i < n; i++) {
+        ctx->h_len[slots[i]] += 1;
+        ctx->h_pend[slots[i]] = (int)ctx->h_fill[slots[i]].size();
+    }
+    CU(cudaStreamSynchronize(ctx->stream));  // the pinned arena is free again
+    return SPARSK_OK;
+}
+
 // --------------------------------------------------------------------------- decode step
 extern "C" int sparsk_decode_step(sparsk_ctx *ctx, int32_t n, const int32_t *slots, const int32_t *token_ids,
                                   const uint8_t *modality, const int32_t *counters, int32_t *next_tokens,
@@ -1345,6 +1614,7 @@ extern "C" int sparsk_decode_step(sparsk_ctx *ctx, int32_t n, const int32_t *slo
                          d.text_period > 0 ? d.text_phase : d.refresh_phase, d.text_exit};
     if (n < 1 || n > B || !slots || !token_ids || !modality || !counters || !next_tokens || !exit_depths)
         return fail(ctx, SPARSK_EINVAL, "decode_step: bad arguments (n=%d)", n);
+    if (d.conf_modalities) return decode_step_conf(ctx, n, slots, token_ids, modality, counters, next_tokens, exit_depths);
     // ---- host mirror of the schedule: validates, and sizes the launches
     std::vector<char> seen(B, 0);
     int n_list[4] = {0, 0, 0, 0};

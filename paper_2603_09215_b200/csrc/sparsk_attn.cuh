@@ -1,69 +1,56 @@
 // Split-KV grouped-query attention over the ragged KV cache (flash-decoding) on tensor cores.
 //
-// One CTA handles one (sequence group, block of query vectors, kv head, KV split).  A group is
-// the block of rows of ONE sequence that a pass processes together: a single row in the lower
-// pass, the pending positions plus the current one in the upper pass (Algorithm 1, full-depth
-// branch: one causal block of at most K rows), a chunk of the prompt in prefill.  All query heads that share
-// the kv head, for all rows of the group, form the M dimension of mma.sync m16n8k16 tiles, so one
-// read of that head's K/V serves them all; row r of the group may look at positions
-// <= pos0 + r (the causal mask of the block on top of the whole earlier cache).
+// A work item is (sequence group, block of 16 query vectors, kv head, KV split) and belongs to ONE
+// warp.  A group is the block of rows of ONE sequence that a pass processes together: a single
+// row in the lower pass, the pending positions plus the current one in the upper pass
+// (Algorithm 1, full-depth branch: one causal block of at most K rows), a chunk of the prompt in
+// prefill.  The query heads that share the kv head, for the rows of the group, form the M
+// dimension of mma.sync m16n8k16 tiles, so one read of that head's K/V serves sixteen of them;
+// row r of the group may look at positions <= pos0 + r (the causal mask of the block on top of
+// the whole earlier cache).
 //
-// The split's positions are dealt to the CTA's four warps as contiguous sub-ranges.  Each warp
-// streams its own 16-position K/V tiles into a private three-stage shared-memory ring with
-// coalesced 16-byte cp.async copies (no CTA-wide barrier in the loop), computes S = Q K^T and
-// O += P V with fp16 MMAs and fp32 accumulators (the cache is fp16; queries and softmax weights
-// enter as two fp16 terms, hi + lo, so that only the cache itself is rounded), and keeps an online softmax whose row maxima
-// and sums are reduced with shuffles inside the four-lane groups that share an accumulator row.
-// The four warps' states are merged through shared memory into one unnormalised partial
-// (acc, running max, running sum) per split; a second kernel merges the splits.
+// The warp keeps its sixteen query vectors as fp16 MMA fragments in registers (scaled by
+// log2(e) / sqrt(hd), so that the softmax works in powers of two), streams 16-position K/V tiles
+// of its split into a private shared-memory ring with coalesced 16-byte cp.async copies (no
+// barrier wider than the warp anywhere), computes S = Q K^T and O += P V with fp16 MMAs and fp32
+// accumulators, and keeps an online softmax whose row maxima and sums are reduced with shuffles
+// inside the four-lane groups that share an accumulator row.  Queries and softmax weights are
+// rounded to fp16 once, like the cache they meet: the same 2^-12 relative error as a cached key
+// or value carries.  The warp writes one unnormalised partial (acc, running max in log2 units
+// turned back to natural-log units, running sum) per (row, query head, split); a second kernel
+// merges the splits.  Items are dealt round-robin to the warps of a persistent grid: a warp's
+// fixed cost per item is a few hundred instructions, which is what lets twelve warps per SM with
+// one tile in flight each keep HBM busy where CTA-wide tiles with a cross-warp merge did not.
 #pragma once
 
 #include "sparsk_common.cuh"
 
 namespace sparsk {
 
-constexpr int AT_THREADS = 128;
-constexpr int AT_TP = 16;        // positions per warp tile
-constexpr int AT_NST = 3;        // ring stages per warp (two when the CTA holds 32 query vectors)
+constexpr int AT_TP = 16;        // positions per tile
 constexpr int AT_MAX_SPLITS = 32;
 constexpr int AT_MIN_SPLIT = 64;
+constexpr int AW_WARPS = 4;      // warps per CTA of the stand-alone kernel
+constexpr int AW_NST = 2;        // ring stages per warp there (default; 3 is the other instantiation)
 
-// How a launch cuts the work: query vectors per CTA (16 or 32), and the KV range into enough
-// splits to fill the machine, none shorter than AT_MIN_SPLIT positions (unless forced), at most
-// AT_MAX_SPLITS.
+// How a launch cuts the work: blocks of 16 query vectors per group, and the KV range into
+// splits so that every warp of the persistent grid gets a few items, none shorter than
+// AT_MIN_SPLIT positions (unless forced), at most AT_MAX_SPLITS.
 struct AttnPlan {
-    int mt;  // m16 tiles per CTA: 1 or 2
     int n_qblk, split_len, n_splits;
 };
-inline AttnPlan attn_plan(int n_sm, int n_groups, int max_grp_rows, int G, int Hkv, int max_len, int forced_split)
+inline AttnPlan attn_plan(int n_workers, int n_groups, int max_grp_rows, int G, int Hkv, int max_len, int forced_split)
 {
     AttnPlan p;
     const int nq = max_grp_rows * G;
-    p.mt = nq > 16 ? 2 : 1;
-    p.n_qblk = (nq + 16 * p.mt - 1) / (16 * p.mt);
+    p.n_qblk = (nq + 15) / 16;
     int split = forced_split;
     if (split <= 0) {
-        // Two CTAs fit an SM.  Cut the KV range so that the CTAs fill whole waves of 2 * n_sm and,
-        // when the work allows, at least four of them (sequences are ragged and the causal cut
-        // makes CTAs unequal: many short CTAs even that out); never below AT_MIN_SPLIT positions.
-        const long slots = 2L * n_sm, base = (long)n_groups * p.n_qblk * Hkv;
-        const int max_s = (int)(max_len / AT_MIN_SPLIT < 1 ? 1 : (max_len / AT_MIN_SPLIT > AT_MAX_SPLITS ? AT_MAX_SPLITS : max_len / AT_MIN_SPLIT));
-        int best_s = 1;
-        double best = -1.0;
-        for (int s = 1; s <= max_s; s++) {
-            const long n = base * s, waves = (n + slots - 1) / slots;
-            const double eff = (double)n / (double)(waves * slots);
-            if (waves >= 4 && eff >= 0.92) {
-                best_s = s;
-                break;
-            }
-            const double score = eff * (double)(waves < 4 ? waves : 4);
-            if (score > best + 1e-9) {
-                best = score;
-                best_s = s;
-            }
-        }
-        split = (max_len + best_s - 1) / best_s;
+        const long base = (long)(n_groups < 1 ? 1 : n_groups) * p.n_qblk * Hkv;
+        long want = (3L * n_workers + base - 1) / base;   // about three items per warp
+        if (want < 1) want = 1;
+        if (want > AT_MAX_SPLITS) want = AT_MAX_SPLITS;
+        split = (int)((max_len + want - 1) / want);
         if (split < AT_MIN_SPLIT) split = AT_MIN_SPLIT;
     }
     split = (split + AT_TP - 1) / AT_TP * AT_TP;
@@ -78,13 +65,8 @@ inline AttnPlan attn_plan(int n_sm, int n_groups, int max_grp_rows, int G, int H
     p.n_splits = n_splits;
     return p;
 }
-inline size_t attn_smem_bytes(int head_dim, int mt)
-{
-    const size_t kp = head_dim + 8;
-    const size_t q = (size_t)2 * 16 * mt * kp * 2, ring = (size_t)4 * (mt == 2 ? 2 : AT_NST) * 2 * AT_TP * kp * 2;
-    const size_t merge = (size_t)4 * 16 * mt * (head_dim + 2) * 4;
-    return q + (ring > merge ? ring : merge);
-}
+// shared memory of one warp's K/V ring
+inline size_t attn_warp_bytes(int head_dim, int stages) { return (size_t)stages * 2 * AT_TP * (head_dim + 8) * 2; }
 
 struct AttnArgs {
     const bf16 *q;            // [rows][Hq*hd], already rotated
@@ -100,6 +82,7 @@ struct AttnArgs {
     int n_slots;              // slots in the cache; rows naming another slot are skipped
     int n_rows;               // rows in q/out; groups reaching beyond them are skipped
     int nq_min, nq_max;       // only groups with this many query vectors per kv head (another launch takes the rest)
+    int max_groups;           // host bound on the number of groups (sizes the item space)
 };
 
 __device__ __forceinline__ void cp_async16(void *dst, const void *src, int src_bytes)
@@ -134,72 +117,30 @@ __device__ __forceinline__ void mma_f16(float (&d)[4], const uint32_t (&a)[4], u
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// The work of one CTA (group * n_qblk + query block, kv head, split) by 128 threads; `sync` is the
-// barrier of those threads.  Also the attention phase of the persistent layer kernel, which runs
-// it on four-warp groups over virtual block indices.
-struct AttnCtaSync {
-    __device__ void operator()() const { __syncthreads(); }
-};
-template <int HD, int MT, int NS, class Sync>
-__device__ __forceinline__ void attn_partial_body(const AttnArgs &a, int bx, int hk, int sp, unsigned char *at_smem, int tid,
-                                                  Sync sync)
+// One item, by one warp: query vectors [16 qb, 16 qb + 16) of a group whose first row is row0
+// (nrows rows of slot `slot`, first at position pos0), kv head hk, split sp of `splits` splits of
+// split_len positions.  `wr` is the warp's ring of NS stages.  Writes the item's partial.
+// QREG: the query fragments stay in registers for the whole item (32 registers at head dimension
+// 128); otherwise they are parked in `qs` ([16][HD + 8] of shared memory) and re-read per tile,
+// for callers whose register budget is spoken for.
+template <int HD, int NS, bool QREG>
+__device__ __forceinline__ void attn_item(const AttnArgs &a, int qb, int hk, int sp, int splits, int split_len, int row0,
+                                          int nrows, int slot, int pos0, kv_t *wr, kv_t *qs, int lane)
 {
-    constexpr int QB = 16 * MT;     // query vectors per CTA
     constexpr int KP = HD + 8;      // padded row: ldmatrix rows fall into distinct banks
     constexpr int CH = HD / 8;      // 16-byte chunks per row
-    kv_t *Qs = reinterpret_cast<kv_t *>(at_smem);  // [QB][KP] hi terms
-    kv_t *Ql = Qs + QB * KP;                       // [QB][KP] lo terms
-    kv_t *ring = Ql + QB * KP;                     // [4 warps][NS][K,V][AT_TP][KP]
-
-    const int g = bx / a.n_qblk, qb = bx % a.n_qblk;
-    if (g >= *a.n_groups) return;
+    constexpr float LOG2E = 1.4426950408889634f, LN2 = 0.6931471805599453f;
     const int G = a.Hq / a.Hkv;
-    const int row0 = a.grp_row0[g], nrows = a.grp_nrows[g];
-    if (row0 < 0 || nrows < 1 || row0 + nrows > a.n_rows) return;
-    const int nq = nrows * G;
-    const int q0 = qb * QB;
-    if (q0 >= nq || nq < a.nq_min || nq > a.nq_max) return;
-    const int nq_here = min(QB, nq - q0);
-    const int slot = a.row_slot[row0], pos0 = a.row_pos[row0];
-    const int lane = tid & 31, warp = tid >> 5;
-
-    // positions this CTA may look at: its split, cut at the last query row's own position
-    // (and at the cache itself: a descriptor that points outside it reads nothing)
-    const int last_row = (q0 + nq_here - 1) / G;
+    const int nq = nrows * G, q0 = qb * 16;
+    const int nq_here = min(16, nq - q0);
+    // positions this item may look at: its split, cut at the last query row's own position
+    // (and at the cache itself: a row that points outside it reads nothing)
     const bool sane = slot >= 0 && slot < a.n_slots && pos0 >= 0;
+    const int last_row = (q0 + nq_here - 1) / G;
     const int kv_end_all = sane ? min(pos0 + last_row + 1, a.S) : 0;
-    const int s_beg = sp * a.split_len;
-    const int s_end = min(s_beg + a.split_len, kv_end_all);
-
-    for (int i = tid; i < QB * CH; i += AT_THREADS) {
-        const int qi = i / CH, c = i % CH;
-        uint4 hi = make_uint4(0, 0, 0, 0), lo = hi;
-        if (qi < nq_here) {
-            const int qg = q0 + qi, r = qg / G, j = qg % G;
-            const size_t off = (size_t)(row0 + r) * a.Hq * HD + (hk * G + j) * HD + c * 8;
-            if (a.q32) {
-                const float4 x0 = *reinterpret_cast<const float4 *>(a.q32 + off);
-                const float4 x1 = *reinterpret_cast<const float4 *>(a.q32 + off + 4);
-                const float v[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-                split8_h(v, hi, lo);
-            } else {
-                float v[8];
-                unpack8(*reinterpret_cast<const uint4 *>(a.q + off), v);  // bf16 queries, widened
-                split8_h(v, hi, lo);
-            }
-        }
-        *reinterpret_cast<uint4 *>(&Qs[qi * KP + c * 8]) = hi;
-        *reinterpret_cast<uint4 *>(&Ql[qi * KP + c * 8]) = lo;
-    }
-    sync();
-
-    // this warp's share of the split
-    const int span = max(s_end - s_beg, 0);
-    const int per = (((span + 3) >> 2) + AT_TP - 1) / AT_TP * AT_TP;
-    const int w_beg = s_beg + warp * per;
-    const int w_end = min(w_beg + per, s_end);
+    const int w_beg = sp * split_len;
+    const int w_end = min(w_beg + split_len, kv_end_all);
     const int n_tiles = w_end > w_beg ? (w_end - w_beg + AT_TP - 1) / AT_TP : 0;
-    kv_t *wr = ring + (size_t)warp * NS * 2 * AT_TP * KP;
     const kv_t *kbase = a.kc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
     const kv_t *vbase = a.vc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
 
@@ -215,106 +156,162 @@ __device__ __forceinline__ void attn_partial_body(const AttnArgs &a, int bx, int
             cp_async16(&vt[r * KP + c * 8], vbase + off, ok ? 16 : 0);
         }
     };
-
-    float o[MT][HD / 8][4], m_run[MT][2], l_run[MT][2];
+    // The ring: tiles t .. t + NS - 1 are in flight or in use while tile t is computed; every
+    // refill is its own commit group (empty ones included), so "all but the newest NS - 1 groups"
+    // always means "tile t has landed".
+    __syncwarp();  // the previous item's last reads of the ring are over
 #pragma unroll
-    for (int mt = 0; mt < MT; mt++) {
-        m_run[mt][0] = m_run[mt][1] = -INFINITY;
-        l_run[mt][0] = l_run[mt][1] = 0.f;
-#pragma unroll
-        for (int nt = 0; nt < HD / 8; nt++)
-#pragma unroll
-            for (int e = 0; e < 4; e++) o[mt][nt][e] = 0.f;
-    }
-    // last position each of this thread's accumulator rows may see
-    int limit[MT][2];
-#pragma unroll
-    for (int mt = 0; mt < MT; mt++)
-#pragma unroll
-        for (int hf = 0; hf < 2; hf++) {
-            const int qi = mt * 16 + (lane >> 2) + hf * 8;
-            limit[mt][hf] = qi < nq_here ? pos0 + (q0 + qi) / G : -1;
-        }
-    const float scale = rsqrtf((float)HD);
-
-#pragma unroll
-    for (int t = 0; t < NS - 1; t++) {
+    for (int t = 0; t < NS; t++) {
         if (t < n_tiles) issue(t);
         cp_async_commit();
     }
+
+    // the queries, as A fragments (row = lane / 4 and + 8, columns 2 (lane % 4) + {0, 1, 8, 9} of
+    // every 16-column step), while the first tiles are on their way
+    uint32_t qa[QREG ? HD / 16 : 1][4];
+    const float qscale = rsqrtf((float)HD) * LOG2E;
+    {
+        const int qi0 = lane >> 2, qi1 = qi0 + 8, c0 = (lane & 3) * 2;
+        const bool h0 = qi0 < nq_here && n_tiles > 0, h1 = qi1 < nq_here && n_tiles > 0;
+        const int g0 = q0 + (h0 ? qi0 : 0), g1 = q0 + (h1 ? qi1 : 0);
+        const size_t o0 = (size_t)(row0 + g0 / G) * a.Hq * HD + (hk * G + g0 % G) * HD + c0;
+        const size_t o1 = (size_t)(row0 + g1 / G) * a.Hq * HD + (hk * G + g1 % G) * HD + c0;
+#pragma unroll
+        for (int ks = 0; ks < HD / 16; ks++) {
+            float2 x00 = make_float2(0.f, 0.f), x01 = x00, x10 = x00, x11 = x00;
+            if (a.q32) {
+                if (h0) {
+                    x00 = *reinterpret_cast<const float2 *>(a.q32 + o0 + ks * 16);
+                    x01 = *reinterpret_cast<const float2 *>(a.q32 + o0 + ks * 16 + 8);
+                }
+                if (h1) {
+                    x10 = *reinterpret_cast<const float2 *>(a.q32 + o1 + ks * 16);
+                    x11 = *reinterpret_cast<const float2 *>(a.q32 + o1 + ks * 16 + 8);
+                }
+            } else {
+                if (h0) {
+                    const uint32_t u0 = *reinterpret_cast<const uint32_t *>(a.q + o0 + ks * 16);
+                    const uint32_t u1 = *reinterpret_cast<const uint32_t *>(a.q + o0 + ks * 16 + 8);
+                    x00 = make_float2(bf_lo(u0), bf_hi(u0));
+                    x01 = make_float2(bf_lo(u1), bf_hi(u1));
+                }
+                if (h1) {
+                    const uint32_t u0 = *reinterpret_cast<const uint32_t *>(a.q + o1 + ks * 16);
+                    const uint32_t u1 = *reinterpret_cast<const uint32_t *>(a.q + o1 + ks * 16 + 8);
+                    x10 = make_float2(bf_lo(u0), bf_hi(u0));
+                    x11 = make_float2(bf_lo(u1), bf_hi(u1));
+                }
+            }
+            const uint32_t f0 = pack_h2(x00.x * qscale, x00.y * qscale), f1 = pack_h2(x10.x * qscale, x10.y * qscale);
+            const uint32_t f2 = pack_h2(x01.x * qscale, x01.y * qscale), f3 = pack_h2(x11.x * qscale, x11.y * qscale);
+            if (QREG) {
+                qa[ks][0] = f0; qa[ks][1] = f1; qa[ks][2] = f2; qa[ks][3] = f3;
+            } else {
+                *reinterpret_cast<uint32_t *>(&qs[qi0 * KP + ks * 16 + c0]) = f0;
+                *reinterpret_cast<uint32_t *>(&qs[qi1 * KP + ks * 16 + c0]) = f1;
+                *reinterpret_cast<uint32_t *>(&qs[qi0 * KP + ks * 16 + c0 + 8]) = f2;
+                *reinterpret_cast<uint32_t *>(&qs[qi1 * KP + ks * 16 + c0 + 8]) = f3;
+            }
+        }
+        if (!QREG) __syncwarp();
+    }
+
+    float o[HD / 8][4], m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+#pragma unroll
+    for (int nt = 0; nt < HD / 8; nt++)
+#pragma unroll
+        for (int e = 0; e < 4; e++) o[nt][e] = 0.f;
+    // last position each of this thread's two accumulator rows may see
+    int limit[2];
+#pragma unroll
+    for (int hf = 0; hf < 2; hf++) {
+        const int qi = (lane >> 2) + hf * 8;
+        limit[hf] = qi < nq_here ? pos0 + (q0 + qi) / G : -1;
+    }
+    const int lim_min = pos0 + q0 / G;  // the smallest limit among the item's query vectors
+
     for (int t = 0; t < n_tiles; t++) {
-        cp_async_wait<NS - 2>();
+        cp_async_wait<NS - 1>();  // tile t has landed
         __syncwarp();
-        if (t + NS - 1 < n_tiles) issue(t + NS - 1);
-        cp_async_commit();
         const kv_t *Kt = wr + (size_t)(t % NS) * 2 * AT_TP * KP, *Vt = Kt + AT_TP * KP;
         const int p0 = w_beg + t * AT_TP;
 
-        // S = Q K^T for 16 positions
-        float s[MT][2][4];
+        // S = Q K^T for 16 positions, in log2 units; two accumulator chains
+        float s[2][4], s2[2][4];
 #pragma unroll
-        for (int mt = 0; mt < MT; mt++)
+        for (int nt = 0; nt < 2; nt++)
+#pragma unroll
+            for (int e = 0; e < 4; e++) s[nt][e] = s2[nt][e] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < HD / 16; ks += 2) {
+            uint32_t kb[4], kb2[4];
+            ldsm_x4(kb, &Kt[((lane & 7) + ((lane >> 4) << 3)) * KP + ks * 16 + ((lane >> 3) & 1) * 8]);
+            ldsm_x4(kb2, &Kt[((lane & 7) + ((lane >> 4) << 3)) * KP + (ks + 1) * 16 + ((lane >> 3) & 1) * 8]);
+            if (QREG) {
+                mma_f16(s[0], qa[ks], kb[0], kb[1]);
+                mma_f16(s[1], qa[ks], kb[2], kb[3]);
+                mma_f16(s2[0], qa[ks + 1], kb2[0], kb2[1]);
+                mma_f16(s2[1], qa[ks + 1], kb2[2], kb2[3]);
+            } else {
+                uint32_t q1[4], q2[4];
+                const int qoff = ((lane & 7) + ((lane >> 3) & 1) * 8) * KP + (lane >> 4) * 8;
+                ldsm_x4(q1, &qs[qoff + ks * 16]);
+                ldsm_x4(q2, &qs[qoff + (ks + 1) * 16]);
+                mma_f16(s[0], q1, kb[0], kb[1]);
+                mma_f16(s[1], q1, kb[2], kb[3]);
+                mma_f16(s2[0], q2, kb2[0], kb2[1]);
+                mma_f16(s2[1], q2, kb2[2], kb2[3]);
+            }
+        }
+        // online softmax; P as the A operand of the second product.  A tile wholly inside what
+        // every query vector of the item may see (all but the last of an item) needs no masking;
+        // accumulator rows without a query vector then carry numbers nobody reads.
+        const bool full = p0 + AT_TP <= w_end && p0 + AT_TP - 1 <= lim_min;
+        uint32_t pa[4];
+        float alpha[2];
+#pragma unroll
+        for (int hf = 0; hf < 2; hf++) {
+            float v[4];
+            float tmax = -INFINITY;
 #pragma unroll
             for (int nt = 0; nt < 2; nt++)
 #pragma unroll
-                for (int e = 0; e < 4; e++) s[mt][nt][e] = 0.f;
+                for (int e = 0; e < 2; e++) {
+                    const int p = p0 + nt * 8 + (lane & 3) * 2 + e;
+                    const bool ok = full || (p < w_end && p <= limit[hf]);
+                    v[nt * 2 + e] = ok ? s[nt][hf * 2 + e] + s2[nt][hf * 2 + e] : -INFINITY;
+                    tmax = fmaxf(tmax, v[nt * 2 + e]);
+                }
+            tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
+            tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
+            const float m_new = fmaxf(m_run[hf], tmax);
+            float psum = 0.f;
+            alpha[hf] = 1.f;
+            if (m_new != -INFINITY) {
+                alpha[hf] = exp2f(m_run[hf] - m_new);  // 2^(-inf) = 0 on the first live tile
 #pragma unroll
-        for (int ks = 0; ks < HD / 16; ks++) {
-            uint32_t kb[4];
-            ldsm_x4(kb, &Kt[((lane & 7) + ((lane >> 4) << 3)) * KP + ks * 16 + ((lane >> 3) & 1) * 8]);
+                for (int i = 0; i < 4; i++) {
+                    v[i] = exp2f(v[i] - m_new);
+                    psum += v[i];
+                }
+            } else {
 #pragma unroll
-            for (int mt = 0; mt < MT; mt++) {
-                uint32_t qa[4], ql[4];
-                const int qoff = (mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * KP + ks * 16 + (lane >> 4) * 8;
-                ldsm_x4(qa, &Qs[qoff]);
-                ldsm_x4(ql, &Ql[qoff]);
-                mma_f16(s[mt][0], qa, kb[0], kb[1]);
-                mma_f16(s[mt][1], qa, kb[2], kb[3]);
-                mma_f16(s[mt][0], ql, kb[0], kb[1]);
-                mma_f16(s[mt][1], ql, kb[2], kb[3]);
+                for (int i = 0; i < 4; i++) v[i] = 0.f;
             }
+            l_run[hf] = l_run[hf] * alpha[hf] + psum;  // per-thread share; lanes are summed at the end
+            m_run[hf] = m_new;
+            pa[hf] = pack_h2(v[0], v[1]);      // positions 0..7 of the tile
+            pa[2 + hf] = pack_h2(v[2], v[3]);  // positions 8..15
         }
-        // online softmax; P as the A operand of the second product
-        uint32_t pa[MT][4], pl[MT][4];
+        // the accumulator is rescaled only when some row's maximum moved (after the first tiles
+        // of an item that is rare)
+        if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) {
 #pragma unroll
-        for (int mt = 0; mt < MT; mt++) {
-#pragma unroll
-            for (int hf = 0; hf < 2; hf++) {
-                float v[4];
-                float tmax = -INFINITY;
-#pragma unroll
-                for (int nt = 0; nt < 2; nt++)
-#pragma unroll
-                    for (int e = 0; e < 2; e++) {
-                        const int p = p0 + nt * 8 + (lane & 3) * 2 + e;
-                        const bool ok = p < w_end && p <= limit[mt][hf];
-                        v[nt * 2 + e] = ok ? s[mt][nt][hf * 2 + e] * scale : -INFINITY;
-                        tmax = fmaxf(tmax, v[nt * 2 + e]);
-                    }
-                tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
-                tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
-                const float m_new = fmaxf(m_run[mt][hf], tmax);
-                float alpha = 1.f, psum = 0.f;
-                if (m_new != -INFINITY) {
-                    alpha = __expf(m_run[mt][hf] - m_new);  // exp(-inf) = 0 on the first live tile
-#pragma unroll
-                    for (int i = 0; i < 4; i++) {
-                        v[i] = __expf(v[i] - m_new);
-                        psum += v[i];
-                    }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 4; i++) v[i] = 0.f;
-                }
-                l_run[mt][hf] = l_run[mt][hf] * alpha + psum;  // per-thread share; lanes are summed at the end
-                m_run[mt][hf] = m_new;
-                split_pair_h(v[0], v[1], pa[mt][hf], pl[mt][hf]);          // positions 0..7 of the tile
-                split_pair_h(v[2], v[3], pa[mt][2 + hf], pl[mt][2 + hf]);  // positions 8..15
-#pragma unroll
-                for (int nt = 0; nt < HD / 8; nt++) {
-                    o[mt][nt][hf * 2] *= alpha;
-                    o[mt][nt][hf * 2 + 1] *= alpha;
-                }
+            for (int nt = 0; nt < HD / 8; nt++) {
+                o[nt][0] *= alpha[0];
+                o[nt][1] *= alpha[0];
+                o[nt][2] *= alpha[1];
+                o[nt][3] *= alpha[1];
             }
         }
         // O += P V
@@ -322,87 +319,81 @@ __device__ __forceinline__ void attn_partial_body(const AttnArgs &a, int bx, int
         for (int np = 0; np < HD / 16; np++) {
             uint32_t vb[4];
             ldsm_x4_t(vb, &Vt[((lane & 7) + ((lane >> 3) & 1) * 8) * KP + np * 16 + (lane >> 4) * 8]);
-#pragma unroll
-            for (int mt = 0; mt < MT; mt++) {
-                mma_f16(o[mt][2 * np], pa[mt], vb[0], vb[1]);
-                mma_f16(o[mt][2 * np + 1], pa[mt], vb[2], vb[3]);
-                mma_f16(o[mt][2 * np], pl[mt], vb[0], vb[1]);
-                mma_f16(o[mt][2 * np + 1], pl[mt], vb[2], vb[3]);
-            }
+            mma_f16(o[2 * np], pa, vb[0], vb[1]);
+            mma_f16(o[2 * np + 1], pa, vb[2], vb[3]);
         }
+        __syncwarp();  // every lane is done with this stage: refill it
+        if (t + NS < n_tiles) issue(t + NS);
+        cp_async_commit();
     }
     cp_async_wait<0>();
-    sync();  // every warp is done with its ring: reuse it for the merge
-
-    // merge the four warps' states
-    float *Ow = reinterpret_cast<float *>(ring);   // [4][QB][HD]
-    float *mw = Ow + 4 * QB * HD, *lw = mw + 4 * QB;  // [4][QB] each
+    // this item's partial (an empty split leaves max = -inf, sum = 0, which the merge ignores)
 #pragma unroll
-    for (int mt = 0; mt < MT; mt++)
+    for (int hf = 0; hf < 2; hf++) {
+        float l = l_run[hf];
+        l += __shfl_xor_sync(0xffffffffu, l, 1);
+        l += __shfl_xor_sync(0xffffffffu, l, 2);
+        const int qi = (lane >> 2) + hf * 8;
+        if (qi < nq_here) {
+            const int qg = q0 + qi, r = qg / G, j = qg % G;
+            const size_t cell = ((size_t)(row0 + r) * a.Hq + hk * G + j) * splits + sp;
+            if ((lane & 3) == 0) a.part_ml[cell] = make_float2(m_run[hf] * LN2, l);  // max back in natural-log units
 #pragma unroll
-        for (int hf = 0; hf < 2; hf++) {
-            float l = l_run[mt][hf];
-            l += __shfl_xor_sync(0xffffffffu, l, 1);
-            l += __shfl_xor_sync(0xffffffffu, l, 2);
-            const int qi = mt * 16 + (lane >> 2) + hf * 8;
-            if ((lane & 3) == 0) {
-                mw[warp * QB + qi] = m_run[mt][hf];
-                lw[warp * QB + qi] = l;
-            }
-#pragma unroll
-            for (int nt = 0; nt < HD / 8; nt++) {
-                float2 v2 = make_float2(o[mt][nt][hf * 2], o[mt][nt][hf * 2 + 1]);
-                *reinterpret_cast<float2 *>(&Ow[((size_t)warp * QB + qi) * HD + nt * 8 + (lane & 3) * 2]) = v2;
-            }
+            for (int nt = 0; nt < HD / 8; nt++)
+                *reinterpret_cast<float2 *>(a.part_o + cell * HD + nt * 8 + (lane & 3) * 2) =
+                    make_float2(o[nt][hf * 2], o[nt][hf * 2 + 1]);
         }
-    sync();
-    // partials (an empty split leaves max = -inf, sum = 0, which the merge of the splits ignores)
-    for (int idx = tid; idx < nq_here * HD; idx += AT_THREADS) {
-        const int qi = idx / HD, d = idx % HD;
-        float M = -INFINITY;
-#pragma unroll
-        for (int w = 0; w < 4; w++) M = fmaxf(M, mw[w * QB + qi]);
-        float acc = 0.f, L = 0.f;
-#pragma unroll
-        for (int w = 0; w < 4; w++) {
-            const float mwv = mw[w * QB + qi];
-            if (mwv == -INFINITY) continue;
-            const float wgt = __expf(mwv - M);
-            acc += Ow[((size_t)w * QB + qi) * HD + d] * wgt;
-            L += lw[w * QB + qi] * wgt;
-        }
-        const int qg = q0 + qi, r = qg / G, j = qg % G;
-        const size_t cell = ((size_t)(row0 + r) * a.Hq + hk * G + j) * a.n_splits + sp;
-        a.part_o[cell * HD + d] = acc;
-        if (d == 0) a.part_ml[cell] = make_float2(M, L);
     }
 }
 
-template <int HD, int MT>
-__global__ void __launch_bounds__(AT_THREADS) attn_partial_kernel(AttnArgs a)
+// Persistent grid of warps; item i = ((g * n_qblk + qb) * Hkv + hk) * n_splits + sp goes to warp
+// i mod (number of warps), warps numbered so that consecutive items land on different SMs.
+template <int HD, int NST>
+__global__ void __launch_bounds__(AW_WARPS * 32) attn_warp_kernel(AttnArgs a)
 {
-    extern __shared__ __align__(16) unsigned char at_smem_dyn[];
+    extern __shared__ __align__(16) unsigned char aw_smem[];
     griddep_launch();
     griddep_wait();
-    attn_partial_body<HD, MT, (MT == 2 ? 2 : AT_NST)>(a, blockIdx.x, blockIdx.y, blockIdx.z, at_smem_dyn, threadIdx.x,
-                                                      AttnCtaSync());
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    kv_t *wr = reinterpret_cast<kv_t *>(aw_smem) + (size_t)warp * NST * 2 * AT_TP * (HD + 8);
+    const int G = a.Hq / a.Hkv;
+    const int n_groups = min(*a.n_groups, a.max_groups);
+    const long n_items = (long)n_groups * a.n_qblk * a.Hkv * a.n_splits;
+    const long n_workers = (long)gridDim.x * AW_WARPS;
+    for (long item = (long)warp * gridDim.x + blockIdx.x; item < n_items; item += n_workers) {
+        long t = item;
+        const int sp = (int)(t % a.n_splits); t /= a.n_splits;
+        const int hk = (int)(t % a.Hkv); t /= a.Hkv;
+        const int qb = (int)(t % a.n_qblk), g = (int)(t / a.n_qblk);
+        const int row0 = a.grp_row0[g], nrows = a.grp_nrows[g];
+        if (row0 < 0 || nrows < 1 || row0 + nrows > a.n_rows) continue;
+        const int nq = nrows * G;
+        if (qb * 16 >= nq || nq < a.nq_min || nq > a.nq_max) continue;
+        attn_item<HD, NST, true>(a, qb, hk, sp, a.n_splits, a.split_len, row0, nrows, a.row_slot[row0], a.row_pos[row0], wr,
+                                    nullptr, lane);
+    }
 }
 
-typedef void (*AttnPartialFn)(AttnArgs);
-// The instantiation for a head dimension (64 or 128) and a query block of 16 * mt vectors, with
-// its dynamic shared-memory limit raised on first use.
-inline cudaError_t attn_partial_fn(int head_dim, int mt, AttnPartialFn *fn)
+// The grid of the stand-alone kernel: as many CTAs as fit the SMs (registers allow three).
+inline int attn_warp_ctas_per_sm(int head_dim, int stages)
+{
+    const size_t per_cta = AW_WARPS * attn_warp_bytes(head_dim, stages) + 1024;
+    const int by_smem = (int)((size_t)227 * 1024 / per_cta);
+    return by_smem < 1 ? 1 : (by_smem > 3 ? 3 : by_smem);
+}
+typedef void (*AttnWarpFn)(AttnArgs);
+// The instantiation for a head dimension (64 or 128) and a ring depth (2 or 3), its dynamic
+// shared-memory limit raised on first use.
+inline cudaError_t attn_warp_fn(int head_dim, int stages, AttnWarpFn *fn)
 {
     static PerDevice<bool> ready_dev[4];
-    const int idx = (head_dim == 128 ? 2 : 0) + (mt == 2 ? 1 : 0);
-    AttnPartialFn f = idx == 3 ? attn_partial_kernel<128, 2>
-                      : idx == 2 ? attn_partial_kernel<128, 1>
-                      : idx == 1 ? attn_partial_kernel<64, 2>
-                                 : attn_partial_kernel<64, 1>;
+    const int idx = (head_dim == 128 ? 2 : 0) + (stages == 3 ? 1 : 0);
+    AttnWarpFn f = idx == 3 ? attn_warp_kernel<128, 3> : idx == 2 ? attn_warp_kernel<128, 2>
+                   : idx == 1 ? attn_warp_kernel<64, 3> : attn_warp_kernel<64, 2>;
     bool &ready = ready_dev[idx].here();
     if (!ready) {
         const cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   (int)attn_smem_bytes(head_dim, mt));
+                                                   (int)(AW_WARPS * attn_warp_bytes(head_dim, stages)));
         if (e != cudaSuccess) return e;
         ready = true;
     }

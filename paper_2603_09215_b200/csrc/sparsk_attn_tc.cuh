@@ -2,22 +2,23 @@
 //
 // A refresh step of a sequence with 16 query heads per kv head and three pending positions has
 // 64 query vectors that share one K/V stream (Algorithm 1: the pending positions and the current
-// one go through the upper layers as one causal block).  With two-term fp16 operands that is 128
-// flop per cache byte: beyond what mma.sync delivers, so the block kernel of sparsk_attn.cuh is
-// tensor-bound there.  This kernel runs the same arithmetic on tcgen05:
+// one go through the upper layers as one causal block): 64 flop per cache byte and more for
+// prefill chunks, where the warp-per-item mma.sync kernel of sparsk_attn.cuh would re-read the
+// cache once per 16 query vectors.  This kernel runs the same arithmetic on tcgen05 (queries and
+// softmax weights rounded to fp16 once, like the cache they multiply):
 //
-//   S = Q K^T : A = the block's query vectors (up to 128 rows, hi and lo fp16 planes) held in TMEM,
+//   S = Q K^T : A = the block's query vectors (up to 128 rows, fp16) held in TMEM,
 //               stored there once with tcgen05.st (lane = query vector, elements packed two per
 //               column); B = a [64 positions x 128] K tile exactly as TMA delivers it from the
 //               cache (K-major); accumulator [128 x 64] fp32 in TMEM
-//   O += P V  : A = the tile's softmax weights (hi and lo planes), written by the softmax warps
+//   O += P V  : A = the tile's softmax weights (fp16), written by the softmax warps
 //               straight into TMEM; B = the V tile as delivered (positions x head dim = MN-major);
 //               accumulated over all tiles in a [128 x 128] fp32 TMEM accumulator that the softmax
 //               warps rescale in place (tcgen05.ld / st) when a tile raises a row's reference maximum
 // With both A operands in TMEM an MMA reads only its K or V slice from shared memory (2 or 4 KB
 // instead of 6 or 8): with the operands in shared memory the MMAs ran at 80 and 120 cycles each
-// against 32 and 64 at the tensor rate.  All 512 TMEM columns are used: scores 2 x 64, output
-// 128, weights 2 x 64, queries 128.
+// against 32 and 64 at the tensor rate.  TMEM columns: scores 2 x 64, output 128, weights 2 x 32
+// (of a 64-column slot each), queries 64 (of 128).
 //
 // CTA = (group, block of 128 query vectors, kv head, KV split); warp 0 issues the TMA copies of a
 // K ring (TA_KST tiles) and a V ring (TA_VST tiles), warp 1 issues the MMAs and owns the TMEM
@@ -168,7 +169,7 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
     const uint32_t tmem_base = tmem_base_s;
     const uint32_t t_s0 = tmem_base + TA_C_S, t_o = tmem_base + TA_C_O, t_p = tmem_base + TA_C_P, t_q = tmem_base + TA_C_Q;
 
-    // ---- the queries, as two fp16 planes in TMEM (thread = query vector = lane; 16-bit elements
+    // ---- the queries, as an fp16 plane in TMEM (thread = query vector = lane; 16-bit elements
     // packed two per column): the A operand of every score MMA, stored once.  The two warps of a
     // lane quadrant take 64 of the 128 head dimensions each.
     if (warp >= 2 && n_tiles > 0) {
@@ -179,21 +180,18 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
 #pragma unroll
         for (int blk = 0; blk < 2; blk++) {  // 32 elements = 16 packed columns per store
-            uint32_t hi[16], lo[16];
+            uint32_t hi[16];
 #pragma unroll
             for (int c = 0; c < 4; c++) {
-                uint4 h4 = make_uint4(0, 0, 0, 0), l4 = h4;
+                uint4 h4 = make_uint4(0, 0, 0, 0);
                 if (have) {
                     const float4 x0 = *reinterpret_cast<const float4 *>(src + blk * 32 + c * 8);
                     const float4 x1 = *reinterpret_cast<const float4 *>(src + blk * 32 + c * 8 + 4);
-                    const float v[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-                    split8_h(v, h4, l4);
+                    h4 = make_uint4(pack_h2(x0.x, x0.y), pack_h2(x0.z, x0.w), pack_h2(x1.x, x1.y), pack_h2(x1.z, x1.w));
                 }
                 hi[c * 4] = h4.x; hi[c * 4 + 1] = h4.y; hi[c * 4 + 2] = h4.z; hi[c * 4 + 3] = h4.w;
-                lo[c * 4] = l4.x; lo[c * 4 + 1] = l4.y; lo[c * 4 + 2] = l4.z; lo[c * 4 + 3] = l4.w;
             }
             tmem_st16(t_q + lane_addr + (uint32_t)(half * 32 + blk * 16), hi);
-            tmem_st16(t_q + lane_addr + 64 + (uint32_t)(half * 32 + blk * 16), lo);
         }
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
     }
@@ -243,7 +241,6 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
                 for (int kk = 0; kk < TA_HD / 16; kk++) {  // 16 head dimensions = 8 packed TMEM columns of the queries
                     const uint64_t db = dk0 + (uint64_t)(((kk >> 2) * 8192 + (kk & 3) * 32) >> 4);
                     umma_f16_ts(d, t_q + (uint32_t)kk * 8, db, idesc_s, kk > 0);
-                    umma_f16_ts(d, t_q + 64 + (uint32_t)kk * 8, db, idesc_s, 1);
                 }
                 umma_commit(&k_empty[st]);  // the K tile is free once the scores are computed
                 umma_commit(&s_full[b]);
@@ -259,12 +256,11 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
                 if (!(ok = mbar_wait(&p_full[b], (t >> 1) & 1, giving_up, args.status))) break;
                 tc_fence_after();
                 const uint64_t dv0 = umma_desc_sw128_mn(v0 + (uint32_t)st * TA_T_BYTES, 8192);
-                const uint32_t tp = t_p + (uint32_t)b * 64;  // this tile's weights: hi plane, lo plane 32 columns on
+                const uint32_t tp = t_p + (uint32_t)b * 64;  // this tile's weights
 #pragma unroll
                 for (int kk = 0; kk < TA_NT / 16; kk++) {  // 16 positions = 8 packed columns
                     const uint64_t dv = dv0 + (uint64_t)((kk * 2048) >> 4);
                     umma_f16_ts(t_o, tp + (uint32_t)kk * 8, dv, idesc_o, t > 0 || kk > 0);
-                    umma_f16_ts(t_o, tp + 32 + (uint32_t)kk * 8, dv, idesc_o, 1);
                 }
                 umma_commit(&v_empty[st]);  // the V tile and this buffer of weights are free once these have read them
                 umma_commit(&o_full[b]);
@@ -365,7 +361,7 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
                     break;
                 }
                 // The reference maximum is allowed to lag the true one by TA_RAISE (weights then reach
-                // 2^11, which two fp16 terms and fp32 sums carry without loss): otherwise some lane of
+                // 2^11, which fp16 and fp32 sums carry at full precision): otherwise some lane of
                 // the warp would see a new maximum in most tiles and the accumulator would be
                 // rescaled nearly every time.  Partials stay exact: (o, l) are relative to m_run.
                 const bool raise = tmax > m_run + TA_RAISE;
@@ -373,7 +369,7 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
                 const float factor = raise ? exp2f(m_run - m_new) : 1.f;  // 2^(-inf) = 0 on the first live tile
                 const float m_ref = m_new == -INFINITY ? 0.f : m_new;    // a row that has seen nothing yet: all weights 0
                 float psum = 0.f;
-                uint4 whi[4], wlo[4];
+                uint4 whi[4];
 #pragma unroll
                 for (int c = 0; c < 4; c++) {
                     float w[8];
@@ -382,7 +378,7 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
                         w[i] = exp2f(__uint_as_float(sr[c >> 1][(c & 1) * 8 + i]) - m_ref);  // 2^(-inf) = 0 for masked positions
                         psum += w[i];
                     }
-                    split8_h(w, whi[c], wlo[c]);
+                    whi[c] = make_uint4(pack_h2(w[0], w[1]), pack_h2(w[2], w[3]), pack_h2(w[4], w[5]), pack_h2(w[6], w[7]));
                 }
                 // The weights go to buffer b, which the product of tile t - 2 has read by the time
                 // o_full[b] completes; a rescaling needs every product so far in the accumulator.  A
@@ -416,15 +412,13 @@ __global__ void __launch_bounds__(TA_THREADS, 1)
                     }
                 }
                 if (ok) {
-                    uint32_t ph[16], pl[16];
+                    uint32_t ph[16];
 #pragma unroll
                     for (int c = 0; c < 4; c++) {
                         ph[c * 4] = whi[c].x; ph[c * 4 + 1] = whi[c].y; ph[c * 4 + 2] = whi[c].z; ph[c * 4 + 3] = whi[c].w;
-                        pl[c * 4] = wlo[c].x; pl[c * 4 + 1] = wlo[c].y; pl[c * 4 + 2] = wlo[c].z; pl[c * 4 + 3] = wlo[c].w;
                     }
                     const uint32_t tp = t_p + lane_addr + (uint32_t)(b * 64 + half * 16);
                     tmem_st16(tp, ph);
-                    tmem_st16(tp + 32, pl);
                     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                     tc_fence_before();
                     mbar_arrive(&p_full[b]);

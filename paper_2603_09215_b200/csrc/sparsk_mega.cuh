@@ -53,7 +53,7 @@ constexpr int MK_MAX_SPLITS = 32;             // the merge keeps one split per l
 // phase moves along), or the attention warps' query blocks and K/V rings.
 inline size_t mk_attn_bytes(int head_dim)
 {
-    return (size_t)MK_ATT_WARPS * (2 * 16 + MK_ATT_NST * 2 * AT_TP) * (head_dim + 8) * 2;
+    return (size_t)MK_ATT_WARPS * (16 * (head_dim + 8) * 2 + attn_warp_bytes(head_dim, MK_ATT_NST));
 }
 // k-steps of M fp32 activation rows that fit the area
 __host__ __device__ inline int mk_act_window(int M) { return MK_AREA_BYTES / (M * MK_BOX_COLS * 4); }

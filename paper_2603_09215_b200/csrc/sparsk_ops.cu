@@ -1,6 +1,7 @@
 // Stand-alone entry points for single kernels of the decode path (C ABI in include/sparsk.h).
 // They run exactly the kernels a decode step runs, on caller-described inputs, so that one
 // stage can be driven, checked and profiled on its own.
+#include <algorithm>
 #include <cstdint>
 
 #include "../../include/sparsk.h"
@@ -54,15 +55,18 @@ int sparsk_attention_launch(const sparsk_attn_args *p, char *scratch, cudaStream
     a.out = (bf16 *)p->out;
     a.Hq = p->n_q_heads; a.Hkv = p->n_kv_heads; a.S = p->cache_len; a.n_slots = p->n_slots; a.n_rows = p->n_rows;
     a.nq_min = 0; a.nq_max = 1 << 30;
-    const AttnPlan pl = attn_plan(n_sm, p->n_groups, p->max_grp_rows, p->n_q_heads / p->n_kv_heads,
+    const int warp_ctas = n_sm * attn_warp_ctas_per_sm(p->head_dim, AW_NST);
+    const AttnPlan pl = attn_plan(warp_ctas * AW_WARPS, p->n_groups, p->max_grp_rows, p->n_q_heads / p->n_kv_heads,
                                   p->n_kv_heads, p->max_len, 0);
     a.n_qblk = pl.n_qblk; a.split_len = pl.split_len; a.n_splits = pl.n_splits;
+    a.max_groups = p->n_groups;
     set_int_kernel<<<1, 1, 0, st>>>(counts, p->n_groups);
     set_int_kernel<<<1, 1, 0, st>>>(counts + 1, p->n_rows);
-    const dim3 grid(p->n_groups * pl.n_qblk, p->n_kv_heads, pl.n_splits);
-    AttnPartialFn fn;
-    if (attn_partial_fn(p->head_dim, pl.mt, &fn) != cudaSuccess) return SPARSK_ECUDA;
-    fn<<<grid, AT_THREADS, attn_smem_bytes(p->head_dim, pl.mt), st>>>(a);
+    const long n_items = (long)p->n_groups * pl.n_qblk * p->n_kv_heads * pl.n_splits;
+    const int grid = (int)std::max<long>(1, std::min<long>(warp_ctas, (n_items + AW_WARPS - 1) / AW_WARPS));
+    AttnWarpFn fn;
+    if (attn_warp_fn(p->head_dim, AW_NST, &fn) != cudaSuccess) return SPARSK_ECUDA;
+    fn<<<grid, AW_WARPS * 32, AW_WARPS * attn_warp_bytes(p->head_dim, AW_NST), st>>>(a);
     if (p->head_dim == 128) attn_merge_kernel<128><<<dim3(p->n_rows, p->n_q_heads), 128, 0, st>>>(a, counts + 1);
     else attn_merge_kernel<64><<<dim3(p->n_rows, p->n_q_heads), 64, 0, st>>>(a, counts + 1);
     return cudaGetLastError() == cudaSuccess ? SPARSK_OK : SPARSK_ECUDA;

@@ -226,6 +226,83 @@ static __global__ void put_current_kernel(StepDesc sd, const float *__restrict__
     for (int i = threadIdx.x; i < d / 4; i += blockDim.x) d4[i] = s4[i];
 }
 
+// ---------------------------------------------------------------------------------------
+// Confidence-based exit (Sec. V-B, compared method 3): after a layer's head has left the logits
+// of the candidate rows in `logits` ([seq][V]), one block per row computes the entropy (natural
+// logarithm) of softmax over the row's modality range [lo, hi): with m = max z, S = sum e^(z-m),
+// T = sum (z-m) e^(z-m):  H = ln S - T / S.  Two passes over a row that sits in the L2.
+// ---------------------------------------------------------------------------------------
+static __global__ void __launch_bounds__(1024) entropy_kernel(const float *__restrict__ logits, const int *__restrict__ rows,
+                                                       const int *__restrict__ row_mod, int n, int V, int Vt,
+                                                       float *__restrict__ ent_out)
+{
+    __shared__ float red[32], red2[32];
+    griddep_wait();
+    const int i = blockIdx.x;
+    if (i >= n) return;
+    const int b = rows[i];
+    const int lo = row_mod[i] ? Vt : 0, hi = row_mod[i] ? V : Vt;
+    const float *z = logits + (size_t)b * V;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float mx = -INFINITY;
+    for (int k = lo + threadIdx.x; k < hi; k += blockDim.x) mx = fmaxf(mx, z[k]);
+    mx = warp_max(mx);
+    if (lane == 0) red[warp] = mx;
+    __syncthreads();
+    mx = red[0];
+    for (int w = 1; w < (int)(blockDim.x >> 5); w++) mx = fmaxf(mx, red[w]);
+    __syncthreads();
+    float S = 0.f, T = 0.f;
+    for (int k = lo + threadIdx.x; k < hi; k += blockDim.x) {
+        const float x = z[k] - mx, e = __expf(x);
+        S += e;
+        T += x * e;
+    }
+    S = warp_sum(S);
+    T = warp_sum(T);
+    if (lane == 0) {
+        red[warp] = S;
+        red2[warp] = T;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float s = 0.f, t = 0.f;
+        for (int w = 0; w < (int)(blockDim.x >> 5); w++) {
+            s += red[w];
+            t += red2[w];
+        }
+        ent_out[i] = hi > lo ? logf(s) - t / s : 0.f;
+    }
+}
+
+// Rows between the residual-stream buffers of a pass and their homes.  Row i of `buf` belongs to
+// sequence index seq[i] of the step; src[i] >= 0: pending position src[i] of that sequence's
+// slot (pending store), src[i] < 0: the sequence's current position (row seq[i] of h_lo).
+// to_buf = 1 gathers, 0 scatters back.
+static __global__ void rows_move_kernel(float *__restrict__ buf, float *__restrict__ h_lo, float *__restrict__ pend_h,
+                                 const int *__restrict__ row_slot, const int *__restrict__ row_seq,
+                                 const int *__restrict__ row_src, int n, int d, int max_pending, int to_buf)
+{
+    griddep_wait();
+    const int i = blockIdx.x;
+    if (i >= n) return;
+    const int src = row_src[i];
+    float *home = src >= 0 ? pend_h + ((size_t)row_slot[i] * max_pending + src) * d : h_lo + (size_t)row_seq[i] * d;
+    float4 *a = reinterpret_cast<float4 *>(buf + (size_t)i * d), *b = reinterpret_cast<float4 *>(home);
+    for (int k = threadIdx.x; k < d / 4; k += blockDim.x) {
+        if (to_buf) a[k] = b[k];
+        else b[k] = a[k];
+    }
+}
+
+// Clears the arg-max cells of the listed sequences (a head is about to be consulted again).
+static __global__ void clear_keys_kernel(unsigned long long *__restrict__ keys, const int *__restrict__ rows, int n)
+{
+    griddep_wait();
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) keys[rows[i]] = 0ull;
+}
+
 // End of step: emit tokens and depths, advance lengths, grow or clear the pending sets.
 static __global__ void finish_kernel(StepDesc sd, int n, int *__restrict__ kv_len, int *__restrict__ pend_cnt,
                               int *__restrict__ next_tokens, int *__restrict__ exit_depths, int L)

@@ -56,6 +56,8 @@ WORKLOADS = {
                           exit_layer=2, refresh_period=4, refresh_phase=0, random_phase=False),
     "prof_step4_b64": dict(shape="step4", batch=64, prompt=(256, 512), steps=64, n_text=1, n_speech=4,
                            exit_layer=2, refresh_period=4, refresh_phase=0, random_phase=True),
+    "prof_step4_b64_ragged": dict(shape="step4", batch=64, prompt=(256, 2048), steps=64, n_text=1, n_speech=4,
+                                  exit_layer=2, refresh_period=4, refresh_phase=0, random_phase=True),
     "prof_glm4_b128": dict(shape="glm4", batch=128, prompt=(8192, 8192), steps=64, n_text=13,
                            n_speech=26, exit_layer=3, refresh_period=4, refresh_phase=0,
                            random_phase=True),
