@@ -64,6 +64,26 @@ def step_bytes(d, depths, mods, lens, pend):
     return total
 
 
+def step_bytes_dyn(d, depths, mods, lens):
+    """The same model for steps whose depths the library decided (confidence-based exit, Sec. V-B):
+    layer l's weights once if any sequence ran it, each sequence's KV prefix for the layers it ran,
+    and the head slice of every layer consulted: from conf_start up to the layer a confidence step
+    left at (the projections that are wasted when the step goes on, Sec. V-C), or the head it
+    was read from for a scheduled step."""
+    L = d["n_layers"]
+    kvb = 2 * d["n_kv_heads"] * d["head_dim"] * 2
+    total = layer_weight_bytes(d) * max(depths)
+    heads = set()
+    for dep, m, ln in zip(depths, mods, lens):
+        total += dep * ((ln + 1) * kvb + kvb)
+        if (d.get("conf_modalities", 0) >> (1 if m else 0)) & 1:
+            heads |= {(l, m) for l in range(d["conf_start"], min(dep, L - 1) + 1)}
+        heads.add((dep, m))
+    for _, m in heads:
+        total += (d["vocab_speech"] if m else d["vocab_text"]) * d["d_model"] * 2 + d["d_model"] * 2
+    return total + len(depths) * d["d_model"] * 2
+
+
 # --------------------------------------------------------------------------- clocks
 class ClockSampler:
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -149,8 +169,11 @@ class Runner:
         self.B = B
         K = dims["refresh_period"]
         max_len = max(len(p) for p in prompts) + total_steps + 8
-        self.ctx = binding.Sparsk(dims, gw, B, max_len, max(K - 1, 1) if dims["exit_layer"] < dims["n_layers"] else 1,
-                                  prefill_rows=64)
+        max_pending = max(K - 1, 1) if dims["exit_layer"] < dims["n_layers"] else 1
+        if dims.get("conf_modalities", 0):
+            max_pending = max(max_pending, wl["n_speech"] + 1)   # a whole chunk may leave early
+        self.last_depths = None
+        self.ctx = binding.Sparsk(dims, gw, B, max_len, max_pending, prefill_rows=64)
         for k, v in (options or {}).items():
             self.ctx.set_option(k, v)
         # nucleus sampling (Sec. V-A decodes the 28-layer backbone with it): a table of uniform
@@ -200,6 +223,15 @@ class Runner:
             if (m == 0 and te == 0) or (m == 1 and te == 2):
                 return L
             return L if c % K == r else e
+        if d.get("conf_modalities", 0):
+            # the library decided the depths: read them back (the step has synchronised already)
+            depths = [int(x) for x in (self.last_depths if self.last_depths is not None else self.dep.cpu().numpy())]
+            self.bytes += step_bytes_dyn(d, depths, mods, self.lens)
+            self.mega_seen = self.ctx.route_counts()["mega"]
+            for i, dep in enumerate(depths):
+                self.lens[i] += 1
+                self.depth_log.append((int(mods[i]), dep))
+            return
         depths = [depth(m, c) for m, c in zip(mods, ctrs)]
         self.bytes += step_bytes(d, depths, mods, self.lens, self.pend)
         kvb = 2 * d["n_kv_heads"] * d["head_dim"] * 2
@@ -232,12 +264,14 @@ class Runner:
             for mods, ctrs in sched:
                 self._next_uniforms()
                 self.ctx.decode_step_host(self.slots, self.host_tok, mods, ctrs, nt, dp)
+                self.last_depths = dp
                 self.host_tok[:] = nt
                 self._account(mods, ctrs)
         else:
             for mods, ctrs in sched:
                 self._next_uniforms()
                 self.ctx.decode_step(self.slots, self.tok[0], mods, ctrs, self.tok[1], self.dep)
+                self.last_depths = None
                 self.tok.reverse()
                 self._account(mods, ctrs)
         self.g += n_cycles * cyc
@@ -388,6 +422,9 @@ def main():
     ap.add_argument("--time-kernel", default="mega", choices=sorted(KC))
     ap.add_argument("--sampling", default=None, metavar="T,P",
                     help="nucleus sampling with temperature T and top_p P (the paper's 0.7,0.9) instead of the arg max")
+    ap.add_argument("--conf", default=None, metavar="START,THRESHOLD",
+                    help="decode speech steps with confidence-based exit (Sec. V-B) from layer START with the given "
+                         "entropy threshold (the paper: 26,0.1 for the 28-layer backbone, 36,0.5 for the 40-layer one)")
     ap.add_argument("--exit-layer", type=int, default=None, help="override the workload's exit layer e (sweep cells)")
     ap.add_argument("--period", type=int, default=None, help="override the workload's refresh period K (sweep cells)")
     args = ap.parse_args()
@@ -397,6 +434,11 @@ def main():
     wl, dims, prompts, phi, off = workload_setup(args.workload, rank, args.exit_layer, args.period)
     cyc = wl["n_text"] + wl["n_speech"]
     L = dims["n_layers"]
+    head_layers = [wl["exit_layer"], L]
+    if args.conf:
+        c_start, c_thr = args.conf.split(",")
+        dims.update(conf_modalities=2, conf_start=int(c_start), conf_threshold=float(c_thr))
+        head_layers += list(range(int(c_start), L))
     cfg = {"workload": args.workload, "shape": wl["shape"], "batch_per_gpu": wl["batch"],
            "prompt_len": list(wl["prompt"]), "interleave": f'{wl["n_text"]}:{wl["n_speech"]}',
            "exit_layer": wl["exit_layer"], "refresh_period": wl["refresh_period"],
@@ -443,7 +485,7 @@ def main():
         torch.cuda.synchronize()
 
     t_setup = time.time()
-    w = synth.make_weights(dims, seed=0, head_layers=[wl["exit_layer"], L])
+    w = synth.make_weights(dims, seed=0, head_layers=head_layers)
     gw = binding.upload_weights(w)
     opts = {}
     for o in args.option:
@@ -451,6 +493,8 @@ def main():
         opts[k] = int(v)
     sampling = tuple(float(x) for x in args.sampling.split(",")) if args.sampling else None
     cfg["decoding"] = f"nucleus T={sampling[0]} top_p={sampling[1]}" if sampling else "greedy (restricted arg max)"
+    if args.conf:
+        cfg["speech_exit"] = f"confidence-based from layer {dims['conf_start']}, entropy threshold {dims['conf_threshold']}"
     synthetic_kv = max(wl["prompt"]) > 4096      # long prompts: cache contents are stand-ins
     extra = (W + args.steps) * 2 + 8
     total_steps = extra * cyc

@@ -310,6 +310,13 @@ int sparsk_phase_trace(sparsk_ctx *ctx, int64_t *out_ns /*host*/, int32_t capaci
  * in the paper: measurement only. */
 int64_t sparsk_launch_count(const sparsk_ctx *ctx);
 
+/* Confidence-based exit (Sec. V-B): the entropies the last decode step saw.  out[i * L + l] is
+ * the entropy of head g_l's prediction for the i-th sequence of that step (l in [conf_start, L)),
+ * or -1 where the head was not consulted (the sequence had left, or follows the schedule).  Host
+ * array of n_seqs * L floats; n_seqs at most the last step's.  Parity hook: a checker can judge
+ * the depths the step chose against entropies of its own. */
+int sparsk_conf_entropies(const sparsk_ctx *ctx, int32_t n_seqs, float *out /*host*/);
+
 /* Which implementation the layer passes so far went through (a pass = one layer over one row
  * set): layer_passes[0] persistent layer-range kernel (1-2 rows), [1] tcgen05 kernels launched
  * per projection, [2] small-batch GEMV kernels.  Lets a benchmark

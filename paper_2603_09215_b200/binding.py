@@ -19,7 +19,7 @@ EXPORTS = ("sparsk_workspace_bytes", "sparsk_create", "sparsk_prefill", "sparsk_
            "sparsk_decode_step_host", "sparsk_reset_slot", "sparsk_import_kv", "sparsk_export_kv",
            "sparsk_set_len", "sparsk_slot_state", "sparsk_set_debug", "sparsk_set_option",
            "sparsk_kernel_time", "sparsk_kernel_time_by_class", "sparsk_check", "sparsk_phase_trace", "sparsk_attention", "sparsk_attention_scratch_bytes", "sparsk_attention_static", "sparsk_sampling_scratch_bytes", "sparsk_set_sampling", "sparsk_nucleus_sample",
-           "sparsk_launch_count", "sparsk_route_counts", "sparsk_last_error", "sparsk_destroy")
+           "sparsk_launch_count", "sparsk_route_counts", "sparsk_conf_entropies", "sparsk_last_error", "sparsk_destroy")
 
 OK, EINVAL, ECAPACITY, ENOHEAD, ECUDA, ESTATE, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
 
@@ -115,6 +115,8 @@ def load():
     L.sparsk_check.argtypes = [vp]
     L.sparsk_launch_count.restype = C.c_int64
     L.sparsk_launch_count.argtypes = [vp]
+    L.sparsk_conf_entropies.restype = C.c_int
+    L.sparsk_conf_entropies.argtypes = [vp, C.c_int32, C.POINTER(C.c_float)]
     L.sparsk_route_counts.restype = C.c_int
     L.sparsk_route_counts.argtypes = [vp, C.POINTER(C.c_int64)]
     L.sparsk_last_error.restype = C.c_char_p
@@ -365,6 +367,13 @@ class Sparsk:
 
     def launch_count(self) -> int:
         return self.lib.sparsk_launch_count(self.h)
+
+    def conf_entropies(self, n_seqs: int) -> np.ndarray:
+        """[n_seqs, L] entropies the last decode step saw per layer (column l, -1 where no head was consulted)."""
+        L = self.cd.n_layers
+        out = np.empty((n_seqs, L), np.float32)
+        self._check(self.lib.sparsk_conf_entropies(self.h, n_seqs, out.ctypes.data_as(C.POINTER(C.c_float))))
+        return out
 
     def route_counts(self) -> dict:
         """Layer passes so far by implementation."""

@@ -113,6 +113,7 @@ struct sparsk_ctx {
     int *conf_rows_dev;            // device: [slot R][pos R][src R][seq R][grp_row0 B][grp_nrows B][n_groups][n_rows]
     int *conf_list_dev;            // device: [rows B][modality B]
     float *conf_ent_dev, *conf_ent_host;  // entropies of a layer's candidates (device, pinned host)
+    std::vector<float> conf_trace; // last step: entropy seen at layer l (1-based, < L) by sequence i at [i * L + l], or -1
     float *conf_logits;            // device [B][V] when neither the parity hook nor a sampler lends a buffer
     int inject_timeout;            // test hook: the next persistent launch waits for a barrier count nobody reaches
     int64_t route_layers[3];       // layer passes so far by implementation: see sparsk_route_counts
@@ -1141,6 +1142,14 @@ extern "C" int sparsk_destroy(sparsk_ctx *ctx)
 
 extern "C" const char *sparsk_last_error(const sparsk_ctx *ctx) { return good(ctx) ? ctx->err : "invalid context"; }
 extern "C" int64_t sparsk_launch_count(const sparsk_ctx *ctx) { return good(ctx) ? ctx->launches : -1; }
+extern "C" int sparsk_conf_entropies(const sparsk_ctx *ctx, int32_t n_seqs, float *out)
+{
+    if (!good(ctx)) return SPARSK_ESTATE;
+    const int L = ctx->dm.n_layers;
+    if (!out || n_seqs < 0 || (size_t)n_seqs * L > ctx->conf_trace.size()) return SPARSK_EINVAL;
+    for (size_t k = 0; k < (size_t)n_seqs * L; k++) out[k] = ctx->conf_trace[k];
+    return SPARSK_OK;
+}
 extern "C" int sparsk_route_counts(const sparsk_ctx *ctx, int64_t *layer_passes)
 {
     if (!good(ctx)) return SPARSK_ESTATE;
@@ -1486,6 +1495,7 @@ static int decode_step_conf(sparsk_ctx *ctx, int32_t n, const int32_t *slots, co
 
     std::vector<int> active(n);
     for (int i = 0; i < n; i++) active[i] = i;
+    ctx->conf_trace.assign((size_t)n * L, -1.f);
     int l = 1;
     while (!active.empty()) {
         // ---- where this segment ends
@@ -1574,8 +1584,10 @@ static int decode_step_conf(sparsk_ctx *ctx, int32_t n, const int32_t *slots, co
                       d.vocab_text, ctx->conf_ent_dev));
             CU(cudaMemcpyAsync(ctx->conf_ent_host, ctx->conf_ent_dev, sizeof(float) * asking.size(), cudaMemcpyDeviceToHost, ctx->stream));
             CU(cudaStreamSynchronize(ctx->stream));
-            for (size_t k = 0; k < asking.size(); k++)
+            for (size_t k = 0; k < asking.size(); k++) {
+                ctx->conf_trace[(size_t)asking[k] * L + seg_end] = ctx->conf_ent_host[k];
                 if (ctx->conf_ent_host[k] < d.conf_threshold) leaving.push_back(asking[k]);
+            }
         }
         for (int i : leaving) {
             const int rc = leave(i, seg_end);

@@ -37,7 +37,7 @@ class Model:
 @pytest.fixture(scope="module")
 def step_model():
     _need_gpu()
-    m = Model("step", [20, 28])
+    m = Model("step", [20, 26, 27, 28])
     yield m
     del m.gw
     torch.cuda.empty_cache()
@@ -190,3 +190,59 @@ def test_config5_sweep_depths(glm_model, e, K):
     interleave cycle are exactly the schedule's (checked inside the driver for every step)."""
     st = _run(glm_model, "cfg5_glm_b128", steps=39, g0=0, n_checked=0, lens=[64] * 128, exit_layer=e, period=K)
     assert st["steps"] == 39
+
+
+def test_confidence_exit_step_shape(step_model):
+    """Confidence-based exit (Sec. V-B) at the Step shape with the paper's start layer for that
+    backbone (row S3: layer 26) on speech steps, from a stand-in cache of 511 positions.  With the
+    paper's threshold 0.1 random heads are never confident (their entropy is near ln 6561): every
+    speech step pays for the heads of layers 26 and 27 and runs all 28 layers, the wasted
+    projection of Sec. V-C.  With an infinite threshold every speech step leaves at layer 26 and
+    the next text step carries the pending positions through layers 27 and 28."""
+    from oracle import oracle as ora
+    from tests import parity_util as pu
+    from paper_2603_09215_b200 import binding
+    for thr, want_speech in ((0.1, 28), (float("inf"), 26)):
+        dims = synth.model_dims("step", 20, 4, 0, conf_modalities=2, conf_start=26, conf_threshold=thr)
+        g = binding.Sparsk(dims, step_model.gw, 1, 511 + 16, 8)
+        om = ora.OracleModel(dims, step_model.w, max_len=511 + 16)
+        sq = om.new_seq(8)
+        k, v = synth.synth_kv(dims, 511, seed=1000)
+        from oracle.bruteforce import bf16_to_f64
+        dev = lambda a: torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16).to(torch.float16)
+        for layer in range(1, 29):
+            g.import_kv(0, layer, 0, dev(k[layer - 1]), dev(v[layer - 1]))
+            kf, vf = bf16_to_f64(k[layer - 1]), bf16_to_f64(v[layer - 1])
+            for p in range(511):
+                sq.set_kv(layer, p, kf[p], vf[p])
+        g.set_len(0, 511)
+        sq.set_len(511)
+        V, Vt = dims["vocab_text"] + dims["vocab_speech"], dims["vocab_text"]
+        dbg_h = torch.zeros((1, dims["d_model"]), dtype=torch.float32, device="cuda")
+        dbg_z = torch.zeros((1, V), dtype=torch.float32, device="cuda")
+        g.set_debug(dbg_h, dbg_z)
+        tok = torch.tensor([1234], dtype=torch.int32, device="cuda")
+        ot, od = torch.zeros(1, dtype=torch.int32, device="cuda"), torch.zeros(1, dtype=torch.int32, device="cuda")
+        nxt = 1234
+        for step in range(7):
+            m, c = synth.interleave(step, 1, 4)
+            tok[0] = nxt
+            g.decode_step([0], tok, [m], [c], ot, od)
+            g.check()
+            dep = int(od.cpu()[0])
+            assert dep == (28 if m == 0 else want_speech), (step, m, dep)
+            r = sq.decode_step_dyn(nxt, m, c, forced_depth=dep)
+            ent = g.conf_entropies(1)[0]
+            for l in (26, 27):
+                if m == 1 and l <= dep and l < 28:
+                    assert abs(float(ent[l]) - r["entropies"][l - 1]) <= 1e-3, (l, ent[l], r["entropies"][l - 1])
+                    assert (float(ent[l]) < thr) == (l == dep)
+            lo, hi = (0, Vt) if m == 0 else (Vt, V)
+            H, Z = dbg_h.cpu().numpy().astype(np.float64)[0], dbg_z.cpu().numpy().astype(np.float64)[0]
+            assert pu.rel_err(H, r["hidden"]) <= pu.REL_TOL
+            assert pu.rel_err(Z[lo:hi], r["logits"][lo:hi]) <= pu.REL_TOL
+            if r["margin"] > pu.MARGIN:
+                assert int(ot.cpu()[0]) == r["token"]
+            nxt = r["token"]
+            assert g.slot_state(0) == (sq.len, len(sq.pending))
+        g.close()
