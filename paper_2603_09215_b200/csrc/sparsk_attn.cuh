@@ -346,8 +346,10 @@ __device__ __forceinline__ void attn_item(const AttnArgs &a, int qb, int hk, int
     }
 }
 
-// Persistent grid of warps; item i = ((g * n_qblk + qb) * Hkv + hk) * n_splits + sp goes to warp
-// i mod (number of warps), warps numbered so that consecutive items land on different SMs.
+// Persistent grid of warps; item i = ((g * Hkv + hk) * n_splits + sp) * n_qblk + qb goes to warp
+// i mod (number of warps), warps numbered so that consecutive items land on different SMs: the
+// query blocks of one (group, kv head, split) run side by side, and all but the first find
+// their K/V tiles in the L2.
 template <int HD, int NST>
 __global__ void __launch_bounds__(AW_WARPS * 32) attn_warp_kernel(AttnArgs a)
 {
@@ -362,9 +364,9 @@ __global__ void __launch_bounds__(AW_WARPS * 32) attn_warp_kernel(AttnArgs a)
     const long n_workers = (long)gridDim.x * AW_WARPS;
     for (long item = (long)warp * gridDim.x + blockIdx.x; item < n_items; item += n_workers) {
         long t = item;
+        const int qb = (int)(t % a.n_qblk); t /= a.n_qblk;
         const int sp = (int)(t % a.n_splits); t /= a.n_splits;
-        const int hk = (int)(t % a.Hkv); t /= a.Hkv;
-        const int qb = (int)(t % a.n_qblk), g = (int)(t / a.n_qblk);
+        const int hk = (int)(t % a.Hkv), g = (int)(t / a.Hkv);
         const int row0 = a.grp_row0[g], nrows = a.grp_nrows[g];
         if (row0 < 0 || nrows < 1 || row0 + nrows > a.n_rows) continue;
         const int nq = nrows * G;
