@@ -160,7 +160,8 @@ def cycle_schedule(wl, phi, off, g0, n):
 class Runner:
     """Drives one library context through decode steps with tokens kept on the device."""
 
-    def __init__(self, dims, gw, wl, prompts, phi, off, total_steps, options=None, synthetic_kv=False, sampling=None):
+    def __init__(self, dims, gw, wl, prompts, phi, off, total_steps, options=None, synthetic_kv=False, sampling=None,
+                 prefill_rows=64):
         import torch
         from paper_2603_09215_b200 import binding
         self.torch = torch
@@ -173,7 +174,7 @@ class Runner:
         if dims.get("conf_modalities", 0):
             max_pending = max(max_pending, wl["n_speech"] + 1)   # a whole chunk may leave early
         self.last_depths = None
-        self.ctx = binding.Sparsk(dims, gw, B, max_len, max_pending, prefill_rows=64)
+        self.ctx = binding.Sparsk(dims, gw, B, max_len, max_pending, prefill_rows=prefill_rows)
         for k, v in (options or {}).items():
             self.ctx.set_option(k, v)
         # nucleus sampling (Sec. V-A decodes the 28-layer backbone with it): a table of uniform
@@ -425,6 +426,7 @@ def main():
     ap.add_argument("--conf", default=None, metavar="START,THRESHOLD",
                     help="decode speech steps with confidence-based exit (Sec. V-B) from layer START with the given "
                          "entropy threshold (the paper: 26,0.1 for the 28-layer backbone, 36,0.5 for the 40-layer one)")
+    ap.add_argument("--prefill-rows", type=int, default=64, help="rows per prefill pass (a prompt chunk)")
     ap.add_argument("--exit-layer", type=int, default=None, help="override the workload's exit layer e (sweep cells)")
     ap.add_argument("--period", type=int, default=None, help="override the workload's refresh period K (sweep cells)")
     args = ap.parse_args()
@@ -498,7 +500,7 @@ def main():
     synthetic_kv = max(wl["prompt"]) > 4096      # long prompts: cache contents are stand-ins
     extra = (W + args.steps) * 2 + 8
     total_steps = extra * cyc
-    run = Runner(dims, gw, wl, prompts, phi, off, total_steps, opts, synthetic_kv, sampling)
+    run = Runner(dims, gw, wl, prompts, phi, off, total_steps, opts, synthetic_kv, sampling, args.prefill_rows)
     cfg["cache_fill"] = "stand-in values (imported)" if synthetic_kv else "real prefill of random prompts"
     setup_s = time.time() - t_setup
 
