@@ -4,7 +4,19 @@
 namespace sparsk {
 
 // ------------------------------------------------------------------ activations -> shared memory
-// Columns [c0, c0 + ncols) of the M activation rows, as fp32, row m at act + m * ncols.  With h:
+// Where column i (a multiple of 4) of a row sits inside the activation area.  A lane of a
+// consumer warp needs the eight columns 8 lane .. 8 lane + 7 of a 256-column step (the columns of
+// its 16-byte weight unit); read as two float4 at a 32-byte stride they would collide two ways on
+// the banks, so each 256-column step is stored as two planes of 128 floats: columns 8 l + 0..3 at
+// [4 l], columns 8 l + 4..7 at [128 + 4 l], and the two reads of a warp are both conflict-free.
+__device__ __forceinline__ int mk_act_slot(int i)
+{
+    const int ci = i & (MK_BOX_COLS - 1);
+    return (i - ci) + ((ci >> 2) & 1) * (MK_BOX_COLS / 2) + (ci >> 3) * 4;
+}
+
+// Columns [c0, c0 + ncols) of the M activation rows, as fp32, row m at act + m * ncols (in the
+// layout of mk_act_slot).  With h:
 // x = h / sqrt(mean(h^2) + eps) * gain; otherwise a copy of the fp32 rows x.  Columns at or
 // beyond K are zeros (the last weight box is zero-filled there too).  ncols is a multiple of 256.
 template <int M>
@@ -41,12 +53,12 @@ __device__ __forceinline__ void mk_load_act(float *act, int c0, int ncols, int K
                     o = make_float4(p.x * inv * bf_lo(g2.x), p.y * inv * bf_hi(g2.x), p.z * inv * bf_lo(g2.y),
                                     p.w * inv * bf_hi(g2.y));
                 }
-                *reinterpret_cast<float4 *>(dst + i) = o;
+                *reinterpret_cast<float4 *>(dst + mk_act_slot(i)) = o;
             }
         } else {
             const float *src = x + (size_t)m * K;
             for (int i = tid * 4; i < ncols; i += T * 4)
-                *reinterpret_cast<float4 *>(dst + i) =
+                *reinterpret_cast<float4 *>(dst + mk_act_slot(i)) =
                     c0 + i < K ? *reinterpret_cast<const float4 *>(src + c0 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
     }
@@ -96,8 +108,8 @@ __device__ __forceinline__ bool mk_project(int type, const MkArgs &a, const MkLa
             unpack8(*reinterpret_cast<const uint4 *>(slot + MK_BOX_BYTES), w1);
 #pragma unroll
             for (int m = 0; m < M; m++) {
-                const float *xp = act + (size_t)m * ncols + (ks - win0) * MK_BOX_COLS + lane * 8;
-                const float4 xa = *reinterpret_cast<const float4 *>(xp), xb = *reinterpret_cast<const float4 *>(xp + 4);
+                const float *xp = act + (size_t)m * ncols + (ks - win0) * MK_BOX_COLS + lane * 4;
+                const float4 xa = *reinterpret_cast<const float4 *>(xp), xb = *reinterpret_cast<const float4 *>(xp + MK_BOX_COLS / 2);
                 const float xv[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
 #pragma unroll
                 for (int j = 0; j < 8; j++) {
