@@ -186,10 +186,11 @@ int sparsk_set_debug(sparsk_ctx *ctx, float *exit_hidden /*device or NULL*/,
                      float *exit_logits /*device or NULL*/);
 
 /* Tuning knobs, by name (no counterpart in the paper: implementation choices): "gemm_min_rows" (row count from which the tcgen05 path is used; a
- * large value keeps everything on the GEMV path), "mega" (0/1: run passes of one
- * or two rows as one persistent kernel per layer range; default 1), "mega_max_rows" (1..4: the
- * largest pass that kernel takes; default 2, above which its CUDA-core inner loop falls behind
- * HBM), "gemm_kb" (1: one 64-element block of the inner
+ * large value keeps everything on the GEMV path), "mega" (0/1: run passes of up to
+ * four rows as one persistent kernel per layer range; default 1), "mega_max_rows" (1..4: the
+ * largest pass that kernel takes; default 4. Passes of three and four rows use its tensor-core
+ * inner loop, which needs d_model, d_ffn and n_heads * head_dim to be multiples of 64; other
+ * shapes stop at two rows), "gemm_kb" (1: one 64-element block of the inner
  * dimension per TMA copy instead of two; 0 = automatic), "attn_split" (positions
  * per KV split), "pdl" (0/1, programmatic dependent launch between the kernels of a step; default 1),
  * "gemv_ks" / "gemv_r" (override the GEMV team width / rows per group; 0 = automatic),

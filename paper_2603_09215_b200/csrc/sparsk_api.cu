@@ -106,6 +106,7 @@ struct sparsk_ctx {
     int mk_trace_n;                // entries the last launch wrote
     unsigned long long mk_bar_base;
     int mega, mk_ok, mk_coop, mk_max_rows;
+    bool mk_tc_ok;                 // the shape allows the persistent kernel's tensor-core form (3-4 rows)
     // confidence-based exit (dims.conf_modalities != 0): the host drives the step layer by layer
     std::vector<std::vector<int>> h_fill;  // per slot: layer each pending position has been carried to
     int *conf_host;                // pinned arena for the row sets of a step's segments
@@ -801,15 +802,30 @@ bool build_mega(sparsk_ctx *c)
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
     };
+    // the swizzled three-dimensional view needs inner dimensions that are whole 64-element blocks
+    c->mk_tc_ok = d.d_model % 64 == 0 && d.d_ffn % 64 == 0 && qd % 64 == 0;
+    auto enc_sw = [&](CUtensorMap *m, const void *base, size_t rows, size_t cols) {
+        const cuuint64_t dims[3] = {64, (cuuint64_t)rows, (cuuint64_t)(cols / 64)};
+        const cuuint64_t strides[2] = {(cuuint64_t)cols * 2, 128};
+        const cuuint32_t box[3] = {64, (cuuint32_t)MK_BOX_ROWS, (cuuint32_t)(MK_BOX_COLS / 64)};
+        const cuuint32_t es[3] = {1, 1, 1};
+        return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, es,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    };
     c->mk_host.resize(d.n_layers);
     bool ok = true;
     for (int l = 0; l < d.n_layers; l++) {
         MkLayer &m = c->mk_host[l];
         memset(&m, 0, sizeof m);
-        ok = ok && enc(&m.map_q, c->wq[l], qd, d.d_model) && enc(&m.map_k, c->wk[l], kd, d.d_model) &&
-             enc(&m.map_v, c->wv[l], kd, d.d_model) && enc(&m.map_o, c->wo[l], d.d_model, qd) &&
-             enc(&m.map_g, c->w_gate[l], d.d_ffn, d.d_model) && enc(&m.map_u, c->w_up[l], d.d_ffn, d.d_model) &&
-             enc(&m.map_d, c->w_down[l], d.d_model, d.d_ffn);
+        const void *mats[MKW_N] = {c->wq[l], c->wk[l], c->wv[l], c->wo[l], c->w_gate[l], c->w_up[l], c->w_down[l]};
+        const size_t rows[MKW_N] = {qd, kd, kd, (size_t)d.d_model, (size_t)d.d_ffn, (size_t)d.d_ffn, (size_t)d.d_model};
+        const size_t cols[MKW_N] = {(size_t)d.d_model, (size_t)d.d_model, (size_t)d.d_model, qd, (size_t)d.d_model,
+                                    (size_t)d.d_model, (size_t)d.d_ffn};
+        for (int k = 0; k < MKW_N; k++) {
+            ok = ok && enc(&m.map[k], mats[k], rows[k], cols[k]);
+            if (c->mk_tc_ok) ok = ok && enc_sw(&m.map[MKW_N + k], mats[k], rows[k], cols[k]);
+        }
         m.attn_gain = c->attn_norm[l];
         m.mlp_gain = c->mlp_norm[l];
         m.kc = c->kcache + l * lstride;
@@ -829,12 +845,12 @@ bool build_mega(sparsk_ctx *c)
     return true;
 }
 
-size_t mega_smem(const sparsk_dims &) { return (size_t)MK_SLOTS * MK_SLOT_BYTES + MK_AREA_BYTES; }
+size_t mega_smem(const sparsk_dims &) { return (size_t)MK_SLOTS * MK_SLOT_BYTES + MK_AREA_BYTES + 1024; }
 
 // Can a pass of n_rows rows go through the persistent kernel?
 bool use_mega(const sparsk_ctx *c, int n_rows)
 {
-    return c->mega && c->mk_ok && c->mk_coop && n_rows >= 1 && n_rows <= c->mk_max_rows &&
+    return c->mega && c->mk_ok && c->mk_coop && n_rows >= 1 && n_rows <= c->mk_max_rows && (n_rows <= 2 || c->mk_tc_ok) &&
            mk_attn_bytes(c->dm.head_dim) <= MK_AREA_BYTES && c->dm.head_dim % (2 * MK_BOX_ROWS) == 0;
 }
 
@@ -1040,7 +1056,7 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
     ctx->tc_kb = 0;
     ctx->gemm_smem_kb = 220;
     ctx->gemm_cps = 1;
-    ctx->mk_max_rows = 2;
+    ctx->mk_max_rows = MK_MAX_ROWS;
     ctx->attn_tc = 1; ctx->attn_tc_min_q = 33; ctx->attn_stages = AW_NST;
     ctx->inject_timeout = 0;
     ctx->trim_last = 1;

@@ -58,11 +58,15 @@ inline size_t mk_attn_bytes(int head_dim)
 // k-steps of M fp32 activation rows that fit the area
 __host__ __device__ inline int mk_act_window(int M) { return MK_AREA_BYTES / (M * MK_BOX_COLS * 4); }
 
+enum { MKW_Q = 0, MKW_K, MKW_V, MKW_O, MKW_G, MKW_U, MKW_D, MKW_N };
 enum { MK_QKV = 0, MK_ATTN = 1, MK_MERGE = 2, MK_OPROJ = 3, MK_GATEUP = 4, MK_DOWN = 5 };
 
 // One layer's worth of what the phases need (device array, one entry per layer).
 struct MkLayer {
-    CUtensorMap map_q, map_k, map_v, map_o, map_g, map_u, map_d;  // [256 x 16] boxes, no swizzle
+    // per matrix (MKW_*): [16 rows x 256 columns] boxes without swizzle (passes of one or two rows),
+    // then, MKW_N entries on, the same boxes as four 64-column blocks with the 128-byte swizzle
+    // (view [64][rows][K/64], box {64, 16, 4}; passes of three and four rows read them with ldmatrix)
+    CUtensorMap map[14];
     const bf16 *attn_gain, *mlp_gain;
     kv_t *kc, *vc;  // this layer's cache [slot][Hkv][S][hd]
 };
@@ -145,23 +149,23 @@ __device__ __forceinline__ void mk_band(int type, const MkArgs &a, const MkLayer
         if (b < nq + nk) {
             const bool isq = b < nq;
             const int bb = isq ? b : b - nq;
-            map[0] = map[1] = isq ? &L->map_q : &L->map_k;
+            map[0] = map[1] = &L->map[isq ? MKW_Q : MKW_K];
             row[0] = (bb / per_head) * a.hd + (bb % per_head) * MK_BOX_ROWS;
             row[1] = row[0] + half;
         } else {
-            map[0] = map[1] = &L->map_v;
+            map[0] = map[1] = &L->map[MKW_V];
             row[0] = (b - nq - nk) * 2 * MK_BOX_ROWS;
             row[1] = row[0] + MK_BOX_ROWS;
         }
         break;
     }
     case MK_GATEUP:
-        map[0] = &L->map_g;
-        map[1] = &L->map_u;
+        map[0] = &L->map[MKW_G];
+        map[1] = &L->map[MKW_U];
         row[0] = row[1] = b * MK_BOX_ROWS;
         break;
     default:
-        map[0] = map[1] = type == MK_OPROJ ? &L->map_o : &L->map_d;
+        map[0] = map[1] = &L->map[type == MK_OPROJ ? MKW_O : MKW_D];
         row[0] = b * 2 * MK_BOX_ROWS;
         row[1] = row[0] + MK_BOX_ROWS;
     }
@@ -214,6 +218,7 @@ struct MkShared {
     int giving_up, never;
     int row_slot[MK_MAX_ROWS], row_pos[MK_MAX_ROWS], grp_row0[MK_MAX_ROWS], grp_nrows[MK_MAX_ROWS];  // copies of the row set
     float red[MK_CW];
+    float red_rows[MK_MAX_ROWS][MK_CW];  // per-row partial sums of squares (tensor-core form: all rows at once)
 };
 
 // Consumers only: wait until every CTA has arrived at this barrier.

@@ -60,8 +60,9 @@ __global__ void __launch_bounds__(MK_THREADS, 1) mega_kernel(const MkArgs a)
 {
     extern __shared__ __align__(1024) unsigned char mk_smem[];
     __shared__ MkShared sh;
-    unsigned char *ring = mk_smem;                                     // MK_SLOTS x 16 KB
-    unsigned char *area = mk_smem + (size_t)MK_SLOTS * MK_SLOT_BYTES;  // activations / attention rings
+    // the swizzled boxes of the tensor-core form need the ring on a 1024-byte boundary
+    unsigned char *ring = mk_smem + ((1024u - (smem_u32(mk_smem) & 1023u)) & 1023u);  // MK_SLOTS x 16 KB
+    unsigned char *area = ring + (size_t)MK_SLOTS * MK_SLOT_BYTES;     // activations / attention rings
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (int s = 0; s < MK_SLOTS; s++) {
@@ -100,8 +101,11 @@ __global__ void __launch_bounds__(MK_THREADS, 1) mega_kernel(const MkArgs a)
                     const CUtensorMap *map[2];
                     int row[2];
                     mk_band(ld.type, a, a.layers + ld.l, ld.band(), map, row);
-                    tma_load_2d(smem_u32(ring) + s * MK_SLOT_BYTES + lane * MK_BOX_BYTES, map[lane], &sh.full[s],
-                                ld.ks * MK_BOX_COLS, row[lane]);
+                    const uint32_t dst = smem_u32(ring) + s * MK_SLOT_BYTES + lane * MK_BOX_BYTES;
+                    if (M >= 3)  // the same box as four swizzled 64-column blocks (entries MKW_N on)
+                        tma_load_3d(dst, map[lane] + MKW_N, &sh.full[s], 0, row[lane], ld.ks * (MK_BOX_COLS / 64));
+                    else
+                        tma_load_2d(dst, map[lane], &sh.full[s], ld.ks * MK_BOX_COLS, row[lane]);
                 }
             }
             ld.advance(a);
@@ -118,13 +122,12 @@ __global__ void __launch_bounds__(MK_THREADS, 1) mega_kernel(const MkArgs a)
         uint32_t it = 0;
         unsigned long long epoch = a.bar_base;
         if (blockIdx.x == 0 && threadIdx.x == 0 && a.trace) a.trace[0] = global_ns();
-        float *act = reinterpret_cast<float *>(area);
         bool ok = true;
         const int qd = a.Hq * a.hd;
         for (int l = a.layer_begin; l < a.layer_end && ok; l++) {
             const MkLayer *L = a.layers + l;
             // q/k/v
-            if (!(ok = mk_project<M>(MK_QKV, a, L, act, a.d, a.h, nullptr, L->attn_gain, ring, &sh, it))) break;
+            if (!(ok = mk_proj<M>(MK_QKV, a, L, area, a.d, a.h, nullptr, L->attn_gain, ring, &sh, it))) break;
             if (!(ok = mk_grid_barrier(a, &sh, epoch))) break;
             // attention and the merge of its splits
             mk_attention<HD>(a, L, area, &sh);
@@ -132,12 +135,12 @@ __global__ void __launch_bounds__(MK_THREADS, 1) mega_kernel(const MkArgs a)
             mk_merge<HD>(a);
             if (!(ok = mk_grid_barrier(a, &sh, epoch))) break;
             // O-projection
-            if (!(ok = mk_project<M>(MK_OPROJ, a, L, act, qd, nullptr, a.attn_o, nullptr, ring, &sh, it))) break;
+            if (!(ok = mk_proj<M>(MK_OPROJ, a, L, area, qd, nullptr, a.attn_o, nullptr, ring, &sh, it))) break;
             if (!(ok = mk_grid_barrier(a, &sh, epoch))) break;
             // MLP
-            if (!(ok = mk_project<M>(MK_GATEUP, a, L, act, a.d, a.h, nullptr, L->mlp_gain, ring, &sh, it))) break;
+            if (!(ok = mk_proj<M>(MK_GATEUP, a, L, area, a.d, a.h, nullptr, L->mlp_gain, ring, &sh, it))) break;
             if (!(ok = mk_grid_barrier(a, &sh, epoch))) break;
-            if (!(ok = mk_project<M>(MK_DOWN, a, L, act, a.F, nullptr, a.act, nullptr, ring, &sh, it))) break;
+            if (!(ok = mk_proj<M>(MK_DOWN, a, L, area, a.F, nullptr, a.act, nullptr, ring, &sh, it))) break;
             if (!(ok = mk_grid_barrier(a, &sh, epoch))) break;
         }
         if (!ok && threadIdx.x == 0) sh.giving_up = 1;

@@ -266,3 +266,30 @@ def test_timeout_is_reported_once_and_the_context_recovers(util):
     ln, pend = P.g.slot_state(0)
     P.check_cache(0, range(1, 5), ln - pend)
     P.close()
+
+
+MICRO256 = dict(n_layers=3, d_model=256, n_q_heads=4, n_kv_heads=2, head_dim=64, d_ffn=512,
+                vocab_text=301, vocab_speech=99, rms_eps=1e-6, rope_base=10000.0)
+
+
+@pytest.mark.parametrize("K,maxp", [(4, 3), (3, 2)])
+def test_persistent_kernel_tensor_core_form_for_three_and_four_rows(util, K, maxp):
+    """Flushes of two and three pending rows (passes of three and four rows) inside the persistent
+    layer-range kernel: its tensor-core form (swizzled weight boxes, mma.sync, two-term
+    activations), on a shape whose inner dimensions are whole 64-element blocks."""
+    dims = synth.model_dims(MICRO256, 1, K, 0)
+    w = synth.make_weights(dims, seed=9)
+    prompt = synth.make_prompts(dims, 1, 23, 23, seed=2)[0]
+    P = util.Pair(dims, w, 1, 23 + 64, maxp, prefill_rows=16, options={"mega_max_rows": 4})
+    P.prefill([prompt])
+    before = P.g.route_counts()
+    for g in range(30):
+        m, c = synth.interleave(g, 1, K)
+        P.step([m], [c])
+    after = P.g.route_counts()
+    assert after["tc"] == before["tc"] and after["gemv"] == before["gemv"]      # every decode pass ran in the persistent kernel
+    assert P.stats["max_flush"] == K - 1
+    ln, pend = P.g.slot_state(0)
+    P.check_cache(0, range(1, 4), ln - pend)
+    print("mega tc", P.stats)
+    P.close()
