@@ -75,6 +75,10 @@ struct sparsk_ctx {
     bf16 *attn_o_lo, *act_lo, *xnorm_lo;  // second bf16 term of the tensor-core path's activations
     float *part_o;
     float2 *part_ml;
+    unsigned *attn_ticket;       // device: item counter of the attention kernel (only ever grows)
+    unsigned attn_ticket_base;   // host: its value once every launch so far has finished
+    int attn_dynamic;            // option: deal attention items by ticket (1, default) or round-robin (0)
+    int attn_ctas;               // option: CTAs of the attention kernel (0: as many as fit the SMs)
     // pinned staging ring for the per-step host arrays
     int *stage_host[STAGE_RING];
     cudaEvent_t stage_ev[STAGE_RING];
@@ -222,6 +226,7 @@ size_t carve(sparsk_ctx *c, const sparsk_dims *d, char *base)
     MkLayer *mkl = w.take<MkLayer>(L);
     unsigned long long *mkb = w.take<unsigned long long>(1);
     int *mka = w.take<int>(1);
+    unsigned *atk = w.take<unsigned>(1);
     float *mkao = w.take<float>((size_t)MK_MAX_ROWS * qrow), *mkact = w.take<float>((size_t)MK_MAX_ROWS * d->d_ffn);
     unsigned long long *mkt = w.take<unsigned long long>(1 + 6 * L);
     const size_t cells = std::max<size_t>(R * MAX_SPLITS, (size_t)MK_MAX_ROWS * MK_MAX_SPLITS) * d->n_q_heads;
@@ -237,7 +242,7 @@ size_t carve(sparsk_ctx *c, const sparsk_dims *d, char *base)
         c->h_lo = hlo; c->h_up = hup; c->qbuf = q; c->attn_o = ao; c->act = act; c->xnorm = xn; c->qkv_part = qp;
         c->attn_o_lo = aol; c->act_lo = actl; c->xnorm_lo = xnl;
         c->mk_layers = mkl; c->mk_bar = mkb; c->mk_abort = mka; c->mk_attn_o = mkao; c->mk_act = mkact; c->mk_trace = mkt;
-        c->part_o = po; c->part_ml = pml;
+        c->part_o = po; c->part_ml = pml; c->attn_ticket = atk;
     }
     return align_up(w.off, 256);
 }
@@ -338,6 +343,7 @@ struct RowSet {
     int max_len;    // longest prefix any row attends to (host)
     int n_big;      // groups with at least attn_tc_min_q query vectors per kv head (0: not counted, assume all)
     const float *q; // the rows' queries if they are not the context's query buffer (NULL: they are)
+    long sum_len;   // total of the groups' prefix lengths (host; 0: unknown)
 };
 
 cudaError_t run_qkv(sparsk_ctx *c, int layer, const float *h, const RowSet &rs)
@@ -463,10 +469,10 @@ cudaError_t run_attn(sparsk_ctx *c, int layer, const RowSet &rs)
     // groups the tcgen05 kernel takes (the host knows every group's row count) and the rest
     const int n_big = blocks_tc ? (rs.n_big > 0 ? rs.n_big : rs.n_groups_h) : 0;
     const int n_small = rs.n_groups_h - n_big;
-    const int warp_ctas = c->n_sm * attn_warp_ctas_per_sm(d.head_dim, c->attn_stages);
+    const int warp_ctas = c->attn_ctas > 0 ? c->attn_ctas : c->n_sm * attn_warp_ctas_per_sm(d.head_dim, c->attn_stages);
     const int small_rows = blocks_tc ? std::max(1, std::min(rs.max_grp_rows, (c->attn_tc_min_q - 1) / G)) : rs.max_grp_rows;
     AttnPlan pl = attn_plan(warp_ctas * AW_WARPS, blocks_tc ? std::max(1, n_small) : rs.n_groups_h, small_rows, G,
-                            d.n_kv_heads, rs.max_len, c->attn_split);
+                            d.n_kv_heads, rs.max_len, c->attn_split, blocks_tc ? 0 : rs.sum_len);
     if (blocks_tc) {
         // Groups with many query vectors per kv head go to the tcgen05 kernel (one CTA per SM, tiles
         // of 64 positions), the others to the mma.sync kernel; both launches cover all groups, a CTA
@@ -529,8 +535,15 @@ cudaError_t run_attn(sparsk_ctx *c, int layer, const RowSet &rs)
         AttnWarpFn fn;
         e = attn_warp_fn(d.head_dim, c->attn_stages, &fn);
         if (e != cudaSuccess) return e;
+        if (c->attn_dynamic && n_items < (1L << 31)) {
+            a.ticket = c->attn_ticket;
+            a.ticket_base = c->attn_ticket_base;
+        }
         e = launch(c, fn, dim3(grid), dim3(AW_WARPS * 32), AW_WARPS * attn_warp_bytes(d.head_dim, c->attn_stages), a);
         if (e != cudaSuccess) return e;
+        // the items beyond the warps' first ones are drawn once each, and every warp draws one
+        // ticket beyond its last item
+        if (a.ticket && n_items > (long)grid * AW_WARPS) c->attn_ticket_base += (unsigned)n_items;
     }
     if (d.head_dim == 128) return launch(c, attn_merge_kernel<128>, dim3(rs.n_rows, d.n_q_heads), dim3(128), 0, a, rs.n_rows_dev);
     return launch(c, attn_merge_kernel<64>, dim3(rs.n_rows, d.n_q_heads), dim3(64), 0, a, rs.n_rows_dev);
@@ -1059,6 +1072,7 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
     ctx->mk_max_rows = MK_MAX_ROWS;
     ctx->attn_tc = 1; ctx->attn_tc_min_q = 33; ctx->attn_stages = AW_NST;
     ctx->inject_timeout = 0;
+    ctx->attn_ticket_base = 0; ctx->attn_dynamic = 1; ctx->attn_ctas = 0;
     ctx->trim_last = 1;
     ctx->conf_host = nullptr; ctx->conf_ent_host = nullptr;
     ctx->h_fill.assign(dims->max_seqs, std::vector<int>());
@@ -1126,6 +1140,7 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
             (ce = cudaMemsetAsync(ctx->kv_len, 0, sizeof(int) * dims->max_seqs, ctx->stream)) != cudaSuccess ||
             (ce = cudaMemsetAsync(ctx->pend_cnt, 0, sizeof(int) * dims->max_seqs, ctx->stream)) != cudaSuccess ||
             (ce = cudaMemsetAsync(ctx->sd.counts, 0, sizeof(int) * 8, ctx->stream)) != cudaSuccess ||
+            (ce = cudaMemsetAsync(ctx->attn_ticket, 0, sizeof(unsigned), ctx->stream)) != cudaSuccess ||
             (ce = cudaMemsetAsync(ctx->qkv_part, 0, sizeof(float) * (size_t)ctx->cap_rows * (dims->n_q_heads + 2 * dims->n_kv_heads) * dims->head_dim, ctx->stream)) != cudaSuccess ||
             (ce = cudaStreamSynchronize(ctx->stream)) != cudaSuccess) {
             rc = fail(ctx, SPARSK_ECUDA, "table upload failed: %s", cudaGetErrorString(ce));
@@ -1223,6 +1238,8 @@ extern "C" int sparsk_set_option(sparsk_ctx *ctx, const char *name, int64_t valu
     else if (!strcmp(name, "gemv_ks") && (value == 0 || value == 1 || value == 2 || value == 4 || value == 8 || value == 16)) ctx->gv_ks = (int)value;
     else if (!strcmp(name, "mega") && (value == 0 || value == 1)) ctx->mega = (int)value;
     else if (!strcmp(name, "attn_stages") && (value == 2 || value == 3)) ctx->attn_stages = (int)value;
+    else if (!strcmp(name, "attn_dynamic") && (value == 0 || value == 1)) ctx->attn_dynamic = (int)value;
+    else if (!strcmp(name, "attn_ctas") && value >= 0 && value <= 65535) ctx->attn_ctas = (int)value;
     else if (!strcmp(name, "attn_tc") && (value == 0 || value == 1)) ctx->attn_tc = (int)value;
     else if (!strcmp(name, "attn_tc_min_q") && value >= 1 && value <= (1 << 20)) ctx->attn_tc_min_q = (int)value;
     else if (!strcmp(name, "mega_max_rows") && value >= 1 && value <= MK_MAX_ROWS) ctx->mk_max_rows = (int)value;
@@ -1274,7 +1291,9 @@ static int read_status(sparsk_ctx *ctx)
     if (status & ST_TIMEOUT) {
         CU(cudaMemsetAsync(ctx->mk_bar, 0, sizeof(unsigned long long), ctx->stream));
         CU(cudaMemsetAsync(ctx->mk_abort, 0, sizeof(int), ctx->stream));
+        CU(cudaMemsetAsync(ctx->attn_ticket, 0, sizeof(unsigned), ctx->stream));
         ctx->mk_bar_base = 0;
+        ctx->attn_ticket_base = 0;
         return fail(ctx, SPARSK_ETIMEOUT, "a bounded in-kernel wait ran out");
     }
     if (status & ST_BAD_TOKEN) return fail(ctx, SPARSK_EINVAL, "a token id was outside the vocabulary (clamped)");
@@ -1647,6 +1666,7 @@ extern "C" int sparsk_decode_step(sparsk_ctx *ctx, int32_t n, const int32_t *slo
     std::vector<char> seen(B, 0);
     int n_list[4] = {0, 0, 0, 0};
     int m_up = 0, n_grp = 0, max_grp = 1, max_len_lo = 0, max_len_up = 0, n_big = 0;
+    long sum_len_lo = 0, sum_len_up = 0;
     const int G_heads = d.n_q_heads / d.n_kv_heads;
     for (int i = 0; i < n; i++) {
         const int s = slots[i];
@@ -1661,7 +1681,9 @@ extern "C" int sparsk_decode_step(sparsk_ctx *ctx, int32_t n, const int32_t *slo
             return fail(ctx, SPARSK_ECAPACITY, "decode_step: slot %d would hold %d pending positions (max_pending %d)", s, ctx->h_pend[s] + 1, d.max_pending);
         n_list[(full ? 2 : 0) + (modality[i] ? 1 : 0)]++;
         max_len_lo = std::max(max_len_lo, ctx->h_len[s] + 1);
+        sum_len_lo += ctx->h_len[s] + 1;
         if (full && e < L) {
+            sum_len_up += ctx->h_len[s] + 1;
             m_up += ctx->h_pend[s] + 1;
             n_grp++;
             max_grp = std::max(max_grp, ctx->h_pend[s] + 1);
@@ -1701,6 +1723,7 @@ extern "C" int sparsk_decode_step(sparsk_ctx *ctx, int32_t n, const int32_t *slo
     // ---- lower pass: layers 1..e over all sequences
     RowSet lo{ctx->sd.slot, ctx->sd.lo_pos, ctx->sd.lo_grp_row0, ctx->sd.lo_grp_nrows, ctx->sd.counts + CNT_NSEQ,
               ctx->sd.counts + CNT_NSEQ, n, n, 1, max_len_lo};
+    lo.sum_len = sum_len_lo;
     CU(run_layers(ctx, 1, e, ctx->h_lo, lo));
     // ---- early exits: keep h^(e), read the token from g_e
     if (n_list[0] + n_list[1]) {
@@ -1716,6 +1739,7 @@ extern "C" int sparsk_decode_step(sparsk_ctx *ctx, int32_t n, const int32_t *slo
                   (const float *)ctx->pend_h, ctx->h_up, d.d_model, d.max_pending));
         RowSet up{ctx->sd.up_slot, ctx->sd.up_pos, ctx->sd.up_grp_row0, ctx->sd.up_grp_nrows, ctx->sd.counts + CNT_NGRP,
                   ctx->sd.counts + CNT_MUP, m_up, n_grp, max_grp, max_len_up, n_big};
+        up.sum_len = sum_len_up;
         // Layer L gives the pending rows nothing but their K/V: nothing reads their h^(L).  When the
         // step has pending rows and the rest of the layer is cheaper on one row per sequence
         // (attention over long prefixes, projections with enough rows to be tensor-bound), the
@@ -1734,6 +1758,7 @@ extern "C" int sparsk_decode_step(sparsk_ctx *ctx, int32_t n, const int32_t *slo
                       (const float *)ctx->qbuf, ctx->h_last, ctx->q_last, ctx->last_slot, ctx->last_pos, d.d_model, qd));
             RowSet last{ctx->last_slot, ctx->last_pos, ctx->sd.lo_grp_row0, ctx->sd.lo_grp_nrows, ctx->sd.counts + CNT_NGRP,
                         ctx->sd.counts + CNT_NGRP, n_grp, n_grp, 1, max_len_up, 0, ctx->q_last};
+            last.sum_len = sum_len_up;
             CU(run_layer_back(ctx, L, ctx->h_last, last));
             CU(launch(ctx, put_current_kernel, dim3(n_grp), dim3(256), 0, ctx->sd, (const float *)ctx->h_last, ctx->h_up,
                       d.d_model));

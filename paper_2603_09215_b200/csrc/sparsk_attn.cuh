@@ -39,19 +39,23 @@ constexpr int AW_NST = 2;        // ring stages per warp there (default; 3 is th
 struct AttnPlan {
     int n_qblk, split_len, n_splits;
 };
-inline AttnPlan attn_plan(int n_workers, int n_groups, int max_grp_rows, int G, int Hkv, int max_len, int forced_split)
+// `sum_len` is the total of the groups' prefix lengths when the caller knows it (0: assume every
+// group is as long as the longest): with ragged lengths the splits past a short group's end are
+// empty items, and sizing by the real total keeps the number of items with work near 1.75 per
+// warp whatever the spread of the lengths (shorter items add set-up, longer ones a ragged end).
+inline AttnPlan attn_plan(int n_workers, int n_groups, int max_grp_rows, int G, int Hkv, int max_len, int forced_split,
+                          long sum_len = 0)
 {
     AttnPlan p;
     const int nq = max_grp_rows * G;
     p.n_qblk = (nq + 15) / 16;
     int split = forced_split;
     if (split <= 0) {
-        const long base = (long)(n_groups < 1 ? 1 : n_groups) * p.n_qblk * Hkv;
-        long want = (3L * n_workers + base - 1) / base;   // about three items per warp
-        if (want < 1) want = 1;
-        if (want > AT_MAX_SPLITS) want = AT_MAX_SPLITS;
-        split = (int)((max_len + want - 1) / want);
+        const long groups = n_groups < 1 ? 1 : n_groups;
+        const long total = (sum_len > 0 ? sum_len : groups * (long)max_len) * p.n_qblk * Hkv;  // positions x heads to visit
+        split = (int)(total * 4 / (7L * n_workers));  // 1.75 items per warp (measured best at 64 ragged sequences)
         if (split < AT_MIN_SPLIT) split = AT_MIN_SPLIT;
+        if (split > max_len) split = max_len < 1 ? 1 : max_len;
     }
     split = (split + AT_TP - 1) / AT_TP * AT_TP;
     int n_splits = (max_len + split - 1) / split;
@@ -83,6 +87,14 @@ struct AttnArgs {
     int n_rows;               // rows in q/out; groups reaching beyond them are skipped
     int nq_min, nq_max;       // only groups with this many query vectors per kv head (another launch takes the rest)
     int max_groups;           // host bound on the number of groups (sizes the item space)
+    // Dynamic dealing of items (optional): a counter that only ever grows.  With W warps and
+    // n > W items, warp w starts on item w and ticket ticket_base + t stands for item W + t
+    // (unsigned arithmetic, so the counter may wrap); every warp draws exactly one ticket beyond
+    // its last item, so the launch adds n to the counter, which is how the host knows the next
+    // launch's base without reading it.  With n <= W no ticket is drawn.  NULL: items are dealt
+    // round-robin.
+    unsigned *ticket;
+    unsigned ticket_base;
 };
 
 __device__ __forceinline__ void cp_async16(void *dst, const void *src, int src_bytes)
@@ -141,6 +153,14 @@ __device__ __forceinline__ void attn_item(const AttnArgs &a, int qb, int hk, int
     const int w_beg = sp * split_len;
     const int w_end = min(w_beg + split_len, kv_end_all);
     const int n_tiles = w_end > w_beg ? (w_end - w_beg + AT_TP - 1) / AT_TP : 0;
+    if (n_tiles == 0) {
+        // an empty split: max = -inf, sum = 0 is all the merge looks at
+        for (int qi = lane; qi < nq_here; qi += 32) {
+            const int qg = q0 + qi;
+            a.part_ml[((size_t)(row0 + qg / G) * a.Hq + hk * G + qg % G) * splits + sp] = make_float2(-INFINITY, 0.f);
+        }
+        return;
+    }
     const kv_t *kbase = a.kc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
     const kv_t *vbase = a.vc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
 
@@ -346,10 +366,13 @@ __device__ __forceinline__ void attn_item(const AttnArgs &a, int qb, int hk, int
     }
 }
 
-// Persistent grid of warps; item i = ((g * Hkv + hk) * n_splits + sp) * n_qblk + qb goes to warp
-// i mod (number of warps), warps numbered so that consecutive items land on different SMs: the
-// query blocks of one (group, kv head, split) run side by side, and all but the first find
-// their K/V tiles in the L2.
+// Persistent grid of warps; item i = ((sp * groups + g) * Hkv + hk) * n_qblk + qb: the query
+// blocks of one (group, kv head, split) run side by side, and all but the first find their K/V
+// tiles in the L2; the splits that short groups leave empty come last.  With a ticket counter
+// the warps draw items as they finish (ragged lengths make the items of a round-robin deal
+// uneven: a third of the warps idle on average at 64 sequences of 256..2048 positions);
+// without one, item i goes to warp i mod (number of warps), warps numbered so that consecutive
+// items land on different SMs.
 template <int HD, int NST>
 __global__ void __launch_bounds__(AW_WARPS * 32) attn_warp_kernel(AttnArgs a)
 {
@@ -360,13 +383,26 @@ __global__ void __launch_bounds__(AW_WARPS * 32) attn_warp_kernel(AttnArgs a)
     kv_t *wr = reinterpret_cast<kv_t *>(aw_smem) + (size_t)warp * NST * 2 * AT_TP * (HD + 8);
     const int G = a.Hq / a.Hkv;
     const int n_groups = min(*a.n_groups, a.max_groups);
-    const long n_items = (long)n_groups * a.n_qblk * a.Hkv * a.n_splits;
-    const long n_workers = (long)gridDim.x * AW_WARPS;
-    for (long item = (long)warp * gridDim.x + blockIdx.x; item < n_items; item += n_workers) {
-        long t = item;
+    const unsigned n_items = (unsigned)a.max_groups * a.n_qblk * a.Hkv * a.n_splits;
+    const unsigned n_workers = gridDim.x * AW_WARPS;
+    // every warp's first item is its own number (no counter, no latency); tickets number the
+    // items beyond that first round, so a launch with no more items than warps draws none
+    const bool dynamic = a.ticket != nullptr && n_items > n_workers;
+    auto draw = [&]() -> unsigned {
+        unsigned t = 0;
+        if (lane == 0) t = atomicAdd(a.ticket, 1u) - a.ticket_base;
+        return n_workers + __shfl_sync(0xffffffffu, t, 0);
+    };
+    unsigned item = (unsigned)warp * gridDim.x + blockIdx.x;
+    while (item < n_items) {
+        // the next ticket is drawn before this item's work, so that its latency is hidden
+        const unsigned next = dynamic ? draw() : item + n_workers;
+        unsigned t = item;
+        item = next;
         const int qb = (int)(t % a.n_qblk); t /= a.n_qblk;
-        const int sp = (int)(t % a.n_splits); t /= a.n_splits;
-        const int hk = (int)(t % a.Hkv), g = (int)(t / a.Hkv);
+        const int hk = (int)(t % a.Hkv); t /= a.Hkv;
+        const int g = (int)(t % a.max_groups), sp = (int)(t / a.max_groups);
+        if (g >= n_groups) continue;
         const int row0 = a.grp_row0[g], nrows = a.grp_nrows[g];
         if (row0 < 0 || nrows < 1 || row0 + nrows > a.n_rows) continue;
         const int nq = nrows * G;

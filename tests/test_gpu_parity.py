@@ -232,6 +232,27 @@ def test_every_route_for_small_passes(util, options):
     P.close()
 
 
+@pytest.mark.parametrize("options", [{"attn_ctas": 2, "attn_split": 16, "mega": 0},
+                                     {"attn_ctas": 2, "attn_split": 16, "mega": 0, "attn_dynamic": 0},
+                                     {"attn_ctas": 1, "mega": 0, "gemm_min_rows": 1}])
+def test_attention_items_drawn_from_the_counter(util, options):
+    """Many more attention work items than warps (the kernel held to one or two CTAs, four ragged
+    sequences, short splits): the warps draw items from the ticket counter, launch after launch
+    (the host predicts the counter's value instead of resetting it), or take every n-th item."""
+    dims = synth.model_dims("tiny", 2, 4, 0)
+    w = synth.make_weights(dims, seed=0)
+    prompts = synth.make_prompts(dims, 4, 9, 150, seed=21)
+    P = util.Pair(dims, w, 4, 200, 3, prefill_rows=16, options=options)
+    P.prefill(prompts)
+    for g in range(14):
+        mc = [synth.interleave(g + 2 * i, 1, 4) for i in range(4)]
+        P.step([m for m, _ in mc], [c for _, c in mc])
+    for s_ in range(4):
+        ln, pend = P.g.slot_state(s_)
+        P.check_cache(s_, range(1, 5), ln - pend)
+    P.close()
+
+
 def test_timeout_is_reported_once_and_the_context_recovers(util):
     """A bounded in-kernel wait that runs out: the persistent kernel is told a grid-barrier count
     that no CTA can reach (a host-side test hook; nothing faults or hangs), its wait ends at the
