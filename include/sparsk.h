@@ -194,7 +194,9 @@ int sparsk_set_debug(sparsk_ctx *ctx, float *exit_hidden /*device or NULL*/,
  * dimension per TMA copy instead of two; 0 = automatic), "attn_split" (positions
  * per KV split), "attn_dynamic" (0/1: the attention kernel's warps draw their work items from a
  * counter as they finish instead of taking every n-th one; default 1), "attn_ctas" (CTAs of that
- * kernel; 0 = as many as fit the SMs), "pdl" (0/1, programmatic dependent launch between the kernels of a step; default 1),
+ * kernel; 0 = as many as fit the SMs), "attn_tma" (0/1: its K/V tiles arrive as TMA boxes with the
+ * 128-byte swizzle instead of per-lane 16-byte copies; default 1), "attn_stages" (2 or 3 tiles per
+ * warp's ring), "pdl" (0/1, programmatic dependent launch between the kernels of a step; default 1),
  * "gemv_ks" / "gemv_r" (override the GEMV team width / rows per group; 0 = automatic),
  * "trim_last_layer" (0/1/2: in a full-depth step, pending rows leave layer L after its K/V
  * projection, since Algorithm 1's full-depth branch reads h^(L) of the current position only; 1,

@@ -98,6 +98,8 @@ struct sparsk_ctx {
     bool tc_ok;
     std::vector<TmaPair> tm_wq, tm_wk, tm_wv, tm_wo, tm_wg, tm_wu, tm_wd, tm_head;
     TmaPair tm_x[5], tm_ao[5], tm_act[5], tm_x_lo[5], tm_ao_lo[5], tm_act_lo[5];
+    std::vector<CUtensorMap> tm_kc16, tm_vc16;  // per layer: the cache as rows of head_dim numbers, boxes of 16 rows (attn_warp_tma_kernel)
+    int attn_tma, attn_tma_ok;               // option (default 1); the maps above exist
     std::vector<CUtensorMap> tm_kc, tm_vc;  // per layer: the cache viewed as [64][slots * Hkv * S rows][hd / 64], boxes of [64][64][2]
     int attn_stages;                        // K/V ring depth of the warp-per-item attention kernel (2 or 3)
     int attn_tc, attn_tc_min_q;             // tcgen05 attention for blocks of at least this many query vectors
@@ -531,19 +533,26 @@ cudaError_t run_attn(sparsk_ctx *c, int layer, const RowSet &rs)
     if (!blocks_tc || (c->attn_tc_min_q > 1 && n_small > 0)) {
         // every group is in the item space (the kernel skips those the other kernel takes)
         const long n_items = (long)rs.n_groups_h * a.n_qblk * d.n_kv_heads * a.n_splits;
-        const int grid = (int)std::max<long>(1, std::min<long>(warp_ctas, (n_items + AW_WARPS - 1) / AW_WARPS));
-        AttnWarpFn fn;
-        e = attn_warp_fn(d.head_dim, c->attn_stages, &fn);
+        const bool tma = c->attn_tma && c->attn_tma_ok;
+        int warps = AW_WARPS;
+        AttnWarpFn fn = nullptr;
+        AttnWarpTmaFn fn_tma = nullptr;
+        e = tma ? attn_warp_tma_fn(d.head_dim, c->attn_stages, &fn_tma, &warps) : attn_warp_fn(d.head_dim, c->attn_stages, &fn);
         if (e != cudaSuccess) return e;
+        const int grid = (int)std::max<long>(1, std::min<long>(warp_ctas, (n_items + warps - 1) / warps));
         if (c->attn_dynamic && n_items < (1L << 31)) {
             a.ticket = c->attn_ticket;
             a.ticket_base = c->attn_ticket_base;
         }
-        e = launch(c, fn, dim3(grid), dim3(AW_WARPS * 32), AW_WARPS * attn_warp_bytes(d.head_dim, c->attn_stages), a);
+        if (tma)
+            e = launch(c, fn_tma, dim3(grid), dim3(warps * 32), attn_warp_tma_bytes(d.head_dim, c->attn_stages, warps),
+                       c->tm_kc16[layer - 1], c->tm_vc16[layer - 1], a, c->sd.counts + CNT_STATUS);
+        else
+            e = launch(c, fn, dim3(grid), dim3(warps * 32), AW_WARPS * attn_warp_bytes(d.head_dim, c->attn_stages), a);
         if (e != cudaSuccess) return e;
         // the items beyond the warps' first ones are drawn once each, and every warp draws one
         // ticket beyond its last item
-        if (a.ticket && n_items > (long)grid * AW_WARPS) c->attn_ticket_base += (unsigned)n_items;
+        if (a.ticket && n_items > (long)grid * warps) c->attn_ticket_base += (unsigned)n_items;
     }
     if (d.head_dim == 128) return launch(c, attn_merge_kernel<128>, dim3(rs.n_rows, d.n_q_heads), dim3(128), 0, a, rs.n_rows_dev);
     return launch(c, attn_merge_kernel<64>, dim3(rs.n_rows, d.n_q_heads), dim3(64), 0, a, rs.n_rows_dev);
@@ -604,6 +613,21 @@ bool build_maps(sparsk_ctx *c)
     fill(c->tm_wv, c->wv, kd, d.d_model, 2 * GM_BM); fill(c->tm_wo, c->wo, d.d_model, qd, 2 * GM_BM);
     fill(c->tm_wg, c->w_gate, d.d_ffn, d.d_model, GM_BM); fill(c->tm_wu, c->w_up, d.d_ffn, d.d_model, GM_BM);
     fill(c->tm_wd, c->w_down, d.d_model, d.d_ffn, 2 * GM_BM); fill(c->tm_head, c->head_proj, V, d.d_model, 2 * GM_BM);
+    if (d.head_dim == 64 || d.head_dim == 128) {
+        const size_t lstride = (size_t)d.max_seqs * d.n_kv_heads * d.max_seq_len * d.head_dim;
+        const size_t rows = (size_t)d.max_seqs * d.n_kv_heads * d.max_seq_len;
+        c->tm_kc16.resize(L);
+        c->tm_vc16.resize(L);
+        bool ok16 = rows < (1ull << 31);
+        for (int l = 0; l < L && ok16; l++) {
+            TmaPair t;
+            ok16 = ok16 && encode_maps(fn, &t, c->kcache + l * lstride, rows, d.head_dim, AT_TP, CU_TENSOR_MAP_DATA_TYPE_FLOAT16);
+            c->tm_kc16[l] = d.head_dim == 128 ? t.m3 : t.m2;
+            ok16 = ok16 && encode_maps(fn, &t, c->vcache + l * lstride, rows, d.head_dim, AT_TP, CU_TENSOR_MAP_DATA_TYPE_FLOAT16);
+            c->tm_vc16[l] = d.head_dim == 128 ? t.m3 : t.m2;
+        }
+        c->attn_tma_ok = ok16 ? 1 : 0;
+    }
     if (d.head_dim == TA_HD) {
         const size_t lstride = (size_t)d.max_seqs * d.n_kv_heads * d.max_seq_len * d.head_dim;
         c->tm_kc.resize(L);
@@ -1073,6 +1097,7 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
     ctx->attn_tc = 1; ctx->attn_tc_min_q = 33; ctx->attn_stages = AW_NST;
     ctx->inject_timeout = 0;
     ctx->attn_ticket_base = 0; ctx->attn_dynamic = 1; ctx->attn_ctas = 0;
+    ctx->attn_tma = 1; ctx->attn_tma_ok = 0;
     ctx->trim_last = 1;
     ctx->conf_host = nullptr; ctx->conf_ent_host = nullptr;
     ctx->h_fill.assign(dims->max_seqs, std::vector<int>());
@@ -1239,6 +1264,7 @@ extern "C" int sparsk_set_option(sparsk_ctx *ctx, const char *name, int64_t valu
     else if (!strcmp(name, "mega") && (value == 0 || value == 1)) ctx->mega = (int)value;
     else if (!strcmp(name, "attn_stages") && (value == 2 || value == 3)) ctx->attn_stages = (int)value;
     else if (!strcmp(name, "attn_dynamic") && (value == 0 || value == 1)) ctx->attn_dynamic = (int)value;
+    else if (!strcmp(name, "attn_tma") && (value == 0 || value == 1)) ctx->attn_tma = (int)value;
     else if (!strcmp(name, "attn_ctas") && value >= 0 && value <= 65535) ctx->attn_ctas = (int)value;
     else if (!strcmp(name, "attn_tc") && (value == 0 || value == 1)) ctx->attn_tc = (int)value;
     else if (!strcmp(name, "attn_tc_min_q") && value >= 1 && value <= (1 << 20)) ctx->attn_tc_min_q = (int)value;

@@ -129,17 +129,37 @@ __device__ __forceinline__ void mma_f16(float (&d)[4], const uint32_t (&a)[4], u
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// The TMA-fed form of a warp's ring: tiles arrive as tensor-map boxes of 16 positions with the
+// 128-byte swizzle (no padding, one copy per tile and matrix instead of sixteen cp.async per
+// lane), each stage with an mbarrier of its own whose phases run on across the warp's items.
+struct AttnTma {
+    const CUtensorMap *mk, *mv;  // this layer's K and V cache as rows of head_dim fp16 numbers
+    uint64_t *bars;              // the warp's NS barriers
+    uint32_t seq;                // tiles this warp has consumed so far (stage = seq mod NS)
+    volatile int *giving_up;     // CTA-wide: a wait ran out
+    int *status;                 // device status word
+};
+// Element offset of 16-byte chunk c of row `row` inside a swizzled tile: blocks of 16 rows x 64
+// elements (one per 64 elements of the head dimension), chunk index XOR row mod 8.
+template <int HD>
+__device__ __forceinline__ int at_swz(int row, int c)
+{
+    return (HD > 64 ? (c >> 3) * (AT_TP * 64) : 0) + row * 64 + (((c & 7) ^ (row & 7)) << 3);
+}
+
 // One item, by one warp: query vectors [16 qb, 16 qb + 16) of a group whose first row is row0
 // (nrows rows of slot `slot`, first at position pos0), kv head hk, split sp of `splits` splits of
 // split_len positions.  `wr` is the warp's ring of NS stages.  Writes the item's partial.
 // QREG: the query fragments stay in registers for the whole item (32 registers at head dimension
 // 128); otherwise they are parked in `qs` ([16][HD + 8] of shared memory) and re-read per tile,
 // for callers whose register budget is spoken for.
-template <int HD, int NS, bool QREG>
+template <int HD, int NS, bool QREG, bool TMA = false>
 __device__ __forceinline__ void attn_item(const AttnArgs &a, int qb, int hk, int sp, int splits, int split_len, int row0,
-                                          int nrows, int slot, int pos0, kv_t *wr, kv_t *qs, int lane)
+                                          int nrows, int slot, int pos0, kv_t *wr, kv_t *qs, int lane,
+                                          AttnTma *tm = nullptr)
 {
-    constexpr int KP = HD + 8;      // padded row: ldmatrix rows fall into distinct banks
+    constexpr int KP = HD + 8;      // padded row (cp.async form; also the parked queries): ldmatrix rows fall into distinct banks
+    constexpr int TP = TMA ? HD : KP;  // row pitch of a K/V tile in the ring
     constexpr int CH = HD / 8;      // 16-byte chunks per row
     constexpr float LOG2E = 1.4426950408889634f, LN2 = 0.6931471805599453f;
     const int G = a.Hq / a.Hkv;
@@ -164,16 +184,34 @@ __device__ __forceinline__ void attn_item(const AttnArgs &a, int qb, int hk, int
     const kv_t *kbase = a.kc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
     const kv_t *vbase = a.vc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
 
+    const uint32_t seq0 = TMA ? tm->seq : 0u;
     auto issue = [&](int t) {
-        kv_t *kt = wr + (size_t)(t % NS) * 2 * AT_TP * KP, *vt = kt + AT_TP * KP;
+        const int st = (int)((seq0 + (uint32_t)t) % NS);
+        kv_t *kt = wr + (size_t)st * 2 * AT_TP * TP, *vt = kt + AT_TP * TP;
         const int p0 = w_beg + t * AT_TP;
+        if constexpr (TMA) {
+            // rows past the split's end arrive as whatever the cache holds there (or zeros beyond
+            // the cache): the scores mask them, the value rows are cleared after landing
+            if (lane == 0) {
+                const int y = (slot * a.Hkv + hk) * a.S + p0;
+                mbar_expect_tx(&tm->bars[st], 2u * AT_TP * HD * (uint32_t)sizeof(kv_t));
+                if (HD > 64) {
+                    tma_load_3d(smem_u32(kt), tm->mk, &tm->bars[st], 0, y, 0);
+                    tma_load_3d(smem_u32(vt), tm->mv, &tm->bars[st], 0, y, 0);
+                } else {
+                    tma_load_2d(smem_u32(kt), tm->mk, &tm->bars[st], 0, y);
+                    tma_load_2d(smem_u32(vt), tm->mv, &tm->bars[st], 0, y);
+                }
+            }
+        } else {
 #pragma unroll
-        for (int i = lane; i < AT_TP * CH; i += 32) {
-            const int r = i / CH, c = i % CH;
-            const bool ok = p0 + r < w_end;                  // rows past the end are zero-filled
-            const size_t off = (size_t)(ok ? p0 + r : w_beg) * HD + c * 8;
-            cp_async16(&kt[r * KP + c * 8], kbase + off, ok ? 16 : 0);
-            cp_async16(&vt[r * KP + c * 8], vbase + off, ok ? 16 : 0);
+            for (int i = lane; i < AT_TP * CH; i += 32) {
+                const int r = i / CH, c = i % CH;
+                const bool ok = p0 + r < w_end;                  // rows past the end are zero-filled
+                const size_t off = (size_t)(ok ? p0 + r : w_beg) * HD + c * 8;
+                cp_async16(&kt[r * KP + c * 8], kbase + off, ok ? 16 : 0);
+                cp_async16(&vt[r * KP + c * 8], vbase + off, ok ? 16 : 0);
+            }
         }
     };
     // The ring: tiles t .. t + NS - 1 are in flight or in use while tile t is computed; every
@@ -183,7 +221,7 @@ __device__ __forceinline__ void attn_item(const AttnArgs &a, int qb, int hk, int
 #pragma unroll
     for (int t = 0; t < NS; t++) {
         if (t < n_tiles) issue(t);
-        cp_async_commit();
+        if (!TMA) cp_async_commit();
     }
 
     // the queries, as A fragments (row = lane / 4 and + 8, columns 2 (lane % 4) + {0, 1, 8, 9} of
@@ -251,10 +289,23 @@ __device__ __forceinline__ void attn_item(const AttnArgs &a, int qb, int hk, int
     const int lim_min = pos0 + q0 / G;  // the smallest limit among the item's query vectors
 
     for (int t = 0; t < n_tiles; t++) {
-        cp_async_wait<NS - 1>();  // tile t has landed
-        __syncwarp();
-        const kv_t *Kt = wr + (size_t)(t % NS) * 2 * AT_TP * KP, *Vt = Kt + AT_TP * KP;
+        const int st = (int)((seq0 + (uint32_t)t) % NS);
+        kv_t *Kt = wr + (size_t)st * 2 * AT_TP * TP, *Vt = Kt + AT_TP * TP;
         const int p0 = w_beg + t * AT_TP;
+        if constexpr (TMA) {
+            if (!mbar_wait(&tm->bars[st], ((seq0 + (uint32_t)t) / NS) & 1u, tm->giving_up, tm->status)) return;
+            if (p0 + AT_TP > w_end) {
+                // value rows past the end meet a weight of exactly zero, which must not meet a
+                // NaN or an infinity: clear them
+                const int nv = w_end - p0;
+                for (int i = lane; i < (AT_TP - nv) * CH; i += 32)
+                    *reinterpret_cast<uint4 *>(&Vt[at_swz<HD>(nv + i / CH, i % CH)]) = make_uint4(0u, 0u, 0u, 0u);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            }
+        } else {
+            cp_async_wait<NS - 1>();  // tile t has landed
+        }
+        __syncwarp();
 
         // S = Q K^T for 16 positions, in log2 units; two accumulator chains
         float s[2][4], s2[2][4];
@@ -265,8 +316,14 @@ __device__ __forceinline__ void attn_item(const AttnArgs &a, int qb, int hk, int
 #pragma unroll
         for (int ks = 0; ks < HD / 16; ks += 2) {
             uint32_t kb[4], kb2[4];
-            ldsm_x4(kb, &Kt[((lane & 7) + ((lane >> 4) << 3)) * KP + ks * 16 + ((lane >> 3) & 1) * 8]);
-            ldsm_x4(kb2, &Kt[((lane & 7) + ((lane >> 4) << 3)) * KP + (ks + 1) * 16 + ((lane >> 3) & 1) * 8]);
+            const int krow = (lane & 7) + ((lane >> 4) << 3), kch = (lane >> 3) & 1;
+            if constexpr (TMA) {
+                ldsm_x4(kb, &Kt[at_swz<HD>(krow, ks * 2 + kch)]);
+                ldsm_x4(kb2, &Kt[at_swz<HD>(krow, (ks + 1) * 2 + kch)]);
+            } else {
+                ldsm_x4(kb, &Kt[krow * KP + ks * 16 + kch * 8]);
+                ldsm_x4(kb2, &Kt[krow * KP + (ks + 1) * 16 + kch * 8]);
+            }
             if (QREG) {
                 mma_f16(s[0], qa[ks], kb[0], kb[1]);
                 mma_f16(s[1], qa[ks], kb[2], kb[3]);
@@ -338,15 +395,18 @@ __device__ __forceinline__ void attn_item(const AttnArgs &a, int qb, int hk, int
 #pragma unroll
         for (int np = 0; np < HD / 16; np++) {
             uint32_t vb[4];
-            ldsm_x4_t(vb, &Vt[((lane & 7) + ((lane >> 3) & 1) * 8) * KP + np * 16 + (lane >> 4) * 8]);
+            const int vrow = (lane & 7) + ((lane >> 3) & 1) * 8;
+            if constexpr (TMA) ldsm_x4_t(vb, &Vt[at_swz<HD>(vrow, np * 2 + (lane >> 4))]);
+            else ldsm_x4_t(vb, &Vt[vrow * KP + np * 16 + (lane >> 4) * 8]);
             mma_f16(o[2 * np], pa, vb[0], vb[1]);
             mma_f16(o[2 * np + 1], pa, vb[2], vb[3]);
         }
         __syncwarp();  // every lane is done with this stage: refill it
         if (t + NS < n_tiles) issue(t + NS);
-        cp_async_commit();
+        if (!TMA) cp_async_commit();
     }
-    cp_async_wait<0>();
+    if constexpr (TMA) tm->seq = seq0 + (uint32_t)n_tiles;
+    else cp_async_wait<0>();
     // this item's partial (an empty split leaves max = -inf, sum = 0, which the merge ignores)
 #pragma unroll
     for (int hf = 0; hf < 2; hf++) {
@@ -410,6 +470,87 @@ __global__ void __launch_bounds__(AW_WARPS * 32) attn_warp_kernel(AttnArgs a)
         attn_item<HD, NST, true>(a, qb, hk, sp, a.n_splits, a.split_len, row0, nrows, a.row_slot[row0], a.row_pos[row0], wr,
                                     nullptr, lane);
     }
+}
+
+// The same grid with TMA-fed rings (callers that hold tensor maps of the cache: the decode
+// path).  Without the padding and with one copy per tile a warp's stage is 16 positions x
+// head_dim x 2 matrices x 2 bytes, so three CTAs per SM hold either four warps with two stages or
+// three warps with three.
+template <int HD, int NST, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32) attn_warp_tma_kernel(const __grid_constant__ CUtensorMap map_k,
+                                                                      const __grid_constant__ CUtensorMap map_v, AttnArgs a,
+                                                                      int *status)
+{
+    extern __shared__ __align__(1024) unsigned char awt_smem[];
+    __shared__ __align__(8) uint64_t bars[WARPS][NST];
+    __shared__ int giving_up_s;
+    griddep_launch();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        for (int w = 0; w < WARPS; w++)
+            for (int s = 0; s < NST; s++) mbar_init(&bars[w][s], 1);
+        giving_up_s = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    griddep_wait();
+    // swizzled tiles want 1024-byte alignment
+    unsigned char *ring = awt_smem + ((1024u - (smem_u32(awt_smem) & 1023u)) & 1023u);
+    kv_t *wr = reinterpret_cast<kv_t *>(ring) + (size_t)warp * NST * 2 * AT_TP * HD;
+    AttnTma tm;
+    tm.mk = &map_k; tm.mv = &map_v; tm.bars = bars[warp]; tm.seq = 0; tm.giving_up = &giving_up_s; tm.status = status;
+    const int G = a.Hq / a.Hkv;
+    const int n_groups = min(*a.n_groups, a.max_groups);
+    const unsigned n_items = (unsigned)a.max_groups * a.n_qblk * a.Hkv * a.n_splits;
+    const unsigned n_workers = gridDim.x * WARPS;
+    const bool dynamic = a.ticket != nullptr && n_items > n_workers;
+    auto draw = [&]() -> unsigned {
+        unsigned t = 0;
+        if (lane == 0) t = atomicAdd(a.ticket, 1u) - a.ticket_base;
+        return n_workers + __shfl_sync(0xffffffffu, t, 0);
+    };
+    unsigned item = (unsigned)warp * gridDim.x + blockIdx.x;
+    while (item < n_items) {
+        const unsigned next = dynamic ? draw() : item + n_workers;
+        unsigned t = item;
+        item = next;
+        const int qb = (int)(t % a.n_qblk); t /= a.n_qblk;
+        const int hk = (int)(t % a.Hkv); t /= a.Hkv;
+        const int g = (int)(t % a.max_groups), sp = (int)(t / a.max_groups);
+        if (g >= n_groups) continue;
+        const int row0 = a.grp_row0[g], nrows = a.grp_nrows[g];
+        if (row0 < 0 || nrows < 1 || row0 + nrows > a.n_rows) continue;
+        const int nq = nrows * G;
+        if (qb * 16 >= nq || nq < a.nq_min || nq > a.nq_max) continue;
+        attn_item<HD, NST, true, true>(a, qb, hk, sp, a.n_splits, a.split_len, row0, nrows, a.row_slot[row0],
+                                       a.row_pos[row0], wr, nullptr, lane, &tm);
+        // a wait that ran out: the warp keeps drawing (the ticket count must come out) but works no more
+        if (giving_up_s) a.nq_max = -1;
+    }
+}
+inline size_t attn_warp_tma_bytes(int head_dim, int stages, int warps)
+{
+    return (size_t)warps * stages * 2 * AT_TP * head_dim * sizeof(kv_t) + 1024;
+}
+typedef void (*AttnWarpTmaFn)(const CUtensorMap, const CUtensorMap, AttnArgs, int *);
+// The instantiation for a head dimension (64 or 128) and a ring depth (2: four warps per CTA,
+// 3: three), its dynamic shared-memory limit raised on first use.
+inline cudaError_t attn_warp_tma_fn(int head_dim, int stages, AttnWarpTmaFn *fn, int *warps)
+{
+    static PerDevice<bool> ready_dev[4];
+    const int idx = (head_dim == 128 ? 2 : 0) + (stages == 3 ? 1 : 0);
+    AttnWarpTmaFn f = idx == 3 ? attn_warp_tma_kernel<128, 3, 3> : idx == 2 ? attn_warp_tma_kernel<128, 2, 4>
+                      : idx == 1 ? attn_warp_tma_kernel<64, 3, 3> : attn_warp_tma_kernel<64, 2, 4>;
+    *warps = stages == 3 ? 3 : 4;
+    bool &ready = ready_dev[idx].here();
+    if (!ready) {
+        const cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   (int)attn_warp_tma_bytes(head_dim, stages, *warps));
+        if (e != cudaSuccess) return e;
+        ready = true;
+    }
+    *fn = f;
+    return cudaSuccess;
 }
 
 // The grid of the stand-alone kernel: as many CTAs as fit the SMs (registers allow three).

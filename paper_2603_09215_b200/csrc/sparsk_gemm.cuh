@@ -40,7 +40,7 @@ constexpr int GM_BLK_BYTES = GM_BM * GM_BK * 2;  // one accumulator's weights fo
 constexpr int GM_MAX_STAGES = 6;
 constexpr int GM_CHUNK = 16;                   // accumulator columns per epilogue chunk
 constexpr int GM_XCHG_BYTES = GM_CHUNK * GM_BM * 4;
-constexpr unsigned long long GM_TIMEOUT_NS = 2000000000ull;
+constexpr unsigned long long GM_TIMEOUT_NS = WAIT_TIMEOUT_NS;
 
 // A unit of work is two accumulators of 128 weight rows each: either 256 consecutive rows of one
 // matrix (one TMA box), or 128 rows of matrix 0 and the same 128 rows of matrix 1 ("pair": gate
@@ -62,73 +62,7 @@ struct GemmArgs {
     int *status;   // device status word
 };
 
-// ------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ unsigned long long global_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_test(uint64_t *bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait for a phase of an mbarrier.  Returns false if the CTA is giving up (another
-// thread did, or this wait outlasted `limit_ns`); the caller then leaves its loop.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *giving_up, int *status,
-                                          unsigned long long limit_ns = GM_TIMEOUT_NS)
-{
-    unsigned long long t0 = 0;
-    for (uint32_t spin = 0;; ++spin) {
-        if (mbar_test(bar, parity)) return true;
-        if (spin > 64) __nanosleep(32);
-        if ((spin & 255u) == 255u) {
-            if (*giving_up) return false;
-            const unsigned long long now = global_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > limit_ns) {
-                *giving_up = 1;
-                if (status) atomicOr(status, ST_TIMEOUT);
-                return false;
-            }
-        }
-    }
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint64_t *bar, int x, int y)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
-        : "memory");
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint64_t *bar, int x, int y, int z)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
-        : "memory");
-}
+// (mbarrier, TMA and timer wrappers: sparsk_common.cuh)
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 // Shared-memory matrix descriptor of a K-major tile stored with the 128-byte swizzle: rows are
