@@ -426,6 +426,258 @@ __device__ __forceinline__ void attn_item(const AttnArgs &a, int qb, int hk, int
     }
 }
 
+// A warp's K/V ring, in either form: `issue` starts the copies of tile t of the split
+// [w_beg, w_end), `wait` blocks until tile t has landed (false: a bounded wait ran out) and says
+// where it is, `release` hands the stage back and refills it, `finish` closes the item.
+template <int HD, int NS, bool TMA>
+struct AtRing {
+    static constexpr int KP = HD + 8;          // padded row of the cp.async form
+    static constexpr int TP = TMA ? HD : KP;   // row pitch of a tile in the ring
+    static constexpr int CH = HD / 8;          // 16-byte chunks per row
+    kv_t *wr;
+    AttnTma *tm;
+    const kv_t *kbase, *vbase;
+    int w_beg, w_end, y0, lane, n_tiles;
+    uint32_t seq0;
+
+    // element offset of 16-byte chunk c of row `row` inside a tile
+    __device__ __forceinline__ static int off(int row, int c) { return TMA ? at_swz<HD>(row, c) : row * KP + c * 8; }
+    __device__ __forceinline__ int stage(int t) const { return (int)((seq0 + (uint32_t)t) % NS); }
+    __device__ __forceinline__ void issue(int t) const
+    {
+        const int st = stage(t);
+        kv_t *kt = wr + (size_t)st * 2 * AT_TP * TP, *vt = kt + AT_TP * TP;
+        const int p0 = w_beg + t * AT_TP;
+        if constexpr (TMA) {
+            if (lane == 0) {
+                mbar_expect_tx(&tm->bars[st], 2u * AT_TP * HD * (uint32_t)sizeof(kv_t));
+                if (HD > 64) {
+                    tma_load_3d(smem_u32(kt), tm->mk, &tm->bars[st], 0, y0 + p0, 0);
+                    tma_load_3d(smem_u32(vt), tm->mv, &tm->bars[st], 0, y0 + p0, 0);
+                } else {
+                    tma_load_2d(smem_u32(kt), tm->mk, &tm->bars[st], 0, y0 + p0);
+                    tma_load_2d(smem_u32(vt), tm->mv, &tm->bars[st], 0, y0 + p0);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int i = lane; i < AT_TP * CH; i += 32) {
+                const int r = i / CH, c = i % CH;
+                const bool ok = p0 + r < w_end;                  // rows past the end are zero-filled
+                const size_t o = (size_t)(ok ? p0 + r : w_beg) * HD + c * 8;
+                cp_async16(&kt[r * KP + c * 8], kbase + o, ok ? 16 : 0);
+                cp_async16(&vt[r * KP + c * 8], vbase + o, ok ? 16 : 0);
+            }
+        }
+    }
+    __device__ __forceinline__ void start() const
+    {
+        __syncwarp();  // the previous item's last reads of the ring are over
+#pragma unroll
+        for (int t = 0; t < NS; t++) {
+            if (t < n_tiles) issue(t);
+            if (!TMA) cp_async_commit();
+        }
+    }
+    __device__ __forceinline__ bool wait(int t, const kv_t *&Kt, const kv_t *&Vt) const
+    {
+        const int st = stage(t);
+        kv_t *kt = wr + (size_t)st * 2 * AT_TP * TP, *vt = kt + AT_TP * TP;
+        if constexpr (TMA) {
+            if (!mbar_wait(&tm->bars[st], ((seq0 + (uint32_t)t) / NS) & 1u, tm->giving_up, tm->status)) return false;
+            const int p0 = w_beg + t * AT_TP;
+            if (p0 + AT_TP > w_end) {
+                // value rows past the end meet a weight of exactly zero, which must not meet a
+                // NaN or an infinity: clear them
+                const int nv = w_end - p0;
+                for (int i = lane; i < (AT_TP - nv) * CH; i += 32)
+                    *reinterpret_cast<uint4 *>(&vt[at_swz<HD>(nv + i / CH, i % CH)]) = make_uint4(0u, 0u, 0u, 0u);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            }
+        } else {
+            cp_async_wait<NS - 1>();
+        }
+        __syncwarp();
+        Kt = kt;
+        Vt = vt;
+        return true;
+    }
+    __device__ __forceinline__ void release(int t) const
+    {
+        __syncwarp();  // every lane is done with this stage: refill it
+        if (t + NS < n_tiles) issue(t + NS);
+        if (!TMA) cp_async_commit();
+    }
+    __device__ __forceinline__ void finish() const
+    {
+        if constexpr (TMA) tm->seq = seq0 + (uint32_t)n_tiles;
+        else cp_async_wait<0>();
+    }
+};
+
+__device__ __forceinline__ uint32_t movmatrix_t(uint32_t x)
+{
+    uint32_t y;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+    return y;
+}
+
+// One item of at most eight query vectors, by one warp, in the transposed form: with few query
+// heads per kv head (a single row of a group) the sixteen-row M dimension of the form above is
+// half empty, so here the POSITIONS are the M dimension.  S^T = K Q^T (K tile as the A operand,
+// the queries as eight B columns, 16 registers for the whole item), the softmax runs down the
+// columns (maxima and sums across the eight lane groups), P^T becomes the B operand of
+// O^T = V^T P^T through two 8x8 register transposes, and V^T is read with transposing ldmatrix.
+// Half the MMAs, half the accumulators and a quarter of the exponentials of the other form;
+// the partial it writes is the same.
+template <int HD, int NS, bool TMA>
+__device__ __forceinline__ void attn_item_t(const AttnArgs &a, int hk, int sp, int splits, int split_len, int row0,
+                                            int nrows, int slot, int pos0, kv_t *wr, int lane, AttnTma *tm = nullptr)
+{
+    constexpr float LOG2E = 1.4426950408889634f, LN2 = 0.6931471805599453f;
+    typedef AtRing<HD, NS, TMA> Ring;
+    const int G = a.Hq / a.Hkv;
+    const int nq = nrows * G;  // <= 8
+    const bool sane = slot >= 0 && slot < a.n_slots && pos0 >= 0;
+    const int kv_end_all = sane ? min(pos0 + nrows, a.S) : 0;
+    Ring ring;
+    ring.w_beg = sp * split_len;
+    ring.w_end = min(ring.w_beg + split_len, kv_end_all);
+    ring.n_tiles = ring.w_end > ring.w_beg ? (ring.w_end - ring.w_beg + AT_TP - 1) / AT_TP : 0;
+    if (ring.n_tiles == 0) {
+        for (int qi = lane; qi < nq; qi += 32)
+            a.part_ml[((size_t)(row0 + qi / G) * a.Hq + hk * G + qi % G) * splits + sp] = make_float2(-INFINITY, 0.f);
+        return;
+    }
+    ring.wr = wr; ring.tm = tm; ring.lane = lane;
+    ring.kbase = a.kc + ((size_t)slot * a.Hkv + hk) * a.S * HD;
+    ring.vbase = a.vc + ((size_t)slot * a.Hkv + hk) * a.S * HD;
+    ring.y0 = (slot * a.Hkv + hk) * a.S;
+    ring.seq0 = TMA ? tm->seq : 0u;
+    ring.start();
+
+    // the queries as B fragments: column lane / 4, elements 2 (lane % 4) + {0, 1, 8, 9} of every
+    // 16-element step, scaled by log2(e) / sqrt(hd)
+    uint32_t qf[HD / 16][2];
+    {
+        const int qi = lane >> 2, c0 = (lane & 3) * 2;
+        const bool have = qi < nq;
+        const size_t o = (size_t)(row0 + (have ? qi / G : 0)) * a.Hq * HD + (hk * G + (have ? qi % G : 0)) * HD + c0;
+        const float qscale = rsqrtf((float)HD) * LOG2E;
+#pragma unroll
+        for (int ks = 0; ks < HD / 16; ks++) {
+            float2 x0 = make_float2(0.f, 0.f), x1 = x0;
+            if (have) {
+                if (a.q32) {
+                    x0 = *reinterpret_cast<const float2 *>(a.q32 + o + ks * 16);
+                    x1 = *reinterpret_cast<const float2 *>(a.q32 + o + ks * 16 + 8);
+                } else {
+                    const uint32_t u0 = *reinterpret_cast<const uint32_t *>(a.q + o + ks * 16);
+                    const uint32_t u1 = *reinterpret_cast<const uint32_t *>(a.q + o + ks * 16 + 8);
+                    x0 = make_float2(bf_lo(u0), bf_hi(u0));
+                    x1 = make_float2(bf_lo(u1), bf_hi(u1));
+                }
+            }
+            qf[ks][0] = pack_h2(x0.x * qscale, x0.y * qscale);
+            qf[ks][1] = pack_h2(x1.x * qscale, x1.y * qscale);
+        }
+    }
+    // this thread's two query vectors (accumulator columns) and the last position each may see
+    int limit[2];
+#pragma unroll
+    for (int e = 0; e < 2; e++) {
+        const int qi = (lane & 3) * 2 + e;
+        limit[e] = qi < nq ? pos0 + qi / G : -1;
+    }
+    float o[HD / 16][4], m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+#pragma unroll
+    for (int mt = 0; mt < HD / 16; mt++)
+#pragma unroll
+        for (int e = 0; e < 4; e++) o[mt][e] = 0.f;
+
+    for (int t = 0; t < ring.n_tiles; t++) {
+        const kv_t *Kt, *Vt;
+        if (!ring.wait(t, Kt, Vt)) return;
+        const int p0 = ring.w_beg + t * AT_TP;
+        // S^T for 16 positions x 8 query vectors, two accumulator chains
+        float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int ks = 0; ks < HD / 16; ks += 2) {
+            uint32_t ka[4], kb[4];
+            ldsm_x4(ka, &Kt[Ring::off(lane & 15, ks * 2 + (lane >> 4))]);
+            ldsm_x4(kb, &Kt[Ring::off(lane & 15, (ks + 1) * 2 + (lane >> 4))]);
+            mma_f16(s0, ka, qf[ks][0], qf[ks][1]);
+            mma_f16(s1, kb, qf[ks + 1][0], qf[ks + 1][1]);
+        }
+        // online softmax down the columns; accumulator rows are positions lane / 4 and + 8
+        const bool full = p0 + AT_TP <= ring.w_end && p0 + AT_TP - 1 <= pos0;
+        float pv[2][2], alpha[2];
+#pragma unroll
+        for (int e = 0; e < 2; e++) {
+#pragma unroll
+            for (int j = 0; j < 2; j++) {
+                const int p = p0 + (lane >> 2) + j * 8;
+                const bool ok = full || (p < ring.w_end && p <= limit[e]);
+                pv[e][j] = ok ? s0[j * 2 + e] + s1[j * 2 + e] : -INFINITY;
+            }
+            float tmax = fmaxf(pv[e][0], pv[e][1]);
+            tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 4));
+            tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 8));
+            tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 16));
+            const float m_new = fmaxf(m_run[e], tmax);
+            alpha[e] = 1.f;
+            if (m_new != -INFINITY) {
+                alpha[e] = exp2f(m_run[e] - m_new);
+                pv[e][0] = exp2f(pv[e][0] - m_new);
+                pv[e][1] = exp2f(pv[e][1] - m_new);
+            } else {
+                pv[e][0] = pv[e][1] = 0.f;
+            }
+            l_run[e] = l_run[e] * alpha[e] + pv[e][0] + pv[e][1];  // per-thread share; lanes are summed at the end
+            m_run[e] = m_new;
+        }
+        // P^T as the B operand: the accumulator layout of an 8x8 block (row = position, two
+        // columns = query vectors) transposed is the operand layout (row = query vector ...)
+        const uint32_t b0 = movmatrix_t(pack_h2(pv[0][0], pv[1][0]));  // positions 0..7 of the tile
+        const uint32_t b1 = movmatrix_t(pack_h2(pv[0][1], pv[1][1]));  // positions 8..15
+        if (__any_sync(0xffffffffu, alpha[0] != 1.f || alpha[1] != 1.f)) {
+#pragma unroll
+            for (int mt = 0; mt < HD / 16; mt++) {
+                o[mt][0] *= alpha[0];
+                o[mt][1] *= alpha[1];
+                o[mt][2] *= alpha[0];
+                o[mt][3] *= alpha[1];
+            }
+        }
+        // O^T += V^T P^T: sixteen dimensions per MMA, V read transposed
+#pragma unroll
+        for (int mt = 0; mt < HD / 16; mt++) {
+            uint32_t va[4];
+            ldsm_x4_t(va, &Vt[Ring::off((lane & 7) + ((lane >> 4) << 3), mt * 2 + ((lane >> 3) & 1))]);
+            mma_f16(o[mt], va, b0, b1);
+        }
+        ring.release(t);
+    }
+    ring.finish();
+#pragma unroll
+    for (int e = 0; e < 2; e++) {
+        float l = l_run[e];
+        l += __shfl_xor_sync(0xffffffffu, l, 4);
+        l += __shfl_xor_sync(0xffffffffu, l, 8);
+        l += __shfl_xor_sync(0xffffffffu, l, 16);
+        const int qi = (lane & 3) * 2 + e;
+        if (qi < nq) {
+            const size_t cell = ((size_t)(row0 + qi / G) * a.Hq + hk * G + qi % G) * splits + sp;
+            if ((lane >> 2) == 0) a.part_ml[cell] = make_float2(m_run[e] * LN2, l);
+#pragma unroll
+            for (int mt = 0; mt < HD / 16; mt++) {
+                a.part_o[cell * HD + mt * 16 + (lane >> 2)] = o[mt][e];
+                a.part_o[cell * HD + mt * 16 + 8 + (lane >> 2)] = o[mt][2 + e];
+            }
+        }
+    }
+}
+
 // Persistent grid of warps; item i = ((sp * groups + g) * Hkv + hk) * n_qblk + qb: the query
 // blocks of one (group, kv head, split) run side by side, and all but the first find their K/V
 // tiles in the L2; the splits that short groups leave empty come last.  With a ticket counter
@@ -467,8 +719,12 @@ __global__ void __launch_bounds__(AW_WARPS * 32) attn_warp_kernel(AttnArgs a)
         if (row0 < 0 || nrows < 1 || row0 + nrows > a.n_rows) continue;
         const int nq = nrows * G;
         if (qb * 16 >= nq || nq < a.nq_min || nq > a.nq_max) continue;
-        attn_item<HD, NST, true>(a, qb, hk, sp, a.n_splits, a.split_len, row0, nrows, a.row_slot[row0], a.row_pos[row0], wr,
-                                    nullptr, lane);
+        if (nq <= 8)
+            attn_item_t<HD, NST, false>(a, hk, sp, a.n_splits, a.split_len, row0, nrows, a.row_slot[row0], a.row_pos[row0], wr,
+                                        lane);
+        else
+            attn_item<HD, NST, true>(a, qb, hk, sp, a.n_splits, a.split_len, row0, nrows, a.row_slot[row0], a.row_pos[row0],
+                                     wr, nullptr, lane);
     }
 }
 
@@ -522,8 +778,12 @@ __global__ void __launch_bounds__(WARPS * 32) attn_warp_tma_kernel(const __grid_
         if (row0 < 0 || nrows < 1 || row0 + nrows > a.n_rows) continue;
         const int nq = nrows * G;
         if (qb * 16 >= nq || nq < a.nq_min || nq > a.nq_max) continue;
-        attn_item<HD, NST, true, true>(a, qb, hk, sp, a.n_splits, a.split_len, row0, nrows, a.row_slot[row0],
-                                       a.row_pos[row0], wr, nullptr, lane, &tm);
+        if (nq <= 8)
+            attn_item_t<HD, NST, true>(a, hk, sp, a.n_splits, a.split_len, row0, nrows, a.row_slot[row0], a.row_pos[row0], wr,
+                                       lane, &tm);
+        else
+            attn_item<HD, NST, true, true>(a, qb, hk, sp, a.n_splits, a.split_len, row0, nrows, a.row_slot[row0],
+                                           a.row_pos[row0], wr, nullptr, lane, &tm);
         // a wait that ran out: the warp keeps drawing (the ticket count must come out) but works no more
         if (giving_up_s) a.nq_max = -1;
     }
