@@ -147,32 +147,178 @@ __device__ __forceinline__ int at_swz(int row, int c)
     return (HD > 64 ? (c >> 3) * (AT_TP * 64) : 0) + row * 64 + (((c & 7) ^ (row & 7)) << 3);
 }
 
-// One item, by one warp: query vectors [16 qb, 16 qb + 16) of a group whose first row is row0
-// (nrows rows of slot `slot`, first at position pos0), kv head hk, split sp of `splits` splits of
-// split_len positions.  `wr` is the warp's ring of NS stages.  Writes the item's partial.
+// What a warp knows of an item before it starts: who it is for, and the span of positions it reads.
+struct AtItem {
+    int qb, hk, sp, row0, nrows, slot, pos0;
+    int nq;                          // query vectors of the group per kv head
+    int w_beg, w_end, n_tiles, y0;   // positions [w_beg, w_end) in tiles of 16; first cache row of (slot, hk)
+    bool valid;                      // false: not an item of this launch (no partial either)
+};
+// Item number idx of a launch -> descriptor.  Straight-line code: every load is clamped instead of
+// skipped, so the loads of one level go out together.
+__device__ __forceinline__ AtItem at_resolve(const AttnArgs &a, unsigned idx, unsigned n_items, int n_groups,
+                                             const int *grp_row0, const int *grp_nrows, const int *row_slot,
+                                             const int *row_pos)
+{
+    AtItem it;
+    const int G = a.Hq / a.Hkv;
+    unsigned t = idx < n_items ? idx : 0u;
+    it.qb = (int)(t % a.n_qblk); t /= a.n_qblk;
+    it.hk = (int)(t % a.Hkv); t /= a.Hkv;
+    const int g = (int)(t % a.max_groups);
+    it.sp = (int)(t / a.max_groups);
+    bool ok = idx < n_items && g < n_groups;
+    const int gc = ok ? g : 0;
+    it.row0 = grp_row0[gc];
+    it.nrows = grp_nrows[gc];
+    ok = ok && it.row0 >= 0 && it.nrows >= 1 && it.row0 + it.nrows <= a.n_rows;
+    const int rc = ok ? it.row0 : 0;
+    it.slot = row_slot[rc];
+    it.pos0 = row_pos[rc];
+    it.nq = it.nrows * G;
+    ok = ok && it.qb * 16 < it.nq && it.nq >= a.nq_min && it.nq <= a.nq_max;
+    // positions the item may look at: its split, cut at the last query row's own position (and
+    // at the cache itself: a row that points outside it reads nothing)
+    const bool sane = it.slot >= 0 && it.slot < a.n_slots && it.pos0 >= 0;
+    const int nq_here = min(16, it.nq - it.qb * 16);
+    const int last_row = (it.qb * 16 + nq_here - 1) / G;
+    const int kv_end_all = ok && sane ? min(it.pos0 + last_row + 1, a.S) : 0;
+    it.w_beg = it.sp * a.split_len;
+    it.w_end = min(it.w_beg + a.split_len, kv_end_all);
+    it.n_tiles = it.w_end > it.w_beg ? (it.w_end - it.w_beg + AT_TP - 1) / AT_TP : 0;
+    it.y0 = ((sane ? it.slot : 0) * a.Hkv + it.hk) * a.S;
+    it.valid = ok;
+    return it;
+}
+// A warp's K/V ring, in either form: `issue` starts the copies of tile t of the split
+// [w_beg, w_end), `wait` blocks until tile t has landed (false: a bounded wait ran out) and says
+// where it is, `release` hands the stage back and refills it, `finish` closes the item.
+template <int HD, int NS, bool TMA>
+struct AtRing {
+    static constexpr int KP = HD + 8;          // padded row of the cp.async form
+    static constexpr int TP = TMA ? HD : KP;   // row pitch of a tile in the ring
+    static constexpr int CH = HD / 8;          // 16-byte chunks per row
+    kv_t *wr;
+    AttnTma *tm;
+    const kv_t *kbase, *vbase;
+    int w_beg, w_end, y0, lane, n_tiles;
+    uint32_t seq0;
+
+    __device__ __forceinline__ AtRing(const AttnArgs &a, const AtItem &it, kv_t *wr_, int lane_, AttnTma *tm_)
+        : wr(wr_), tm(tm_), kbase(a.kc + (size_t)it.y0 * HD), vbase(a.vc + (size_t)it.y0 * HD), w_beg(it.w_beg),
+          w_end(it.w_end), y0(it.y0), lane(lane_), n_tiles(it.n_tiles), seq0(TMA ? tm_->seq : 0u)
+    {
+    }
+
+    // element offset of 16-byte chunk c of row `row` inside a tile
+    __device__ __forceinline__ static int off(int row, int c) { return TMA ? at_swz<HD>(row, c) : row * KP + c * 8; }
+    __device__ __forceinline__ int stage(int t) const { return (int)((seq0 + (uint32_t)t) % NS); }
+    // TMA form: the tile whose first cache row is y, as tile number `seq` of this warp.  Rows past a
+    // split's end arrive as whatever the cache holds there (zeros beyond the cache): the scores
+    // mask them, the value rows are cleared after landing.
+    __device__ __forceinline__ void issue_tma(int y, uint32_t seq) const
+    {
+        if (lane == 0) {
+            const int st = (int)(seq % NS);
+            kv_t *kt = wr + (size_t)st * 2 * AT_TP * TP, *vt = kt + AT_TP * TP;
+            mbar_expect_tx(&tm->bars[st], 2u * AT_TP * HD * (uint32_t)sizeof(kv_t));
+            if (HD > 64) {
+                tma_load_3d(smem_u32(kt), tm->mk, &tm->bars[st], 0, y, 0);
+                tma_load_3d(smem_u32(vt), tm->mv, &tm->bars[st], 0, y, 0);
+            } else {
+                tma_load_2d(smem_u32(kt), tm->mk, &tm->bars[st], 0, y);
+                tma_load_2d(smem_u32(vt), tm->mv, &tm->bars[st], 0, y);
+            }
+        }
+    }
+    __device__ __forceinline__ void issue(int t) const
+    {
+        const int st = stage(t);
+        kv_t *kt = wr + (size_t)st * 2 * AT_TP * TP, *vt = kt + AT_TP * TP;
+        const int p0 = w_beg + t * AT_TP;
+        if constexpr (TMA) {
+            issue_tma(y0 + p0, seq0 + (uint32_t)t);
+        } else {
+#pragma unroll
+            for (int i = lane; i < AT_TP * CH; i += 32) {
+                const int r = i / CH, c = i % CH;
+                const bool ok = p0 + r < w_end;                  // rows past the end are zero-filled
+                const size_t o = (size_t)(ok ? p0 + r : w_beg) * HD + c * 8;
+                cp_async16(&kt[r * KP + c * 8], kbase + o, ok ? 16 : 0);
+                cp_async16(&vt[r * KP + c * 8], vbase + o, ok ? 16 : 0);
+            }
+        }
+    }
+    __device__ __forceinline__ void start() const
+    {
+        __syncwarp();  // the previous item's last reads of the ring are over
+#pragma unroll
+        for (int t = 0; t < NS; t++) {
+            if (t < n_tiles) issue(t);
+            if (!TMA) cp_async_commit();
+        }
+    }
+    __device__ __forceinline__ bool wait(int t, const kv_t *&Kt, const kv_t *&Vt) const
+    {
+        const int st = stage(t);
+        kv_t *kt = wr + (size_t)st * 2 * AT_TP * TP, *vt = kt + AT_TP * TP;
+        if constexpr (TMA) {
+            if (!mbar_wait(&tm->bars[st], ((seq0 + (uint32_t)t) / NS) & 1u, tm->giving_up, tm->status)) return false;
+            const int p0 = w_beg + t * AT_TP;
+            if (p0 + AT_TP > w_end) {
+                // value rows past the end meet a weight of exactly zero, which must not meet a
+                // NaN or an infinity: clear them
+                const int nv = w_end - p0;
+                for (int i = lane; i < (AT_TP - nv) * CH; i += 32)
+                    *reinterpret_cast<uint4 *>(&vt[at_swz<HD>(nv + i / CH, i % CH)]) = make_uint4(0u, 0u, 0u, 0u);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            }
+        } else {
+            cp_async_wait<NS - 1>();
+        }
+        __syncwarp();
+        Kt = kt;
+        Vt = vt;
+        return true;
+    }
+    __device__ __forceinline__ void release(int t) const
+    {
+        __syncwarp();  // every lane is done with this stage: refill it
+        if (t + NS < n_tiles) issue(t + NS);
+        if (!TMA) cp_async_commit();
+    }
+    __device__ __forceinline__ void finish() const
+    {
+        if constexpr (TMA) tm->seq = seq0 + (uint32_t)n_tiles;
+        else cp_async_wait<0>();
+    }
+};
+
+__device__ __forceinline__ uint32_t movmatrix_t(uint32_t x)
+{
+    uint32_t y;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+    return y;
+}
+
+// One item, by one warp: query vectors [16 qb, 16 qb + 16) of a group (rows row0 .. row0 + nrows - 1
+// of slot `slot`, the first at position pos0), kv head hk, split sp.  `wr` is the warp's ring of
+// NS stages.  Writes the item's partial.
 // QREG: the query fragments stay in registers for the whole item (32 registers at head dimension
 // 128); otherwise they are parked in `qs` ([16][HD + 8] of shared memory) and re-read per tile,
 // for callers whose register budget is spoken for.
 template <int HD, int NS, bool QREG, bool TMA = false>
-__device__ __forceinline__ void attn_item(const AttnArgs &a, int qb, int hk, int sp, int splits, int split_len, int row0,
-                                          int nrows, int slot, int pos0, kv_t *wr, kv_t *qs, int lane,
+__device__ __forceinline__ void attn_item(const AttnArgs &a, const AtItem &it, kv_t *wr, kv_t *qs, int lane,
                                           AttnTma *tm = nullptr)
 {
-    constexpr int KP = HD + 8;      // padded row (cp.async form; also the parked queries): ldmatrix rows fall into distinct banks
-    constexpr int TP = TMA ? HD : KP;  // row pitch of a K/V tile in the ring
-    constexpr int CH = HD / 8;      // 16-byte chunks per row
+    typedef AtRing<HD, NS, TMA> Ring;
+    constexpr int KP = HD + 8;      // padded row of the parked queries: ldmatrix rows fall into distinct banks
     constexpr float LOG2E = 1.4426950408889634f, LN2 = 0.6931471805599453f;
-    const int G = a.Hq / a.Hkv;
-    const int nq = nrows * G, q0 = qb * 16;
+    const int G = a.Hq / a.Hkv, splits = a.n_splits;
+    const int qb = it.qb, hk = it.hk, sp = it.sp, row0 = it.row0, pos0 = it.pos0;
+    const int nq = it.nq, q0 = qb * 16;
     const int nq_here = min(16, nq - q0);
-    // positions this item may look at: its split, cut at the last query row's own position
-    // (and at the cache itself: a row that points outside it reads nothing)
-    const bool sane = slot >= 0 && slot < a.n_slots && pos0 >= 0;
-    const int last_row = (q0 + nq_here - 1) / G;
-    const int kv_end_all = sane ? min(pos0 + last_row + 1, a.S) : 0;
-    const int w_beg = sp * split_len;
-    const int w_end = min(w_beg + split_len, kv_end_all);
-    const int n_tiles = w_end > w_beg ? (w_end - w_beg + AT_TP - 1) / AT_TP : 0;
+    const int w_beg = it.w_beg, w_end = it.w_end, n_tiles = it.n_tiles;
     if (n_tiles == 0) {
         // an empty split: max = -inf, sum = 0 is all the merge looks at
         for (int qi = lane; qi < nq_here; qi += 32) {
@@ -181,48 +327,8 @@ __device__ __forceinline__ void attn_item(const AttnArgs &a, int qb, int hk, int
         }
         return;
     }
-    const kv_t *kbase = a.kc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
-    const kv_t *vbase = a.vc + ((size_t)(sane ? slot : 0) * a.Hkv + hk) * a.S * HD;
-
-    const uint32_t seq0 = TMA ? tm->seq : 0u;
-    auto issue = [&](int t) {
-        const int st = (int)((seq0 + (uint32_t)t) % NS);
-        kv_t *kt = wr + (size_t)st * 2 * AT_TP * TP, *vt = kt + AT_TP * TP;
-        const int p0 = w_beg + t * AT_TP;
-        if constexpr (TMA) {
-            // rows past the split's end arrive as whatever the cache holds there (or zeros beyond
-            // the cache): the scores mask them, the value rows are cleared after landing
-            if (lane == 0) {
-                const int y = (slot * a.Hkv + hk) * a.S + p0;
-                mbar_expect_tx(&tm->bars[st], 2u * AT_TP * HD * (uint32_t)sizeof(kv_t));
-                if (HD > 64) {
-                    tma_load_3d(smem_u32(kt), tm->mk, &tm->bars[st], 0, y, 0);
-                    tma_load_3d(smem_u32(vt), tm->mv, &tm->bars[st], 0, y, 0);
-                } else {
-                    tma_load_2d(smem_u32(kt), tm->mk, &tm->bars[st], 0, y);
-                    tma_load_2d(smem_u32(vt), tm->mv, &tm->bars[st], 0, y);
-                }
-            }
-        } else {
-#pragma unroll
-            for (int i = lane; i < AT_TP * CH; i += 32) {
-                const int r = i / CH, c = i % CH;
-                const bool ok = p0 + r < w_end;                  // rows past the end are zero-filled
-                const size_t off = (size_t)(ok ? p0 + r : w_beg) * HD + c * 8;
-                cp_async16(&kt[r * KP + c * 8], kbase + off, ok ? 16 : 0);
-                cp_async16(&vt[r * KP + c * 8], vbase + off, ok ? 16 : 0);
-            }
-        }
-    };
-    // The ring: tiles t .. t + NS - 1 are in flight or in use while tile t is computed; every
-    // refill is its own commit group (empty ones included), so "all but the newest NS - 1 groups"
-    // always means "tile t has landed".
-    __syncwarp();  // the previous item's last reads of the ring are over
-#pragma unroll
-    for (int t = 0; t < NS; t++) {
-        if (t < n_tiles) issue(t);
-        if (!TMA) cp_async_commit();
-    }
+    Ring ring(a, it, wr, lane, tm);
+    ring.start();
 
     // the queries, as A fragments (row = lane / 4 and + 8, columns 2 (lane % 4) + {0, 1, 8, 9} of
     // every 16-column step), while the first tiles are on their way
@@ -289,23 +395,9 @@ __device__ __forceinline__ void attn_item(const AttnArgs &a, int qb, int hk, int
     const int lim_min = pos0 + q0 / G;  // the smallest limit among the item's query vectors
 
     for (int t = 0; t < n_tiles; t++) {
-        const int st = (int)((seq0 + (uint32_t)t) % NS);
-        kv_t *Kt = wr + (size_t)st * 2 * AT_TP * TP, *Vt = Kt + AT_TP * TP;
+        const kv_t *Kt, *Vt;
+        if (!ring.wait(t, Kt, Vt)) return;
         const int p0 = w_beg + t * AT_TP;
-        if constexpr (TMA) {
-            if (!mbar_wait(&tm->bars[st], ((seq0 + (uint32_t)t) / NS) & 1u, tm->giving_up, tm->status)) return;
-            if (p0 + AT_TP > w_end) {
-                // value rows past the end meet a weight of exactly zero, which must not meet a
-                // NaN or an infinity: clear them
-                const int nv = w_end - p0;
-                for (int i = lane; i < (AT_TP - nv) * CH; i += 32)
-                    *reinterpret_cast<uint4 *>(&Vt[at_swz<HD>(nv + i / CH, i % CH)]) = make_uint4(0u, 0u, 0u, 0u);
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            }
-        } else {
-            cp_async_wait<NS - 1>();  // tile t has landed
-        }
-        __syncwarp();
 
         // S = Q K^T for 16 positions, in log2 units; two accumulator chains
         float s[2][4], s2[2][4];
@@ -317,13 +409,8 @@ __device__ __forceinline__ void attn_item(const AttnArgs &a, int qb, int hk, int
         for (int ks = 0; ks < HD / 16; ks += 2) {
             uint32_t kb[4], kb2[4];
             const int krow = (lane & 7) + ((lane >> 4) << 3), kch = (lane >> 3) & 1;
-            if constexpr (TMA) {
-                ldsm_x4(kb, &Kt[at_swz<HD>(krow, ks * 2 + kch)]);
-                ldsm_x4(kb2, &Kt[at_swz<HD>(krow, (ks + 1) * 2 + kch)]);
-            } else {
-                ldsm_x4(kb, &Kt[krow * KP + ks * 16 + kch * 8]);
-                ldsm_x4(kb2, &Kt[krow * KP + (ks + 1) * 16 + kch * 8]);
-            }
+            ldsm_x4(kb, &Kt[Ring::off(krow, ks * 2 + kch)]);
+            ldsm_x4(kb2, &Kt[Ring::off(krow, (ks + 1) * 2 + kch)]);
             if (QREG) {
                 mma_f16(s[0], qa[ks], kb[0], kb[1]);
                 mma_f16(s[1], qa[ks], kb[2], kb[3]);
@@ -396,17 +483,13 @@ __device__ __forceinline__ void attn_item(const AttnArgs &a, int qb, int hk, int
         for (int np = 0; np < HD / 16; np++) {
             uint32_t vb[4];
             const int vrow = (lane & 7) + ((lane >> 3) & 1) * 8;
-            if constexpr (TMA) ldsm_x4_t(vb, &Vt[at_swz<HD>(vrow, np * 2 + (lane >> 4))]);
-            else ldsm_x4_t(vb, &Vt[vrow * KP + np * 16 + (lane >> 4) * 8]);
+            ldsm_x4_t(vb, &Vt[Ring::off(vrow, np * 2 + (lane >> 4))]);
             mma_f16(o[2 * np], pa, vb[0], vb[1]);
             mma_f16(o[2 * np + 1], pa, vb[2], vb[3]);
         }
-        __syncwarp();  // every lane is done with this stage: refill it
-        if (t + NS < n_tiles) issue(t + NS);
-        if (!TMA) cp_async_commit();
+        ring.release(t);
     }
-    if constexpr (TMA) tm->seq = seq0 + (uint32_t)n_tiles;
-    else cp_async_wait<0>();
+    ring.finish();
     // this item's partial (an empty split leaves max = -inf, sum = 0, which the merge ignores)
 #pragma unroll
     for (int hf = 0; hf < 2; hf++) {
@@ -426,102 +509,6 @@ __device__ __forceinline__ void attn_item(const AttnArgs &a, int qb, int hk, int
     }
 }
 
-// A warp's K/V ring, in either form: `issue` starts the copies of tile t of the split
-// [w_beg, w_end), `wait` blocks until tile t has landed (false: a bounded wait ran out) and says
-// where it is, `release` hands the stage back and refills it, `finish` closes the item.
-template <int HD, int NS, bool TMA>
-struct AtRing {
-    static constexpr int KP = HD + 8;          // padded row of the cp.async form
-    static constexpr int TP = TMA ? HD : KP;   // row pitch of a tile in the ring
-    static constexpr int CH = HD / 8;          // 16-byte chunks per row
-    kv_t *wr;
-    AttnTma *tm;
-    const kv_t *kbase, *vbase;
-    int w_beg, w_end, y0, lane, n_tiles;
-    uint32_t seq0;
-
-    // element offset of 16-byte chunk c of row `row` inside a tile
-    __device__ __forceinline__ static int off(int row, int c) { return TMA ? at_swz<HD>(row, c) : row * KP + c * 8; }
-    __device__ __forceinline__ int stage(int t) const { return (int)((seq0 + (uint32_t)t) % NS); }
-    __device__ __forceinline__ void issue(int t) const
-    {
-        const int st = stage(t);
-        kv_t *kt = wr + (size_t)st * 2 * AT_TP * TP, *vt = kt + AT_TP * TP;
-        const int p0 = w_beg + t * AT_TP;
-        if constexpr (TMA) {
-            if (lane == 0) {
-                mbar_expect_tx(&tm->bars[st], 2u * AT_TP * HD * (uint32_t)sizeof(kv_t));
-                if (HD > 64) {
-                    tma_load_3d(smem_u32(kt), tm->mk, &tm->bars[st], 0, y0 + p0, 0);
-                    tma_load_3d(smem_u32(vt), tm->mv, &tm->bars[st], 0, y0 + p0, 0);
-                } else {
-                    tma_load_2d(smem_u32(kt), tm->mk, &tm->bars[st], 0, y0 + p0);
-                    tma_load_2d(smem_u32(vt), tm->mv, &tm->bars[st], 0, y0 + p0);
-                }
-            }
-        } else {
-#pragma unroll
-            for (int i = lane; i < AT_TP * CH; i += 32) {
-                const int r = i / CH, c = i % CH;
-                const bool ok = p0 + r < w_end;                  // rows past the end are zero-filled
-                const size_t o = (size_t)(ok ? p0 + r : w_beg) * HD + c * 8;
-                cp_async16(&kt[r * KP + c * 8], kbase + o, ok ? 16 : 0);
-                cp_async16(&vt[r * KP + c * 8], vbase + o, ok ? 16 : 0);
-            }
-        }
-    }
-    __device__ __forceinline__ void start() const
-    {
-        __syncwarp();  // the previous item's last reads of the ring are over
-#pragma unroll
-        for (int t = 0; t < NS; t++) {
-            if (t < n_tiles) issue(t);
-            if (!TMA) cp_async_commit();
-        }
-    }
-    __device__ __forceinline__ bool wait(int t, const kv_t *&Kt, const kv_t *&Vt) const
-    {
-        const int st = stage(t);
-        kv_t *kt = wr + (size_t)st * 2 * AT_TP * TP, *vt = kt + AT_TP * TP;
-        if constexpr (TMA) {
-            if (!mbar_wait(&tm->bars[st], ((seq0 + (uint32_t)t) / NS) & 1u, tm->giving_up, tm->status)) return false;
-            const int p0 = w_beg + t * AT_TP;
-            if (p0 + AT_TP > w_end) {
-                // value rows past the end meet a weight of exactly zero, which must not meet a
-                // NaN or an infinity: clear them
-                const int nv = w_end - p0;
-                for (int i = lane; i < (AT_TP - nv) * CH; i += 32)
-                    *reinterpret_cast<uint4 *>(&vt[at_swz<HD>(nv + i / CH, i % CH)]) = make_uint4(0u, 0u, 0u, 0u);
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            }
-        } else {
-            cp_async_wait<NS - 1>();
-        }
-        __syncwarp();
-        Kt = kt;
-        Vt = vt;
-        return true;
-    }
-    __device__ __forceinline__ void release(int t) const
-    {
-        __syncwarp();  // every lane is done with this stage: refill it
-        if (t + NS < n_tiles) issue(t + NS);
-        if (!TMA) cp_async_commit();
-    }
-    __device__ __forceinline__ void finish() const
-    {
-        if constexpr (TMA) tm->seq = seq0 + (uint32_t)n_tiles;
-        else cp_async_wait<0>();
-    }
-};
-
-__device__ __forceinline__ uint32_t movmatrix_t(uint32_t x)
-{
-    uint32_t y;
-    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
-    return y;
-}
-
 // One item of at most eight query vectors, by one warp, in the transposed form: with few query
 // heads per kv head (a single row of a group) the sixteen-row M dimension of the form above is
 // half empty, so here the POSITIONS are the M dimension.  S^T = K Q^T (K tile as the A operand,
@@ -531,29 +518,19 @@ __device__ __forceinline__ uint32_t movmatrix_t(uint32_t x)
 // Half the MMAs, half the accumulators and a quarter of the exponentials of the other form;
 // the partial it writes is the same.
 template <int HD, int NS, bool TMA>
-__device__ __forceinline__ void attn_item_t(const AttnArgs &a, int hk, int sp, int splits, int split_len, int row0,
-                                            int nrows, int slot, int pos0, kv_t *wr, int lane, AttnTma *tm = nullptr)
+__device__ __forceinline__ void attn_item_t(const AttnArgs &a, const AtItem &it, kv_t *wr, int lane, AttnTma *tm = nullptr)
 {
     constexpr float LOG2E = 1.4426950408889634f, LN2 = 0.6931471805599453f;
     typedef AtRing<HD, NS, TMA> Ring;
-    const int G = a.Hq / a.Hkv;
-    const int nq = nrows * G;  // <= 8
-    const bool sane = slot >= 0 && slot < a.n_slots && pos0 >= 0;
-    const int kv_end_all = sane ? min(pos0 + nrows, a.S) : 0;
-    Ring ring;
-    ring.w_beg = sp * split_len;
-    ring.w_end = min(ring.w_beg + split_len, kv_end_all);
-    ring.n_tiles = ring.w_end > ring.w_beg ? (ring.w_end - ring.w_beg + AT_TP - 1) / AT_TP : 0;
-    if (ring.n_tiles == 0) {
+    const int G = a.Hq / a.Hkv, splits = a.n_splits;
+    const int hk = it.hk, sp = it.sp, row0 = it.row0, pos0 = it.pos0;
+    const int nq = it.nq;  // <= 8
+    if (it.n_tiles == 0) {
         for (int qi = lane; qi < nq; qi += 32)
             a.part_ml[((size_t)(row0 + qi / G) * a.Hq + hk * G + qi % G) * splits + sp] = make_float2(-INFINITY, 0.f);
         return;
     }
-    ring.wr = wr; ring.tm = tm; ring.lane = lane;
-    ring.kbase = a.kc + ((size_t)slot * a.Hkv + hk) * a.S * HD;
-    ring.vbase = a.vc + ((size_t)slot * a.Hkv + hk) * a.S * HD;
-    ring.y0 = (slot * a.Hkv + hk) * a.S;
-    ring.seq0 = TMA ? tm->seq : 0u;
+    Ring ring(a, it, wr, lane, tm);
     ring.start();
 
     // the queries as B fragments: column lane / 4, elements 2 (lane % 4) + {0, 1, 8, 9} of every
@@ -693,7 +670,6 @@ __global__ void __launch_bounds__(AW_WARPS * 32) attn_warp_kernel(AttnArgs a)
     griddep_wait();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     kv_t *wr = reinterpret_cast<kv_t *>(aw_smem) + (size_t)warp * NST * 2 * AT_TP * (HD + 8);
-    const int G = a.Hq / a.Hkv;
     const int n_groups = min(*a.n_groups, a.max_groups);
     const unsigned n_items = (unsigned)a.max_groups * a.n_qblk * a.Hkv * a.n_splits;
     const unsigned n_workers = gridDim.x * AW_WARPS;
@@ -709,22 +685,11 @@ __global__ void __launch_bounds__(AW_WARPS * 32) attn_warp_kernel(AttnArgs a)
     while (item < n_items) {
         // the next ticket is drawn before this item's work, so that its latency is hidden
         const unsigned next = dynamic ? draw() : item + n_workers;
-        unsigned t = item;
+        const AtItem it = at_resolve(a, item, n_items, n_groups, a.grp_row0, a.grp_nrows, a.row_slot, a.row_pos);
         item = next;
-        const int qb = (int)(t % a.n_qblk); t /= a.n_qblk;
-        const int hk = (int)(t % a.Hkv); t /= a.Hkv;
-        const int g = (int)(t % a.max_groups), sp = (int)(t / a.max_groups);
-        if (g >= n_groups) continue;
-        const int row0 = a.grp_row0[g], nrows = a.grp_nrows[g];
-        if (row0 < 0 || nrows < 1 || row0 + nrows > a.n_rows) continue;
-        const int nq = nrows * G;
-        if (qb * 16 >= nq || nq < a.nq_min || nq > a.nq_max) continue;
-        if (nq <= 8)
-            attn_item_t<HD, NST, false>(a, hk, sp, a.n_splits, a.split_len, row0, nrows, a.row_slot[row0], a.row_pos[row0], wr,
-                                        lane);
-        else
-            attn_item<HD, NST, true>(a, qb, hk, sp, a.n_splits, a.split_len, row0, nrows, a.row_slot[row0], a.row_pos[row0],
-                                     wr, nullptr, lane);
+        if (!it.valid) continue;
+        if (it.nq <= 8) attn_item_t<HD, NST, false>(a, it, wr, lane);
+        else attn_item<HD, NST, true>(a, it, wr, nullptr, lane);
     }
 }
 
@@ -755,7 +720,6 @@ __global__ void __launch_bounds__(WARPS * 32) attn_warp_tma_kernel(const __grid_
     kv_t *wr = reinterpret_cast<kv_t *>(ring) + (size_t)warp * NST * 2 * AT_TP * HD;
     AttnTma tm;
     tm.mk = &map_k; tm.mv = &map_v; tm.bars = bars[warp]; tm.seq = 0; tm.giving_up = &giving_up_s; tm.status = status;
-    const int G = a.Hq / a.Hkv;
     const int n_groups = min(*a.n_groups, a.max_groups);
     const unsigned n_items = (unsigned)a.max_groups * a.n_qblk * a.Hkv * a.n_splits;
     const unsigned n_workers = gridDim.x * WARPS;
@@ -768,24 +732,12 @@ __global__ void __launch_bounds__(WARPS * 32) attn_warp_tma_kernel(const __grid_
     unsigned item = (unsigned)warp * gridDim.x + blockIdx.x;
     while (item < n_items) {
         const unsigned next = dynamic ? draw() : item + n_workers;
-        unsigned t = item;
+        const AtItem it = at_resolve(a, item, n_items, n_groups, a.grp_row0, a.grp_nrows, a.row_slot, a.row_pos);
         item = next;
-        const int qb = (int)(t % a.n_qblk); t /= a.n_qblk;
-        const int hk = (int)(t % a.Hkv); t /= a.Hkv;
-        const int g = (int)(t % a.max_groups), sp = (int)(t / a.max_groups);
-        if (g >= n_groups) continue;
-        const int row0 = a.grp_row0[g], nrows = a.grp_nrows[g];
-        if (row0 < 0 || nrows < 1 || row0 + nrows > a.n_rows) continue;
-        const int nq = nrows * G;
-        if (qb * 16 >= nq || nq < a.nq_min || nq > a.nq_max) continue;
-        if (nq <= 8)
-            attn_item_t<HD, NST, true>(a, hk, sp, a.n_splits, a.split_len, row0, nrows, a.row_slot[row0], a.row_pos[row0], wr,
-                                       lane, &tm);
-        else
-            attn_item<HD, NST, true, true>(a, qb, hk, sp, a.n_splits, a.split_len, row0, nrows, a.row_slot[row0],
-                                           a.row_pos[row0], wr, nullptr, lane, &tm);
-        // a wait that ran out: the warp keeps drawing (the ticket count must come out) but works no more
-        if (giving_up_s) a.nq_max = -1;
+        // after a wait that ran out the warp keeps drawing (the ticket count must come out) but works no more
+        if (!it.valid || giving_up_s) continue;
+        if (it.nq <= 8) attn_item_t<HD, NST, true>(a, it, wr, lane, &tm);
+        else attn_item<HD, NST, true, true>(a, it, wr, nullptr, lane, &tm);
     }
 }
 inline size_t attn_warp_tma_bytes(int head_dim, int stages, int warps)

@@ -19,19 +19,16 @@ __device__ __forceinline__ void mk_attention(const MkArgs &a, const MkLayer *L, 
     at.q = nullptr; at.q32 = a.q_buf; at.kc = L->kc; at.vc = L->vc;
     at.part_o = a.part_o; at.part_ml = a.part_ml;
     at.Hq = a.Hq; at.Hkv = a.Hkv; at.S = a.S; at.n_slots = a.n_slots; at.n_rows = a.n_rows;
-    const int G = a.Hq / a.Hkv;
-    const int n_workers = gridDim.x * MK_ATT_WARPS, worker = warp * gridDim.x + blockIdx.x;
-    const int n_qblk = a.att_qblk;
-    const int n_items = a.n_groups * n_qblk * a.Hkv * a.att_splits;
-    for (int item = worker; item < n_items; item += n_workers) {
-        int t = item;
-        const int sp = t % a.att_splits; t /= a.att_splits;
-        const int hk = t % a.Hkv; t /= a.Hkv;
-        const int qb = t % n_qblk, g = t / n_qblk;
-        const int row0 = sh->grp_row0[g], nrows = sh->grp_nrows[g];
-        if (row0 < 0 || nrows < 1 || row0 + nrows > a.n_rows || qb * 16 >= nrows * G) continue;
-        attn_item<HD, MK_ATT_NST, false>(at, qb, hk, sp, a.att_splits, a.att_split_len, row0, nrows, sh->row_slot[row0],
-                                         sh->row_pos[row0], wr, qs, lane);
+    at.n_qblk = a.att_qblk; at.n_splits = a.att_splits; at.split_len = a.att_split_len; at.max_groups = a.n_groups;
+    at.nq_min = 0; at.nq_max = 1 << 30;
+    const unsigned n_workers = gridDim.x * MK_ATT_WARPS, worker = warp * gridDim.x + blockIdx.x;
+    const unsigned n_items = (unsigned)a.n_groups * a.att_qblk * a.Hkv * a.att_splits;
+    for (unsigned item = worker; item < n_items; item += n_workers) {
+        const AtItem it = at_resolve(at, item, n_items, a.n_groups, sh->grp_row0, sh->grp_nrows, sh->row_slot, sh->row_pos);
+        if (!it.valid) continue;
+        // a single row's query heads (at most eight per kv head) take the transposed form
+        if (it.nq <= 8) attn_item_t<HD, MK_ATT_NST, false>(at, it, wr, lane);
+        else attn_item<HD, MK_ATT_NST, false>(at, it, wr, qs, lane);
     }
 }
 

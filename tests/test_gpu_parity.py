@@ -232,13 +232,17 @@ def test_every_route_for_small_passes(util, options):
     P.close()
 
 
-@pytest.mark.parametrize("options", [{"attn_ctas": 2, "attn_split": 16, "mega": 0},
+@pytest.mark.parametrize("options", [{"attn_ctas": 2, "attn_split": 16, "mega": 0}, {"attn_ctas": 2, "attn_split": 32, "mega": 0},
+                                     {"attn_ctas": 3, "attn_split": 48, "mega": 0, "attn_stages": 3},
+                                     {"attn_ctas": 1, "attn_split": 64, "mega": 0, "attn_tma": 0},
                                      {"attn_ctas": 2, "attn_split": 16, "mega": 0, "attn_dynamic": 0},
                                      {"attn_ctas": 1, "mega": 0, "gemm_min_rows": 1}])
 def test_attention_items_drawn_from_the_counter(util, options):
     """Many more attention work items than warps (the kernel held to one or two CTAs, four ragged
     sequences, short splits): the warps draw items from the ticket counter, launch after launch
-    (the host predicts the counter's value instead of resetting it), or take every n-th item."""
+    (the host predicts the counter's value instead of resetting it), or take every n-th item.
+    Splits of one, two and three tiles with ragged ends, so that items shorter than, as long as and
+    longer than a warp's ring follow one another and each starts its successor's first tiles."""
     dims = synth.model_dims("tiny", 2, 4, 0)
     w = synth.make_weights(dims, seed=0)
     prompts = synth.make_prompts(dims, 4, 9, 150, seed=21)
