@@ -31,10 +31,14 @@ __device__ __forceinline__ void mk_load_act(float *act, int c0, int ncols, int K
         float *dst = act + (size_t)m * ncols;
         if (h) {
             const float *src = h + (size_t)m * K;
+            // a row that is loaded whole is parked in the area on its way through the sum of
+            // squares and scaled in place afterwards: one trip to the L2 instead of two
+            const bool whole = c0 == 0 && ncols >= K;
             float ss = 0.f;
-            for (int i = tid * 4; i < K; i += T * 4) {
-                const float4 v = *reinterpret_cast<const float4 *>(src + i);
+            for (int i = tid * 4; i < (whole ? ncols : K); i += T * 4) {
+                const float4 v = i < K ? *reinterpret_cast<const float4 *>(src + i) : make_float4(0.f, 0.f, 0.f, 0.f);
                 ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+                if (whole) *reinterpret_cast<float4 *>(dst + mk_act_slot(i)) = v;
             }
             ss = warp_sum(ss);
             if (lane == 0) sh->red[warp] = ss;
@@ -44,16 +48,26 @@ __device__ __forceinline__ void mk_load_act(float *act, int c0, int ncols, int K
             for (int w = 0; w < MK_CW; w++) tot += sh->red[w];
             mk_consumer_sync();
             const float inv = rsqrtf(tot / (float)K + eps);
-            for (int i = tid * 4; i < ncols; i += T * 4) {
-                float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-                const int k = c0 + i;
-                if (k < K) {
-                    const float4 p = *reinterpret_cast<const float4 *>(src + k);
-                    const uint2 g2 = *reinterpret_cast<const uint2 *>(gain + k);
-                    o = make_float4(p.x * inv * bf_lo(g2.x), p.y * inv * bf_hi(g2.x), p.z * inv * bf_lo(g2.y),
-                                    p.w * inv * bf_hi(g2.y));
+            if (whole) {
+                for (int i = tid * 4; i < K; i += T * 4) {   // the thread's own float4s again
+                    float4 *q = reinterpret_cast<float4 *>(dst + mk_act_slot(i));
+                    const float4 p = *q;
+                    const uint2 g2 = *reinterpret_cast<const uint2 *>(gain + i);
+                    *q = make_float4(p.x * inv * bf_lo(g2.x), p.y * inv * bf_hi(g2.x), p.z * inv * bf_lo(g2.y),
+                                     p.w * inv * bf_hi(g2.y));
                 }
-                *reinterpret_cast<float4 *>(dst + mk_act_slot(i)) = o;
+            } else {
+                for (int i = tid * 4; i < ncols; i += T * 4) {
+                    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+                    const int k = c0 + i;
+                    if (k < K) {
+                        const float4 p = *reinterpret_cast<const float4 *>(src + k);
+                        const uint2 g2 = *reinterpret_cast<const uint2 *>(gain + k);
+                        o = make_float4(p.x * inv * bf_lo(g2.x), p.y * inv * bf_hi(g2.x), p.z * inv * bf_lo(g2.y),
+                                        p.w * inv * bf_hi(g2.y));
+                    }
+                    *reinterpret_cast<float4 *>(dst + mk_act_slot(i)) = o;
+                }
             }
         } else {
             const float *src = x + (size_t)m * K;
