@@ -29,10 +29,10 @@ if ROOT not in sys.path:
 from paper_2603_09215_b200 import synth  # noqa: E402
 
 # DRAM bytes (read + write) per algorithmic byte of the persistent kernel, from its profiler capture
-# on a two-layer launch (935.44 MB read + 10.0 MB written against 934.3 MB algorithmic); a launch's
+# on a two-layer launch (935.29 MB read + 7.0 MB written against 934.3 MB algorithmic); a launch's
 # traffic is its layers' weights and cache, so it grows in proportion to the layer passes and the
 # ratio carries over to the full-size launches timed here.
-MEGA_DRAM_PER_ALGORITHMIC_BYTE = (935.44 + 10.0) / 934.3
+MEGA_DRAM_PER_ALGORITHMIC_BYTE = (935.29 + 7.0) / 934.3
 
 KC = {"qkv": 1, "attn": 2, "oproj": 3, "gateup": 4, "down": 5, "head": 6, "mega": 7, "all": 8}
 

@@ -81,6 +81,7 @@ struct sparsk_ctx {
     int attn_ctas;               // option: CTAs of the attention kernel (0: as many as fit the SMs)
     // pinned staging ring for the per-step host arrays
     int *stage_host[STAGE_RING];
+    int *io_host;                // pinned: [B] tokens in, [B] tokens out, [B] depths out, status (decode_step_host)
     cudaEvent_t stage_ev[STAGE_RING];
     int stage_next;
     // host mirror of per-slot state
@@ -1110,6 +1111,7 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
     ctx->cur_class = KC_MISC; ctx->time_class = KC_MISC; ctx->tev_used = 0;
     ctx->stage_next = 0;
     for (int i = 0; i < STAGE_RING; i++) { ctx->stage_host[i] = nullptr; ctx->stage_ev[i] = nullptr; }
+    ctx->io_host = nullptr;
 
     int rc = SPARSK_OK;
     do {
@@ -1125,6 +1127,9 @@ extern "C" int sparsk_create(const sparsk_dims *dims, const sparsk_weights *w, v
                 (ce = cudaEventCreateWithFlags(&ctx->stage_ev[i], cudaEventDisableTiming)) != cudaSuccess)
                 rc = fail(ctx, SPARSK_ECUDA, "staging setup failed: %s", cudaGetErrorString(ce));
         }
+        if (rc == SPARSK_OK &&
+            (ce = cudaHostAlloc((void **)&ctx->io_host, sizeof(int) * (3 * (size_t)dims->max_seqs + 1), cudaHostAllocDefault)) != cudaSuccess)
+            rc = fail(ctx, SPARSK_ECUDA, "staging setup failed: %s", cudaGetErrorString(ce));
         if (rc) break;
         if (dims->conf_modalities) {
             // one region per segment of a step (at most one per layer, plus lists per consulted layer)
@@ -1188,6 +1193,7 @@ extern "C" int sparsk_destroy(sparsk_ctx *ctx)
         if (ctx->stage_host[i]) cudaFreeHost(ctx->stage_host[i]);
         if (ctx->stage_ev[i]) cudaEventDestroy(ctx->stage_ev[i]);
     }
+    if (ctx->io_host) cudaFreeHost(ctx->io_host);
     for (cudaEvent_t ev : ctx->tev) cudaEventDestroy(ev);
     if (ctx->conf_host) cudaFreeHost(ctx->conf_host);
     if (ctx->conf_ent_host) cudaFreeHost(ctx->conf_ent_host);
@@ -1308,11 +1314,17 @@ extern "C" int sparsk_kernel_time(sparsk_ctx *ctx, double *total_ms, int64_t *n_
 // return code.  After a timeout the persistent kernels' grid-barrier counter, its host mirror and
 // the abort word start over, so that the next launch does not find a stale abort request or a
 // counter that no longer matches its base.
+static int act_on_status(sparsk_ctx *ctx, int status);
 static int read_status(sparsk_ctx *ctx)
 {
     int status = 0;
     CU(cudaMemcpyAsync(&status, ctx->sd.counts + CNT_STATUS, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
     CU(cudaStreamSynchronize(ctx->stream));
+    return act_on_status(ctx, status);
+}
+// What a status word read back from the device (the stream is idle) means for the caller.
+static int act_on_status(sparsk_ctx *ctx, int status)
+{
     if (status) CU(cudaMemsetAsync(ctx->sd.counts + CNT_STATUS, 0, sizeof(int), ctx->stream));
     if (status & ST_TIMEOUT) {
         CU(cudaMemsetAsync(ctx->mk_bar, 0, sizeof(unsigned long long), ctx->stream));
@@ -1837,10 +1849,20 @@ extern "C" int sparsk_decode_step_host(sparsk_ctx *ctx, int32_t n, const int32_t
     for (int i = 0; i < n; i++)
         if (token_ids[i] < 0 || token_ids[i] >= V)
             return fail(ctx, SPARSK_EINVAL, "decode_step_host: token_ids[%d]=%d is outside the vocabulary [0, %d)", i, token_ids[i], V);
-    CU(cudaMemcpyAsync(ctx->tok_dev, token_ids, sizeof(int) * n, cudaMemcpyHostToDevice, ctx->stream));
+    // Everything crosses the bus through one pinned buffer, so that the copies are truly
+    // asynchronous and the host waits once per step (a copy to or from pageable memory makes the
+    // host wait for it; three of them in a row after the step cost 30 us of idle GPU per step).
+    const int B = ctx->dm.max_seqs;
+    int *io = ctx->io_host;
+    memcpy(io, token_ids, sizeof(int) * n);
+    CU(cudaMemcpyAsync(ctx->tok_dev, io, sizeof(int) * n, cudaMemcpyHostToDevice, ctx->stream));
     const int rc = sparsk_decode_step(ctx, n, slots, ctx->tok_dev, modality, counters, ctx->out_tok_dev, ctx->out_depth_dev);
     if (rc != SPARSK_OK) return rc;
-    CU(cudaMemcpyAsync(next_tokens, ctx->out_tok_dev, sizeof(int) * n, cudaMemcpyDeviceToHost, ctx->stream));
-    CU(cudaMemcpyAsync(exit_depths, ctx->out_depth_dev, sizeof(int) * n, cudaMemcpyDeviceToHost, ctx->stream));
-    return read_status(ctx);
+    CU(cudaMemcpyAsync(io + B, ctx->out_tok_dev, sizeof(int) * n, cudaMemcpyDeviceToHost, ctx->stream));
+    CU(cudaMemcpyAsync(io + 2 * B, ctx->out_depth_dev, sizeof(int) * n, cudaMemcpyDeviceToHost, ctx->stream));
+    CU(cudaMemcpyAsync(io + 3 * B, ctx->sd.counts + CNT_STATUS, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+    CU(cudaStreamSynchronize(ctx->stream));
+    memcpy(next_tokens, io + B, sizeof(int) * n);
+    memcpy(exit_depths, io + 2 * B, sizeof(int) * n);
+    return act_on_status(ctx, io[3 * B]);
 }
