@@ -41,6 +41,7 @@ def oracle_out(q, k, v, row_slot, row_pos, Hq, Hkv, hd):
     (7, 1, 128, 1200, [(0, 1100, 4), (1, 17, 1), (2, 640, 2)]),                  # 7 q heads per kv head
     (32, 2, 128, 700, [(1, 600, 4), (0, 3, 2)]),                                 # 16 per kv head: 2 q blocks
     (6, 2, 64, 400, [(0, 100, 40)]),                                             # prefill-like block of 40 rows
+    (8, 2, 128, 500, [(0, 14, 2), (1, 15, 2), (2, 16, 2), (0, 400, 1), (1, 47, 2)]),  # two rows = 8 query vectors: the transposed form, masks at tile edges
 ])
 def test_attention_matches_oracle(Hq, Hkv, hd, S, groups):
     if not torch.cuda.is_available():
