@@ -523,7 +523,10 @@ def main():
     sampler = ClockSampler(uuid)
     sampler.start()
     b0 = run.bytes
+    # a profiler started with "--profile-from-start off" sees exactly this timed region
+    torch.cuda.profiler.start()
     ms, ntok, launches = timed(run, args.steps)
+    torch.cuda.profiler.stop()
     clocks = sampler.stop()
     step_b = (run.bytes - b0)
     value = job_tokens_per_s(ntok, ms, world)
