@@ -11,16 +11,24 @@
 //
 // The warp keeps its sixteen query vectors as fp16 MMA fragments in registers (scaled by
 // log2(e) / sqrt(hd), so that the softmax works in powers of two), streams 16-position K/V tiles
-// of its split into a private shared-memory ring with coalesced 16-byte cp.async copies (no
-// barrier wider than the warp anywhere), computes S = Q K^T and O += P V with fp16 MMAs and fp32
-// accumulators, and keeps an online softmax whose row maxima and sums are reduced with shuffles
-// inside the four-lane groups that share an accumulator row.  Queries and softmax weights are
-// rounded to fp16 once, like the cache they meet: the same 2^-12 relative error as a cached key
-// or value carries.  The warp writes one unnormalised partial (acc, running max in log2 units
-// turned back to natural-log units, running sum) per (row, query head, split); a second kernel
-// merges the splits.  Items are dealt round-robin to the warps of a persistent grid: a warp's
-// fixed cost per item is a few hundred instructions, which is what lets twelve warps per SM with
-// one tile in flight each keep HBM busy where CTA-wide tiles with a cross-warp merge did not.
+// of its split into a private shared-memory ring (no barrier wider than the warp anywhere),
+// computes S = Q K^T and O += P V with fp16 MMAs and fp32 accumulators, and keeps an online
+// softmax whose row maxima and sums are reduced with shuffles inside the four-lane groups that
+// share an accumulator row.  Queries and softmax weights are rounded to fp16 once, like the cache
+// they meet: the same 2^-12 relative error as a cached key or value carries.  The warp writes one
+// unnormalised partial (acc, running max in log2 units turned back to natural-log units, running
+// sum) per (row, query head, split); a second kernel merges the splits.
+//
+// Two forms of the ring: coalesced 16-byte cp.async copies into padded rows (callers that pass
+// plain cache pointers: the stand-alone entry points, the persistent kernel), or one TMA box per
+// tile and matrix with the 128-byte swizzle and an mbarrier per stage (the decode path, which
+// holds tensor maps of its cache).  Two forms of an item: the one above, and a transposed one for
+// groups of at most eight query vectors (a single row at up to eight query heads per kv head),
+// where the positions are the M dimension and the work per tile halves (attn_item_t).
+// Items are dealt to the warps of a persistent grid, each warp's first by its number and the rest,
+// when there are more items than warps, from a ticket counter as warps finish: a warp's fixed cost
+// per item is a few hundred instructions, which is what lets twelve warps per SM with one tile
+// in flight each keep HBM busy where CTA-wide tiles with a cross-warp merge did not.
 #pragma once
 
 #include "sparsk_common.cuh"
