@@ -801,28 +801,42 @@ inline cudaError_t attn_warp_fn(int head_dim, int stages, AttnWarpFn *fn)
 }
 
 // Merge the splits of every (row, query head): out = sum_s acc_s e^{m_s - M} / sum_s l_s e^{m_s - M}.
+// One block per (row, head), one thread per output dimension.  The splits' weights are worked out
+// once (thread s takes split s) and parked in shared memory, so that the loop over the splits is
+// a row of independent loads and not a chain of (max, sum) look-ups in front of every one.
 template <int HD>
 __global__ void __launch_bounds__(HD) attn_merge_kernel(AttnArgs a, const int *__restrict__ n_rows)
 {
+    __shared__ float w_s[AT_MAX_SPLITS];
+    __shared__ float den_s;
     griddep_launch();
     griddep_wait();
     const int row = blockIdx.x, head = blockIdx.y;
     if (row >= *n_rows) return;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const size_t cell0 = ((size_t)row * a.Hq + head) * a.n_splits;
-    float M = -INFINITY;
-    for (int s = 0; s < a.n_splits; s++) M = fmaxf(M, a.part_ml[cell0 + s].x);
-    float den = 0.f, num = 0.f;
+    // a.n_splits <= AT_MAX_SPLITS = 32 <= HD: the first warp holds one split per lane
+    float2 ml = make_float2(-INFINITY, 0.f);
+    if (tid < a.n_splits) ml = a.part_ml[cell0 + tid];
+    if (warp == 0) {
+        const float M = warp_max(ml.x);
+        const float w = ml.x == -INFINITY ? 0.f : __expf(ml.x - M);
+        const float den = warp_sum(ml.y * w);
+        if (lane < AT_MAX_SPLITS) w_s[lane] = w;
+        if (lane == 0) den_s = den;
+    }
+    __syncthreads();
+    const float den = den_s;
+    float num = 0.f;
+#pragma unroll 4
     for (int s = 0; s < a.n_splits; s++) {
-        const float2 ml = a.part_ml[cell0 + s];
-        if (ml.x == -INFINITY) continue;
-        const float w = __expf(ml.x - M);
-        den += ml.y * w;
-        num += a.part_o[(cell0 + s) * HD + threadIdx.x] * w;
+        const float w = w_s[s];
+        if (w != 0.f) num += a.part_o[(cell0 + s) * HD + tid] * w;  // an empty split's partial is never read
     }
     const float val = den > 0.f ? num / den : 0.f;
     const bf16 hi = __float2bfloat16(val);
-    a.out[(size_t)row * a.Hq * HD + head * HD + threadIdx.x] = hi;
-    if (a.out_lo) a.out_lo[(size_t)row * a.Hq * HD + head * HD + threadIdx.x] = __float2bfloat16(val - __bfloat162float(hi));
+    a.out[(size_t)row * a.Hq * HD + head * HD + tid] = hi;
+    if (a.out_lo) a.out_lo[(size_t)row * a.Hq * HD + head * HD + tid] = __float2bfloat16(val - __bfloat162float(hi));
 }
 
 }  // namespace sparsk
